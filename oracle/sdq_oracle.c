@@ -1,0 +1,429 @@
+/*
+ * SDQ oracle -- TEST INFRASTRUCTURE, NOT THE PRODUCT.
+ *
+ * A plain, slow, obviously-correct CPU statement of what the SDQ decomposed linear layer computes
+ * (arXiv 2406.13868, Section 5: Stage 1 sparsification, Stage 2 decomposition, Stage 3
+ * quantization, and the "LLM inference performance" paragraph O = O_o + O_i).  It shares no code,
+ * header, table or helper with the CUDA library; only tests, the smoke check and the CPU-baseline
+ * leg of the benchmark may call it.
+ *
+ * Everything is written in the order and notation of the paper's stages:
+ *   W  --(local N:M outlier extraction per S-Vector of 8 along K)-->  W_o  (outliers, 8-bit float)
+ *      --(N:M magnitude pruning of the remaining values)          -->  W_i  (inliers, 4-bit float)
+ *   A  --> A_o (8-bit float), A_i (4-bit float with per-Q-Vector power-of-two scale)
+ *   O  = A_o * W_o^T + A_i * W_i^T                     accumulated in fp64
+ *
+ * Number formats are decoded/encoded by exhaustive nearest-value search over the list of
+ * representable values in fp64 -- no bit tricks -- so that the rounding rule is visible:
+ * round to nearest, ties to the code whose last bit is 0, saturate at the largest finite value.
+ *
+ * Pins (tests/ -m "not gpu"): exhaustive codec checks against closed forms and torch CPU casts,
+ * N:M invariants from the paper, brute force over all C(8,n) selections, an independent dense
+ * "definition" of the decomposition, brute-force matmul, one-hot read-back, exact power-of-two
+ * scaling, and the paper's printed bits-per-weight / throughput arithmetic.
+ * Parity unpinned: none of the functions in this file (model-quality numbers of the paper are not
+ * computed here at all).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define SDQO_GRAN_PAIR 0 /* inlier pattern: keep 2 of the 4 adjacent pairs in every 8 (pair-wise 4:8) */
+#define SDQO_GRAN_ELEM 1 /* inlier pattern: keep 2 of every 4 elements (element-wise 2:4)            */
+#define SDQO_SCALE_OCP_FLOOR 0  /* E = floor(log2 amax) - 2   (OCP MX rule, may saturate in (6,8)) */
+#define SDQO_SCALE_CEIL_NOSAT 1 /* E = smallest integer with amax <= 6 * 2^E                        */
+
+typedef struct {
+  int out_n;      /* outliers kept per S-Vector of 8 along K: 0, 1 or 2          */
+  int in_gran;    /* SDQO_GRAN_*                                                */
+  int in_block;   /* Q-Vector: logical K per inlier / 4-bit activation scale (32|64) */
+  int scale_rule; /* SDQO_SCALE_*                                               */
+} sdqo_config;
+
+/* ------------------------------------------------------------------ number formats */
+
+/* bf16 bit pattern -> value (bf16 is the upper half of an IEEE fp32) */
+double sdqo_bf16_to_double(uint16_t h) {
+  uint32_t u = ((uint32_t)h) << 16;
+  float f;
+  memcpy(&f, &u, sizeof f);
+  return (double)f;
+}
+
+/* E2M1: 1 sign, 2 exponent (bias 1), 1 mantissa bit. Magnitudes by code 0..7. */
+static const double E2M1_MAG[8] = {0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0};
+
+double sdqo_e2m1_decode(uint8_t code) {
+  double m = E2M1_MAG[code & 7];
+  return (code & 8) ? -m : m;
+}
+
+/* E4M3 (OCP "FN" flavour): 1 sign, 4 exponent (bias 7), 3 mantissa; no infinity; magnitude codes
+ * 0x00..0x7E are finite (0x7F is NaN); largest finite value 448. */
+static double e4m3_mag(int mcode) {
+  int e = (mcode >> 3) & 15, m = mcode & 7;
+  if (e == 0) return ldexp((double)m / 8.0, -6);   /* subnormals: m/8 * 2^-6 */
+  return ldexp(1.0 + (double)m / 8.0, e - 7);
+}
+
+double sdqo_e4m3_decode(uint8_t code) {
+  double m = e4m3_mag(code & 0x7F);
+  return (code & 0x80) ? -m : m;
+}
+
+/* E8M0: value 2^(code-127); code 255 (NaN) never produced here. */
+double sdqo_e8m0_decode(uint8_t code) { return ldexp(1.0, (int)code - 127); }
+
+/* nearest representable magnitude among n_codes ascending magnitudes; ties -> even code;
+ * anything above the largest magnitude saturates to it. */
+static int nearest_code(double a, int n_codes, double (*mag)(int)) {
+  if (a >= mag(n_codes - 1)) return n_codes - 1;   /* saturate (also keeps huge inputs away from the tie rule) */
+  int best = 0;
+  double best_d = fabs(a - mag(0));
+  for (int c = 1; c < n_codes; ++c) {
+    double d = fabs(a - mag(c));
+    if (d < best_d || (d == best_d && (c & 1) == 0)) { best = c; best_d = d; }
+  }
+  return best;
+}
+static double e2m1_mag_fn(int c) { return E2M1_MAG[c]; }
+
+/* sign of v is kept even when the magnitude rounds to zero (so -0 encodes as 0x8 / 0x80) */
+uint8_t sdqo_e2m1_encode(double v) {
+  int c = nearest_code(fabs(v), 8, e2m1_mag_fn);
+  return (uint8_t)(c | (signbit(v) ? 8 : 0));
+}
+uint8_t sdqo_e4m3_encode(double v) {
+  int c = nearest_code(fabs(v), 127, e4m3_mag);
+  return (uint8_t)(c | (signbit(v) ? 0x80 : 0));
+}
+
+/* smallest integer e with amax <= vmax * 2^e ; amax == 0 -> 0 */
+static int ceil_exp(double amax, double vmax) {
+  if (amax == 0.0) return 0;
+  int e = -200;
+  while (amax > ldexp(vmax, e)) ++e;
+  return e;
+}
+/* floor(log2 amax) for amax > 0 */
+static int floor_log2(double amax) {
+  int e = -200;
+  while (ldexp(1.0, e + 1) <= amax) ++e;
+  return e;
+}
+
+/* E8M0 code of the Q-Vector scale for 4-bit values whose largest magnitude is amax */
+uint8_t sdqo_e8m0_scale_code(double amax, int scale_rule) {
+  if (amax == 0.0) return 0;
+  int E = (scale_rule == SDQO_SCALE_OCP_FLOOR) ? floor_log2(amax) - 2 : ceil_exp(amax, 6.0);
+  int c = E + 127;
+  if (c < 0) c = 0;
+  if (c > 254) c = 254;
+  return (uint8_t)c;
+}
+
+/* exponent e of the power-of-two scale 2^e used for 8-bit (E4M3) operands: nothing saturates */
+int sdqo_fp8_scale_exp(double amax) { return ceil_exp(amax, 448.0); }
+
+/* magnitude key used by every "largest" selection: the 15 low bits of the bf16 pattern */
+static int mag_key(uint16_t h) { return (int)(h & 0x7FFF); }
+
+static int is_finite_bf16(uint16_t h) { return (h & 0x7F80) != 0x7F80; }
+
+/* ------------------------------------------------------------------ Stage 2 + 1 + 3 on one weight matrix
+ *
+ * W        [N][K] bf16 bit patterns, row-major (row = output feature, K contiguous)
+ * Canonical outputs, one code per byte (layout-free parity surface):
+ *   in_code  [N][K/2]      E2M1 codes of the kept inlier slots in ascending k
+ *   in_meta  [N][K/8] (PAIR: j0 | j1<<2, kept pair indices 0..3 of the group of 8)
+ *            [N][K/4] (ELEM: i0 | i1<<2, kept element indices 0..3 of the group of 4)
+ *   in_scale [N][K/in_block] E8M0 code
+ *   out_code [N][K/8][out_n] E4M3 codes; out_idx same shape, position 0..7 inside the group, ascending
+ *   out_sexp [N]           e of the per-row outlier scale 2^e (int32)
+ * returns 0, or -1 on a bad argument, -2 if W holds a non-finite value.
+ */
+int sdqo_decompose(const uint16_t* W, int64_t N, int64_t K, const sdqo_config* cfg,
+                   uint8_t* in_code, uint8_t* in_meta, uint8_t* in_scale,
+                   uint8_t* out_code, uint8_t* out_idx, int32_t* out_sexp) {
+  if (!W || !cfg || N <= 0 || K <= 0 || K % 64 != 0) return -1;
+  if (cfg->out_n < 0 || cfg->out_n > 2) return -1;
+  if (cfg->in_block != 32 && cfg->in_block != 64) return -1;
+  const int on = cfg->out_n, Bs = cfg->in_block;
+  const int64_t G8 = K / 8;
+  for (int64_t i = 0; i < N * K; ++i)
+    if (!is_finite_bf16(W[i])) return -2;
+
+  uint8_t* is_out = (uint8_t*)malloc((size_t)K);   /* 1 where the element went to W_o            */
+  uint8_t* kept = (uint8_t*)malloc((size_t)K);     /* 1 where the element is a kept inlier SLOT  */
+  for (int64_t n = 0; n < N; ++n) {
+    const uint16_t* w = W + n * K;
+    memset(is_out, 0, (size_t)K);
+    memset(kept, 0, (size_t)K);
+
+    /* Stage 2, local outlier extraction: the out_n largest |w| of every S-Vector of 8 */
+    double out_amax = 0.0;
+    for (int64_t g = 0; g < G8; ++g) {
+      int chosen[2] = {-1, -1};
+      for (int t = 0; t < on; ++t) {
+        int best = -1;
+        for (int i = 0; i < 8; ++i) {
+          if (is_out[8 * g + i]) continue;
+          if (best < 0 || mag_key(w[8 * g + i]) > mag_key(w[8 * g + best])) best = i;
+        }
+        is_out[8 * g + best] = 1;
+        chosen[t] = best;
+      }
+      if (on == 2 && chosen[0] > chosen[1]) { int t = chosen[0]; chosen[0] = chosen[1]; chosen[1] = t; }
+      for (int t = 0; t < on; ++t) {
+        out_idx[(n * G8 + g) * on + t] = (uint8_t)chosen[t];
+        double a = fabs(sdqo_bf16_to_double(w[8 * g + chosen[t]]));
+        if (a > out_amax) out_amax = a;
+      }
+    }
+    /* Stage 3 for outliers: per-row power-of-two scale, E4M3 codes of w / 2^e */
+    const int e = sdqo_fp8_scale_exp(out_amax);
+    out_sexp[n] = e;
+    for (int64_t g = 0; g < G8; ++g)
+      for (int t = 0; t < on; ++t) {
+        int i = out_idx[(n * G8 + g) * on + t];
+        out_code[(n * G8 + g) * on + t] = sdqo_e4m3_encode(ldexp(sdqo_bf16_to_double(w[8 * g + i]), -e));
+      }
+
+    /* Stage 1 on the remaining values: N:M magnitude pruning */
+    if (cfg->in_gran == SDQO_GRAN_PAIR) {
+      for (int64_t g = 0; g < G8; ++g) {
+        float score[4];
+        for (int j = 0; j < 4; ++j) {
+          float a0 = is_out[8 * g + 2 * j] ? 0.0f : (float)fabs(sdqo_bf16_to_double(w[8 * g + 2 * j]));
+          float a1 = is_out[8 * g + 2 * j + 1] ? 0.0f : (float)fabs(sdqo_bf16_to_double(w[8 * g + 2 * j + 1]));
+          volatile float s = a0 + a1;             /* one fp32 round-to-nearest add */
+          score[j] = s;
+        }
+        int j0 = -1, j1 = -1;
+        for (int j = 0; j < 4; ++j) if (j0 < 0 || score[j] > score[j0]) j0 = j;
+        for (int j = 0; j < 4; ++j) if (j != j0 && (j1 < 0 || score[j] > score[j1])) j1 = j;
+        if (j0 > j1) { int t = j0; j0 = j1; j1 = t; }
+        in_meta[n * G8 + g] = (uint8_t)(j0 | (j1 << 2));
+        kept[8 * g + 2 * j0] = kept[8 * g + 2 * j0 + 1] = 1;
+        kept[8 * g + 2 * j1] = kept[8 * g + 2 * j1 + 1] = 1;
+      }
+    } else {
+      for (int64_t h = 0; h < K / 4; ++h) {
+        int i0 = -1, i1 = -1;
+        for (int i = 0; i < 4; ++i) {
+          if (is_out[4 * h + i]) continue;
+          if (i0 < 0 || mag_key(w[4 * h + i]) > mag_key(w[4 * h + i0])) i0 = i;
+        }
+        for (int i = 0; i < 4; ++i) {
+          if (is_out[4 * h + i] || i == i0) continue;
+          if (i1 < 0 || mag_key(w[4 * h + i]) > mag_key(w[4 * h + i1])) i1 = i;
+        }
+        if (i0 > i1) { int t = i0; i0 = i1; i1 = t; }
+        in_meta[n * (K / 4) + h] = (uint8_t)(i0 | (i1 << 2));
+        kept[4 * h + i0] = kept[4 * h + i1] = 1;
+      }
+    }
+
+    /* Stage 3 for inliers: per Q-Vector E8M0 scale over the kept inlier values, then E2M1 codes.
+       A kept slot that holds an outlier position carries the value +0. */
+    for (int64_t b = 0; b < K / Bs; ++b) {
+      double amax = 0.0;
+      for (int64_t k = b * Bs; k < (b + 1) * Bs; ++k)
+        if (kept[k] && !is_out[k]) {
+          double a = fabs(sdqo_bf16_to_double(w[k]));
+          if (a > amax) amax = a;
+        }
+      in_scale[n * (K / Bs) + b] = sdqo_e8m0_scale_code(amax, cfg->scale_rule);
+    }
+    int64_t slot = 0;
+    for (int64_t k = 0; k < K; ++k) {
+      if (!kept[k]) continue;
+      uint8_t code = 0;
+      if (!is_out[k]) {
+        int c = in_scale[n * (K / Bs) + k / Bs];
+        code = sdqo_e2m1_encode(ldexp(sdqo_bf16_to_double(w[k]), 127 - c));
+      }
+      in_code[n * (K / 2) + slot++] = code;
+    }
+  }
+  free(is_out);
+  free(kept);
+  return 0;
+}
+
+/* Dequantize the canonical arrays of ONE weight matrix back to dense W_i and W_o (fp64, [N][K]). */
+int sdqo_dequant_weights(int64_t N, int64_t K, const sdqo_config* cfg,
+                         const uint8_t* in_code, const uint8_t* in_meta, const uint8_t* in_scale,
+                         const uint8_t* out_code, const uint8_t* out_idx, const int32_t* out_sexp,
+                         double* W_in, double* W_out) {
+  const int on = cfg->out_n, Bs = cfg->in_block;
+  const int64_t G8 = K / 8;
+  memset(W_in, 0, sizeof(double) * (size_t)(N * K));
+  memset(W_out, 0, sizeof(double) * (size_t)(N * K));
+  for (int64_t n = 0; n < N; ++n) {
+    int64_t slot = 0;
+    if (cfg->in_gran == SDQO_GRAN_PAIR) {
+      for (int64_t g = 0; g < G8; ++g) {
+        int nib = in_meta[n * G8 + g];
+        int jj[2] = {nib & 3, (nib >> 2) & 3};
+        for (int t = 0; t < 2; ++t)
+          for (int u = 0; u < 2; ++u) {
+            int64_t k = 8 * g + 2 * jj[t] + u;
+            W_in[n * K + k] = sdqo_e2m1_decode(in_code[n * (K / 2) + slot++]) *
+                              sdqo_e8m0_decode(in_scale[n * (K / Bs) + k / Bs]);
+          }
+      }
+    } else {
+      for (int64_t h = 0; h < K / 4; ++h) {
+        int nib = in_meta[n * (K / 4) + h];
+        int ii[2] = {nib & 3, (nib >> 2) & 3};
+        for (int t = 0; t < 2; ++t) {
+          int64_t k = 4 * h + ii[t];
+          W_in[n * K + k] = sdqo_e2m1_decode(in_code[n * (K / 2) + slot++]) *
+                            sdqo_e8m0_decode(in_scale[n * (K / Bs) + k / Bs]);
+        }
+      }
+    }
+    for (int64_t g = 0; g < G8; ++g)
+      for (int t = 0; t < on; ++t) {
+        int64_t k = 8 * g + out_idx[(n * G8 + g) * on + t];
+        W_out[n * K + k] = ldexp(sdqo_e4m3_decode(out_code[(n * G8 + g) * on + t]), out_sexp[n]);
+      }
+  }
+  return 0;
+}
+
+/* ------------------------------------------------------------------ activations: A -> A_i (4-bit), A_o (8-bit)
+ * X [M][K] bf16 patterns.  xq4_code [M][K] E2M1 codes, xq4_scale [M][K/in_block] E8M0 codes,
+ * xq8_code [M][K] E4M3 codes, xq8_sexp [M] exponent e of the per-token scale 2^e.
+ * +-Inf saturates to the largest finite value; NaN is rejected (-2). */
+int sdqo_quantize_act(const uint16_t* X, int64_t M, int64_t K, const sdqo_config* cfg,
+                      uint8_t* xq4_code, uint8_t* xq4_scale, uint8_t* xq8_code, int32_t* xq8_sexp) {
+  if (!X || !cfg || M <= 0 || K <= 0) return -1;
+  if (cfg->in_block != 32 && cfg->in_block != 64) return -1;
+  if (K % cfg->in_block != 0) return -1;
+  const int Bs = cfg->in_block;
+  const double BF16_MAX = 3.3895313892515355e38;
+  for (int64_t m = 0; m < M; ++m) {
+    const uint16_t* x = X + m * K;
+    double row_amax = 0.0;
+    for (int64_t k = 0; k < K; ++k) {
+      if ((x[k] & 0x7F80) == 0x7F80 && (x[k] & 0x007F)) return -2; /* NaN */
+    }
+    for (int64_t b = 0; b < K / Bs; ++b) {
+      double amax = 0.0;
+      for (int64_t k = b * Bs; k < (b + 1) * Bs; ++k) {
+        double a = fabs(sdqo_bf16_to_double(x[k]));
+        if (isinf(a)) a = BF16_MAX;
+        if (a > amax) amax = a;
+      }
+      if (amax > row_amax) row_amax = amax;
+      uint8_t c = sdqo_e8m0_scale_code(amax, cfg->scale_rule);
+      xq4_scale[m * (K / Bs) + b] = c;
+      for (int64_t k = b * Bs; k < (b + 1) * Bs; ++k) {
+        double v = sdqo_bf16_to_double(x[k]);
+        if (isinf(v)) v = copysign(BF16_MAX, v);
+        xq4_code[m * K + k] = sdqo_e2m1_encode(ldexp(v, 127 - (int)c));
+      }
+    }
+    const int e = sdqo_fp8_scale_exp(row_amax);
+    xq8_sexp[m] = e;
+    for (int64_t k = 0; k < K; ++k) {
+      double v = sdqo_bf16_to_double(x[k]);
+      if (isinf(v)) v = copysign(BF16_MAX, v);
+      xq8_code[m * K + k] = sdqo_e4m3_encode(ldexp(v, -e));
+    }
+  }
+  return 0;
+}
+
+/* ------------------------------------------------------------------ the decomposed product, fp64
+ * Y[m][n] = sum_k A_i[m][k] * W_i[n][k]  +  sum_k A_o[m][k] * W_o[n][k]        (O = O_i + O_o)
+ * Rows n in [n_begin, n_end) and tokens m in [0, M) are produced into Y [M][n_end-n_begin].
+ * Only the non-zero weights are visited; every term is formed and added in fp64. */
+int sdqo_linear(int64_t M, int64_t N, int64_t K, const sdqo_config* cfg,
+                const uint8_t* in_code, const uint8_t* in_meta, const uint8_t* in_scale,
+                const uint8_t* out_code, const uint8_t* out_idx, const int32_t* out_sexp,
+                const uint8_t* xq4_code, const uint8_t* xq4_scale, const uint8_t* xq8_code, const int32_t* xq8_sexp,
+                int64_t n_begin, int64_t n_end, double* Y, int n_threads) {
+  if (n_begin < 0 || n_end > N || n_begin > n_end) return -1;
+  const int on = cfg->out_n, Bs = cfg->in_block;
+  const int64_t G8 = K / 8, NB = n_end - n_begin;
+  double* A_i = (double*)malloc(sizeof(double) * (size_t)(M * K));
+  double* A_o = (double*)malloc(sizeof(double) * (size_t)(M * K));
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t k = 0; k < K; ++k) {
+      A_i[m * K + k] = sdqo_e2m1_decode(xq4_code[m * K + k]) * sdqo_e8m0_decode(xq4_scale[m * (K / Bs) + k / Bs]);
+      A_o[m * K + k] = ldexp(sdqo_e4m3_decode(xq8_code[m * K + k]), xq8_sexp[m]);
+    }
+#pragma omp parallel num_threads(n_threads > 0 ? n_threads : 1)
+  {
+    int32_t* ki = (int32_t*)malloc(sizeof(int32_t) * (size_t)(K / 2));
+    double* wi = (double*)malloc(sizeof(double) * (size_t)(K / 2));
+    int32_t* ko = (int32_t*)malloc(sizeof(int32_t) * (size_t)(G8 * 2));
+    double* wo = (double*)malloc(sizeof(double) * (size_t)(G8 * 2));
+#pragma omp for schedule(static)
+    for (int64_t n = n_begin; n < n_end; ++n) {
+      /* positions and values of the non-zeros of row n of W_i and W_o */
+      int64_t ni = 0, no = 0, slot = 0;
+      if (cfg->in_gran == SDQO_GRAN_PAIR) {
+        for (int64_t g = 0; g < G8; ++g) {
+          int nib = in_meta[n * G8 + g];
+          int jj[2] = {nib & 3, (nib >> 2) & 3};
+          for (int t = 0; t < 2; ++t)
+            for (int u = 0; u < 2; ++u) {
+              int64_t k = 8 * g + 2 * jj[t] + u;
+              ki[ni] = (int32_t)k;
+              wi[ni++] = sdqo_e2m1_decode(in_code[n * (K / 2) + slot++]) *
+                         sdqo_e8m0_decode(in_scale[n * (K / Bs) + k / Bs]);
+            }
+        }
+      } else {
+        for (int64_t h = 0; h < K / 4; ++h) {
+          int nib = in_meta[n * (K / 4) + h];
+          int ii[2] = {nib & 3, (nib >> 2) & 3};
+          for (int t = 0; t < 2; ++t) {
+            int64_t k = 4 * h + ii[t];
+            ki[ni] = (int32_t)k;
+            wi[ni++] = sdqo_e2m1_decode(in_code[n * (K / 2) + slot++]) *
+                       sdqo_e8m0_decode(in_scale[n * (K / Bs) + k / Bs]);
+          }
+        }
+      }
+      for (int64_t g = 0; g < G8; ++g)
+        for (int t = 0; t < on; ++t) {
+          ko[no] = (int32_t)(8 * g + out_idx[(n * G8 + g) * on + t]);
+          wo[no++] = ldexp(sdqo_e4m3_decode(out_code[(n * G8 + g) * on + t]), out_sexp[n]);
+        }
+      for (int64_t m = 0; m < M; ++m) {
+        double acc = 0.0;
+        for (int64_t t = 0; t < ni; ++t) acc += A_i[m * K + ki[t]] * wi[t];
+        for (int64_t t = 0; t < no; ++t) acc += A_o[m * K + ko[t]] * wo[t];
+        Y[m * NB + (n - n_begin)] = acc;
+      }
+    }
+    free(ki); free(wi); free(ko); free(wo);
+  }
+  free(A_i);
+  free(A_o);
+  return 0;
+}
+
+/* ------------------------------------------------------------------ the paper's accounting (Section 3)
+ * Average bits per weight element of the compressed format: data + index metadata + scale metadata.
+ * An N:M part with b-bit values stores N*b data bits and N*ceil(log2 M) index bits per S-Vector of M
+ * ("ELLPACK-like": one index per non-zero); a scale of s bits per Q-Vector of q logical elements
+ * adds s/q. */
+double sdqo_bits_per_weight_part(int n, int m, int value_bits, int scale_bits, int qvec) {
+  int idx_bits = 0;
+  while ((1 << idx_bits) < m) ++idx_bits;
+  if (n == m) idx_bits = 0; /* dense: no index metadata */
+  double bits = ((double)n * value_bits + (double)n * idx_bits) / (double)m;
+  if (qvec > 0) bits += (double)scale_bits / (double)qvec;
+  return bits;
+}
+
+/* Effective compute throughput model: an N:M part computed with b-bit operands costs
+ * (N/M) * (b/16) of the fp16-dense time; the SDQ layer costs the sum of its two parts. */
+double sdqo_relative_cost(int n, int m, int bits) { return ((double)n / m) * ((double)bits / 16.0); }

@@ -1,0 +1,98 @@
+"""An independent dense statement of the SDQ decomposition used ONLY to pin the oracle.
+
+It never builds packed arrays: it computes masks and quantized dense matrices directly with
+vectorised numpy, threshold-based E2M1 rounding and torch's own float8_e4m3fn cast, i.e. with none
+of the oracle's routines.
+"""
+import numpy as np
+import torch
+
+E2M1_VALUES = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+
+
+def bf16_to_f64(bits):
+    return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).double().numpy()
+
+
+def q_e2m1(v):
+    """round |v| to the E2M1 grid, ties to the neighbour with even code, saturate at 6; keeps sign."""
+    a = np.abs(v)
+    mids = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0])
+    tie_up = np.array([False, True, False, True, False, True, False])
+    code = np.zeros(a.shape, dtype=np.int64)
+    for i in range(7):
+        code = np.where((a > mids[i]) | ((a == mids[i]) & tie_up[i]), i + 1, code)
+    return np.copysign(E2M1_VALUES[code], v)
+
+
+def q_e4m3(v):
+    t = torch.from_numpy(np.ascontiguousarray(v)).to(torch.float32)
+    assert (t.abs() <= 448).all()
+    return t.to(torch.float8_e4m3fn).double().numpy()
+
+
+def floor_log2(a):
+    m, e = np.frexp(a)          # a = m * 2^e, m in [0.5, 1)
+    return e - 1
+
+
+def ceil_exp(amax, vmax):
+    """smallest integer e with amax <= vmax * 2^e (amax > 0)"""
+    e = np.ceil(np.log2(amax / vmax)).astype(np.int64)
+    e = np.where(amax > np.ldexp(vmax, e), e + 1, e)
+    e = np.where(amax <= np.ldexp(vmax, e - 1), e - 1, e)
+    return e
+
+
+def block_scale_exp(amax, rule_floor):
+    E = np.where(amax > 0, floor_log2(np.where(amax > 0, amax, 1.0)) - 2 if rule_floor
+                 else ceil_exp(np.where(amax > 0, amax, 1.0), 6.0), -127)
+    return np.clip(E, -127, 127)
+
+
+def top_mask(keys, n):
+    """mask of the n largest along the last axis, ties to the lower index"""
+    order = np.argsort(-keys, axis=-1, kind="stable")
+    mask = np.zeros(keys.shape, dtype=bool)
+    np.put_along_axis(mask, order[..., :n], True, axis=-1)
+    return mask
+
+
+def decompose_dense(W_bits, out_n, pair, block, rule_floor):
+    """returns (W_in_hat, W_out_hat, mask_in_slots, mask_out) as dense [N, K] arrays"""
+    W = bf16_to_f64(W_bits)
+    N, K = W.shape
+    A = np.abs(W)
+    mask_out = top_mask(A.reshape(N, K // 8, 8), out_n).reshape(N, K) if out_n else np.zeros((N, K), bool)
+    R = np.where(mask_out, 0.0, A)
+    if pair:
+        r32 = R.astype(np.float32).reshape(N, K // 8, 4, 2)
+        score = (r32[..., 0] + r32[..., 1]).astype(np.float32)
+        keep_pair = top_mask(score, 2)
+        slots = np.repeat(keep_pair, 2, axis=-1).reshape(N, K)
+    else:
+        keys = np.where(mask_out, -1.0, A).reshape(N, K // 4, 4)
+        slots = top_mask(keys, 2).reshape(N, K)
+    inl = slots & ~mask_out
+    Win = np.where(inl, W, 0.0)
+    amax = np.abs(Win).reshape(N, K // block, block).max(-1)
+    E = block_scale_exp(amax, rule_floor)
+    Es = np.repeat(E, block, axis=1)
+    Win_hat = np.where(inl, np.ldexp(q_e2m1(np.ldexp(Win, -Es)), Es), 0.0)
+    Wout = np.where(mask_out, W, 0.0)
+    oamax = np.abs(Wout).max(axis=1)
+    e = np.where(oamax > 0, ceil_exp(np.where(oamax > 0, oamax, 1.0), 448.0), 0)[:, None]
+    Wout_hat = np.ldexp(q_e4m3(np.ldexp(Wout, -e)), e)
+    return Win_hat, Wout_hat, slots, mask_out
+
+
+def quantize_act_dense(X_bits, block, rule_floor):
+    X = bf16_to_f64(X_bits)
+    M, K = X.shape
+    amax = np.abs(X).reshape(M, K // block, block).max(-1)
+    Es = np.repeat(block_scale_exp(amax, rule_floor), block, axis=1)
+    A_i = np.ldexp(q_e2m1(np.ldexp(X, -Es)), Es)
+    ramax = np.abs(X).max(axis=1)
+    e = np.where(ramax > 0, ceil_exp(np.where(ramax > 0, ramax, 1.0), 448.0), 0)[:, None]
+    A_o = np.ldexp(q_e4m3(np.ldexp(X, -e)), e)
+    return A_i, A_o

@@ -1,0 +1,187 @@
+"""Pins for the oracle's decomposition (Stages 1-3) and activation quantization."""
+import itertools
+
+import numpy as np
+import pytest
+
+import sdq_synth
+from oracle import sdq_oracle as so
+from tests.indep_definition import bf16_to_f64, decompose_dense, quantize_act_dense
+
+CFGS = [so.Config(1, so.GRAN_PAIR, 64, so.SCALE_OCP_FLOOR),
+        so.Config(1, so.GRAN_ELEM, 32, so.SCALE_OCP_FLOOR),
+        so.Config(2, so.GRAN_PAIR, 64, so.SCALE_CEIL_NOSAT),
+        so.Config(0, so.GRAN_PAIR, 64, so.SCALE_OCP_FLOOR),
+        so.Config(2, so.GRAN_ELEM, 64, so.SCALE_OCP_FLOOR),
+        so.Config(0, so.GRAN_ELEM, 32, so.SCALE_CEIL_NOSAT)]
+
+
+def tiny_W(N=64, K=256, seed=0):
+    return sdq_synth.bf16_bits(sdq_synth.make_weight(N, K, seed))
+
+
+@pytest.mark.parametrize("cfg", CFGS)
+def test_nm_invariants(cfg):
+    """at most out_n outliers per 8; exactly 2 kept pairs per 8 / 2 kept per 4; disjoint supports"""
+    Wb = tiny_W()
+    p = so.decompose(Wb, cfg)
+    W_in, W_out = so.dequant_weights(p)
+    N, K = Wb.shape
+    assert ((W_out != 0).reshape(N, K // 8, 8).sum(-1) <= cfg.out_n).all()
+    assert not ((W_in != 0) & (W_out != 0)).any()
+    if cfg.in_gran == so.GRAN_PAIR:
+        j0, j1 = p.in_meta & 3, (p.in_meta >> 2) & 3
+        assert (j0 < j1).all()
+        pair_nz = (W_in != 0).reshape(N, K // 8, 4, 2).any(-1)
+        assert (pair_nz.sum(-1) <= 2).all()
+    else:
+        i0, i1 = p.in_meta & 3, (p.in_meta >> 2) & 3
+        assert (i0 < i1).all()
+        assert ((W_in != 0).reshape(N, K // 4, 4).sum(-1) <= 2).all()
+    if cfg.out_n:
+        assert (np.diff(p.out_idx.astype(int), axis=-1) > 0).all()
+        assert (p.out_idx < 8).all()
+
+
+@pytest.mark.parametrize("cfg", CFGS)
+def test_matches_independent_dense_definition(cfg):
+    """W_in + W_out equals the pruned-quantized W computed by an independent routine"""
+    for seed in (0, 1):
+        Wb = tiny_W(48, 512, seed)
+        p = so.decompose(Wb, cfg)
+        W_in, W_out = so.dequant_weights(p)
+        ref_in, ref_out, slots, mask_out = decompose_dense(Wb, cfg.out_n, cfg.in_gran == so.GRAN_PAIR, cfg.in_block,
+                                                           cfg.scale_rule == so.SCALE_OCP_FLOOR)
+        assert np.array_equal(W_out, ref_out)
+        assert np.array_equal(W_in, ref_in)
+        assert np.array_equal(W_in + W_out, ref_in + ref_out)
+
+
+def test_selection_brute_force_all_choices():
+    """chosen outlier set maximises kept magnitude and is lexicographically first among maximisers;
+    same for the kept pair set (pair score) -- enumerated over all C(8,n) / C(4,2) choices"""
+    rng = np.random.default_rng(5)
+    # few distinct magnitudes -> many ties
+    vals = np.array([0.0, 0.5, 1.0, 1.0, 2.0, -2.0, 3.0, -0.5])
+    W = rng.choice(vals, size=(32, 64))
+    import torch
+    Wb = sdq_synth.bf16_bits(torch.from_numpy(W).to(torch.bfloat16))
+    for out_n in (1, 2):
+        cfg = so.Config(out_n, so.GRAN_PAIR, 64, so.SCALE_OCP_FLOOR)
+        p = so.decompose(Wb, cfg)
+        for n in range(W.shape[0]):
+            for g in range(W.shape[1] // 8):
+                a = np.abs(W[n, 8 * g:8 * g + 8])
+                best, best_set = -1.0, None
+                for comb in itertools.combinations(range(8), out_n):
+                    s = a[list(comb)].sum()
+                    if s > best:
+                        best, best_set = s, comb
+                # lexicographically first maximiser under "largest first, lower index on ties"
+                order = sorted(range(8), key=lambda i: (-a[i], i))[:out_n]
+                assert a[order].sum() == best
+                assert tuple(p.out_idx[n, g]) == tuple(sorted(order))
+                r = a.copy()
+                r[order] = 0.0
+                score = r.reshape(4, 2).sum(-1)
+                bestp = max(itertools.combinations(range(4), 2), key=lambda c: (score[list(c)].sum(), ))
+                porder = sorted(sorted(range(4), key=lambda j: (-score[j], j))[:2])
+                assert score[porder].sum() == score[list(bestp)].sum()
+                assert (int(p.in_meta[n, g]) & 3, int(p.in_meta[n, g]) >> 2) == tuple(porder)
+
+
+def test_on_grid_weights_round_trip_exactly():
+    """weights that already lie on the E2M1*2^E / E4M3*2^e grids with a valid pattern survive unchanged"""
+    rng = np.random.default_rng(3)
+    N, K = 16, 256
+    W = np.zeros((N, K))
+    e2m1 = np.array([0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+    for n in range(N):
+        for g in range(K // 8):
+            o = rng.integers(0, 8)
+            W[n, 8 * g + o] = rng.choice([-1, 1]) * 16.0 * (1 + rng.integers(0, 8) / 8)   # E4M3-exact, dominates
+            pairs = [j for j in range(4)]
+            free = [j for j in pairs if j != o // 2]
+            keep = rng.choice(free, size=2, replace=False)
+            for j in keep:
+                for u in range(2):
+                    W[n, 8 * g + 2 * j + u] = rng.choice([-1, 1]) * rng.choice(e2m1) * 0.125
+        # make sure every 64-block has amax = 6*0.125 so the shared scale is 2^-3 under both rules
+        for b in range(K // 64):
+            g = 8 * b
+            o_pos = np.nonzero(np.abs(W[n, 8 * g:8 * g + 8]) >= 16)[0][0]
+            j = [j for j in range(4) if j != o_pos // 2 and W[n, 8 * g + 2 * j] != 0][0]
+            W[n, 8 * g + 2 * j] = 0.75
+    import torch
+    Wb = sdq_synth.bf16_bits(torch.from_numpy(W).to(torch.bfloat16))
+    assert np.array_equal(bf16_to_f64(Wb), W)
+    for rule in (so.SCALE_OCP_FLOOR, so.SCALE_CEIL_NOSAT):
+        p = so.decompose(Wb, so.Config(1, so.GRAN_PAIR, 64, rule))
+        W_in, W_out = so.dequant_weights(p)
+        assert np.array_equal(W_in + W_out, W)
+
+
+def test_ceil_rule_never_saturates_floor_rule_only_in_6_to_8():
+    Wb = tiny_W(64, 512, 9)
+    W = bf16_to_f64(Wb)
+    for rule in (so.SCALE_OCP_FLOOR, so.SCALE_CEIL_NOSAT):
+        cfg = so.Config(1, so.GRAN_PAIR, 64, rule)
+        p = so.decompose(Wb, cfg)
+        W_in, _ = so.dequant_weights(p)
+        sc = np.repeat(np.ldexp(1.0, p.in_scale.astype(int) - 127), 64, axis=1)
+        scaled = np.abs(np.where(W_in != 0, W, 0.0)) / sc
+        if rule == so.SCALE_CEIL_NOSAT:
+            assert scaled.max() <= 6.0
+        else:
+            assert scaled.max() < 8.0
+
+
+def test_all_zero_and_ties_pick_lowest_indices():
+    Wb = np.zeros((4, 128), np.uint16)
+    p = so.decompose(Wb, so.Config(2, so.GRAN_PAIR, 64, so.SCALE_OCP_FLOOR))
+    assert (p.out_idx[..., 0] == 0).all() and (p.out_idx[..., 1] == 1).all()
+    assert (p.in_meta == (0 | (1 << 2))).all()
+    assert (p.in_code == 0).all() and (p.in_scale == 0).all() and (p.out_sexp == 0).all()
+    p = so.decompose(Wb, so.Config(1, so.GRAN_ELEM, 32, so.SCALE_OCP_FLOOR))
+    # group of 4 that contains the outlier (position 0) keeps elements 1,2; the other keeps 0,1
+    assert (p.in_meta[:, 0::2] == (1 | (2 << 2))).all()
+    assert (p.in_meta[:, 1::2] == (0 | (1 << 2))).all()
+
+
+def test_nonfinite_weight_rejected():
+    Wb = tiny_W(8, 128, 0)
+    Wb[3, 5] = 0x7F80
+    with pytest.raises(ValueError):
+        so.decompose(Wb, so.Config())
+
+
+@pytest.mark.parametrize("cfg", CFGS[:3])
+def test_activation_quantization_matches_independent_definition(cfg):
+    Xb = sdq_synth.bf16_bits(sdq_synth.make_act(24, 512, 4, n_outlier_channels=5))
+    q = so.quantize_act(Xb, cfg)
+    A_i, A_o = so.dequant_act(q)
+    ref_i, ref_o = quantize_act_dense(Xb, cfg.in_block, cfg.scale_rule == so.SCALE_OCP_FLOOR)
+    assert np.array_equal(A_i, ref_i)
+    assert np.array_equal(A_o, ref_o)
+    # nothing saturates in the 8-bit copy; it is within half an E4M3 ulp (2^-4 relative) of x
+    X = bf16_to_f64(Xb)
+    assert (np.abs(A_o - X) <= np.abs(X) * 2.0 ** -4 + 2.0 ** (q.xq8_sexp[:, None].astype(float) - 10)).all()
+
+
+def test_block64_scale_is_max_of_the_two_block32_scales():
+    Xb = sdq_synth.bf16_bits(sdq_synth.make_act(16, 256, 11))
+    q64 = so.quantize_act(Xb, so.Config(1, so.GRAN_PAIR, 64, so.SCALE_OCP_FLOOR))
+    q32 = so.quantize_act(Xb, so.Config(1, so.GRAN_PAIR, 32, so.SCALE_OCP_FLOOR))
+    assert np.array_equal(q64.xq4_scale, q32.xq4_scale.reshape(16, -1, 2).max(-1))
+
+
+def test_activation_inf_saturates_nan_rejected():
+    Xb = sdq_synth.bf16_bits(sdq_synth.make_act(2, 128, 1))
+    Xb[0, 3] = 0x7F80   # +inf
+    Xb[1, 9] = 0xFF80   # -inf
+    q = so.quantize_act(Xb, so.Config())
+    assert q.xq4_code[0, 3] == 7 and q.xq4_code[1, 9] == 15
+    assert q.xq8_code[0, 3] in (0x7E, 0x7D, 0x7C, 0x7B, 0x7A, 0x79, 0x78)  # top binade, no NaN code
+    Xb[0, 0] = 0x7FC0
+    with pytest.raises(ValueError):
+        so.quantize_act(Xb, so.Config())
