@@ -1,0 +1,156 @@
+/*
+ * sdq.h -- C-ABI of the B200 (sm_100a) SDQ decomposed linear layer
+ *
+ *     Y = A_i * W_i^T + A_o * W_o^T
+ *
+ * following "SDQ: Sparse Decomposed Quantization for LLM Inference" (arXiv 2406.13868):
+ *   Section 5, Stage 1 (N:M magnitude sparsification), Stage 2 (local N:M outlier extraction per
+ *   S-Vector), Stage 3 (different number formats for inliers and outliers, activations quantized
+ *   accordingly) and the paragraph "LLM inference performance" (O = O_o + O_i).
+ *
+ * Conventions
+ *   W [N, K] bf16, row-major (row = output feature, K contiguous);  X [M, K] bf16;  Y [M, N].
+ *   "device" pointers are CUDA device memory of the current device; "host" pointers are plain
+ *   host memory.  The library never allocates or frees device memory: every buffer is owned by the
+ *   caller and sized with the *_size queries.  All launches go to the caller's stream; nothing
+ *   synchronises unless stated.  Every function returns a status code; nothing throws or aborts.
+ *   Preconditions: N % 128 == 0, K % 256 == 0, M >= 1, 16-byte aligned pointers, finite weights.
+ */
+#ifndef SDQ_H_
+#define SDQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SDQ_OK = 0,
+  SDQ_ERR_INVALID_ARG = 1,      /* null pointer, bad enum value                              */
+  SDQ_ERR_SHAPE = 2,            /* N, K, M violate the preconditions or operands disagree    */
+  SDQ_ERR_ALIGNMENT = 3,        /* pointer or leading dimension not 16-byte aligned          */
+  SDQ_ERR_UNSUPPORTED = 4,      /* valid config that this kernel set cannot execute          */
+  SDQ_ERR_BUFFER_TOO_SMALL = 5, /* caller buffer smaller than the matching *_size query      */
+  SDQ_ERR_NONFINITE = 6,        /* Inf/NaN weight seen by sdq_decompose                      */
+  SDQ_ERR_CUDA = 7,             /* a CUDA runtime call failed (launch error etc.)            */
+  SDQ_ERR_TIMEOUT = 8           /* a bounded device-side wait gave up (sticky device status) */
+} sdq_status_t;
+
+enum { SDQ_GRAN_PAIR = 0, SDQ_GRAN_ELEM = 1 };           /* inlier N:M granularity            */
+enum { SDQ_SCALE_OCP_FLOOR = 0, SDQ_SCALE_CEIL_NOSAT = 1 }; /* E8M0 Q-Vector scale rule        */
+
+/* "pattern, formats" of the decomposition (Section 5, Stages 1-3).
+ *   out_n      outliers extracted per S-Vector of 8 consecutive K (Stage 2): 0, 1 or 2; stored as
+ *              FP8-E4M3 with one power-of-two scale per weight row.
+ *   in_gran    how the remaining values are pruned to 50% (Stage 1, magnitude metric):
+ *              SDQ_GRAN_PAIR keeps the 2 adjacent pairs (of 4) with the largest |a|+|b| in every 8
+ *              (the pattern the sparse FP4 tensor core consumes); SDQ_GRAN_ELEM keeps the 2 largest
+ *              of every 4 (decompose/export only; sdq_linear returns SDQ_ERR_UNSUPPORTED).
+ *   in_block   Q-Vector length: logical K sharing one E8M0 scale, for W_i and for the 4-bit
+ *              activations (64 is what sdq_linear executes; 32 is decompose/quantize/export only).
+ *   scale_rule E8M0 exponent from the Q-Vector's largest magnitude a: OCP_FLOOR = floor(log2 a) - 2,
+ *              CEIL_NOSAT = smallest E with a <= 6 * 2^E.
+ */
+typedef struct {
+  int32_t out_n;
+  int32_t in_gran;
+  int32_t in_block;
+  int32_t scale_rule;
+} sdq_config_t;
+
+/* Host-side descriptor of a packed weight matrix (filled by sdq_decompose; plain data, may be
+ * copied; `dev` stays owned by the caller).  off[] are byte offsets of the sections inside dev:
+ *   0 inlier stages  1 outlier stages (tensor-core 2:4 form)  2 outlier row-scale atoms
+ *   3 compact outlier codes  4 compact outlier indices  5 outlier scale exponents  6,7 reserved */
+typedef struct {
+  void* dev;
+  size_t bytes;
+  int64_t N, K;
+  sdq_config_t cfg;
+  size_t off[8];
+} sdq_packed_t;
+
+/* Host-side descriptor of a quantized activation matrix (filled by sdq_quantize_act).
+ *   off: 0 activation stages (4-bit codes | 8-bit codes | 4-bit scales per 128-token x 256-K tile)
+ *        1 per-token 8-bit scale atoms   2 per-token 8-bit scale exponents   3.. reserved */
+typedef struct {
+  void* dev;
+  size_t bytes;
+  int64_t M, K;
+  sdq_config_t cfg;
+  size_t off[6];
+} sdq_act_t;
+
+/* Layout-free copies of the packed arrays, one code per byte, for bit-exact comparison
+ * (all pointers: device memory, caller-owned, sizes in elements given beside each field). */
+typedef struct {
+  uint8_t* in_code;   /* [N][K/2]   E2M1 codes of the kept inlier slots in ascending k            */
+  uint8_t* in_meta;   /* [N][K/8] (PAIR) or [N][K/4] (ELEM): i0 | i1<<2, kept indices, ascending  */
+  uint8_t* in_scale;  /* [N][K/in_block] E8M0 codes                                               */
+  uint8_t* out_code;  /* [N][K/8][out_n] E4M3 codes                                               */
+  uint8_t* out_idx;   /* [N][K/8][out_n] position 0..7 in the S-Vector, ascending                 */
+  int32_t* out_sexp;  /* [N] exponent e of the row scale 2^e                                      */
+} sdq_canonical_t;
+
+typedef struct {
+  uint8_t* xq4_code;  /* [M][K] E2M1 codes           */
+  uint8_t* xq4_scale; /* [M][K/in_block] E8M0 codes  */
+  uint8_t* xq8_code;  /* [M][K] E4M3 codes           */
+  int32_t* xq8_sexp;  /* [M] exponent e of the per-token scale 2^e */
+} sdq_act_canonical_t;
+
+/* Size of the packed-weight buffer for an N x K matrix.  *bytes: what sdq_decompose needs;
+ * *algorithmic_bytes: the paper's accounting (Section 3.3: values + one index per non-zero + one
+ * scale per Q-Vector), the numerator of the decode GB/s metric.  Either out pointer may be NULL. */
+sdq_status_t sdq_packed_size(int64_t N, int64_t K, const sdq_config_t* cfg, size_t* bytes,
+                             size_t* algorithmic_bytes);
+
+/* Section 5, Stages 2 -> 1 -> 3 on one weight matrix: per S-Vector of 8 along K take the out_n
+ * largest |w| as outliers, prune the rest to the inlier N:M pattern by magnitude, quantize
+ * outliers to E4M3 with a per-row power-of-two scale and inliers to E2M1 with an E8M0 scale per
+ * Q-Vector, and write codes, scales and sparsity metadata in the tiled layout sdq_linear streams.
+ *   W (device) [N][ldw] bf16, ldw >= K elements; packed_buf (device) >= *bytes of sdq_packed_size;
+ *   out (host) receives the descriptor.  Enqueues on `stream`, then synchronises that stream once
+ *   to read back the non-finite flag.  Errors: INVALID_ARG, SHAPE, ALIGNMENT, BUFFER_TOO_SMALL,
+ *   NONFINITE (buffer contents undefined), CUDA. */
+sdq_status_t sdq_decompose(const void* W_bf16, int64_t N, int64_t K, int64_t ldw, const sdq_config_t* cfg,
+                           void* packed_buf, size_t packed_bytes, sdq_packed_t* out, void* stream);
+
+/* Untile a packed weight buffer into the canonical arrays (parity surface). Asynchronous. */
+sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canonical_t* out, void* stream);
+
+/* Size of the quantized-activation buffer for M tokens of K features. */
+sdq_status_t sdq_act_size(int64_t M, int64_t K, const sdq_config_t* cfg, size_t* bytes);
+
+/* "We also quantize activations accordingly" (Section 5, Stage 3; A -> A_o, A_i in Section 5.1):
+ * per token and Q-Vector an E8M0 scale and E2M1 codes (A_i); per token a power-of-two scale and
+ * E4M3 codes (A_o).  X (device) [M][ldx] bf16; xq_buf (device) >= sdq_act_size bytes; out (host).
+ * +-Inf saturates, NaN input is undefined.  Asynchronous on `stream`. */
+sdq_status_t sdq_quantize_act(const void* X_bf16, int64_t M, int64_t K, int64_t ldx, const sdq_config_t* cfg,
+                              void* xq_buf, size_t xq_bytes, sdq_act_t* out, void* stream);
+
+/* Untile a quantized activation buffer into canonical arrays (parity surface). Asynchronous. */
+sdq_status_t sdq_act_export(const sdq_act_t* Xq, const sdq_act_canonical_t* out, void* stream);
+
+/* The decomposed product of Section 5.1, O = O_o + O_i, both sparse products accumulated in fp32 in
+ * one accumulator: Y[m][n] = sum_k A_i[m][k] W_i[n][k] + sum_k A_o[m][k] W_o[n][k].
+ *   Xq, P (host descriptors; K and cfg must agree); Y (device) [M][ldy] bf16 (round to nearest even
+ *   of the fp32 accumulator); ldy >= N elements, ldy % 8 == 0.  Asynchronous on `stream`.
+ *   Errors: INVALID_ARG, SHAPE, ALIGNMENT, UNSUPPORTED (in_gran != PAIR or in_block != 64), CUDA. */
+sdq_status_t sdq_linear(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y_bf16, int64_t ldy, void* stream);
+
+/* Same product, storing the fp32 accumulator itself (the value the bf16 output is rounded from). */
+sdq_status_t sdq_linear_f32(const sdq_act_t* Xq, const sdq_packed_t* P, float* Y_f32, int64_t ldy, void* stream);
+
+/* Synchronises `stream` and returns the sticky device-side status (SDQ_OK or SDQ_ERR_TIMEOUT when a
+ * bounded wait inside a kernel gave up), clearing it. */
+sdq_status_t sdq_device_status(void* stream);
+
+const char* sdq_status_string(sdq_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SDQ_H_ */

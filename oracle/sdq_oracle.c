@@ -123,8 +123,15 @@ uint8_t sdqo_e8m0_scale_code(double amax, int scale_rule) {
   return (uint8_t)c;
 }
 
-/* exponent e of the power-of-two scale 2^e used for 8-bit (E4M3) operands: nothing saturates */
-int sdqo_fp8_scale_exp(double amax) { return ceil_exp(amax, 448.0); }
+/* exponent e of the power-of-two scale 2^e used for 8-bit (E4M3) operands: nothing saturates.
+ * The scale must be expressible as an E8M0 byte (code e + 127 in 0..254), so e is limited to
+ * [-127, 127]; only rows whose largest magnitude is below 448 * 2^-127 are affected. */
+int sdqo_fp8_scale_exp(double amax) {
+  int e = ceil_exp(amax, 448.0);
+  if (e < -127) e = -127;
+  if (e > 127) e = 127;
+  return e;
+}
 
 /* magnitude key used by every "largest" selection: the 15 low bits of the bf16 pattern */
 static int mag_key(uint16_t h) { return (int)(h & 0x7FFF); }

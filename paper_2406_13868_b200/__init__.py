@@ -1,0 +1,207 @@
+"""B200-native SDQ decomposed linear layer: thin Python binding over the C-ABI in include/sdq.h.
+
+Argument marshalling only -- every step of the path (weight decomposition + packing, activation
+quantization, the fused sparse GEMM) runs in the CUDA kernels of libsdq_b200.so.  PyTorch supplies
+device memory and streams.  There is no CPU fallback: importing works without a GPU (so the build can
+be checked), but every compute call needs the CUDA library and a CUDA tensor.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass, field
+
+import torch
+
+from .build import LIB, build
+
+GRAN_PAIR, GRAN_ELEM = 0, 1
+SCALE_OCP_FLOOR, SCALE_CEIL_NOSAT = 0, 1
+
+STATUS = ["ok", "invalid_arg", "shape", "alignment", "unsupported", "buffer_too_small", "nonfinite", "cuda", "timeout"]
+
+
+class SdqError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s failed: %s (%d)" % (where, STATUS[code] if 0 <= code < len(STATUS) else "?", code))
+
+
+class Config(ctypes.Structure):
+    """`pattern, formats` of the decomposition (sdq_config_t)."""
+    _fields_ = [("out_n", ctypes.c_int32), ("in_gran", ctypes.c_int32), ("in_block", ctypes.c_int32),
+                ("scale_rule", ctypes.c_int32)]
+
+    def __init__(self, out_n=1, in_gran=GRAN_PAIR, in_block=64, scale_rule=SCALE_OCP_FLOOR):
+        super().__init__(out_n, in_gran, in_block, scale_rule)
+
+
+class _Packed(ctypes.Structure):
+    _fields_ = [("dev", ctypes.c_void_p), ("bytes", ctypes.c_size_t), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("cfg", Config), ("off", ctypes.c_size_t * 8)]
+
+
+class _Act(ctypes.Structure):
+    _fields_ = [("dev", ctypes.c_void_p), ("bytes", ctypes.c_size_t), ("M", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("cfg", Config), ("off", ctypes.c_size_t * 6)]
+
+
+class _Canon(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp")]
+
+
+class _ActCanon(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp")]
+
+
+EXPORTS = ["sdq_packed_size", "sdq_decompose", "sdq_packed_export", "sdq_act_size", "sdq_quantize_act", "sdq_act_export",
+           "sdq_linear", "sdq_linear_f32", "sdq_device_status", "sdq_status_string"]
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the CUDA library; raises if it has not been built (there is no fallback path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB):
+            raise RuntimeError("libsdq_b200.so is missing: run `python -c 'import __graft_entry__ as g; g.build()'` "
+                               "(the SDQ path has no CPU or PyTorch fallback)")
+        L = ctypes.CDLL(LIB)
+        vp, i64, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t
+        L.sdq_packed_size.argtypes = [i64, i64, ctypes.POINTER(Config), ctypes.POINTER(sz), ctypes.POINTER(sz)]
+        L.sdq_decompose.argtypes = [vp, i64, i64, i64, ctypes.POINTER(Config), vp, sz, ctypes.POINTER(_Packed), vp]
+        L.sdq_packed_export.argtypes = [ctypes.POINTER(_Packed), ctypes.POINTER(_Canon), vp]
+        L.sdq_act_size.argtypes = [i64, i64, ctypes.POINTER(Config), ctypes.POINTER(sz)]
+        L.sdq_quantize_act.argtypes = [vp, i64, i64, i64, ctypes.POINTER(Config), vp, sz, ctypes.POINTER(_Act), vp]
+        L.sdq_act_export.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_ActCanon), vp]
+        L.sdq_linear.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_Packed), vp, i64, vp]
+        L.sdq_linear_f32.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_Packed), vp, i64, vp]
+        L.sdq_device_status.argtypes = [vp]
+        L.sdq_status_string.argtypes = [ctypes.c_int]
+        L.sdq_status_string.restype = ctypes.c_char_p
+        for n in EXPORTS[:-1]:
+            getattr(L, n).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise SdqError(code, where)
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _need_cuda(t: torch.Tensor, name: str):
+    if not t.is_cuda:
+        raise ValueError("%s must be a CUDA tensor (the SDQ path has no CPU fallback)" % name)
+
+
+@dataclass
+class PackedWeight:
+    """A decomposed + packed weight matrix: caller-owned device buffer plus its host descriptor."""
+    buf: torch.Tensor
+    desc: _Packed
+    N: int
+    K: int
+    cfg: Config
+    algorithmic_bytes: int
+
+
+@dataclass
+class QuantAct:
+    buf: torch.Tensor
+    desc: _Act
+    M: int
+    K: int
+    cfg: Config
+
+
+def packed_size(N: int, K: int, cfg: Config):
+    b, a = ctypes.c_size_t(), ctypes.c_size_t()
+    _check(lib().sdq_packed_size(N, K, ctypes.byref(cfg), ctypes.byref(b), ctypes.byref(a)), "sdq_packed_size")
+    return b.value, a.value
+
+
+def act_size(M: int, K: int, cfg: Config) -> int:
+    b = ctypes.c_size_t()
+    _check(lib().sdq_act_size(M, K, ctypes.byref(cfg), ctypes.byref(b)), "sdq_act_size")
+    return b.value
+
+
+def sdq_decompose(W: torch.Tensor, cfg: Config | None = None, buf: torch.Tensor | None = None) -> PackedWeight:
+    """W [N, K] bf16 CUDA tensor -> packed inlier/outlier parts (sdq_decompose of the C-ABI)."""
+    cfg = cfg or Config()
+    _need_cuda(W, "W")
+    assert W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
+    N, K = W.shape
+    nbytes, algo = packed_size(N, K, cfg)
+    if buf is None:
+        buf = torch.empty(nbytes, dtype=torch.uint8, device=W.device)
+    d = _Packed()
+    _check(lib().sdq_decompose(W.data_ptr(), N, K, W.stride(0), ctypes.byref(cfg), buf.data_ptr(), buf.numel(),
+                               ctypes.byref(d), _stream()), "sdq_decompose")
+    return PackedWeight(buf, d, N, K, cfg, algo)
+
+
+def sdq_quantize_act(X: torch.Tensor, cfg: Config | None = None, buf: torch.Tensor | None = None) -> QuantAct:
+    """X [M, K] bf16 CUDA tensor -> 4-bit block-scaled and 8-bit per-token-scaled activations."""
+    cfg = cfg or Config()
+    _need_cuda(X, "X")
+    assert X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    M, K = X.shape
+    if buf is None:
+        buf = torch.empty(act_size(M, K, cfg), dtype=torch.uint8, device=X.device)
+    d = _Act()
+    _check(lib().sdq_quantize_act(X.data_ptr(), M, K, X.stride(0), ctypes.byref(cfg), buf.data_ptr(), buf.numel(),
+                                  ctypes.byref(d), _stream()), "sdq_quantize_act")
+    return QuantAct(buf, d, M, K, cfg)
+
+
+def sdq_linear(xq: QuantAct, p: PackedWeight, out: torch.Tensor | None = None, f32: bool = False) -> torch.Tensor:
+    """Y [M, N] = A_i W_i^T + A_o W_o^T (bf16, or the fp32 accumulator itself with f32=True)."""
+    dt = torch.float32 if f32 else torch.bfloat16
+    if out is None:
+        out = torch.empty((xq.M, p.N), dtype=dt, device=p.buf.device)
+    assert out.dtype == dt and out.shape == (xq.M, p.N) and out.stride(1) == 1
+    fn = lib().sdq_linear_f32 if f32 else lib().sdq_linear
+    _check(fn(ctypes.byref(xq.desc), ctypes.byref(p.desc), out.data_ptr(), out.stride(0), _stream()), "sdq_linear")
+    return out
+
+
+def packed_export(p: PackedWeight) -> dict:
+    N, K, on = p.N, p.K, p.cfg.out_n
+    dev = p.buf.device
+    nmeta = K // 8 if p.cfg.in_gran == GRAN_PAIR else K // 4
+    t = dict(in_code=torch.zeros((N, K // 2), dtype=torch.uint8, device=dev),
+             in_meta=torch.zeros((N, nmeta), dtype=torch.uint8, device=dev),
+             in_scale=torch.zeros((N, K // p.cfg.in_block), dtype=torch.uint8, device=dev),
+             out_code=torch.zeros((N, K // 8, max(on, 1)), dtype=torch.uint8, device=dev),
+             out_idx=torch.zeros((N, K // 8, max(on, 1)), dtype=torch.uint8, device=dev),
+             out_sexp=torch.zeros((N,), dtype=torch.int32, device=dev))
+    c = _Canon(*[t[n].data_ptr() for n in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp")])
+    _check(lib().sdq_packed_export(ctypes.byref(p.desc), ctypes.byref(c), _stream()), "sdq_packed_export")
+    if on == 0:
+        t["out_code"] = t["out_code"][:, :, :0]
+        t["out_idx"] = t["out_idx"][:, :, :0]
+    return t
+
+
+def act_export(xq: QuantAct) -> dict:
+    M, K = xq.M, xq.K
+    dev = xq.buf.device
+    t = dict(xq4_code=torch.zeros((M, K), dtype=torch.uint8, device=dev),
+             xq4_scale=torch.zeros((M, K // xq.cfg.in_block), dtype=torch.uint8, device=dev),
+             xq8_code=torch.zeros((M, K), dtype=torch.uint8, device=dev),
+             xq8_sexp=torch.zeros((M,), dtype=torch.int32, device=dev))
+    c = _ActCanon(*[t[n].data_ptr() for n in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp")])
+    _check(lib().sdq_act_export(ctypes.byref(xq.desc), ctypes.byref(c), _stream()), "sdq_act_export")
+    return t
+
+
+def device_status() -> int:
+    """Synchronises the current stream and returns (and clears) the sticky device-side status."""
+    return lib().sdq_device_status(_stream())

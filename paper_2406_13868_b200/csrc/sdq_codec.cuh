@@ -1,0 +1,53 @@
+// Device-side number-format helpers of the packer and the activation quantizer.
+// E2M1 / E4M3 encoding uses the hardware converters (round to nearest even, saturate to the largest
+// finite value); scales are powers of two so every scaling below is exact.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp4.h>
+#include <cuda_fp8.h>
+#include <stdint.h>
+
+namespace sdq {
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }
+
+// a = f * 2^p with f in [1, 2):  returns p and f (a > 0, finite; subnormals handled)
+__device__ __forceinline__ void split_pow2(float a, int& p, float& f) {
+  p = ilogbf(a);
+  f = scalbnf(a, -p);
+}
+
+// E8M0 code of the Q-Vector scale of 4-bit values whose largest magnitude is amax
+//   rule 0: E = floor(log2 amax) - 2      rule 1: E = smallest integer with amax <= 6 * 2^E
+__device__ __forceinline__ uint32_t e8m0_scale_code(float amax, int rule) {
+  if (amax == 0.0f) return 0u;
+  int p;
+  float f;
+  split_pow2(amax, p, f);
+  int E = (rule == 0) ? (p - 2) : ((f <= 1.5f) ? (p - 2) : (p - 1));
+  int c = E + 127;
+  return (uint32_t)min(max(c, 0), 254);
+}
+
+// exponent e of the power-of-two scale of an 8-bit (E4M3, max 448 = 1.75 * 2^8) operand:
+// the smallest integer with amax <= 448 * 2^e, limited to what an E8M0 byte can carry
+__device__ __forceinline__ int fp8_scale_exp(float amax) {
+  if (amax == 0.0f) return 0;
+  int p;
+  float f;
+  split_pow2(amax, p, f);
+  int e = (f <= 1.75f) ? (p - 8) : (p - 7);
+  return min(max(e, -127), 127);
+}
+
+// two floats -> two E2M1 codes in one byte (x in the low nibble)
+__device__ __forceinline__ uint32_t e2m1x2(float x, float y) {
+  return (uint32_t)__nv_cvt_float2_to_fp4x2(make_float2(x, y), __NV_E2M1, cudaRoundNearest);
+}
+// two floats -> two E4M3 codes in 16 bits (x in the low byte)
+__device__ __forceinline__ uint32_t e4m3x2(float x, float y) {
+  return (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(x, y), __NV_SATFINITE, __NV_E4M3);
+}
+__device__ __forceinline__ uint32_t e4m3x1(float x) { return (uint32_t)__nv_cvt_float_to_fp8(x, __NV_SATFINITE, __NV_E4M3); }
+
+}  // namespace sdq

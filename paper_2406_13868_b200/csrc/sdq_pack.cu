@@ -1,0 +1,284 @@
+// Offline weight decomposition + packing (Section 5, Stage 2 -> Stage 1 -> Stage 3) and its exporter.
+//
+// One CTA per weight row; one thread per S-Vector of 8 consecutive K (a single 16-byte load).
+// Pass 1 finds the row's largest outlier magnitude (the per-row power-of-two scale); pass 2 selects
+// outliers, prunes the rest pair-wise, derives the Q-Vector scales by an 8-lane shuffle reduction
+// (8 S-Vectors = 64 K), encodes, and scatters into the stage-tiled layout of sdq_layout.h.
+#include "sdq_codec.cuh"
+#include "sdq_internal.h"
+#include "sdq_layout.h"
+
+namespace sdq {
+
+struct GroupSel {
+  uint32_t key[8];   // 15-bit magnitude keys
+  int o0, o1;        // outlier positions (ascending), -1 if absent
+};
+
+// positions of the out_n largest magnitudes, ties to the lower index
+__device__ __forceinline__ void select_outliers(const uint32_t (&key)[8], int out_n, int& o0, int& o1) {
+  o0 = o1 = -1;
+  if (out_n >= 1) {
+    int b = 0;
+#pragma unroll
+    for (int i = 1; i < 8; ++i)
+      if (key[i] > key[b]) b = i;
+    o0 = b;
+  }
+  if (out_n >= 2) {
+    int b = -1;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (i == o0) continue;
+      if (b < 0 || key[i] > key[b]) b = i;
+    }
+    o1 = b;
+    if (o0 > o1) { int t = o0; o0 = o1; o1 = t; }
+  }
+}
+
+__device__ __forceinline__ void load_group(const __nv_bfloat16* w, uint32_t (&bits)[8]) {
+  const uint4 v = *reinterpret_cast<const uint4*>(w);
+  const uint32_t r[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    bits[2 * i] = r[i] & 0xFFFFu;
+    bits[2 * i + 1] = r[i] >> 16;
+  }
+}
+
+__global__ void __launch_bounds__(128)
+pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t ldw, sdq_config_t cfg, uint8_t* __restrict__ blob,
+            PackedOffsets off, uint32_t* __restrict__ flags)
+{
+  const int64_t n = blockIdx.x;
+  const int tid = threadIdx.x;
+  const int G = (int)(K / 8);
+  const int out_n = cfg.out_n;
+  const __nv_bfloat16* wrow = W + n * ldw;
+  __shared__ uint32_t s_red[4];
+  __shared__ int s_e;
+
+  // ---- pass 1: largest outlier magnitude of the row, non-finite check
+  uint32_t okey_max = 0, bad = 0;
+  for (int g = tid; g < G; g += 128) {
+    uint32_t bits[8], key[8];
+    load_group(wrow + 8 * g, bits);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      key[i] = bits[i] & 0x7FFFu;
+      bad |= (key[i] >= 0x7F80u);
+    }
+    int o0, o1;
+    select_outliers(key, out_n, o0, o1);
+    if (o0 >= 0) okey_max = max(okey_max, key[o0]);
+    if (o1 >= 0) okey_max = max(okey_max, key[o1]);
+  }
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) {
+    okey_max = max(okey_max, __shfl_xor_sync(0xffffffffu, okey_max, s));
+    bad |= __shfl_xor_sync(0xffffffffu, bad, s);
+  }
+  if ((tid & 31) == 0) s_red[tid >> 5] = okey_max;
+  if (bad && (tid & 31) == 0) atomicOr(&flags[FLAG_NONFINITE], 1u);
+  __syncthreads();
+  if (tid == 0) {
+    uint32_t m = max(max(s_red[0], s_red[1]), max(s_red[2], s_red[3]));
+    s_e = fp8_scale_exp(bf16_bits_to_float(m));
+  }
+  __syncthreads();
+  const int e = s_e;
+
+  const int64_t rt = n / TILE_ROWS;
+  const uint32_t r = (uint32_t)(n % TILE_ROWS);
+  const int T1 = (int)(K / K1), T2 = (int)(K / K2);
+  const int W1B = w1_bytes(out_n);
+  uint8_t* w1_base = blob + off.w1 + (size_t)rt * T1 * W1B;
+  uint8_t* w2_base = blob + off.w2 + (size_t)rt * T2 * W2_BYTES;
+
+  if (tid == 0) {
+    reinterpret_cast<int32_t*>(blob + off.osexp)[n] = e;
+    const uint32_t c = (uint32_t)(e + 127);
+    *reinterpret_cast<uint32_t*>(blob + off.sfa_out + (size_t)rt * SF_ATOM_BYTES + sf_off(r, 0)) = c * 0x01010101u;
+  }
+
+  // ---- pass 2 (G is a multiple of 32, so whole warps iterate together)
+  for (int g = tid; g < G; g += 128) {
+    uint32_t bits[8], key[8];
+    load_group(wrow + 8 * g, bits);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) key[i] = bits[i] & 0x7FFFu;
+    int o0, o1;
+    select_outliers(key, out_n, o0, o1);
+
+    // Stage 1 on the remaining values: keep the 2 pairs (of 4) with the largest |a| + |b|
+    float score[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float a0 = (2 * j == o0 || 2 * j == o1) ? 0.0f : bf16_bits_to_float(key[2 * j]);
+      const float a1 = (2 * j + 1 == o0 || 2 * j + 1 == o1) ? 0.0f : bf16_bits_to_float(key[2 * j + 1]);
+      score[j] = __fadd_rn(a0, a1);
+    }
+    int j0 = 0;
+#pragma unroll
+    for (int j = 1; j < 4; ++j)
+      if (score[j] > score[j0]) j0 = j;
+    int j1 = -1;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (j == j0) continue;
+      if (j1 < 0 || score[j] > score[j1]) j1 = j;
+    }
+    if (j0 > j1) { int t = j0; j0 = j1; j1 = t; }
+    const int slot_pos[4] = {2 * j0, 2 * j0 + 1, 2 * j1, 2 * j1 + 1};
+
+    // Stage 3, inliers: Q-Vector (64 K = 8 S-Vectors = 8 lanes) largest kept magnitude -> E8M0 scale
+    uint32_t ikey = 0;
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      const int p = slot_pos[s];
+      if (p != o0 && p != o1) ikey = max(ikey, key[p]);
+    }
+    ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 1));
+    ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 2));
+    ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 4));
+    const uint32_t c = e8m0_scale_code(bf16_bits_to_float(ikey), cfg.scale_rule);
+    float v[4];
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      const int p = slot_pos[s];
+      v[s] = (p == o0 || p == o1) ? 0.0f : scalbnf(bf16_bits_to_float(bits[p]), 127 - (int)c);
+    }
+    const uint32_t codes = e2m1x2(v[0], v[1]) | (e2m1x2(v[2], v[3]) << 8);
+
+    const int k1 = g >> 4, k2 = g >> 5;
+    uint8_t* w1 = w1_base + (size_t)k1 * W1B;
+    uint8_t* w2 = w2_base + (size_t)k2 * W2_BYTES;
+    *reinterpret_cast<uint16_t*>(w1 + a_off(r, (uint32_t)(g & 15) * 2)) = (uint16_t)codes;
+    // metadata nibble j0 | j1<<2; two S-Vectors share a byte (even one in the low nibble)
+    uint32_t nib = (uint32_t)(j0 | (j1 << 2));
+    const uint32_t nib_hi = __shfl_down_sync(0xffffffffu, nib, 1);
+    if ((g & 1) == 0) w2[r * 16 + ((g & 31) >> 1)] = (uint8_t)(nib | (nib_hi << 4));
+    if ((g & 7) == 0) w2[E_IN_BYTES + sf_off(r, (uint32_t)((g >> 3) & 3))] = (uint8_t)c;
+
+    if (out_n > 0) {
+      // Stage 3, outliers: E4M3 codes of w / 2^e; compact arrays plus the 2:4 embedding the sparse
+      // FP8 tensor-core path consumes (per 4 K: two ascending slot indices, unused slots hold +0)
+      const uint32_t c0 = e4m3x1(scalbnf(bf16_bits_to_float(bits[o0]), -e));
+      const uint32_t c1 = (o1 >= 0) ? e4m3x1(scalbnf(bf16_bits_to_float(bits[o1]), -e)) : 0u;
+      uint8_t* oc = blob + off.ocode + ((size_t)n * G + g) * out_n;
+      uint8_t* oi = blob + off.oidx + ((size_t)n * G + g) * out_n;
+      oc[0] = (uint8_t)c0;
+      oi[0] = (uint8_t)o0;
+      if (out_n == 2) { oc[1] = (uint8_t)c1; oi[1] = (uint8_t)o1; }
+      uint32_t stored = 0, meta = 0;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int a = (o0 >= 4 * h && o0 < 4 * h + 4) ? (o0 - 4 * h) : -1;
+        const int b = (o1 >= 4 * h && o1 < 4 * h + 4) ? (o1 - 4 * h) : -1;
+        int i0, i1;
+        uint32_t s0 = 0, s1 = 0;
+        if (a >= 0 && b >= 0) { i0 = a; i1 = b; s0 = c0; s1 = c1; }
+        else if (a >= 0 || b >= 0) {
+          const int p = (a >= 0) ? a : b;
+          const uint32_t cc = (a >= 0) ? c0 : c1;
+          if (p < 3) { i0 = p; i1 = 3; s0 = cc; } else { i0 = 0; i1 = 3; s1 = cc; }
+        } else { i0 = 0; i1 = 1; }
+        stored |= (s0 | (s1 << 8)) << (16 * h);
+        meta |= (uint32_t)(i0 | (i1 << 2)) << (4 * h);
+      }
+      *reinterpret_cast<uint32_t*>(w1 + A_IN_BYTES + a_off(r, (uint32_t)(g & 15) * 4)) = stored;
+      w1[A_IN_BYTES + A_OUT_BYTES + r * 16 + (g & 15)] = (uint8_t)meta;
+    }
+  }
+}
+
+// packed buffer -> canonical arrays (one code per byte)
+__global__ void __launch_bounds__(128)
+export_packed_kernel(const uint8_t* __restrict__ blob, int64_t N, int64_t K, sdq_config_t cfg, PackedOffsets off, sdq_canonical_t out)
+{
+  const int64_t n = blockIdx.x;
+  const int G = (int)(K / 8), out_n = cfg.out_n;
+  const int64_t rt = n / TILE_ROWS;
+  const uint32_t r = (uint32_t)(n % TILE_ROWS);
+  const int T1 = (int)(K / K1), T2 = (int)(K / K2), W1B = w1_bytes(out_n);
+  const uint8_t* w1_base = blob + off.w1 + (size_t)rt * T1 * W1B;
+  const uint8_t* w2_base = blob + off.w2 + (size_t)rt * T2 * W2_BYTES;
+  for (int g = threadIdx.x; g < G; g += 128) {
+    const uint8_t* w1 = w1_base + (size_t)(g >> 4) * W1B;
+    const uint8_t* w2 = w2_base + (size_t)(g >> 5) * W2_BYTES;
+    const uint32_t codes = *reinterpret_cast<const uint16_t*>(w1 + a_off(r, (uint32_t)(g & 15) * 2));
+    uint8_t* ic = out.in_code + (size_t)n * (K / 2) + 4 * g;
+    ic[0] = codes & 15; ic[1] = (codes >> 4) & 15; ic[2] = (codes >> 8) & 15; ic[3] = (codes >> 12) & 15;
+    const uint32_t mb = w2[r * 16 + ((g & 31) >> 1)];
+    out.in_meta[(size_t)n * G + g] = (uint8_t)((g & 1) ? (mb >> 4) : (mb & 15));
+    if ((g & 7) == 0) out.in_scale[(size_t)n * (K / 64) + (g >> 3)] = w2[E_IN_BYTES + sf_off(r, (uint32_t)((g >> 3) & 3))];
+    for (int t = 0; t < out_n; ++t) {
+      out.out_code[((size_t)n * G + g) * out_n + t] = blob[off.ocode + ((size_t)n * G + g) * out_n + t];
+      out.out_idx[((size_t)n * G + g) * out_n + t] = blob[off.oidx + ((size_t)n * G + g) * out_n + t];
+    }
+  }
+  if (threadIdx.x == 0) out.out_sexp[n] = reinterpret_cast<const int32_t*>(blob + off.osexp)[n];
+}
+
+}  // namespace sdq
+
+using namespace sdq;
+
+static bool cfg_ok(const sdq_config_t* c) {
+  return c && c->out_n >= 0 && c->out_n <= 2 && (c->in_gran == SDQ_GRAN_PAIR || c->in_gran == SDQ_GRAN_ELEM) &&
+         (c->in_block == 32 || c->in_block == 64) && (c->scale_rule == SDQ_SCALE_OCP_FLOOR || c->scale_rule == SDQ_SCALE_CEIL_NOSAT);
+}
+
+extern "C" sdq_status_t sdq_packed_size(int64_t N, int64_t K, const sdq_config_t* cfg, size_t* bytes, size_t* algorithmic_bytes)
+{
+  if (!cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
+  if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2) return SDQ_ERR_SHAPE;
+  if (cfg->in_gran != SDQ_GRAN_PAIR || cfg->in_block != 64) return SDQ_ERR_UNSUPPORTED;
+  if (bytes) *bytes = packed_offsets(N, K, cfg->out_n).total;
+  if (algorithmic_bytes) {
+    // per weight: 4-bit values on half the positions (2) + two 2-bit pair indices per 8 (0.5) + one
+    // 8-bit scale per 64 (0.125) + out_n * (8 value + 3 index bits) per 8; plus one 32-bit row scale
+    const double bits = 2.0 + 0.5 + 0.125 + cfg->out_n * 11.0 / 8.0;
+    *algorithmic_bytes = (size_t)((double)N * (double)K * bits / 8.0) + (cfg->out_n ? (size_t)N * 4 : 0);
+  }
+  return SDQ_OK;
+}
+
+extern "C" sdq_status_t sdq_decompose(const void* W, int64_t N, int64_t K, int64_t ldw, const sdq_config_t* cfg, void* packed_buf,
+                                      size_t packed_bytes, sdq_packed_t* out, void* stream)
+{
+  if (!W || !packed_buf || !out || !cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
+  if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2 || ldw < K) return SDQ_ERR_SHAPE;
+  if (cfg->in_gran != SDQ_GRAN_PAIR || cfg->in_block != 64) return SDQ_ERR_UNSUPPORTED;
+  if (((uintptr_t)W & 15) || ((uintptr_t)packed_buf & 15) || (ldw % 8)) return SDQ_ERR_ALIGNMENT;
+  const PackedOffsets off = packed_offsets(N, K, cfg->out_n);
+  if (packed_bytes < off.total) return SDQ_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  uint32_t* flags = device_flags();
+  if (!flags) return SDQ_ERR_CUDA;
+  if (cudaMemsetAsync(flags + FLAG_NONFINITE, 0, sizeof(uint32_t), st) != cudaSuccess) return SDQ_ERR_CUDA;
+  pack_kernel<<<(unsigned)N, 128, 0, st>>>((const __nv_bfloat16*)W, N, K, ldw, *cfg, (uint8_t*)packed_buf, off, flags);
+  if (cudaGetLastError() != cudaSuccess) return SDQ_ERR_CUDA;
+  uint32_t nonfinite = 0;
+  if (cudaMemcpyAsync(&nonfinite, flags + FLAG_NONFINITE, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SDQ_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return SDQ_ERR_CUDA;
+  out->dev = packed_buf;
+  out->bytes = off.total;
+  out->N = N;
+  out->K = K;
+  out->cfg = *cfg;
+  for (int i = 0; i < 8; ++i) out->off[i] = 0;
+  out->off[0] = off.w1; out->off[1] = off.w2; out->off[2] = off.sfa_out;
+  out->off[3] = off.ocode; out->off[4] = off.oidx; out->off[5] = off.osexp;
+  return nonfinite ? SDQ_ERR_NONFINITE : SDQ_OK;
+}
+
+extern "C" sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canonical_t* out, void* stream)
+{
+  if (!P || !out || !P->dev || !out->in_code || !out->in_meta || !out->in_scale || !out->out_sexp) return SDQ_ERR_INVALID_ARG;
+  if (P->cfg.out_n > 0 && (!out->out_code || !out->out_idx)) return SDQ_ERR_INVALID_ARG;
+  const PackedOffsets off = packed_offsets(P->N, P->K, P->cfg.out_n);
+  export_packed_kernel<<<(unsigned)P->N, 128, 0, (cudaStream_t)stream>>>((const uint8_t*)P->dev, P->N, P->K, P->cfg, off, *out);
+  return cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
+}

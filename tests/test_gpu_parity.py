@@ -1,0 +1,157 @@
+"""GPU parity: the CUDA path against the CPU oracle, element by element, through the C-ABI."""
+import numpy as np
+import pytest
+import torch
+
+import sdq_synth
+from oracle import sdq_oracle as so
+
+pytestmark = pytest.mark.gpu
+
+
+def sdq():
+    import paper_2406_13868_b200 as m
+    return m
+
+
+def ocfg(out_n=1, rule=0):
+    return so.Config(out_n, so.GRAN_PAIR, 64, rule)
+
+
+def y_close(y_gpu, y_ref):
+    """spec criterion on the fp32 accumulator: |d| <= 1e-3 * (|y| + 1e-2)"""
+    d = np.abs(y_gpu.astype(np.float64) - y_ref)
+    tol = 1e-3 * (np.abs(y_ref) + 1e-2)
+    return d, tol
+
+
+def run_case(M, N, K, seed, out_n=1, rule=0, n_out_ch=None, check_rows=None):
+    m = sdq()
+    cfg = m.Config(out_n, m.GRAN_PAIR, 64, rule)
+    W = sdq_synth.make_weight(N, K, seed)
+    X = sdq_synth.make_act(M, K, seed, n_outlier_channels=n_out_ch)
+    p = m.sdq_decompose(W.cuda(), cfg)
+    xq = m.sdq_quantize_act(X.cuda(), cfg)
+    y32 = m.sdq_linear(xq, p, f32=True)
+    y16 = m.sdq_linear(xq, p)
+    assert m.device_status() == 0
+    op = so.decompose(sdq_synth.bf16_bits(W), ocfg(out_n, rule))
+    oq = so.quantize_act(sdq_synth.bf16_bits(X), ocfg(out_n, rule))
+    pe = {k: v.cpu().numpy() for k, v in m.packed_export(p).items()}
+    ae = {k: v.cpu().numpy() for k, v in m.act_export(xq).items()}
+    for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp"):
+        assert np.array_equal(pe[name], getattr(op, name)), name
+    for name in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp"):
+        assert np.array_equal(ae[name], getattr(oq, name)), name
+    if check_rows is None:
+        yref = so.linear(oq, op)
+        yg = y32.cpu().numpy()
+        y16g = y16.float().cpu().numpy()
+    else:
+        n0, n1 = check_rows
+        yref = so.linear(oq, op, n0, n1)
+        yg = y32[:, n0:n1].cpu().numpy()
+        y16g = y16[:, n0:n1].float().cpu().numpy()
+    d, tol = y_close(yg, yref)
+    assert (d <= tol).all(), (d.max(), (d / tol).max())
+    # bf16 output is the round-to-nearest-even of the fp32 accumulator
+    assert np.array_equal(y16g, torch.from_numpy(yg).to(torch.bfloat16).float().numpy())
+    return float((d / tol).max())
+
+
+def test_tiny_config_seed0():
+    """C1: X 8x256 with 2 of 256 outlier channels x30, W 256x256"""
+    run_case(8, 256, 256, 0, n_out_ch=2)
+
+
+@pytest.mark.parametrize("out_n", [0, 1, 2])
+@pytest.mark.parametrize("rule", [0, 1])
+def test_patterns_and_scale_rules(out_n, rule):
+    run_case(40, 256, 512, 3 + out_n, out_n=out_n, rule=rule)
+
+
+@pytest.mark.parametrize("M", [1, 3, 16, 17, 33, 65, 128, 129, 300])
+def test_ragged_token_counts(M):
+    run_case(M, 128, 768, 10 + M)
+
+
+def test_several_tiles_long_k():
+    run_case(200, 384, 2816, 21)   # K = 11 x 256: more stages than the pipeline is deep
+
+
+def test_one_hot_readback_through_the_tensor_core():
+    """X = identity rows (1.0 is exact in both activation formats): Y^T must equal W_in + W_out exactly"""
+    m = sdq()
+    cfg = m.Config()
+    N, K = 128, 512
+    W = sdq_synth.make_weight(N, K, 5)
+    p = m.sdq_decompose(W.cuda(), cfg)
+    X = torch.eye(K, dtype=torch.bfloat16)
+    xq = m.sdq_quantize_act(X.cuda(), cfg)
+    y = m.sdq_linear(xq, p, f32=True).cpu().numpy().astype(np.float64)
+    W_in, W_out = so.dequant_weights(so.decompose(sdq_synth.bf16_bits(W), ocfg()))
+    assert np.array_equal(y, (W_in + W_out).T)
+
+
+def test_hardware_converters_match_oracle_exhaustively():
+    """all 65536 bf16 patterns through the activation quantizer (finite ones), several magnitudes"""
+    m = sdq()
+    bits = np.arange(65536, dtype=np.uint16)
+    finite = (bits & 0x7F80) != 0x7F80
+    vals = bits[finite]
+    K = 256
+    pad = (-len(vals)) % K
+    vals = np.concatenate([vals, np.zeros(pad, np.uint16)])
+    rng = np.random.default_rng(0)
+    rng.shuffle(vals)
+    Xb = vals.reshape(-1, K)
+    X = sdq_synth.bits_to_bf16(Xb)
+    for rule in (0, 1):
+        cfg = m.Config(1, m.GRAN_PAIR, 64, rule)
+        ae = {k: v.cpu().numpy() for k, v in m.act_export(m.sdq_quantize_act(X.cuda(), cfg)).items()}
+        oq = so.quantize_act(Xb, ocfg(1, rule))
+        for name in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp"):
+            assert np.array_equal(ae[name], getattr(oq, name)), name
+    # and sorted by magnitude so that blocks hold similar exponents (exercises every rounding boundary)
+    order = np.argsort(vals & 0x7FFF, kind="stable")
+    Xb2 = vals[order].reshape(-1, K)
+    ae = {k: v.cpu().numpy() for k, v in m.act_export(m.sdq_quantize_act(sdq_synth.bits_to_bf16(Xb2).cuda(), m.Config())).items()}
+    oq = so.quantize_act(Xb2, ocfg())
+    for name in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp"):
+        assert np.array_equal(ae[name], getattr(oq, name)), name
+
+
+def test_packer_ties_zeros_and_negative_zero():
+    m = sdq()
+    rng = np.random.default_rng(1)
+    vals = np.array([0.0, -0.0, 0.5, -0.5, 1.0, 1.0, -2.0, 2.0, 3.0, 1e-30, -1e-30, 448.0, 6.0, -6.0, 7.0, 0.75])
+    W = torch.from_numpy(rng.choice(vals, size=(128, 512))).to(torch.bfloat16)
+    W[5] = 0
+    for out_n in (0, 1, 2):
+        for rule in (0, 1):
+            cfg = m.Config(out_n, m.GRAN_PAIR, 64, rule)
+            pe = {k: v.cpu().numpy() for k, v in m.packed_export(m.sdq_decompose(W.cuda(), cfg)).items()}
+            op = so.decompose(sdq_synth.bf16_bits(W), ocfg(out_n, rule))
+            for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp"):
+                assert np.array_equal(pe[name], getattr(op, name)), (name, out_n, rule)
+
+
+def test_errors_are_status_codes():
+    m = sdq()
+    W = sdq_synth.make_weight(128, 256, 0).cuda()
+    with pytest.raises(m.SdqError) as e:
+        m.sdq_decompose(W[:, :128].contiguous())           # K not a multiple of 256
+    assert e.value.code == 2
+    with pytest.raises(m.SdqError) as e:
+        m.sdq_decompose(W, m.Config(1, m.GRAN_ELEM, 32, 0))  # decompose-only reading not built yet
+    assert e.value.code == 4
+    Wbad = W.clone()
+    Wbad[3, 7] = float("inf")
+    with pytest.raises(m.SdqError) as e:
+        m.sdq_decompose(Wbad)
+    assert e.value.code == 6
+    p = m.sdq_decompose(W)
+    xq = m.sdq_quantize_act(sdq_synth.make_act(4, 512, 0).cuda())
+    with pytest.raises(m.SdqError) as e:
+        m.sdq_linear(xq, p)                                  # K mismatch
+    assert e.value.code == 2
