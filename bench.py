@@ -1,0 +1,341 @@
+#!/usr/bin/env python
+"""Benchmark of the SDQ decomposed linear layer on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" is one pass of the hot path over one batch of synthetic input shaped like the MLP of a
+LLaMA-7B decoder layer at prefill: quantize X [2048, 4096] -> gate and up projections (4096 -> 11008,
+sharing the quantized X) -> quantize H [2048, 11008] -> down projection (11008 -> 4096).  Weights are
+decomposed and packed offline (untimed).  The headline value is dense-equivalent TFLOP/s of the whole
+step (2*M*N*K per projection).  A second, separately timed region measures the decode shape
+(M in {1, 16}, 4096 x 4096 attention projection, rotating over 32 distinct layers) in GB/s of
+algorithmic compressed-weight bytes and is reported under "decode".
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import sdq_synth  # noqa: E402
+
+METRIC = "sdq_linear_dense_equiv_tflops_prefill"
+UNIT = "TFLOP/s"
+WORKLOAD = "llama7b_mlp_prefill_M2048 (gate,up 4096->11008; down 11008->4096; 1:8 FP8 outlier + pair-wise 4:8 MXFP4 inlier, block 64)"
+M_PREFILL, D_MODEL, D_FF = 2048, 4096, 11008
+# Mixed-instruction tensor roofline: per dense-equivalent flop the layer issues one sparse-FP4 flop
+# (nominally 8x the bf16 rate) and one sparse-FP8 flop (4x): peak = bf16_peak / (1/8 + 1/4).
+MIXED_PEAK_OVER_BF16 = 1.0 / (1.0 / 8.0 + 1.0 / 4.0)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm=d["hbm_gbs"], bf16=d["bf16_tflops"], bf16_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]),
+                    source="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """samples nvidia-smi clocks / throttle reasons while the timed region runs"""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                                       "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1])); mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        # median over the upper half of the samples = clocks under load (the sampler also sees idle edges)
+        hi = sorted(sm)[len(sm) // 2:]
+        return {"sm_mhz": statistics.median(hi), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------------------------- oracle arm
+class OracleSample:
+    """The CPU oracle (as it stands) on a bounded sample of the prefill workload: `rows_x` tokens through
+    the first `n_rows_w` output features of the gate projection; activation quantization is inside the
+    timed region, the weight decomposition is offline (untimed), exactly as on the GPU arm."""
+
+    def __init__(self, rows_x: int, n_rows_w: int = D_FF, seed: int = 3000):
+        from oracle import sdq_oracle as so
+        self.so = so
+        self.cfg = so.Config(1, so.GRAN_PAIR, 64, so.SCALE_OCP_FLOOR)
+        W = sdq_synth.bf16_bits(sdq_synth.make_weight(n_rows_w, D_MODEL, seed + 1))
+        self.X = sdq_synth.bf16_bits(sdq_synth.make_act(rows_x, D_MODEL, seed + 4))
+        self.p = so.decompose(W, self.cfg)
+        self.threads = os.cpu_count() or 1
+        self.flops = 2.0 * rows_x * n_rows_w * D_MODEL
+        self.desc = "%d of 2048 tokens x %d of 11008 gate rows x K=4096 (quantize_act + product, fp64 accumulate)" % (rows_x, n_rows_w)
+
+    def run(self):
+        t0 = time.perf_counter()
+        q = self.so.quantize_act(self.X, self.cfg)
+        self.so.linear(q, self.p, threads=self.threads)
+        dt = time.perf_counter() - t0
+        return self.flops / dt / 1e12, dt
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    # each step is a bounded sample; sized so that a 20+3 step run still ends within a few minutes
+    sample = OracleSample(rows_x=256)
+    vals, secs = [], []
+    for i in range(args.warmup + args.steps):
+        v, dt = sample.run()
+        if i >= args.warmup:
+            vals.append(v); secs.append(dt)
+    v = sum(vals) / len(vals)
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * sum(secs) / len(secs), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": sample.desc},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": sample.threads, "kind": "oracle", "sample": sample.desc},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------- CUDA arm
+def run_ours(args):
+    import paper_2406_13868_b200 as sdq
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    cfg = sdq.Config(1, sdq.GRAN_PAIR, 64, sdq.SCALE_OCP_FLOOR)
+    peaks = measured_peaks()
+
+    # ---- synthetic layer (seed = config index * 1000 + rank; weak scaling: every rank has its own batch)
+    seed = 3000 + rank
+    Wg = sdq_synth.make_weight(D_FF, D_MODEL, seed + 1, device=str(dev))
+    Wu = sdq_synth.make_weight(D_FF, D_MODEL, seed + 2, device=str(dev))
+    Wd = sdq_synth.make_weight(D_MODEL, D_FF, seed + 3, device=str(dev))
+    X = sdq_synth.make_act(M_PREFILL, D_MODEL, seed + 4, device=str(dev))
+    H = sdq_synth.make_act(M_PREFILL, D_FF, seed + 5, device=str(dev))
+    Pg, Pu, Pd = (sdq.sdq_decompose(w, cfg) for w in (Wg, Wu, Wd))
+    del Wg, Wu, Wd
+    bx = torch.empty(sdq.act_size(M_PREFILL, D_MODEL, cfg), dtype=torch.uint8, device=dev)
+    bh = torch.empty(sdq.act_size(M_PREFILL, D_FF, cfg), dtype=torch.uint8, device=dev)
+    Yg = torch.empty((M_PREFILL, D_FF), dtype=torch.bfloat16, device=dev)
+    Yu = torch.empty_like(Yg)
+    Yd = torch.empty((M_PREFILL, D_MODEL), dtype=torch.bfloat16, device=dev)
+    flops_step = 3 * 2.0 * M_PREFILL * D_MODEL * D_FF
+    launches_per_step = 5
+
+    ev = []   # (kind, start, end) per launch in the timed region
+
+    def step(record=False):
+        def timed(kind, fn):
+            if record:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); r = fn(); b.record(); ev.append((kind, a, b))
+                return r
+            return fn()
+        xq = timed("quant", lambda: sdq.sdq_quantize_act(X, cfg, bx))
+        timed("gemm", lambda: sdq.sdq_linear(xq, Pg, Yg))
+        timed("gemm", lambda: sdq.sdq_linear(xq, Pu, Yu))
+        hq = timed("quant", lambda: sdq.sdq_quantize_act(H, cfg, bh))
+        timed("gemm", lambda: sdq.sdq_linear(hq, Pd, Yd))
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    assert sdq.device_status() == 0, "device-side timeout flag set"
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.1)
+    barrier(); torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step(record=True)
+    e1.record()
+    torch.cuda.synchronize(); barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    assert sdq.device_status() == 0, "device-side timeout flag set"
+    t_ms = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+    ms_step = float(t_ms.item()) / args.steps
+    value = world * flops_step / (ms_step * 1e-3) / 1e12
+
+    gemm_ms = [a.elapsed_time(b) for k, a, b in ev if k == "gemm"]
+    quant_ms = [a.elapsed_time(b) for k, a, b in ev if k == "quant"]
+    gemm_tf = (flops_step * args.steps) / (sum(gemm_ms) * 1e-3) / 1e12
+    mixed_peak = peaks["bf16"] * MIXED_PEAK_OVER_BF16
+    roofline = {"kernel": "sdq_linear_kernel", "bound": "tensor", "achieved": gemm_tf, "peak": mixed_peak, "unit": "TFLOP/s",
+                "frac": gemm_tf / mixed_peak, "traffic": None,
+                "peak_basis": "%s bf16 burst %.1f TF/s x 8/3 (sparse FP4 at 8x + sparse FP8 at 4x per dense-equivalent flop)" % (peaks["source"], peaks["bf16"]),
+                "avg_launch_ms": sum(gemm_ms) / len(gemm_ms), "launches": len(gemm_ms),
+                "frac_of_sparse_fp4_peak": gemm_tf / (8 * peaks["bf16"])}
+    quant_bytes = (M_PREFILL * D_MODEL + M_PREFILL * D_FF) * (2 + 0.5 + 1.0 + 1.0 / 64)
+    quant = {"kernel": "quant_act_kernel", "bound": "hbm", "achieved": quant_bytes * args.steps / (sum(quant_ms) * 1e-3) / 1e9,
+             "peak": peaks["hbm"], "unit": "GB/s"}
+    quant["frac"] = quant["achieved"] / quant["peak"]
+
+    if rank != 0:
+        return
+    # ---- decode shape (C2): 4096x4096, M in {1,16}, rotating over 32 distinct packed layers (> L2)
+    decode = measure_decode(sdq, cfg, dev, peaks)
+    # ---- end to end through the public API with host buffers (pinned), copies inside the timed region
+    e2e = measure_e2e(sdq, cfg, dev, X, H, (Pg, Pu, Pd), (bx, bh), (Yg, Yu, Yd), flops_step, max(3, args.steps // 2))
+    sample = OracleSample(rows_x=1024)
+    v, dt = sample.run()
+    threads, desc = sample.threads, sample.desc
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp4+fp8 (E2M1/E4M3 products, fp32 accumulate)",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD, "tokens_per_gpu": M_PREFILL, "l2": "packed weights + activations of one step exceed L2 (150 MB > 126 MB)",
+                       "parallelism": "dp%d (independent batches, no collective)" % world},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline, "quantizer_roofline": quant, "decode": decode,
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc, "seconds": dt}}
+    print(json.dumps(line))
+
+
+def measure_decode(sdq, cfg, dev, peaks, layers: int = 32, reps: int = 20):
+    N = K = 4096
+    packs = []
+    for i in range(layers):
+        W = sdq_synth.make_weight(N, K, 2000 + i, device=str(dev))
+        packs.append(sdq.sdq_decompose(W, cfg))
+        del W
+    algo = packs[0].algorithmic_bytes
+    out = {}
+    for M in (1, 16):
+        X = sdq_synth.make_act(M, K, 2100 + M, device=str(dev))
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+        xb = torch.empty(sdq.act_size(M, K, cfg), dtype=torch.uint8, device=dev)
+        xq = sdq.sdq_quantize_act(X, cfg, xb)
+        for p in packs:
+            sdq.sdq_linear(xq, p, Y)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            for p in packs:
+                sdq.sdq_linear(xq, p, Y)
+        b.record()
+        torch.cuda.synchronize()
+        us = a.elapsed_time(b) * 1e3 / (reps * layers)
+        gbs = algo / (us * 1e-6) / 1e9
+        out["M%d" % M] = {"us_per_layer": us, "weight_GBps_algorithmic": gbs, "frac_of_hbm_peak": gbs / peaks["hbm"]}
+    out["workload"] = "llama7b_attn_proj_decode 4096x4096, %d distinct layers in rotation (%.0f MB packed > L2), sdq_linear only" % (
+        layers, layers * packs[0].buf.numel() / 1e6)
+    out["algorithmic_bytes_per_layer"] = algo
+    out["stored_bytes_per_layer"] = int(packs[0].buf.numel())
+    out["hbm_peak_GBps"] = peaks["hbm"]
+    return out
+
+
+def measure_e2e(sdq, cfg, dev, X, H, packs, bufs, outs, flops_step, steps):
+    Xh, Hh = X.cpu().pin_memory(), H.cpu().pin_memory()
+    Yh = [torch.empty(o.shape, dtype=o.dtype).pin_memory() for o in outs]
+    Xd, Hd = torch.empty_like(X), torch.empty_like(H)
+
+    def step():
+        Xd.copy_(Xh, non_blocking=True)
+        Hd.copy_(Hh, non_blocking=True)
+        xq = sdq.sdq_quantize_act(Xd, cfg, bufs[0])
+        sdq.sdq_linear(xq, packs[0], outs[0])
+        sdq.sdq_linear(xq, packs[1], outs[1])
+        hq = sdq.sdq_quantize_act(Hd, cfg, bufs[1])
+        sdq.sdq_linear(hq, packs[2], outs[2])
+        for yh, yd in zip(Yh, outs):
+            yh.copy_(yd, non_blocking=True)
+    for _ in range(2):
+        step()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps):
+        step()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / steps
+    return {"value": flops_step / (ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms,
+            "h2d_bytes_per_step": int(Xh.numel() * 2 + Hh.numel() * 2), "d2h_bytes_per_step": int(sum(y.numel() * 2 for y in Yh))}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
