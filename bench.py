@@ -323,15 +323,43 @@ def measure_e2e(sdq, cfg, dev, X, H, packs, bufs, outs, flops_step, steps):
             "h2d_bytes_per_step": int(Xh.numel() * 2 + Hh.numel() * 2), "d2h_bytes_per_step": int(sum(y.numel() * 2 for y in Yh))}
 
 
+def run_case(args):
+    """Small single-kernel cases for profiler captures (few launches, a few hundred MB on the device)."""
+    import paper_2406_13868_b200 as sdq
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    cfg = sdq.Config(1, sdq.GRAN_PAIR, 64, sdq.SCALE_OCP_FLOOR)
+    if args.case == "gemm_prefill":
+        M, K, N = M_PREFILL, D_MODEL, D_FF
+    elif args.case == "gemm_decode":
+        M, K, N = 16, 4096, 4096
+    else:
+        M, K, N = M_PREFILL, D_FF, 128
+    W = sdq_synth.make_weight(N, K, 1, device=str(dev))
+    X = sdq_synth.make_act(M, K, 2, device=str(dev))
+    P = sdq.sdq_decompose(W, cfg)
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+    for _ in range(args.steps):
+        xq = sdq.sdq_quantize_act(X, cfg)
+        sdq.sdq_linear(xq, P, Y)
+    torch.cuda.synchronize()
+    assert sdq.device_status() == 0
+    print(json.dumps({"case": args.case, "M": M, "N": N, "K": K, "launches": args.steps}))
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--case", default=None, choices=["gemm_prefill", "gemm_decode", "quant"],
+                    help="run only a small single-kernel case (for profiler captures) and exit")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.impl == "reference":
+    if args.case:
+        run_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -17,22 +17,20 @@
 namespace sdq {
 
 constexpr int LIN_THREADS = 192;
-constexpr int NSTAGE = 5;
-constexpr int STAGE_BYTES = A_IN_BYTES + A_OUT_BYTES + E_OUT_BYTES + W2_BYTES + B4_BYTES + B8_BYTES + X2_BYTES;  // 41984
-constexpr int SM_W1 = 0;
-constexpr int SM_W2 = SM_W1 + A_IN_BYTES + A_OUT_BYTES + E_OUT_BYTES;  // 14336
-constexpr int SM_B4 = SM_W2 + W2_BYTES;                                // 16896
-constexpr int SM_B8 = SM_B4 + B4_BYTES;                                // 25088
-constexpr int SM_X2 = SM_B8 + B8_BYTES;                                // 41472
-constexpr int SM_SFOUT = NSTAGE * STAGE_BYTES;                         // two 512 B atoms
-constexpr int SM_BARS = SM_SFOUT + 2 * SF_ATOM_BYTES;
-constexpr int LIN_SMEM = SM_BARS + 256 + 1024;                         // + alignment slack
+constexpr int NSLOT = 5;
+constexpr int SLOT_BYTES = 45056;              // one ring slot holds either an inlier or an outlier stage
+constexpr int SL_A = 0;                        // WI record (A_in | E_in | SFA_in) or WO record (A_out | E_out)
+constexpr int SL_B = 10752;                    // B4 (256 K) or B8 (128 K) of up to 256 tokens: 32768 B
+constexpr int SL_SF = SL_B + 32768;            // inlier: SFB_in atoms (2 x 512); outlier stage 0: SFA_out | SFB_out x 2
+constexpr int SM_BARS = NSLOT * SLOT_BYTES;
+constexpr int LIN_SMEM = SM_BARS + 128 + 1024; // + barriers + alignment slack
 
 // TMEM columns
-constexpr uint32_t TM_D = 0;         // accumulator: up to 128 columns
-constexpr uint32_t TM_META = 256;    // 2 buffers x 16 columns: E_in 4 | SFA_in 4 | SFB_in 4 | E_out 4
-constexpr uint32_t TM_SFA_OUT = 384;
-constexpr uint32_t TM_SFB_OUT = 388;
+constexpr uint32_t TM_D = 0;          // accumulator: up to 256 columns (tokens)
+constexpr uint32_t TM_I = 256;        // 2 buffers x 16 columns: E_in 4 | SFA_in 4 | SFB_in 8
+constexpr uint32_t TM_EO = 288;       // 2 buffers x 4 columns: E_out
+constexpr uint32_t TM_SFA_OUT = 296;  // 4 columns
+constexpr uint32_t TM_SFB_OUT = 300;  // 8 columns
 
 struct LinearParams {
   const uint8_t* w;      // packed weights
@@ -41,7 +39,9 @@ struct LinearParams {
   ActOffsets aoff;
   int64_t M, N, K;
   int out_n;
-  int n_tile;            // tokens per CTA: 16..128, multiple of 16
+  int n_tile;            // tokens per tile: 16, 32, 64, 128 or 256
+  int n_mtiles;          // ceil(M / n_tile)
+  int total_tiles;       // (N / 128) * n_mtiles
   void* Y;
   int64_t ldy;
   uint32_t* flags;
@@ -55,24 +55,20 @@ sdq_linear_kernel(const LinearParams p)
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint8_t* sm = smem_raw + ((1024 - (ptx::smem_u32(smem_raw) & 1023)) & 1023);
   uint64_t* full = reinterpret_cast<uint64_t*>(sm + SM_BARS);
-  uint64_t* empty = full + NSTAGE;
-  uint64_t* sf_full = empty + NSTAGE;
-  uint64_t* acc_full = sf_full + 1;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
+  uint64_t* empty = full + NSLOT;
+  uint64_t* acc_full = empty + NSLOT;
+  uint64_t* acc_empty = acc_full + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
 
-  const int64_t rt = blockIdx.x, mtile = blockIdx.y;
   const int n_tile = p.n_tile;
-  const int T1 = (int)(p.K / K1), T2 = (int)(p.K / K2);
-  const int W1B = w1_bytes(p.out_n);
-  // token tile of this CTA inside the 128-token activation tiles
-  const int64_t m0 = mtile * n_tile;
-  const int64_t mt = m0 / TILE_TOK;
-  const uint32_t t0 = (uint32_t)(m0 % TILE_TOK);   // multiple of n_tile (n_tile divides 128 or is 128-aligned)
+  const int RT = (int)(p.N / TILE_ROWS);
+  const int T1 = p.out_n ? (int)(p.K / K1) : 0, T2 = (int)(p.K / K2);
+  const int n_atiles = (n_tile + TILE_TOK - 1) / TILE_TOK;     // 128-token activation tiles per token tile
 
   if (tid == 0) {
-    for (int s = 0; s < NSTAGE; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
-    ptx::mbar_init(sf_full, 1);
+    for (int s = 0; s < NSLOT; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
     ptx::mbar_init(acc_full, 1);
+    ptx::mbar_init(acc_empty, 4);
     ptx::fence_barrier_init();
   }
   if (warp == 1) ptx::tmem_alloc(tmem_slot, 512);
@@ -83,31 +79,47 @@ sdq_linear_kernel(const LinearParams p)
 
   if (warp == 0) {
     if (lane == 0) {
-      // ---------------- producer: one bulk copy per operand block per stage
-      const uint8_t* w1 = p.w + p.poff.w1 + (size_t)rt * T1 * W1B;
-      const uint8_t* w2 = p.w + p.poff.w2 + (size_t)rt * T2 * W2_BYTES;
-      const uint8_t* x1 = p.x + p.aoff.x1 + (size_t)mt * T1 * X1_BYTES;
-      const uint8_t* x2 = p.x + p.aoff.x2 + (size_t)mt * T2 * X2_BYTES;
-      const uint32_t b4_bytes = (uint32_t)n_tile * 64u, b8_bytes = (uint32_t)n_tile * 128u;
-      if (p.out_n) {
-        ptx::mbar_expect_tx(sf_full, 2 * SF_ATOM_BYTES);
-        ptx::bulk_g2s(sm + SM_SFOUT, p.w + p.poff.sfa_out + (size_t)rt * SF_ATOM_BYTES, SF_ATOM_BYTES, sf_full);
-        ptx::bulk_g2s(sm + SM_SFOUT + SF_ATOM_BYTES, p.x + p.aoff.sfb_out + (size_t)mt * SF_ATOM_BYTES, SF_ATOM_BYTES, sf_full);
-      }
+      // ---------------- producer: bulk copies, inlier stages of the tile first, then its outlier stages
       bool ok = true;
-      for (int it = 0; it < T1 && ok; ++it) {
-        const int s = it % NSTAGE;
-        if (it >= NSTAGE) ok = ptx::mbar_wait(&empty[s], ((it / NSTAGE) - 1) & 1);
-        if (!ok) break;
-        uint8_t* st = sm + (size_t)s * STAGE_BYTES;
-        const uint32_t tx = (uint32_t)W1B + W2_BYTES + b4_bytes + (p.out_n ? b8_bytes : 0u) + X2_BYTES;
-        ptx::mbar_expect_tx(&full[s], tx);
-        ptx::bulk_g2s(st + SM_W1, w1 + (size_t)it * W1B, (uint32_t)W1B, &full[s]);
-        ptx::bulk_g2s(st + SM_W2, w2 + (size_t)(it >> 1) * W2_BYTES, W2_BYTES, &full[s]);
-        ptx::bulk_g2s(st + SM_B4, x1 + (size_t)it * X1_BYTES + (size_t)(t0 >> 3) * 512, b4_bytes, &full[s]);
-        if (p.out_n)
-          ptx::bulk_g2s(st + SM_B8, x1 + (size_t)it * X1_BYTES + B4_BYTES + (size_t)(t0 >> 3) * 1024, b8_bytes, &full[s]);
-        ptx::bulk_g2s(st + SM_X2, x2 + (size_t)(it >> 1) * X2_BYTES, X2_BYTES, &full[s]);
+      uint32_t it = 0;
+      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+        const int rt = tile % RT, mtile = tile / RT;
+        const int64_t m0 = (int64_t)mtile * n_tile;
+        const int64_t mt = m0 / TILE_TOK;
+        const int have = (int)min((int64_t)n_atiles, p.aoff.MT - mt);     // activation tiles that exist
+        const uint32_t tok_bytes = (uint32_t)min(n_tile, TILE_TOK) * 128u;   // bytes per activation tile per stage
+        const uint8_t* wi = p.w + p.poff.wi + (size_t)rt * T2 * WI_BYTES;
+        const uint8_t* wo = p.w + p.poff.wo + (size_t)rt * T1 * WO_BYTES;
+        const uint8_t* xi = p.x + p.aoff.xi + (size_t)mt * T2 * XI_BYTES;
+        const uint8_t* xo = p.x + p.aoff.xo + (size_t)mt * T1 * XO_BYTES;
+        for (int k = 0; k < T2 + T1 && ok; ++k, ++it) {
+          const uint32_t s = it % NSLOT;
+          if (it >= NSLOT) ok = ptx::mbar_wait(&empty[s], ((it / NSLOT) - 1) & 1);
+          if (!ok) break;
+          uint8_t* st = sm + (size_t)s * SLOT_BYTES;
+          if (k < T2) {
+            ptx::mbar_expect_tx(&full[s], WI_BYTES + (uint32_t)have * (tok_bytes + SF_ATOM_BYTES));
+            ptx::bulk_g2s(st + SL_A, wi + (size_t)k * WI_BYTES, WI_BYTES, &full[s]);
+            for (int a = 0; a < have; ++a) {
+              const uint8_t* src = xi + ((size_t)a * T2 + k) * XI_BYTES;
+              ptx::bulk_g2s(st + SL_B + a * B4_BYTES, src, tok_bytes, &full[s]);
+              ptx::bulk_g2s(st + SL_SF + a * SF_ATOM_BYTES, src + B4_BYTES, SF_ATOM_BYTES, &full[s]);
+            }
+          } else {
+            const int k1 = k - T2;
+            const uint32_t sf_bytes = (k1 == 0) ? (uint32_t)(1 + have) * SF_ATOM_BYTES : 0u;
+            ptx::mbar_expect_tx(&full[s], WO_BYTES + (uint32_t)have * tok_bytes + sf_bytes);
+            ptx::bulk_g2s(st + SL_A, wo + (size_t)k1 * WO_BYTES, WO_BYTES, &full[s]);
+            for (int a = 0; a < have; ++a)
+              ptx::bulk_g2s(st + SL_B + a * B8_BYTES, xo + ((size_t)a * T1 + k1) * XO_BYTES, tok_bytes, &full[s]);
+            if (k1 == 0) {
+              ptx::bulk_g2s(st + SL_SF, p.w + p.poff.sfa_out + (size_t)rt * SF_ATOM_BYTES, SF_ATOM_BYTES, &full[s]);
+              for (int a = 0; a < have; ++a)
+                ptx::bulk_g2s(st + SL_SF + (1 + a) * SF_ATOM_BYTES, p.x + p.aoff.sfb_out + (size_t)(mt + a) * SF_ATOM_BYTES,
+                              SF_ATOM_BYTES, &full[s]);
+            }
+          }
+        }
       }
       if (!ok) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
     }
@@ -116,68 +128,107 @@ sdq_linear_kernel(const LinearParams p)
       // ---------------- MMA issuer
       bool ok = true;
       const uint32_t smb = ptx::smem_u32(sm);
-      if (p.out_n) {
-        ok = ptx::mbar_wait(sf_full, 0);
-        ptx::tc_fence_after();
-        ptx::tc_cp_32x128b_warpx4(tmem + TM_SFA_OUT, ptx::smem_desc(smb + SM_SFOUT, 0, 128));
-        ptx::tc_cp_32x128b_warpx4(tmem + TM_SFB_OUT, ptx::smem_desc(smb + SM_SFOUT + SF_ATOM_BYTES, 0, 128));
-      }
-      // SFB atoms hold 128 tokens as (t%32)*16 + (t/32)*4: a token tile starting at t0 reads column t0/32
-      // and, inside the column, rows from t0%32 -- only tiles of 32+ tokens or t0%32==0 keep that simple,
-      // so small tiles (n_tile < 32) always start at t0 % 32 == 0 (enforced by the host).
-      const uint32_t sfb_col = t0 >> 5;
-      for (int it = 0; it < T1 && ok; ++it) {
-        const int s = it % NSTAGE;
-        ok = ptx::mbar_wait(&full[s], (it / NSTAGE) & 1);
-        if (!ok) break;
-        ptx::tc_fence_after();
-        const uint32_t st = smb + (uint32_t)s * STAGE_BYTES;
-        const uint32_t meta = tmem + TM_META + 16u * (uint32_t)(it & 1);
-        const uint32_t half = (uint32_t)(it & 1);
-        ptx::tc_cp_128x128b(meta + 0, ptx::smem_desc(st + SM_W2, 0, 128));
-        ptx::tc_cp_32x128b_warpx4(meta + 4, ptx::smem_desc(st + SM_W2 + E_IN_BYTES, 0, 128));
-        ptx::tc_cp_32x128b_warpx4(meta + 8, ptx::smem_desc(st + SM_X2, 0, 128));
-        if (p.out_n) ptx::tc_cp_128x128b(meta + 12, ptx::smem_desc(st + SM_W1 + A_IN_BYTES + A_OUT_BYTES, 0, 128));
-        // inliers: 128 logical K, scales 2*half and 2*half+1 of the 256-K atoms
-        ptx::mma_sp_mxf4(tmem + TM_D, ptx::smem_desc(st + SM_W1, 2048, 128), ptx::smem_desc(st + SM_B4, 128, 512),
-                         ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, true, 2 * half, 2 * half), meta + 0 + 2 * half,
-                         meta + 4, meta + 8 + sfb_col, it > 0 ? 1u : 0u);
-        if (p.out_n) {
-#pragma unroll
-          for (uint32_t j = 0; j < 2; ++j)
-            ptx::mma_sp_mxf8(tmem + TM_D, ptx::smem_desc(st + SM_W1 + A_IN_BYTES + j * 4096, 2048, 128),
-                             ptx::smem_desc(st + SM_B8 + j * 512, 128, 1024),
-                             ptx::idesc_block_scaled(128, (uint32_t)n_tile, 0, true, 0, 0), meta + 12 + 2 * j, tmem + TM_SFA_OUT,
-                             tmem + TM_SFB_OUT + sfb_col, 1u);
+      uint32_t it = 0, tcount = 0;
+      const uint32_t id4[2] = {ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, true, 0, 0),
+                               ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, true, 2, 2)};
+      const uint32_t id8 = ptx::idesc_block_scaled(128, (uint32_t)n_tile, 0, true, 0, 0);
+      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
+        if (tcount > 0) {   // the epilogue must have drained the accumulator of the previous tile
+          ok = ptx::mbar_wait(acc_empty, (tcount - 1) & 1);
+          if (!ok) break;
+          ptx::tc_fence_after();
         }
-        ptx::tc_commit(&empty[s]);
+        for (int k = 0; k < T2 + T1 && ok; ++k, ++it) {
+          const uint32_t s = it % NSLOT;
+          ok = ptx::mbar_wait(&full[s], (it / NSLOT) & 1);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          const uint32_t st = smb + s * SLOT_BYTES;
+          if (k < T2) {
+            // inlier stage: 256 logical K = 2 sparse MXFP4 MMAs; metadata and scale atoms go to TMEM first
+            const uint32_t mb = tmem + TM_I + 16u * (uint32_t)(k & 1);
+            ptx::tc_cp_128x128b(mb + 0, ptx::smem_desc(st + SL_A + A_IN_BYTES, 0, 128));
+            ptx::tc_cp_32x128b_warpx4(mb + 4, ptx::smem_desc(st + SL_A + A_IN_BYTES + E_IN_BYTES, 0, 128));
+            ptx::tc_cp_32x128b_warpx4(mb + 8, ptx::smem_desc(st + SL_SF, 0, 128));
+            if (n_atiles > 1) ptx::tc_cp_32x128b_warpx4(mb + 12, ptx::smem_desc(st + SL_SF + SF_ATOM_BYTES, 0, 128));
+#pragma unroll
+            for (uint32_t j = 0; j < 2; ++j)
+              ptx::mma_sp_mxf4(tmem + TM_D, ptx::smem_desc(st + SL_A + j * 4096, 128, 256),
+                               ptx::smem_desc(st + SL_B + j * 512, 128, 1024), id4[j], mb + 2 * j, mb + 4, mb + 8,
+                               (k > 0 || j > 0) ? 1u : 0u);
+          } else {
+            // outlier stage: 128 logical K = 2 sparse FP8 MMAs; the row / token scales (E8M0) arrive with stage 0
+            const int k1 = k - T2;
+            const uint32_t eb = tmem + TM_EO + 4u * (uint32_t)(k1 & 1);
+            ptx::tc_cp_128x128b(eb, ptx::smem_desc(st + SL_A + A_OUT_BYTES, 0, 128));
+            if (k1 == 0) {
+              ptx::tc_cp_32x128b_warpx4(tmem + TM_SFA_OUT, ptx::smem_desc(st + SL_SF, 0, 128));
+              ptx::tc_cp_32x128b_warpx4(tmem + TM_SFB_OUT, ptx::smem_desc(st + SL_SF + SF_ATOM_BYTES, 0, 128));
+              if (n_atiles > 1)
+                ptx::tc_cp_32x128b_warpx4(tmem + TM_SFB_OUT + 4, ptx::smem_desc(st + SL_SF + 2 * SF_ATOM_BYTES, 0, 128));
+            }
+#pragma unroll
+            for (uint32_t j = 0; j < 2; ++j)
+              ptx::mma_sp_mxf8(tmem + TM_D, ptx::smem_desc(st + SL_A + j * 4096, 128, 256),
+                               ptx::smem_desc(st + SL_B + j * 512, 128, 1024), id8, eb + 2 * j, tmem + TM_SFA_OUT,
+                               tmem + TM_SFB_OUT, 1u);
+          }
+          ptx::tc_commit(&empty[s]);
+        }
+        ptx::tc_commit(acc_full);
       }
-      ptx::tc_commit(acc_full);
       if (!ok) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
     }
   } else {
     // ---------------- epilogue: warp w owns TMEM lanes 32*(w%4) .. +31 (weight rows), columns = tokens
-    const bool ok = ptx::mbar_wait(acc_full, 0);
-    ptx::tc_fence_after();
-    if (!ok) {
-      if (lane == 0) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
-    } else {
-      const uint32_t q = warp & 3;
-      const int64_t n = rt * TILE_ROWS + q * 32 + lane;
-      for (int c0 = 0; c0 < n_tile; c0 += 16) {
-        uint32_t v[16];
-        ptx::tmem_ld_32x32b_x16(tmem + ((q * 32u) << 16) + TM_D + (uint32_t)c0, v);
-        ptx::tmem_ld_wait();
+    const uint32_t q = warp & 3;
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
+      const int rt = tile % RT, mtile = tile / RT;
+      const int64_t m0 = (int64_t)mtile * n_tile;
+      const int n_valid = (int)min((int64_t)n_tile, p.M - m0);
+      ok = ptx::mbar_wait(acc_full, tcount & 1);
+      ptx::tc_fence_after();
+      if (!ok) break;
+      const int64_t n = (int64_t)rt * TILE_ROWS + q * 32 + lane;
+      for (int c0 = 0; c0 < n_tile; c0 += 32) {
+        uint32_t v[32];
+        if (c0 < n_valid) {
+          ptx::tmem_ld_32x32b_x32(tmem + ((q * 32u) << 16) + TM_D + (uint32_t)c0, v);
+          ptx::tmem_ld_wait();
+        }
+        if (c0 + 32 >= n_tile) {      // accumulator fully read: hand TMEM back before the stores
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(acc_empty);
+        }
+        if (c0 >= n_valid) continue;
+        if (F32_OUT) {
+          float* Y = reinterpret_cast<float*>(p.Y);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int64_t m = m0 + c0 + j;
-          if (m < p.M) {
-            if (F32_OUT) reinterpret_cast<float*>(p.Y)[m * p.ldy + n] = __uint_as_float(v[j]);
-            else reinterpret_cast<__nv_bfloat16*>(p.Y)[m * p.ldy + n] = __float2bfloat16_rn(__uint_as_float(v[j]));
+          for (int j = 0; j < 32; ++j)
+            if (c0 + j < n_valid) Y[(m0 + c0 + j) * p.ldy + n] = __uint_as_float(v[j]);
+        } else {
+          // pair lanes so that each lane stores two adjacent output features (4 bytes) of one token
+          __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(p.Y);
+          const bool odd = lane & 1;
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            const uint32_t send = odd ? v[j] : v[j + 1];
+            const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
+            const float lo = __uint_as_float(odd ? recv : v[j]);        // feature n (even lane) / n-1 (odd lane)
+            const float hi = __uint_as_float(odd ? v[j + 1] : recv);
+            const int tok = c0 + j + (odd ? 1 : 0);
+            if (tok < n_valid) {
+              const __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
+              *reinterpret_cast<__nv_bfloat162*>(Y + (m0 + tok) * p.ldy + (n & ~(int64_t)1)) = pk;
+            }
           }
         }
       }
     }
+    if (!ok && lane == 0) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
   }
   ptx::tc_fence_before();
   __syncthreads();
@@ -210,11 +261,18 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   p.M = Xq->M; p.N = P->N; p.K = P->K;
   p.out_n = P->cfg.out_n;
   const int64_t M = Xq->M;
-  p.n_tile = M >= 128 ? 128 : (M > 64 ? 128 : (M > 32 ? 64 : (M > 16 ? 32 : 16)));
+  p.n_tile = M > 128 ? 256 : (M > 64 ? 128 : (M > 32 ? 64 : (M > 16 ? 32 : 16)));
+  p.n_mtiles = (int)((M + p.n_tile - 1) / p.n_tile);
+  p.total_tiles = (int)(P->N / TILE_ROWS) * p.n_mtiles;
   p.Y = Y; p.ldy = ldy;
   p.flags = device_flags();
   if (!p.flags) return SDQ_ERR_CUDA;
-  dim3 grid((unsigned)(P->N / TILE_ROWS), (unsigned)((M + p.n_tile - 1) / p.n_tile));
+  static int sm_count = 0;
+  if (!sm_count) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SDQ_ERR_CUDA;
+  }
+  dim3 grid((unsigned)(p.total_tiles < sm_count ? p.total_tiles : sm_count));
   if (f32) sdq_linear_kernel<true><<<grid, LIN_THREADS, LIN_SMEM, (cudaStream_t)stream>>>(p);
   else sdq_linear_kernel<false><<<grid, LIN_THREADS, LIN_SMEM, (cudaStream_t)stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;

@@ -92,9 +92,8 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
   const int64_t rt = n / TILE_ROWS;
   const uint32_t r = (uint32_t)(n % TILE_ROWS);
   const int T1 = (int)(K / K1), T2 = (int)(K / K2);
-  const int W1B = w1_bytes(out_n);
-  uint8_t* w1_base = blob + off.w1 + (size_t)rt * T1 * W1B;
-  uint8_t* w2_base = blob + off.w2 + (size_t)rt * T2 * W2_BYTES;
+  uint8_t* wi_base = blob + off.wi + (size_t)rt * T2 * WI_BYTES;
+  uint8_t* wo_base = blob + off.wo + (size_t)rt * T1 * WO_BYTES;
 
   if (tid == 0) {
     reinterpret_cast<int32_t*>(blob + off.osexp)[n] = e;
@@ -152,14 +151,15 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     const uint32_t codes = e2m1x2(v[0], v[1]) | (e2m1x2(v[2], v[3]) << 8);
 
     const int k1 = g >> 4, k2 = g >> 5;
-    uint8_t* w1 = w1_base + (size_t)k1 * W1B;
-    uint8_t* w2 = w2_base + (size_t)k2 * W2_BYTES;
-    *reinterpret_cast<uint16_t*>(w1 + a_off(r, (uint32_t)(g & 15) * 2)) = (uint16_t)codes;
+    uint8_t* wi = wi_base + (size_t)k2 * WI_BYTES;
+    uint8_t* wo = wo_base + (size_t)k1 * WO_BYTES;
+    // 32 S-Vectors per 256-K stage, 2 code bytes each: bytes 0..31 = K-block 0, 32..63 = K-block 1
+    *reinterpret_cast<uint16_t*>(wi + a_off(r, (uint32_t)(g & 31) * 2)) = (uint16_t)codes;
     // metadata nibble j0 | j1<<2; two S-Vectors share a byte (even one in the low nibble)
     uint32_t nib = (uint32_t)(j0 | (j1 << 2));
     const uint32_t nib_hi = __shfl_down_sync(0xffffffffu, nib, 1);
-    if ((g & 1) == 0) w2[r * 16 + ((g & 31) >> 1)] = (uint8_t)(nib | (nib_hi << 4));
-    if ((g & 7) == 0) w2[E_IN_BYTES + sf_off(r, (uint32_t)((g >> 3) & 3))] = (uint8_t)c;
+    if ((g & 1) == 0) wi[A_IN_BYTES + r * 16 + ((g & 31) >> 1)] = (uint8_t)(nib | (nib_hi << 4));
+    if ((g & 7) == 0) wi[A_IN_BYTES + E_IN_BYTES + sf_off(r, (uint32_t)((g >> 3) & 3))] = (uint8_t)c;
 
     if (out_n > 0) {
       // Stage 3, outliers: E4M3 codes of w / 2^e; compact arrays plus the 2:4 embedding the sparse
@@ -187,8 +187,9 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
         stored |= (s0 | (s1 << 8)) << (16 * h);
         meta |= (uint32_t)(i0 | (i1 << 2)) << (4 * h);
       }
-      *reinterpret_cast<uint32_t*>(w1 + A_IN_BYTES + a_off(r, (uint32_t)(g & 15) * 4)) = stored;
-      w1[A_IN_BYTES + A_OUT_BYTES + r * 16 + (g & 15)] = (uint8_t)meta;
+      // 16 S-Vectors per 128-K stage, 4 stored bytes each: bytes 0..31 = K-block 0 (64 K), 32..63 = K-block 1
+      *reinterpret_cast<uint32_t*>(wo + a_off(r, (uint32_t)(g & 15) * 4)) = stored;
+      wo[A_OUT_BYTES + r * 16 + (g & 15)] = (uint8_t)meta;
     }
   }
 }
@@ -201,18 +202,16 @@ export_packed_kernel(const uint8_t* __restrict__ blob, int64_t N, int64_t K, sdq
   const int G = (int)(K / 8), out_n = cfg.out_n;
   const int64_t rt = n / TILE_ROWS;
   const uint32_t r = (uint32_t)(n % TILE_ROWS);
-  const int T1 = (int)(K / K1), T2 = (int)(K / K2), W1B = w1_bytes(out_n);
-  const uint8_t* w1_base = blob + off.w1 + (size_t)rt * T1 * W1B;
-  const uint8_t* w2_base = blob + off.w2 + (size_t)rt * T2 * W2_BYTES;
+  const int T2 = (int)(K / K2);
+  const uint8_t* wi_base = blob + off.wi + (size_t)rt * T2 * WI_BYTES;
   for (int g = threadIdx.x; g < G; g += 128) {
-    const uint8_t* w1 = w1_base + (size_t)(g >> 4) * W1B;
-    const uint8_t* w2 = w2_base + (size_t)(g >> 5) * W2_BYTES;
-    const uint32_t codes = *reinterpret_cast<const uint16_t*>(w1 + a_off(r, (uint32_t)(g & 15) * 2));
+    const uint8_t* wi = wi_base + (size_t)(g >> 5) * WI_BYTES;
+    const uint32_t codes = *reinterpret_cast<const uint16_t*>(wi + a_off(r, (uint32_t)(g & 31) * 2));
     uint8_t* ic = out.in_code + (size_t)n * (K / 2) + 4 * g;
     ic[0] = codes & 15; ic[1] = (codes >> 4) & 15; ic[2] = (codes >> 8) & 15; ic[3] = (codes >> 12) & 15;
-    const uint32_t mb = w2[r * 16 + ((g & 31) >> 1)];
+    const uint32_t mb = wi[A_IN_BYTES + r * 16 + ((g & 31) >> 1)];
     out.in_meta[(size_t)n * G + g] = (uint8_t)((g & 1) ? (mb >> 4) : (mb & 15));
-    if ((g & 7) == 0) out.in_scale[(size_t)n * (K / 64) + (g >> 3)] = w2[E_IN_BYTES + sf_off(r, (uint32_t)((g >> 3) & 3))];
+    if ((g & 7) == 0) out.in_scale[(size_t)n * (K / 64) + (g >> 3)] = wi[A_IN_BYTES + E_IN_BYTES + sf_off(r, (uint32_t)((g >> 3) & 3))];
     for (int t = 0; t < out_n; ++t) {
       out.out_code[((size_t)n * G + g) * out_n + t] = blob[off.ocode + ((size_t)n * G + g) * out_n + t];
       out.out_idx[((size_t)n * G + g) * out_n + t] = blob[off.oidx + ((size_t)n * G + g) * out_n + t];
@@ -269,7 +268,7 @@ extern "C" sdq_status_t sdq_decompose(const void* W, int64_t N, int64_t K, int64
   out->K = K;
   out->cfg = *cfg;
   for (int i = 0; i < 8; ++i) out->off[i] = 0;
-  out->off[0] = off.w1; out->off[1] = off.w2; out->off[2] = off.sfa_out;
+  out->off[0] = off.wi; out->off[1] = off.wo; out->off[2] = off.sfa_out;
   out->off[3] = off.ocode; out->off[4] = off.oidx; out->off[5] = off.osexp;
   return nonfinite ? SDQ_ERR_NONFINITE : SDQ_OK;
 }

@@ -59,8 +59,8 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
   const int64_t mt = m / TILE_TOK;
   const uint32_t t = (uint32_t)(m % TILE_TOK);
   const int T1 = (int)(K / K1), T2 = (int)(K / K2);
-  uint8_t* x1_base = buf + off.x1 + (size_t)mt * T1 * X1_BYTES;
-  uint8_t* x2_base = buf + off.x2 + (size_t)mt * T2 * X2_BYTES;
+  uint8_t* xi_base = buf + off.xi + (size_t)mt * T2 * XI_BYTES;
+  uint8_t* xo_base = buf + off.xo + (size_t)mt * T1 * XO_BYTES;
   if (tid == 0) {
     reinterpret_cast<int32_t*>(buf + off.sexp)[m] = e;
     *reinterpret_cast<uint32_t*>(buf + off.sfb_out + (size_t)mt * SF_ATOM_BYTES + sf_off(t, 0)) = (uint32_t)(e + 127) * 0x01010101u;
@@ -88,11 +88,11 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
       if (i < 2) q8lo |= p << (16 * i); else q8hi |= p << (16 * (i - 2));
     }
     const int k1 = (int)(k >> 7), k2 = (int)(k >> 8);
-    const uint32_t kk = (uint32_t)(k & 127);
-    uint8_t* x1 = x1_base + (size_t)k1 * X1_BYTES;
-    *reinterpret_cast<uint32_t*>(x1 + b4_off(t, kk >> 1)) = q4;
-    *reinterpret_cast<uint2*>(x1 + B4_BYTES + b8_off(t, kk)) = make_uint2(q8lo, q8hi);
-    if ((k & 63) == 0) x2_base[(size_t)k2 * X2_BYTES + sf_off(t, (uint32_t)((k >> 6) & 3))] = (uint8_t)c;
+    uint8_t* xi = xi_base + (size_t)k2 * XI_BYTES;
+    uint8_t* xo = xo_base + (size_t)k1 * XO_BYTES;
+    *reinterpret_cast<uint32_t*>(xi + b_off(t, (uint32_t)(k & 255) >> 1)) = q4;
+    *reinterpret_cast<uint2*>(xo + b_off(t, (uint32_t)(k & 127))) = make_uint2(q8lo, q8hi);
+    if ((k & 63) == 0) xi[B4_BYTES + sf_off(t, (uint32_t)((k >> 6) & 3))] = (uint8_t)c;
   }
 }
 
@@ -103,15 +103,15 @@ export_act_kernel(const uint8_t* __restrict__ buf, int64_t M, int64_t K, ActOffs
   const int64_t mt = m / TILE_TOK;
   const uint32_t t = (uint32_t)(m % TILE_TOK);
   const int T1 = (int)(K / K1), T2 = (int)(K / K2);
-  const uint8_t* x1_base = buf + off.x1 + (size_t)mt * T1 * X1_BYTES;
-  const uint8_t* x2_base = buf + off.x2 + (size_t)mt * T2 * X2_BYTES;
+  const uint8_t* xi_base = buf + off.xi + (size_t)mt * T2 * XI_BYTES;
+  const uint8_t* xo_base = buf + off.xo + (size_t)mt * T1 * XO_BYTES;
   for (int64_t k = threadIdx.x; k < K; k += QA_THREADS) {
-    const uint8_t* x1 = x1_base + (size_t)(k >> 7) * X1_BYTES;
-    const uint32_t kk = (uint32_t)(k & 127);
-    const uint32_t b = x1[b4_off(t, kk >> 1)];
-    out.xq4_code[(size_t)m * K + k] = (uint8_t)((kk & 1) ? (b >> 4) : (b & 15));
-    out.xq8_code[(size_t)m * K + k] = x1[B4_BYTES + b8_off(t, kk)];
-    if ((k & 63) == 0) out.xq4_scale[(size_t)m * (K / 64) + (k >> 6)] = x2_base[(size_t)(k >> 8) * X2_BYTES + sf_off(t, (uint32_t)((k >> 6) & 3))];
+    const uint8_t* xi = xi_base + (size_t)(k >> 8) * XI_BYTES;
+    const uint8_t* xo = xo_base + (size_t)(k >> 7) * XO_BYTES;
+    const uint32_t b = xi[b_off(t, (uint32_t)(k & 255) >> 1)];
+    out.xq4_code[(size_t)m * K + k] = (uint8_t)((k & 1) ? (b >> 4) : (b & 15));
+    out.xq8_code[(size_t)m * K + k] = xo[b_off(t, (uint32_t)(k & 127))];
+    if ((k & 63) == 0) out.xq4_scale[(size_t)m * (K / 64) + (k >> 6)] = xi[B4_BYTES + sf_off(t, (uint32_t)((k >> 6) & 3))];
   }
   if (threadIdx.x == 0) out.xq8_sexp[m] = reinterpret_cast<const int32_t*>(buf + off.sexp)[m];
 }
@@ -151,7 +151,7 @@ extern "C" sdq_status_t sdq_quantize_act(const void* X, int64_t M, int64_t K, in
   out->K = K;
   out->cfg = *cfg;
   for (int i = 0; i < 6; ++i) out->off[i] = 0;
-  out->off[0] = off.x1; out->off[1] = off.x2; out->off[2] = off.sfb_out; out->off[3] = off.sexp;
+  out->off[0] = off.xi; out->off[1] = off.xo; out->off[2] = off.sfb_out; out->off[3] = off.sexp;
   return SDQ_OK;
 }
 
