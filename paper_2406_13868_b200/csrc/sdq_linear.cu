@@ -12,6 +12,7 @@
 
 #include "sdq_internal.h"
 #include "sdq_layout.h"
+#include "sdq_linear.h"
 #include "sdq_ptx.cuh"
 
 namespace sdq {
@@ -22,8 +23,9 @@ constexpr int SLOT_BYTES = 45056;              // one ring slot holds either an 
 constexpr int SL_A = 0;                        // WI record (A_in | E_in | SFA_in) or WO record (A_out | E_out)
 constexpr int SL_B = 10752;                    // B4 (256 K) or B8 (128 K) of up to 256 tokens: 32768 B
 constexpr int SL_SF = SL_B + 32768;            // inlier: SFB_in atoms (2 x 512); outlier stage 0: SFA_out | SFB_out x 2
-constexpr int SM_BARS = NSLOT * SLOT_BYTES;
-constexpr int LIN_SMEM = SM_BARS + 128 + 1024; // + barriers + alignment slack
+constexpr int SM_STG = NSLOT * SLOT_BYTES;      // epilogue transpose buffer: 16 tokens x 128 features bf16
+constexpr int SM_BARS = SM_STG + 4096;
+constexpr int LIN_SMEM = SM_BARS + 128 + 128;  // + barriers + alignment slack
 
 // TMEM columns
 constexpr uint32_t TM_D = 0;          // accumulator: up to 256 columns (tokens)
@@ -32,20 +34,7 @@ constexpr uint32_t TM_EO = 288;       // 2 buffers x 4 columns: E_out
 constexpr uint32_t TM_SFA_OUT = 296;  // 4 columns
 constexpr uint32_t TM_SFB_OUT = 300;  // 8 columns
 
-struct LinearParams {
-  const uint8_t* w;      // packed weights
-  const uint8_t* x;      // quantized activations
-  PackedOffsets poff;
-  ActOffsets aoff;
-  int64_t M, N, K;
-  int out_n;
-  int n_tile;            // tokens per tile: 16, 32, 64, 128 or 256
-  int n_mtiles;          // ceil(M / n_tile)
-  int total_tiles;       // (N / 128) * n_mtiles
-  void* Y;
-  int64_t ldy;
-  uint32_t* flags;
-};
+
 
 template <bool F32_OUT>
 __global__ void __launch_bounds__(LIN_THREADS, 1)
@@ -53,7 +42,7 @@ sdq_linear_kernel(const LinearParams p)
 {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  uint8_t* sm = smem_raw + ((1024 - (ptx::smem_u32(smem_raw) & 1023)) & 1023);
+  uint8_t* sm = smem_raw + ((128 - (ptx::smem_u32(smem_raw) & 127)) & 127);
   uint64_t* full = reinterpret_cast<uint64_t*>(sm + SM_BARS);
   uint64_t* empty = full + NSLOT;
   uint64_t* acc_full = empty + NSLOT;
@@ -78,8 +67,9 @@ sdq_linear_kernel(const LinearParams p)
   const uint32_t tmem = *tmem_slot;
 
   if (warp == 0) {
-    if (lane == 0) {
-      // ---------------- producer: bulk copies, inlier stages of the tile first, then its outlier stages
+    if (lane < NSLOT) {
+      // ---------------- producer: bulk copies, inlier stages of the tile first, then its outlier stages.
+      // Lane l owns ring slot l, so the barrier round trips of different slots overlap.
       bool ok = true;
       uint32_t it = 0;
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
@@ -94,6 +84,7 @@ sdq_linear_kernel(const LinearParams p)
         const uint8_t* xo = p.x + p.aoff.xo + (size_t)mt * T1 * XO_BYTES;
         for (int k = 0; k < T2 + T1 && ok; ++k, ++it) {
           const uint32_t s = it % NSLOT;
+          if (s != lane) continue;
           if (it >= NSLOT) ok = ptx::mbar_wait(&empty[s], ((it / NSLOT) - 1) & 1);
           if (!ok) break;
           uint8_t* st = sm + (size_t)s * SLOT_BYTES;
@@ -129,6 +120,7 @@ sdq_linear_kernel(const LinearParams p)
       bool ok = true;
       const uint32_t smb = ptx::smem_u32(sm);
       uint32_t it = 0, tcount = 0;
+      bool ready = false;
       const uint32_t id4[2] = {ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, true, 0, 0),
                                ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, true, 2, 2)};
       const uint32_t id8 = ptx::idesc_block_scaled(128, (uint32_t)n_tile, 0, true, 0, 0);
@@ -140,9 +132,11 @@ sdq_linear_kernel(const LinearParams p)
         }
         for (int k = 0; k < T2 + T1 && ok; ++k, ++it) {
           const uint32_t s = it % NSLOT;
-          ok = ptx::mbar_wait(&full[s], (it / NSLOT) & 1);
+          if (!ready) ok = ptx::mbar_wait(&full[s], (it / NSLOT) & 1);
           if (!ok) break;
           ptx::tc_fence_after();
+          // poll the next slot now: the answer is back by the time this stage's instructions are issued
+          ready = ptx::mbar_test(&full[(it + 1) % NSLOT], ((it + 1) / NSLOT) & 1);
           const uint32_t st = smb + s * SLOT_BYTES;
           if (k < T2) {
             // inlier stage: 256 logical K = 2 sparse MXFP4 MMAs; metadata and scale atoms go to TMEM first
@@ -191,40 +185,42 @@ sdq_linear_kernel(const LinearParams p)
       ok = ptx::mbar_wait(acc_full, tcount & 1);
       ptx::tc_fence_after();
       if (!ok) break;
-      const int64_t n = (int64_t)rt * TILE_ROWS + q * 32 + lane;
-      for (int c0 = 0; c0 < n_tile; c0 += 32) {
-        uint32_t v[32];
+      const int64_t n0 = (int64_t)rt * TILE_ROWS;
+      const uint32_t et = (warp - 2) * 32 + lane;     // 0..127 among the epilogue threads
+#pragma unroll 1
+      for (int c0 = 0; c0 < n_tile; c0 += 16) {
+        uint32_t v[16];
         if (c0 < n_valid) {
-          ptx::tmem_ld_32x32b_x32(tmem + ((q * 32u) << 16) + TM_D + (uint32_t)c0, v);
+          ptx::tmem_ld_32x32b_x16(tmem + ((q * 32u) << 16) + TM_D + (uint32_t)c0, v);
           ptx::tmem_ld_wait();
         }
-        if (c0 + 32 >= n_tile) {      // accumulator fully read: hand TMEM back before the stores
+        if (c0 + 16 >= n_tile) {      // accumulator fully read: hand TMEM back before the stores
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(acc_empty);
         }
-        if (c0 >= n_valid) continue;
+        if (c0 >= n_valid) continue;  // uniform over the four epilogue warps
         if (F32_OUT) {
           float* Y = reinterpret_cast<float*>(p.Y);
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (c0 + j < n_valid) Y[(m0 + c0 + j) * p.ldy + n] = __uint_as_float(v[j]);
+          for (int j = 0; j < 16; ++j)
+            if (c0 + j < n_valid) Y[(m0 + c0 + j) * p.ldy + n0 + q * 32 + lane] = __uint_as_float(v[j]);
         } else {
-          // pair lanes so that each lane stores two adjacent output features (4 bytes) of one token
-          __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(p.Y);
-          const bool odd = lane & 1;
+          // transpose through shared memory: [16 tokens][128 features] bf16, then 16-byte stores of full 256 B rows
+          __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(sm + SM_STG);
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            const uint32_t send = odd ? v[j] : v[j + 1];
-            const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
-            const float lo = __uint_as_float(odd ? recv : v[j]);        // feature n (even lane) / n-1 (odd lane)
-            const float hi = __uint_as_float(odd ? v[j + 1] : recv);
-            const int tok = c0 + j + (odd ? 1 : 0);
-            if (tok < n_valid) {
-              const __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
-              *reinterpret_cast<__nv_bfloat162*>(Y + (m0 + tok) * p.ldy + (n & ~(int64_t)1)) = pk;
+          for (int j = 0; j < 16; ++j) stg[j * 128 + q * 32 + lane] = __float2bfloat16_rn(__uint_as_float(v[j]));
+          ptx::named_bar_sync(1, 128);
+          __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(p.Y);
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            const uint32_t idx = i * 128 + et, tok = idx >> 4, seg = idx & 15;
+            if (c0 + (int)tok < n_valid) {
+              const uint4 w = *reinterpret_cast<const uint4*>(stg + tok * 128 + seg * 8);
+              *reinterpret_cast<uint4*>(Y + (m0 + c0 + tok) * p.ldy + n0 + seg * 8) = w;
             }
           }
+          ptx::named_bar_sync(1, 128);   // the buffer is rewritten by the next chunk
         }
       }
     }

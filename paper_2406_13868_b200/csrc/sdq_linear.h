@@ -1,0 +1,26 @@
+// Launch parameters of the fused GEMM kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sdq_internal.h"
+#include "sdq_layout.h"
+
+namespace sdq {
+
+struct LinearParams {
+  const uint8_t* w;      // packed weights
+  const uint8_t* x;      // quantized activations
+  PackedOffsets poff;
+  ActOffsets aoff;
+  int64_t M, N, K;
+  int out_n;
+  int n_tile;            // tokens per tile: 16, 32, 64, 128 or 256
+  int n_mtiles;          // ceil(M / n_tile)
+  int total_tiles;       // (N / 128) * n_mtiles
+  void* Y;
+  int64_t ldy;
+  uint32_t* flags;
+};
+
+}  // namespace sdq

@@ -79,6 +79,27 @@ def test_several_tiles_long_k():
     run_case(200, 384, 2816, 21)   # K = 11 x 256: more stages than the pipeline is deep
 
 
+@pytest.mark.parametrize("M,N,K,out_n", [(129, 256, 512, 1), (256, 256, 768, 1), (300, 512, 1024, 2), (520, 256, 2816, 1),
+                                         (384, 512, 512, 0), (1000, 1024, 256, 1)])
+def test_cta_pair_kernel_shapes(M, N, K, out_n):
+    """even number of 128-row tiles and more than 128 tokens: the 256x256 CTA-pair kernel, ragged token tails"""
+    run_case(M, N, K, 100 + M, out_n=out_n)
+
+
+def test_one_hot_readback_pair_kernel():
+    m = sdq()
+    cfg = m.Config()
+    N, K = 256, 512
+    W = sdq_synth.make_weight(N, K, 6)
+    p = m.sdq_decompose(W.cuda(), cfg)
+    X = torch.eye(K, dtype=torch.bfloat16)
+    xq = m.sdq_quantize_act(X.cuda(), cfg)
+    y = m.sdq_linear(xq, p, f32=True).cpu().numpy().astype(np.float64)
+    W_in, W_out = so.dequant_weights(so.decompose(sdq_synth.bf16_bits(W), ocfg()))
+    assert np.array_equal(y, (W_in + W_out).T)
+    assert m.device_status() == 0
+
+
 def test_one_hot_readback_through_the_tensor_core():
     """X = identity rows (1.0 is exact in both activation formats): Y^T must equal W_in + W_out exactly"""
     m = sdq()
