@@ -144,6 +144,22 @@ sdq_status_t sdq_linear(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y_bf16
 /* Same product, storing the fp32 accumulator itself (the value the bf16 output is rounded from). */
 sdq_status_t sdq_linear_f32(const sdq_act_t* Xq, const sdq_packed_t* P, float* Y_f32, int64_t ldy, void* stream);
 
+/* The same product with a caller-owned scratch buffer (device).  With few tokens (M <= 128) a weight row
+ * tile has too little work for one thread block per SM, so the K range of every row tile is split over
+ * several blocks; each writes an fp32 partial tile to the workspace and the last one to arrive adds them in
+ * split order, so the result does not depend on timing (O = O_o + O_i of Section 5.1 is unchanged; only the
+ * summation over K is regrouped, hence Y may differ from sdq_linear in the last fp32 bits).
+ *   sdq_workspace_size: bytes needed for (M, N, K) on the current device (0 when no split would be used).
+ *   sdq_workspace_init: zeroes a workspace once after allocation (asynchronous); calls leave it zeroed.
+ *   A workspace must not be shared by calls that can overlap on the GPU.  ws may be NULL (no split).
+ *   Errors as sdq_linear, plus BUFFER_TOO_SMALL. */
+sdq_status_t sdq_workspace_size(int64_t M, int64_t N, int64_t K, const sdq_config_t* cfg, size_t* bytes);
+sdq_status_t sdq_workspace_init(void* ws, size_t ws_bytes, void* stream);
+sdq_status_t sdq_linear_ws(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y_bf16, int64_t ldy, void* ws, size_t ws_bytes,
+                           void* stream);
+sdq_status_t sdq_linear_f32_ws(const sdq_act_t* Xq, const sdq_packed_t* P, float* Y_f32, int64_t ldy, void* ws, size_t ws_bytes,
+                               void* stream);
+
 /* Synchronises `stream` and returns the sticky device-side status (SDQ_OK or SDQ_ERR_TIMEOUT when a
  * bounded wait inside a kernel gave up), clearing it. */
 sdq_status_t sdq_device_status(void* stream);

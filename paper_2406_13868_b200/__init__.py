@@ -55,7 +55,8 @@ class _ActCanon(ctypes.Structure):
 
 
 EXPORTS = ["sdq_packed_size", "sdq_decompose", "sdq_packed_export", "sdq_act_size", "sdq_quantize_act", "sdq_act_export",
-           "sdq_linear", "sdq_linear_f32", "sdq_device_status", "sdq_status_string"]
+           "sdq_linear", "sdq_linear_f32", "sdq_workspace_size", "sdq_workspace_init", "sdq_linear_ws", "sdq_linear_f32_ws",
+           "sdq_device_status", "sdq_status_string"]
 
 _lib = None
 
@@ -77,6 +78,10 @@ def lib() -> ctypes.CDLL:
         L.sdq_act_export.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_ActCanon), vp]
         L.sdq_linear.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_Packed), vp, i64, vp]
         L.sdq_linear_f32.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_Packed), vp, i64, vp]
+        L.sdq_workspace_size.argtypes = [i64, i64, i64, ctypes.POINTER(Config), ctypes.POINTER(sz)]
+        L.sdq_workspace_init.argtypes = [vp, sz, vp]
+        L.sdq_linear_ws.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_Packed), vp, i64, vp, sz, vp]
+        L.sdq_linear_f32_ws.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_Packed), vp, i64, vp, sz, vp]
         L.sdq_device_status.argtypes = [vp]
         L.sdq_status_string.argtypes = [ctypes.c_int]
         L.sdq_status_string.restype = ctypes.c_char_p
@@ -161,14 +166,37 @@ def sdq_quantize_act(X: torch.Tensor, cfg: Config | None = None, buf: torch.Tens
     return QuantAct(buf, d, M, K, cfg)
 
 
-def sdq_linear(xq: QuantAct, p: PackedWeight, out: torch.Tensor | None = None, f32: bool = False) -> torch.Tensor:
-    """Y [M, N] = A_i W_i^T + A_o W_o^T (bf16, or the fp32 accumulator itself with f32=True)."""
+def workspace_size(M: int, N: int, K: int, cfg: Config) -> int:
+    b = ctypes.c_size_t()
+    _check(lib().sdq_workspace_size(M, N, K, ctypes.byref(cfg), ctypes.byref(b)), "sdq_workspace_size")
+    return b.value
+
+
+def make_workspace(M: int, N: int, K: int, cfg: Config, device) -> torch.Tensor | None:
+    """Allocates (with torch) and zeroes the split-K scratch buffer for a call shape; None if none is needed."""
+    n = workspace_size(M, N, K, cfg)
+    if n == 0:
+        return None
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    _check(lib().sdq_workspace_init(ws.data_ptr(), ws.numel(), _stream()), "sdq_workspace_init")
+    return ws
+
+
+def sdq_linear(xq: QuantAct, p: PackedWeight, out: torch.Tensor | None = None, f32: bool = False,
+               workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """Y [M, N] = A_i W_i^T + A_o W_o^T (bf16, or the fp32 accumulator itself with f32=True).
+    `workspace` (from make_workspace) enables the split-K path for few tokens."""
     dt = torch.float32 if f32 else torch.bfloat16
     if out is None:
         out = torch.empty((xq.M, p.N), dtype=dt, device=p.buf.device)
     assert out.dtype == dt and out.shape == (xq.M, p.N) and out.stride(1) == 1
-    fn = lib().sdq_linear_f32 if f32 else lib().sdq_linear
-    _check(fn(ctypes.byref(xq.desc), ctypes.byref(p.desc), out.data_ptr(), out.stride(0), _stream()), "sdq_linear")
+    if workspace is None:
+        fn = lib().sdq_linear_f32 if f32 else lib().sdq_linear
+        _check(fn(ctypes.byref(xq.desc), ctypes.byref(p.desc), out.data_ptr(), out.stride(0), _stream()), "sdq_linear")
+    else:
+        fn = lib().sdq_linear_f32_ws if f32 else lib().sdq_linear_ws
+        _check(fn(ctypes.byref(xq.desc), ctypes.byref(p.desc), out.data_ptr(), out.stride(0), workspace.data_ptr(),
+                  workspace.numel(), _stream()), "sdq_linear_ws")
     return out
 
 

@@ -40,6 +40,12 @@ __device__ __forceinline__ int fp8_scale_exp(float amax) {
   return min(max(e, -127), 127);
 }
 
+// 2^(127 - c) for an E8M0 code c <= 253 and 2^(-e) for an 8-bit scale exponent e in [-127, 120], built from
+// the exponent field: multiplying by them is exact (the products here never overflow; results too small for
+// fp32 are far below half of the smallest E2M1 / E4M3 step and round to zero either way)
+__device__ __forceinline__ float pow2_inv_e8m0(uint32_t c) { return __uint_as_float((254u - c) << 23); }
+__device__ __forceinline__ float pow2_neg(int e) { return __uint_as_float((uint32_t)(127 - e) << 23); }
+
 // two floats -> two E2M1 codes in one byte (x in the low nibble)
 __device__ __forceinline__ uint32_t e2m1x2(float x, float y) {
   return (uint32_t)__nv_cvt_float2_to_fp4x2(make_float2(x, y), __NV_E2M1, cudaRoundNearest);

@@ -81,7 +81,7 @@ inline PackedOffsets packed_offsets(int64_t N, int64_t K, int out_n) {
 }
 
 struct ActOffsets {
-  size_t xi, xo, sfb_out, sexp, total;
+  size_t xi, xo, sfb_out, sexp, amax, total;
   int64_t MT;
 };
 inline ActOffsets act_offsets(int64_t M, int64_t K) {
@@ -93,7 +93,8 @@ inline ActOffsets act_offsets(int64_t M, int64_t K) {
   o.xo = al(o.xi + MT * T2 * XI_BYTES);
   o.sfb_out = al(o.xo + MT * T1 * XO_BYTES);
   o.sexp = al(o.sfb_out + MT * SF_ATOM_BYTES);
-  o.total = al(o.sexp + MT * TILE_TOK * 4);
+  o.amax = al(o.sexp + MT * TILE_TOK * 4);                       // per-token chunk maxima [MT*128][ceil(K/1024)] f32
+  o.total = al(o.amax + MT * TILE_TOK * ((size_t)(K + 1023) / 1024) * 4);
   return o;
 }
 

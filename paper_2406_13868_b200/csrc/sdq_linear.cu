@@ -1,13 +1,17 @@
 // Fused decomposed GEMM  Y = A_i W_i^T + A_o W_o^T   (Section 5.1: O = O_i + O_o)
 //
-// The sparse operand of tcgen05.mma.sp is A, so the kernel computes Y^T = W X^T: the 128 weight rows
-// of a tile sit on the 128 TMEM lanes, tokens on the accumulator columns.  Per 128 logical K:
-//   1 x tcgen05.mma.sp kind::mxf4      (pair-wise 4:8 E2M1 inliers x E2M1 activations, E8M0 per 64 K)
-//   2 x tcgen05.mma.sp kind::mxf8f6f4  (1:8 / 2:8 E4M3 outliers embedded in 2:4 x E4M3 activations;
-//                                       the power-of-two row / token scales ride in as E8M0 factors)
-// all into ONE fp32 TMEM accumulator.  Warp roles: warp 0 = bulk-copy (TMA) producer, warp 1 = TMEM
-// owner + MMA issuer (also moves metadata / scale atoms smem -> TMEM with tcgen05.cp), warps 2..5 =
-// epilogue (tcgen05.ld, convert, transposed store).  Every wait is bounded; a timeout sets a sticky flag.
+// The sparse operand of tcgen05.mma.sp is A, so the kernel computes Y^T = W X^T: the 128 weight rows of a
+// tile sit on the 128 TMEM lanes, tokens on the accumulator columns.  A tile first runs its inlier K loop
+//   2 x tcgen05.mma.sp kind::mxf4 per 256 K     (pair-wise 4:8 E2M1 inliers x E2M1 activations, E8M0 per 64 K)
+// then its outlier K loop
+//   2 x tcgen05.mma.sp kind::mxf8f6f4 per 128 K (1:8 / 2:8 E4M3 outliers embedded in 2:4 x E4M3 activations;
+//                                                the power-of-two row / token scales ride in as E8M0 factors)
+// both into ONE fp32 TMEM accumulator.  Persistent CTAs walk tiles of 128 rows x up to 256 tokens.
+// Warp roles: warp 0 = bulk-copy (TMA) producer, warp 1 = TMEM owner + MMA issuer (also moves metadata and
+// scale atoms smem -> TMEM with tcgen05.cp), warps 2..5 = epilogue (tcgen05.ld, convert, shared-memory
+// transpose, 16-byte row stores).  For few tokens the K range of a row tile is split over several CTAs; the
+// fp32 partial tiles go to a caller-provided workspace and the last CTA to arrive adds them in split order
+// (deterministic).  Every wait is bounded; a timeout sets a sticky flag.
 #include <cuda_bf16.h>
 
 #include "sdq_internal.h"
@@ -18,14 +22,13 @@
 namespace sdq {
 
 constexpr int LIN_THREADS = 192;
-constexpr int NSLOT = 5;
-constexpr int SLOT_BYTES = 45056;              // one ring slot holds either an inlier or an outlier stage
+constexpr int MAX_SLOTS = 16;
 constexpr int SL_A = 0;                        // WI record (A_in | E_in | SFA_in) or WO record (A_out | E_out)
-constexpr int SL_B = 10752;                    // B4 (256 K) or B8 (128 K) of up to 256 tokens: 32768 B
-constexpr int SL_SF = SL_B + 32768;            // inlier: SFB_in atoms (2 x 512); outlier stage 0: SFA_out | SFB_out x 2
-constexpr int SM_STG = NSLOT * SLOT_BYTES;      // epilogue transpose buffer: 16 tokens x 128 features bf16
+constexpr int SL_B = 10752;                    // B4 (256 K) or B8 (128 K) of n_tile tokens: n_tile * 128 B
+constexpr int RING_BYTES = 225280;             // ring of nslot slots of slot_bytes each
+constexpr int SM_STG = RING_BYTES;             // epilogue transpose buffer: 16 tokens x 128 features bf16
 constexpr int SM_BARS = SM_STG + 4096;
-constexpr int LIN_SMEM = SM_BARS + 128 + 128;  // + barriers + alignment slack
+constexpr int LIN_SMEM = SM_BARS + 320 + 128;  // + barriers + alignment slack
 
 // TMEM columns
 constexpr uint32_t TM_D = 0;          // accumulator: up to 256 columns (tokens)
@@ -34,7 +37,26 @@ constexpr uint32_t TM_EO = 288;       // 2 buffers x 4 columns: E_out
 constexpr uint32_t TM_SFA_OUT = 296;  // 4 columns
 constexpr uint32_t TM_SFB_OUT = 300;  // 8 columns
 
+// slot = | A record 10752 | B n_tile*128 | scale atoms 1536 |  (inlier: SFB_in x n_atiles; first outlier stage:
+// SFA_out | SFB_out x n_atiles)
+__host__ __device__ inline int slot_bytes_for(int n_tile) { return SL_B + n_tile * 128 + 1536; }
 
+struct TileCoord {
+  int rt, mtile, split;
+  int i0, i1, o0, o1;   // inlier stages [i0, i1) of T2, outlier stages [o0, o1) of T1
+};
+__device__ __forceinline__ TileCoord tile_coord(const LinearParams& p, int tile, int RT, int T1, int T2) {
+  TileCoord c;
+  c.split = tile % p.ksplit;
+  const int rest = tile / p.ksplit;
+  c.rt = rest % RT;
+  c.mtile = rest / RT;
+  c.i0 = (int)((int64_t)c.split * T2 / p.ksplit);
+  c.i1 = (int)((int64_t)(c.split + 1) * T2 / p.ksplit);
+  c.o0 = (int)((int64_t)c.split * T1 / p.ksplit);
+  c.o1 = (int)((int64_t)(c.split + 1) * T1 / p.ksplit);
+  return c;
+}
 
 template <bool F32_OUT>
 __global__ void __launch_bounds__(LIN_THREADS, 1)
@@ -44,18 +66,21 @@ sdq_linear_kernel(const LinearParams p)
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint8_t* sm = smem_raw + ((128 - (ptx::smem_u32(smem_raw) & 127)) & 127);
   uint64_t* full = reinterpret_cast<uint64_t*>(sm + SM_BARS);
-  uint64_t* empty = full + NSLOT;
-  uint64_t* acc_full = empty + NSLOT;
+  uint64_t* empty = full + MAX_SLOTS;
+  uint64_t* acc_full = empty + MAX_SLOTS;
   uint64_t* acc_empty = acc_full + 1;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
+  uint32_t* last_flag = tmem_slot + 1;
 
   const int n_tile = p.n_tile;
   const int RT = (int)(p.N / TILE_ROWS);
   const int T1 = p.out_n ? (int)(p.K / K1) : 0, T2 = (int)(p.K / K2);
   const int n_atiles = (n_tile + TILE_TOK - 1) / TILE_TOK;     // 128-token activation tiles per token tile
+  const uint32_t nslot = (uint32_t)p.nslot, slot_bytes = (uint32_t)p.slot_bytes;
+  const uint32_t sl_sf = SL_B + (uint32_t)n_tile * 128u;
 
   if (tid == 0) {
-    for (int s = 0; s < NSLOT; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
+    for (uint32_t s = 0; s < nslot; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
     ptx::mbar_init(acc_full, 1);
     ptx::mbar_init(acc_empty, 4);
     ptx::fence_barrier_init();
@@ -67,49 +92,49 @@ sdq_linear_kernel(const LinearParams p)
   const uint32_t tmem = *tmem_slot;
 
   if (warp == 0) {
-    if (lane < NSLOT) {
-      // ---------------- producer: bulk copies, inlier stages of the tile first, then its outlier stages.
-      // Lane l owns ring slot l, so the barrier round trips of different slots overlap.
+    if (lane == 0) {
+      // ---------------- producer: bulk copies, inlier stages of the tile first, then its outlier stages
       bool ok = true;
-      uint32_t it = 0;
+      uint32_t s = 0, wrapped = 0, ph = 0;   // ring slot, whether the ring has wrapped, phase parity of `empty`
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-        const int rt = tile % RT, mtile = tile / RT;
-        const int64_t m0 = (int64_t)mtile * n_tile;
+        const TileCoord tc = tile_coord(p, tile, RT, T1, T2);
+        const int64_t m0 = (int64_t)tc.mtile * n_tile;
         const int64_t mt = m0 / TILE_TOK;
-        const int have = (int)min((int64_t)n_atiles, p.aoff.MT - mt);     // activation tiles that exist
+        const int have = (int)min((int64_t)n_atiles, p.aoff.MT - mt);        // activation tiles that exist
         const uint32_t tok_bytes = (uint32_t)min(n_tile, TILE_TOK) * 128u;   // bytes per activation tile per stage
-        const uint8_t* wi = p.w + p.poff.wi + (size_t)rt * T2 * WI_BYTES;
-        const uint8_t* wo = p.w + p.poff.wo + (size_t)rt * T1 * WO_BYTES;
-        const uint8_t* xi = p.x + p.aoff.xi + (size_t)mt * T2 * XI_BYTES;
-        const uint8_t* xo = p.x + p.aoff.xo + (size_t)mt * T1 * XO_BYTES;
-        for (int k = 0; k < T2 + T1 && ok; ++k, ++it) {
-          const uint32_t s = it % NSLOT;
-          if (s != lane) continue;
-          if (it >= NSLOT) ok = ptx::mbar_wait(&empty[s], ((it / NSLOT) - 1) & 1);
-          if (!ok) break;
-          uint8_t* st = sm + (size_t)s * SLOT_BYTES;
-          if (k < T2) {
+        const uint8_t* wi = p.w + p.poff.wi + ((size_t)tc.rt * T2 + tc.i0) * WI_BYTES;
+        const uint8_t* wo = p.w + p.poff.wo + ((size_t)tc.rt * T1 + tc.o0) * WO_BYTES;
+        const uint8_t* xi = p.x + p.aoff.xi + ((size_t)mt * T2 + tc.i0) * XI_BYTES;
+        const uint8_t* xo = p.x + p.aoff.xo + ((size_t)mt * T1 + tc.o0) * XO_BYTES;
+        const int ni = tc.i1 - tc.i0, no = tc.o1 - tc.o0;
+        for (int k = 0; k < ni + no; ++k) {
+          if (wrapped && !(ok = ptx::mbar_wait(&empty[s], ph ^ 1))) break;
+          uint8_t* st = sm + (size_t)s * slot_bytes;
+          if (k < ni) {
             ptx::mbar_expect_tx(&full[s], WI_BYTES + (uint32_t)have * (tok_bytes + SF_ATOM_BYTES));
-            ptx::bulk_g2s(st + SL_A, wi + (size_t)k * WI_BYTES, WI_BYTES, &full[s]);
+            ptx::bulk_g2s(st + SL_A, wi, WI_BYTES, &full[s]);
             for (int a = 0; a < have; ++a) {
-              const uint8_t* src = xi + ((size_t)a * T2 + k) * XI_BYTES;
+              const uint8_t* src = xi + (size_t)a * T2 * XI_BYTES;
               ptx::bulk_g2s(st + SL_B + a * B4_BYTES, src, tok_bytes, &full[s]);
-              ptx::bulk_g2s(st + SL_SF + a * SF_ATOM_BYTES, src + B4_BYTES, SF_ATOM_BYTES, &full[s]);
+              ptx::bulk_g2s(st + sl_sf + a * SF_ATOM_BYTES, src + B4_BYTES, SF_ATOM_BYTES, &full[s]);
             }
+            wi += WI_BYTES;
+            xi += XI_BYTES;
           } else {
-            const int k1 = k - T2;
-            const uint32_t sf_bytes = (k1 == 0) ? (uint32_t)(1 + have) * SF_ATOM_BYTES : 0u;
-            ptx::mbar_expect_tx(&full[s], WO_BYTES + (uint32_t)have * tok_bytes + sf_bytes);
-            ptx::bulk_g2s(st + SL_A, wo + (size_t)k1 * WO_BYTES, WO_BYTES, &full[s]);
-            for (int a = 0; a < have; ++a)
-              ptx::bulk_g2s(st + SL_B + a * B8_BYTES, xo + ((size_t)a * T1 + k1) * XO_BYTES, tok_bytes, &full[s]);
-            if (k1 == 0) {
-              ptx::bulk_g2s(st + SL_SF, p.w + p.poff.sfa_out + (size_t)rt * SF_ATOM_BYTES, SF_ATOM_BYTES, &full[s]);
+            const bool first = (k == ni);
+            ptx::mbar_expect_tx(&full[s], WO_BYTES + (uint32_t)have * tok_bytes + (first ? (uint32_t)(1 + have) * SF_ATOM_BYTES : 0u));
+            ptx::bulk_g2s(st + SL_A, wo, WO_BYTES, &full[s]);
+            for (int a = 0; a < have; ++a) ptx::bulk_g2s(st + SL_B + a * B8_BYTES, xo + (size_t)a * T1 * XO_BYTES, tok_bytes, &full[s]);
+            if (first) {
+              ptx::bulk_g2s(st + sl_sf, p.w + p.poff.sfa_out + (size_t)tc.rt * SF_ATOM_BYTES, SF_ATOM_BYTES, &full[s]);
               for (int a = 0; a < have; ++a)
-                ptx::bulk_g2s(st + SL_SF + (1 + a) * SF_ATOM_BYTES, p.x + p.aoff.sfb_out + (size_t)(mt + a) * SF_ATOM_BYTES,
+                ptx::bulk_g2s(st + sl_sf + (1 + a) * SF_ATOM_BYTES, p.x + p.aoff.sfb_out + (size_t)(mt + a) * SF_ATOM_BYTES,
                               SF_ATOM_BYTES, &full[s]);
             }
+            wo += WO_BYTES;
+            xo += XO_BYTES;
           }
+          if (++s == nslot) { s = 0; wrapped = 1; ph ^= 1; }
         }
       }
       if (!ok) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
@@ -119,55 +144,62 @@ sdq_linear_kernel(const LinearParams p)
       // ---------------- MMA issuer
       bool ok = true;
       const uint32_t smb = ptx::smem_u32(sm);
-      uint32_t it = 0, tcount = 0;
+      uint32_t s = 0, ph = 0, tcount = 0;
       bool ready = false;
       const uint32_t id4[2] = {ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, true, 0, 0),
                                ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, true, 2, 2)};
       const uint32_t id8 = ptx::idesc_block_scaled(128, (uint32_t)n_tile, 0, true, 0, 0);
+      // descriptors of slot 0; slot s adds s * slot_bytes / 16 to the start-address field
+      const uint64_t d_a = ptx::smem_desc(smb + SL_A, 128, 256), d_b = ptx::smem_desc(smb + SL_B, 128, 1024);
+      const uint64_t d_e_in = ptx::smem_desc(smb + SL_A + A_IN_BYTES, 0, 128);
+      const uint64_t d_sfa_in = ptx::smem_desc(smb + SL_A + A_IN_BYTES + E_IN_BYTES, 0, 128);
+      const uint64_t d_e_out = ptx::smem_desc(smb + SL_A + A_OUT_BYTES, 0, 128);
+      const uint64_t d_sf0 = ptx::smem_desc(smb + sl_sf, 0, 128), d_sf1 = ptx::smem_desc(smb + sl_sf + SF_ATOM_BYTES, 0, 128);
+      const uint64_t d_sf2 = ptx::smem_desc(smb + sl_sf + 2 * SF_ATOM_BYTES, 0, 128);
+      const uint32_t slot16 = slot_bytes >> 4;
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
+        const TileCoord tc = tile_coord(p, tile, RT, T1, T2);
+        const int ni = tc.i1 - tc.i0, no = tc.o1 - tc.o0;
         if (tcount > 0) {   // the epilogue must have drained the accumulator of the previous tile
           ok = ptx::mbar_wait(acc_empty, (tcount - 1) & 1);
           if (!ok) break;
           ptx::tc_fence_after();
         }
-        for (int k = 0; k < T2 + T1 && ok; ++k, ++it) {
-          const uint32_t s = it % NSLOT;
-          if (!ready) ok = ptx::mbar_wait(&full[s], (it / NSLOT) & 1);
+        uint32_t acc = 0;   // the first MMA of the tile overwrites the accumulator
+        for (int k = 0; k < ni + no; ++k) {
+          if (!ready) ok = ptx::mbar_wait(&full[s], ph);
           if (!ok) break;
           ptx::tc_fence_after();
+          const uint32_t sn = (s + 1 == nslot) ? 0 : s + 1;
           // poll the next slot now: the answer is back by the time this stage's instructions are issued
-          ready = ptx::mbar_test(&full[(it + 1) % NSLOT], ((it + 1) / NSLOT) & 1);
-          const uint32_t st = smb + s * SLOT_BYTES;
-          if (k < T2) {
+          ready = ptx::mbar_test(&full[sn], sn ? ph : ph ^ 1);
+          const uint64_t so = (uint64_t)(s * slot16);
+          if (k < ni) {
             // inlier stage: 256 logical K = 2 sparse MXFP4 MMAs; metadata and scale atoms go to TMEM first
             const uint32_t mb = tmem + TM_I + 16u * (uint32_t)(k & 1);
-            ptx::tc_cp_128x128b(mb + 0, ptx::smem_desc(st + SL_A + A_IN_BYTES, 0, 128));
-            ptx::tc_cp_32x128b_warpx4(mb + 4, ptx::smem_desc(st + SL_A + A_IN_BYTES + E_IN_BYTES, 0, 128));
-            ptx::tc_cp_32x128b_warpx4(mb + 8, ptx::smem_desc(st + SL_SF, 0, 128));
-            if (n_atiles > 1) ptx::tc_cp_32x128b_warpx4(mb + 12, ptx::smem_desc(st + SL_SF + SF_ATOM_BYTES, 0, 128));
-#pragma unroll
-            for (uint32_t j = 0; j < 2; ++j)
-              ptx::mma_sp_mxf4(tmem + TM_D, ptx::smem_desc(st + SL_A + j * 4096, 128, 256),
-                               ptx::smem_desc(st + SL_B + j * 512, 128, 1024), id4[j], mb + 2 * j, mb + 4, mb + 8,
-                               (k > 0 || j > 0) ? 1u : 0u);
+            ptx::tc_cp_128x128b(mb + 0, d_e_in + so);
+            ptx::tc_cp_32x128b_warpx4(mb + 4, d_sfa_in + so);
+            ptx::tc_cp_32x128b_warpx4(mb + 8, d_sf0 + so);
+            if (n_atiles > 1) ptx::tc_cp_32x128b_warpx4(mb + 12, d_sf1 + so);
+            ptx::mma_sp_mxf4(tmem + TM_D, d_a + so, d_b + so, id4[0], mb, mb + 4, mb + 8, acc);
+            ptx::mma_sp_mxf4(tmem + TM_D, d_a + so + (4096 >> 4), d_b + so + (512 >> 4), id4[1], mb + 2, mb + 4, mb + 8, 1u);
           } else {
-            // outlier stage: 128 logical K = 2 sparse FP8 MMAs; the row / token scales (E8M0) arrive with stage 0
-            const int k1 = k - T2;
-            const uint32_t eb = tmem + TM_EO + 4u * (uint32_t)(k1 & 1);
-            ptx::tc_cp_128x128b(eb, ptx::smem_desc(st + SL_A + A_OUT_BYTES, 0, 128));
-            if (k1 == 0) {
-              ptx::tc_cp_32x128b_warpx4(tmem + TM_SFA_OUT, ptx::smem_desc(st + SL_SF, 0, 128));
-              ptx::tc_cp_32x128b_warpx4(tmem + TM_SFB_OUT, ptx::smem_desc(st + SL_SF + SF_ATOM_BYTES, 0, 128));
-              if (n_atiles > 1)
-                ptx::tc_cp_32x128b_warpx4(tmem + TM_SFB_OUT + 4, ptx::smem_desc(st + SL_SF + 2 * SF_ATOM_BYTES, 0, 128));
+            // outlier stage: 128 logical K = 2 sparse FP8 MMAs; the row / token scales (E8M0) arrive with the first one
+            const uint32_t eb = tmem + TM_EO + 4u * (uint32_t)(k & 1);
+            ptx::tc_cp_128x128b(eb, d_e_out + so);
+            if (k == ni) {
+              ptx::tc_cp_32x128b_warpx4(tmem + TM_SFA_OUT, d_sf0 + so);
+              ptx::tc_cp_32x128b_warpx4(tmem + TM_SFB_OUT, d_sf1 + so);
+              if (n_atiles > 1) ptx::tc_cp_32x128b_warpx4(tmem + TM_SFB_OUT + 4, d_sf2 + so);
             }
-#pragma unroll
-            for (uint32_t j = 0; j < 2; ++j)
-              ptx::mma_sp_mxf8(tmem + TM_D, ptx::smem_desc(st + SL_A + j * 4096, 128, 256),
-                               ptx::smem_desc(st + SL_B + j * 512, 128, 1024), id8, eb + 2 * j, tmem + TM_SFA_OUT,
-                               tmem + TM_SFB_OUT, 1u);
+            ptx::mma_sp_mxf8(tmem + TM_D, d_a + so, d_b + so, id8, eb, tmem + TM_SFA_OUT, tmem + TM_SFB_OUT, acc);
+            ptx::mma_sp_mxf8(tmem + TM_D, d_a + so + (4096 >> 4), d_b + so + (512 >> 4), id8, eb + 2, tmem + TM_SFA_OUT,
+                             tmem + TM_SFB_OUT, 1u);
           }
+          acc = 1;
           ptx::tc_commit(&empty[s]);
+          s = sn;
+          if (sn == 0) ph ^= 1;
         }
         ptx::tc_commit(acc_full);
       }
@@ -176,17 +208,20 @@ sdq_linear_kernel(const LinearParams p)
   } else {
     // ---------------- epilogue: warp w owns TMEM lanes 32*(w%4) .. +31 (weight rows), columns = tokens
     const uint32_t q = warp & 3;
+    const uint32_t et = (warp - 2) * 32 + lane;     // 0..127 among the epilogue threads
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
-      const int rt = tile % RT, mtile = tile / RT;
-      const int64_t m0 = (int64_t)mtile * n_tile;
+      const TileCoord tc = tile_coord(p, tile, RT, T1, T2);
+      const int64_t m0 = (int64_t)tc.mtile * n_tile;
       const int n_valid = (int)min((int64_t)n_tile, p.M - m0);
       ok = ptx::mbar_wait(acc_full, tcount & 1);
       ptx::tc_fence_after();
       if (!ok) break;
-      const int64_t n0 = (int64_t)rt * TILE_ROWS;
-      const uint32_t et = (warp - 2) * 32 + lane;     // 0..127 among the epilogue threads
+      const int64_t n0 = (int64_t)tc.rt * TILE_ROWS;
+      // split-K: this CTA's fp32 partial tile [token][128 rows] in the workspace
+      float* part = p.ksplit > 1 ? p.ws_partial + ((size_t)(tc.rt * p.n_mtiles + tc.mtile) * p.ksplit + tc.split) * (size_t)n_tile * TILE_ROWS
+                                 : nullptr;
 #pragma unroll 1
       for (int c0 = 0; c0 < n_tile; c0 += 16) {
         uint32_t v[16];
@@ -200,7 +235,11 @@ sdq_linear_kernel(const LinearParams p)
           if (lane == 0) ptx::mbar_arrive(acc_empty);
         }
         if (c0 >= n_valid) continue;  // uniform over the four epilogue warps
-        if (F32_OUT) {
+        if (part) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (c0 + j < n_valid) part[(size_t)(c0 + j) * TILE_ROWS + q * 32 + lane] = __uint_as_float(v[j]);
+        } else if (F32_OUT) {
           float* Y = reinterpret_cast<float*>(p.Y);
 #pragma unroll
           for (int j = 0; j < 16; ++j)
@@ -223,6 +262,42 @@ sdq_linear_kernel(const LinearParams p)
           ptx::named_bar_sync(1, 128);   // the buffer is rewritten by the next chunk
         }
       }
+      if (part) {
+        // the last CTA of this (row tile, token tile) to finish adds the partial tiles in split order
+        __threadfence();
+        ptx::named_bar_sync(1, 128);
+        uint32_t* counter = p.ws_counter + tc.rt * p.n_mtiles + tc.mtile;
+        if (et == 0) {
+          const uint32_t old = atomicAdd(counter, 1u);
+          *last_flag = (old == (uint32_t)p.ksplit - 1) ? 1u : 0u;
+        }
+        ptx::named_bar_sync(1, 128);
+        if (*last_flag) {
+          __threadfence();
+          const float* base = p.ws_partial + (size_t)(tc.rt * p.n_mtiles + tc.mtile) * p.ksplit * (size_t)n_tile * TILE_ROWS;
+          // 8 tokens at a time: the loads of one split are independent, only the adds follow split order
+          for (int t0 = 0; t0 < n_valid; t0 += 8) {
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 2
+            for (int sp = 0; sp < p.ksplit; ++sp) {
+              const float* src = base + ((size_t)sp * n_tile + t0) * TILE_ROWS + et;
+              float v[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) v[j] = (t0 + j < n_valid) ? __ldcg(src + (size_t)j * TILE_ROWS) : 0.0f;
+#pragma unroll
+              for (int j = 0; j < 8; ++j) acc[j] += v[j];
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              if (t0 + j < n_valid) {
+                if (F32_OUT) reinterpret_cast<float*>(p.Y)[(m0 + t0 + j) * p.ldy + n0 + et] = acc[j];
+                else reinterpret_cast<__nv_bfloat16*>(p.Y)[(m0 + t0 + j) * p.ldy + n0 + et] = __float2bfloat16_rn(acc[j]);
+              }
+          }
+          if (et == 0) *counter = 0u;     // ready for the next call
+        }
+        ptx::named_bar_sync(1, 128);       // last_flag is rewritten by the next tile
+      }
     }
     if (!ok && lane == 0) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
   }
@@ -235,13 +310,46 @@ sdq_linear_kernel(const LinearParams p)
 
 using namespace sdq;
 
-static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y, int64_t ldy, void* stream, bool f32)
+static int sm_count_cached() {
+  static int sm_count = 0;
+  if (!sm_count) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sm_count = 0;
+  }
+  return sm_count;
+}
+
+// number of K splits for a call: only for M <= 128 (one token tile), as many as keep one CTA per SM,
+// never more than the inlier stages so that every split owns at least one
+static int choose_ksplit(int64_t M, int64_t N, int64_t K, int sm_count) {
+  if (M > 128 || sm_count <= 0) return 1;
+  const int RT = (int)(N / TILE_ROWS), T2 = (int)(K / K2);
+  int ks = sm_count / RT;
+  if (ks > T2) ks = T2;
+  if (ks > 32) ks = 32;
+  return ks < 1 ? 1 : ks;
+}
+static int n_tile_for(int64_t M) { return M > 128 ? 256 : (M > 64 ? 128 : (M > 32 ? 64 : (M > 16 ? 32 : 16))); }
+
+extern "C" sdq_status_t sdq_workspace_size(int64_t M, int64_t N, int64_t K, const sdq_config_t* cfg, size_t* bytes)
+{
+  if (!cfg || !bytes) return SDQ_ERR_INVALID_ARG;
+  if (M <= 0 || N <= 0 || K <= 0 || N % TILE_ROWS || K % K2) return SDQ_ERR_SHAPE;
+  const int ks = choose_ksplit(M, N, K, sm_count_cached());
+  const size_t RT = (size_t)(N / TILE_ROWS);
+  // counters first (one per row tile, 256 B aligned), then ks fp32 partial tiles per row tile
+  *bytes = ks > 1 ? ((RT * 4 + 255) & ~(size_t)255) + RT * (size_t)ks * (size_t)n_tile_for(M) * TILE_ROWS * 4 : 0;
+  return SDQ_OK;
+}
+
+static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y, int64_t ldy, void* ws, size_t ws_bytes,
+                                  void* stream, bool f32)
 {
   if (!Xq || !P || !Y || !Xq->dev || !P->dev) return SDQ_ERR_INVALID_ARG;
   if (Xq->K != P->K || Xq->M <= 0 || P->N <= 0 || P->N % TILE_ROWS || P->K % K2 || ldy < P->N) return SDQ_ERR_SHAPE;
   if (Xq->cfg.in_block != P->cfg.in_block || Xq->cfg.scale_rule != P->cfg.scale_rule) return SDQ_ERR_SHAPE;
   if (P->cfg.in_gran != SDQ_GRAN_PAIR || P->cfg.in_block != 64) return SDQ_ERR_UNSUPPORTED;
-  if (((uintptr_t)Y & 15) || (ldy % 8)) return SDQ_ERR_ALIGNMENT;
+  if (((uintptr_t)Y & 15) || (ldy % 8) || ((uintptr_t)ws & 15)) return SDQ_ERR_ALIGNMENT;
   static bool attr_set[2] = {false, false};
   if (!attr_set[f32]) {
     cudaError_t e = f32 ? cudaFuncSetAttribute(sdq_linear_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM)
@@ -249,6 +357,8 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
     if (e != cudaSuccess) return SDQ_ERR_CUDA;
     attr_set[f32] = true;
   }
+  const int sm_count = sm_count_cached();
+  if (!sm_count) return SDQ_ERR_CUDA;
   LinearParams p;
   p.w = (const uint8_t*)P->dev;
   p.x = (const uint8_t*)Xq->dev;
@@ -257,17 +367,29 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   p.M = Xq->M; p.N = P->N; p.K = P->K;
   p.out_n = P->cfg.out_n;
   const int64_t M = Xq->M;
-  p.n_tile = M > 128 ? 256 : (M > 64 ? 128 : (M > 32 ? 64 : (M > 16 ? 32 : 16)));
+  p.n_tile = n_tile_for(M);
   p.n_mtiles = (int)((M + p.n_tile - 1) / p.n_tile);
-  p.total_tiles = (int)(P->N / TILE_ROWS) * p.n_mtiles;
+  p.slot_bytes = slot_bytes_for(p.n_tile);
+  p.nslot = RING_BYTES / p.slot_bytes;
+  if (p.nslot > MAX_SLOTS) p.nslot = MAX_SLOTS;
+  p.ksplit = 1;
+  p.ws_counter = nullptr;
+  p.ws_partial = nullptr;
+  if (ws) {
+    const int ks = choose_ksplit(M, P->N, P->K, sm_count);
+    size_t need = 0;
+    sdq_workspace_size(M, P->N, P->K, &P->cfg, &need);
+    if (ks > 1) {
+      if (ws_bytes < need) return SDQ_ERR_BUFFER_TOO_SMALL;
+      p.ksplit = ks;
+      p.ws_counter = (uint32_t*)ws;
+      p.ws_partial = (float*)((uint8_t*)ws + (((size_t)(P->N / TILE_ROWS) * 4 + 255) & ~(size_t)255));
+    }
+  }
+  p.total_tiles = (int)(P->N / TILE_ROWS) * p.n_mtiles * p.ksplit;
   p.Y = Y; p.ldy = ldy;
   p.flags = device_flags();
   if (!p.flags) return SDQ_ERR_CUDA;
-  static int sm_count = 0;
-  if (!sm_count) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SDQ_ERR_CUDA;
-  }
   dim3 grid((unsigned)(p.total_tiles < sm_count ? p.total_tiles : sm_count));
   if (f32) sdq_linear_kernel<true><<<grid, LIN_THREADS, LIN_SMEM, (cudaStream_t)stream>>>(p);
   else sdq_linear_kernel<false><<<grid, LIN_THREADS, LIN_SMEM, (cudaStream_t)stream>>>(p);
@@ -275,7 +397,22 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
 }
 
 extern "C" sdq_status_t sdq_linear(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y, int64_t ldy, void* stream)
-{ return launch_linear(Xq, P, Y, ldy, stream, false); }
+{ return launch_linear(Xq, P, Y, ldy, nullptr, 0, stream, false); }
 
 extern "C" sdq_status_t sdq_linear_f32(const sdq_act_t* Xq, const sdq_packed_t* P, float* Y, int64_t ldy, void* stream)
-{ return launch_linear(Xq, P, (void*)Y, ldy, stream, true); }
+{ return launch_linear(Xq, P, (void*)Y, ldy, nullptr, 0, stream, true); }
+
+extern "C" sdq_status_t sdq_workspace_init(void* ws, size_t ws_bytes, void* stream)
+{
+  if (!ws) return SDQ_ERR_INVALID_ARG;
+  if ((uintptr_t)ws & 15) return SDQ_ERR_ALIGNMENT;
+  return cudaMemsetAsync(ws, 0, ws_bytes, (cudaStream_t)stream) == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
+}
+
+extern "C" sdq_status_t sdq_linear_ws(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y, int64_t ldy, void* ws, size_t ws_bytes,
+                                      void* stream)
+{ return launch_linear(Xq, P, Y, ldy, ws, ws_bytes, stream, false); }
+
+extern "C" sdq_status_t sdq_linear_f32_ws(const sdq_act_t* Xq, const sdq_packed_t* P, float* Y, int64_t ldy, void* ws, size_t ws_bytes,
+                                          void* stream)
+{ return launch_linear(Xq, P, (void*)Y, ldy, ws, ws_bytes, stream, true); }

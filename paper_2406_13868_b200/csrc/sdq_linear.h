@@ -17,7 +17,11 @@ struct LinearParams {
   int out_n;
   int n_tile;            // tokens per tile: 16, 32, 64, 128 or 256
   int n_mtiles;          // ceil(M / n_tile)
-  int total_tiles;       // (N / 128) * n_mtiles
+  int total_tiles;       // (N / 128) * n_mtiles * ksplit
+  int nslot, slot_bytes; // shared-memory ring geometry (depends on n_tile)
+  int ksplit;            // CTAs sharing the K range of one row tile (1 = no split)
+  uint32_t* ws_counter;  // split-K workspace: arrival counters [row tile], zero between calls
+  float* ws_partial;     // split-K workspace: fp32 partial tiles [row tile][split][token][128 rows]
   void* Y;
   int64_t ldy;
   uint32_t* flags;

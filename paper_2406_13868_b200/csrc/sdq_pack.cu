@@ -146,7 +146,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
       const int p = slot_pos[s];
-      v[s] = (p == o0 || p == o1) ? 0.0f : scalbnf(bf16_bits_to_float(bits[p]), 127 - (int)c);
+      v[s] = (p == o0 || p == o1) ? 0.0f : bf16_bits_to_float(bits[p]) * pow2_inv_e8m0(c);
     }
     const uint32_t codes = e2m1x2(v[0], v[1]) | (e2m1x2(v[2], v[3]) << 8);
 
@@ -164,8 +164,8 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     if (out_n > 0) {
       // Stage 3, outliers: E4M3 codes of w / 2^e; compact arrays plus the 2:4 embedding the sparse
       // FP8 tensor-core path consumes (per 4 K: two ascending slot indices, unused slots hold +0)
-      const uint32_t c0 = e4m3x1(scalbnf(bf16_bits_to_float(bits[o0]), -e));
-      const uint32_t c1 = (o1 >= 0) ? e4m3x1(scalbnf(bf16_bits_to_float(bits[o1]), -e)) : 0u;
+      const uint32_t c0 = e4m3x1(bf16_bits_to_float(bits[o0]) * pow2_neg(e));
+      const uint32_t c1 = (o1 >= 0) ? e4m3x1(bf16_bits_to_float(bits[o1]) * pow2_neg(e)) : 0u;
       uint8_t* oc = blob + off.ocode + ((size_t)n * G + g) * out_n;
       uint8_t* oi = blob + off.oidx + ((size_t)n * G + g) * out_n;
       oc[0] = (uint8_t)c0;

@@ -1,10 +1,13 @@
 // Runtime activation quantization A -> A_i (E2M1 + E8M0 per 64 K) and A_o (E4M3 + per-token power-of-two
 // scale), "we also quantize activations accordingly" (Section 5, Stage 3; A_o / A_i of Section 5.1).
 //
-// One CTA per token row, 16-byte loads (8 bf16 per thread per step).  Pass 1 reduces the row's largest
-// magnitude (the 8-bit scale needs the whole row); pass 2 re-reads the row (L2 resident), reduces each
-// 64-K Q-Vector over 8 lanes by warp shuffle, converts with the hardware E2M1 / E4M3 converters and
-// stores packed codes straight into the stage-tiled layout the GEMM streams with bulk copies.
+// Two launches.  `act_amax_kernel` reduces, per token, the largest magnitude of each 1024-K chunk (the
+// per-token 8-bit scale needs the whole row before anything can be stored).  `quant_act_kernel` then encodes:
+// one CTA per (group of 8 tokens = one row group of the tiled operand layout, 1024-K chunk).  A warp works
+// on one 64-K Q-Vector of all 8 tokens at a time: 4 lanes per token, 16 elements (two 16-byte loads) per
+// lane, so the Q-Vector maximum is a 4-lane shuffle and every store instruction writes whole 128-byte lines
+// of the stage-tiled layout (8 tokens x 16 B per core matrix).  Codes come from the hardware E2M1 / E4M3
+// converters and go straight into the layout the GEMM streams.
 #include "sdq_codec.cuh"
 #include "sdq_internal.h"
 #include "sdq_layout.h"
@@ -12,87 +15,119 @@
 namespace sdq {
 
 constexpr int QA_THREADS = 256;
+constexpr int QA_WARPS = QA_THREADS / 32;
+constexpr int QA_CHUNK_QV = 16;                          // Q-Vectors (64 K each) per CTA: 1024 K
 
-__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&x)[8]) {
-  const uint4 v = *reinterpret_cast<const uint4*>(p);
-  const uint32_t r[4] = {v.x, v.y, v.z, v.w};
+__device__ __forceinline__ void load16(const __nv_bfloat16* p, float (&x)[16]) {
+  const uint4 a = reinterpret_cast<const uint4*>(p)[0], b = reinterpret_cast<const uint4*>(p)[1];
+  const uint32_t r[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < 8; ++i) {
     x[2 * i] = __uint_as_float(r[i] << 16);
     x[2 * i + 1] = __uint_as_float(r[i] & 0xFFFF0000u);
   }
 }
-// |x| with +-Inf replaced by the largest finite bf16 (saturation), as a float
+// |x| with +-Inf replaced by the largest finite bf16 (saturation)
 __device__ __forceinline__ float sat_abs(float x) { return fminf(fabsf(x), 3.3895313892515355e38f); }
 __device__ __forceinline__ float sat(float x) { return copysignf(sat_abs(x), x); }
 
+// partial[m][chunk] = max |x| of token m over its 1024-K chunk
 __global__ void __launch_bounds__(QA_THREADS)
-quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int64_t ldx, sdq_config_t cfg, uint8_t* __restrict__ buf,
-                 ActOffsets off)
+act_amax_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int64_t ldx, float* __restrict__ partial, int n_chunks)
 {
-  const int64_t m = blockIdx.x;
-  const int tid = threadIdx.x;
-  const __nv_bfloat16* x = X + m * ldx;
-  __shared__ float s_red[QA_THREADS / 32];
-  __shared__ int s_e;
-
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int t = lane >> 2, l = lane & 3;
+  const int64_t m = (int64_t)blockIdx.x * 8 + t;
+  const bool live = m < M;
+  const int NB = (int)(K / 64);
+  const int b0 = blockIdx.y * QA_CHUNK_QV;
+  __shared__ float s_amax[QA_WARPS][8];
   float amax = 0.0f;
-  for (int64_t k = (int64_t)tid * 8; k < K; k += QA_THREADS * 8) {
-    float v[8];
-    load8(x + k, v);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) amax = fmaxf(amax, sat_abs(v[i]));
+  for (int i = 0; i < QA_CHUNK_QV / QA_WARPS; ++i) {
+    const int b = b0 + warp + i * QA_WARPS;
+    if (live && b < NB) {
+      float v[16];
+      load16(X + m * ldx + (int64_t)b * 64 + l * 16, v);
+#pragma unroll
+      for (int j = 0; j < 16; ++j) amax = fmaxf(amax, sat_abs(v[j]));
+    }
   }
-#pragma unroll
-  for (int s = 16; s > 0; s >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, s));
-  if ((tid & 31) == 0) s_red[tid >> 5] = amax;
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+  if (l == 0) s_amax[warp][t] = amax;
   __syncthreads();
-  if (tid == 0) {
+  if (tid < 8 && (int64_t)blockIdx.x * 8 + tid < M) {
     float a = 0.0f;
 #pragma unroll
-    for (int i = 0; i < QA_THREADS / 32; ++i) a = fmaxf(a, s_red[i]);
-    s_e = fp8_scale_exp(a);
+    for (int w = 0; w < QA_WARPS; ++w) a = fmaxf(a, s_amax[w][tid]);
+    partial[((int64_t)blockIdx.x * 8 + tid) * n_chunks + blockIdx.y] = a;
   }
-  __syncthreads();
-  const int e = s_e;
+}
+
+__global__ void __launch_bounds__(QA_THREADS)
+quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int64_t ldx, sdq_config_t cfg, uint8_t* __restrict__ buf,
+                 ActOffsets off, const float* __restrict__ partial, int n_chunks)
+{
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int t = lane >> 2, l = lane & 3;                 // token within the group of 8, quarter of the Q-Vector
+  const int64_t m = (int64_t)blockIdx.x * 8 + t;
+  const bool live = m < M;
+  const int NB = (int)(K / 64);                           // Q-Vectors per row
+  const int b0 = blockIdx.y * QA_CHUNK_QV;
+
+  // per-token 8-bit scale from the chunk maxima of the whole row
+  float ramax = 0.0f;
+  if (live)
+    for (int c = l; c < n_chunks; c += 4) ramax = fmaxf(ramax, partial[m * n_chunks + c]);
+  ramax = fmaxf(ramax, __shfl_xor_sync(0xffffffffu, ramax, 1));
+  ramax = fmaxf(ramax, __shfl_xor_sync(0xffffffffu, ramax, 2));
+  const int e = fp8_scale_exp(ramax);
+  const float s8 = pow2_neg(e);
 
   const int64_t mt = m / TILE_TOK;
-  const uint32_t t = (uint32_t)(m % TILE_TOK);
+  const uint32_t tk = (uint32_t)(m % TILE_TOK);
   const int T1 = (int)(K / K1), T2 = (int)(K / K2);
   uint8_t* xi_base = buf + off.xi + (size_t)mt * T2 * XI_BYTES;
   uint8_t* xo_base = buf + off.xo + (size_t)mt * T1 * XO_BYTES;
-  if (tid == 0) {
+  if (live && blockIdx.y == 0 && warp == 0 && l == 0) {
     reinterpret_cast<int32_t*>(buf + off.sexp)[m] = e;
-    *reinterpret_cast<uint32_t*>(buf + off.sfb_out + (size_t)mt * SF_ATOM_BYTES + sf_off(t, 0)) = (uint32_t)(e + 127) * 0x01010101u;
+    *reinterpret_cast<uint32_t*>(buf + off.sfb_out + (size_t)mt * SF_ATOM_BYTES + sf_off(tk, 0)) = (uint32_t)(e + 127) * 0x01010101u;
   }
 
-  // K is a multiple of 256, so every warp-iteration covers whole 64-K Q-Vectors (8 lanes each)
-  for (int64_t k = (int64_t)tid * 8; k < K; k += QA_THREADS * 8) {
-    float v[8];
-    load8(x + k, v);
+#pragma unroll
+  for (int i = 0; i < QA_CHUNK_QV / QA_WARPS; ++i) {
+    const int b = b0 + warp + i * QA_WARPS;              // uniform over the warp
+    if (b >= NB) break;
+    float v[16];
+    if (live) load16(X + m * ldx + (int64_t)b * 64 + l * 16, v);
+    else {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) v[j] = 0.0f;
+    }
     float bmax = 0.0f;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      v[i] = sat(v[i]);
-      bmax = fmaxf(bmax, fabsf(v[i]));
+    for (int j = 0; j < 16; ++j) {
+      v[j] = sat(v[j]);
+      bmax = fmaxf(bmax, fabsf(v[j]));
     }
     bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
     bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
-    bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 4));
     const uint32_t c = e8m0_scale_code(bmax, cfg.scale_rule);
-    uint32_t q4 = 0, q8lo = 0, q8hi = 0;
+    uint32_t q4[2] = {0, 0}, q8[4] = {0, 0, 0, 0};
+    const float s4 = pow2_inv_e8m0(c);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      q4 |= e2m1x2(scalbnf(v[2 * i], 127 - (int)c), scalbnf(v[2 * i + 1], 127 - (int)c)) << (8 * i);
-      const uint32_t p = e4m3x2(scalbnf(v[2 * i], -e), scalbnf(v[2 * i + 1], -e));
-      if (i < 2) q8lo |= p << (16 * i); else q8hi |= p << (16 * (i - 2));
+    for (int j = 0; j < 8; ++j) {
+      q4[j >> 2] |= e2m1x2(v[2 * j] * s4, v[2 * j + 1] * s4) << (8 * (j & 3));
+      q8[j >> 1] |= e4m3x2(v[2 * j] * s8, v[2 * j + 1] * s8) << (16 * (j & 1));
     }
-    const int k1 = (int)(k >> 7), k2 = (int)(k >> 8);
-    uint8_t* xi = xi_base + (size_t)k2 * XI_BYTES;
-    uint8_t* xo = xo_base + (size_t)k1 * XO_BYTES;
-    *reinterpret_cast<uint32_t*>(xi + b_off(t, (uint32_t)(k & 255) >> 1)) = q4;
-    *reinterpret_cast<uint2*>(xo + b_off(t, (uint32_t)(k & 127))) = make_uint2(q8lo, q8hi);
-    if ((k & 63) == 0) xi[B4_BYTES + sf_off(t, (uint32_t)((k >> 6) & 3))] = (uint8_t)c;
+    if (!live) continue;
+    const uint32_t k = (uint32_t)b * 64 + l * 16;          // first element of this lane
+    uint8_t* xi = xi_base + (size_t)(k >> 8) * XI_BYTES;
+    uint8_t* xo = xo_base + (size_t)(k >> 7) * XO_BYTES;
+    *reinterpret_cast<uint2*>(xi + b_off(tk, (k & 255) >> 1)) = make_uint2(q4[0], q4[1]);
+    *reinterpret_cast<uint4*>(xo + b_off(tk, k & 127)) = make_uint4(q8[0], q8[1], q8[2], q8[3]);
+    if (l == 0) xi[B4_BYTES + sf_off(tk, (uint32_t)(b & 3))] = (uint8_t)c;
   }
 }
 
@@ -143,7 +178,11 @@ extern "C" sdq_status_t sdq_quantize_act(const void* X, int64_t M, int64_t K, in
   if (((uintptr_t)X & 15) || ((uintptr_t)xq_buf & 15) || (ldx % 8)) return SDQ_ERR_ALIGNMENT;
   const ActOffsets off = act_offsets(M, K);
   if (xq_bytes < off.total) return SDQ_ERR_BUFFER_TOO_SMALL;
-  quant_act_kernel<<<(unsigned)M, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, *cfg, (uint8_t*)xq_buf, off);
+  const int n_chunks = (int)((K / 64 + QA_CHUNK_QV - 1) / QA_CHUNK_QV);
+  float* partial = reinterpret_cast<float*>((uint8_t*)xq_buf + off.amax);
+  const dim3 grid((unsigned)((M + 7) / 8), (unsigned)n_chunks);
+  act_amax_kernel<<<grid, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, partial, n_chunks);
+  quant_act_kernel<<<grid, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, *cfg, (uint8_t*)xq_buf, off, partial, n_chunks);
   if (cudaGetLastError() != cudaSuccess) return SDQ_ERR_CUDA;
   out->dev = xq_buf;
   out->bytes = off.total;

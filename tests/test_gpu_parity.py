@@ -100,6 +100,33 @@ def test_one_hot_readback_pair_kernel():
     assert m.device_status() == 0
 
 
+@pytest.mark.parametrize("M,N,K,out_n", [(1, 512, 2048, 1), (16, 256, 4096, 1), (7, 1024, 1024, 2), (100, 256, 2816, 1),
+                                         (16, 256, 512, 0), (3, 128, 4096, 1)])
+def test_split_k_with_workspace(M, N, K, out_n):
+    """few tokens + workspace: K split over several thread blocks, partial tiles added in split order;
+    the result must meet the same criterion and be identical from call to call"""
+    m = sdq()
+    cfg = m.Config(out_n, m.GRAN_PAIR, 64, 0)
+    W = sdq_synth.make_weight(N, K, 200 + M)
+    X = sdq_synth.make_act(M, K, 200 + M)
+    p = m.sdq_decompose(W.cuda(), cfg)
+    xq = m.sdq_quantize_act(X.cuda(), cfg)
+    ws = m.make_workspace(M, N, K, cfg, "cuda")
+    assert ws is not None and m.workspace_size(M, N, K, cfg) == ws.numel()
+    y1 = m.sdq_linear(xq, p, f32=True, workspace=ws)
+    y2 = m.sdq_linear(xq, p, f32=True, workspace=ws)     # workspace is left ready for the next call
+    y16 = m.sdq_linear(xq, p, workspace=ws)
+    assert m.device_status() == 0
+    assert torch.equal(y1, y2)
+    assert torch.equal(y16, y1.to(torch.bfloat16))
+    yref = so.linear(so.quantize_act(sdq_synth.bf16_bits(X), ocfg(out_n)), so.decompose(sdq_synth.bf16_bits(W), ocfg(out_n)))
+    d, tol = y_close(y1.cpu().numpy(), yref)
+    assert (d <= tol).all(), (d.max(), (d / tol).max())
+    with pytest.raises(m.SdqError) as e:
+        m.sdq_linear(xq, p, workspace=ws[:256])
+    assert e.value.code == 5
+
+
 def test_one_hot_readback_through_the_tensor_core():
     """X = identity rows (1.0 is exact in both activation formats): Y^T must equal W_in + W_out exactly"""
     m = sdq()
