@@ -7,9 +7,10 @@
 //   2 x tcgen05.mma.sp kind::mxf8f6f4 per 128 K (1:8 / 2:8 E4M3 outliers embedded in 2:4 x E4M3 activations;
 //                                                the power-of-two row / token scales ride in as E8M0 factors)
 // both into ONE fp32 TMEM accumulator.  Persistent CTAs walk tiles of 128 rows x up to 256 tokens.
-// Warp roles: warp 0 = bulk-copy (TMA) producer, warp 1 = TMEM owner + MMA issuer (also moves metadata and
-// scale atoms smem -> TMEM with tcgen05.cp), warps 2..5 = epilogue (tcgen05.ld, convert, shared-memory
-// transpose, 16-byte row stores).  For few tokens the K range of a row tile is split over several CTAs; the
+// Warp roles: warps 0, 6, 7 = bulk-copy (TMA) producers for weights, activations and scale atoms (issuing a
+// bulk copy costs one thread ~50 ns, so the copies of a stage are spread over three threads), warp 1 = TMEM
+// owner + MMA issuer (also moves metadata and scale atoms smem -> TMEM with tcgen05.cp), warps 2..5 =
+// epilogue (tcgen05.ld, convert, shared-memory transpose, 16-byte row stores).  For few tokens the K range of a row tile is split over several CTAs; the
 // fp32 partial tiles go to a caller-provided workspace and the last CTA to arrive adds them in split order
 // (deterministic).  Every wait is bounded; a timeout sets a sticky flag.
 #include <cuda_bf16.h>
@@ -21,7 +22,7 @@
 
 namespace sdq {
 
-constexpr int LIN_THREADS = 192;
+constexpr int LIN_THREADS = 256;   // warps: 0 weight producer, 1 MMA issuer, 2..5 epilogue, 6 activation producer, 7 scale-atom producer
 constexpr int MAX_SLOTS = 16;
 constexpr int SL_A = 0;                        // WI record (A_in | E_in | SFA_in) or WO record (A_out | E_out)
 constexpr int SL_B = 10752;                    // B4 (256 K) or B8 (128 K) of n_tile tokens: n_tile * 128 B
@@ -51,10 +52,10 @@ __device__ __forceinline__ TileCoord tile_coord(const LinearParams& p, int tile,
   const int rest = tile / p.ksplit;
   c.rt = rest % RT;
   c.mtile = rest / RT;
-  c.i0 = (int)((int64_t)c.split * T2 / p.ksplit);
-  c.i1 = (int)((int64_t)(c.split + 1) * T2 / p.ksplit);
-  c.o0 = (int)((int64_t)c.split * T1 / p.ksplit);
-  c.o1 = (int)((int64_t)(c.split + 1) * T1 / p.ksplit);
+  c.i0 = c.split * T2 / p.ksplit;           // 32-bit: split < 32, T1 <= K/128
+  c.i1 = (c.split + 1) * T2 / p.ksplit;
+  c.o0 = c.split * T1 / p.ksplit;
+  c.o1 = (c.split + 1) * T1 / p.ksplit;
   return c;
 }
 
@@ -80,7 +81,7 @@ sdq_linear_kernel(const LinearParams p)
   const uint32_t sl_sf = SL_B + (uint32_t)n_tile * 128u;
 
   if (tid == 0) {
-    for (uint32_t s = 0; s < nslot; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
+    for (uint32_t s = 0; s < nslot; ++s) { ptx::mbar_init(&full[s], 3); ptx::mbar_init(&empty[s], 1); }
     ptx::mbar_init(acc_full, 1);
     ptx::mbar_init(acc_empty, 4);
     ptx::fence_barrier_init();
@@ -91,48 +92,61 @@ sdq_linear_kernel(const LinearParams p)
   ptx::tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  if (warp == 0) {
+  if (warp == 0 || warp >= 6) {
     if (lane == 0) {
-      // ---------------- producer: bulk copies, inlier stages of the tile first, then its outlier stages
+      // ---------------- producers: role 0 = weight records, role 1 = activation codes, role 2 = scale atoms.
+      // Each arrives once per stage on full[s] with the bytes it is about to copy.
+      const int role = warp == 0 ? 0 : (int)warp - 5;
       bool ok = true;
       uint32_t s = 0, wrapped = 0, ph = 0;   // ring slot, whether the ring has wrapped, phase parity of `empty`
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
         const TileCoord tc = tile_coord(p, tile, RT, T1, T2);
-        const int64_t m0 = (int64_t)tc.mtile * n_tile;
-        const int64_t mt = m0 / TILE_TOK;
-        const int have = (int)min((int64_t)n_atiles, p.aoff.MT - mt);        // activation tiles that exist
+        const int mt = tc.mtile * n_tile / TILE_TOK;
+        const int have = min(n_atiles, (int)p.aoff.MT - mt);                 // activation tiles that exist
         const uint32_t tok_bytes = (uint32_t)min(n_tile, TILE_TOK) * 128u;   // bytes per activation tile per stage
         const uint8_t* wi = p.w + p.poff.wi + ((size_t)tc.rt * T2 + tc.i0) * WI_BYTES;
         const uint8_t* wo = p.w + p.poff.wo + ((size_t)tc.rt * T1 + tc.o0) * WO_BYTES;
         const uint8_t* xi = p.x + p.aoff.xi + ((size_t)mt * T2 + tc.i0) * XI_BYTES;
         const uint8_t* xo = p.x + p.aoff.xo + ((size_t)mt * T1 + tc.o0) * XO_BYTES;
+        const size_t xi_tile = (size_t)T2 * XI_BYTES, xo_tile = (size_t)T1 * XO_BYTES;
         const int ni = tc.i1 - tc.i0, no = tc.o1 - tc.o0;
         for (int k = 0; k < ni + no; ++k) {
           if (wrapped && !(ok = ptx::mbar_wait(&empty[s], ph ^ 1))) break;
           uint8_t* st = sm + (size_t)s * slot_bytes;
-          if (k < ni) {
-            ptx::mbar_expect_tx(&full[s], WI_BYTES + (uint32_t)have * (tok_bytes + SF_ATOM_BYTES));
-            ptx::bulk_g2s(st + SL_A, wi, WI_BYTES, &full[s]);
-            for (int a = 0; a < have; ++a) {
-              const uint8_t* src = xi + (size_t)a * T2 * XI_BYTES;
-              ptx::bulk_g2s(st + SL_B + a * B4_BYTES, src, tok_bytes, &full[s]);
-              ptx::bulk_g2s(st + sl_sf + a * SF_ATOM_BYTES, src + B4_BYTES, SF_ATOM_BYTES, &full[s]);
+          const bool first_o = (k == ni);
+          if (role == 0) {
+            if (k < ni) {
+              ptx::mbar_expect_tx(&full[s], WI_BYTES);
+              ptx::bulk_g2s(st + SL_A, wi, WI_BYTES, &full[s]);
+              wi += WI_BYTES;
+            } else {
+              ptx::mbar_expect_tx(&full[s], WO_BYTES + (first_o ? SF_ATOM_BYTES : 0u));
+              ptx::bulk_g2s(st + SL_A, wo, WO_BYTES, &full[s]);
+              if (first_o) ptx::bulk_g2s(st + sl_sf, p.w + p.poff.sfa_out + (size_t)tc.rt * SF_ATOM_BYTES, SF_ATOM_BYTES, &full[s]);
+              wo += WO_BYTES;
             }
-            wi += WI_BYTES;
-            xi += XI_BYTES;
+          } else if (role == 1) {
+            ptx::mbar_expect_tx(&full[s], (uint32_t)have * tok_bytes);
+            if (k < ni) {
+              for (int a = 0; a < have; ++a) ptx::bulk_g2s(st + SL_B + a * B4_BYTES, xi + a * xi_tile, tok_bytes, &full[s]);
+              xi += XI_BYTES;
+            } else {
+              for (int a = 0; a < have; ++a) ptx::bulk_g2s(st + SL_B + a * B8_BYTES, xo + a * xo_tile, tok_bytes, &full[s]);
+              xo += XO_BYTES;
+            }
           } else {
-            const bool first = (k == ni);
-            ptx::mbar_expect_tx(&full[s], WO_BYTES + (uint32_t)have * tok_bytes + (first ? (uint32_t)(1 + have) * SF_ATOM_BYTES : 0u));
-            ptx::bulk_g2s(st + SL_A, wo, WO_BYTES, &full[s]);
-            for (int a = 0; a < have; ++a) ptx::bulk_g2s(st + SL_B + a * B8_BYTES, xo + (size_t)a * T1 * XO_BYTES, tok_bytes, &full[s]);
-            if (first) {
-              ptx::bulk_g2s(st + sl_sf, p.w + p.poff.sfa_out + (size_t)tc.rt * SF_ATOM_BYTES, SF_ATOM_BYTES, &full[s]);
+            if (k < ni) {
+              ptx::mbar_expect_tx(&full[s], (uint32_t)have * SF_ATOM_BYTES);
+              for (int a = 0; a < have; ++a) ptx::bulk_g2s(st + sl_sf + a * SF_ATOM_BYTES, xi + a * xi_tile + B4_BYTES, SF_ATOM_BYTES, &full[s]);
+              xi += XI_BYTES;
+            } else if (first_o) {
+              ptx::mbar_expect_tx(&full[s], (uint32_t)have * SF_ATOM_BYTES);
               for (int a = 0; a < have; ++a)
-                ptx::bulk_g2s(st + sl_sf + (1 + a) * SF_ATOM_BYTES, p.x + p.aoff.sfb_out + (size_t)(mt + a) * SF_ATOM_BYTES,
-                              SF_ATOM_BYTES, &full[s]);
+                ptx::bulk_g2s(st + sl_sf + (1 + a) * SF_ATOM_BYTES, p.x + p.aoff.sfb_out + (size_t)(mt + a) * SF_ATOM_BYTES, SF_ATOM_BYTES,
+                              &full[s]);
+            } else {
+              ptx::mbar_arrive(&full[s]);
             }
-            wo += WO_BYTES;
-            xo += XO_BYTES;
           }
           if (++s == nslot) { s = 0; wrapped = 1; ph ^= 1; }
         }
@@ -205,7 +219,7 @@ sdq_linear_kernel(const LinearParams p)
       }
       if (!ok) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
     }
-  } else {
+  } else if (warp >= 2 && warp <= 5) {
     // ---------------- epilogue: warp w owns TMEM lanes 32*(w%4) .. +31 (weight rows), columns = tokens
     const uint32_t q = warp & 3;
     const uint32_t et = (warp - 2) * 32 + lane;     // 0..127 among the epilogue threads
