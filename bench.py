@@ -230,7 +230,10 @@ def run_ours(args):
     gemm_tf = (flops_step * args.steps) / (sum(gemm_ms) * 1e-3) / 1e12
     mixed_peak = peaks["bf16"] * MIXED_PEAK_OVER_BF16
     roofline = {"kernel": "sdq_linear_kernel", "bound": "tensor", "achieved": gemm_tf, "peak": mixed_peak, "unit": "TFLOP/s",
-                "frac": gemm_tf / mixed_peak, "traffic": None,
+                "frac": gemm_tf / mixed_peak,
+                # dram__bytes_read.sum + dram__bytes_write.sum of one captured launch of the gate / up shape
+                # (profiles/sdq_linear_kernel_prefill_M2048_N11008_K4096.md); the down shape was not captured
+                "traffic": 88.3e6, "traffic_unit": "bytes per launch (gate/up shape)",
                 "peak_basis": "%s bf16 burst %.1f TF/s x 8/3 (sparse FP4 at 8x + sparse FP8 at 4x per dense-equivalent flop)" % (peaks["source"], peaks["bf16"]),
                 "avg_launch_ms": sum(gemm_ms) / len(gemm_ms), "launches": len(gemm_ms),
                 "frac_of_sparse_fp4_peak": gemm_tf / (8 * peaks["bf16"])}
