@@ -160,6 +160,25 @@ sdq_status_t sdq_linear_ws(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y_b
 sdq_status_t sdq_linear_f32_ws(const sdq_act_t* Xq, const sdq_packed_t* P, float* Y_f32, int64_t ldy, void* ws, size_t ws_bytes,
                                void* stream);
 
+/* Built-in scratch variant of sdq_linear_ws (the paper has no counterpart: this is a packaging choice of the
+ * library, not part of the method).
+ *   For callers that hold nothing but their input and output pointers and cannot obtain device memory: a
+ *   plug-in running inside someone else's inference server whose memory pool was handed out at start-up, a
+ *   host thread on a latency path where a device allocation (which may synchronise the whole device) is not
+ *   acceptable, or any caller that must not call cudaMalloc.  The split-K scratch is a fixed array of
+ *   SDQ_STATIC_WS_BYTES inside the library's device image; every GPU that loads the library carries it until
+ *   the process exits.  The call allocates and frees nothing.
+ *   Same arguments, result and errors as sdq_linear; the result equals sdq_linear_ws with a caller workspace
+ *   bit for bit.  Shapes whose scratch need (sdq_workspace_size) exceeds SDQ_STATIC_WS_BYTES are refused with
+ *   SDQ_ERR_BUFFER_TOO_SMALL; shapes that need no scratch run as sdq_linear.
+ *   The first call on each device looks up the device address of the array (cudaGetSymbolAddress with that
+ *   device current); make that first call before any stream capture begins.  All calls on a device share the
+ *   one array and it keeps the previous call's contents (the counters are cleared on the stream at the start of
+ *   every call): two calls that can overlap on the GPU (different streams) race on it -- serialise them or use
+ *   sdq_linear_ws with separate workspaces. */
+#define SDQ_STATIC_WS_BYTES (4u << 20)
+sdq_status_t sdq_linear_noalloc(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y_bf16, int64_t ldy, void* stream);
+
 /* Synchronises `stream` and returns the sticky device-side status (SDQ_OK or SDQ_ERR_TIMEOUT when a
  * bounded wait inside a kernel gave up), clearing it. */
 sdq_status_t sdq_device_status(void* stream);

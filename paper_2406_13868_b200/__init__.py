@@ -55,7 +55,7 @@ class _ActCanon(ctypes.Structure):
 
 
 EXPORTS = ["sdq_packed_size", "sdq_decompose", "sdq_packed_export", "sdq_act_size", "sdq_quantize_act", "sdq_act_export",
-           "sdq_linear", "sdq_linear_f32", "sdq_workspace_size", "sdq_workspace_init", "sdq_linear_ws", "sdq_linear_f32_ws",
+           "sdq_linear", "sdq_linear_f32", "sdq_workspace_size", "sdq_workspace_init", "sdq_linear_ws", "sdq_linear_f32_ws", "sdq_linear_noalloc",
            "sdq_device_status", "sdq_status_string"]
 
 _lib = None
@@ -82,6 +82,7 @@ def lib() -> ctypes.CDLL:
         L.sdq_workspace_init.argtypes = [vp, sz, vp]
         L.sdq_linear_ws.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_Packed), vp, i64, vp, sz, vp]
         L.sdq_linear_f32_ws.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_Packed), vp, i64, vp, sz, vp]
+        L.sdq_linear_noalloc.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_Packed), vp, i64, vp]
         L.sdq_device_status.argtypes = [vp]
         L.sdq_status_string.argtypes = [ctypes.c_int]
         L.sdq_status_string.restype = ctypes.c_char_p
@@ -197,6 +198,18 @@ def sdq_linear(xq: QuantAct, p: PackedWeight, out: torch.Tensor | None = None, f
         fn = lib().sdq_linear_f32_ws if f32 else lib().sdq_linear_ws
         _check(fn(ctypes.byref(xq.desc), ctypes.byref(p.desc), out.data_ptr(), out.stride(0), workspace.data_ptr(),
                   workspace.numel(), _stream()), "sdq_linear_ws")
+    return out
+
+
+STATIC_WS_BYTES = 4 << 20
+
+
+def sdq_linear_noalloc(xq: QuantAct, p: PackedWeight, out: torch.Tensor) -> torch.Tensor:
+    """sdq_linear for callers that may not allocate device memory: the split-K scratch is a fixed array inside the
+    library (STATIC_WS_BYTES); `out` must be supplied.  Calls that can overlap on the GPU must not share it."""
+    assert out.dtype == torch.bfloat16 and out.shape == (xq.M, p.N) and out.stride(1) == 1
+    _check(lib().sdq_linear_noalloc(ctypes.byref(xq.desc), ctypes.byref(p.desc), out.data_ptr(), out.stride(0), _stream()),
+           "sdq_linear_noalloc")
     return out
 
 

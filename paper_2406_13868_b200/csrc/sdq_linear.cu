@@ -430,3 +430,41 @@ extern "C" sdq_status_t sdq_linear_ws(const sdq_act_t* Xq, const sdq_packed_t* P
 extern "C" sdq_status_t sdq_linear_f32_ws(const sdq_act_t* Xq, const sdq_packed_t* P, float* Y, int64_t ldy, void* ws, size_t ws_bytes,
                                           void* stream)
 { return launch_linear(Xq, P, (void*)Y, ldy, ws, ws_bytes, stream, true); }
+
+// ---------------------------------------------------------------------------------------------------------
+// Allocation-free variant of sdq_linear_ws (see include/sdq.h).  The split-K scratch lives in this library's
+// own device image instead of a caller buffer.
+namespace sdq {
+static __device__ __align__(256) unsigned char g_static_ws[SDQ_STATIC_WS_BYTES];
+}
+
+// Device address of the built-in scratch for the current device.  `g_static_ws` in host code is only a handle
+// for the symbol, not an address a kernel could use, so the address is asked from the runtime, once per
+// device and with that device current.
+static void* static_ws_address() {
+  static void* cache[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!cache[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress((void**)&ptr, sdq::g_static_ws) != cudaSuccess) return nullptr;
+    cache[dev] = ptr;
+  }
+  return cache[dev];
+}
+
+extern "C" sdq_status_t sdq_linear_noalloc(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y, int64_t ldy, void* stream)
+{
+  if (!Xq || !P) return SDQ_ERR_INVALID_ARG;
+  size_t need = 0;
+  const sdq_status_t st = sdq_workspace_size(Xq->M, P->N, P->K, &P->cfg, &need);
+  if (st != SDQ_OK) return st;
+  if (need == 0) return launch_linear(Xq, P, Y, ldy, nullptr, 0, stream, false);   // this shape uses no scratch
+  if (need > (size_t)SDQ_STATIC_WS_BYTES) return SDQ_ERR_BUFFER_TOO_SMALL;
+  void* ws = static_ws_address();
+  if (!ws) return SDQ_ERR_CUDA;
+  // the array keeps whatever the previous call left: the arrival counters must start at zero
+  const size_t counter_bytes = ((size_t)(P->N / TILE_ROWS) * 4 + 255) & ~(size_t)255;
+  if (cudaMemsetAsync(ws, 0, counter_bytes, (cudaStream_t)stream) != cudaSuccess) return SDQ_ERR_CUDA;
+  return launch_linear(Xq, P, Y, ldy, ws, need, stream, false);
+}
