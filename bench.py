@@ -148,6 +148,17 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def aggregate_over_ranks(ms_local: float, units_per_rank: float, world: int, device="cpu"):
+    """Whole-job throughput under weak scaling: every rank processed `units_per_rank` in `ms_local`; the job took
+    the MAX over ranks (all-reduce), and processed world * units_per_rank.  Returns (units per second, max ms)."""
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item())
+    return world * units_per_rank / (ms * 1e-3), ms
+
+
 # ----------------------------------------------------------------------------------------------- CUDA arm
 def run_ours(args):
     import paper_2406_13868_b200 as sdq
@@ -218,12 +229,9 @@ def run_ours(args):
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
     assert sdq.device_status() == 0, "device-side timeout flag set"
-    t_ms = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        import torch.distributed as dist
-        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-    ms_step = float(t_ms.item()) / args.steps
-    value = world * flops_step / (ms_step * 1e-3) / 1e12
+    flops_per_s, ms_max = aggregate_over_ranks(ms_total, flops_step * args.steps, world, dev)
+    ms_step = ms_max / args.steps
+    value = flops_per_s / 1e12
 
     gemm_ms = [a.elapsed_time(b) for k, a, b in ev if k == "gemm"]
     quant_ms = [a.elapsed_time(b) for k, a, b in ev if k == "quant"]

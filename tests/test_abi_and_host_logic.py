@@ -1,0 +1,94 @@
+"""CPU-side checks: the C-ABI library loads and exports every symbol include/sdq.h declares, host-only entry points
+validate their arguments, and the multi-rank aggregation of bench.py works over gloo with two ranks."""
+import ctypes
+import os
+import re
+import subprocess
+import sys
+
+import pytest
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def m():
+    import paper_2406_13868_b200 as mod
+    mod.build()
+    return mod
+
+
+def declared_symbols():
+    src = open(os.path.join(ROOT, "include", "sdq.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(sdq_[a-z0-9_]+)\s*\(", src)))
+
+
+def test_library_exports_every_declared_symbol(m):
+    names = declared_symbols()
+    assert "sdq_decompose" in names and "sdq_quantize_act" in names and "sdq_linear" in names
+    L = m.lib()
+    for n in names:
+        assert hasattr(L, n), n
+    assert sorted(m.EXPORTS) == names
+
+
+def test_size_queries_and_argument_errors_without_a_gpu(m):
+    L = m.lib()
+    cfg = m.Config()
+    b, a = ctypes.c_size_t(), ctypes.c_size_t()
+    assert L.sdq_packed_size(4096, 4096, ctypes.byref(cfg), ctypes.byref(b), ctypes.byref(a)) == 0
+    assert a.value == 4096 * 4096 // 2 + 4096 * 4      # 4.0 bits per weight + one fp32 scale per row
+    assert b.value >= a.value
+    assert L.sdq_packed_size(4096, 4000, ctypes.byref(cfg), ctypes.byref(b), ctypes.byref(a)) == 2   # K % 256
+    assert L.sdq_packed_size(100, 4096, ctypes.byref(cfg), ctypes.byref(b), ctypes.byref(a)) == 2    # N % 128
+    bad = m.Config(3, 0, 64, 0)
+    assert L.sdq_packed_size(128, 256, ctypes.byref(bad), ctypes.byref(b), ctypes.byref(a)) == 1
+    elem = m.Config(1, m.GRAN_ELEM, 32, 0)
+    assert L.sdq_packed_size(128, 256, ctypes.byref(elem), ctypes.byref(b), ctypes.byref(a)) == 4
+    assert L.sdq_act_size(1, 4096, ctypes.byref(cfg), ctypes.byref(b)) == 0 and b.value > 4096 * 3 // 2
+    assert L.sdq_act_size(0, 4096, ctypes.byref(cfg), ctypes.byref(b)) == 2
+    # null pointers are rejected before anything is launched
+    assert L.sdq_decompose(None, 128, 256, 256, ctypes.byref(cfg), None, 0, None, None) == 1
+    assert L.sdq_linear(None, None, None, 0, None) == 1
+    assert L.sdq_linear_noalloc(None, None, None, 0, None) == 1
+    assert L.sdq_status_string(8) == b"device-side bounded wait timed out"
+    assert L.sdq_status_string(0) == b"ok"
+
+
+def test_compute_calls_refuse_cpu_tensors(m):
+    W = torch.zeros((128, 256), dtype=torch.bfloat16)
+    with pytest.raises(ValueError):
+        m.sdq_decompose(W)
+    with pytest.raises(ValueError):
+        m.sdq_quantize_act(W)
+
+
+_WORKER = r"""
+import os, sys, torch, torch.distributed as dist
+sys.path.insert(0, sys.argv[1])
+import bench
+rank, world = int(sys.argv[2]), int(sys.argv[3])
+os.environ["MASTER_ADDR"] = "127.0.0.1"; os.environ["MASTER_PORT"] = sys.argv[4]
+dist.init_process_group("gloo", rank=rank, world_size=world)
+ms_local = 10.0 if rank == 0 else 12.5          # the slower rank sets the job time
+rate, ms = bench.aggregate_over_ranks(ms_local, 1000.0, world)
+assert ms == 12.5, ms
+assert abs(rate - world * 1000.0 / 12.5e-3) < 1e-6, rate
+dist.barrier()
+dist.destroy_process_group()
+print("ok", rank)
+"""
+
+
+def test_weak_scaling_aggregation_two_ranks_gloo(tmp_path):
+    script = tmp_path / "worker.py"
+    script.write_text(_WORKER)
+    port = str(29500 + os.getpid() % 2000)
+    procs = [subprocess.Popen([sys.executable, str(script), ROOT, str(r), "2", port], stdout=subprocess.PIPE, stderr=subprocess.STDOUT)
+             for r in range(2)]
+    outs = [p.communicate(timeout=120)[0].decode() for p in procs]
+    for p, o in zip(procs, outs):
+        assert p.returncode == 0, o
+        assert "ok" in o
