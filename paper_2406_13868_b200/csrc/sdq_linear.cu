@@ -26,17 +26,14 @@ constexpr int LIN_THREADS = 256;   // warps: 0 weight producer, 1 MMA issuer, 2.
 constexpr int MAX_SLOTS = 16;
 constexpr int SL_A = 0;                        // WI record (A_in | E_in | SFA_in) or WO record (A_out | E_out)
 constexpr int SL_B = 10752;                    // B4 (256 K) or B8 (128 K) of n_tile tokens: n_tile * 128 B
-constexpr int RING_BYTES = 225280;             // ring of nslot slots of slot_bytes each
-constexpr int SM_STG = RING_BYTES;             // epilogue transpose buffer: 16 tokens x 128 features bf16
-constexpr int SM_BARS = SM_STG + 4096;
-constexpr int LIN_SMEM = SM_BARS + 320 + 128;  // + barriers + alignment slack
+constexpr int RING_BYTES = 225280;             // largest ring: nslot slots of slot_bytes each
+constexpr int SM_TAIL = 4096 + 320 + 128;      // epilogue transpose buffer (16 tokens x 128 features bf16) + barriers + slack
+constexpr int LIN_SMEM_MAX = RING_BYTES + SM_TAIL;
 
-// TMEM columns
-constexpr uint32_t TM_D = 0;          // accumulator: up to 256 columns (tokens)
-constexpr uint32_t TM_I = 256;        // 2 buffers x 16 columns: E_in 4 | SFA_in 4 | SFB_in 8
-constexpr uint32_t TM_EO = 288;       // 2 buffers x 4 columns: E_out
-constexpr uint32_t TM_SFA_OUT = 296;  // 4 columns
-constexpr uint32_t TM_SFB_OUT = 300;  // 8 columns
+// TMEM columns: accumulator at 0 (n_tile columns, tokens), then 52 columns of metadata / scales at `meta_col`:
+//   +0  2 buffers x 16: E_in 4 | SFA_in 4 | SFB_in 8      +32 2 buffers x 4: E_out      +40 SFA_out 4      +44 SFB_out 8
+constexpr uint32_t TM_D = 0;
+constexpr uint32_t TM_META_COLS = 52;
 
 // slot = | A record 10752 | B n_tile*128 | scale atoms 1536 |  (inlier: SFB_in x n_atiles; first outlier stage:
 // SFA_out | SFB_out x n_atiles)
@@ -66,6 +63,8 @@ sdq_linear_kernel(const LinearParams p)
   extern __shared__ uint8_t smem_raw[];
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint8_t* sm = smem_raw + ((128 - (ptx::smem_u32(smem_raw) & 127)) & 127);
+  const uint32_t SM_STG = (uint32_t)p.ring_bytes, SM_BARS = SM_STG + 4096;
+  const uint32_t TM_I = (uint32_t)p.meta_col, TM_EO = TM_I + 32, TM_SFA_OUT = TM_I + 40, TM_SFB_OUT = TM_I + 44;
   uint64_t* full = reinterpret_cast<uint64_t*>(sm + SM_BARS);
   uint64_t* empty = full + MAX_SLOTS;
   uint64_t* acc_full = empty + MAX_SLOTS;
@@ -80,13 +79,16 @@ sdq_linear_kernel(const LinearParams p)
   const uint32_t nslot = (uint32_t)p.nslot, slot_bytes = (uint32_t)p.slot_bytes;
   const uint32_t sl_sf = SL_B + (uint32_t)n_tile * 128u;
 
+  // the coordinates of the first tile are worked out by every thread while the barriers and TMEM are being set up
+  // (a lone thread needs ~0.5 us for the integer divisions, which would otherwise delay the first copies)
+  const TileCoord first_tc = tile_coord(p, (int)blockIdx.x, RT, T1, T2);
   if (tid == 0) {
     for (uint32_t s = 0; s < nslot; ++s) { ptx::mbar_init(&full[s], 3); ptx::mbar_init(&empty[s], 1); }
     ptx::mbar_init(acc_full, 1);
     ptx::mbar_init(acc_empty, 4);
     ptx::fence_barrier_init();
   }
-  if (warp == 1) ptx::tmem_alloc(tmem_slot, 512);
+  if (warp == 1) ptx::tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
@@ -100,7 +102,7 @@ sdq_linear_kernel(const LinearParams p)
       bool ok = true;
       uint32_t s = 0, wrapped = 0, ph = 0;   // ring slot, whether the ring has wrapped, phase parity of `empty`
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-        const TileCoord tc = tile_coord(p, tile, RT, T1, T2);
+        const TileCoord tc = (tile == (int)blockIdx.x) ? first_tc : tile_coord(p, tile, RT, T1, T2);
         const int mt = tc.mtile * n_tile / TILE_TOK;
         const int have = min(n_atiles, (int)p.aoff.MT - mt);                 // activation tiles that exist
         const uint32_t tok_bytes = (uint32_t)min(n_tile, TILE_TOK) * 128u;   // bytes per activation tile per stage
@@ -111,7 +113,7 @@ sdq_linear_kernel(const LinearParams p)
         const size_t xi_tile = (size_t)T2 * XI_BYTES, xo_tile = (size_t)T1 * XO_BYTES;
         const int ni = tc.i1 - tc.i0, no = tc.o1 - tc.o0;
         for (int k = 0; k < ni + no; ++k) {
-          if (wrapped && !(ok = ptx::mbar_wait(&empty[s], ph ^ 1))) break;
+          if (wrapped && p.release && !(ok = ptx::mbar_wait(&empty[s], ph ^ 1))) break;
           uint8_t* st = sm + (size_t)s * slot_bytes;
           const bool first_o = (k == ni);
           if (role == 0) {
@@ -172,7 +174,7 @@ sdq_linear_kernel(const LinearParams p)
       const uint64_t d_sf2 = ptx::smem_desc(smb + sl_sf + 2 * SF_ATOM_BYTES, 0, 128);
       const uint32_t slot16 = slot_bytes >> 4;
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
-        const TileCoord tc = tile_coord(p, tile, RT, T1, T2);
+        const TileCoord tc = (tcount == 0) ? first_tc : tile_coord(p, tile, RT, T1, T2);
         const int ni = tc.i1 - tc.i0, no = tc.o1 - tc.o0;
         if (tcount > 0) {   // the epilogue must have drained the accumulator of the previous tile
           ok = ptx::mbar_wait(acc_empty, (tcount - 1) & 1);
@@ -211,7 +213,7 @@ sdq_linear_kernel(const LinearParams p)
                              tmem + TM_SFB_OUT, 1u);
           }
           acc = 1;
-          ptx::tc_commit(&empty[s]);
+          if (p.release) ptx::tc_commit(&empty[s]);   // ring slots are reused only when a CTA runs more stages than slots
           s = sn;
           if (sn == 0) ph ^= 1;
         }
@@ -226,7 +228,7 @@ sdq_linear_kernel(const LinearParams p)
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
-      const TileCoord tc = tile_coord(p, tile, RT, T1, T2);
+      const TileCoord tc = (tcount == 0) ? first_tc : tile_coord(p, tile, RT, T1, T2);
       const int64_t m0 = (int64_t)tc.mtile * n_tile;
       const int n_valid = (int)min((int64_t)n_tile, p.M - m0);
       ok = ptx::mbar_wait(acc_full, tcount & 1);
@@ -234,8 +236,10 @@ sdq_linear_kernel(const LinearParams p)
       if (!ok) break;
       const int64_t n0 = (int64_t)tc.rt * TILE_ROWS;
       // split-K: this CTA's fp32 partial tile [token][128 rows] in the workspace
-      float* part = p.ksplit > 1 ? p.ws_partial + ((size_t)(tc.rt * p.n_mtiles + tc.mtile) * p.ksplit + tc.split) * (size_t)n_tile * TILE_ROWS
-                                 : nullptr;
+      float* part = nullptr;
+      if (p.cluster_ks > 1) part = reinterpret_cast<float*>(sm);   // the ring is idle once the accumulator is complete
+      else if (p.ksplit > 1)
+        part = p.ws_partial + ((size_t)(tc.rt * p.n_mtiles + tc.mtile) * p.ksplit + tc.split) * (size_t)n_tile * TILE_ROWS;
 #pragma unroll 1
       for (int c0 = 0; c0 < n_tile; c0 += 16) {
         uint32_t v[16];
@@ -276,7 +280,7 @@ sdq_linear_kernel(const LinearParams p)
           ptx::named_bar_sync(1, 128);   // the buffer is rewritten by the next chunk
         }
       }
-      if (part) {
+      if (part && p.cluster_ks <= 1) {
         // the last CTA of this (row tile, token tile) to finish adds the partial tiles in split order
         __threadfence();
         ptx::named_bar_sync(1, 128);
@@ -315,9 +319,33 @@ sdq_linear_kernel(const LinearParams p)
     }
     if (!ok && lane == 0) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
   }
+  if (p.cluster_ks > 1) {
+    // ---------------- cluster split-K: one tile per CTA; CTA r adds rows [r*128/ks, (r+1)*128/ks) of all members
+    ptx::cluster_sync();                         // every member's partial tile is in its shared memory
+    if (warp >= 2 && warp <= 5) {
+      const uint32_t et = (warp - 2) * 32 + lane;
+      const uint32_t ks = (uint32_t)p.cluster_ks, rank = ptx::cluster_ctarank();
+      const uint32_t rows_per = TILE_ROWS / ks;
+      const int n_valid = (int)min((int64_t)n_tile, p.M - (int64_t)first_tc.mtile * n_tile);
+      const int64_t m0 = (int64_t)first_tc.mtile * n_tile, n0 = (int64_t)first_tc.rt * TILE_ROWS;
+      const uint32_t local = ptx::smem_u32(sm);
+      for (uint32_t idx = et; idx < rows_per * (uint32_t)n_valid; idx += 128) {
+        const uint32_t row = rank * rows_per + idx % rows_per, tok = idx / rows_per;
+        float v[8];
+#pragma unroll
+        for (uint32_t sp = 0; sp < 8; ++sp) v[sp] = sp < ks ? ptx::ld_dsmem_f32(local + (tok * TILE_ROWS + row) * 4, sp) : 0.0f;
+        float acc = 0.0f;
+#pragma unroll
+        for (uint32_t sp = 0; sp < 8; ++sp) acc += v[sp];          // rank order; absent members contribute +0
+        if (F32_OUT) reinterpret_cast<float*>(p.Y)[(m0 + tok) * p.ldy + n0 + row] = acc;
+        else reinterpret_cast<__nv_bfloat16*>(p.Y)[(m0 + tok) * p.ldy + n0 + row] = __float2bfloat16_rn(acc);
+      }
+    }
+    ptx::cluster_sync();                         // nobody leaves while its shared memory may still be read
+  }
   ptx::tc_fence_before();
   __syncthreads();
-  if (warp == 1) ptx::tmem_dealloc(tmem, 512);
+  if (warp == 1) ptx::tmem_dealloc(tmem, (uint32_t)p.tmem_cols);
 }
 
 }  // namespace sdq
@@ -338,7 +366,8 @@ static int sm_count_cached() {
 static int choose_ksplit(int64_t M, int64_t N, int64_t K, int sm_count) {
   if (M > 128 || sm_count <= 0) return 1;
   const int RT = (int)(N / TILE_ROWS), T2 = (int)(K / K2);
-  int ks = sm_count / RT;
+  // few tokens: short K chains and two small CTAs per SM hide the per-CTA latencies best
+  int ks = (M <= 32 ? 2 * sm_count : sm_count) / RT;
   if (ks > T2) ks = T2;
   if (ks > 32) ks = 32;
   return ks < 1 ? 1 : ks;
@@ -366,8 +395,8 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   if (((uintptr_t)Y & 15) || (ldy % 8) || ((uintptr_t)ws & 15)) return SDQ_ERR_ALIGNMENT;
   static bool attr_set[2] = {false, false};
   if (!attr_set[f32]) {
-    cudaError_t e = f32 ? cudaFuncSetAttribute(sdq_linear_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM)
-                        : cudaFuncSetAttribute(sdq_linear_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM);
+    cudaError_t e = f32 ? cudaFuncSetAttribute(sdq_linear_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX)
+                        : cudaFuncSetAttribute(sdq_linear_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX);
     if (e != cudaSuccess) return SDQ_ERR_CUDA;
     attr_set[f32] = true;
   }
@@ -384,11 +413,21 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   p.n_tile = n_tile_for(M);
   p.n_mtiles = (int)((M + p.n_tile - 1) / p.n_tile);
   p.slot_bytes = slot_bytes_for(p.n_tile);
-  p.nslot = RING_BYTES / p.slot_bytes;
-  if (p.nslot > MAX_SLOTS) p.nslot = MAX_SLOTS;
   p.ksplit = 1;
+  p.cluster_ks = 1;
   p.ws_counter = nullptr;
   p.ws_partial = nullptr;
+  if (!ws && M <= 32) {
+    // cluster split-K: power-of-two cluster of up to 8 CTAs per row tile, about two CTAs per SM in total
+    const int RT = (int)(P->N / TILE_ROWS), T2c = (int)(P->K / K2);
+    int ks = 8;
+    while (ks > 1 && (ks * RT > 2 * sm_count || ks > T2c)) ks >>= 1;
+    const int T1c = p.out_n ? (int)(P->K / K1) : 0;
+    const int stages = (T2c + ks - 1) / ks + (T1c + ks - 1) / ks;
+    int max_slots_c = RING_BYTES / p.slot_bytes;
+    if (max_slots_c > MAX_SLOTS) max_slots_c = MAX_SLOTS;
+    if (ks > 1 && stages <= max_slots_c) { p.ksplit = ks; p.cluster_ks = ks; }
+  }
   if (ws) {
     const int ks = choose_ksplit(M, P->N, P->K, sm_count);
     size_t need = 0;
@@ -404,10 +443,41 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   p.Y = Y; p.ldy = ldy;
   p.flags = device_flags();
   if (!p.flags) return SDQ_ERR_CUDA;
-  dim3 grid((unsigned)(p.total_tiles < sm_count ? p.total_tiles : sm_count));
-  if (f32) sdq_linear_kernel<true><<<grid, LIN_THREADS, LIN_SMEM, (cudaStream_t)stream>>>(p);
-  else sdq_linear_kernel<false><<<grid, LIN_THREADS, LIN_SMEM, (cudaStream_t)stream>>>(p);
-  return cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
+  // ring geometry: a CTA that runs a single tile with no more stages than fit never reuses a slot, needs only as
+  // much shared memory as its stages take (so that small CTAs share an SM) and skips the slot-release traffic
+  const int T1 = p.out_n ? (int)(P->K / K1) : 0, T2 = (int)(P->K / K2);
+  const int stages_per_tile = (T2 + p.ksplit - 1) / p.ksplit + (T1 + p.ksplit - 1) / p.ksplit;
+  int max_slots = RING_BYTES / p.slot_bytes;
+  if (max_slots > MAX_SLOTS) max_slots = MAX_SLOTS;
+  int grid_x;
+  if (p.total_tiles <= 2 * sm_count && stages_per_tile <= max_slots && p.n_tile <= 32) {
+    grid_x = p.total_tiles;
+    p.nslot = stages_per_tile;
+    p.release = 0;
+  } else {
+    grid_x = p.total_tiles < sm_count ? p.total_tiles : sm_count;
+    p.nslot = max_slots;
+    p.release = 1;
+  }
+  p.ring_bytes = p.nslot * p.slot_bytes;
+  p.meta_col = p.n_tile < 32 ? 32 : p.n_tile;
+  int cols = p.meta_col + (int)TM_META_COLS;
+  p.tmem_cols = cols <= 128 ? 128 : (cols <= 256 ? 256 : 512);
+  const int smem = p.ring_bytes + SM_TAIL;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3((unsigned)grid_x);
+  lc.blockDim = dim3(LIN_THREADS);
+  lc.dynamicSmemBytes = (size_t)smem;
+  lc.stream = (cudaStream_t)stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)p.cluster_ks;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  lc.attrs = attr;
+  lc.numAttrs = p.cluster_ks > 1 ? 1 : 0;
+  const cudaError_t le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false>, p);
+  return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
 }
 
 extern "C" sdq_status_t sdq_linear(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y, int64_t ldy, void* stream)

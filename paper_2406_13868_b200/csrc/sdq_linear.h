@@ -19,7 +19,12 @@ struct LinearParams {
   int n_mtiles;          // ceil(M / n_tile)
   int total_tiles;       // (N / 128) * n_mtiles * ksplit
   int nslot, slot_bytes; // shared-memory ring geometry (depends on n_tile)
+  int ring_bytes;        // nslot * slot_bytes; the transpose buffer and the barriers follow
+  int release;           // 1: ring slots are reused (producer waits on `empty`, MMA issuer commits to it)
+  int tmem_cols;         // TMEM columns to allocate (128, 256 or 512)
+  int meta_col;          // first TMEM column of the metadata / scale buffers
   int ksplit;            // CTAs sharing the K range of one row tile (1 = no split)
+  int cluster_ks;        // > 1: those CTAs form a cluster and reduce through distributed shared memory
   uint32_t* ws_counter;  // split-K workspace: arrival counters [row tile], zero between calls
   float* ws_partial;     // split-K workspace: fp32 partial tiles [row tile][split][token][128 rows]
   void* Y;

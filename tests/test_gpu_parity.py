@@ -127,6 +127,28 @@ def test_split_k_with_workspace(M, N, K, out_n):
     assert e.value.code == 5
 
 
+@pytest.mark.parametrize("M,N,K,out_n", [(1, 512, 4096, 1), (16, 1024, 4096, 1), (32, 256, 2048, 2), (5, 4096, 1024, 1),
+                                         (16, 256, 1024, 0), (2, 128, 11008, 1)])
+def test_cluster_split_k_few_tokens(M, N, K, out_n):
+    """up to 32 tokens without a workspace: the thread blocks of a row tile form a cluster and add their partial
+    tiles through distributed shared memory in rank order -- same criterion, identical from call to call"""
+    m = sdq()
+    cfg = m.Config(out_n, m.GRAN_PAIR, 64, 0)
+    W = sdq_synth.make_weight(N, K, 300 + M)
+    X = sdq_synth.make_act(M, K, 300 + M)
+    p = m.sdq_decompose(W.cuda(), cfg)
+    xq = m.sdq_quantize_act(X.cuda(), cfg)
+    y1 = m.sdq_linear(xq, p, f32=True)
+    y2 = m.sdq_linear(xq, p, f32=True)
+    y16 = m.sdq_linear(xq, p)
+    assert m.device_status() == 0
+    assert torch.equal(y1, y2)
+    assert torch.equal(y16, y1.to(torch.bfloat16))
+    yref = so.linear(so.quantize_act(sdq_synth.bf16_bits(X), ocfg(out_n)), so.decompose(sdq_synth.bf16_bits(W), ocfg(out_n)))
+    d, tol = y_close(y1.cpu().numpy(), yref)
+    assert (d <= tol).all(), (d.max(), (d / tol).max())
+
+
 def test_one_hot_readback_through_the_tensor_core():
     """X = identity rows (1.0 is exact in both activation formats): Y^T must equal W_in + W_out exactly"""
     m = sdq()
