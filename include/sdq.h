@@ -47,7 +47,8 @@ enum { SDQ_SCALE_OCP_FLOOR = 0, SDQ_SCALE_CEIL_NOSAT = 1 }; /* E8M0 Q-Vector sca
  *   in_gran    how the remaining values are pruned to 50% (Stage 1, magnitude metric):
  *              SDQ_GRAN_PAIR keeps the 2 adjacent pairs (of 4) with the largest |a|+|b| in every 8
  *              (the pattern the sparse FP4 tensor core consumes); SDQ_GRAN_ELEM keeps the 2 largest
- *              of every 4 (decompose/export only; sdq_linear returns SDQ_ERR_UNSUPPORTED).
+ *              of every 4 (decompose / export only: the buffer then holds the canonical arrays and
+ *              sdq_linear returns SDQ_ERR_UNSUPPORTED).
  *   in_block   Q-Vector length: logical K sharing one E8M0 scale, for W_i and for the 4-bit
  *              activations (64 is what sdq_linear executes; 32 is decompose/quantize/export only).
  *   scale_rule E8M0 exponent from the Q-Vector's largest magnitude a: OCP_FLOOR = floor(log2 a) - 2,

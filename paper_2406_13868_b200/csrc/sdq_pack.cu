@@ -7,6 +7,7 @@
 #include "sdq_codec.cuh"
 #include "sdq_internal.h"
 #include "sdq_layout.h"
+#include "sdq_plain.h"
 
 namespace sdq {
 
@@ -233,12 +234,12 @@ extern "C" sdq_status_t sdq_packed_size(int64_t N, int64_t K, const sdq_config_t
 {
   if (!cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
   if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2) return SDQ_ERR_SHAPE;
-  if (cfg->in_gran != SDQ_GRAN_PAIR || cfg->in_block != 64) return SDQ_ERR_UNSUPPORTED;
-  if (bytes) *bytes = packed_offsets(N, K, cfg->out_n).total;
+  if (bytes) *bytes = is_tensor_core_reading(*cfg) ? packed_offsets(N, K, cfg->out_n).total : plain_packed_offsets(N, K, *cfg).total;
   if (algorithmic_bytes) {
-    // per weight: 4-bit values on half the positions (2) + two 2-bit pair indices per 8 (0.5) + one
-    // 8-bit scale per 64 (0.125) + out_n * (8 value + 3 index bits) per 8; plus one 32-bit row scale
-    const double bits = 2.0 + 0.5 + 0.125 + cfg->out_n * 11.0 / 8.0;
+    // per weight: 4-bit values on half the positions (2) + index metadata (pair-wise: two 2-bit pair indices per 8 =
+    // 0.5; element-wise: two 2-bit indices per 4 = 1) + one 8-bit scale per Q-Vector + out_n * (8 value + 3 index
+    // bits) per 8; plus one 32-bit row scale
+    const double bits = 2.0 + (cfg->in_gran == SDQ_GRAN_PAIR ? 0.5 : 1.0) + 8.0 / cfg->in_block + cfg->out_n * 11.0 / 8.0;
     *algorithmic_bytes = (size_t)((double)N * (double)K * bits / 8.0) + (cfg->out_n ? (size_t)N * 4 : 0);
   }
   return SDQ_OK;
@@ -249,27 +250,34 @@ extern "C" sdq_status_t sdq_decompose(const void* W, int64_t N, int64_t K, int64
 {
   if (!W || !packed_buf || !out || !cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
   if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2 || ldw < K) return SDQ_ERR_SHAPE;
-  if (cfg->in_gran != SDQ_GRAN_PAIR || cfg->in_block != 64) return SDQ_ERR_UNSUPPORTED;
   if (((uintptr_t)W & 15) || ((uintptr_t)packed_buf & 15) || (ldw % 8)) return SDQ_ERR_ALIGNMENT;
+  const bool tc = is_tensor_core_reading(*cfg);
   const PackedOffsets off = packed_offsets(N, K, cfg->out_n);
-  if (packed_bytes < off.total) return SDQ_ERR_BUFFER_TOO_SMALL;
+  const PlainPackedOffsets poff = plain_packed_offsets(N, K, *cfg);
+  if (packed_bytes < (tc ? off.total : poff.total)) return SDQ_ERR_BUFFER_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
   uint32_t* flags = device_flags();
   if (!flags) return SDQ_ERR_CUDA;
   if (cudaMemsetAsync(flags + FLAG_NONFINITE, 0, sizeof(uint32_t), st) != cudaSuccess) return SDQ_ERR_CUDA;
-  pack_kernel<<<(unsigned)N, 128, 0, st>>>((const __nv_bfloat16*)W, N, K, ldw, *cfg, (uint8_t*)packed_buf, off, flags);
+  if (tc) pack_kernel<<<(unsigned)N, 128, 0, st>>>((const __nv_bfloat16*)W, N, K, ldw, *cfg, (uint8_t*)packed_buf, off, flags);
+  else launch_pack_plain(W, N, K, ldw, *cfg, packed_buf, flags, st);
   if (cudaGetLastError() != cudaSuccess) return SDQ_ERR_CUDA;
   uint32_t nonfinite = 0;
   if (cudaMemcpyAsync(&nonfinite, flags + FLAG_NONFINITE, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SDQ_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return SDQ_ERR_CUDA;
   out->dev = packed_buf;
-  out->bytes = off.total;
+  out->bytes = tc ? off.total : poff.total;
   out->N = N;
   out->K = K;
   out->cfg = *cfg;
   for (int i = 0; i < 8; ++i) out->off[i] = 0;
-  out->off[0] = off.wi; out->off[1] = off.wo; out->off[2] = off.sfa_out;
-  out->off[3] = off.ocode; out->off[4] = off.oidx; out->off[5] = off.osexp;
+  if (tc) {
+    out->off[0] = off.wi; out->off[1] = off.wo; out->off[2] = off.sfa_out;
+    out->off[3] = off.ocode; out->off[4] = off.oidx; out->off[5] = off.osexp;
+  } else {
+    out->off[0] = poff.in_code; out->off[1] = poff.in_meta; out->off[2] = poff.in_scale;
+    out->off[3] = poff.out_code; out->off[4] = poff.out_idx; out->off[5] = poff.osexp;
+  }
   return nonfinite ? SDQ_ERR_NONFINITE : SDQ_OK;
 }
 
@@ -277,6 +285,22 @@ extern "C" sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canon
 {
   if (!P || !out || !P->dev || !out->in_code || !out->in_meta || !out->in_scale || !out->out_sexp) return SDQ_ERR_INVALID_ARG;
   if (P->cfg.out_n > 0 && (!out->out_code || !out->out_idx)) return SDQ_ERR_INVALID_ARG;
+  if (!is_tensor_core_reading(P->cfg)) {
+    // the buffer already holds the canonical arrays
+    const PlainPackedOffsets o = plain_packed_offsets(P->N, P->K, P->cfg);
+    const uint8_t* b = (const uint8_t*)P->dev;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t n = (size_t)P->N, k = (size_t)P->K, on = (size_t)P->cfg.out_n;
+    bool ok = cudaMemcpyAsync(out->in_code, b + o.in_code, n * k / 2, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(out->in_meta, b + o.in_meta, n * (P->cfg.in_gran == SDQ_GRAN_PAIR ? k / 8 : k / 4), cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(out->in_scale, b + o.in_scale, n * k / (size_t)P->cfg.in_block, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+    if (on) {
+      ok = ok && cudaMemcpyAsync(out->out_code, b + o.out_code, n * (k / 8) * on, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+      ok = ok && cudaMemcpyAsync(out->out_idx, b + o.out_idx, n * (k / 8) * on, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+    }
+    ok = ok && cudaMemcpyAsync(out->out_sexp, b + o.osexp, n * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+    return ok ? SDQ_OK : SDQ_ERR_CUDA;
+  }
   const PackedOffsets off = packed_offsets(P->N, P->K, P->cfg.out_n);
   export_packed_kernel<<<(unsigned)P->N, 128, 0, (cudaStream_t)stream>>>((const uint8_t*)P->dev, P->N, P->K, P->cfg, off, *out);
   return cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;

@@ -1,0 +1,247 @@
+// The readings of the decomposition that the sparse tensor core cannot execute -- element-wise 2:4 inliers
+// (SDQ_GRAN_ELEM) and / or one scale per 32 logical K (in_block = 32), i.e. the literal "2:4, block-32 MXFP4" wording
+// -- are decompose / quantize / export only.  Their buffers simply hold the canonical arrays (one code per byte,
+// sections in the order of sdq_canonical_t / sdq_act_canonical_t); sdq_linear refuses them.
+// Same algorithm as sdq_pack.cu / sdq_quant_act.cu (Section 5, Stage 2 -> Stage 1 -> Stage 3), same thread mapping:
+// one thread per S-Vector of 8 weights, 4 lanes x 16 elements per token and Q-Vector pair for activations.
+#include "sdq_codec.cuh"
+#include "sdq_internal.h"
+#include "sdq_layout.h"
+#include "sdq_plain.h"
+
+namespace sdq {
+
+__device__ __forceinline__ void load_group8(const __nv_bfloat16* w, uint32_t (&bits)[8]) {
+  const uint4 v = *reinterpret_cast<const uint4*>(w);
+  const uint32_t r[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    bits[2 * i] = r[i] & 0xFFFFu;
+    bits[2 * i + 1] = r[i] >> 16;
+  }
+}
+__device__ __forceinline__ void pick_outliers(const uint32_t (&key)[8], int out_n, int& o0, int& o1) {
+  o0 = o1 = -1;
+  if (out_n >= 1) {
+    int b = 0;
+#pragma unroll
+    for (int i = 1; i < 8; ++i)
+      if (key[i] > key[b]) b = i;
+    o0 = b;
+  }
+  if (out_n >= 2) {
+    int b = -1;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (i == o0) continue;
+      if (b < 0 || key[i] > key[b]) b = i;
+    }
+    o1 = b;
+    if (o0 > o1) { int t = o0; o0 = o1; o1 = t; }
+  }
+}
+
+__global__ void __launch_bounds__(128)
+pack_plain_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t ldw, sdq_config_t cfg, uint8_t* __restrict__ blob,
+                  PlainPackedOffsets off, uint32_t* __restrict__ flags)
+{
+  const int64_t n = blockIdx.x;
+  const int tid = threadIdx.x;
+  const int G = (int)(K / 8), out_n = cfg.out_n, Bs = cfg.in_block;
+  const bool pair = cfg.in_gran == SDQ_GRAN_PAIR;
+  const __nv_bfloat16* wrow = W + n * ldw;
+  __shared__ uint32_t s_red[4];
+  __shared__ int s_e;
+
+  uint32_t okey_max = 0, bad = 0;
+  for (int g = tid; g < G; g += 128) {
+    uint32_t bits[8], key[8];
+    load_group8(wrow + 8 * g, bits);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      key[i] = bits[i] & 0x7FFFu;
+      bad |= (key[i] >= 0x7F80u);
+    }
+    int o0, o1;
+    pick_outliers(key, out_n, o0, o1);
+    if (o0 >= 0) okey_max = max(okey_max, key[o0]);
+    if (o1 >= 0) okey_max = max(okey_max, key[o1]);
+  }
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) {
+    okey_max = max(okey_max, __shfl_xor_sync(0xffffffffu, okey_max, s));
+    bad |= __shfl_xor_sync(0xffffffffu, bad, s);
+  }
+  if ((tid & 31) == 0) s_red[tid >> 5] = okey_max;
+  if (bad && (tid & 31) == 0) atomicOr(&flags[FLAG_NONFINITE], 1u);
+  __syncthreads();
+  if (tid == 0) s_e = fp8_scale_exp(bf16_bits_to_float(max(max(s_red[0], s_red[1]), max(s_red[2], s_red[3]))));
+  __syncthreads();
+  const int e = s_e;
+  if (tid == 0) reinterpret_cast<int32_t*>(blob + off.osexp)[n] = e;
+
+  for (int g = tid; g < G; g += 128) {
+    uint32_t bits[8], key[8];
+    load_group8(wrow + 8 * g, bits);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) key[i] = bits[i] & 0x7FFFu;
+    int o0, o1;
+    pick_outliers(key, out_n, o0, o1);
+    int slot_pos[4];
+    if (pair) {
+      float score[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float a0 = (2 * j == o0 || 2 * j == o1) ? 0.0f : bf16_bits_to_float(key[2 * j]);
+        const float a1 = (2 * j + 1 == o0 || 2 * j + 1 == o1) ? 0.0f : bf16_bits_to_float(key[2 * j + 1]);
+        score[j] = __fadd_rn(a0, a1);
+      }
+      int j0 = 0;
+#pragma unroll
+      for (int j = 1; j < 4; ++j)
+        if (score[j] > score[j0]) j0 = j;
+      int j1 = -1;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (j == j0) continue;
+        if (j1 < 0 || score[j] > score[j1]) j1 = j;
+      }
+      if (j0 > j1) { int t = j0; j0 = j1; j1 = t; }
+      slot_pos[0] = 2 * j0; slot_pos[1] = 2 * j0 + 1; slot_pos[2] = 2 * j1; slot_pos[3] = 2 * j1 + 1;
+      blob[off.in_meta + (size_t)n * G + g] = (uint8_t)(j0 | (j1 << 2));
+    } else {
+      // element-wise 2:4: in each group of 4 keep the 2 largest magnitudes among the non-outlier positions
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        int i0 = -1, i1 = -1;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int p = 4 * h + i;
+          if (p == o0 || p == o1) continue;
+          if (i0 < 0 || key[p] > key[4 * h + i0]) i0 = i;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int p = 4 * h + i;
+          if (p == o0 || p == o1 || i == i0) continue;
+          if (i1 < 0 || key[p] > key[4 * h + i1]) i1 = i;
+        }
+        if (i0 > i1) { int t = i0; i0 = i1; i1 = t; }
+        slot_pos[2 * h] = 4 * h + i0;
+        slot_pos[2 * h + 1] = 4 * h + i1;
+        blob[off.in_meta + (size_t)n * (2 * G) + 2 * g + h] = (uint8_t)(i0 | (i1 << 2));
+      }
+    }
+    // Q-Vector maximum over the kept inlier values: Bs = 64 -> 8 S-Vectors (8 lanes); Bs = 32 -> 4 lanes
+    uint32_t ikey = 0;
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      const int p = slot_pos[s];
+      if (p != o0 && p != o1) ikey = max(ikey, key[p]);
+    }
+    ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 1));
+    ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 2));
+    if (Bs == 64) ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 4));
+    const uint32_t c = e8m0_scale_code(bf16_bits_to_float(ikey), cfg.scale_rule);
+    const int lanes_per_q = Bs / 8;
+    if ((g % lanes_per_q) == 0) blob[off.in_scale + (size_t)n * (K / Bs) + g / lanes_per_q] = (uint8_t)c;
+    float v[4];
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      const int p = slot_pos[s];
+      v[s] = (p == o0 || p == o1) ? 0.0f : bf16_bits_to_float(bits[p]) * pow2_inv_e8m0(c);
+    }
+    const uint32_t c01 = e2m1x2(v[0], v[1]), c23 = e2m1x2(v[2], v[3]);
+    uint8_t* ic = blob + off.in_code + (size_t)n * (K / 2) + 4 * g;
+    ic[0] = c01 & 15; ic[1] = c01 >> 4; ic[2] = c23 & 15; ic[3] = c23 >> 4;
+    if (out_n > 0) {
+      uint8_t* oc = blob + off.out_code + ((size_t)n * G + g) * out_n;
+      uint8_t* oi = blob + off.out_idx + ((size_t)n * G + g) * out_n;
+      oc[0] = (uint8_t)e4m3x1(bf16_bits_to_float(bits[o0]) * pow2_neg(e));
+      oi[0] = (uint8_t)o0;
+      if (out_n == 2) {
+        oc[1] = (uint8_t)e4m3x1(bf16_bits_to_float(bits[o1]) * pow2_neg(e));
+        oi[1] = (uint8_t)o1;
+      }
+    }
+  }
+}
+
+// activations, one scale per 32 K: 4 lanes x 16 elements per token and 64 K, a Q-Vector is a lane pair
+__global__ void __launch_bounds__(256)
+quant_act_plain_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int64_t ldx, sdq_config_t cfg, uint8_t* __restrict__ buf,
+                       PlainActOffsets off, const float* __restrict__ partial, int n_chunks)
+{
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int t = lane >> 2, l = lane & 3;
+  const int64_t m = (int64_t)blockIdx.x * 8 + t;
+  const bool live = m < M;
+  const int NB = (int)(K / 64);
+  const int b0 = blockIdx.y * 16;
+  float ramax = 0.0f;
+  if (live)
+    for (int c = l; c < n_chunks; c += 4) ramax = fmaxf(ramax, partial[m * n_chunks + c]);
+  ramax = fmaxf(ramax, __shfl_xor_sync(0xffffffffu, ramax, 1));
+  ramax = fmaxf(ramax, __shfl_xor_sync(0xffffffffu, ramax, 2));
+  const int e = fp8_scale_exp(ramax);
+  const float s8 = pow2_neg(e);
+  if (live && blockIdx.y == 0 && warp == 0 && l == 0) reinterpret_cast<int32_t*>(buf + off.sexp)[m] = e;
+  for (int i = 0; i < 2; ++i) {
+    const int b = b0 + warp + i * 8;
+    if (b >= NB) break;
+    float v[16];
+    if (live) {
+      const __nv_bfloat16* px = X + m * ldx + (int64_t)b * 64 + l * 16;
+      const uint4 a = reinterpret_cast<const uint4*>(px)[0], bb = reinterpret_cast<const uint4*>(px)[1];
+      const uint32_t r[8] = {a.x, a.y, a.z, a.w, bb.x, bb.y, bb.z, bb.w};
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        v[2 * j] = __uint_as_float(r[j] << 16);
+        v[2 * j + 1] = __uint_as_float(r[j] & 0xFFFF0000u);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) v[j] = 0.0f;
+    }
+    float bmax = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      v[j] = copysignf(fminf(fabsf(v[j]), 3.3895313892515355e38f), v[j]);
+      bmax = fmaxf(bmax, fabsf(v[j]));
+    }
+    bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
+    if (cfg.in_block == 64) bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
+    const uint32_t c = e8m0_scale_code(bmax, cfg.scale_rule);
+    const float s4 = pow2_inv_e8m0(c);
+    if (!live) continue;
+    const int64_t k = (int64_t)b * 64 + l * 16;
+    uint8_t* c4 = buf + off.xq4_code + (size_t)m * K + k;
+    uint8_t* c8 = buf + off.xq8_code + (size_t)m * K + k;
+    uint32_t q4[4], q8[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t a = e2m1x2(v[4 * j] * s4, v[4 * j + 1] * s4), bq = e2m1x2(v[4 * j + 2] * s4, v[4 * j + 3] * s4);
+      q4[j] = (a & 15) | ((a >> 4) << 8) | ((bq & 15) << 16) | ((bq >> 4) << 24);
+      q8[j] = e4m3x2(v[4 * j] * s8, v[4 * j + 1] * s8) | (e4m3x2(v[4 * j + 2] * s8, v[4 * j + 3] * s8) << 16);
+    }
+    *reinterpret_cast<uint4*>(c4) = make_uint4(q4[0], q4[1], q4[2], q4[3]);
+    *reinterpret_cast<uint4*>(c8) = make_uint4(q8[0], q8[1], q8[2], q8[3]);
+    const int Bs = cfg.in_block;
+    if ((k % Bs) == 0) buf[off.xq4_scale + (size_t)m * (K / Bs) + k / Bs] = (uint8_t)c;
+  }
+}
+
+void launch_pack_plain(const void* W, int64_t N, int64_t K, int64_t ldw, const sdq_config_t& cfg, void* buf, uint32_t* flags,
+                       cudaStream_t st)
+{
+  pack_plain_kernel<<<(unsigned)N, 128, 0, st>>>((const __nv_bfloat16*)W, N, K, ldw, cfg, (uint8_t*)buf, plain_packed_offsets(N, K, cfg), flags);
+}
+void launch_quant_plain(const void* X, int64_t M, int64_t K, int64_t ldx, const sdq_config_t& cfg, void* buf, const float* partial,
+                        int n_chunks, cudaStream_t st)
+{
+  const dim3 grid((unsigned)((M + 7) / 8), (unsigned)n_chunks);
+  quant_act_plain_kernel<<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, M, K, ldx, cfg, (uint8_t*)buf, plain_act_offsets(M, K, cfg), partial,
+                                                 n_chunks);
+}
+
+}  // namespace sdq

@@ -11,6 +11,7 @@
 #include "sdq_codec.cuh"
 #include "sdq_internal.h"
 #include "sdq_layout.h"
+#include "sdq_plain.h"
 
 namespace sdq {
 
@@ -164,8 +165,7 @@ extern "C" sdq_status_t sdq_act_size(int64_t M, int64_t K, const sdq_config_t* c
 {
   if (!act_cfg_ok(cfg) || !bytes) return SDQ_ERR_INVALID_ARG;
   if (M <= 0 || K <= 0 || K % K2) return SDQ_ERR_SHAPE;
-  if (cfg->in_block != 64) return SDQ_ERR_UNSUPPORTED;
-  *bytes = act_offsets(M, K).total;
+  *bytes = cfg->in_block == 64 ? act_offsets(M, K).total : plain_act_offsets(M, K, *cfg).total;
   return SDQ_OK;
 }
 
@@ -174,29 +174,43 @@ extern "C" sdq_status_t sdq_quantize_act(const void* X, int64_t M, int64_t K, in
 {
   if (!X || !xq_buf || !out || !act_cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
   if (M <= 0 || K <= 0 || K % K2 || ldx < K) return SDQ_ERR_SHAPE;
-  if (cfg->in_block != 64) return SDQ_ERR_UNSUPPORTED;
   if (((uintptr_t)X & 15) || ((uintptr_t)xq_buf & 15) || (ldx % 8)) return SDQ_ERR_ALIGNMENT;
+  const bool tiled = cfg->in_block == 64;
   const ActOffsets off = act_offsets(M, K);
-  if (xq_bytes < off.total) return SDQ_ERR_BUFFER_TOO_SMALL;
+  const PlainActOffsets poff = plain_act_offsets(M, K, *cfg);
+  if (xq_bytes < (tiled ? off.total : poff.total)) return SDQ_ERR_BUFFER_TOO_SMALL;
   const int n_chunks = (int)((K / 64 + QA_CHUNK_QV - 1) / QA_CHUNK_QV);
-  float* partial = reinterpret_cast<float*>((uint8_t*)xq_buf + off.amax);
+  float* partial = reinterpret_cast<float*>((uint8_t*)xq_buf + (tiled ? off.amax : poff.amax));
   const dim3 grid((unsigned)((M + 7) / 8), (unsigned)n_chunks);
   act_amax_kernel<<<grid, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, partial, n_chunks);
-  quant_act_kernel<<<grid, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, *cfg, (uint8_t*)xq_buf, off, partial, n_chunks);
+  if (tiled) quant_act_kernel<<<grid, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, *cfg, (uint8_t*)xq_buf, off, partial, n_chunks);
+  else launch_quant_plain(X, M, K, ldx, *cfg, xq_buf, partial, n_chunks, (cudaStream_t)stream);
   if (cudaGetLastError() != cudaSuccess) return SDQ_ERR_CUDA;
   out->dev = xq_buf;
-  out->bytes = off.total;
+  out->bytes = tiled ? off.total : poff.total;
   out->M = M;
   out->K = K;
   out->cfg = *cfg;
   for (int i = 0; i < 6; ++i) out->off[i] = 0;
-  out->off[0] = off.xi; out->off[1] = off.xo; out->off[2] = off.sfb_out; out->off[3] = off.sexp;
+  if (tiled) { out->off[0] = off.xi; out->off[1] = off.xo; out->off[2] = off.sfb_out; out->off[3] = off.sexp; }
+  else { out->off[0] = poff.xq4_code; out->off[1] = poff.xq4_scale; out->off[2] = poff.xq8_code; out->off[3] = poff.sexp; }
   return SDQ_OK;
 }
 
 extern "C" sdq_status_t sdq_act_export(const sdq_act_t* Xq, const sdq_act_canonical_t* out, void* stream)
 {
   if (!Xq || !out || !Xq->dev || !out->xq4_code || !out->xq4_scale || !out->xq8_code || !out->xq8_sexp) return SDQ_ERR_INVALID_ARG;
+  if (Xq->cfg.in_block != 64) {
+    const PlainActOffsets o = plain_act_offsets(Xq->M, Xq->K, Xq->cfg);
+    const uint8_t* b = (const uint8_t*)Xq->dev;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t m = (size_t)Xq->M, k = (size_t)Xq->K;
+    bool ok = cudaMemcpyAsync(out->xq4_code, b + o.xq4_code, m * k, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(out->xq4_scale, b + o.xq4_scale, m * k / (size_t)Xq->cfg.in_block, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(out->xq8_code, b + o.xq8_code, m * k, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(out->xq8_sexp, b + o.sexp, m * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+    return ok ? SDQ_OK : SDQ_ERR_CUDA;
+  }
   const ActOffsets off = act_offsets(Xq->M, Xq->K);
   export_act_kernel<<<(unsigned)Xq->M, QA_THREADS, 0, (cudaStream_t)stream>>>((const uint8_t*)Xq->dev, Xq->M, Xq->K, off, *out);
   return cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;

@@ -45,8 +45,9 @@ def test_size_queries_and_argument_errors_without_a_gpu(m):
     assert L.sdq_packed_size(100, 4096, ctypes.byref(cfg), ctypes.byref(b), ctypes.byref(a)) == 2    # N % 128
     bad = m.Config(3, 0, 64, 0)
     assert L.sdq_packed_size(128, 256, ctypes.byref(bad), ctypes.byref(b), ctypes.byref(a)) == 1
-    elem = m.Config(1, m.GRAN_ELEM, 32, 0)
-    assert L.sdq_packed_size(128, 256, ctypes.byref(elem), ctypes.byref(b), ctypes.byref(a)) == 4
+    elem = m.Config(1, m.GRAN_ELEM, 32, 0)      # literal "2:4, block-32" reading: 2 + 1 + 0.25 + 1.375 bits per weight
+    assert L.sdq_packed_size(128, 256, ctypes.byref(elem), ctypes.byref(b), ctypes.byref(a)) == 0
+    assert a.value == int(128 * 256 * 4.625 / 8) + 128 * 4
     assert L.sdq_act_size(1, 4096, ctypes.byref(cfg), ctypes.byref(b)) == 0 and b.value > 4096 * 3 // 2
     assert L.sdq_act_size(0, 4096, ctypes.byref(cfg), ctypes.byref(b)) == 2
     # null pointers are rejected before anything is launched

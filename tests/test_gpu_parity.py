@@ -206,14 +206,46 @@ def test_packer_ties_zeros_and_negative_zero():
                 assert np.array_equal(pe[name], getattr(op, name)), (name, out_n, rule)
 
 
+@pytest.mark.parametrize("gran,block", [(1, 32), (1, 64), (0, 32)])
+@pytest.mark.parametrize("out_n", [0, 1, 2])
+def test_literal_readings_element_wise_2of4_and_block32(gran, block, out_n):
+    """element-wise 2:4 inliers and / or one scale per 32 K (the literal '2:4, block-32 MXFP4' wording): packer and
+    activation quantizer are bit-exact against the oracle; these readings are decompose / quantize / export only"""
+    m = sdq()
+    for rule in (0, 1):
+        cfg = m.Config(out_n, gran, block, rule)
+        oc = so.Config(out_n, gran, block, rule)
+        W = sdq_synth.make_weight(256, 1024, 40 + out_n)
+        X = sdq_synth.make_act(37, 1024, 41 + out_n)
+        pe = {k: v.cpu().numpy() for k, v in m.packed_export(m.sdq_decompose(W.cuda(), cfg)).items()}
+        op = so.decompose(sdq_synth.bf16_bits(W), oc)
+        for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp"):
+            assert np.array_equal(pe[name], getattr(op, name)), (name, rule)
+        ae = {k: v.cpu().numpy() for k, v in m.act_export(m.sdq_quantize_act(X.cuda(), cfg)).items()}
+        oq = so.quantize_act(sdq_synth.bf16_bits(X), oc)
+        for name in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp"):
+            assert np.array_equal(ae[name], getattr(oq, name)), (name, rule)
+    # ties, zeros and -0 under the element-wise pattern
+    rng = np.random.default_rng(2)
+    vals = np.array([0.0, -0.0, 0.5, -0.5, 1.0, 1.0, -2.0, 2.0, 3.0, 1e-30, 448.0, 6.0, 7.0, 0.75])
+    Wt = torch.from_numpy(rng.choice(vals, size=(128, 512))).to(torch.bfloat16)
+    cfg, oc = m.Config(out_n, gran, block, 0), so.Config(out_n, gran, block, 0)
+    pe = {k: v.cpu().numpy() for k, v in m.packed_export(m.sdq_decompose(Wt.cuda(), cfg)).items()}
+    op = so.decompose(sdq_synth.bf16_bits(Wt), oc)
+    for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp"):
+        assert np.array_equal(pe[name], getattr(op, name)), name
+
+
 def test_errors_are_status_codes():
     m = sdq()
     W = sdq_synth.make_weight(128, 256, 0).cuda()
     with pytest.raises(m.SdqError) as e:
         m.sdq_decompose(W[:, :128].contiguous())           # K not a multiple of 256
     assert e.value.code == 2
+    p_elem = m.sdq_decompose(W, m.Config(1, m.GRAN_ELEM, 32, 0))            # decompose-only reading ...
+    xq32 = m.sdq_quantize_act(sdq_synth.make_act(4, 256, 0).cuda(), m.Config(1, m.GRAN_ELEM, 32, 0))
     with pytest.raises(m.SdqError) as e:
-        m.sdq_decompose(W, m.Config(1, m.GRAN_ELEM, 32, 0))  # decompose-only reading not built yet
+        m.sdq_linear(xq32, p_elem)                                          # ... which the tensor core cannot run
     assert e.value.code == 4
     Wbad = W.clone()
     Wbad[3, 7] = float("inf")
