@@ -383,8 +383,103 @@ def run_case(args):
     print(json.dumps({"case": args.case, "M": M, "N": N, "K": K, "launches": args.steps}))
 
 
+def time_graph(fn, reps=10):
+    """captures fn() once in a CUDA graph and returns the mean replay time in ms"""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        fn()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        fn()
+    g.replay()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        g.replay()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+def run_sweep(args):
+    """Extra measurements for the other configurations (not the contract line): the OPT-6.7B FFN with the outlier
+    pattern swept, and all 224 linear layers of a 32-layer LLaMA-7B-shaped decoder back to back for a sweep of
+    token counts (quantize_act where a new activation enters + sdq_linear, one CUDA graph per token count)."""
+    import paper_2406_13868_b200 as sdq
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    peaks = measured_peaks()
+    out = {"peaks": peaks}
+    # ---- config 4: OPT-6.7B FFN, M = 4096
+    M = 4096
+    X = sdq_synth.make_act(M, 4096, 4001, device="cuda")
+    H = sdq_synth.make_act(M, 16384, 4002, device="cuda")
+    W1 = sdq_synth.make_weight(16384, 4096, 4003, device="cuda")
+    W2 = sdq_synth.make_weight(4096, 16384, 4004, device="cuda")
+    Y1 = torch.empty((M, 16384), dtype=torch.bfloat16, device=dev)
+    Y2 = torch.empty((M, 4096), dtype=torch.bfloat16, device=dev)
+    c4 = {}
+    for on, name in ((1, "1:8"), (2, "2:8"), (0, "none")):
+        cfg = sdq.Config(on, sdq.GRAN_PAIR, 64, 0)
+        P1, P2 = sdq.sdq_decompose(W1, cfg), sdq.sdq_decompose(W2, cfg)
+        xq, hq = sdq.sdq_quantize_act(X, cfg), sdq.sdq_quantize_act(H, cfg)
+        t1 = time_graph(lambda: sdq.sdq_linear(xq, P1, Y1))
+        t2 = time_graph(lambda: sdq.sdq_linear(hq, P2, Y2))
+        fl = 2.0 * M * 4096 * 16384
+        c4[name] = {"fc1_ms": t1, "fc1_TFLOPs": fl / t1 / 1e9, "fc2_ms": t2, "fc2_TFLOPs": fl / t2 / 1e9}
+        del P1, P2, xq, hq
+    out["opt67b_ffn_M4096_outlier_sweep"] = c4
+    del X, H, W1, W2, Y1, Y2
+    # ---- config 5: 32 layers x (q, k, v, o, gate, up, down)
+    cfg = sdq.Config(1, sdq.GRAN_PAIR, 64, 0)
+    shapes = [(4096, 4096)] * 4 + [(11008, 4096)] * 2 + [(4096, 11008)]
+    layers = []
+    algo = 0
+    for l in range(32):
+        ps = []
+        for i, (N, K) in enumerate(shapes):
+            W = sdq_synth.make_weight(N, K, 5000 + 10 * l + i, device="cuda")
+            ps.append(sdq.sdq_decompose(W, cfg))
+            algo += ps[-1].algorithmic_bytes
+            del W
+        layers.append(ps)
+    c5 = {"algorithmic_weight_bytes": algo}
+    for M in (1, 16, 128, 1024, 8192):
+        X = sdq_synth.make_act(M, 4096, 5500 + M, n_outlier_channels=41, device="cuda")
+        Hh = sdq_synth.make_act(M, 11008, 5600 + M, n_outlier_channels=110, device="cuda")
+        bx = torch.empty(sdq.act_size(M, 4096, cfg), dtype=torch.uint8, device=dev)
+        bh = torch.empty(sdq.act_size(M, 11008, cfg), dtype=torch.uint8, device=dev)
+        Ya = torch.empty((M, 4096), dtype=torch.bfloat16, device=dev)
+        Yb = torch.empty((M, 11008), dtype=torch.bfloat16, device=dev)
+
+        def model():
+            for ps in layers:
+                xq = sdq.sdq_quantize_act(X, cfg, bx)          # input of q, k, v
+                for j in range(3):
+                    sdq.sdq_linear(xq, ps[j], Ya)
+                xq = sdq.sdq_quantize_act(X, cfg, bx)          # input of o
+                sdq.sdq_linear(xq, ps[3], Ya)
+                xq = sdq.sdq_quantize_act(X, cfg, bx)          # input of gate, up
+                sdq.sdq_linear(xq, ps[4], Yb)
+                sdq.sdq_linear(xq, ps[5], Yb)
+                hq = sdq.sdq_quantize_act(Hh, cfg, bh)         # input of down
+                sdq.sdq_linear(hq, ps[6], Ya)
+        ms = time_graph(model, reps=3 if M >= 1024 else 10)
+        flops = 2.0 * M * sum(n * k for n, k in shapes) * 32
+        c5["M%d" % M] = {"ms_per_model_pass": ms, "dense_equiv_TFLOPs": flops / ms / 1e9, "weight_GBps_algorithmic": algo / ms / 1e6,
+                         "frac_of_hbm_peak": algo / ms / 1e6 / peaks["hbm"], "frac_of_mixed_tensor_peak": flops / ms / 1e9 / (peaks["bf16"] * MIXED_PEAK_OVER_BF16)}
+    out["llama7b_32_layers_224_linears"] = c5
+    assert sdq.device_status() == 0
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--sweep", action="store_true", help="measure the other configurations (OPT FFN outlier sweep, whole-model pass) and exit")
     ap.add_argument("--case", default=None, choices=["gemm_prefill", "gemm_decode", "quant"],
                     help="run only a small single-kernel case (for profiler captures) and exit")
     ap.add_argument("--gpus", type=int, default=1)
@@ -393,7 +488,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.case:
+    if args.sweep:
+        run_sweep(args)
+    elif args.case:
         run_case(args)
     elif args.impl == "reference":
         run_reference(args)
