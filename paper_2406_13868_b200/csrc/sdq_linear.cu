@@ -417,16 +417,14 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   p.cluster_ks = 1;
   p.ws_counter = nullptr;
   p.ws_partial = nullptr;
-  if (!ws && M <= 32) {
-    // cluster split-K: power-of-two cluster of up to 8 CTAs per row tile, about two CTAs per SM in total
+  if (!ws && M <= 128) {
+    // cluster split-K: power-of-two cluster of up to 8 CTAs per row tile; up to 32 tokens the CTAs are small enough
+    // for two per SM, beyond that one per SM
     const int RT = (int)(P->N / TILE_ROWS), T2c = (int)(P->K / K2);
+    const int cta_budget = (M <= 32 ? 2 : 1) * sm_count;
     int ks = 8;
-    while (ks > 1 && (ks * RT > 2 * sm_count || ks > T2c)) ks >>= 1;
-    const int T1c = p.out_n ? (int)(P->K / K1) : 0;
-    const int stages = (T2c + ks - 1) / ks + (T1c + ks - 1) / ks;
-    int max_slots_c = RING_BYTES / p.slot_bytes;
-    if (max_slots_c > MAX_SLOTS) max_slots_c = MAX_SLOTS;
-    if (ks > 1 && stages <= max_slots_c) { p.ksplit = ks; p.cluster_ks = ks; }
+    while (ks > 1 && (ks * RT > cta_budget || ks > T2c)) ks >>= 1;
+    if (ks > 1) { p.ksplit = ks; p.cluster_ks = ks; }
   }
   if (ws) {
     const int ks = choose_ksplit(M, P->N, P->K, sm_count);
@@ -454,6 +452,10 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
     grid_x = p.total_tiles;
     p.nslot = stages_per_tile;
     p.release = 0;
+  } else if (p.cluster_ks > 1) {
+    grid_x = p.total_tiles;          // one tile per CTA (the cluster reduction relies on it); total_tiles <= SM count
+    p.nslot = max_slots;
+    p.release = 1;
   } else {
     grid_x = p.total_tiles < sm_count ? p.total_tiles : sm_count;
     p.nslot = max_slots;

@@ -128,9 +128,10 @@ def test_split_k_with_workspace(M, N, K, out_n):
 
 
 @pytest.mark.parametrize("M,N,K,out_n", [(1, 512, 4096, 1), (16, 1024, 4096, 1), (32, 256, 2048, 2), (5, 4096, 1024, 1),
-                                         (16, 256, 1024, 0), (2, 128, 11008, 1)])
+                                         (16, 256, 1024, 0), (2, 128, 11008, 1), (33, 512, 4096, 1), (128, 1024, 4096, 1),
+                                         (100, 256, 11008, 2), (64, 4096, 2048, 1)])
 def test_cluster_split_k_few_tokens(M, N, K, out_n):
-    """up to 32 tokens without a workspace: the thread blocks of a row tile form a cluster and add their partial
+    """up to 128 tokens without a workspace: the thread blocks of a row tile form a cluster and add their partial
     tiles through distributed shared memory in rank order -- same criterion, identical from call to call"""
     m = sdq()
     cfg = m.Config(out_n, m.GRAN_PAIR, 64, 0)
