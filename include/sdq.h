@@ -139,6 +139,10 @@ sdq_status_t sdq_act_export(const sdq_act_t* Xq, const sdq_act_canonical_t* out,
  * one accumulator: Y[m][n] = sum_k A_i[m][k] W_i[n][k] + sum_k A_o[m][k] W_o[n][k].
  *   Xq, P (host descriptors; K and cfg must agree); Y (device) [M][ldy] bf16 (round to nearest even
  *   of the fp32 accumulator); ldy >= N elements, ldy % 8 == 0.  Asynchronous on `stream`.
+ *   For M <= 128 the kernel is enqueued with programmatic stream serialization: it may begin (set-up, reading the packed
+ *   weights) while the previous kernel of the stream is still finishing, and waits for that kernel before it
+ *   reads Xq or writes Y.  The packed weights must therefore be complete before the call is enqueued
+ *   (sdq_decompose synchronises its stream, so a buffer it returned always is).
  *   Errors: INVALID_ARG, SHAPE, ALIGNMENT, UNSUPPORTED (in_gran != PAIR or in_block != 64), CUDA. */
 sdq_status_t sdq_linear(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y_bf16, int64_t ldy, void* stream);
 

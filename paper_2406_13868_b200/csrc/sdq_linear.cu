@@ -43,28 +43,39 @@ struct TileCoord {
   int rt, mtile, split;
   int i0, i1, o0, o1;   // inlier stages [i0, i1) of T2, outlier stages [o0, o1) of T1
 };
-__device__ __forceinline__ TileCoord tile_coord(const LinearParams& p, int tile, int RT, int T1, int T2) {
+__device__ __forceinline__ TileCoord tile_coord(int ksplit, int tile, int RT, int T1, int T2) {
   TileCoord c;
-  c.split = tile % p.ksplit;
-  const int rest = tile / p.ksplit;
+  if (ksplit == 1) {
+    c.split = 0; c.rt = tile % RT; c.mtile = tile / RT;
+    c.i0 = 0; c.i1 = T2; c.o0 = 0; c.o1 = T1;
+    return c;
+  }
+  c.split = tile % ksplit;
+  const int rest = tile / ksplit;
   c.rt = rest % RT;
   c.mtile = rest / RT;
-  c.i0 = c.split * T2 / p.ksplit;           // 32-bit: split < 32, T1 <= K/128
-  c.i1 = (c.split + 1) * T2 / p.ksplit;
-  c.o0 = c.split * T1 / p.ksplit;
-  c.o1 = (c.split + 1) * T1 / p.ksplit;
+  c.i0 = c.split * T2 / ksplit;           // 32-bit: split < 32, T1 <= K/128
+  c.i1 = (c.split + 1) * T2 / ksplit;
+  c.o0 = c.split * T1 / ksplit;
+  c.o1 = (c.split + 1) * T1 / ksplit;
   return c;
 }
 
-template <bool F32_OUT>
+// FLEX = false: the many-token instantiation (n_tile = 256, 5 ring slots, 512 TMEM columns, no K split) with every
+// geometry constant known at compile time -- the single-thread issue loops are latency-bound, so each runtime
+// parameter they touch costs time.  FLEX = true: geometry from the launch parameters (few tokens, split K).
+template <bool F32_OUT, bool FLEX>
 __global__ void __launch_bounds__(LIN_THREADS, 1)
 sdq_linear_kernel(const LinearParams p)
 {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint8_t* sm = smem_raw + ((128 - (ptx::smem_u32(smem_raw) & 127)) & 127);
-  const uint32_t SM_STG = (uint32_t)p.ring_bytes, SM_BARS = SM_STG + 4096;
-  const uint32_t TM_I = (uint32_t)p.meta_col, TM_EO = TM_I + 32, TM_SFA_OUT = TM_I + 40, TM_SFB_OUT = TM_I + 44;
+  const int ksplit = FLEX ? p.ksplit : 1, cluster_ks = FLEX ? p.cluster_ks : 1;
+  const bool release = FLEX ? (p.release != 0) : true;
+  const uint32_t SM_STG = FLEX ? (uint32_t)p.ring_bytes : (uint32_t)RING_BYTES, SM_BARS = SM_STG + 4096;
+  const uint32_t TM_I = FLEX ? (uint32_t)p.meta_col : 256u, TM_EO = TM_I + 32, TM_SFA_OUT = TM_I + 40, TM_SFB_OUT = TM_I + 44;
+  const uint32_t tmem_cols = FLEX ? (uint32_t)p.tmem_cols : 512u;
   uint64_t* full = reinterpret_cast<uint64_t*>(sm + SM_BARS);
   uint64_t* empty = full + MAX_SLOTS;
   uint64_t* acc_full = empty + MAX_SLOTS;
@@ -72,23 +83,24 @@ sdq_linear_kernel(const LinearParams p)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
   uint32_t* last_flag = tmem_slot + 1;
 
-  const int n_tile = p.n_tile;
+  const int n_tile = FLEX ? p.n_tile : 256;
   const int RT = (int)(p.N / TILE_ROWS);
   const int T1 = p.out_n ? (int)(p.K / K1) : 0, T2 = (int)(p.K / K2);
   const int n_atiles = (n_tile + TILE_TOK - 1) / TILE_TOK;     // 128-token activation tiles per token tile
-  const uint32_t nslot = (uint32_t)p.nslot, slot_bytes = (uint32_t)p.slot_bytes;
+  const uint32_t nslot = FLEX ? (uint32_t)p.nslot : 5u, slot_bytes = FLEX ? (uint32_t)p.slot_bytes : 45056u;
   const uint32_t sl_sf = SL_B + (uint32_t)n_tile * 128u;
 
   // the coordinates of the first tile are worked out by every thread while the barriers and TMEM are being set up
   // (a lone thread needs ~0.5 us for the integer divisions, which would otherwise delay the first copies)
-  const TileCoord first_tc = tile_coord(p, (int)blockIdx.x, RT, T1, T2);
+  const TileCoord first_tc = tile_coord(ksplit, (int)blockIdx.x, RT, T1, T2);
+  if (tid == 0) ptx::griddep_launch_dependents();   // the next launch may be scheduled as soon as every CTA got here
   if (tid == 0) {
     for (uint32_t s = 0; s < nslot; ++s) { ptx::mbar_init(&full[s], 3); ptx::mbar_init(&empty[s], 1); }
     ptx::mbar_init(acc_full, 1);
     ptx::mbar_init(acc_empty, 4);
     ptx::fence_barrier_init();
   }
-  if (warp == 1) ptx::tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
+  if (warp == 1) ptx::tmem_alloc(tmem_slot, tmem_cols);
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
@@ -99,10 +111,11 @@ sdq_linear_kernel(const LinearParams p)
       // ---------------- producers: role 0 = weight records, role 1 = activation codes, role 2 = scale atoms.
       // Each arrives once per stage on full[s] with the bytes it is about to copy.
       const int role = warp == 0 ? 0 : (int)warp - 5;
+      if (role != 0) ptx::griddep_wait();    // activations and their scales come from an earlier kernel; weights do not
       bool ok = true;
       uint32_t s = 0, wrapped = 0, ph = 0;   // ring slot, whether the ring has wrapped, phase parity of `empty`
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-        const TileCoord tc = (tile == (int)blockIdx.x) ? first_tc : tile_coord(p, tile, RT, T1, T2);
+        const TileCoord tc = (tile == (int)blockIdx.x) ? first_tc : tile_coord(ksplit, tile, RT, T1, T2);
         const int mt = tc.mtile * n_tile / TILE_TOK;
         const int have = min(n_atiles, (int)p.aoff.MT - mt);                 // activation tiles that exist
         const uint32_t tok_bytes = (uint32_t)min(n_tile, TILE_TOK) * 128u;   // bytes per activation tile per stage
@@ -113,7 +126,7 @@ sdq_linear_kernel(const LinearParams p)
         const size_t xi_tile = (size_t)T2 * XI_BYTES, xo_tile = (size_t)T1 * XO_BYTES;
         const int ni = tc.i1 - tc.i0, no = tc.o1 - tc.o0;
         for (int k = 0; k < ni + no; ++k) {
-          if (wrapped && p.release && !(ok = ptx::mbar_wait(&empty[s], ph ^ 1))) break;
+          if (wrapped && release && !(ok = ptx::mbar_wait(&empty[s], ph ^ 1))) break;
           uint8_t* st = sm + (size_t)s * slot_bytes;
           const bool first_o = (k == ni);
           if (role == 0) {
@@ -174,7 +187,7 @@ sdq_linear_kernel(const LinearParams p)
       const uint64_t d_sf2 = ptx::smem_desc(smb + sl_sf + 2 * SF_ATOM_BYTES, 0, 128);
       const uint32_t slot16 = slot_bytes >> 4;
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
-        const TileCoord tc = (tcount == 0) ? first_tc : tile_coord(p, tile, RT, T1, T2);
+        const TileCoord tc = (tcount == 0) ? first_tc : tile_coord(ksplit, tile, RT, T1, T2);
         const int ni = tc.i1 - tc.i0, no = tc.o1 - tc.o0;
         if (tcount > 0) {   // the epilogue must have drained the accumulator of the previous tile
           ok = ptx::mbar_wait(acc_empty, (tcount - 1) & 1);
@@ -213,7 +226,7 @@ sdq_linear_kernel(const LinearParams p)
                              tmem + TM_SFB_OUT, 1u);
           }
           acc = 1;
-          if (p.release) ptx::tc_commit(&empty[s]);   // ring slots are reused only when a CTA runs more stages than slots
+          if (release) ptx::tc_commit(&empty[s]);   // ring slots are reused only when a CTA runs more stages than slots
           s = sn;
           if (sn == 0) ph ^= 1;
         }
@@ -227,8 +240,9 @@ sdq_linear_kernel(const LinearParams p)
     const uint32_t et = (warp - 2) * 32 + lane;     // 0..127 among the epilogue threads
     uint32_t tcount = 0;
     bool ok = true;
+    ptx::griddep_wait();                            // Y and the workspace may still be in use by the previous kernel
     for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
-      const TileCoord tc = (tcount == 0) ? first_tc : tile_coord(p, tile, RT, T1, T2);
+      const TileCoord tc = (tcount == 0) ? first_tc : tile_coord(ksplit, tile, RT, T1, T2);
       const int64_t m0 = (int64_t)tc.mtile * n_tile;
       const int n_valid = (int)min((int64_t)n_tile, p.M - m0);
       ok = ptx::mbar_wait(acc_full, tcount & 1);
@@ -237,9 +251,9 @@ sdq_linear_kernel(const LinearParams p)
       const int64_t n0 = (int64_t)tc.rt * TILE_ROWS;
       // split-K: this CTA's fp32 partial tile [token][128 rows] in the workspace
       float* part = nullptr;
-      if (p.cluster_ks > 1) part = reinterpret_cast<float*>(sm);   // the ring is idle once the accumulator is complete
-      else if (p.ksplit > 1)
-        part = p.ws_partial + ((size_t)(tc.rt * p.n_mtiles + tc.mtile) * p.ksplit + tc.split) * (size_t)n_tile * TILE_ROWS;
+      if (cluster_ks > 1) part = reinterpret_cast<float*>(sm);   // the ring is idle once the accumulator is complete
+      else if (ksplit > 1)
+        part = p.ws_partial + ((size_t)(tc.rt * p.n_mtiles + tc.mtile) * ksplit + tc.split) * (size_t)n_tile * TILE_ROWS;
 #pragma unroll 1
       for (int c0 = 0; c0 < n_tile; c0 += 16) {
         uint32_t v[16];
@@ -280,24 +294,24 @@ sdq_linear_kernel(const LinearParams p)
           ptx::named_bar_sync(1, 128);   // the buffer is rewritten by the next chunk
         }
       }
-      if (part && p.cluster_ks <= 1) {
+      if (part && cluster_ks <= 1) {
         // the last CTA of this (row tile, token tile) to finish adds the partial tiles in split order
         __threadfence();
         ptx::named_bar_sync(1, 128);
         uint32_t* counter = p.ws_counter + tc.rt * p.n_mtiles + tc.mtile;
         if (et == 0) {
           const uint32_t old = atomicAdd(counter, 1u);
-          *last_flag = (old == (uint32_t)p.ksplit - 1) ? 1u : 0u;
+          *last_flag = (old == (uint32_t)ksplit - 1) ? 1u : 0u;
         }
         ptx::named_bar_sync(1, 128);
         if (*last_flag) {
           __threadfence();
-          const float* base = p.ws_partial + (size_t)(tc.rt * p.n_mtiles + tc.mtile) * p.ksplit * (size_t)n_tile * TILE_ROWS;
+          const float* base = p.ws_partial + (size_t)(tc.rt * p.n_mtiles + tc.mtile) * ksplit * (size_t)n_tile * TILE_ROWS;
           // 8 tokens at a time: the loads of one split are independent, only the adds follow split order
           for (int t0 = 0; t0 < n_valid; t0 += 8) {
             float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll 2
-            for (int sp = 0; sp < p.ksplit; ++sp) {
+            for (int sp = 0; sp < ksplit; ++sp) {
               const float* src = base + ((size_t)sp * n_tile + t0) * TILE_ROWS + et;
               float v[8];
 #pragma unroll
@@ -319,12 +333,12 @@ sdq_linear_kernel(const LinearParams p)
     }
     if (!ok && lane == 0) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
   }
-  if (p.cluster_ks > 1) {
+  if (cluster_ks > 1) {
     // ---------------- cluster split-K: one tile per CTA; CTA r adds rows [r*128/ks, (r+1)*128/ks) of all members
     ptx::cluster_sync();                         // every member's partial tile is in its shared memory
     if (warp >= 2 && warp <= 5) {
       const uint32_t et = (warp - 2) * 32 + lane;
-      const uint32_t ks = (uint32_t)p.cluster_ks, rank = ptx::cluster_ctarank();
+      const uint32_t ks = (uint32_t)cluster_ks, rank = ptx::cluster_ctarank();
       const uint32_t rows_per = TILE_ROWS / ks;
       const int n_valid = (int)min((int64_t)n_tile, p.M - (int64_t)first_tc.mtile * n_tile);
       const int64_t m0 = (int64_t)first_tc.mtile * n_tile, n0 = (int64_t)first_tc.rt * TILE_ROWS;
@@ -345,7 +359,7 @@ sdq_linear_kernel(const LinearParams p)
   }
   ptx::tc_fence_before();
   __syncthreads();
-  if (warp == 1) ptx::tmem_dealloc(tmem, (uint32_t)p.tmem_cols);
+  if (warp == 1) ptx::tmem_dealloc(tmem, tmem_cols);
 }
 
 }  // namespace sdq
@@ -393,12 +407,14 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   if (Xq->cfg.in_block != P->cfg.in_block || Xq->cfg.scale_rule != P->cfg.scale_rule) return SDQ_ERR_SHAPE;
   if (P->cfg.in_gran != SDQ_GRAN_PAIR || P->cfg.in_block != 64) return SDQ_ERR_UNSUPPORTED;
   if (((uintptr_t)Y & 15) || (ldy % 8) || ((uintptr_t)ws & 15)) return SDQ_ERR_ALIGNMENT;
-  static bool attr_set[2] = {false, false};
-  if (!attr_set[f32]) {
-    cudaError_t e = f32 ? cudaFuncSetAttribute(sdq_linear_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX)
-                        : cudaFuncSetAttribute(sdq_linear_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX);
-    if (e != cudaSuccess) return SDQ_ERR_CUDA;
-    attr_set[f32] = true;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(sdq_linear_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess)
+      return SDQ_ERR_CUDA;
+    attr_set = true;
   }
   const int sm_count = sm_count_cached();
   if (!sm_count) return SDQ_ERR_CUDA;
@@ -471,14 +487,26 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   lc.blockDim = dim3(LIN_THREADS);
   lc.dynamicSmemBytes = (size_t)smem;
   lc.stream = (cudaStream_t)stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)p.cluster_ks;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
+  // early launch pays where per-launch latencies dominate (few tokens); large problems measured slower with it
+  cudaLaunchAttribute attr[2];
+  int na = 0;
+  if (M <= 128) {
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  if (p.cluster_ks > 1) {
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = (unsigned)p.cluster_ks;
+    attr[na].val.clusterDim.y = 1;
+    attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
   lc.attrs = attr;
-  lc.numAttrs = p.cluster_ks > 1 ? 1 : 0;
-  const cudaError_t le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false>, p);
+  lc.numAttrs = na;
+  const bool flex = !(p.n_tile == 256 && p.ksplit == 1 && p.nslot == 5 && p.release == 1);
+  const cudaError_t le = flex ? (f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, true>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, true>, p))
+                              : (f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, false>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, false>, p));
   return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
 }
 

@@ -72,6 +72,8 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
 {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int t = lane >> 2, l = lane & 3;                 // token within the group of 8, quarter of the Q-Vector
+  // a following sdq_linear may start its set-up and weight copies now; it waits for this grid before reading codes
+  if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int64_t m = (int64_t)blockIdx.x * 8 + t;
   const bool live = m < M;
   const int NB = (int)(K / 64);                           // Q-Vectors per row
