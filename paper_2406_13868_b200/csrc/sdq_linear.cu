@@ -22,12 +22,13 @@
 
 namespace sdq {
 
-constexpr int LIN_THREADS = 256;   // warps: 0 weight producer, 1 MMA issuer, 2..5 epilogue, 6 activation producer, 7 scale-atom producer
+constexpr int LIN_THREADS = 288;   // warps: 0 weight producer, 1 MMA issuer, 2..5 epilogue, 6 activation producer, 7 scale-atom producer,
+                                   // 8 metadata / scale mover (many-token instantiation only)
 constexpr int MAX_SLOTS = 16;
 constexpr int SL_A = 0;                        // WI record (A_in | E_in | SFA_in) or WO record (A_out | E_out)
 constexpr int SL_B = 10752;                    // B4 (256 K) or B8 (128 K) of n_tile tokens: n_tile * 128 B
 constexpr int RING_BYTES = 225280;             // largest ring: nslot slots of slot_bytes each
-constexpr int SM_TAIL = 4096 + 320 + 128;      // epilogue transpose buffer (16 tokens x 128 features bf16) + barriers + slack
+constexpr int SM_TAIL = 4096 + 448 + 128;      // epilogue transpose buffer (16 tokens x 128 features bf16) + barriers + slack
 constexpr int LIN_SMEM_MAX = RING_BYTES + SM_TAIL;
 
 // TMEM columns: accumulator at 0 (n_tile columns, tokens), then 52 columns of metadata / scales at `meta_col`:
@@ -78,7 +79,8 @@ sdq_linear_kernel(const LinearParams p)
   const uint32_t tmem_cols = FLEX ? (uint32_t)p.tmem_cols : 512u;
   uint64_t* full = reinterpret_cast<uint64_t*>(sm + SM_BARS);
   uint64_t* empty = full + MAX_SLOTS;
-  uint64_t* acc_full = empty + MAX_SLOTS;
+  uint64_t* meta_full = empty + MAX_SLOTS;          // FLEX = false: metadata / scales of slot s are in TMEM
+  uint64_t* acc_full = meta_full + MAX_SLOTS;
   uint64_t* acc_empty = acc_full + 1;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
   uint32_t* last_flag = tmem_slot + 1;
@@ -95,7 +97,7 @@ sdq_linear_kernel(const LinearParams p)
   const TileCoord first_tc = tile_coord(ksplit, (int)blockIdx.x, RT, T1, T2);
   if (tid == 0) ptx::griddep_launch_dependents();   // the next launch may be scheduled as soon as every CTA got here
   if (tid == 0) {
-    for (uint32_t s = 0; s < nslot; ++s) { ptx::mbar_init(&full[s], 3); ptx::mbar_init(&empty[s], 1); }
+    for (uint32_t s = 0; s < nslot; ++s) { ptx::mbar_init(&full[s], 3); ptx::mbar_init(&empty[s], 1); ptx::mbar_init(&meta_full[s], 1); }
     ptx::mbar_init(acc_full, 1);
     ptx::mbar_init(acc_empty, 4);
     ptx::fence_barrier_init();
@@ -106,7 +108,7 @@ sdq_linear_kernel(const LinearParams p)
   ptx::tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  if (warp == 0 || warp >= 6) {
+  if (warp == 0 || warp == 6 || warp == 7) {
     if (lane == 0) {
       // ---------------- producers: role 0 = weight records, role 1 = activation codes, role 2 = scale atoms.
       // Each arrives once per stage on full[s] with the bytes it is about to copy.
@@ -195,6 +197,32 @@ sdq_linear_kernel(const LinearParams p)
           ptx::tc_fence_after();
         }
         uint32_t acc = 0;   // the first MMA of the tile overwrites the accumulator
+        if constexpr (!FLEX) {
+          // many tokens: warp 8 has already moved the metadata and scales of slot s to TMEM (16 columns per slot, the
+          // outlier scales in one of two per-tile buffers); this thread only issues the MMAs
+          const uint32_t sfo = tmem + 256u + 80u + 12u * (tcount & 1);
+          for (int k = 0; k < ni + no; ++k) {
+            if (!ready) ok = ptx::mbar_wait(&meta_full[s], ph);
+            if (!ok) break;
+            ptx::tc_fence_after();
+            const uint32_t sn = (s + 1 == nslot) ? 0 : s + 1;
+            ready = ptx::mbar_test(&meta_full[sn], sn ? ph : ph ^ 1);
+            const uint64_t so = (uint64_t)(s * slot16);
+            const uint32_t mb = tmem + 256u + 16u * s;
+            if (k < ni) {
+              ptx::mma_sp_mxf4(tmem + TM_D, d_a + so, d_b + so, id4[0], mb, mb + 4, mb + 8, acc);
+              ptx::mma_sp_mxf4(tmem + TM_D, d_a + so + (4096 >> 4), d_b + so + (512 >> 4), id4[1], mb + 2, mb + 4, mb + 8, 1u);
+            } else {
+              ptx::mma_sp_mxf8(tmem + TM_D, d_a + so, d_b + so, id8, mb, sfo, sfo + 4, acc);
+              ptx::mma_sp_mxf8(tmem + TM_D, d_a + so + (4096 >> 4), d_b + so + (512 >> 4), id8, mb + 2, sfo, sfo + 4, 1u);
+            }
+            acc = 1;
+            ptx::tc_commit(&empty[s]);
+            s = sn;
+            if (sn == 0) ph ^= 1;
+          }
+          ptx::tc_commit(acc_full);
+        } else {
         for (int k = 0; k < ni + no; ++k) {
           if (!ready) ok = ptx::mbar_wait(&full[s], ph);
           if (!ok) break;
@@ -231,6 +259,47 @@ sdq_linear_kernel(const LinearParams p)
           if (sn == 0) ph ^= 1;
         }
         ptx::tc_commit(acc_full);
+        }
+      }
+      if (!ok) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
+    }
+  } else if (warp == 8) {
+    if (!FLEX && lane == 0) {
+      // ---------------- metadata / scale mover: smem -> TMEM (tcgen05.cp) for every slot as soon as it has landed, so
+      // that the MMA issuer's instruction stream holds nothing but MMAs.  TMEM buffer s belongs to ring slot s: it is
+      // free again exactly when the slot is (the producers refill a slot only after its MMAs have completed).
+      bool ok = true;
+      const uint32_t smb = ptx::smem_u32(sm);
+      uint32_t s = 0, ph = 0, tcount = 0;
+      const uint64_t d_e_in = ptx::smem_desc(smb + SL_A + A_IN_BYTES, 0, 128);
+      const uint64_t d_sfa_in = ptx::smem_desc(smb + SL_A + A_IN_BYTES + E_IN_BYTES, 0, 128);
+      const uint64_t d_e_out = ptx::smem_desc(smb + SL_A + A_OUT_BYTES, 0, 128);
+      const uint64_t d_sf0 = ptx::smem_desc(smb + sl_sf, 0, 128), d_sf1 = ptx::smem_desc(smb + sl_sf + SF_ATOM_BYTES, 0, 128);
+      const uint64_t d_sf2 = ptx::smem_desc(smb + sl_sf + 2 * SF_ATOM_BYTES, 0, 128);
+      const uint32_t slot16 = slot_bytes >> 4;
+      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
+        const uint32_t sfo = tmem + 256u + 80u + 12u * (tcount & 1);
+        for (int k = 0; k < T2 + T1; ++k) {
+          if (!(ok = ptx::mbar_wait(&full[s], ph))) break;
+          ptx::tc_fence_after();
+          const uint64_t so = (uint64_t)(s * slot16);
+          const uint32_t mb = tmem + 256u + 16u * s;
+          if (k < T2) {
+            ptx::tc_cp_128x128b(mb + 0, d_e_in + so);
+            ptx::tc_cp_32x128b_warpx4(mb + 4, d_sfa_in + so);
+            ptx::tc_cp_32x128b_warpx4(mb + 8, d_sf0 + so);
+            ptx::tc_cp_32x128b_warpx4(mb + 12, d_sf1 + so);
+          } else {
+            ptx::tc_cp_128x128b(mb + 0, d_e_out + so);
+            if (k == T2) {
+              ptx::tc_cp_32x128b_warpx4(sfo, d_sf0 + so);
+              ptx::tc_cp_32x128b_warpx4(sfo + 4, d_sf1 + so);
+              ptx::tc_cp_32x128b_warpx4(sfo + 8, d_sf2 + so);
+            }
+          }
+          ptx::tc_commit(&meta_full[s]);
+          if (++s == nslot) { s = 0; ph ^= 1; }
+        }
       }
       if (!ok) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
     }
