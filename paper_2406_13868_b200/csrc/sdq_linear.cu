@@ -531,9 +531,9 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   const int T1 = p.out_n ? (int)(P->K / K1) : 0, T2 = (int)(P->K / K2);
   const int stages_per_tile = (T2 + p.ksplit - 1) / p.ksplit + (T1 + p.ksplit - 1) / p.ksplit;
   int max_slots = RING_BYTES / p.slot_bytes;
-  if (p.total_tiles > sm_count) {
-    // more CTAs than SMs (few tokens): the grid is one wave only if two CTAs share an SM, so a ring gets half of
-    // an SM's shared memory (228 KB, 1 KB of it reserved per CTA)
+  if (p.cluster_ks > 1 && p.total_tiles > sm_count) {
+    // cluster split K with more CTAs than SMs (few tokens, one tile per CTA): the grid is one wave only if two CTAs
+    // share an SM, so a ring gets half of an SM's shared memory (228 KB, 1 KB of it reserved per CTA)
     const int half = (233472 / 2 - 1024 - SM_TAIL) / p.slot_bytes;
     if (half < max_slots) max_slots = half;
   }
