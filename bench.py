@@ -374,10 +374,9 @@ def run_case(args):
     X = sdq_synth.make_act(M, K, 2, device=str(dev))
     P = sdq.sdq_decompose(W, cfg)
     Y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
-    ws = sdq.make_workspace(M, N, K, cfg, dev)
     for _ in range(args.steps):
         xq = sdq.sdq_quantize_act(X, cfg)
-        sdq.sdq_linear(xq, P, Y, workspace=ws)
+        sdq.sdq_linear(xq, P, Y)
     torch.cuda.synchronize()
     assert sdq.device_status() == 0
     print(json.dumps({"case": args.case, "M": M, "N": N, "K": K, "launches": args.steps}))
