@@ -1,13 +1,15 @@
 // Runtime activation quantization A -> A_i (E2M1 + E8M0 per 64 K) and A_o (E4M3 + per-token power-of-two
 // scale), "we also quantize activations accordingly" (Section 5, Stage 3; A_o / A_i of Section 5.1).
 //
-// Two launches.  `act_amax_kernel` reduces, per token, the largest magnitude of each 1024-K chunk (the
-// per-token 8-bit scale needs the whole row before anything can be stored).  `quant_act_kernel` then encodes:
-// one CTA per (group of 8 tokens = one row group of the tiled operand layout, 1024-K chunk).  A warp works
-// on one 64-K Q-Vector of all 8 tokens at a time: 4 lanes per token, 16 elements (two 16-byte loads) per
-// lane, so the Q-Vector maximum is a 4-lane shuffle and every store instruction writes whole 128-byte lines
-// of the stage-tiled layout (8 tokens x 16 B per core matrix).  Codes come from the hardware E2M1 / E4M3
-// converters and go straight into the layout the GEMM streams.
+// The per-token 8-bit scale needs the whole row before anything can be stored.  Rows up to 16384 long take one
+// launch (`quant_act_fused_kernel`): the CTAs of a thread-block cluster split the Q-Vectors of a group of 8 tokens,
+// keep their elements in registers, exchange the per-token maxima through distributed shared memory and encode.
+// Longer rows take two launches: `act_amax_kernel` reduces, per token, the largest magnitude of each 1024-K chunk,
+// `quant_act_kernel` then encodes, one CTA per (group of 8 tokens = one row group of the tiled operand layout,
+// 1024-K chunk).  In both a warp works on one 64-K Q-Vector of all 8 tokens at a time: 4 lanes per token, 16
+// elements (two 16-byte loads) per lane, so the Q-Vector maximum is a 4-lane shuffle and every store instruction
+// writes whole 128-byte lines of the stage-tiled layout (8 tokens x 16 B per core matrix).  Codes come from the
+// hardware E2M1 / E4M3 converters and go straight into the layout the GEMM streams.
 #include "sdq_codec.cuh"
 #include "sdq_internal.h"
 #include "sdq_layout.h"
@@ -134,6 +136,113 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
   }
 }
 
+// Single pass: the CTAs of a cluster share one group of 8 tokens and split its Q-Vectors; every thread keeps its
+// elements in registers (packed bf16) from the one read of X, the per-token maxima meet through distributed shared
+// memory, and the codes are produced from the registers.  Same arithmetic as the two-kernel path, which stays for
+// rows too long for the register budget (K > 64 * QA_WARPS * QF_MAX_IT * 8 = 16384) and for the block-32 reading.
+constexpr int QF_MAX_IT = 4;                             // Q-Vectors per warp
+template <int IT>
+__global__ void __launch_bounds__(QA_THREADS)
+quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int64_t ldx, sdq_config_t cfg, uint8_t* __restrict__ buf,
+                       ActOffsets off)
+{
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int t = lane >> 2, l = lane & 3;                 // token within the group of 8, quarter of the Q-Vector
+  if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const uint32_t cx = gridDim.x, rank = blockIdx.x;      // cluster = the gridDim.x CTAs of one token group
+  const int64_t m = (int64_t)blockIdx.y * 8 + t;
+  const bool live = m < M;
+  const int NB = (int)(K / 64);
+  const int per_cta = (NB + (int)cx - 1) / (int)cx;
+  const int b_begin = (int)rank * per_cta, b_end = min(NB, b_begin + per_cta);
+  __shared__ float s_warp[QA_WARPS][8];
+  __shared__ float s_all[8][8];                          // [cluster rank][token]: every CTA's maxima, pushed by their owners
+
+  uint4 raw[IT][2];
+  float amax = 0.0f;
+#pragma unroll
+  for (int i = 0; i < IT; ++i) {
+    const int b = b_begin + warp + i * QA_WARPS;
+    raw[i][0] = raw[i][1] = make_uint4(0, 0, 0, 0);
+    if (live && b < b_end) {
+      const uint4* p = reinterpret_cast<const uint4*>(X + m * ldx + (int64_t)b * 64 + l * 16);
+      raw[i][0] = p[0];
+      raw[i][1] = p[1];
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < IT; ++i) {
+    const uint32_t r[8] = {raw[i][0].x, raw[i][0].y, raw[i][0].z, raw[i][0].w, raw[i][1].x, raw[i][1].y, raw[i][1].z, raw[i][1].w};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      amax = fmaxf(amax, sat_abs(__uint_as_float(r[j] << 16)));
+      amax = fmaxf(amax, sat_abs(__uint_as_float(r[j] & 0xFFFF0000u)));
+    }
+  }
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+  if (l == 0) s_warp[warp][t] = amax;
+  __syncthreads();
+  if (tid < 8 * (int)cx) {
+    // thread (peer, token): this CTA's maximum of the token goes into row `rank` of the peer's table
+    const int tok = tid & 7;
+    const uint32_t peer = (uint32_t)tid >> 3;
+    float a = 0.0f;
+#pragma unroll
+    for (int w = 0; w < QA_WARPS; ++w) a = fmaxf(a, s_warp[w][tok]);
+    uint32_t ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"((uint32_t)__cvta_generic_to_shared(&s_all[rank][tok])), "r"(peer));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra), "f"(a) : "memory");
+  }
+  // one barrier: every push is visible after it, and nobody touches another CTA's memory afterwards
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+  float ramax = 0.0f;
+  for (uint32_t c = 0; c < cx; ++c) ramax = fmaxf(ramax, s_all[c][t]);
+  const int e = fp8_scale_exp(ramax);
+  const float s8 = pow2_neg(e);
+
+  const int64_t mt = m / TILE_TOK;
+  const uint32_t tk = (uint32_t)(m % TILE_TOK);
+  const int T1 = (int)(K / K1), T2 = (int)(K / K2);
+  uint8_t* xi_base = buf + off.xi + (size_t)mt * T2 * XI_BYTES;
+  uint8_t* xo_base = buf + off.xo + (size_t)mt * T1 * XO_BYTES;
+  if (live && rank == 0 && warp == 0 && l == 0) {
+    reinterpret_cast<int32_t*>(buf + off.sexp)[m] = e;
+    *reinterpret_cast<uint32_t*>(buf + off.sfb_out + (size_t)mt * SF_ATOM_BYTES + sf_off(tk, 0)) = (uint32_t)(e + 127) * 0x01010101u;
+  }
+#pragma unroll
+  for (int i = 0; i < IT; ++i) {
+    const int b = b_begin + warp + i * QA_WARPS;          // uniform over the warp
+    if (b >= b_end) break;
+    const uint32_t r[8] = {raw[i][0].x, raw[i][0].y, raw[i][0].z, raw[i][0].w, raw[i][1].x, raw[i][1].y, raw[i][1].z, raw[i][1].w};
+    float v[16];
+    float bmax = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      v[2 * j] = sat(__uint_as_float(r[j] << 16));
+      v[2 * j + 1] = sat(__uint_as_float(r[j] & 0xFFFF0000u));
+      bmax = fmaxf(bmax, fmaxf(fabsf(v[2 * j]), fabsf(v[2 * j + 1])));
+    }
+    bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
+    bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
+    const uint32_t c = e8m0_scale_code(bmax, cfg.scale_rule);
+    uint32_t q4[2] = {0, 0}, q8[4] = {0, 0, 0, 0};
+    const float s4 = pow2_inv_e8m0(c);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      q4[j >> 2] |= e2m1x2(v[2 * j] * s4, v[2 * j + 1] * s4) << (8 * (j & 3));
+      q8[j >> 1] |= e4m3x2(v[2 * j] * s8, v[2 * j + 1] * s8) << (16 * (j & 1));
+    }
+    if (!live) continue;
+    const uint32_t k = (uint32_t)b * 64 + l * 16;          // first element of this lane
+    uint8_t* xi = xi_base + (size_t)(k >> 8) * XI_BYTES;
+    uint8_t* xo = xo_base + (size_t)(k >> 7) * XO_BYTES;
+    *reinterpret_cast<uint2*>(xi + b_off(tk, (k & 255) >> 1)) = make_uint2(q4[0], q4[1]);
+    *reinterpret_cast<uint4*>(xo + b_off(tk, k & 127)) = make_uint4(q8[0], q8[1], q8[2], q8[3]);
+    if (l == 0) xi[B4_BYTES + sf_off(tk, (uint32_t)(b & 3))] = (uint8_t)c;
+  }
+}
+
 __global__ void __launch_bounds__(QA_THREADS)
 export_act_kernel(const uint8_t* __restrict__ buf, int64_t M, int64_t K, ActOffsets off, sdq_act_canonical_t out)
 {
@@ -184,10 +293,38 @@ extern "C" sdq_status_t sdq_quantize_act(const void* X, int64_t M, int64_t K, in
   const int n_chunks = (int)((K / 64 + QA_CHUNK_QV - 1) / QA_CHUNK_QV);
   float* partial = reinterpret_cast<float*>((uint8_t*)xq_buf + (tiled ? off.amax : poff.amax));
   const dim3 grid((unsigned)((M + 7) / 8), (unsigned)n_chunks);
+  // cluster size for the single-pass kernel: enough CTAs per token group that a warp keeps at most QF_MAX_IT Q-Vectors
+  const int NB = (int)(K / 64);
+  const int cx = (NB + QA_WARPS * QF_MAX_IT - 1) / (QA_WARPS * QF_MAX_IT);
+  if (tiled && cx <= 8) {
+    const int it = ((NB + cx - 1) / cx + QA_WARPS - 1) / QA_WARPS;      // 1..QF_MAX_IT
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3((unsigned)cx, (unsigned)((M + 7) / 8));
+    lc.blockDim = dim3(QA_THREADS);
+    lc.stream = (cudaStream_t)stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cx;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    const __nv_bfloat16* Xb = (const __nv_bfloat16*)X;
+    uint8_t* bufp = (uint8_t*)xq_buf;
+    cudaError_t le;
+    switch (it) {
+      case 1: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<1>, Xb, M, K, ldx, *cfg, bufp, off); break;
+      case 2: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<2>, Xb, M, K, ldx, *cfg, bufp, off); break;
+      case 3: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<3>, Xb, M, K, ldx, *cfg, bufp, off); break;
+      default: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<4>, Xb, M, K, ldx, *cfg, bufp, off); break;
+    }
+    if (le != cudaSuccess || cudaGetLastError() != cudaSuccess) return SDQ_ERR_CUDA;
+  } else {
   act_amax_kernel<<<grid, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, partial, n_chunks);
   if (tiled) quant_act_kernel<<<grid, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, *cfg, (uint8_t*)xq_buf, off, partial, n_chunks);
   else launch_quant_plain(X, M, K, ldx, *cfg, xq_buf, partial, n_chunks, (cudaStream_t)stream);
   if (cudaGetLastError() != cudaSuccess) return SDQ_ERR_CUDA;
+  }
   out->dev = xq_buf;
   out->bytes = tiled ? off.total : poff.total;
   out->M = M;
