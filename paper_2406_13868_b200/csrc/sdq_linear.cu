@@ -14,6 +14,7 @@
 // fp32 partial tiles go to a caller-provided workspace and the last CTA to arrive adds them in split order
 // (deterministic).  Every wait is bounded; a timeout sets a sticky flag.
 #include <cuda_bf16.h>
+#include <stdlib.h>
 
 #include "sdq_internal.h"
 #include "sdq_layout.h"
@@ -562,14 +563,12 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   lc.blockDim = dim3(LIN_THREADS);
   lc.dynamicSmemBytes = (size_t)smem;
   lc.stream = (cudaStream_t)stream;
-  // early launch pays where per-launch latencies dominate (few tokens); large problems measured slower with it
+  // the kernel may be scheduled while the previous one in the stream drains: set-up and weight copies overlap its tail
   cudaLaunchAttribute attr[2];
   int na = 0;
-  if (M <= 128) {
-    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[na].val.programmaticStreamSerializationAllowed = 1;
-    ++na;
-  }
+  attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[na].val.programmaticStreamSerializationAllowed = 1;
+  ++na;
   if (p.cluster_ks > 1) {
     attr[na].id = cudaLaunchAttributeClusterDimension;
     attr[na].val.clusterDim.x = (unsigned)p.cluster_ks;

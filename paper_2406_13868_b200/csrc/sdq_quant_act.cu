@@ -148,6 +148,8 @@ quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K
 {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int t = lane >> 2, l = lane & 3;                 // token within the group of 8, quarter of the Q-Vector
+  // launched with programmatic stream serialization: X may still be being written by the previous kernel
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const uint32_t cx = gridDim.x, rank = blockIdx.x;      // cluster = the gridDim.x CTAs of one token group
   const int64_t m = (int64_t)blockIdx.y * 8 + t;
@@ -302,13 +304,15 @@ extern "C" sdq_status_t sdq_quantize_act(const void* X, int64_t M, int64_t K, in
     lc.gridDim = dim3((unsigned)cx, (unsigned)((M + 7) / 8));
     lc.blockDim = dim3(QA_THREADS);
     lc.stream = (cudaStream_t)stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)cx;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
-    lc.numAttrs = 1;
+    lc.numAttrs = 2;
     const __nv_bfloat16* Xb = (const __nv_bfloat16*)X;
     uint8_t* bufp = (uint8_t*)xq_buf;
     cudaError_t le;
