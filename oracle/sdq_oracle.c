@@ -134,7 +134,6 @@ int sdqo_fp8_scale_exp(double amax) {
 }
 
 /* magnitude key used by every "largest" selection: the 15 low bits of the bf16 pattern */
-static int mag_key(uint16_t h) { return (int)(h & 0x7FFF); }
 
 static int is_finite_bf16(uint16_t h) { return (h & 0x7F80) != 0x7F80; }
 
@@ -150,10 +149,26 @@ static int is_finite_bf16(uint16_t h) { return (h & 0x7F80) != 0x7F80; }
  *   out_sexp [N]           e of the per-row outlier scale 2^e (int32)
  * returns 0, or -1 on a bad argument, -2 if W holds a non-finite value.
  */
-int sdqo_decompose(const uint16_t* W, int64_t N, int64_t K, const sdqo_config* cfg,
-                   uint8_t* in_code, uint8_t* in_meta, uint8_t* in_scale,
-                   uint8_t* out_code, uint8_t* out_idx, int32_t* out_sexp) {
+/* Significance of element k of a row for the selections of Stage 2 (which values are outliers) and Stage 1 (which
+   values survive pruning).  Without a channel weight it is the magnitude |w| (Section 5, Stage 1: "the most
+   straightforward metric is magnitude").  With one it is the weight-activation product |w| * c[k], c[k] being a
+   per-input-channel activation norm from calibration (Section 5, Stage 1 / Stage 2 and the decomposition-stage
+   sensitivity study: product-based outlier extraction, outliers taken in descending order).  The product is ONE
+   fp32 round-to-nearest multiply so that any implementation can reproduce the order exactly; with c == 1 it is |w|. */
+static float significance(uint16_t w, const float* col_weight, int64_t k) {
+  const float a = (float)fabs(sdqo_bf16_to_double(w));
+  if (!col_weight) return a;
+  volatile float p = a * col_weight[k];
+  return p;
+}
+
+int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_config* cfg, const float* col_weight,
+                          uint8_t* in_code, uint8_t* in_meta, uint8_t* in_scale,
+                          uint8_t* out_code, uint8_t* out_idx, int32_t* out_sexp) {
   if (!W || !cfg || N <= 0 || K <= 0 || K % 64 != 0) return -1;
+  if (col_weight)
+    for (int64_t k = 0; k < K; ++k)
+      if (!(col_weight[k] >= 0.0f) || isinf(col_weight[k])) return -3;
   if (cfg->out_n < 0 || cfg->out_n > 2) return -1;
   if (cfg->in_block != 32 && cfg->in_block != 64) return -1;
   const int on = cfg->out_n, Bs = cfg->in_block;
@@ -163,12 +178,15 @@ int sdqo_decompose(const uint16_t* W, int64_t N, int64_t K, const sdqo_config* c
 
   uint8_t* is_out = (uint8_t*)malloc((size_t)K);   /* 1 where the element went to W_o            */
   uint8_t* kept = (uint8_t*)malloc((size_t)K);     /* 1 where the element is a kept inlier SLOT  */
+  float* sig = (float*)malloc((size_t)K * sizeof(float));
   for (int64_t n = 0; n < N; ++n) {
     const uint16_t* w = W + n * K;
     memset(is_out, 0, (size_t)K);
     memset(kept, 0, (size_t)K);
+    for (int64_t k = 0; k < K; ++k) sig[k] = significance(w[k], col_weight, k);
 
-    /* Stage 2, local outlier extraction: the out_n largest |w| of every S-Vector of 8 */
+    /* Stage 2, local outlier extraction: the out_n most significant values of every S-Vector of 8
+       (largest first, ties to the lower index) */
     double out_amax = 0.0;
     for (int64_t g = 0; g < G8; ++g) {
       int chosen[2] = {-1, -1};
@@ -176,7 +194,7 @@ int sdqo_decompose(const uint16_t* W, int64_t N, int64_t K, const sdqo_config* c
         int best = -1;
         for (int i = 0; i < 8; ++i) {
           if (is_out[8 * g + i]) continue;
-          if (best < 0 || mag_key(w[8 * g + i]) > mag_key(w[8 * g + best])) best = i;
+          if (best < 0 || sig[8 * g + i] > sig[8 * g + best]) best = i;
         }
         is_out[8 * g + best] = 1;
         chosen[t] = best;
@@ -197,13 +215,13 @@ int sdqo_decompose(const uint16_t* W, int64_t N, int64_t K, const sdqo_config* c
         out_code[(n * G8 + g) * on + t] = sdqo_e4m3_encode(ldexp(sdqo_bf16_to_double(w[8 * g + i]), -e));
       }
 
-    /* Stage 1 on the remaining values: N:M magnitude pruning */
+    /* Stage 1 on the remaining values: N:M pruning by significance */
     if (cfg->in_gran == SDQO_GRAN_PAIR) {
       for (int64_t g = 0; g < G8; ++g) {
         float score[4];
         for (int j = 0; j < 4; ++j) {
-          float a0 = is_out[8 * g + 2 * j] ? 0.0f : (float)fabs(sdqo_bf16_to_double(w[8 * g + 2 * j]));
-          float a1 = is_out[8 * g + 2 * j + 1] ? 0.0f : (float)fabs(sdqo_bf16_to_double(w[8 * g + 2 * j + 1]));
+          float a0 = is_out[8 * g + 2 * j] ? 0.0f : sig[8 * g + 2 * j];
+          float a1 = is_out[8 * g + 2 * j + 1] ? 0.0f : sig[8 * g + 2 * j + 1];
           volatile float s = a0 + a1;             /* one fp32 round-to-nearest add */
           score[j] = s;
         }
@@ -220,11 +238,11 @@ int sdqo_decompose(const uint16_t* W, int64_t N, int64_t K, const sdqo_config* c
         int i0 = -1, i1 = -1;
         for (int i = 0; i < 4; ++i) {
           if (is_out[4 * h + i]) continue;
-          if (i0 < 0 || mag_key(w[4 * h + i]) > mag_key(w[4 * h + i0])) i0 = i;
+          if (i0 < 0 || sig[4 * h + i] > sig[4 * h + i0]) i0 = i;
         }
         for (int i = 0; i < 4; ++i) {
           if (is_out[4 * h + i] || i == i0) continue;
-          if (i1 < 0 || mag_key(w[4 * h + i]) > mag_key(w[4 * h + i1])) i1 = i;
+          if (i1 < 0 || sig[4 * h + i] > sig[4 * h + i1]) i1 = i;
         }
         if (i0 > i1) { int t = i0; i0 = i1; i1 = t; }
         in_meta[n * (K / 4) + h] = (uint8_t)(i0 | (i1 << 2));
@@ -256,7 +274,15 @@ int sdqo_decompose(const uint16_t* W, int64_t N, int64_t K, const sdqo_config* c
   }
   free(is_out);
   free(kept);
+  free(sig);
   return 0;
+}
+
+/* magnitude metric: the decomposition of Section 5 with |w| as the significance */
+int sdqo_decompose(const uint16_t* W, int64_t N, int64_t K, const sdqo_config* cfg,
+                   uint8_t* in_code, uint8_t* in_meta, uint8_t* in_scale,
+                   uint8_t* out_code, uint8_t* out_idx, int32_t* out_sexp) {
+  return sdqo_decompose_metric(W, N, K, cfg, (const float*)0, in_code, in_meta, in_scale, out_code, out_idx, out_sexp);
 }
 
 /* Dequantize the canonical arrays of ONE weight matrix back to dense W_i and W_o (fp64, [N][K]). */

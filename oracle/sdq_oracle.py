@@ -72,6 +72,7 @@ def lib():
         L.sdqo_relative_cost.restype = ctypes.c_double
         L.sdqo_relative_cost.argtypes = [ctypes.c_int] * 3
         L.sdqo_decompose.restype = ctypes.c_int
+        L.sdqo_decompose_metric.restype = ctypes.c_int
         L.sdqo_dequant_weights.restype = ctypes.c_int
         L.sdqo_quantize_act.restype = ctypes.c_int
         L.sdqo_linear.restype = ctypes.c_int
@@ -109,7 +110,9 @@ class QAct:
     xq8_sexp: np.ndarray   # [M] i32, per-token scale = 2^xq8_sexp
 
 
-def decompose(W_bits: np.ndarray, cfg: Config) -> Packed:
+def decompose(W_bits: np.ndarray, cfg: Config, col_weight=None) -> Packed:
+    """Stage 2 / 1 / 3 of Section 5.  col_weight: optional per-input-channel activation norm c[k] >= 0 (fp32); the
+    significance of an element is then the weight-activation product |w| * c[k] instead of the magnitude."""
     W_bits = np.ascontiguousarray(W_bits, dtype=np.uint16)
     N, K = W_bits.shape
     nmeta = K // 8 if cfg.in_gran == GRAN_PAIR else K // 4
@@ -120,9 +123,15 @@ def decompose(W_bits: np.ndarray, cfg: Config) -> Packed:
                np.zeros((N, K // 8, on), np.uint8), np.zeros((N, K // 8, on), np.uint8),
                np.zeros((N,), np.int32))
     c = cfg.c()
-    rc = lib().sdqo_decompose(_p(W_bits), ctypes.c_int64(N), ctypes.c_int64(K), ctypes.byref(c),
-                              _p(p.in_code), _p(p.in_meta), _p(p.in_scale), _p(p.out_code), _p(p.out_idx),
-                              _p(p.out_sexp))
+    if col_weight is None:
+        cw = None
+    else:
+        cw_arr = np.ascontiguousarray(col_weight, dtype=np.float32)
+        assert cw_arr.shape == (K,)
+        cw = _p(cw_arr)
+    rc = lib().sdqo_decompose_metric(_p(W_bits), ctypes.c_int64(N), ctypes.c_int64(K), ctypes.byref(c), cw,
+                                     _p(p.in_code), _p(p.in_meta), _p(p.in_scale), _p(p.out_code), _p(p.out_idx),
+                                     _p(p.out_sexp))
     if rc != 0:
         raise ValueError("sdqo_decompose failed: %d" % rc)
     return p

@@ -58,11 +58,14 @@ def top_mask(keys, n):
     return mask
 
 
-def decompose_dense(W_bits, out_n, pair, block, rule_floor):
-    """returns (W_in_hat, W_out_hat, mask_in_slots, mask_out) as dense [N, K] arrays"""
+def decompose_dense(W_bits, out_n, pair, block, rule_floor, col_weight=None):
+    """returns (W_in_hat, W_out_hat, mask_in_slots, mask_out) as dense [N, K] arrays; with col_weight the
+    selections rank by the fp32 product |w| * c[k] instead of |w| (the values that get quantized do not change)"""
     W = bf16_to_f64(W_bits)
     N, K = W.shape
     A = np.abs(W)
+    if col_weight is not None:
+        A = (A.astype(np.float32) * np.asarray(col_weight, dtype=np.float32)[None, :]).astype(np.float32).astype(np.float64)
     mask_out = top_mask(A.reshape(N, K // 8, 8), out_n).reshape(N, K) if out_n else np.zeros((N, K), bool)
     R = np.where(mask_out, 0.0, A)
     if pair:

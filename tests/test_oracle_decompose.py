@@ -185,3 +185,68 @@ def test_activation_inf_saturates_nan_rejected():
     Xb[0, 0] = 0x7FC0
     with pytest.raises(ValueError):
         so.quantize_act(Xb, so.Config())
+
+
+# ---------------------------------------------------------------- weight-activation product metric
+def lognormal_channel_weight(K, seed):
+    rng = np.random.default_rng(seed)
+    c = np.exp(rng.normal(0.0, 1.0, K)).astype(np.float32)
+    c[rng.integers(0, K, max(1, K // 64))] *= 30.0        # a few heavy input channels, as in make_act
+    return c
+
+
+@pytest.mark.parametrize("cfg", CFGS)
+def test_product_metric_with_unit_or_power_of_two_channel_weight_is_the_magnitude_metric(cfg):
+    """|w| * 1 == |w| and |w| * 2^t preserves every order and every tie: the packed arrays must not change"""
+    Wb = tiny_W(32, 512, 7)
+    ref = so.decompose(Wb, cfg)
+    for c in (np.ones(512, np.float32), np.full(512, 2.0 ** -9, np.float32), np.full(512, 64.0, np.float32)):
+        p = so.decompose(Wb, cfg, col_weight=c)
+        for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp"):
+            assert np.array_equal(getattr(p, name), getattr(ref, name)), name
+
+
+def test_product_metric_hand_example():
+    """Section 5 (Stage 1): a tiny weight whose activation is huge matters.  Row of one S-Vector of 8 (padded to 64
+    with zeros): magnitudes pick position 0 (0.5) as the outlier, products with c[7] = 10 pick position 7 (0.09375*10)."""
+    import torch
+    w = np.zeros((1, 64))
+    w[0, :8] = [0.5, 0.125, 0.125, 0.125, 0.125, 0.125, 0.125, 0.09375]
+    Wb = sdq_synth.bf16_bits(torch.from_numpy(w).to(torch.bfloat16))
+    cfg = so.Config(1, so.GRAN_PAIR, 64, so.SCALE_OCP_FLOOR)
+    assert so.decompose(Wb, cfg).out_idx[0, 0, 0] == 0
+    c = np.ones(64, np.float32)
+    c[7] = 10.0
+    p = so.decompose(Wb, cfg, col_weight=c)
+    assert p.out_idx[0, 0, 0] == 7
+    W_in, W_out = so.dequant_weights(p)
+    assert W_out[0, 7] == 0.09375 and np.count_nonzero(W_out[0, :8]) == 1      # the VALUE is untouched by the metric
+    # remaining products: 0.5, 0.125 x6 -> pair scores (0.625, 0.25, 0.25, 0.125): pairs 0 and 1 are kept
+    assert p.in_meta[0, 0] == (0 | (1 << 2))
+    assert W_in[0, 0] == 0.5 and W_in[0, 6] == 0.0 and W_in[0, 7] == 0.0
+
+
+@pytest.mark.parametrize("cfg", CFGS)
+def test_product_metric_matches_independent_dense_definition(cfg):
+    for seed in (3, 4):
+        Wb = tiny_W(40, 512, seed)
+        c = lognormal_channel_weight(512, seed)
+        p = so.decompose(Wb, cfg, col_weight=c)
+        W_in, W_out = so.dequant_weights(p)
+        ref_in, ref_out, slots, mask_out = decompose_dense(Wb, cfg.out_n, cfg.in_gran == so.GRAN_PAIR, cfg.in_block,
+                                                           cfg.scale_rule == so.SCALE_OCP_FLOOR, col_weight=c)
+        assert np.array_equal(W_out, ref_out)
+        assert np.array_equal(W_in, ref_in)
+        N, K = Wb.shape
+        assert ((W_out != 0).reshape(N, K // 8, 8).sum(-1) <= cfg.out_n).all()
+        assert not ((W_in != 0) & (W_out != 0)).any()
+
+
+def test_product_metric_rejects_bad_channel_weight():
+    Wb = tiny_W(4, 64, 0)
+    cfg = CFGS[0]
+    for bad in (-1.0, np.inf, np.nan):
+        c = np.ones(64, np.float32)
+        c[5] = bad
+        with pytest.raises(ValueError):
+            so.decompose(Wb, cfg, col_weight=c)
