@@ -33,7 +33,7 @@ typedef enum {
   SDQ_ERR_ALIGNMENT = 3,        /* pointer or leading dimension not 16-byte aligned          */
   SDQ_ERR_UNSUPPORTED = 4,      /* valid config that this kernel set cannot execute          */
   SDQ_ERR_BUFFER_TOO_SMALL = 5, /* caller buffer smaller than the matching *_size query      */
-  SDQ_ERR_NONFINITE = 6,        /* Inf/NaN weight seen by sdq_decompose                      */
+  SDQ_ERR_NONFINITE = 6,        /* Inf/NaN weight (or bad channel weight) seen by sdq_decompose */
   SDQ_ERR_CUDA = 7,             /* a CUDA runtime call failed (launch error etc.)            */
   SDQ_ERR_TIMEOUT = 8           /* a bounded device-side wait gave up (sticky device status) */
 } sdq_status_t;
@@ -118,6 +118,20 @@ sdq_status_t sdq_packed_size(int64_t N, int64_t K, const sdq_config_t* cfg, size
  *   NONFINITE (buffer contents undefined), CUDA. */
 sdq_status_t sdq_decompose(const void* W_bf16, int64_t N, int64_t K, int64_t ldw, const sdq_config_t* cfg,
                            void* packed_buf, size_t packed_bytes, sdq_packed_t* out, void* stream);
+
+/* The same decomposition with the weight-activation product as the significance metric (Section 5,
+ * Stage 1: "a weight value itself is tiny, [but] the corresponding activation is huge"; the
+ * decomposition-stage study finds product-based outlier extraction best): the selections -- which
+ * out_n values of an S-Vector are outliers and which inlier pairs / elements survive pruning -- rank
+ * by |w[n][k]| * col_weight[k] (one fp32 round-to-nearest multiply, largest first, ties to the lower
+ * k; a pair's score is the fp32 sum of its two products) instead of |w|.  Values, scales and formats
+ * are untouched by the metric.
+ *   col_weight (device) [K] fp32, 16-byte aligned, every entry finite and >= 0 -- typically the norm
+ *   of input channel k over a calibration set.  NULL gives sdq_decompose exactly.
+ *   Errors as sdq_decompose; a negative, infinite or NaN channel weight reports NONFINITE. */
+sdq_status_t sdq_decompose_metric(const void* W_bf16, int64_t N, int64_t K, int64_t ldw, const sdq_config_t* cfg,
+                                  const float* col_weight, void* packed_buf, size_t packed_bytes,
+                                  sdq_packed_t* out, void* stream);
 
 /* Untile a packed weight buffer into the canonical arrays (parity surface). Asynchronous. */
 sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canonical_t* out, void* stream);

@@ -54,7 +54,7 @@ class _ActCanon(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp")]
 
 
-EXPORTS = ["sdq_packed_size", "sdq_decompose", "sdq_packed_export", "sdq_act_size", "sdq_quantize_act", "sdq_act_export",
+EXPORTS = ["sdq_packed_size", "sdq_decompose", "sdq_decompose_metric", "sdq_packed_export", "sdq_act_size", "sdq_quantize_act", "sdq_act_export",
            "sdq_linear", "sdq_linear_f32", "sdq_workspace_size", "sdq_workspace_init", "sdq_linear_ws", "sdq_linear_f32_ws", "sdq_linear_noalloc",
            "sdq_device_status", "sdq_status_string"]
 
@@ -72,6 +72,7 @@ def lib() -> ctypes.CDLL:
         vp, i64, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t
         L.sdq_packed_size.argtypes = [i64, i64, ctypes.POINTER(Config), ctypes.POINTER(sz), ctypes.POINTER(sz)]
         L.sdq_decompose.argtypes = [vp, i64, i64, i64, ctypes.POINTER(Config), vp, sz, ctypes.POINTER(_Packed), vp]
+        L.sdq_decompose_metric.argtypes = [vp, i64, i64, i64, ctypes.POINTER(Config), vp, vp, sz, ctypes.POINTER(_Packed), vp]
         L.sdq_packed_export.argtypes = [ctypes.POINTER(_Packed), ctypes.POINTER(_Canon), vp]
         L.sdq_act_size.argtypes = [i64, i64, ctypes.POINTER(Config), ctypes.POINTER(sz)]
         L.sdq_quantize_act.argtypes = [vp, i64, i64, i64, ctypes.POINTER(Config), vp, sz, ctypes.POINTER(_Act), vp]
@@ -138,8 +139,10 @@ def act_size(M: int, K: int, cfg: Config) -> int:
     return b.value
 
 
-def sdq_decompose(W: torch.Tensor, cfg: Config | None = None, buf: torch.Tensor | None = None) -> PackedWeight:
-    """W [N, K] bf16 CUDA tensor -> packed inlier/outlier parts (sdq_decompose of the C-ABI)."""
+def sdq_decompose(W: torch.Tensor, cfg: Config | None = None, buf: torch.Tensor | None = None,
+                  col_weight: torch.Tensor | None = None) -> PackedWeight:
+    """W [N, K] bf16 CUDA tensor -> packed inlier/outlier parts (sdq_decompose of the C-ABI; with col_weight [K] fp32,
+    sdq_decompose_metric: selections rank by the weight-activation product |w| * col_weight[k])."""
     cfg = cfg or Config()
     _need_cuda(W, "W")
     assert W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
@@ -148,8 +151,14 @@ def sdq_decompose(W: torch.Tensor, cfg: Config | None = None, buf: torch.Tensor 
     if buf is None:
         buf = torch.empty(nbytes, dtype=torch.uint8, device=W.device)
     d = _Packed()
-    _check(lib().sdq_decompose(W.data_ptr(), N, K, W.stride(0), ctypes.byref(cfg), buf.data_ptr(), buf.numel(),
-                               ctypes.byref(d), _stream()), "sdq_decompose")
+    if col_weight is None:
+        _check(lib().sdq_decompose(W.data_ptr(), N, K, W.stride(0), ctypes.byref(cfg), buf.data_ptr(), buf.numel(),
+                                   ctypes.byref(d), _stream()), "sdq_decompose")
+    else:
+        _need_cuda(col_weight, "col_weight")
+        assert col_weight.dtype == torch.float32 and col_weight.shape == (K,) and col_weight.is_contiguous()
+        _check(lib().sdq_decompose_metric(W.data_ptr(), N, K, W.stride(0), ctypes.byref(cfg), col_weight.data_ptr(), buf.data_ptr(),
+                                          buf.numel(), ctypes.byref(d), _stream()), "sdq_decompose_metric")
     return PackedWeight(buf, d, N, K, cfg, algo)
 
 

@@ -56,4 +56,28 @@ __device__ __forceinline__ uint32_t e4m3x2(float x, float y) {
 }
 __device__ __forceinline__ uint32_t e4m3x1(float x) { return (uint32_t)__nv_cvt_float_to_fp8(x, __NV_SATFINITE, __NV_E4M3); }
 
+// selection keys of one S-Vector: the 15-bit magnitude itself, or -- with a per-input-channel weight c[k] -- the bit
+// pattern of the fp32 product |w| * c[k] (one round-to-nearest multiply; non-negative floats order like their bits).
+// Returns nonzero if a channel weight is negative, infinite or NaN.
+__device__ __forceinline__ uint32_t selection_keys(const uint32_t (&key)[8], const float* __restrict__ colw, int g, uint32_t (&skey)[8]) {
+  if (!colw) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) skey[i] = key[i];
+    return 0;
+  }
+  const float4 c0 = reinterpret_cast<const float4*>(colw + 8 * g)[0], c1 = reinterpret_cast<const float4*>(colw + 8 * g)[1];
+  const float c[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+  uint32_t bad = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    bad |= !(c[i] >= 0.0f && c[i] <= 3.4028234663852886e38f);
+    skey[i] = __float_as_uint(__fmul_rn(bf16_bits_to_float(key[i]), c[i]));
+  }
+  return bad;
+}
+// significance of position i as a float (for the pair score)
+__device__ __forceinline__ float key_value(uint32_t key, uint32_t skey, bool weighted) {
+  return weighted ? __uint_as_float(skey) : bf16_bits_to_float(key);
+}
+
 }  // namespace sdq

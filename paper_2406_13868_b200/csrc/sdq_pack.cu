@@ -49,8 +49,8 @@ __device__ __forceinline__ void load_group(const __nv_bfloat16* w, uint32_t (&bi
 }
 
 __global__ void __launch_bounds__(128)
-pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t ldw, sdq_config_t cfg, uint8_t* __restrict__ blob,
-            PackedOffsets off, uint32_t* __restrict__ flags)
+pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t ldw, sdq_config_t cfg, const float* __restrict__ colw,
+            uint8_t* __restrict__ blob, PackedOffsets off, uint32_t* __restrict__ flags)
 {
   const int64_t n = blockIdx.x;
   const int tid = threadIdx.x;
@@ -70,8 +70,10 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
       key[i] = bits[i] & 0x7FFFu;
       bad |= (key[i] >= 0x7F80u);
     }
+    uint32_t skey[8];
+    bad |= selection_keys(key, colw, g, skey);
     int o0, o1;
-    select_outliers(key, out_n, o0, o1);
+    select_outliers(skey, out_n, o0, o1);
     if (o0 >= 0) okey_max = max(okey_max, key[o0]);
     if (o1 >= 0) okey_max = max(okey_max, key[o1]);
   }
@@ -108,15 +110,17 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     load_group(wrow + 8 * g, bits);
 #pragma unroll
     for (int i = 0; i < 8; ++i) key[i] = bits[i] & 0x7FFFu;
+    uint32_t skey[8];
+    selection_keys(key, colw, g, skey);
     int o0, o1;
-    select_outliers(key, out_n, o0, o1);
+    select_outliers(skey, out_n, o0, o1);
 
-    // Stage 1 on the remaining values: keep the 2 pairs (of 4) with the largest |a| + |b|
+    // Stage 1 on the remaining values: keep the 2 pairs (of 4) with the largest summed significance
     float score[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const float a0 = (2 * j == o0 || 2 * j == o1) ? 0.0f : bf16_bits_to_float(key[2 * j]);
-      const float a1 = (2 * j + 1 == o0 || 2 * j + 1 == o1) ? 0.0f : bf16_bits_to_float(key[2 * j + 1]);
+      const float a0 = (2 * j == o0 || 2 * j == o1) ? 0.0f : key_value(key[2 * j], skey[2 * j], colw != nullptr);
+      const float a1 = (2 * j + 1 == o0 || 2 * j + 1 == o1) ? 0.0f : key_value(key[2 * j + 1], skey[2 * j + 1], colw != nullptr);
       score[j] = __fadd_rn(a0, a1);
     }
     int j0 = 0;
@@ -247,8 +251,14 @@ extern "C" sdq_status_t sdq_packed_size(int64_t N, int64_t K, const sdq_config_t
 
 extern "C" sdq_status_t sdq_decompose(const void* W, int64_t N, int64_t K, int64_t ldw, const sdq_config_t* cfg, void* packed_buf,
                                       size_t packed_bytes, sdq_packed_t* out, void* stream)
+{ return sdq_decompose_metric(W, N, K, ldw, cfg, nullptr, packed_buf, packed_bytes, out, stream); }
+
+extern "C" sdq_status_t sdq_decompose_metric(const void* W, int64_t N, int64_t K, int64_t ldw, const sdq_config_t* cfg,
+                                             const float* col_weight, void* packed_buf, size_t packed_bytes, sdq_packed_t* out,
+                                             void* stream)
 {
   if (!W || !packed_buf || !out || !cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
+  if ((uintptr_t)col_weight & 15) return SDQ_ERR_ALIGNMENT;
   if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2 || ldw < K) return SDQ_ERR_SHAPE;
   if (((uintptr_t)W & 15) || ((uintptr_t)packed_buf & 15) || (ldw % 8)) return SDQ_ERR_ALIGNMENT;
   const bool tc = is_tensor_core_reading(*cfg);
@@ -259,8 +269,8 @@ extern "C" sdq_status_t sdq_decompose(const void* W, int64_t N, int64_t K, int64
   uint32_t* flags = device_flags();
   if (!flags) return SDQ_ERR_CUDA;
   if (cudaMemsetAsync(flags + FLAG_NONFINITE, 0, sizeof(uint32_t), st) != cudaSuccess) return SDQ_ERR_CUDA;
-  if (tc) pack_kernel<<<(unsigned)N, 128, 0, st>>>((const __nv_bfloat16*)W, N, K, ldw, *cfg, (uint8_t*)packed_buf, off, flags);
-  else launch_pack_plain(W, N, K, ldw, *cfg, packed_buf, flags, st);
+  if (tc) pack_kernel<<<(unsigned)N, 128, 0, st>>>((const __nv_bfloat16*)W, N, K, ldw, *cfg, col_weight, (uint8_t*)packed_buf, off, flags);
+  else launch_pack_plain(W, N, K, ldw, *cfg, col_weight, packed_buf, flags, st);
   if (cudaGetLastError() != cudaSuccess) return SDQ_ERR_CUDA;
   uint32_t nonfinite = 0;
   if (cudaMemcpyAsync(&nonfinite, flags + FLAG_NONFINITE, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SDQ_ERR_CUDA;

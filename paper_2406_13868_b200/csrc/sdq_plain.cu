@@ -42,8 +42,8 @@ __device__ __forceinline__ void pick_outliers(const uint32_t (&key)[8], int out_
 }
 
 __global__ void __launch_bounds__(128)
-pack_plain_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t ldw, sdq_config_t cfg, uint8_t* __restrict__ blob,
-                  PlainPackedOffsets off, uint32_t* __restrict__ flags)
+pack_plain_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t ldw, sdq_config_t cfg, const float* __restrict__ colw,
+                  uint8_t* __restrict__ blob, PlainPackedOffsets off, uint32_t* __restrict__ flags)
 {
   const int64_t n = blockIdx.x;
   const int tid = threadIdx.x;
@@ -62,8 +62,10 @@ pack_plain_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int
       key[i] = bits[i] & 0x7FFFu;
       bad |= (key[i] >= 0x7F80u);
     }
+    uint32_t skey[8];
+    bad |= selection_keys(key, colw, g, skey);
     int o0, o1;
-    pick_outliers(key, out_n, o0, o1);
+    pick_outliers(skey, out_n, o0, o1);
     if (o0 >= 0) okey_max = max(okey_max, key[o0]);
     if (o1 >= 0) okey_max = max(okey_max, key[o1]);
   }
@@ -85,15 +87,17 @@ pack_plain_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int
     load_group8(wrow + 8 * g, bits);
 #pragma unroll
     for (int i = 0; i < 8; ++i) key[i] = bits[i] & 0x7FFFu;
+    uint32_t skey[8];
+    selection_keys(key, colw, g, skey);
     int o0, o1;
-    pick_outliers(key, out_n, o0, o1);
+    pick_outliers(skey, out_n, o0, o1);
     int slot_pos[4];
     if (pair) {
       float score[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const float a0 = (2 * j == o0 || 2 * j == o1) ? 0.0f : bf16_bits_to_float(key[2 * j]);
-        const float a1 = (2 * j + 1 == o0 || 2 * j + 1 == o1) ? 0.0f : bf16_bits_to_float(key[2 * j + 1]);
+        const float a0 = (2 * j == o0 || 2 * j == o1) ? 0.0f : key_value(key[2 * j], skey[2 * j], colw != nullptr);
+        const float a1 = (2 * j + 1 == o0 || 2 * j + 1 == o1) ? 0.0f : key_value(key[2 * j + 1], skey[2 * j + 1], colw != nullptr);
         score[j] = __fadd_rn(a0, a1);
       }
       int j0 = 0;
@@ -110,7 +114,7 @@ pack_plain_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int
       slot_pos[0] = 2 * j0; slot_pos[1] = 2 * j0 + 1; slot_pos[2] = 2 * j1; slot_pos[3] = 2 * j1 + 1;
       blob[off.in_meta + (size_t)n * G + g] = (uint8_t)(j0 | (j1 << 2));
     } else {
-      // element-wise 2:4: in each group of 4 keep the 2 largest magnitudes among the non-outlier positions
+      // element-wise 2:4: in each group of 4 keep the 2 most significant among the non-outlier positions
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         int i0 = -1, i1 = -1;
@@ -118,13 +122,13 @@ pack_plain_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int
         for (int i = 0; i < 4; ++i) {
           const int p = 4 * h + i;
           if (p == o0 || p == o1) continue;
-          if (i0 < 0 || key[p] > key[4 * h + i0]) i0 = i;
+          if (i0 < 0 || skey[p] > skey[4 * h + i0]) i0 = i;
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int p = 4 * h + i;
           if (p == o0 || p == o1 || i == i0) continue;
-          if (i1 < 0 || key[p] > key[4 * h + i1]) i1 = i;
+          if (i1 < 0 || skey[p] > skey[4 * h + i1]) i1 = i;
         }
         if (i0 > i1) { int t = i0; i0 = i1; i1 = t; }
         slot_pos[2 * h] = 4 * h + i0;
@@ -231,10 +235,11 @@ quant_act_plain_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K
   }
 }
 
-void launch_pack_plain(const void* W, int64_t N, int64_t K, int64_t ldw, const sdq_config_t& cfg, void* buf, uint32_t* flags,
-                       cudaStream_t st)
+void launch_pack_plain(const void* W, int64_t N, int64_t K, int64_t ldw, const sdq_config_t& cfg, const float* col_weight, void* buf,
+                       uint32_t* flags, cudaStream_t st)
 {
-  pack_plain_kernel<<<(unsigned)N, 128, 0, st>>>((const __nv_bfloat16*)W, N, K, ldw, cfg, (uint8_t*)buf, plain_packed_offsets(N, K, cfg), flags);
+  pack_plain_kernel<<<(unsigned)N, 128, 0, st>>>((const __nv_bfloat16*)W, N, K, ldw, cfg, col_weight, (uint8_t*)buf,
+                                                 plain_packed_offsets(N, K, cfg), flags);
 }
 void launch_quant_plain(const void* X, int64_t M, int64_t K, int64_t ldx, const sdq_config_t& cfg, void* buf, const float* partial,
                         int n_chunks, cudaStream_t st)

@@ -42,8 +42,8 @@ inline PlainActOffsets plain_act_offsets(int64_t M, int64_t K, const sdq_config_
   return o;
 }
 
-void launch_pack_plain(const void* W, int64_t N, int64_t K, int64_t ldw, const sdq_config_t& cfg, void* buf, uint32_t* flags,
-                       cudaStream_t st);
+void launch_pack_plain(const void* W, int64_t N, int64_t K, int64_t ldw, const sdq_config_t& cfg, const float* col_weight, void* buf,
+                       uint32_t* flags, cudaStream_t st);
 void launch_quant_plain(const void* X, int64_t M, int64_t K, int64_t ldx, const sdq_config_t& cfg, void* buf, const float* partial,
                         int n_chunks, cudaStream_t st);
 

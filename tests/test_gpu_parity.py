@@ -210,6 +210,44 @@ def test_activation_quantizer_row_lengths(M, K, rule):
         assert np.array_equal(ae[name], getattr(oq, name)), name
 
 
+@pytest.mark.parametrize("gran,block", [(1, 64), (0, 32), (0, 64)])
+@pytest.mark.parametrize("out_n", [0, 1, 2])
+def test_product_metric_packer(gran, block, out_n):
+    """sdq_decompose_metric: selections by |w| * c[k]; packed arrays bit-exact against the oracle for the tensor-core
+    layout and for the literal readings, the product-metric weights run through the GEMM, and bad channel weights are
+    reported."""
+    m = sdq()
+    N, K, M = 256, 1024, 24
+    cfg = m.Config(out_n, gran, block, 0)
+    oc = so.Config(out_n, gran, block, 0)
+    W = sdq_synth.make_weight(N, K, 40 + out_n)
+    rng = np.random.default_rng(17)
+    c = np.exp(rng.normal(0.0, 1.0, K)).astype(np.float32)
+    c[rng.integers(0, K, 12)] *= 30.0
+    c[5] = 0.0                                    # a dead input channel never wins a selection
+    p = m.sdq_decompose(W.cuda(), cfg, col_weight=torch.from_numpy(c).cuda())
+    op = so.decompose(sdq_synth.bf16_bits(W), oc, col_weight=c)
+    pe = {k: v.cpu().numpy() for k, v in m.packed_export(p).items()}
+    for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp"):
+        assert np.array_equal(pe[name], getattr(op, name)), name
+    # it does change the selection (otherwise the test would prove nothing)
+    om = so.decompose(sdq_synth.bf16_bits(W), oc)
+    assert not np.array_equal(op.in_meta, om.in_meta)
+    if gran == m.GRAN_PAIR and block == 64:
+        X = sdq_synth.make_act(M, K, 41)
+        xq = m.sdq_quantize_act(X.cuda(), cfg)
+        y = m.sdq_linear(xq, p, f32=True).cpu().numpy()
+        oq = so.quantize_act(sdq_synth.bf16_bits(X), oc)
+        d, tol = y_close(y, so.linear(oq, op))
+        assert (d <= tol).all()
+    for bad in (-1.0, float("inf"), float("nan")):
+        cb = c.copy()
+        cb[100] = bad
+        with pytest.raises(m.SdqError) as ei:
+            m.sdq_decompose(W.cuda(), cfg, col_weight=torch.from_numpy(cb).cuda())
+        assert ei.value.code == 6
+
+
 def test_packer_ties_zeros_and_negative_zero():
     m = sdq()
     rng = np.random.default_rng(1)
