@@ -9,10 +9,15 @@
 // both into ONE fp32 TMEM accumulator.  Persistent CTAs walk tiles of 128 rows x up to 256 tokens.
 // Warp roles: warps 0, 6, 7 = bulk-copy (TMA) producers for weights, activations and scale atoms (issuing a
 // bulk copy costs one thread ~50 ns, so the copies of a stage are spread over three threads), warp 1 = TMEM
-// owner + MMA issuer (also moves metadata and scale atoms smem -> TMEM with tcgen05.cp), warps 2..5 =
-// epilogue (tcgen05.ld, convert, shared-memory transpose, 16-byte row stores).  For few tokens the K range of a row tile is split over several CTAs; the
-// fp32 partial tiles go to a caller-provided workspace and the last CTA to arrive adds them in split order
-// (deterministic).  Every wait is bounded; a timeout sets a sticky flag.
+// owner + MMA issuer, warps 2..5 = epilogue (tcgen05.ld, convert, shared-memory transpose, 16-byte row stores),
+// warp 8 = mover of metadata and scale atoms smem -> TMEM (tcgen05.cp) in the many-token instantiation; with
+// runtime geometry the MMA issuer does those copies itself.
+// For few tokens the K range of a row tile is split over several CTAs: either a thread-block cluster whose members
+// keep their fp32 partial tiles in shared memory and each add one slice of rows over all members in rank order
+// (no global scratch), or, with a caller-provided workspace, partial tiles in global memory that the last CTA to
+// arrive adds in split order.  Both orders are fixed.  Launches carry programmatic stream serialization: the
+// kernel lets its successor be scheduled at once and itself waits for its predecessor only before it reads
+// activations or writes Y.  Every wait is bounded; a timeout sets a sticky flag.
 #include <cuda_bf16.h>
 #include <stdlib.h>
 
@@ -32,8 +37,11 @@ constexpr int RING_BYTES = 225280;             // largest ring: nslot slots of s
 constexpr int SM_TAIL = 4096 + 448 + 128;      // epilogue transpose buffer (16 tokens x 128 features bf16) + barriers + slack
 constexpr int LIN_SMEM_MAX = RING_BYTES + SM_TAIL;
 
-// TMEM columns: accumulator at 0 (n_tile columns, tokens), then 52 columns of metadata / scales at `meta_col`:
+// TMEM columns: accumulator at 0 (n_tile columns, tokens), then metadata / scales.
+// Runtime geometry: 52 columns at `meta_col`:
 //   +0  2 buffers x 16: E_in 4 | SFA_in 4 | SFB_in 8      +32 2 buffers x 4: E_out      +40 SFA_out 4      +44 SFB_out 8
+// Many tokens (512 columns): 16 columns per ring slot at 256 + 16 s (E 4 | SFA 4 | SFB 8; an outlier stage uses the
+// first 4) and two alternating 12-column buffers of outlier row / token scales at 336.
 constexpr uint32_t TM_D = 0;
 constexpr uint32_t TM_META_COLS = 52;
 
