@@ -160,8 +160,11 @@ quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K
   __shared__ float s_warp[QA_WARPS][8];
   __shared__ float s_all[8][8];                          // [cluster rank][token]: every CTA's maxima, pushed by their owners
 
+  // magnitudes are compared as 15-bit integers, two per 32-bit word (max.u16x2); +-Inf counts as the largest finite
+  // bf16: the maxima are clamped once, the elements only in the (rare) lanes that hold an infinity
   uint4 raw[IT][2];
-  float amax = 0.0f;
+  uint32_t qmax[IT];                                      // this lane's largest magnitude bits of Q-Vector i (16 elements)
+  uint32_t m2 = 0;
 #pragma unroll
   for (int i = 0; i < IT; ++i) {
     const int b = b_begin + warp + i * QA_WARPS;
@@ -175,12 +178,14 @@ quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K
 #pragma unroll
   for (int i = 0; i < IT; ++i) {
     const uint32_t r[8] = {raw[i][0].x, raw[i][0].y, raw[i][0].z, raw[i][0].w, raw[i][1].x, raw[i][1].y, raw[i][1].z, raw[i][1].w};
+    uint32_t q = 0;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      amax = fmaxf(amax, sat_abs(__uint_as_float(r[j] << 16)));
-      amax = fmaxf(amax, sat_abs(__uint_as_float(r[j] & 0xFFFF0000u)));
-    }
+    for (int j = 0; j < 8; ++j) q = __vmaxu2(q, r[j] & 0x7FFF7FFFu);
+    q = max(q & 0xFFFFu, q >> 16);                       // > 0x7F7F: the lane holds an infinity (clamped where used)
+    qmax[i] = q;
+    m2 = max(m2, min(q, 0x7F7Fu));
   }
+  float amax = __uint_as_float(m2 << 16);
   amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
   amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
   if (l == 0) s_warp[warp][t] = amax;
@@ -218,15 +223,19 @@ quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K
     if (b >= b_end) break;
     const uint32_t r[8] = {raw[i][0].x, raw[i][0].y, raw[i][0].z, raw[i][0].w, raw[i][1].x, raw[i][1].y, raw[i][1].z, raw[i][1].w};
     float v[16];
-    float bmax = 0.0f;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      v[2 * j] = sat(__uint_as_float(r[j] << 16));
-      v[2 * j + 1] = sat(__uint_as_float(r[j] & 0xFFFF0000u));
-      bmax = fmaxf(bmax, fmaxf(fabsf(v[2 * j]), fabsf(v[2 * j + 1])));
+      v[2 * j] = __uint_as_float(r[j] << 16);
+      v[2 * j + 1] = __uint_as_float(r[j] & 0xFFFF0000u);
     }
-    bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
-    bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
+    if (qmax[i] > 0x7F7Fu) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) v[j] = sat(v[j]);
+    }
+    uint32_t bm = min(qmax[i], 0x7F7Fu);
+    bm = max(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
+    bm = max(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
+    const float bmax = __uint_as_float(bm << 16);
     const uint32_t c = e8m0_scale_code(bmax, cfg.scale_rule);
     uint32_t q4[2] = {0, 0}, q8[4] = {0, 0, 0, 0};
     const float s4 = pow2_inv_e8m0(c);
