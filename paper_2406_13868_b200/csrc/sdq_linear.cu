@@ -34,7 +34,7 @@ constexpr int MAX_SLOTS = 16;
 constexpr int SL_A = 0;                        // WI record (A_in | E_in | SFA_in) or WO record (A_out | E_out)
 constexpr int SL_B = 10752;                    // B4 (256 K) or B8 (128 K) of n_tile tokens: n_tile * 128 B
 constexpr int RING_BYTES = 225280;             // largest ring: nslot slots of slot_bytes each
-constexpr int SM_TAIL = 4096 + 448 + 128;      // epilogue transpose buffer (16 tokens x 128 features bf16) + barriers + slack
+constexpr int SM_TAIL = 4096 + 640 + 128;      // epilogue transpose buffer (16 tokens x 128 features bf16) + barriers + slack
 constexpr int LIN_SMEM_MAX = RING_BYTES + SM_TAIL;
 
 // TMEM columns: accumulator at 0 (n_tile columns, tokens), then metadata / scales.
@@ -89,7 +89,8 @@ sdq_linear_kernel(const LinearParams p)
   uint64_t* full = reinterpret_cast<uint64_t*>(sm + SM_BARS);
   uint64_t* empty = full + MAX_SLOTS;
   uint64_t* meta_full = empty + MAX_SLOTS;          // FLEX = false: metadata / scales of slot s are in TMEM
-  uint64_t* acc_full = meta_full + MAX_SLOTS;
+  uint64_t* full_w = meta_full + MAX_SLOTS;         // FLEX = false: weight record and scale atoms of slot s have landed
+  uint64_t* acc_full = full_w + MAX_SLOTS;
   uint64_t* acc_empty = acc_full + 1;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
   uint32_t* last_flag = tmem_slot + 1;
@@ -106,7 +107,14 @@ sdq_linear_kernel(const LinearParams p)
   const TileCoord first_tc = tile_coord(ksplit, (int)blockIdx.x, RT, T1, T2);
   if (tid == 0) ptx::griddep_launch_dependents();   // the next launch may be scheduled as soon as every CTA got here
   if (tid == 0) {
-    for (uint32_t s = 0; s < nslot; ++s) { ptx::mbar_init(&full[s], 3); ptx::mbar_init(&empty[s], 1); ptx::mbar_init(&meta_full[s], 1); }
+    // FLEX = false: the weight and scale-atom producers arrive on full_w[s] (the mover starts from it while the
+    // larger activation copies are still landing), the activation producer on full[s]
+    for (uint32_t s = 0; s < nslot; ++s) {
+      ptx::mbar_init(&full[s], FLEX ? 3 : 1);
+      ptx::mbar_init(&empty[s], 1);
+      ptx::mbar_init(&meta_full[s], 1);
+      ptx::mbar_init(&full_w[s], 2);
+    }
     ptx::mbar_init(acc_full, 1);
     ptx::mbar_init(acc_empty, 4);
     ptx::fence_barrier_init();
@@ -140,15 +148,16 @@ sdq_linear_kernel(const LinearParams p)
           if (wrapped && release && !(ok = ptx::mbar_wait(&empty[s], ph ^ 1))) break;
           uint8_t* st = sm + (size_t)s * slot_bytes;
           const bool first_o = (k == ni);
+          uint64_t* bw = FLEX ? &full[s] : &full_w[s];
           if (role == 0) {
             if (k < ni) {
-              ptx::mbar_expect_tx(&full[s], WI_BYTES);
-              ptx::bulk_g2s(st + SL_A, wi, WI_BYTES, &full[s]);
+              ptx::mbar_expect_tx(bw, WI_BYTES);
+              ptx::bulk_g2s(st + SL_A, wi, WI_BYTES, bw);
               wi += WI_BYTES;
             } else {
-              ptx::mbar_expect_tx(&full[s], WO_BYTES + (first_o ? SF_ATOM_BYTES : 0u));
-              ptx::bulk_g2s(st + SL_A, wo, WO_BYTES, &full[s]);
-              if (first_o) ptx::bulk_g2s(st + sl_sf, p.w + p.poff.sfa_out + (size_t)tc.rt * SF_ATOM_BYTES, SF_ATOM_BYTES, &full[s]);
+              ptx::mbar_expect_tx(bw, WO_BYTES + (first_o ? SF_ATOM_BYTES : 0u));
+              ptx::bulk_g2s(st + SL_A, wo, WO_BYTES, bw);
+              if (first_o) ptx::bulk_g2s(st + sl_sf, p.w + p.poff.sfa_out + (size_t)tc.rt * SF_ATOM_BYTES, SF_ATOM_BYTES, bw);
               wo += WO_BYTES;
             }
           } else if (role == 1) {
@@ -162,16 +171,16 @@ sdq_linear_kernel(const LinearParams p)
             }
           } else {
             if (k < ni) {
-              ptx::mbar_expect_tx(&full[s], (uint32_t)have * SF_ATOM_BYTES);
-              for (int a = 0; a < have; ++a) ptx::bulk_g2s(st + sl_sf + a * SF_ATOM_BYTES, xi + a * xi_tile + B4_BYTES, SF_ATOM_BYTES, &full[s]);
+              ptx::mbar_expect_tx(bw, (uint32_t)have * SF_ATOM_BYTES);
+              for (int a = 0; a < have; ++a) ptx::bulk_g2s(st + sl_sf + a * SF_ATOM_BYTES, xi + a * xi_tile + B4_BYTES, SF_ATOM_BYTES, bw);
               xi += XI_BYTES;
             } else if (first_o) {
-              ptx::mbar_expect_tx(&full[s], (uint32_t)have * SF_ATOM_BYTES);
+              ptx::mbar_expect_tx(bw, (uint32_t)have * SF_ATOM_BYTES);
               for (int a = 0; a < have; ++a)
                 ptx::bulk_g2s(st + sl_sf + (1 + a) * SF_ATOM_BYTES, p.x + p.aoff.sfb_out + (size_t)(mt + a) * SF_ATOM_BYTES, SF_ATOM_BYTES,
-                              &full[s]);
+                              bw);
             } else {
-              ptx::mbar_arrive(&full[s]);
+              ptx::mbar_arrive(bw);
             }
           }
           if (++s == nslot) { s = 0; wrapped = 1; ph ^= 1; }
@@ -212,6 +221,7 @@ sdq_linear_kernel(const LinearParams p)
           const uint32_t sfo = tmem + 256u + 80u + 12u * (tcount & 1);
           for (int k = 0; k < ni + no; ++k) {
             if (!ready) ok = ptx::mbar_wait(&meta_full[s], ph);
+            if (ok) ok = ptx::mbar_wait(&full[s], ph);          // the activation codes of the slot
             if (!ok) break;
             ptx::tc_fence_after();
             const uint32_t sn = (s + 1 == nslot) ? 0 : s + 1;
@@ -289,7 +299,7 @@ sdq_linear_kernel(const LinearParams p)
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
         const uint32_t sfo = tmem + 256u + 80u + 12u * (tcount & 1);
         for (int k = 0; k < T2 + T1; ++k) {
-          if (!(ok = ptx::mbar_wait(&full[s], ph))) break;
+          if (!(ok = ptx::mbar_wait(&full_w[s], ph))) break;
           ptx::tc_fence_after();
           const uint64_t so = (uint64_t)(s * slot16);
           const uint32_t mb = tmem + 256u + 16u * s;
