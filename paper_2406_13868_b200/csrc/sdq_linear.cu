@@ -431,16 +431,30 @@ sdq_linear_kernel(const LinearParams p)
       const int n_valid = (int)min((int64_t)n_tile, p.M - (int64_t)first_tc.mtile * n_tile);
       const int64_t m0 = (int64_t)first_tc.mtile * n_tile, n0 = (int64_t)first_tc.rt * TILE_ROWS;
       const uint32_t local = ptx::smem_u32(sm);
-      for (uint32_t idx = et; idx < rows_per * (uint32_t)n_valid; idx += 128) {
-        const uint32_t row = rank * rows_per + idx % rows_per, tok = idx / rows_per;
-        float v[8];
+      // four rows x one token per item: one 16-byte load per member, added in rank order
+      uint32_t peer[8];
 #pragma unroll
-        for (uint32_t sp = 0; sp < 8; ++sp) v[sp] = sp < ks ? ptx::ld_dsmem_f32(local + (tok * TILE_ROWS + row) * 4, sp) : 0.0f;
-        float acc = 0.0f;
+      for (uint32_t sp = 0; sp < 8; ++sp) peer[sp] = ptx::mapa_u32(local, sp < ks ? sp : 0u);
+      const uint32_t q_per = rows_per >> 2;                    // 4, 8 or 16 (ks = 8, 4, 2): a power of two
+      const uint32_t q_shift = 31u - (uint32_t)__clz((int)q_per);
+      for (uint32_t idx = et; idx < q_per * (uint32_t)n_valid; idx += 128) {
+        const uint32_t row = rank * rows_per + ((idx & (q_per - 1)) << 2), tok = idx >> q_shift;
+        const uint32_t off = (tok * TILE_ROWS + row) * 4;
+        float4 v[8];
 #pragma unroll
-        for (uint32_t sp = 0; sp < 8; ++sp) acc += v[sp];          // rank order; absent members contribute +0
-        if (F32_OUT) reinterpret_cast<float*>(p.Y)[(m0 + tok) * p.ldy + n0 + row] = acc;
-        else reinterpret_cast<__nv_bfloat16*>(p.Y)[(m0 + tok) * p.ldy + n0 + row] = __float2bfloat16_rn(acc);
+        for (uint32_t sp = 0; sp < 8; ++sp) v[sp] = sp < ks ? ptx::ld_cluster_f32x4(peer[sp] + off) : make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (uint32_t sp = 0; sp < 8; ++sp) { acc.x += v[sp].x; acc.y += v[sp].y; acc.z += v[sp].z; acc.w += v[sp].w; }   // rank order; absent members add +0
+        if (F32_OUT) {
+          *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.Y) + (m0 + tok) * p.ldy + n0 + row) = acc;
+        } else {
+          const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+          uint2 w;
+          w.x = *reinterpret_cast<const uint32_t*>(&lo);
+          w.y = *reinterpret_cast<const uint32_t*>(&hi);
+          *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.Y) + (m0 + tok) * p.ldy + n0 + row) = w;
+        }
       }
     }
     ptx::cluster_sync();                         // nobody leaves while its shared memory may still be read

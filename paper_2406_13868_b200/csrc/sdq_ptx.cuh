@@ -202,6 +202,12 @@ __device__ __forceinline__ void st_async_v4(uint32_t raddr, uint32_t rbar, uint3
                "r"(b), "r"(c), "r"(d), "r"(rbar)
                : "memory");
 }
+// 16-byte load from a shared::cluster address (see mapa_u32)
+__device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t raddr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(raddr) : "memory");
+  return v;
+}
 __device__ __forceinline__ void tmem_alloc_2cta(uint32_t* smem_slot, uint32_t cols) {  // one full warp in EACH CTA
   asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_slot)), "r"(cols)
                : "memory");
