@@ -536,12 +536,17 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   p.ws_counter = nullptr;
   p.ws_partial = nullptr;
   if (!ws && M <= 128) {
-    // cluster split-K: power-of-two cluster of up to 8 CTAs per row tile; up to 32 tokens the CTAs are small enough
-    // for two per SM, beyond that one per SM
+    // cluster split-K: power-of-two cluster of up to 8 CTAs per row tile
     const int RT = (int)(P->N / TILE_ROWS), T2c = (int)(P->K / K2);
-    const int cta_budget = (M <= 32 ? 2 : 1) * sm_count;
-    int ks = 8;
-    while (ks > 1 && (ks * RT > cta_budget || ks > T2c)) ks >>= 1;
+    // CTAs the grid may have: up to 64 tokens the CTAs are small enough for two per SM; from 65 to 128 tokens two
+    // per SM leave only three ring slots, which pays only when one per SM would leave many SMs idle
+    auto split_for = [&](int cta_budget) {
+      int k = 8;
+      while (k > 1 && (k * RT > cta_budget || k > T2c)) k >>= 1;
+      return k;
+    };
+    int ks = split_for((M <= 64 ? 2 : 1) * sm_count);
+    if (M > 64 && ks * RT * 5 <= sm_count * 3) ks = split_for(2 * sm_count);
     if (ks > 1) { p.ksplit = ks; p.cluster_ks = ks; }
   }
   if (ws) {
