@@ -75,7 +75,7 @@ __device__ __forceinline__ TileCoord tile_coord(int ksplit, int tile, int RT, in
 // geometry constant known at compile time -- the single-thread issue loops are latency-bound, so each runtime
 // parameter they touch costs time.  FLEX = true: geometry from the launch parameters (few tokens, split K).
 template <bool F32_OUT, bool FLEX>
-__global__ void __launch_bounds__(LIN_THREADS, 1)
+__global__ void __maxnreg__(96)   // two 9-warp CTAs share an SM only below ~100 registers per thread
 sdq_linear_kernel(const LinearParams p)
 {
   extern __shared__ uint8_t smem_raw[];
