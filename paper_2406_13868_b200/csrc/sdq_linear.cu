@@ -342,8 +342,32 @@ sdq_linear_kernel(const LinearParams p)
       if (cluster_ks > 1) part = reinterpret_cast<float*>(sm);   // the ring is idle once the accumulator is complete
       else if (ksplit > 1)
         part = p.ws_partial + ((size_t)(tc.rt * p.n_mtiles + tc.mtile) * ksplit + tc.split) * (size_t)n_tile * TILE_ROWS;
+      if (part) {
+        // split K: all n_tile token columns of the partial tile go out (the reduction reads only the valid ones); the
+        // TMEM load of the next 16 columns is in flight while the current 16 are stored
+        uint32_t va[16], vb[16];
+        const uint32_t tbase = tmem + ((q * 32u) << 16) + TM_D;
+        float* dst = part + q * 32 + lane;
+        ptx::tmem_ld_32x32b_x16(tbase, va);
 #pragma unroll 1
-      for (int c0 = 0; c0 < n_tile; c0 += 16) {
+        for (int c0 = 0; c0 < n_tile; c0 += 32) {
+          ptx::tmem_ld_wait();
+          if (c0 + 16 < n_tile) ptx::tmem_ld_32x32b_x16(tbase + (uint32_t)(c0 + 16), vb);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) dst[(size_t)(c0 + j) * TILE_ROWS] = __uint_as_float(va[j]);
+          if (c0 + 16 < n_tile) {
+            ptx::tmem_ld_wait();
+            if (c0 + 32 < n_tile) ptx::tmem_ld_32x32b_x16(tbase + (uint32_t)(c0 + 32), va);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) dst[(size_t)(c0 + 16 + j) * TILE_ROWS] = __uint_as_float(vb[j]);
+          }
+        }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(acc_empty);   // accumulator fully read
+      }
+#pragma unroll 1
+      for (int c0 = 0; c0 < (part ? 0 : n_tile); c0 += 16) {
         uint32_t v[16];
         if (c0 < n_valid) {
           ptx::tmem_ld_32x32b_x16(tmem + ((q * 32u) << 16) + TM_D + (uint32_t)c0, v);
@@ -355,11 +379,7 @@ sdq_linear_kernel(const LinearParams p)
           if (lane == 0) ptx::mbar_arrive(acc_empty);
         }
         if (c0 >= n_valid) continue;  // uniform over the four epilogue warps
-        if (part) {
-#pragma unroll
-          for (int j = 0; j < 16; ++j)
-            if (c0 + j < n_valid) part[(size_t)(c0 + j) * TILE_ROWS + q * 32 + lane] = __uint_as_float(v[j]);
-        } else if (F32_OUT) {
+        if (F32_OUT) {
           float* Y = reinterpret_cast<float*>(p.Y);
 #pragma unroll
           for (int j = 0; j < 16; ++j)
@@ -437,15 +457,9 @@ sdq_linear_kernel(const LinearParams p)
       for (uint32_t sp = 0; sp < 8; ++sp) peer[sp] = ptx::mapa_u32(local, sp < ks ? sp : 0u);
       const uint32_t q_per = rows_per >> 2;                    // 4, 8 or 16 (ks = 8, 4, 2): a power of two
       const uint32_t q_shift = 31u - (uint32_t)__clz((int)q_per);
-      for (uint32_t idx = et; idx < q_per * (uint32_t)n_valid; idx += 128) {
+      const uint32_t n_items = q_per * (uint32_t)n_valid;
+      auto out4 = [&](uint32_t idx, const float4& acc) {
         const uint32_t row = rank * rows_per + ((idx & (q_per - 1)) << 2), tok = idx >> q_shift;
-        const uint32_t off = (tok * TILE_ROWS + row) * 4;
-        float4 v[8];
-#pragma unroll
-        for (uint32_t sp = 0; sp < 8; ++sp) v[sp] = sp < ks ? ptx::ld_cluster_f32x4(peer[sp] + off) : make_float4(0.f, 0.f, 0.f, 0.f);
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (uint32_t sp = 0; sp < 8; ++sp) { acc.x += v[sp].x; acc.y += v[sp].y; acc.z += v[sp].z; acc.w += v[sp].w; }   // rank order; absent members add +0
         if (F32_OUT) {
           *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.Y) + (m0 + tok) * p.ldy + n0 + row) = acc;
         } else {
@@ -455,6 +469,27 @@ sdq_linear_kernel(const LinearParams p)
           w.y = *reinterpret_cast<const uint32_t*>(&hi);
           *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.Y) + (m0 + tok) * p.ldy + n0 + row) = w;
         }
+      };
+      auto item_off = [&](uint32_t idx) { return ((idx >> q_shift) * TILE_ROWS + rank * rows_per + ((idx & (q_per - 1)) << 2)) * 4; };
+      // two items per round: up to 16 loads of 16 bytes in flight per thread
+      for (uint32_t idx = et; idx < n_items; idx += 256) {
+        const uint32_t idx2 = idx + 128;
+        const bool two = idx2 < n_items;
+        const uint32_t off = item_off(idx), off2 = item_off(two ? idx2 : idx);
+        float4 v[8], w[8];
+#pragma unroll
+        for (uint32_t sp = 0; sp < 8; ++sp) {
+          v[sp] = sp < ks ? ptx::ld_cluster_f32x4(peer[sp] + off) : make_float4(0.f, 0.f, 0.f, 0.f);
+          w[sp] = (sp < ks && two) ? ptx::ld_cluster_f32x4(peer[sp] + off2) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), acc2 = acc;
+#pragma unroll
+        for (uint32_t sp = 0; sp < 8; ++sp) {   // rank order; absent members add +0
+          acc.x += v[sp].x; acc.y += v[sp].y; acc.z += v[sp].z; acc.w += v[sp].w;
+          acc2.x += w[sp].x; acc2.y += w[sp].y; acc2.z += w[sp].z; acc2.w += w[sp].w;
+        }
+        out4(idx, acc);
+        if (two) out4(idx2, acc2);
       }
     }
     ptx::cluster_sync();                         // nobody leaves while its shared memory may still be read
