@@ -570,18 +570,24 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   p.cluster_ks = 1;
   p.ws_counter = nullptr;
   p.ws_partial = nullptr;
-  if (!ws && M <= 128) {
-    // cluster split-K: power-of-two cluster of up to 8 CTAs per row tile
-    const int RT = (int)(P->N / TILE_ROWS), T2c = (int)(P->K / K2);
-    // CTAs the grid may have: up to 64 tokens the CTAs are small enough for two per SM; from 65 to 128 tokens two
-    // per SM leave only three ring slots, which pays only when one per SM would leave many SMs idle
+  if (!ws) {
+    // cluster split-K: power-of-two cluster of up to 8 CTAs per (row tile, token tile), one tile per CTA
+    const int tiles = (int)(P->N / TILE_ROWS) * p.n_mtiles, T2c = (int)(P->K / K2);
     auto split_for = [&](int cta_budget) {
       int k = 8;
-      while (k > 1 && (k * RT > cta_budget || k > T2c)) k >>= 1;
+      while (k > 1 && ((int64_t)k * tiles > cta_budget || k > T2c)) k >>= 1;
       return k;
     };
-    int ks = split_for((M <= 64 ? 2 : 1) * sm_count);
-    if (M > 64 && ks * RT * 5 <= sm_count * 3) ks = split_for(2 * sm_count);
+    int ks = 1;
+    if (M <= 128) {
+      // CTAs the grid may have: up to 64 tokens the CTAs are small enough for two per SM; from 65 to 128 tokens two
+      // per SM leave only three ring slots, which pays only when one per SM would leave many SMs idle
+      ks = split_for((M <= 64 ? 2 : 1) * sm_count);
+      if (M > 64 && ks * tiles * 5 <= sm_count * 3) ks = split_for(2 * sm_count);
+    } else if (tiles * 2 <= sm_count) {
+      // a few hundred tokens against a narrow weight matrix: fewer 256-token tiles than half the SMs
+      ks = split_for(sm_count);
+    }
     if (ks > 1) { p.ksplit = ks; p.cluster_ks = ks; }
   }
   if (ws) {
