@@ -81,12 +81,20 @@ def test_several_tiles_long_k():
 
 @pytest.mark.parametrize("M,N,K,out_n", [(129, 256, 512, 1), (256, 256, 768, 1), (300, 512, 1024, 2), (520, 256, 2816, 1),
                                          (384, 512, 512, 0), (1000, 1024, 256, 1)])
-def test_cta_pair_kernel_shapes(M, N, K, out_n):
-    """even number of 128-row tiles and more than 128 tokens: the 256x256 CTA-pair kernel, ragged token tails"""
+def test_more_than_128_tokens_few_tiles(M, N, K, out_n):
+    """more than 128 tokens (256-token tiles, ragged token tails) against narrow matrices: few tiles, so the K range
+    of a tile is split over a cluster"""
     run_case(M, N, K, 100 + M, out_n=out_n)
 
 
-def test_one_hot_readback_pair_kernel():
+@pytest.mark.parametrize("M,N,K,out_n", [(300, 5120, 512, 1), (520, 6400, 256, 2), (257, 9600, 256, 0)])
+def test_persistent_many_token_kernel(M, N, K, out_n):
+    """enough 256-token tiles (80, 150, 150) for the persistent many-token instantiation: one and several tiles per
+    CTA, fewer stages than ring slots, a ragged last token tile"""
+    run_case(M, N, K, 200 + M, out_n=out_n)
+
+
+def test_one_hot_readback_512_tokens():
     m = sdq()
     cfg = m.Config()
     N, K = 256, 512
