@@ -142,7 +142,7 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
 // rows too long for the register budget (K > 64 * QA_WARPS * QF_MAX_IT * 8 = 16384) and for the block-32 reading.
 constexpr int QF_MAX_IT = 4;                             // Q-Vectors per warp
 template <int IT>
-__global__ void __launch_bounds__(QA_THREADS)
+__global__ void __launch_bounds__(QA_THREADS, 4)
 quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int64_t ldx, sdq_config_t cfg, uint8_t* __restrict__ buf,
                        ActOffsets off)
 {
