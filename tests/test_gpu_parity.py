@@ -94,6 +94,24 @@ def test_persistent_many_token_kernel(M, N, K, out_n):
     run_case(M, N, K, 200 + M, out_n=out_n)
 
 
+def _random_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        M = int(rng.choice([rng.integers(1, 17), rng.integers(17, 129), rng.integers(129, 700)]))
+        N = 128 * int(rng.integers(1, 9))
+        K = 256 * int(rng.integers(1, 13))
+        out.append((M, N, K, int(rng.integers(0, 3)), int(rng.integers(0, 2))))
+    return out
+
+
+@pytest.mark.parametrize("M,N,K,out_n,rule", _random_shapes(24, 2024))
+def test_seeded_random_shapes(M, N, K, out_n, rule):
+    """seeded random token counts (few / up to 128 / several hundred), widths, depths, outlier counts and scale rules:
+    every launch geometry the host logic can pick for small problems, full parity each"""
+    run_case(M, N, K, 7 * M + N + K, out_n=out_n, rule=rule)
+
+
 def test_one_hot_readback_512_tokens():
     m = sdq()
     cfg = m.Config()
