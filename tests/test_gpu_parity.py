@@ -274,6 +274,40 @@ def test_product_metric_packer(gran, block, out_n):
         assert ei.value.code == 6
 
 
+@pytest.mark.parametrize("M", [5, 200])
+def test_leading_dimensions_larger_than_the_row(M):
+    """W, X and Y are views into wider buffers (ldw > K, ldx > K, ldy > N); nothing outside the views may be written"""
+    m = sdq()
+    cfg = m.Config()
+    N, K = 256, 512
+    W = sdq_synth.make_weight(N, K, 71)
+    X = sdq_synth.make_act(M, K, 72)
+    Wbig = torch.full((N, K + 64), 7.0, dtype=torch.bfloat16, device="cuda")
+    Xbig = torch.full((M, K + 24), -3.0, dtype=torch.bfloat16, device="cuda")
+    Wbig[:, :K] = W.cuda()
+    Xbig[:, :K] = X.cuda()
+    p = m.sdq_decompose(Wbig[:, :K], cfg)
+    xq = m.sdq_quantize_act(Xbig[:, :K], cfg)
+    Ybig = torch.full((M, N + 40), 123.0, dtype=torch.bfloat16, device="cuda")
+    Y32big = torch.full((M, N + 8), 123.0, dtype=torch.float32, device="cuda")
+    m.sdq_linear(xq, p, Ybig[:, :N])
+    m.sdq_linear(xq, p, Y32big[:, :N], f32=True)
+    assert m.device_status() == 0
+    op = so.decompose(sdq_synth.bf16_bits(W), ocfg())
+    oq = so.quantize_act(sdq_synth.bf16_bits(X), ocfg())
+    pe = {k: v.cpu().numpy() for k, v in m.packed_export(p).items()}
+    ae = {k: v.cpu().numpy() for k, v in m.act_export(xq).items()}
+    for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp"):
+        assert np.array_equal(pe[name], getattr(op, name)), name
+    for name in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp"):
+        assert np.array_equal(ae[name], getattr(oq, name)), name
+    y32 = Y32big[:, :N].cpu().numpy()
+    d, tol = y_close(y32, so.linear(oq, op))
+    assert (d <= tol).all()
+    assert np.array_equal(Ybig[:, :N].float().cpu().numpy(), torch.from_numpy(y32).to(torch.bfloat16).float().numpy())
+    assert (Ybig[:, N:] == 123.0).all() and (Y32big[:, N:] == 123.0).all()
+
+
 def test_packer_ties_zeros_and_negative_zero():
     m = sdq()
     rng = np.random.default_rng(1)
