@@ -142,7 +142,9 @@ sdq_status_t sdq_act_size(int64_t M, int64_t K, const sdq_config_t* cfg, size_t*
 /* "We also quantize activations accordingly" (Section 5, Stage 3; A -> A_o, A_i in Section 5.1):
  * per token and Q-Vector an E8M0 scale and E2M1 codes (A_i); per token a power-of-two scale and
  * E4M3 codes (A_o).  X (device) [M][ldx] bf16; xq_buf (device) >= sdq_act_size bytes; out (host).
- * +-Inf saturates, NaN input is undefined.  Asynchronous on `stream`. */
+ * +-Inf saturates, NaN input is undefined.  Asynchronous on `stream`; for K <= 16384 the one kernel it
+ * enqueues carries programmatic stream serialization and waits for the previous kernel of the stream
+ * before it reads X. */
 sdq_status_t sdq_quantize_act(const void* X_bf16, int64_t M, int64_t K, int64_t ldx, const sdq_config_t* cfg,
                               void* xq_buf, size_t xq_bytes, sdq_act_t* out, void* stream);
 
@@ -153,7 +155,7 @@ sdq_status_t sdq_act_export(const sdq_act_t* Xq, const sdq_act_canonical_t* out,
  * one accumulator: Y[m][n] = sum_k A_i[m][k] W_i[n][k] + sum_k A_o[m][k] W_o[n][k].
  *   Xq, P (host descriptors; K and cfg must agree); Y (device) [M][ldy] bf16 (round to nearest even
  *   of the fp32 accumulator); ldy >= N elements, ldy % 8 == 0.  Asynchronous on `stream`.
- *   For M <= 128 the kernel is enqueued with programmatic stream serialization: it may begin (set-up, reading the packed
+ *   The kernel is enqueued with programmatic stream serialization: it may begin (set-up, reading the packed
  *   weights) while the previous kernel of the stream is still finishing, and waits for that kernel before it
  *   reads Xq or writes Y.  The packed weights must therefore be complete before the call is enqueued
  *   (sdq_decompose synchronises its stream, so a buffer it returned always is).
