@@ -133,6 +133,13 @@ sdq_status_t sdq_decompose_metric(const void* W_bf16, int64_t N, int64_t K, int6
                                   const float* col_weight, void* packed_buf, size_t packed_bytes,
                                   sdq_packed_t* out, void* stream);
 
+/* Calibration helper for sdq_decompose_metric (Section 5, Stage 1: metrics that use calibration data):
+ * col_norm[k] = sqrt(sum over the M tokens of X[m][k]^2), the Euclidean norm of input channel k, accumulated
+ * in token order in fp64 and rounded to fp32 (reproducible).
+ *   X (device) [M][ldx] bf16, 4-byte aligned, ldx >= K, K and ldx even; col_norm (device) [K] fp32.
+ *   Asynchronous on `stream`.  Errors: INVALID_ARG, SHAPE, ALIGNMENT, CUDA. */
+sdq_status_t sdq_channel_norm(const void* X_bf16, int64_t M, int64_t K, int64_t ldx, float* col_norm, void* stream);
+
 /* Untile a packed weight buffer into the canonical arrays (parity surface). Asynchronous. */
 sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canonical_t* out, void* stream);
 

@@ -137,6 +137,14 @@ def decompose(W_bits: np.ndarray, cfg: Config, col_weight=None) -> Packed:
     return p
 
 
+def channel_norm(X_bits: np.ndarray) -> np.ndarray:
+    """Euclidean norm of every input channel over the tokens, c[k] = sqrt(sum_m x[m][k]^2) (the activation statistic
+    of the weight-activation product metric, Section 5 Stage 1), in fp64, returned as fp32."""
+    X_bits = np.ascontiguousarray(X_bits, dtype=np.uint16)
+    x = (X_bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    return np.sqrt((x * x).sum(axis=0)).astype(np.float32)
+
+
 def dequant_weights(p: Packed):
     """Dense fp64 (W_in, W_out), each [N, K]."""
     W_in = np.zeros((p.N, p.K), np.float64)

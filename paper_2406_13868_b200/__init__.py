@@ -54,7 +54,7 @@ class _ActCanon(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp")]
 
 
-EXPORTS = ["sdq_packed_size", "sdq_decompose", "sdq_decompose_metric", "sdq_packed_export", "sdq_act_size", "sdq_quantize_act", "sdq_act_export",
+EXPORTS = ["sdq_packed_size", "sdq_decompose", "sdq_decompose_metric", "sdq_channel_norm", "sdq_packed_export", "sdq_act_size", "sdq_quantize_act", "sdq_act_export",
            "sdq_linear", "sdq_linear_f32", "sdq_workspace_size", "sdq_workspace_init", "sdq_linear_ws", "sdq_linear_f32_ws", "sdq_linear_noalloc",
            "sdq_device_status", "sdq_status_string"]
 
@@ -73,6 +73,7 @@ def lib() -> ctypes.CDLL:
         L.sdq_packed_size.argtypes = [i64, i64, ctypes.POINTER(Config), ctypes.POINTER(sz), ctypes.POINTER(sz)]
         L.sdq_decompose.argtypes = [vp, i64, i64, i64, ctypes.POINTER(Config), vp, sz, ctypes.POINTER(_Packed), vp]
         L.sdq_decompose_metric.argtypes = [vp, i64, i64, i64, ctypes.POINTER(Config), vp, vp, sz, ctypes.POINTER(_Packed), vp]
+        L.sdq_channel_norm.argtypes = [vp, i64, i64, i64, vp, vp]
         L.sdq_packed_export.argtypes = [ctypes.POINTER(_Packed), ctypes.POINTER(_Canon), vp]
         L.sdq_act_size.argtypes = [i64, i64, ctypes.POINTER(Config), ctypes.POINTER(sz)]
         L.sdq_quantize_act.argtypes = [vp, i64, i64, i64, ctypes.POINTER(Config), vp, sz, ctypes.POINTER(_Act), vp]
@@ -160,6 +161,17 @@ def sdq_decompose(W: torch.Tensor, cfg: Config | None = None, buf: torch.Tensor 
         _check(lib().sdq_decompose_metric(W.data_ptr(), N, K, W.stride(0), ctypes.byref(cfg), col_weight.data_ptr(), buf.data_ptr(),
                                           buf.numel(), ctypes.byref(d), _stream()), "sdq_decompose_metric")
     return PackedWeight(buf, d, N, K, cfg, algo)
+
+
+def channel_norm(X: torch.Tensor) -> torch.Tensor:
+    """X [M, K] bf16 CUDA tensor -> fp32 [K]: Euclidean norm of every input channel over the tokens
+    (the per-channel weight of the product metric)."""
+    _need_cuda(X, "X")
+    assert X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    M, K = X.shape
+    c = torch.empty(K, dtype=torch.float32, device=X.device)
+    _check(lib().sdq_channel_norm(X.data_ptr(), M, K, X.stride(0), c.data_ptr(), _stream()), "sdq_channel_norm")
+    return c
 
 
 def sdq_quantize_act(X: torch.Tensor, cfg: Config | None = None, buf: torch.Tensor | None = None) -> QuantAct:

@@ -308,6 +308,27 @@ def test_leading_dimensions_larger_than_the_row(M):
     assert (Ybig[:, N:] == 123.0).all() and (Y32big[:, N:] == 123.0).all()
 
 
+@pytest.mark.parametrize("M,K", [(1, 256), (77, 512), (2048, 4096)])
+def test_channel_norm_and_calibrated_decomposition(M, K):
+    """sdq_channel_norm against the fp64 definition (fp64 accumulation on both sides: equal after rounding to fp32, one
+    ulp allowed), then the whole calibrate -> decompose path: the packer fed with the GPU's norms must reproduce the
+    oracle fed with the same norms bit for bit"""
+    m = sdq()
+    X = sdq_synth.make_act(M, K, 300 + M)
+    c = m.channel_norm(X.cuda())
+    ref = so.channel_norm(sdq_synth.bf16_bits(X))
+    cg = c.cpu().numpy()
+    assert np.all(np.abs(cg.astype(np.float64) - ref.astype(np.float64)) <= np.spacing(ref).astype(np.float64))
+    if K <= 512:
+        cfg = m.Config()
+        W = sdq_synth.make_weight(256, K, 301)
+        p = m.sdq_decompose(W.cuda(), cfg, col_weight=c)
+        op = so.decompose(sdq_synth.bf16_bits(W), ocfg(), col_weight=cg)
+        pe = {k: v.cpu().numpy() for k, v in m.packed_export(p).items()}
+        for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp"):
+            assert np.array_equal(pe[name], getattr(op, name)), name
+
+
 def test_packer_ties_zeros_and_negative_zero():
     m = sdq()
     rng = np.random.default_rng(1)

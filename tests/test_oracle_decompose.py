@@ -250,3 +250,26 @@ def test_product_metric_rejects_bad_channel_weight():
         c[5] = bad
         with pytest.raises(ValueError):
             so.decompose(Wb, cfg, col_weight=c)
+
+
+def test_channel_norm_closed_forms():
+    """c[k] = sqrt(sum_m x[m][k]^2): a constant column of value v over M tokens gives |v| sqrt(M); a one-hot column gives
+    the magnitude of its entry; a 3-4-12 column gives 13; zeros give 0"""
+    import torch
+    M, K = 16, 8
+    x = np.zeros((M, K))
+    x[:, 0] = -0.5                  # 0.5 * sqrt(16) = 2
+    x[5, 1] = 3.0                   # one-hot
+    x[0, 2], x[1, 2], x[2, 2] = 3.0, -4.0, 12.0
+    x[:, 3] = np.arange(M)          # sqrt(sum i^2) = sqrt(1240)
+    Xb = sdq_synth.bf16_bits(torch.from_numpy(x).to(torch.bfloat16))
+    c = so.channel_norm(Xb)
+    assert c.dtype == np.float32 and c.shape == (K,)
+    assert c[0] == 2.0 and c[1] == 3.0 and c[2] == 13.0
+    assert c[3] == np.float32(np.sqrt(1240.0))
+    assert (c[4:] == 0).all()
+    # invariance to the order of the tokens, scaling by a power of two
+    perm = np.random.default_rng(0).permutation(M)
+    assert np.array_equal(so.channel_norm(Xb[perm]), c)
+    Xb4 = sdq_synth.bf16_bits(torch.from_numpy(x * 4).to(torch.bfloat16))
+    assert np.array_equal(so.channel_norm(Xb4), c * 4)
