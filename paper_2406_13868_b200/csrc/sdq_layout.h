@@ -49,6 +49,16 @@ constexpr int B4_BYTES = 16384;       // 128 tokens x 256 K
 constexpr int XI_BYTES = B4_BYTES + SF_ATOM_BYTES;                   // 16896
 constexpr int B8_BYTES = 16384;       // 128 tokens x 128 K
 constexpr int XO_BYTES = B8_BYTES;
+// One scale per 32 logical K (in_block = 32, run by kind::mxf4nvf4 .block16) doubles the scale atoms of the inlier
+// records: one atom per 128-K block (4 scales of 32 K each) instead of one per 256 K (4 scales of 64 K each).
+__host__ __device__ inline int sf_atoms(bool b32) { return b32 ? 2 : 1; }
+__host__ __device__ inline int wi_bytes(bool b32) { return A_IN_BYTES + E_IN_BYTES + sf_atoms(b32) * SF_ATOM_BYTES; }
+__host__ __device__ inline int xi_bytes(bool b32) { return B4_BYTES + sf_atoms(b32) * SF_ATOM_BYTES; }
+// byte of the inlier scale of scale block `blk` (counted inside its 256-K record) of row / token `row` inside the
+// record's scale atoms: block 64 -> atom 0, slot blk (0..3); block 32 -> atom blk / 4, slot blk % 4
+__host__ __device__ inline uint32_t in_sf_off(bool b32, uint32_t row, uint32_t blk) {
+  return (b32 ? (blk >> 2) * SF_ATOM_BYTES : 0u) + (row & 31) * 16 + (row >> 5) * 4 + (blk & 3);
+}
 
 // byte offset inside an operand block of K-blocks of `kb_bytes` whose rows carry `row_bytes` per K-block
 //   A operands: row_bytes 32, kb_bytes 4096 (LBO 128, SBO 256);  B operands: one block, row_bytes 128 (SBO 1024)
@@ -66,12 +76,12 @@ constexpr size_t HEADER_BYTES = 256;
 struct PackedOffsets {
   size_t wi, wo, sfa_out, ocode, oidx, osexp, total;
 };
-inline PackedOffsets packed_offsets(int64_t N, int64_t K, int out_n) {
+inline PackedOffsets packed_offsets(int64_t N, int64_t K, int out_n, bool b32 = false) {
   PackedOffsets o;
   const size_t RT = (size_t)(N / TILE_ROWS), T1 = (size_t)(K / K1), T2 = (size_t)(K / K2);
   auto al = [](size_t x) { return (x + 255) & ~(size_t)255; };
   o.wi = HEADER_BYTES;
-  o.wo = al(o.wi + RT * T2 * WI_BYTES);
+  o.wo = al(o.wi + RT * T2 * (size_t)wi_bytes(b32));
   o.sfa_out = al(o.wo + (out_n ? RT * T1 * WO_BYTES : 0));
   o.ocode = al(o.sfa_out + RT * SF_ATOM_BYTES);
   o.oidx = al(o.ocode + (size_t)N * (size_t)(K / 8) * (size_t)out_n);
@@ -84,13 +94,13 @@ struct ActOffsets {
   size_t xi, xo, sfb_out, sexp, amax, total;
   int64_t MT;
 };
-inline ActOffsets act_offsets(int64_t M, int64_t K) {
+inline ActOffsets act_offsets(int64_t M, int64_t K, bool b32 = false) {
   ActOffsets o;
   const size_t MT = (size_t)((M + TILE_TOK - 1) / TILE_TOK), T1 = (size_t)(K / K1), T2 = (size_t)(K / K2);
   auto al = [](size_t x) { return (x + 255) & ~(size_t)255; };
   o.MT = (int64_t)MT;
   o.xi = 0;
-  o.xo = al(o.xi + MT * T2 * XI_BYTES);
+  o.xo = al(o.xi + MT * T2 * (size_t)xi_bytes(b32));
   o.sfb_out = al(o.xo + MT * T1 * XO_BYTES);
   o.sexp = al(o.sfb_out + MT * SF_ATOM_BYTES);
   o.amax = al(o.sexp + MT * TILE_TOK * 4);                       // per-token chunk maxima [MT*128][ceil(K/1024)] f32

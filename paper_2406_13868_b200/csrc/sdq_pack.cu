@@ -95,7 +95,9 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
   const int64_t rt = n / TILE_ROWS;
   const uint32_t r = (uint32_t)(n % TILE_ROWS);
   const int T1 = (int)(K / K1), T2 = (int)(K / K2);
-  uint8_t* wi_base = blob + off.wi + (size_t)rt * T2 * WI_BYTES;
+  const bool b32 = cfg.in_block == 32;
+  const int wib = wi_bytes(b32);
+  uint8_t* wi_base = blob + off.wi + (size_t)rt * T2 * wib;
   uint8_t* wo_base = blob + off.wo + (size_t)rt * T1 * WO_BYTES;
 
   if (tid == 0) {
@@ -136,7 +138,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     if (j0 > j1) { int t = j0; j0 = j1; j1 = t; }
     const int slot_pos[4] = {2 * j0, 2 * j0 + 1, 2 * j1, 2 * j1 + 1};
 
-    // Stage 3, inliers: Q-Vector (64 K = 8 S-Vectors = 8 lanes) largest kept magnitude -> E8M0 scale
+    // Stage 3, inliers: Q-Vector (64 K = 8 S-Vectors = 8 lanes, or 32 K = 4 lanes) largest kept magnitude -> E8M0 scale
     uint32_t ikey = 0;
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
@@ -145,7 +147,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     }
     ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 1));
     ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 2));
-    ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 4));
+    if (!b32) ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 4));
     const uint32_t c = e8m0_scale_code(bf16_bits_to_float(ikey), cfg.scale_rule);
     float v[4];
 #pragma unroll
@@ -156,7 +158,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     const uint32_t codes = e2m1x2(v[0], v[1]) | (e2m1x2(v[2], v[3]) << 8);
 
     const int k1 = g >> 4, k2 = g >> 5;
-    uint8_t* wi = wi_base + (size_t)k2 * WI_BYTES;
+    uint8_t* wi = wi_base + (size_t)k2 * wib;
     uint8_t* wo = wo_base + (size_t)k1 * WO_BYTES;
     // 32 S-Vectors per 256-K stage, 2 code bytes each: bytes 0..31 = K-block 0, 32..63 = K-block 1
     *reinterpret_cast<uint16_t*>(wi + a_off(r, (uint32_t)(g & 31) * 2)) = (uint16_t)codes;
@@ -164,7 +166,8 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     uint32_t nib = (uint32_t)(j0 | (j1 << 2));
     const uint32_t nib_hi = __shfl_down_sync(0xffffffffu, nib, 1);
     if ((g & 1) == 0) wi[A_IN_BYTES + r * 16 + ((g & 31) >> 1)] = (uint8_t)(nib | (nib_hi << 4));
-    if ((g & 7) == 0) wi[A_IN_BYTES + E_IN_BYTES + sf_off(r, (uint32_t)((g >> 3) & 3))] = (uint8_t)c;
+    if (b32) { if ((g & 3) == 0) wi[A_IN_BYTES + E_IN_BYTES + in_sf_off(true, r, (uint32_t)((g >> 2) & 7))] = (uint8_t)c; }
+    else if ((g & 7) == 0) wi[A_IN_BYTES + E_IN_BYTES + in_sf_off(false, r, (uint32_t)((g >> 3) & 3))] = (uint8_t)c;
 
     if (out_n > 0) {
       // Stage 3, outliers: E4M3 codes of w / 2^e; compact arrays plus the 2:4 embedding the sparse
@@ -208,15 +211,18 @@ export_packed_kernel(const uint8_t* __restrict__ blob, int64_t N, int64_t K, sdq
   const int64_t rt = n / TILE_ROWS;
   const uint32_t r = (uint32_t)(n % TILE_ROWS);
   const int T2 = (int)(K / K2);
-  const uint8_t* wi_base = blob + off.wi + (size_t)rt * T2 * WI_BYTES;
+  const bool b32 = cfg.in_block == 32;
+  const int wib = wi_bytes(b32);
+  const uint8_t* wi_base = blob + off.wi + (size_t)rt * T2 * wib;
   for (int g = threadIdx.x; g < G; g += 128) {
-    const uint8_t* wi = wi_base + (size_t)(g >> 5) * WI_BYTES;
+    const uint8_t* wi = wi_base + (size_t)(g >> 5) * wib;
     const uint32_t codes = *reinterpret_cast<const uint16_t*>(wi + a_off(r, (uint32_t)(g & 31) * 2));
     uint8_t* ic = out.in_code + (size_t)n * (K / 2) + 4 * g;
     ic[0] = codes & 15; ic[1] = (codes >> 4) & 15; ic[2] = (codes >> 8) & 15; ic[3] = (codes >> 12) & 15;
     const uint32_t mb = wi[A_IN_BYTES + r * 16 + ((g & 31) >> 1)];
     out.in_meta[(size_t)n * G + g] = (uint8_t)((g & 1) ? (mb >> 4) : (mb & 15));
-    if ((g & 7) == 0) out.in_scale[(size_t)n * (K / 64) + (g >> 3)] = wi[A_IN_BYTES + E_IN_BYTES + sf_off(r, (uint32_t)((g >> 3) & 3))];
+    if (b32) { if ((g & 3) == 0) out.in_scale[(size_t)n * (K / 32) + (g >> 2)] = wi[A_IN_BYTES + E_IN_BYTES + in_sf_off(true, r, (uint32_t)((g >> 2) & 7))]; }
+    else if ((g & 7) == 0) out.in_scale[(size_t)n * (K / 64) + (g >> 3)] = wi[A_IN_BYTES + E_IN_BYTES + in_sf_off(false, r, (uint32_t)((g >> 3) & 3))];
     for (int t = 0; t < out_n; ++t) {
       out.out_code[((size_t)n * G + g) * out_n + t] = blob[off.ocode + ((size_t)n * G + g) * out_n + t];
       out.out_idx[((size_t)n * G + g) * out_n + t] = blob[off.oidx + ((size_t)n * G + g) * out_n + t];
@@ -238,7 +244,7 @@ extern "C" sdq_status_t sdq_packed_size(int64_t N, int64_t K, const sdq_config_t
 {
   if (!cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
   if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2) return SDQ_ERR_SHAPE;
-  if (bytes) *bytes = is_tensor_core_reading(*cfg) ? packed_offsets(N, K, cfg->out_n).total : plain_packed_offsets(N, K, *cfg).total;
+  if (bytes) *bytes = is_tensor_core_reading(*cfg) ? packed_offsets(N, K, cfg->out_n, cfg->in_block == 32).total : plain_packed_offsets(N, K, *cfg).total;
   if (algorithmic_bytes) {
     // per weight: 4-bit values on half the positions (2) + index metadata (pair-wise: two 2-bit pair indices per 8 =
     // 0.5; element-wise: two 2-bit indices per 4 = 1) + one 8-bit scale per Q-Vector + out_n * (8 value + 3 index
@@ -262,7 +268,7 @@ extern "C" sdq_status_t sdq_decompose_metric(const void* W, int64_t N, int64_t K
   if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2 || ldw < K) return SDQ_ERR_SHAPE;
   if (((uintptr_t)W & 15) || ((uintptr_t)packed_buf & 15) || (ldw % 8)) return SDQ_ERR_ALIGNMENT;
   const bool tc = is_tensor_core_reading(*cfg);
-  const PackedOffsets off = packed_offsets(N, K, cfg->out_n);
+  const PackedOffsets off = packed_offsets(N, K, cfg->out_n, cfg->in_block == 32);
   const PlainPackedOffsets poff = plain_packed_offsets(N, K, *cfg);
   if (packed_bytes < (tc ? off.total : poff.total)) return SDQ_ERR_BUFFER_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
@@ -311,7 +317,7 @@ extern "C" sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canon
     ok = ok && cudaMemcpyAsync(out->out_sexp, b + o.osexp, n * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
     return ok ? SDQ_OK : SDQ_ERR_CUDA;
   }
-  const PackedOffsets off = packed_offsets(P->N, P->K, P->cfg.out_n);
+  const PackedOffsets off = packed_offsets(P->N, P->K, P->cfg.out_n, P->cfg.in_block == 32);
   export_packed_kernel<<<(unsigned)P->N, 128, 0, (cudaStream_t)stream>>>((const uint8_t*)P->dev, P->N, P->K, P->cfg, off, *out);
   return cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
 }

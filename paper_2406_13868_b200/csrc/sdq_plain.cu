@@ -1,9 +1,8 @@
-// The readings of the decomposition that the sparse tensor core cannot execute -- element-wise 2:4 inliers
-// (SDQ_GRAN_ELEM) and / or one scale per 32 logical K (in_block = 32), i.e. the literal "2:4, block-32 MXFP4" wording
-// -- are decompose / quantize / export only.  Their buffers simply hold the canonical arrays (one code per byte,
-// sections in the order of sdq_canonical_t / sdq_act_canonical_t); sdq_linear refuses them.
-// Same algorithm as sdq_pack.cu / sdq_quant_act.cu (Section 5, Stage 2 -> Stage 1 -> Stage 3), same thread mapping:
-// one thread per S-Vector of 8 weights, 4 lanes x 16 elements per token and Q-Vector pair for activations.
+// The reading of the decomposition that the sparse FP4 tensor core cannot execute -- element-wise 2:4 inliers
+// (SDQ_GRAN_ELEM), the literal "2:4" wording -- is decompose / export only.  Its buffer simply holds the canonical
+// arrays (one code per byte, sections in the order of sdq_canonical_t); sdq_linear refuses it.
+// Same algorithm as sdq_pack.cu (Section 5, Stage 2 -> Stage 1 -> Stage 3), same thread mapping: one thread per
+// S-Vector of 8 weights.
 #include "sdq_codec.cuh"
 #include "sdq_internal.h"
 #include "sdq_layout.h"
@@ -171,82 +170,10 @@ pack_plain_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int
   }
 }
 
-// activations, one scale per 32 K: 4 lanes x 16 elements per token and 64 K, a Q-Vector is a lane pair
-__global__ void __launch_bounds__(256)
-quant_act_plain_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int64_t ldx, sdq_config_t cfg, uint8_t* __restrict__ buf,
-                       PlainActOffsets off, const float* __restrict__ partial, int n_chunks)
-{
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int t = lane >> 2, l = lane & 3;
-  const int64_t m = (int64_t)blockIdx.x * 8 + t;
-  const bool live = m < M;
-  const int NB = (int)(K / 64);
-  const int b0 = blockIdx.y * 16;
-  float ramax = 0.0f;
-  if (live)
-    for (int c = l; c < n_chunks; c += 4) ramax = fmaxf(ramax, partial[m * n_chunks + c]);
-  ramax = fmaxf(ramax, __shfl_xor_sync(0xffffffffu, ramax, 1));
-  ramax = fmaxf(ramax, __shfl_xor_sync(0xffffffffu, ramax, 2));
-  const int e = fp8_scale_exp(ramax);
-  const float s8 = pow2_neg(e);
-  if (live && blockIdx.y == 0 && warp == 0 && l == 0) reinterpret_cast<int32_t*>(buf + off.sexp)[m] = e;
-  for (int i = 0; i < 2; ++i) {
-    const int b = b0 + warp + i * 8;
-    if (b >= NB) break;
-    float v[16];
-    if (live) {
-      const __nv_bfloat16* px = X + m * ldx + (int64_t)b * 64 + l * 16;
-      const uint4 a = reinterpret_cast<const uint4*>(px)[0], bb = reinterpret_cast<const uint4*>(px)[1];
-      const uint32_t r[8] = {a.x, a.y, a.z, a.w, bb.x, bb.y, bb.z, bb.w};
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        v[2 * j] = __uint_as_float(r[j] << 16);
-        v[2 * j + 1] = __uint_as_float(r[j] & 0xFFFF0000u);
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 16; ++j) v[j] = 0.0f;
-    }
-    float bmax = 0.0f;
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      v[j] = copysignf(fminf(fabsf(v[j]), 3.3895313892515355e38f), v[j]);
-      bmax = fmaxf(bmax, fabsf(v[j]));
-    }
-    bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
-    if (cfg.in_block == 64) bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
-    const uint32_t c = e8m0_scale_code(bmax, cfg.scale_rule);
-    const float s4 = pow2_inv_e8m0(c);
-    if (!live) continue;
-    const int64_t k = (int64_t)b * 64 + l * 16;
-    uint8_t* c4 = buf + off.xq4_code + (size_t)m * K + k;
-    uint8_t* c8 = buf + off.xq8_code + (size_t)m * K + k;
-    uint32_t q4[4], q8[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const uint32_t a = e2m1x2(v[4 * j] * s4, v[4 * j + 1] * s4), bq = e2m1x2(v[4 * j + 2] * s4, v[4 * j + 3] * s4);
-      q4[j] = (a & 15) | ((a >> 4) << 8) | ((bq & 15) << 16) | ((bq >> 4) << 24);
-      q8[j] = e4m3x2(v[4 * j] * s8, v[4 * j + 1] * s8) | (e4m3x2(v[4 * j + 2] * s8, v[4 * j + 3] * s8) << 16);
-    }
-    *reinterpret_cast<uint4*>(c4) = make_uint4(q4[0], q4[1], q4[2], q4[3]);
-    *reinterpret_cast<uint4*>(c8) = make_uint4(q8[0], q8[1], q8[2], q8[3]);
-    const int Bs = cfg.in_block;
-    if ((k % Bs) == 0) buf[off.xq4_scale + (size_t)m * (K / Bs) + k / Bs] = (uint8_t)c;
-  }
-}
-
 void launch_pack_plain(const void* W, int64_t N, int64_t K, int64_t ldw, const sdq_config_t& cfg, const float* col_weight, void* buf,
                        uint32_t* flags, cudaStream_t st)
 {
   pack_plain_kernel<<<(unsigned)N, 128, 0, st>>>((const __nv_bfloat16*)W, N, K, ldw, cfg, col_weight, (uint8_t*)buf,
                                                  plain_packed_offsets(N, K, cfg), flags);
 }
-void launch_quant_plain(const void* X, int64_t M, int64_t K, int64_t ldx, const sdq_config_t& cfg, void* buf, const float* partial,
-                        int n_chunks, cudaStream_t st)
-{
-  const dim3 grid((unsigned)((M + 7) / 8), (unsigned)n_chunks);
-  quant_act_plain_kernel<<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, M, K, ldx, cfg, (uint8_t*)buf, plain_act_offsets(M, K, cfg), partial,
-                                                 n_chunks);
-}
-
 }  // namespace sdq

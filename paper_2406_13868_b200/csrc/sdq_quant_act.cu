@@ -93,7 +93,9 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
   const int64_t mt = m / TILE_TOK;
   const uint32_t tk = (uint32_t)(m % TILE_TOK);
   const int T1 = (int)(K / K1), T2 = (int)(K / K2);
-  uint8_t* xi_base = buf + off.xi + (size_t)mt * T2 * XI_BYTES;
+  const bool b32 = cfg.in_block == 32;               // one scale per 32 K: a Q-Vector is a lane pair
+  const int xib = xi_bytes(b32);
+  uint8_t* xi_base = buf + off.xi + (size_t)mt * T2 * xib;
   uint8_t* xo_base = buf + off.xo + (size_t)mt * T1 * XO_BYTES;
   if (live && blockIdx.y == 0 && warp == 0 && l == 0) {
     reinterpret_cast<int32_t*>(buf + off.sexp)[m] = e;
@@ -117,7 +119,7 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
       bmax = fmaxf(bmax, fabsf(v[j]));
     }
     bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
-    bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
+    if (!b32) bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
     const uint32_t c = e8m0_scale_code(bmax, cfg.scale_rule);
     uint32_t q4[2] = {0, 0}, q8[4] = {0, 0, 0, 0};
     const float s4 = pow2_inv_e8m0(c);
@@ -128,11 +130,12 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
     }
     if (!live) continue;
     const uint32_t k = (uint32_t)b * 64 + l * 16;          // first element of this lane
-    uint8_t* xi = xi_base + (size_t)(k >> 8) * XI_BYTES;
+    uint8_t* xi = xi_base + (size_t)(k >> 8) * xib;
     uint8_t* xo = xo_base + (size_t)(k >> 7) * XO_BYTES;
     *reinterpret_cast<uint2*>(xi + b_off(tk, (k & 255) >> 1)) = make_uint2(q4[0], q4[1]);
     *reinterpret_cast<uint4*>(xo + b_off(tk, k & 127)) = make_uint4(q8[0], q8[1], q8[2], q8[3]);
-    if (l == 0) xi[B4_BYTES + sf_off(tk, (uint32_t)(b & 3))] = (uint8_t)c;
+    if (b32) { if ((l & 1) == 0) xi[B4_BYTES + in_sf_off(true, tk, (k >> 5) & 7)] = (uint8_t)c; }
+    else if (l == 0) xi[B4_BYTES + in_sf_off(false, tk, (uint32_t)(b & 3))] = (uint8_t)c;
   }
 }
 
@@ -211,7 +214,9 @@ quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K
   const int64_t mt = m / TILE_TOK;
   const uint32_t tk = (uint32_t)(m % TILE_TOK);
   const int T1 = (int)(K / K1), T2 = (int)(K / K2);
-  uint8_t* xi_base = buf + off.xi + (size_t)mt * T2 * XI_BYTES;
+  const bool b32 = cfg.in_block == 32;               // one scale per 32 K: a Q-Vector is a lane pair
+  const int xib = xi_bytes(b32);
+  uint8_t* xi_base = buf + off.xi + (size_t)mt * T2 * xib;
   uint8_t* xo_base = buf + off.xo + (size_t)mt * T1 * XO_BYTES;
   if (live && rank == 0 && warp == 0 && l == 0) {
     reinterpret_cast<int32_t*>(buf + off.sexp)[m] = e;
@@ -234,7 +239,7 @@ quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K
     }
     uint32_t bm = min(qmax[i], 0x7F7Fu);
     bm = max(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
-    bm = max(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
+    if (!b32) bm = max(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
     const float bmax = __uint_as_float(bm << 16);
     const uint32_t c = e8m0_scale_code(bmax, cfg.scale_rule);
     uint32_t q4[2] = {0, 0}, q8[4] = {0, 0, 0, 0};
@@ -246,30 +251,34 @@ quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K
     }
     if (!live) continue;
     const uint32_t k = (uint32_t)b * 64 + l * 16;          // first element of this lane
-    uint8_t* xi = xi_base + (size_t)(k >> 8) * XI_BYTES;
+    uint8_t* xi = xi_base + (size_t)(k >> 8) * xib;
     uint8_t* xo = xo_base + (size_t)(k >> 7) * XO_BYTES;
     *reinterpret_cast<uint2*>(xi + b_off(tk, (k & 255) >> 1)) = make_uint2(q4[0], q4[1]);
     *reinterpret_cast<uint4*>(xo + b_off(tk, k & 127)) = make_uint4(q8[0], q8[1], q8[2], q8[3]);
-    if (l == 0) xi[B4_BYTES + sf_off(tk, (uint32_t)(b & 3))] = (uint8_t)c;
+    if (b32) { if ((l & 1) == 0) xi[B4_BYTES + in_sf_off(true, tk, (k >> 5) & 7)] = (uint8_t)c; }
+    else if (l == 0) xi[B4_BYTES + in_sf_off(false, tk, (uint32_t)(b & 3))] = (uint8_t)c;
   }
 }
 
 __global__ void __launch_bounds__(QA_THREADS)
-export_act_kernel(const uint8_t* __restrict__ buf, int64_t M, int64_t K, ActOffsets off, sdq_act_canonical_t out)
+export_act_kernel(const uint8_t* __restrict__ buf, int64_t M, int64_t K, int in_block, ActOffsets off, sdq_act_canonical_t out)
 {
   const int64_t m = blockIdx.x;
   const int64_t mt = m / TILE_TOK;
   const uint32_t t = (uint32_t)(m % TILE_TOK);
   const int T1 = (int)(K / K1), T2 = (int)(K / K2);
-  const uint8_t* xi_base = buf + off.xi + (size_t)mt * T2 * XI_BYTES;
+  const bool b32 = in_block == 32;
+  const int xib = xi_bytes(b32);
+  const uint8_t* xi_base = buf + off.xi + (size_t)mt * T2 * xib;
   const uint8_t* xo_base = buf + off.xo + (size_t)mt * T1 * XO_BYTES;
   for (int64_t k = threadIdx.x; k < K; k += QA_THREADS) {
-    const uint8_t* xi = xi_base + (size_t)(k >> 8) * XI_BYTES;
+    const uint8_t* xi = xi_base + (size_t)(k >> 8) * xib;
     const uint8_t* xo = xo_base + (size_t)(k >> 7) * XO_BYTES;
     const uint32_t b = xi[b_off(t, (uint32_t)(k & 255) >> 1)];
     out.xq4_code[(size_t)m * K + k] = (uint8_t)((k & 1) ? (b >> 4) : (b & 15));
     out.xq8_code[(size_t)m * K + k] = xo[b_off(t, (uint32_t)(k & 127))];
-    if ((k & 63) == 0) out.xq4_scale[(size_t)m * (K / 64) + (k >> 6)] = xi[B4_BYTES + sf_off(t, (uint32_t)((k >> 6) & 3))];
+    if (b32) { if ((k & 31) == 0) out.xq4_scale[(size_t)m * (K / 32) + (k >> 5)] = xi[B4_BYTES + in_sf_off(true, t, (uint32_t)((k >> 5) & 7))]; }
+    else if ((k & 63) == 0) out.xq4_scale[(size_t)m * (K / 64) + (k >> 6)] = xi[B4_BYTES + in_sf_off(false, t, (uint32_t)((k >> 6) & 3))];
   }
   if (threadIdx.x == 0) out.xq8_sexp[m] = reinterpret_cast<const int32_t*>(buf + off.sexp)[m];
 }
@@ -287,7 +296,7 @@ extern "C" sdq_status_t sdq_act_size(int64_t M, int64_t K, const sdq_config_t* c
 {
   if (!act_cfg_ok(cfg) || !bytes) return SDQ_ERR_INVALID_ARG;
   if (M <= 0 || K <= 0 || K % K2) return SDQ_ERR_SHAPE;
-  *bytes = cfg->in_block == 64 ? act_offsets(M, K).total : plain_act_offsets(M, K, *cfg).total;
+  *bytes = act_offsets(M, K, cfg->in_block == 32).total;
   return SDQ_OK;
 }
 
@@ -297,17 +306,16 @@ extern "C" sdq_status_t sdq_quantize_act(const void* X, int64_t M, int64_t K, in
   if (!X || !xq_buf || !out || !act_cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
   if (M <= 0 || K <= 0 || K % K2 || ldx < K) return SDQ_ERR_SHAPE;
   if (((uintptr_t)X & 15) || ((uintptr_t)xq_buf & 15) || (ldx % 8)) return SDQ_ERR_ALIGNMENT;
-  const bool tiled = cfg->in_block == 64;
-  const ActOffsets off = act_offsets(M, K);
-  const PlainActOffsets poff = plain_act_offsets(M, K, *cfg);
-  if (xq_bytes < (tiled ? off.total : poff.total)) return SDQ_ERR_BUFFER_TOO_SMALL;
+  const bool b32 = cfg->in_block == 32;
+  const ActOffsets off = act_offsets(M, K, b32);
+  if (xq_bytes < off.total) return SDQ_ERR_BUFFER_TOO_SMALL;
   const int n_chunks = (int)((K / 64 + QA_CHUNK_QV - 1) / QA_CHUNK_QV);
-  float* partial = reinterpret_cast<float*>((uint8_t*)xq_buf + (tiled ? off.amax : poff.amax));
+  float* partial = reinterpret_cast<float*>((uint8_t*)xq_buf + off.amax);
   const dim3 grid((unsigned)((M + 7) / 8), (unsigned)n_chunks);
   // cluster size for the single-pass kernel: enough CTAs per token group that a warp keeps at most QF_MAX_IT Q-Vectors
   const int NB = (int)(K / 64);
   const int cx = (NB + QA_WARPS * QF_MAX_IT - 1) / (QA_WARPS * QF_MAX_IT);
-  if (tiled && cx <= 8) {
+  if (cx <= 8) {
     const int it = ((NB + cx - 1) / cx + QA_WARPS - 1) / QA_WARPS;      // 1..QF_MAX_IT
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3((unsigned)cx, (unsigned)((M + 7) / 8));
@@ -334,36 +342,23 @@ extern "C" sdq_status_t sdq_quantize_act(const void* X, int64_t M, int64_t K, in
     if (le != cudaSuccess || cudaGetLastError() != cudaSuccess) return SDQ_ERR_CUDA;
   } else {
   act_amax_kernel<<<grid, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, partial, n_chunks);
-  if (tiled) quant_act_kernel<<<grid, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, *cfg, (uint8_t*)xq_buf, off, partial, n_chunks);
-  else launch_quant_plain(X, M, K, ldx, *cfg, xq_buf, partial, n_chunks, (cudaStream_t)stream);
+  quant_act_kernel<<<grid, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, *cfg, (uint8_t*)xq_buf, off, partial, n_chunks);
   if (cudaGetLastError() != cudaSuccess) return SDQ_ERR_CUDA;
   }
   out->dev = xq_buf;
-  out->bytes = tiled ? off.total : poff.total;
+  out->bytes = off.total;
   out->M = M;
   out->K = K;
   out->cfg = *cfg;
   for (int i = 0; i < 6; ++i) out->off[i] = 0;
-  if (tiled) { out->off[0] = off.xi; out->off[1] = off.xo; out->off[2] = off.sfb_out; out->off[3] = off.sexp; }
-  else { out->off[0] = poff.xq4_code; out->off[1] = poff.xq4_scale; out->off[2] = poff.xq8_code; out->off[3] = poff.sexp; }
+  out->off[0] = off.xi; out->off[1] = off.xo; out->off[2] = off.sfb_out; out->off[3] = off.sexp;
   return SDQ_OK;
 }
 
 extern "C" sdq_status_t sdq_act_export(const sdq_act_t* Xq, const sdq_act_canonical_t* out, void* stream)
 {
   if (!Xq || !out || !Xq->dev || !out->xq4_code || !out->xq4_scale || !out->xq8_code || !out->xq8_sexp) return SDQ_ERR_INVALID_ARG;
-  if (Xq->cfg.in_block != 64) {
-    const PlainActOffsets o = plain_act_offsets(Xq->M, Xq->K, Xq->cfg);
-    const uint8_t* b = (const uint8_t*)Xq->dev;
-    cudaStream_t st = (cudaStream_t)stream;
-    const size_t m = (size_t)Xq->M, k = (size_t)Xq->K;
-    bool ok = cudaMemcpyAsync(out->xq4_code, b + o.xq4_code, m * k, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(out->xq4_scale, b + o.xq4_scale, m * k / (size_t)Xq->cfg.in_block, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(out->xq8_code, b + o.xq8_code, m * k, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(out->xq8_sexp, b + o.sexp, m * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
-    return ok ? SDQ_OK : SDQ_ERR_CUDA;
-  }
-  const ActOffsets off = act_offsets(Xq->M, Xq->K);
-  export_act_kernel<<<(unsigned)Xq->M, QA_THREADS, 0, (cudaStream_t)stream>>>((const uint8_t*)Xq->dev, Xq->M, Xq->K, off, *out);
+  const ActOffsets off = act_offsets(Xq->M, Xq->K, Xq->cfg.in_block == 32);
+  export_act_kernel<<<(unsigned)Xq->M, QA_THREADS, 0, (cudaStream_t)stream>>>((const uint8_t*)Xq->dev, Xq->M, Xq->K, Xq->cfg.in_block, off, *out);
   return cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
 }
