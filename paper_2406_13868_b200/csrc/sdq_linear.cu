@@ -38,16 +38,21 @@ constexpr int SM_TAIL = 4096 + 640 + 128;      // epilogue transpose buffer (16 
 constexpr int LIN_SMEM_MAX = RING_BYTES + SM_TAIL;
 
 // TMEM columns: accumulator at 0 (n_tile columns, tokens), then metadata / scales.
-// Runtime geometry: 52 columns at `meta_col`:
-//   +0  2 buffers x 16: E_in 4 | SFA_in 4 | SFB_in 8      +32 2 buffers x 4: E_out      +40 SFA_out 4      +44 SFB_out 8
+// Runtime geometry: 84 columns at `meta_col`:
+//   +0  2 buffers x 32: E_in 4 | SFA_in 4 or 8 | SFB_in up to 16     +64 2 buffers x 4: E_out     +72 SFA_out 4     +76 SFB_out 8
+//   (one scale per 64 K: SFA_in 4, SFB_in 4 per token tile; per 32 K: one scale word per 128-K block, so twice as many)
 // Many tokens (512 columns): 16 columns per ring slot at 256 + 16 s (E 4 | SFA 4 | SFB 8; an outlier stage uses the
 // first 4) and two alternating 12-column buffers of outlier row / token scales at 336.
 constexpr uint32_t TM_D = 0;
-constexpr uint32_t TM_META_COLS = 52;
+constexpr uint32_t TM_META_COLS = 84;
 
 // slot = | A record 10752 | B n_tile*128 | scale atoms 1536 |  (inlier: SFB_in x n_atiles; first outlier stage:
 // SFA_out | SFB_out x n_atiles)
-__host__ __device__ inline int slot_bytes_for(int n_tile) { return SL_B + n_tile * 128 + 1536; }
+// (one scale per 32 K: the weight record is 512 B longer and an inlier stage carries two scale atoms per token tile)
+__host__ __device__ inline int slot_bytes_for(int n_tile, bool b32 = false) {
+  const int n_atiles = (n_tile + TILE_TOK - 1) / TILE_TOK, atoms = b32 ? (2 * n_atiles > 1 + n_atiles ? 2 * n_atiles : 1 + n_atiles) : 3;
+  return wi_bytes(b32) + n_tile * 128 + atoms * SF_ATOM_BYTES;
+}
 
 struct TileCoord {
   int rt, mtile, split;
@@ -84,7 +89,7 @@ sdq_linear_kernel(const LinearParams p)
   const int ksplit = FLEX ? p.ksplit : 1, cluster_ks = FLEX ? p.cluster_ks : 1;
   const bool release = FLEX ? (p.release != 0) : true;
   const uint32_t SM_STG = FLEX ? (uint32_t)p.ring_bytes : (uint32_t)RING_BYTES, SM_BARS = SM_STG + 4096;
-  const uint32_t TM_I = FLEX ? (uint32_t)p.meta_col : 256u, TM_EO = TM_I + 32, TM_SFA_OUT = TM_I + 40, TM_SFB_OUT = TM_I + 44;
+  const uint32_t TM_I = FLEX ? (uint32_t)p.meta_col : 256u, TM_EO = TM_I + 64, TM_SFA_OUT = TM_I + 72, TM_SFB_OUT = TM_I + 76;
   const uint32_t tmem_cols = FLEX ? (uint32_t)p.tmem_cols : 512u;
   uint64_t* full = reinterpret_cast<uint64_t*>(sm + SM_BARS);
   uint64_t* empty = full + MAX_SLOTS;
@@ -100,7 +105,10 @@ sdq_linear_kernel(const LinearParams p)
   const int T1 = p.out_n ? (int)(p.K / K1) : 0, T2 = (int)(p.K / K2);
   const int n_atiles = (n_tile + TILE_TOK - 1) / TILE_TOK;     // 128-token activation tiles per token tile
   const uint32_t nslot = FLEX ? (uint32_t)p.nslot : 5u, slot_bytes = FLEX ? (uint32_t)p.slot_bytes : 45056u;
-  const uint32_t sl_sf = SL_B + (uint32_t)n_tile * 128u;
+  const bool b32 = FLEX && p.b32;                          // one scale per 32 K (runtime geometry only)
+  const uint32_t wib = (uint32_t)wi_bytes(b32), xib = (uint32_t)xi_bytes(b32), na = b32 ? 2u : 1u;
+  const uint32_t sl_b = wib;                               // B4 / B8 follow the (longest) weight record
+  const uint32_t sl_sf = sl_b + (uint32_t)n_tile * 128u;
 
   // the coordinates of the first tile are worked out by every thread while the barriers and TMEM are being set up
   // (a lone thread needs ~0.5 us for the integer divisions, which would otherwise delay the first copies)
@@ -138,11 +146,11 @@ sdq_linear_kernel(const LinearParams p)
         const int mt = tc.mtile * n_tile / TILE_TOK;
         const int have = min(n_atiles, (int)p.aoff.MT - mt);                 // activation tiles that exist
         const uint32_t tok_bytes = (uint32_t)min(n_tile, TILE_TOK) * 128u;   // bytes per activation tile per stage
-        const uint8_t* wi = p.w + p.poff.wi + ((size_t)tc.rt * T2 + tc.i0) * WI_BYTES;
+        const uint8_t* wi = p.w + p.poff.wi + ((size_t)tc.rt * T2 + tc.i0) * wib;
         const uint8_t* wo = p.w + p.poff.wo + ((size_t)tc.rt * T1 + tc.o0) * WO_BYTES;
-        const uint8_t* xi = p.x + p.aoff.xi + ((size_t)mt * T2 + tc.i0) * XI_BYTES;
+        const uint8_t* xi = p.x + p.aoff.xi + ((size_t)mt * T2 + tc.i0) * xib;
         const uint8_t* xo = p.x + p.aoff.xo + ((size_t)mt * T1 + tc.o0) * XO_BYTES;
-        const size_t xi_tile = (size_t)T2 * XI_BYTES, xo_tile = (size_t)T1 * XO_BYTES;
+        const size_t xi_tile = (size_t)T2 * xib, xo_tile = (size_t)T1 * XO_BYTES;
         const int ni = tc.i1 - tc.i0, no = tc.o1 - tc.o0;
         for (int k = 0; k < ni + no; ++k) {
           if (wrapped && release && !(ok = ptx::mbar_wait(&empty[s], ph ^ 1))) break;
@@ -151,9 +159,9 @@ sdq_linear_kernel(const LinearParams p)
           uint64_t* bw = FLEX ? &full[s] : &full_w[s];
           if (role == 0) {
             if (k < ni) {
-              ptx::mbar_expect_tx(bw, WI_BYTES);
-              ptx::bulk_g2s(st + SL_A, wi, WI_BYTES, bw);
-              wi += WI_BYTES;
+              ptx::mbar_expect_tx(bw, wib);
+              ptx::bulk_g2s(st + SL_A, wi, wib, bw);
+              wi += wib;
             } else {
               ptx::mbar_expect_tx(bw, WO_BYTES + (first_o ? SF_ATOM_BYTES : 0u));
               ptx::bulk_g2s(st + SL_A, wo, WO_BYTES, bw);
@@ -163,17 +171,18 @@ sdq_linear_kernel(const LinearParams p)
           } else if (role == 1) {
             ptx::mbar_expect_tx(&full[s], (uint32_t)have * tok_bytes);
             if (k < ni) {
-              for (int a = 0; a < have; ++a) ptx::bulk_g2s(st + SL_B + a * B4_BYTES, xi + a * xi_tile, tok_bytes, &full[s]);
-              xi += XI_BYTES;
+              for (int a = 0; a < have; ++a) ptx::bulk_g2s(st + sl_b + a * B4_BYTES, xi + a * xi_tile, tok_bytes, &full[s]);
+              xi += xib;
             } else {
-              for (int a = 0; a < have; ++a) ptx::bulk_g2s(st + SL_B + a * B8_BYTES, xo + a * xo_tile, tok_bytes, &full[s]);
+              for (int a = 0; a < have; ++a) ptx::bulk_g2s(st + sl_b + a * B8_BYTES, xo + a * xo_tile, tok_bytes, &full[s]);
               xo += XO_BYTES;
             }
           } else {
             if (k < ni) {
-              ptx::mbar_expect_tx(bw, (uint32_t)have * SF_ATOM_BYTES);
-              for (int a = 0; a < have; ++a) ptx::bulk_g2s(st + sl_sf + a * SF_ATOM_BYTES, xi + a * xi_tile + B4_BYTES, SF_ATOM_BYTES, bw);
-              xi += XI_BYTES;
+              ptx::mbar_expect_tx(bw, (uint32_t)have * na * SF_ATOM_BYTES);
+              for (int a = 0; a < have; ++a)
+                ptx::bulk_g2s(st + sl_sf + a * na * SF_ATOM_BYTES, xi + a * xi_tile + B4_BYTES, na * SF_ATOM_BYTES, bw);
+              xi += xib;
             } else if (first_o) {
               ptx::mbar_expect_tx(bw, (uint32_t)have * SF_ATOM_BYTES);
               for (int a = 0; a < have; ++a)
@@ -199,7 +208,7 @@ sdq_linear_kernel(const LinearParams p)
                                ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, true, 2, 2)};
       const uint32_t id8 = ptx::idesc_block_scaled(128, (uint32_t)n_tile, 0, true, 0, 0);
       // descriptors of slot 0; slot s adds s * slot_bytes / 16 to the start-address field
-      const uint64_t d_a = ptx::smem_desc(smb + SL_A, 128, 256), d_b = ptx::smem_desc(smb + SL_B, 128, 1024);
+      const uint64_t d_a = ptx::smem_desc(smb + SL_A, 128, 256), d_b = ptx::smem_desc(smb + sl_b, 128, 1024);
       const uint64_t d_e_in = ptx::smem_desc(smb + SL_A + A_IN_BYTES, 0, 128);
       const uint64_t d_sfa_in = ptx::smem_desc(smb + SL_A + A_IN_BYTES + E_IN_BYTES, 0, 128);
       const uint64_t d_e_out = ptx::smem_desc(smb + SL_A + A_OUT_BYTES, 0, 128);
@@ -252,13 +261,25 @@ sdq_linear_kernel(const LinearParams p)
           const uint64_t so = (uint64_t)(s * slot16);
           if (k < ni) {
             // inlier stage: 256 logical K = 2 sparse MXFP4 MMAs; metadata and scale atoms go to TMEM first
-            const uint32_t mb = tmem + TM_I + 16u * (uint32_t)(k & 1);
+            const uint32_t mb = tmem + TM_I + 32u * (uint32_t)(k & 1);
             ptx::tc_cp_128x128b(mb + 0, d_e_in + so);
             ptx::tc_cp_32x128b_warpx4(mb + 4, d_sfa_in + so);
-            ptx::tc_cp_32x128b_warpx4(mb + 8, d_sf0 + so);
-            if (n_atiles > 1) ptx::tc_cp_32x128b_warpx4(mb + 12, d_sf1 + so);
-            ptx::mma_sp_mxf4(tmem + TM_D, d_a + so, d_b + so, id4[0], mb, mb + 4, mb + 8, acc);
-            ptx::mma_sp_mxf4(tmem + TM_D, d_a + so + (4096 >> 4), d_b + so + (512 >> 4), id4[1], mb + 2, mb + 4, mb + 8, 1u);
+            if (!b32) {
+              ptx::tc_cp_32x128b_warpx4(mb + 8, d_sf0 + so);
+              if (n_atiles > 1) ptx::tc_cp_32x128b_warpx4(mb + 12, d_sf1 + so);
+              ptx::mma_sp_mxf4(tmem + TM_D, d_a + so, d_b + so, id4[0], mb, mb + 4, mb + 8, acc);
+              ptx::mma_sp_mxf4(tmem + TM_D, d_a + so + (4096 >> 4), d_b + so + (512 >> 4), id4[1], mb + 2, mb + 4, mb + 8, 1u);
+            } else {
+              // one scale per 32 K: scale word of K-block kb for the weights at mb + 4 + 4 kb, for the tokens at
+              // mb + 12 + 4 n_atiles kb (+ 4 per token tile); the staged atoms are ordered [token tile][K-block]
+              ptx::tc_cp_32x128b_warpx4(mb + 8, d_sfa_in + so + (SF_ATOM_BYTES >> 4));
+              for (uint32_t a = 0; a < (uint32_t)n_atiles; ++a)
+                for (uint32_t kb = 0; kb < 2; ++kb)
+                  ptx::tc_cp_32x128b_warpx4(mb + 12 + 4 * (kb * (uint32_t)n_atiles + a), d_sf0 + so + (((2 * a + kb) * SF_ATOM_BYTES) >> 4));
+              ptx::mma_sp_nvf4(tmem + TM_D, d_a + so, d_b + so, id4[0], mb, mb + 4, mb + 12, acc);
+              ptx::mma_sp_nvf4(tmem + TM_D, d_a + so + (4096 >> 4), d_b + so + (512 >> 4), id4[0], mb + 2, mb + 8,
+                               mb + 12 + 4 * (uint32_t)n_atiles, 1u);
+            }
           } else {
             // outlier stage: 128 logical K = 2 sparse FP8 MMAs; the row / token scales (E8M0) arrive with the first one
             const uint32_t eb = tmem + TM_EO + 4u * (uint32_t)(k & 1);
@@ -542,7 +563,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   if (!Xq || !P || !Y || !Xq->dev || !P->dev) return SDQ_ERR_INVALID_ARG;
   if (Xq->K != P->K || Xq->M <= 0 || P->N <= 0 || P->N % TILE_ROWS || P->K % K2 || ldy < P->N) return SDQ_ERR_SHAPE;
   if (Xq->cfg.in_block != P->cfg.in_block || Xq->cfg.scale_rule != P->cfg.scale_rule) return SDQ_ERR_SHAPE;
-  if (P->cfg.in_gran != SDQ_GRAN_PAIR || P->cfg.in_block != 64) return SDQ_ERR_UNSUPPORTED;
+  if (P->cfg.in_gran != SDQ_GRAN_PAIR) return SDQ_ERR_UNSUPPORTED;
   if (((uintptr_t)Y & 15) || (ldy % 8) || ((uintptr_t)ws & 15)) return SDQ_ERR_ALIGNMENT;
   static bool attr_set = false;
   if (!attr_set) {
@@ -558,14 +579,15 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   LinearParams p;
   p.w = (const uint8_t*)P->dev;
   p.x = (const uint8_t*)Xq->dev;
-  p.poff = packed_offsets(P->N, P->K, P->cfg.out_n);
-  p.aoff = act_offsets(Xq->M, Xq->K);
+  p.b32 = P->cfg.in_block == 32 ? 1 : 0;
+  p.poff = packed_offsets(P->N, P->K, P->cfg.out_n, p.b32 != 0);
+  p.aoff = act_offsets(Xq->M, Xq->K, p.b32 != 0);
   p.M = Xq->M; p.N = P->N; p.K = P->K;
   p.out_n = P->cfg.out_n;
   const int64_t M = Xq->M;
   p.n_tile = n_tile_for(M);
   p.n_mtiles = (int)((M + p.n_tile - 1) / p.n_tile);
-  p.slot_bytes = slot_bytes_for(p.n_tile);
+  p.slot_bytes = slot_bytes_for(p.n_tile, p.b32 != 0);
   p.ksplit = 1;
   p.cluster_ks = 1;
   p.ws_counter = nullptr;
@@ -656,7 +678,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   }
   lc.attrs = attr;
   lc.numAttrs = na;
-  const bool flex = !(p.n_tile == 256 && p.ksplit == 1 && p.nslot == 5 && p.release == 1);
+  const bool flex = !(p.n_tile == 256 && p.ksplit == 1 && p.nslot == 5 && p.release == 1 && !p.b32);
   const cudaError_t le = flex ? (f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, true>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, true>, p))
                               : (f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, false>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, false>, p));
   return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;

@@ -23,6 +23,7 @@ struct LinearParams {
   int release;           // 1: ring slots are reused (producer waits on `empty`, MMA issuer commits to it)
   int tmem_cols;         // TMEM columns to allocate (128, 256 or 512)
   int meta_col;          // first TMEM column of the metadata / scale buffers
+  int b32;               // 1: one inlier / activation scale per 32 K (kind::mxf4nvf4 .block16), runtime geometry only
   int ksplit;            // CTAs sharing the K range of one row tile (1 = no split)
   int cluster_ks;        // > 1: those CTAs form a cluster and reduce through distributed shared memory
   uint32_t* ws_counter;  // split-K workspace: arrival counters [row tile], zero between calls

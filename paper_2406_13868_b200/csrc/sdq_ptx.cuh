@@ -113,6 +113,16 @@ __device__ __forceinline__ void mma_sp_mxf4(uint32_t d, uint64_t adesc, uint64_t
       : "memory");
 }
 // D[128 x N] (+)= A_sparse[128 x 64 logical K] * B[N x 64]^T, E4M3 operands, one E8M0 scale per operand row
+// sparse E2M1 x E2M1 with one UE8M0 scale per 32 logical K for both operands (4 scale bytes per row and MMA of
+// 128 logical K: the whole 32-bit scale word, sf ids 0); pair-wise 4:8 metadata as for kind::mxf4
+__device__ __forceinline__ void mma_sp_nvf4(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t e_tmem,
+                                            uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.sp.cta_group::1.kind::mxf4nvf4.block_scale.block16 [%0], %1, %2, [%7], %3, [%5], [%6], p;\n}" ::"r"(d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem), "r"(e_tmem)
+      : "memory");
+}
 __device__ __forceinline__ void mma_sp_mxf8(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t e_tmem,
                                             uint32_t sfa, uint32_t sfb, uint32_t accumulate) {
   asm volatile(

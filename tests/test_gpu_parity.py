@@ -14,8 +14,8 @@ def sdq():
     return m
 
 
-def ocfg(out_n=1, rule=0):
-    return so.Config(out_n, so.GRAN_PAIR, 64, rule)
+def ocfg(out_n=1, rule=0, block=64):
+    return so.Config(out_n, so.GRAN_PAIR, block, rule)
 
 
 def y_close(y_gpu, y_ref):
@@ -25,9 +25,9 @@ def y_close(y_gpu, y_ref):
     return d, tol
 
 
-def run_case(M, N, K, seed, out_n=1, rule=0, n_out_ch=None, check_rows=None):
+def run_case(M, N, K, seed, out_n=1, rule=0, n_out_ch=None, check_rows=None, block=64):
     m = sdq()
-    cfg = m.Config(out_n, m.GRAN_PAIR, 64, rule)
+    cfg = m.Config(out_n, m.GRAN_PAIR, block, rule)
     W = sdq_synth.make_weight(N, K, seed)
     X = sdq_synth.make_act(M, K, seed, n_outlier_channels=n_out_ch)
     p = m.sdq_decompose(W.cuda(), cfg)
@@ -35,8 +35,8 @@ def run_case(M, N, K, seed, out_n=1, rule=0, n_out_ch=None, check_rows=None):
     y32 = m.sdq_linear(xq, p, f32=True)
     y16 = m.sdq_linear(xq, p)
     assert m.device_status() == 0
-    op = so.decompose(sdq_synth.bf16_bits(W), ocfg(out_n, rule))
-    oq = so.quantize_act(sdq_synth.bf16_bits(X), ocfg(out_n, rule))
+    op = so.decompose(sdq_synth.bf16_bits(W), ocfg(out_n, rule, block))
+    oq = so.quantize_act(sdq_synth.bf16_bits(X), ocfg(out_n, rule, block))
     pe = {k: v.cpu().numpy() for k, v in m.packed_export(p).items()}
     ae = {k: v.cpu().numpy() for k, v in m.act_export(xq).items()}
     for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp"):
@@ -110,6 +110,30 @@ def test_seeded_random_shapes(M, N, K, out_n, rule):
     """seeded random token counts (few / up to 128 / several hundred), widths, depths, outlier counts and scale rules:
     every launch geometry the host logic can pick for small problems, full parity each"""
     run_case(M, N, K, 7 * M + N + K, out_n=out_n, rule=rule)
+
+
+@pytest.mark.parametrize("M,N,K,out_n,rule", [(8, 256, 256, 1, 0), (1, 512, 2048, 1, 0), (16, 256, 4096, 2, 1), (33, 128, 768, 0, 0),
+                                              (100, 256, 2816, 1, 0), (129, 256, 512, 1, 1), (300, 512, 1024, 2, 0),
+                                              (520, 6400, 256, 1, 0)])
+def test_block_32_scales_through_the_tensor_core(M, N, K, out_n, rule):
+    """one E8M0 scale per 32 logical K for the inlier weights and the 4-bit activations (the literal block-32 MXFP4
+    wording): executed by the sparse kind::mxf4nvf4 .block16 MMA; few tokens, cluster split K, several hundred tokens,
+    and enough tiles for persistent CTAs"""
+    run_case(M, N, K, 900 + M, out_n=out_n, rule=rule, block=32)
+
+
+def test_block_32_one_hot_readback():
+    m = sdq()
+    cfg = m.Config(1, m.GRAN_PAIR, 32, 0)
+    N, K = 256, 512
+    W = sdq_synth.make_weight(N, K, 61)
+    p = m.sdq_decompose(W.cuda(), cfg)
+    X = torch.eye(K, dtype=torch.bfloat16)
+    xq = m.sdq_quantize_act(X.cuda(), cfg)
+    y = m.sdq_linear(xq, p, f32=True).cpu().numpy().astype(np.float64)
+    W_in, W_out = so.dequant_weights(so.decompose(sdq_synth.bf16_bits(W), ocfg(block=32)))
+    assert np.array_equal(y, (W_in + W_out).T)
+    assert m.device_status() == 0
 
 
 def test_one_hot_readback_512_tokens():
