@@ -32,7 +32,6 @@ constexpr int LIN_THREADS = 288;   // warps: 0 weight producer, 1 MMA issuer, 2.
                                    // 8 metadata / scale mover (many-token instantiation only)
 constexpr int MAX_SLOTS = 16;
 constexpr int SL_A = 0;                        // WI record (A_in | E_in | SFA_in) or WO record (A_out | E_out)
-constexpr int SL_B = 10752;                    // B4 (256 K) or B8 (128 K) of n_tile tokens: n_tile * 128 B
 constexpr int RING_BYTES = 225280;             // largest ring: nslot slots of slot_bytes each
 constexpr int SM_TAIL = 4096 + 640 + 128;      // epilogue transpose buffer (16 tokens x 128 features bf16) + barriers + slack
 constexpr int LIN_SMEM_MAX = RING_BYTES + SM_TAIL;
@@ -79,7 +78,8 @@ __device__ __forceinline__ TileCoord tile_coord(int ksplit, int tile, int RT, in
 // FLEX = false: the many-token instantiation (n_tile = 256, 5 ring slots, 512 TMEM columns, no K split) with every
 // geometry constant known at compile time -- the single-thread issue loops are latency-bound, so each runtime
 // parameter they touch costs time.  FLEX = true: geometry from the launch parameters (few tokens, split K).
-template <bool F32_OUT, bool FLEX>
+// B32 (many-token instantiation only): one scale per 32 K, four ring slots of 45 KB.
+template <bool F32_OUT, bool FLEX, bool B32>
 __global__ void __maxnreg__(96)   // two 9-warp CTAs share an SM only below ~100 registers per thread
 sdq_linear_kernel(const LinearParams p)
 {
@@ -88,7 +88,8 @@ sdq_linear_kernel(const LinearParams p)
   uint8_t* sm = smem_raw + ((128 - (ptx::smem_u32(smem_raw) & 127)) & 127);
   const int ksplit = FLEX ? p.ksplit : 1, cluster_ks = FLEX ? p.cluster_ks : 1;
   const bool release = FLEX ? (p.release != 0) : true;
-  const uint32_t SM_STG = FLEX ? (uint32_t)p.ring_bytes : (uint32_t)RING_BYTES, SM_BARS = SM_STG + 4096;
+  // the transpose buffer and the barriers follow the ring (many tokens: 5 x 45056, or 4 x 46080 with one scale per 32 K)
+  const uint32_t SM_STG = FLEX ? (uint32_t)p.ring_bytes : (B32 ? 4u * 46080u : (uint32_t)RING_BYTES), SM_BARS = SM_STG + 4096;
   const uint32_t TM_I = FLEX ? (uint32_t)p.meta_col : 256u, TM_EO = TM_I + 64, TM_SFA_OUT = TM_I + 72, TM_SFB_OUT = TM_I + 76;
   const uint32_t tmem_cols = FLEX ? (uint32_t)p.tmem_cols : 512u;
   uint64_t* full = reinterpret_cast<uint64_t*>(sm + SM_BARS);
@@ -104,8 +105,9 @@ sdq_linear_kernel(const LinearParams p)
   const int RT = (int)(p.N / TILE_ROWS);
   const int T1 = p.out_n ? (int)(p.K / K1) : 0, T2 = (int)(p.K / K2);
   const int n_atiles = (n_tile + TILE_TOK - 1) / TILE_TOK;     // 128-token activation tiles per token tile
-  const uint32_t nslot = FLEX ? (uint32_t)p.nslot : 5u, slot_bytes = FLEX ? (uint32_t)p.slot_bytes : 45056u;
-  const bool b32 = FLEX && p.b32;                          // one scale per 32 K (runtime geometry only)
+  const uint32_t nslot = FLEX ? (uint32_t)p.nslot : (B32 ? 4u : 5u), slot_bytes = FLEX ? (uint32_t)p.slot_bytes : (B32 ? 46080u : 45056u);
+  const bool b32 = FLEX ? (p.b32 != 0) : B32;              // one scale per 32 K
+  constexpr uint32_t MS = B32 ? 32u : 16u;                 // many tokens: metadata / scale columns per ring slot
   const uint32_t wib = (uint32_t)wi_bytes(b32), xib = (uint32_t)xi_bytes(b32), na = b32 ? 2u : 1u;
   const uint32_t sl_b = wib;                               // B4 / B8 follow the (longest) weight record
   const uint32_t sl_sf = sl_b + (uint32_t)n_tile * 128u;
@@ -227,7 +229,7 @@ sdq_linear_kernel(const LinearParams p)
         if constexpr (!FLEX) {
           // many tokens: warp 8 has already moved the metadata and scales of slot s to TMEM (16 columns per slot, the
           // outlier scales in one of two per-tile buffers); this thread only issues the MMAs
-          const uint32_t sfo = tmem + 256u + 80u + 12u * (tcount & 1);
+          const uint32_t sfo = tmem + 256u + MS * nslot + 12u * (tcount & 1);
           for (int k = 0; k < ni + no; ++k) {
             if (!ready) ok = ptx::mbar_wait(&meta_full[s], ph);
             if (ok) ok = ptx::mbar_wait(&full[s], ph);          // the activation codes of the slot
@@ -236,10 +238,15 @@ sdq_linear_kernel(const LinearParams p)
             const uint32_t sn = (s + 1 == nslot) ? 0 : s + 1;
             ready = ptx::mbar_test(&meta_full[sn], sn ? ph : ph ^ 1);
             const uint64_t so = (uint64_t)(s * slot16);
-            const uint32_t mb = tmem + 256u + 16u * s;
+            const uint32_t mb = tmem + 256u + MS * s;
             if (k < ni) {
-              ptx::mma_sp_mxf4(tmem + TM_D, d_a + so, d_b + so, id4[0], mb, mb + 4, mb + 8, acc);
-              ptx::mma_sp_mxf4(tmem + TM_D, d_a + so + (4096 >> 4), d_b + so + (512 >> 4), id4[1], mb + 2, mb + 4, mb + 8, 1u);
+              if constexpr (B32) {
+                ptx::mma_sp_nvf4(tmem + TM_D, d_a + so, d_b + so, id4[0], mb, mb + 4, mb + 12, acc);
+                ptx::mma_sp_nvf4(tmem + TM_D, d_a + so + (4096 >> 4), d_b + so + (512 >> 4), id4[0], mb + 2, mb + 8, mb + 20, 1u);
+              } else {
+                ptx::mma_sp_mxf4(tmem + TM_D, d_a + so, d_b + so, id4[0], mb, mb + 4, mb + 8, acc);
+                ptx::mma_sp_mxf4(tmem + TM_D, d_a + so + (4096 >> 4), d_b + so + (512 >> 4), id4[1], mb + 2, mb + 4, mb + 8, 1u);
+              }
             } else {
               ptx::mma_sp_mxf8(tmem + TM_D, d_a + so, d_b + so, id8, mb, sfo, sfo + 4, acc);
               ptx::mma_sp_mxf8(tmem + TM_D, d_a + so + (4096 >> 4), d_b + so + (512 >> 4), id8, mb + 2, sfo, sfo + 4, 1u);
@@ -318,17 +325,27 @@ sdq_linear_kernel(const LinearParams p)
       const uint64_t d_sf2 = ptx::smem_desc(smb + sl_sf + 2 * SF_ATOM_BYTES, 0, 128);
       const uint32_t slot16 = slot_bytes >> 4;
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
-        const uint32_t sfo = tmem + 256u + 80u + 12u * (tcount & 1);
+        const uint32_t sfo = tmem + 256u + MS * nslot + 12u * (tcount & 1);
         for (int k = 0; k < T2 + T1; ++k) {
           if (!(ok = ptx::mbar_wait(&full_w[s], ph))) break;
           ptx::tc_fence_after();
           const uint64_t so = (uint64_t)(s * slot16);
-          const uint32_t mb = tmem + 256u + 16u * s;
+          const uint32_t mb = tmem + 256u + MS * s;
           if (k < T2) {
             ptx::tc_cp_128x128b(mb + 0, d_e_in + so);
             ptx::tc_cp_32x128b_warpx4(mb + 4, d_sfa_in + so);
-            ptx::tc_cp_32x128b_warpx4(mb + 8, d_sf0 + so);
-            ptx::tc_cp_32x128b_warpx4(mb + 12, d_sf1 + so);
+            if constexpr (B32) {
+              // scale words: weights K-block 0 / 1 at +4 / +8; tokens K-block kb, token tile a at +12 + 4 (2 kb + a), staged
+              // as [token tile][K-block]
+              ptx::tc_cp_32x128b_warpx4(mb + 8, d_sfa_in + so + (SF_ATOM_BYTES >> 4));
+              ptx::tc_cp_32x128b_warpx4(mb + 12, d_sf0 + so);
+              ptx::tc_cp_32x128b_warpx4(mb + 20, d_sf1 + so);
+              ptx::tc_cp_32x128b_warpx4(mb + 16, d_sf2 + so);
+              ptx::tc_cp_32x128b_warpx4(mb + 24, d_sf2 + so + (SF_ATOM_BYTES >> 4));
+            } else {
+              ptx::tc_cp_32x128b_warpx4(mb + 8, d_sf0 + so);
+              ptx::tc_cp_32x128b_warpx4(mb + 12, d_sf1 + so);
+            }
           } else {
             ptx::tc_cp_128x128b(mb + 0, d_e_out + so);
             if (k == T2) {
@@ -567,10 +584,12 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   if (((uintptr_t)Y & 15) || (ldy % 8) || ((uintptr_t)ws & 15)) return SDQ_ERR_ALIGNMENT;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(sdq_linear_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
-        cudaFuncSetAttribute(sdq_linear_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
-        cudaFuncSetAttribute(sdq_linear_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
-        cudaFuncSetAttribute(sdq_linear_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess)
+    if (cudaFuncSetAttribute(sdq_linear_kernel<true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess)
       return SDQ_ERR_CUDA;
     attr_set = true;
   }
@@ -678,9 +697,11 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   }
   lc.attrs = attr;
   lc.numAttrs = na;
-  const bool flex = !(p.n_tile == 256 && p.ksplit == 1 && p.nslot == 5 && p.release == 1 && !p.b32);
-  const cudaError_t le = flex ? (f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, true>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, true>, p))
-                              : (f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, false>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, false>, p));
+  const bool flex = !(p.n_tile == 256 && p.ksplit == 1 && p.nslot == (p.b32 ? 4 : 5) && p.release == 1);
+  cudaError_t le;
+  if (flex) le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, true, false>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, true, false>, p);
+  else if (p.b32) le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, false, true>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, false, true>, p);
+  else le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, false, false>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, false, false>, p);
   return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
 }
 
