@@ -50,7 +50,8 @@ enum { SDQ_SCALE_OCP_FLOOR = 0, SDQ_SCALE_CEIL_NOSAT = 1 }; /* E8M0 Q-Vector sca
  *              of every 4 (decompose / export only: the buffer then holds the canonical arrays and
  *              sdq_linear returns SDQ_ERR_UNSUPPORTED).
  *   in_block   Q-Vector length: logical K sharing one E8M0 scale, for W_i and for the 4-bit
- *              activations (64 is what sdq_linear executes; 32 is decompose/quantize/export only).
+ *              activations: 64 or 32.  Both are executed by sdq_linear (64: kind::mxf4 .block32, the
+ *              faster kernel; 32: kind::mxf4nvf4 .block16 with E8M0 scale codes).
  *   scale_rule E8M0 exponent from the Q-Vector's largest magnitude a: OCP_FLOOR = floor(log2 a) - 2,
  *              CEIL_NOSAT = smallest E with a <= 6 * 2^E.
  */
@@ -166,7 +167,7 @@ sdq_status_t sdq_act_export(const sdq_act_t* Xq, const sdq_act_canonical_t* out,
  *   weights) while the previous kernel of the stream is still finishing, and waits for that kernel before it
  *   reads Xq or writes Y.  The packed weights must therefore be complete before the call is enqueued
  *   (sdq_decompose synchronises its stream, so a buffer it returned always is).
- *   Errors: INVALID_ARG, SHAPE, ALIGNMENT, UNSUPPORTED (in_gran != PAIR or in_block != 64), CUDA. */
+ *   Errors: INVALID_ARG, SHAPE, ALIGNMENT, UNSUPPORTED (in_gran != PAIR), CUDA. */
 sdq_status_t sdq_linear(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y_bf16, int64_t ldy, void* stream);
 
 /* Same product, storing the fp32 accumulator itself (the value the bf16 output is rounded from). */
