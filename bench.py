@@ -462,6 +462,15 @@ def run_sweep(args):
         fl = 2.0 * M * 4096 * 16384
         c4[name] = {"fc1_ms": t1, "fc1_TFLOPs": fl / t1 / 1e9, "fc2_ms": t2, "fc2_TFLOPs": fl / t2 / 1e9}
         del P1, P2, xq, hq
+    # the same layers with one scale per 32 K (the literal block-32 MXFP4 wording), 1:8 outliers
+    cfg = sdq.Config(1, sdq.GRAN_PAIR, 32, 0)
+    P1, P2 = sdq.sdq_decompose(W1, cfg), sdq.sdq_decompose(W2, cfg)
+    xq, hq = sdq.sdq_quantize_act(X, cfg), sdq.sdq_quantize_act(H, cfg)
+    t1 = time_graph(lambda: sdq.sdq_linear(xq, P1, Y1))
+    t2 = time_graph(lambda: sdq.sdq_linear(hq, P2, Y2))
+    fl = 2.0 * M * 4096 * 16384
+    c4["1:8, scale block 32"] = {"fc1_ms": t1, "fc1_TFLOPs": fl / t1 / 1e9, "fc2_ms": t2, "fc2_TFLOPs": fl / t2 / 1e9}
+    del P1, P2, xq, hq
     out["opt67b_ffn_M4096_outlier_sweep"] = c4
     del X, H, W1, W2, Y1, Y2
     # ---- config 5: 32 layers x (q, k, v, o, gate, up, down)
