@@ -20,10 +20,10 @@ def sdq():
     return m
 
 
-def check_sampled(M, N, K, seed, out_n=1, n_tok=12, use_ws=False):
+def check_sampled(M, N, K, seed, out_n=1, n_tok=12, use_ws=False, block=64):
     m = sdq()
-    cfg = m.Config(out_n, m.GRAN_PAIR, 64, 0)
-    ocfg = so.Config(out_n, so.GRAN_PAIR, 64, 0)
+    cfg = m.Config(out_n, m.GRAN_PAIR, block, 0)
+    ocfg = so.Config(out_n, so.GRAN_PAIR, block, 0)
     W = sdq_synth.make_weight(N, K, seed, device="cuda")
     X = sdq_synth.make_act(M, K, seed + 1, device="cuda")
     p = m.sdq_decompose(W, cfg)
@@ -69,6 +69,12 @@ def test_llama7b_attention_projection_decode(M, use_ws):
 def test_llama7b_mlp_prefill(N, K):
     """config 3: X 2048 x K; gate/up 4096 -> 11008 and down 11008 -> 4096"""
     check_sampled(2048, N, K, 3000 + N)
+
+
+@pytest.mark.parametrize("M,N,K", [(16, 4096, 4096), (2048, 11008, 4096), (2048, 4096, 11008)])
+def test_scale_block_32_at_full_size(M, N, K):
+    """configs 2 and 3 with one scale per 32 K (the literal block-32 MXFP4 wording)"""
+    check_sampled(M, N, K, 3500 + M, block=32)
 
 
 @pytest.mark.parametrize("out_n", [1, 2, 0])
