@@ -14,6 +14,7 @@
 //            lower k): byte(j, row r, b) at j*4096 + (r/8)*256 + (b/16)*128 + (r%8)*16 + b%16
 //     E_in : 128 rows x 16 B  (one 4-bit pair-index pair per 8 logical K over 256 K)
 //     SFA_in: 4 E8M0 scales (one per 64 K) of 128 rows: byte(r, s) at (r%32)*16 + (r/32)*4 + s
+//             (one scale per 32 K: two such atoms, one per 128-K block, 4 scales each; the record is 11264 B)
 //   section WO[rt][k1] = | A_out 8192 | E_out 2048 |                                     (10240 B)
 //     A_out: two K-blocks j (64 logical K each) of 128 rows x 32 B (stored E4M3 bytes of the 2:4
 //            embedding of the 1:8 / 2:8 outliers), same addressing as A_in
@@ -22,7 +23,7 @@
 //   sections compact outlier codes / indices [N][K/8][out_n] u8 and row scale exponents [N] i32
 //
 // Activation buffer (per 128-token tile mt)
-//   section XI[mt][k2] = | B4 16384 | SFB_in 512 |
+//   section XI[mt][k2] = | B4 16384 | SFB_in 512 |            (one scale per 32 K: SFB_in 2 x 512, as for the weights)
 //     B4: 128 tokens x 128 B (256 K): byte(t, b) at (t/8)*1024 + (b/16)*128 + (t%8)*16 + b%16
 //   section XO[mt][k1] = | B8 16384 |
 //     B8: 128 tokens x 128 B (128 K): same addressing
