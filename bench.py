@@ -270,6 +270,9 @@ def run_ours(args):
         return
     # ---- decode shape (C2): 4096x4096, M in {1,16}, rotating over 32 distinct packed layers (> L2)
     decode = measure_decode(sdq, cfg, dev, peaks)
+    # ---- the same step with one scale per 32 K (the literal block-32 MXFP4 wording), timed the same way
+    cfg32 = sdq.Config(1, sdq.GRAN_PAIR, 32, sdq.SCALE_OCP_FLOOR)
+    b32 = measure_block32_step(sdq, cfg32, dev, rank, X, H, (Yg, Yu, Yd), flops_step, args.steps)
     # ---- end to end through the public API with host buffers (pinned), copies inside the timed region
     e2e = measure_e2e(sdq, cfg, dev, X, H, (Pg, Pu, Pd), (bx, bh), (Yg, Yu, Yd), flops_step, max(3, args.steps // 2))
     sample = OracleSample(rows_x=1024)
@@ -281,7 +284,7 @@ def run_ours(args):
             "config": {"workload": WORKLOAD, "tokens_per_gpu": M_PREFILL, "l2": "packed weights + activations of one step exceed L2 (150 MB > 126 MB)",
                        "parallelism": "dp%d (independent batches, no collective)" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "quantizer_roofline": quant, "decode": decode,
+            "roofline": roofline, "quantizer_roofline": quant, "scale_block_32": b32, "decode": decode,
             "cpu_baseline": {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc, "seconds": dt}}
     print(json.dumps(line))
 
@@ -332,6 +335,39 @@ def measure_decode(sdq, cfg, dev, peaks, layers: int = 32, reps: int = 20):
     out["stored_bytes_per_layer"] = int(packs[0].buf.numel())
     out["hbm_peak_GBps"] = peaks["hbm"]
     return out
+
+
+def measure_block32_step(sdq, cfg, dev, rank, X, H, outs, flops_step, steps):
+    """The benchmark step with in_block = 32 (kind::mxf4nvf4 .block16): fresh packed weights of the same shapes, the
+    same inputs and output buffers; whole-step throughput from one event pair around `steps` steps."""
+    seed = 3000 + rank
+    packs = []
+    for i, (n, k) in enumerate(((D_FF, D_MODEL), (D_FF, D_MODEL), (D_MODEL, D_FF))):
+        W = sdq_synth.make_weight(n, k, seed + 1 + i, device=str(dev))
+        packs.append(sdq.sdq_decompose(W, cfg))
+        del W
+    bx = torch.empty(sdq.act_size(M_PREFILL, D_MODEL, cfg), dtype=torch.uint8, device=dev)
+    bh = torch.empty(sdq.act_size(M_PREFILL, D_FF, cfg), dtype=torch.uint8, device=dev)
+
+    def step():
+        xq = sdq.sdq_quantize_act(X, cfg, bx)
+        sdq.sdq_linear(xq, packs[0], outs[0])
+        sdq.sdq_linear(xq, packs[1], outs[1])
+        hq = sdq.sdq_quantize_act(H, cfg, bh)
+        sdq.sdq_linear(hq, packs[2], outs[2])
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps):
+        step()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / steps
+    assert sdq.device_status() == 0
+    return {"value": flops_step / (ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms,
+            "workload": "the same step with one E8M0 scale per 32 K for inlier weights and 4-bit activations"}
 
 
 def measure_e2e(sdq, cfg, dev, X, H, packs, bufs, outs, flops_step, steps):
