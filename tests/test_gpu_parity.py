@@ -243,18 +243,18 @@ def test_hardware_converters_match_oracle_exhaustively():
 
 
 @pytest.mark.parametrize("M,K", [(13, 256), (8, 2048), (21, 11008), (5, 16384), (3, 16640), (9, 20480)])
-@pytest.mark.parametrize("rule", [0, 1])
-def test_activation_quantizer_row_lengths(M, K, rule):
+@pytest.mark.parametrize("rule,block", [(0, 64), (1, 64), (0, 32), (1, 32)])
+def test_activation_quantizer_row_lengths(M, K, rule, block):
     """Rows up to 16384 take the single-launch cluster kernel (1..8 CTAs per group of 8 tokens), longer rows the
     two-launch path; both must give the oracle's codes and scales bit for bit, ragged token groups included."""
     m = sdq()
-    cfg = m.Config(1, m.GRAN_PAIR, 64, rule)
+    cfg = m.Config(1, m.GRAN_PAIR, block, rule)
     X = sdq_synth.make_act(M, K, 100 + M, n_outlier_channels=max(1, K // 100))
     X[M // 2, K // 3] = float("inf")            # saturates, must not poison the row
     X[0, :64] = 0.0                             # an all-zero Q-Vector
     xq = m.sdq_quantize_act(X.cuda(), cfg)
     assert m.device_status() == 0
-    oq = so.quantize_act(sdq_synth.bf16_bits(X), ocfg(1, rule))
+    oq = so.quantize_act(sdq_synth.bf16_bits(X), ocfg(1, rule, block))
     ae = {k: v.cpu().numpy() for k, v in m.act_export(xq).items()}
     for name in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp"):
         assert np.array_equal(ae[name], getattr(oq, name)), name
