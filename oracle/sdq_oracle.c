@@ -31,6 +31,7 @@
 
 #define SDQO_GRAN_PAIR 0 /* inlier pattern: keep 2 of the 4 adjacent pairs in every 8 (pair-wise 4:8) */
 #define SDQO_GRAN_ELEM 1 /* inlier pattern: keep 2 of every 4 elements (element-wise 2:4)            */
+#define SDQO_GRAN_DENSE 2 /* no Stage 1: every non-outlier value stays an inlier (8:8 = out_n:8 + (8-out_n):8) */
 #define SDQO_SCALE_OCP_FLOOR 0  /* E = floor(log2 amax) - 2   (OCP MX rule, may saturate in (6,8)) */
 #define SDQO_SCALE_CEIL_NOSAT 1 /* E = smallest integer with amax <= 6 * 2^E                        */
 
@@ -141,9 +142,10 @@ static int is_finite_bf16(uint16_t h) { return (h & 0x7F80) != 0x7F80; }
  *
  * W        [N][K] bf16 bit patterns, row-major (row = output feature, K contiguous)
  * Canonical outputs, one code per byte (layout-free parity surface):
- *   in_code  [N][K/2]      E2M1 codes of the kept inlier slots in ascending k
+ *   in_code  [N][K/2]      E2M1 codes of the kept inlier slots in ascending k   (DENSE: [N][K], every position)
  *   in_meta  [N][K/8] (PAIR: j0 | j1<<2, kept pair indices 0..3 of the group of 8)
  *            [N][K/4] (ELEM: i0 | i1<<2, kept element indices 0..3 of the group of 4)
+ *            not touched for DENSE (there is no pattern to record)
  *   in_scale [N][K/in_block] E8M0 code
  *   out_code [N][K/8][out_n] E4M3 codes; out_idx same shape, position 0..7 inside the group, ascending
  *   out_sexp [N]           e of the per-row outlier scale 2^e (int32)
@@ -171,8 +173,10 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
       if (!(col_weight[k] >= 0.0f) || isinf(col_weight[k])) return -3;
   if (cfg->out_n < 0 || cfg->out_n > 2) return -1;
   if (cfg->in_block != 32 && cfg->in_block != 64) return -1;
+  if (cfg->in_gran != SDQO_GRAN_PAIR && cfg->in_gran != SDQO_GRAN_ELEM && cfg->in_gran != SDQO_GRAN_DENSE) return -1;
   const int on = cfg->out_n, Bs = cfg->in_block;
   const int64_t G8 = K / 8;
+  const int64_t slots = cfg->in_gran == SDQO_GRAN_DENSE ? K : K / 2;   /* inlier slots per row */
   for (int64_t i = 0; i < N * K; ++i)
     if (!is_finite_bf16(W[i])) return -2;
 
@@ -215,8 +219,11 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
         out_code[(n * G8 + g) * on + t] = sdqo_e4m3_encode(ldexp(sdqo_bf16_to_double(w[8 * g + i]), -e));
       }
 
-    /* Stage 1 on the remaining values: N:M pruning by significance */
-    if (cfg->in_gran == SDQO_GRAN_PAIR) {
+    /* Stage 1 on the remaining values: N:M pruning by significance.  The dense configuration
+       (Section 5, decomposition-stage study: 8:8 split as 1:8 outliers + 7:8 inliers) skips it. */
+    if (cfg->in_gran == SDQO_GRAN_DENSE) {
+      memset(kept, 1, (size_t)K);
+    } else if (cfg->in_gran == SDQO_GRAN_PAIR) {
       for (int64_t g = 0; g < G8; ++g) {
         float score[4];
         for (int j = 0; j < 4; ++j) {
@@ -269,7 +276,7 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
         int c = in_scale[n * (K / Bs) + k / Bs];
         code = sdqo_e2m1_encode(ldexp(sdqo_bf16_to_double(w[k]), 127 - c));
       }
-      in_code[n * (K / 2) + slot++] = code;
+      in_code[n * slots + slot++] = code;
     }
   }
   free(is_out);
@@ -296,7 +303,10 @@ int sdqo_dequant_weights(int64_t N, int64_t K, const sdqo_config* cfg,
   memset(W_out, 0, sizeof(double) * (size_t)(N * K));
   for (int64_t n = 0; n < N; ++n) {
     int64_t slot = 0;
-    if (cfg->in_gran == SDQO_GRAN_PAIR) {
+    if (cfg->in_gran == SDQO_GRAN_DENSE) {
+      for (int64_t k = 0; k < K; ++k)
+        W_in[n * K + k] = sdqo_e2m1_decode(in_code[n * K + k]) * sdqo_e8m0_decode(in_scale[n * (K / Bs) + k / Bs]);
+    } else if (cfg->in_gran == SDQO_GRAN_PAIR) {
       for (int64_t g = 0; g < G8; ++g) {
         int nib = in_meta[n * G8 + g];
         int jj[2] = {nib & 3, (nib >> 2) & 3};
@@ -392,15 +402,20 @@ int sdqo_linear(int64_t M, int64_t N, int64_t K, const sdqo_config* cfg,
     }
 #pragma omp parallel num_threads(n_threads > 0 ? n_threads : 1)
   {
-    int32_t* ki = (int32_t*)malloc(sizeof(int32_t) * (size_t)(K / 2));
-    double* wi = (double*)malloc(sizeof(double) * (size_t)(K / 2));
+    int32_t* ki = (int32_t*)malloc(sizeof(int32_t) * (size_t)K);
+    double* wi = (double*)malloc(sizeof(double) * (size_t)K);
     int32_t* ko = (int32_t*)malloc(sizeof(int32_t) * (size_t)(G8 * 2));
     double* wo = (double*)malloc(sizeof(double) * (size_t)(G8 * 2));
 #pragma omp for schedule(static)
     for (int64_t n = n_begin; n < n_end; ++n) {
       /* positions and values of the non-zeros of row n of W_i and W_o */
       int64_t ni = 0, no = 0, slot = 0;
-      if (cfg->in_gran == SDQO_GRAN_PAIR) {
+      if (cfg->in_gran == SDQO_GRAN_DENSE) {
+        for (int64_t k = 0; k < K; ++k) {
+          ki[ni] = (int32_t)k;
+          wi[ni++] = sdqo_e2m1_decode(in_code[n * K + k]) * sdqo_e8m0_decode(in_scale[n * (K / Bs) + k / Bs]);
+        }
+      } else if (cfg->in_gran == SDQO_GRAN_PAIR) {
         for (int64_t g = 0; g < G8; ++g) {
           int nib = in_meta[n * G8 + g];
           int jj[2] = {nib & 3, (nib >> 2) & 3};

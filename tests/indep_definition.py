@@ -60,7 +60,8 @@ def top_mask(keys, n):
 
 def decompose_dense(W_bits, out_n, pair, block, rule_floor, col_weight=None):
     """returns (W_in_hat, W_out_hat, mask_in_slots, mask_out) as dense [N, K] arrays; with col_weight the
-    selections rank by the fp32 product |w| * c[k] instead of |w| (the values that get quantized do not change)"""
+    selections rank by the fp32 product |w| * c[k] instead of |w| (the values that get quantized do not change);
+    pair: True = pair-wise 4:8, False = element-wise 2:4, None = no pruning"""
     W = bf16_to_f64(W_bits)
     N, K = W.shape
     A = np.abs(W)
@@ -68,7 +69,9 @@ def decompose_dense(W_bits, out_n, pair, block, rule_floor, col_weight=None):
         A = (A.astype(np.float32) * np.asarray(col_weight, dtype=np.float32)[None, :]).astype(np.float32).astype(np.float64)
     mask_out = top_mask(A.reshape(N, K // 8, 8), out_n).reshape(N, K) if out_n else np.zeros((N, K), bool)
     R = np.where(mask_out, 0.0, A)
-    if pair:
+    if pair is None:                      # no pruning: every non-outlier value stays an inlier
+        slots = np.ones((N, K), bool)
+    elif pair:
         r32 = R.astype(np.float32).reshape(N, K // 8, 4, 2)
         score = (r32[..., 0] + r32[..., 1]).astype(np.float32)
         keep_pair = top_mask(score, 2)

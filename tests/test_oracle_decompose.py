@@ -273,3 +273,85 @@ def test_channel_norm_closed_forms():
     assert np.array_equal(so.channel_norm(Xb[perm]), c)
     Xb4 = sdq_synth.bf16_bits(torch.from_numpy(x * 4).to(torch.bfloat16))
     assert np.array_equal(so.channel_norm(Xb4), c * 4)
+
+
+# ---------------------------------------------------------------- no Stage 1: 8:8 split as out_n:8 outliers + dense inliers
+DENSE_CFGS = [so.Config(1, so.GRAN_DENSE, 32, so.SCALE_OCP_FLOOR),
+              so.Config(2, so.GRAN_DENSE, 32, so.SCALE_CEIL_NOSAT),
+              so.Config(0, so.GRAN_DENSE, 64, so.SCALE_OCP_FLOOR),
+              so.Config(1, so.GRAN_DENSE, 64, so.SCALE_CEIL_NOSAT)]
+
+
+@pytest.mark.parametrize("cfg", DENSE_CFGS)
+def test_dense_inliers_match_independent_dense_definition(cfg):
+    """without pruning, W_in + W_out is the quantized W of an independent routine, with and without a channel weight"""
+    for seed, cw in ((0, None), (1, lognormal_channel_weight(512, 7))):
+        Wb = tiny_W(48, 512, seed)
+        p = so.decompose(Wb, cfg, cw)
+        assert p.in_code.shape == (48, 512) and p.in_meta.size == 0
+        W_in, W_out = so.dequant_weights(p)
+        ref_in, ref_out, slots, mask_out = decompose_dense(Wb, cfg.out_n, None, cfg.in_block,
+                                                           cfg.scale_rule == so.SCALE_OCP_FLOOR, cw)
+        assert slots.all()
+        assert np.array_equal(W_out, ref_out)
+        assert np.array_equal(W_in, ref_in)
+        # every position that is not an outlier holds its own code; the outlier positions hold +0
+        assert (p.in_code[mask_out] == 0).all()
+        assert ((W_out != 0).reshape(48, 64, 8).sum(-1) <= cfg.out_n).all()
+        assert not ((W_in != 0) & (W_out != 0)).any()
+
+
+@pytest.mark.parametrize("out_n", [1, 2])
+def test_dense_inliers_share_stage_2_with_the_pruned_patterns(out_n):
+    """Stage 2 does not depend on Stage 1: the outlier arrays are those of the pair-wise and element-wise patterns"""
+    Wb = tiny_W(32, 256, 11)
+    d = so.decompose(Wb, so.Config(out_n, so.GRAN_DENSE, 64, so.SCALE_OCP_FLOOR))
+    for gran in (so.GRAN_PAIR, so.GRAN_ELEM):
+        p = so.decompose(Wb, so.Config(out_n, gran, 64, so.SCALE_OCP_FLOOR))
+        assert np.array_equal(d.out_idx, p.out_idx) and np.array_equal(d.out_code, p.out_code)
+        assert np.array_equal(d.out_sexp, p.out_sexp)
+        # the pruned W_in is the dense W_in restricted to the kept slots whenever both use the same block scale
+        Wd, _ = so.dequant_weights(d)
+        Wp, _ = so.dequant_weights(p)
+        same_scale = np.repeat(d.in_scale == p.in_scale, 64, axis=1)
+        assert np.array_equal(np.where(same_scale & (Wp != 0), Wd, 0.0), np.where(same_scale, Wp, 0.0))
+
+
+def test_dense_inliers_on_grid_weights_round_trip_exactly():
+    """every element on the E2M1 * 2^E grid (one E4M3-exact dominant value per 8): nothing is lost, W_in + W_out == W"""
+    rng = np.random.default_rng(13)
+    N, K = 16, 256
+    e2m1 = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+    W = rng.choice([-1.0, 1.0], size=(N, K)) * rng.choice(e2m1, size=(N, K)) * 0.125
+    W[:, 1::32] = 0.75                                     # every block of 32 reaches 6 * 2^-3: one scale under both rules
+    for g in range(K // 8):
+        o = (3 * g) % 8
+        if (8 * g + o) % 32 == 1:
+            o += 1
+        W[:, 8 * g + o] = rng.choice([-1, 1], size=N) * 16.0 * (1 + rng.integers(0, 8, size=N) / 8)
+    import torch
+    Wb = sdq_synth.bf16_bits(torch.from_numpy(W).to(torch.bfloat16))
+    assert np.array_equal(bf16_to_f64(Wb), W)
+    for rule in (so.SCALE_OCP_FLOOR, so.SCALE_CEIL_NOSAT):
+        for block in (32, 64):
+            p = so.decompose(Wb, so.Config(1, so.GRAN_DENSE, block, rule))
+            W_in, W_out = so.dequant_weights(p)
+            assert np.array_equal(W_in + W_out, W)
+            assert (np.abs(W_out[W_out != 0]) >= 16).all() and (W_out != 0).sum() == N * K // 8
+
+
+def test_dense_inliers_without_outliers_is_plain_block_scaled_4bit_quantization():
+    """out_n = 0 and no pruning: the weight path is the activation path's 4-bit quantizer applied to W"""
+    Wb = tiny_W(24, 512, 17)
+    for block in (32, 64):
+        for rule in (so.SCALE_OCP_FLOOR, so.SCALE_CEIL_NOSAT):
+            cfg = so.Config(0, so.GRAN_DENSE, block, rule)
+            p = so.decompose(Wb, cfg)
+            q = so.quantize_act(Wb, cfg)
+            assert np.array_equal(p.in_code, q.xq4_code) and np.array_equal(p.in_scale, q.xq4_scale)
+            assert p.out_code.size == 0
+
+
+def test_unknown_inlier_pattern_rejected():
+    with pytest.raises(ValueError):
+        so.decompose(tiny_W(8, 128, 0), so.Config(1, 3, 64, so.SCALE_OCP_FLOOR))

@@ -18,7 +18,8 @@ def make(M, N, K, seed, cfg=CFG):
     return Wb, Xb, so.decompose(Wb, cfg), so.quantize_act(Xb, cfg)
 
 
-@pytest.mark.parametrize("cfg", [CFG, so.Config(2, so.GRAN_ELEM, 32, so.SCALE_CEIL_NOSAT), so.Config(0, so.GRAN_PAIR, 64, 0)])
+@pytest.mark.parametrize("cfg", [CFG, so.Config(2, so.GRAN_ELEM, 32, so.SCALE_CEIL_NOSAT), so.Config(0, so.GRAN_PAIR, 64, 0),
+                                 so.Config(1, so.GRAN_DENSE, 32, so.SCALE_OCP_FLOOR)])
 def test_brute_force_triple_loop(cfg):
     Wb, Xb, p, q = make(3, 16, 128, 2, cfg)
     W_in, W_out = so.dequant_weights(p)
@@ -51,6 +52,21 @@ def test_no_outliers_reduces_to_plain_quantized_gemm():
     assert not W_out.any()
     A_i, _ = so.dequant_act(q)
     assert np.allclose(so.linear(q, p), A_i @ W_in.T, rtol=1e-13, atol=1e-13)
+
+
+def test_dense_inliers_match_independent_definition_end_to_end():
+    cfg = so.Config(1, so.GRAN_DENSE, 32, so.SCALE_CEIL_NOSAT)
+    Wb, Xb, p, q = make(8, 64, 256, 9, cfg)
+    Win, Wout, _, _ = decompose_dense(Wb, 1, None, 32, False)
+    Ai, Ao = quantize_act_dense(Xb, 32, False)
+    assert np.allclose(so.linear(q, p), Ai @ Win.T + Ao @ Wout.T, rtol=1e-12, atol=1e-12)
+    # and it is closer to the unquantized product than the pruned decomposition of the same weights
+    W = torch.from_numpy(Wb.view(np.int16)).view(torch.bfloat16).double().numpy()
+    X = torch.from_numpy(Xb.view(np.int16)).view(torch.bfloat16).double().numpy()
+    cfg_p = so.Config(1, so.GRAN_PAIR, 32, so.SCALE_CEIL_NOSAT)
+    err_dense = np.linalg.norm(so.linear(q, p) - X @ W.T)
+    err_pruned = np.linalg.norm(so.linear(so.quantize_act(Xb, cfg_p), so.decompose(Wb, cfg_p)) - X @ W.T)
+    assert err_dense < err_pruned
 
 
 def test_one_hot_readback_returns_columns_of_W_in_plus_W_out():
@@ -129,3 +145,6 @@ def test_bits_per_weight_of_the_formats_used_here():
     assert so.bits_per_weight(so.Config(0, so.GRAN_PAIR, 64, 0)) == 2.625
     assert so.bits_per_weight(so.Config(2, so.GRAN_PAIR, 64, 0)) == 2.625 + 2.75
     assert so.bits_per_weight(so.Config(1, so.GRAN_ELEM, 32, 0)) == 2 + 1 + 0.25 + 1.375
+    # no pruning: 4-bit value at every position, one 8-bit scale per 32, plus the 1:8 outliers (8-bit value + 3-bit index)
+    assert so.bits_per_weight(so.Config(1, so.GRAN_DENSE, 32, 0)) == 4 + 0.25 + 1.375
+    assert so.bits_per_weight(so.Config(0, so.GRAN_DENSE, 64, 0)) == 4.125
