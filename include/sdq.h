@@ -38,7 +38,7 @@ typedef enum {
   SDQ_ERR_TIMEOUT = 8           /* a bounded device-side wait gave up (sticky device status) */
 } sdq_status_t;
 
-enum { SDQ_GRAN_PAIR = 0, SDQ_GRAN_ELEM = 1 };           /* inlier N:M granularity            */
+enum { SDQ_GRAN_PAIR = 0, SDQ_GRAN_ELEM = 1, SDQ_GRAN_DENSE = 2 }; /* inlier pattern            */
 enum { SDQ_SCALE_OCP_FLOOR = 0, SDQ_SCALE_CEIL_NOSAT = 1 }; /* E8M0 Q-Vector scale rule        */
 
 /* "pattern, formats" of the decomposition (Section 5, Stages 1-3).
@@ -48,7 +48,11 @@ enum { SDQ_SCALE_OCP_FLOOR = 0, SDQ_SCALE_CEIL_NOSAT = 1 }; /* E8M0 Q-Vector sca
  *              SDQ_GRAN_PAIR keeps the 2 adjacent pairs (of 4) with the largest |a|+|b| in every 8
  *              (the pattern the sparse FP4 tensor core consumes); SDQ_GRAN_ELEM keeps the 2 largest
  *              of every 4 (decompose / export only: the buffer then holds the canonical arrays and
- *              sdq_linear returns SDQ_ERR_UNSUPPORTED).
+ *              sdq_linear returns SDQ_ERR_UNSUPPORTED).  SDQ_GRAN_DENSE skips Stage 1: every value that
+ *              is not an outlier stays an inlier (the evaluation's configuration 8:8 = 1:8 outliers +
+ *              7:8 inliers); sdq_linear runs W_i as a dense 4-bit operand.  The dense 4-bit tensor-core
+ *              kind has one scale per 32 K only, so SDQ_GRAN_DENSE requires in_block = 32 (with 64 every
+ *              call returns SDQ_ERR_UNSUPPORTED).
  *   in_block   Q-Vector length: logical K sharing one E8M0 scale, for W_i and for the 4-bit
  *              activations: 64 or 32.  Both are executed by sdq_linear (64: kind::mxf4 .block32, the
  *              faster kernel; 32: kind::mxf4nvf4 .block16 with E8M0 scale codes).
@@ -88,8 +92,10 @@ typedef struct {
 /* Layout-free copies of the packed arrays, one code per byte, for bit-exact comparison
  * (all pointers: device memory, caller-owned, sizes in elements given beside each field). */
 typedef struct {
-  uint8_t* in_code;   /* [N][K/2]   E2M1 codes of the kept inlier slots in ascending k            */
-  uint8_t* in_meta;   /* [N][K/8] (PAIR) or [N][K/4] (ELEM): i0 | i1<<2, kept indices, ascending  */
+  uint8_t* in_code;   /* [N][K/2]   E2M1 codes of the kept inlier slots in ascending k
+                         (DENSE: [N][K], every position; outlier positions hold +0)                */
+  uint8_t* in_meta;   /* [N][K/8] (PAIR) or [N][K/4] (ELEM): i0 | i1<<2, kept indices, ascending
+                         (DENSE: not written, may be NULL)                                         */
   uint8_t* in_scale;  /* [N][K/in_block] E8M0 codes                                               */
   uint8_t* out_code;  /* [N][K/8][out_n] E4M3 codes                                               */
   uint8_t* out_idx;   /* [N][K/8][out_n] position 0..7 in the S-Vector, ascending                 */
@@ -167,7 +173,7 @@ sdq_status_t sdq_act_export(const sdq_act_t* Xq, const sdq_act_canonical_t* out,
  *   weights) while the previous kernel of the stream is still finishing, and waits for that kernel before it
  *   reads Xq or writes Y.  The packed weights must therefore be complete before the call is enqueued
  *   (sdq_decompose synchronises its stream, so a buffer it returned always is).
- *   Errors: INVALID_ARG, SHAPE, ALIGNMENT, UNSUPPORTED (in_gran != PAIR), CUDA. */
+ *   Errors: INVALID_ARG, SHAPE, ALIGNMENT, UNSUPPORTED (in_gran == ELEM), CUDA. */
 sdq_status_t sdq_linear(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y_bf16, int64_t ldy, void* stream);
 
 /* Same product, storing the fp32 accumulator itself (the value the bf16 output is rounded from). */

@@ -15,7 +15,7 @@ import torch
 
 from .build import LIB, build
 
-GRAN_PAIR, GRAN_ELEM = 0, 1
+GRAN_PAIR, GRAN_ELEM, GRAN_DENSE = 0, 1, 2
 SCALE_OCP_FLOOR, SCALE_CEIL_NOSAT = 0, 1
 
 STATUS = ["ok", "invalid_arg", "shape", "alignment", "unsupported", "buffer_too_small", "nonfinite", "cuda", "timeout"]
@@ -237,8 +237,9 @@ def sdq_linear_noalloc(xq: QuantAct, p: PackedWeight, out: torch.Tensor) -> torc
 def packed_export(p: PackedWeight) -> dict:
     N, K, on = p.N, p.K, p.cfg.out_n
     dev = p.buf.device
-    nmeta = K // 8 if p.cfg.in_gran == GRAN_PAIR else K // 4
-    t = dict(in_code=torch.zeros((N, K // 2), dtype=torch.uint8, device=dev),
+    dense = p.cfg.in_gran == GRAN_DENSE
+    nmeta = 0 if dense else (K // 8 if p.cfg.in_gran == GRAN_PAIR else K // 4)
+    t = dict(in_code=torch.zeros((N, K if dense else K // 2), dtype=torch.uint8, device=dev),
              in_meta=torch.zeros((N, nmeta), dtype=torch.uint8, device=dev),
              in_scale=torch.zeros((N, K // p.cfg.in_block), dtype=torch.uint8, device=dev),
              out_code=torch.zeros((N, K // 8, max(on, 1)), dtype=torch.uint8, device=dev),

@@ -15,6 +15,9 @@
 //     E_in : 128 rows x 16 B  (one 4-bit pair-index pair per 8 logical K over 256 K)
 //     SFA_in: 4 E8M0 scales (one per 64 K) of 128 rows: byte(r, s) at (r%32)*16 + (r/32)*4 + s
 //             (one scale per 32 K: two such atoms, one per 128-K block, 4 scales each; the record is 11264 B)
+//   no pruning (dense inliers, one scale per 32 K): WI[rt][k2] = | A_in 16384 | SFA_in 2 x 512 |   (17408 B)
+//     A_in : four K-blocks j (64 K each) of 128 rows x 32 B (all 64 E2M1 codes; outlier positions hold +0), same
+//            addressing; no E_in
 //   section WO[rt][k1] = | A_out 8192 | E_out 2048 |                                     (10240 B)
 //     A_out: two K-blocks j (64 logical K each) of 128 rows x 32 B (stored E4M3 bytes of the 2:4
 //            embedding of the 1:8 / 2:8 outliers), same addressing as A_in
@@ -53,7 +56,12 @@ constexpr int XO_BYTES = B8_BYTES;
 // One scale per 32 logical K (in_block = 32, run by kind::mxf4nvf4 .block16) doubles the scale atoms of the inlier
 // records: one atom per 128-K block (4 scales of 32 K each) instead of one per 256 K (4 scales of 64 K each).
 __host__ __device__ inline int sf_atoms(bool b32) { return b32 ? 2 : 1; }
-__host__ __device__ inline int wi_bytes(bool b32) { return A_IN_BYTES + E_IN_BYTES + sf_atoms(b32) * SF_ATOM_BYTES; }
+// dense inliers (no Stage 1): twice the codes, no pattern metadata
+__host__ __device__ inline int a_in_bytes(bool dense) { return dense ? 2 * A_IN_BYTES : A_IN_BYTES; }
+__host__ __device__ inline int e_in_bytes(bool dense) { return dense ? 0 : E_IN_BYTES; }
+__host__ __device__ inline int wi_bytes(bool b32, bool dense = false) {
+  return a_in_bytes(dense) + e_in_bytes(dense) + sf_atoms(b32) * SF_ATOM_BYTES;
+}
 __host__ __device__ inline int xi_bytes(bool b32) { return B4_BYTES + sf_atoms(b32) * SF_ATOM_BYTES; }
 // byte of the inlier scale of scale block `blk` (counted inside its 256-K record) of row / token `row` inside the
 // record's scale atoms: block 64 -> atom 0, slot blk (0..3); block 32 -> atom blk / 4, slot blk % 4
@@ -63,7 +71,7 @@ __host__ __device__ inline uint32_t in_sf_off(bool b32, uint32_t row, uint32_t b
 
 // byte offset inside an operand block of K-blocks of `kb_bytes` whose rows carry `row_bytes` per K-block
 //   A operands: row_bytes 32, kb_bytes 4096 (LBO 128, SBO 256);  B operands: one block, row_bytes 128 (SBO 1024)
-__host__ __device__ inline uint32_t a_off(uint32_t row, uint32_t byte /*0..63*/) {
+__host__ __device__ inline uint32_t a_off(uint32_t row, uint32_t byte /*0..63; dense inliers 0..127*/) {
   const uint32_t j = byte >> 5, b = byte & 31;
   return j * 4096 + (row >> 3) * 256 + (b >> 4) * 128 + (row & 7) * 16 + (b & 15);
 }
@@ -77,12 +85,12 @@ constexpr size_t HEADER_BYTES = 256;
 struct PackedOffsets {
   size_t wi, wo, sfa_out, ocode, oidx, osexp, total;
 };
-inline PackedOffsets packed_offsets(int64_t N, int64_t K, int out_n, bool b32 = false) {
+inline PackedOffsets packed_offsets(int64_t N, int64_t K, int out_n, bool b32 = false, bool dense = false) {
   PackedOffsets o;
   const size_t RT = (size_t)(N / TILE_ROWS), T1 = (size_t)(K / K1), T2 = (size_t)(K / K2);
   auto al = [](size_t x) { return (x + 255) & ~(size_t)255; };
   o.wi = HEADER_BYTES;
-  o.wo = al(o.wi + RT * T2 * (size_t)wi_bytes(b32));
+  o.wo = al(o.wi + RT * T2 * (size_t)wi_bytes(b32, dense));
   o.sfa_out = al(o.wo + (out_n ? RT * T1 * WO_BYTES : 0));
   o.ocode = al(o.sfa_out + RT * SF_ATOM_BYTES);
   o.oidx = al(o.ocode + (size_t)N * (size_t)(K / 8) * (size_t)out_n);

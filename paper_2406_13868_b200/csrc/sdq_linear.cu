@@ -48,9 +48,10 @@ constexpr uint32_t TM_META_COLS = 84;
 // slot = | A record 10752 | B n_tile*128 | scale atoms 1536 |  (inlier: SFB_in x n_atiles; first outlier stage:
 // SFA_out | SFB_out x n_atiles)
 // (one scale per 32 K: the weight record is 512 B longer and an inlier stage carries two scale atoms per token tile)
-__host__ __device__ inline int slot_bytes_for(int n_tile, bool b32 = false) {
+// (dense inliers: the weight record holds twice the codes and no pattern metadata)
+__host__ __device__ inline int slot_bytes_for(int n_tile, bool b32 = false, bool dense = false) {
   const int n_atiles = (n_tile + TILE_TOK - 1) / TILE_TOK, atoms = b32 ? (2 * n_atiles > 1 + n_atiles ? 2 * n_atiles : 1 + n_atiles) : 3;
-  return wi_bytes(b32) + n_tile * 128 + atoms * SF_ATOM_BYTES;
+  return wi_bytes(b32, dense) + n_tile * 128 + atoms * SF_ATOM_BYTES;
 }
 
 struct TileCoord {
@@ -107,8 +108,9 @@ sdq_linear_kernel(const LinearParams p)
   const int n_atiles = (n_tile + TILE_TOK - 1) / TILE_TOK;     // 128-token activation tiles per token tile
   const uint32_t nslot = FLEX ? (uint32_t)p.nslot : (B32 ? 4u : 5u), slot_bytes = FLEX ? (uint32_t)p.slot_bytes : (B32 ? 46080u : 45056u);
   const bool b32 = FLEX ? (p.b32 != 0) : B32;              // one scale per 32 K
+  const bool dense = FLEX ? (p.dense != 0) : false;        // dense inliers (always with one scale per 32 K)
   constexpr uint32_t MS = B32 ? 32u : 16u;                 // many tokens: metadata / scale columns per ring slot
-  const uint32_t wib = (uint32_t)wi_bytes(b32), xib = (uint32_t)xi_bytes(b32), na = b32 ? 2u : 1u;
+  const uint32_t wib = (uint32_t)wi_bytes(b32, dense), xib = (uint32_t)xi_bytes(b32), na = b32 ? 2u : 1u;
   const uint32_t sl_b = wib;                               // B4 / B8 follow the (longest) weight record
   const uint32_t sl_sf = sl_b + (uint32_t)n_tile * 128u;
 
@@ -209,10 +211,12 @@ sdq_linear_kernel(const LinearParams p)
       const uint32_t id4[2] = {ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, true, 0, 0),
                                ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, true, 2, 2)};
       const uint32_t id8 = ptx::idesc_block_scaled(128, (uint32_t)n_tile, 0, true, 0, 0);
+      const uint32_t idd[2] = {ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, false, 0, 0),      // dense inliers
+                               ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, false, 2, 2)};
       // descriptors of slot 0; slot s adds s * slot_bytes / 16 to the start-address field
       const uint64_t d_a = ptx::smem_desc(smb + SL_A, 128, 256), d_b = ptx::smem_desc(smb + sl_b, 128, 1024);
       const uint64_t d_e_in = ptx::smem_desc(smb + SL_A + A_IN_BYTES, 0, 128);
-      const uint64_t d_sfa_in = ptx::smem_desc(smb + SL_A + A_IN_BYTES + E_IN_BYTES, 0, 128);
+      const uint64_t d_sfa_in = ptx::smem_desc(smb + SL_A + (uint32_t)(a_in_bytes(dense) + e_in_bytes(dense)), 0, 128);
       const uint64_t d_e_out = ptx::smem_desc(smb + SL_A + A_OUT_BYTES, 0, 128);
       const uint64_t d_sf0 = ptx::smem_desc(smb + sl_sf, 0, 128), d_sf1 = ptx::smem_desc(smb + sl_sf + SF_ATOM_BYTES, 0, 128);
       const uint64_t d_sf2 = ptx::smem_desc(smb + sl_sf + 2 * SF_ATOM_BYTES, 0, 128);
@@ -269,7 +273,7 @@ sdq_linear_kernel(const LinearParams p)
           if (k < ni) {
             // inlier stage: 256 logical K = 2 sparse MXFP4 MMAs; metadata and scale atoms go to TMEM first
             const uint32_t mb = tmem + TM_I + 32u * (uint32_t)(k & 1);
-            ptx::tc_cp_128x128b(mb + 0, d_e_in + so);
+            if (!dense) ptx::tc_cp_128x128b(mb + 0, d_e_in + so);
             ptx::tc_cp_32x128b_warpx4(mb + 4, d_sfa_in + so);
             if (!b32) {
               ptx::tc_cp_32x128b_warpx4(mb + 8, d_sf0 + so);
@@ -283,9 +287,19 @@ sdq_linear_kernel(const LinearParams p)
               for (uint32_t a = 0; a < (uint32_t)n_atiles; ++a)
                 for (uint32_t kb = 0; kb < 2; ++kb)
                   ptx::tc_cp_32x128b_warpx4(mb + 12 + 4 * (kb * (uint32_t)n_atiles + a), d_sf0 + so + (((2 * a + kb) * SF_ATOM_BYTES) >> 4));
-              ptx::mma_sp_nvf4(tmem + TM_D, d_a + so, d_b + so, id4[0], mb, mb + 4, mb + 12, acc);
-              ptx::mma_sp_nvf4(tmem + TM_D, d_a + so + (4096 >> 4), d_b + so + (512 >> 4), id4[0], mb + 2, mb + 8,
-                               mb + 12 + 4 * (uint32_t)n_atiles, 1u);
+              if (!dense) {
+                ptx::mma_sp_nvf4(tmem + TM_D, d_a + so, d_b + so, id4[0], mb, mb + 4, mb + 12, acc);
+                ptx::mma_sp_nvf4(tmem + TM_D, d_a + so + (4096 >> 4), d_b + so + (512 >> 4), id4[0], mb + 2, mb + 8,
+                                 mb + 12 + 4 * (uint32_t)n_atiles, 1u);
+              } else {
+                // dense inliers: four MMAs of 64 K; MMA j reads K-block j of the weights (4096 B apart), bytes 32 j .. 32 j + 31
+                // of every token (two 16-byte chunks, 256 B apart per j) and scales 2 (j & 1), 2 (j & 1) + 1 of the scale
+                // word of 128-K block j / 2
+#pragma unroll
+                for (uint32_t j = 0; j < 4; ++j)
+                  ptx::mma_mxf4(tmem + TM_D, d_a + so + ((4096 * j) >> 4), d_b + so + ((256 * j) >> 4), idd[j & 1], mb + 4 + 4 * (j >> 1),
+                                mb + 12 + 4 * (uint32_t)n_atiles * (j >> 1), j ? 1u : acc);
+              }
             }
           } else {
             // outlier stage: 128 logical K = 2 sparse FP8 MMAs; the row / token scales (E8M0) arrive with the first one
@@ -580,7 +594,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   if (!Xq || !P || !Y || !Xq->dev || !P->dev) return SDQ_ERR_INVALID_ARG;
   if (Xq->K != P->K || Xq->M <= 0 || P->N <= 0 || P->N % TILE_ROWS || P->K % K2 || ldy < P->N) return SDQ_ERR_SHAPE;
   if (Xq->cfg.in_block != P->cfg.in_block || Xq->cfg.scale_rule != P->cfg.scale_rule) return SDQ_ERR_SHAPE;
-  if (P->cfg.in_gran != SDQ_GRAN_PAIR) return SDQ_ERR_UNSUPPORTED;
+  if (P->cfg.in_gran != SDQ_GRAN_PAIR && !(P->cfg.in_gran == SDQ_GRAN_DENSE && P->cfg.in_block == 32)) return SDQ_ERR_UNSUPPORTED;
   if (((uintptr_t)Y & 15) || (ldy % 8) || ((uintptr_t)ws & 15)) return SDQ_ERR_ALIGNMENT;
   static bool attr_set = false;
   if (!attr_set) {
@@ -599,14 +613,15 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   p.w = (const uint8_t*)P->dev;
   p.x = (const uint8_t*)Xq->dev;
   p.b32 = P->cfg.in_block == 32 ? 1 : 0;
-  p.poff = packed_offsets(P->N, P->K, P->cfg.out_n, p.b32 != 0);
+  p.dense = P->cfg.in_gran == SDQ_GRAN_DENSE ? 1 : 0;
+  p.poff = packed_offsets(P->N, P->K, P->cfg.out_n, p.b32 != 0, p.dense != 0);
   p.aoff = act_offsets(Xq->M, Xq->K, p.b32 != 0);
   p.M = Xq->M; p.N = P->N; p.K = P->K;
   p.out_n = P->cfg.out_n;
   const int64_t M = Xq->M;
   p.n_tile = n_tile_for(M);
   p.n_mtiles = (int)((M + p.n_tile - 1) / p.n_tile);
-  p.slot_bytes = slot_bytes_for(p.n_tile, p.b32 != 0);
+  p.slot_bytes = slot_bytes_for(p.n_tile, p.b32 != 0, p.dense != 0);
   p.ksplit = 1;
   p.cluster_ks = 1;
   p.ws_counter = nullptr;
@@ -697,7 +712,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   }
   lc.attrs = attr;
   lc.numAttrs = na;
-  const bool flex = !(p.n_tile == 256 && p.ksplit == 1 && p.nslot == (p.b32 ? 4 : 5) && p.release == 1);
+  const bool flex = p.dense || !(p.n_tile == 256 && p.ksplit == 1 && p.nslot == (p.b32 ? 4 : 5) && p.release == 1);
   cudaError_t le;
   if (flex) le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, true, false>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, true, false>, p);
   else if (p.b32) le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, false, true>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, false, true>, p);

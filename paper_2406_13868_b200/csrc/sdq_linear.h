@@ -24,6 +24,7 @@ struct LinearParams {
   int tmem_cols;         // TMEM columns to allocate (128, 256 or 512)
   int meta_col;          // first TMEM column of the metadata / scale buffers
   int b32;               // 1: one inlier / activation scale per 32 K (kind::mxf4nvf4 .block16), runtime geometry only
+  int dense;             // 1: dense inliers (no Stage 1): 4 dense kind::mxf4 MMAs of 64 K per stage, runtime geometry only
   int ksplit;            // CTAs sharing the K range of one row tile (1 = no split)
   int cluster_ks;        // > 1: those CTAs form a cluster and reduce through distributed shared memory
   uint32_t* ws_counter;  // split-K workspace: arrival counters [row tile], zero between calls

@@ -3,7 +3,8 @@
 // One CTA per weight row; one thread per S-Vector of 8 consecutive K (a single 16-byte load).
 // Pass 1 finds the row's largest outlier magnitude (the per-row power-of-two scale); pass 2 selects
 // outliers, prunes the rest pair-wise, derives the Q-Vector scales by an 8-lane shuffle reduction
-// (8 S-Vectors = 64 K), encodes, and scatters into the stage-tiled layout of sdq_layout.h.
+// (8 S-Vectors = 64 K), encodes, and scatters into the stage-tiled layout of sdq_layout.h.  Without Stage 1 (dense
+// inliers) every position that is not an outlier is encoded, with one scale per 32 K.
 #include "sdq_codec.cuh"
 #include "sdq_internal.h"
 #include "sdq_layout.h"
@@ -95,8 +96,8 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
   const int64_t rt = n / TILE_ROWS;
   const uint32_t r = (uint32_t)(n % TILE_ROWS);
   const int T1 = (int)(K / K1), T2 = (int)(K / K2);
-  const bool b32 = cfg.in_block == 32;
-  const int wib = wi_bytes(b32);
+  const bool b32 = cfg.in_block == 32, dense = cfg.in_gran == SDQ_GRAN_DENSE;
+  const int wib = wi_bytes(b32, dense);
   uint8_t* wi_base = blob + off.wi + (size_t)rt * T2 * wib;
   uint8_t* wo_base = blob + off.wo + (size_t)rt * T1 * WO_BYTES;
 
@@ -116,7 +117,31 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     selection_keys(key, colw, g, skey);
     int o0, o1;
     select_outliers(skey, out_n, o0, o1);
+    const int k1 = g >> 4, k2 = g >> 5;
+    uint8_t* wi = wi_base + (size_t)k2 * wib;
+    uint8_t* wo = wo_base + (size_t)k1 * WO_BYTES;
 
+    if (dense) {
+      // no Stage 1: all eight positions are inlier slots (an outlier position holds +0).  Stage 3 with one scale per
+      // 32 K = 4 S-Vectors = 4 lanes
+      uint32_t ikey = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if (i != o0 && i != o1) ikey = max(ikey, key[i]);
+      ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 1));
+      ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 2));
+      const uint32_t c = e8m0_scale_code(bf16_bits_to_float(ikey), cfg.scale_rule);
+      uint32_t codes = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float v0 = (2 * i == o0 || 2 * i == o1) ? 0.0f : bf16_bits_to_float(bits[2 * i]) * pow2_inv_e8m0(c);
+        const float v1 = (2 * i + 1 == o0 || 2 * i + 1 == o1) ? 0.0f : bf16_bits_to_float(bits[2 * i + 1]) * pow2_inv_e8m0(c);
+        codes |= e2m1x2(v0, v1) << (8 * i);
+      }
+      // 32 S-Vectors per 256-K stage, 4 code bytes each: bytes 32 j .. 32 j + 31 = K-block j (64 K)
+      *reinterpret_cast<uint32_t*>(wi + a_off(r, (uint32_t)(g & 31) * 4)) = codes;
+      if ((g & 3) == 0) wi[a_in_bytes(true) + in_sf_off(true, r, (uint32_t)((g >> 2) & 7))] = (uint8_t)c;
+    } else {
     // Stage 1 on the remaining values: keep the 2 pairs (of 4) with the largest summed significance
     float score[4];
 #pragma unroll
@@ -157,9 +182,6 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     }
     const uint32_t codes = e2m1x2(v[0], v[1]) | (e2m1x2(v[2], v[3]) << 8);
 
-    const int k1 = g >> 4, k2 = g >> 5;
-    uint8_t* wi = wi_base + (size_t)k2 * wib;
-    uint8_t* wo = wo_base + (size_t)k1 * WO_BYTES;
     // 32 S-Vectors per 256-K stage, 2 code bytes each: bytes 0..31 = K-block 0, 32..63 = K-block 1
     *reinterpret_cast<uint16_t*>(wi + a_off(r, (uint32_t)(g & 31) * 2)) = (uint16_t)codes;
     // metadata nibble j0 | j1<<2; two S-Vectors share a byte (even one in the low nibble)
@@ -168,6 +190,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     if ((g & 1) == 0) wi[A_IN_BYTES + r * 16 + ((g & 31) >> 1)] = (uint8_t)(nib | (nib_hi << 4));
     if (b32) { if ((g & 3) == 0) wi[A_IN_BYTES + E_IN_BYTES + in_sf_off(true, r, (uint32_t)((g >> 2) & 7))] = (uint8_t)c; }
     else if ((g & 7) == 0) wi[A_IN_BYTES + E_IN_BYTES + in_sf_off(false, r, (uint32_t)((g >> 3) & 3))] = (uint8_t)c;
+    }
 
     if (out_n > 0) {
       // Stage 3, outliers: E4M3 codes of w / 2^e; compact arrays plus the 2:4 embedding the sparse
@@ -211,11 +234,23 @@ export_packed_kernel(const uint8_t* __restrict__ blob, int64_t N, int64_t K, sdq
   const int64_t rt = n / TILE_ROWS;
   const uint32_t r = (uint32_t)(n % TILE_ROWS);
   const int T2 = (int)(K / K2);
-  const bool b32 = cfg.in_block == 32;
-  const int wib = wi_bytes(b32);
+  const bool b32 = cfg.in_block == 32, dense = cfg.in_gran == SDQ_GRAN_DENSE;
+  const int wib = wi_bytes(b32, dense);
   const uint8_t* wi_base = blob + off.wi + (size_t)rt * T2 * wib;
   for (int g = threadIdx.x; g < G; g += 128) {
     const uint8_t* wi = wi_base + (size_t)(g >> 5) * wib;
+    if (dense) {
+      const uint32_t codes = *reinterpret_cast<const uint32_t*>(wi + a_off(r, (uint32_t)(g & 31) * 4));
+      uint8_t* ic = out.in_code + (size_t)n * K + 8 * g;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) ic[i] = (codes >> (4 * i)) & 15;
+      if ((g & 3) == 0) out.in_scale[(size_t)n * (K / 32) + (g >> 2)] = wi[a_in_bytes(true) + in_sf_off(true, r, (uint32_t)((g >> 2) & 7))];
+      for (int t = 0; t < out_n; ++t) {
+        out.out_code[((size_t)n * G + g) * out_n + t] = blob[off.ocode + ((size_t)n * G + g) * out_n + t];
+        out.out_idx[((size_t)n * G + g) * out_n + t] = blob[off.oidx + ((size_t)n * G + g) * out_n + t];
+      }
+      continue;
+    }
     const uint32_t codes = *reinterpret_cast<const uint16_t*>(wi + a_off(r, (uint32_t)(g & 31) * 2));
     uint8_t* ic = out.in_code + (size_t)n * (K / 2) + 4 * g;
     ic[0] = codes & 15; ic[1] = (codes >> 4) & 15; ic[2] = (codes >> 8) & 15; ic[3] = (codes >> 12) & 15;
@@ -236,20 +271,23 @@ export_packed_kernel(const uint8_t* __restrict__ blob, int64_t N, int64_t K, sdq
 using namespace sdq;
 
 static bool cfg_ok(const sdq_config_t* c) {
-  return c && c->out_n >= 0 && c->out_n <= 2 && (c->in_gran == SDQ_GRAN_PAIR || c->in_gran == SDQ_GRAN_ELEM) &&
+  return c && c->out_n >= 0 && c->out_n <= 2 && (c->in_gran == SDQ_GRAN_PAIR || c->in_gran == SDQ_GRAN_ELEM || c->in_gran == SDQ_GRAN_DENSE) &&
          (c->in_block == 32 || c->in_block == 64) && (c->scale_rule == SDQ_SCALE_OCP_FLOOR || c->scale_rule == SDQ_SCALE_CEIL_NOSAT);
 }
 
 extern "C" sdq_status_t sdq_packed_size(int64_t N, int64_t K, const sdq_config_t* cfg, size_t* bytes, size_t* algorithmic_bytes)
 {
   if (!cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
+  if (cfg->in_gran == SDQ_GRAN_DENSE && cfg->in_block != 32) return SDQ_ERR_UNSUPPORTED;
   if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2) return SDQ_ERR_SHAPE;
-  if (bytes) *bytes = is_tensor_core_reading(*cfg) ? packed_offsets(N, K, cfg->out_n, cfg->in_block == 32).total : plain_packed_offsets(N, K, *cfg).total;
+  if (bytes) *bytes = is_tensor_core_reading(*cfg) ? packed_offsets(N, K, cfg->out_n, cfg->in_block == 32, cfg->in_gran == SDQ_GRAN_DENSE).total : plain_packed_offsets(N, K, *cfg).total;
   if (algorithmic_bytes) {
     // per weight: 4-bit values on half the positions (2) + index metadata (pair-wise: two 2-bit pair indices per 8 =
     // 0.5; element-wise: two 2-bit indices per 4 = 1) + one 8-bit scale per Q-Vector + out_n * (8 value + 3 index
     // bits) per 8; plus one 32-bit row scale
-    const double bits = 2.0 + (cfg->in_gran == SDQ_GRAN_PAIR ? 0.5 : 1.0) + 8.0 / cfg->in_block + cfg->out_n * 11.0 / 8.0;
+    // (no pruning: a 4-bit value on every position and no index metadata)
+    const double inl = cfg->in_gran == SDQ_GRAN_DENSE ? 4.0 : 2.0 + (cfg->in_gran == SDQ_GRAN_PAIR ? 0.5 : 1.0);
+    const double bits = inl + 8.0 / cfg->in_block + cfg->out_n * 11.0 / 8.0;
     *algorithmic_bytes = (size_t)((double)N * (double)K * bits / 8.0) + (cfg->out_n ? (size_t)N * 4 : 0);
   }
   return SDQ_OK;
@@ -264,11 +302,12 @@ extern "C" sdq_status_t sdq_decompose_metric(const void* W, int64_t N, int64_t K
                                              void* stream)
 {
   if (!W || !packed_buf || !out || !cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
+  if (cfg->in_gran == SDQ_GRAN_DENSE && cfg->in_block != 32) return SDQ_ERR_UNSUPPORTED;
   if ((uintptr_t)col_weight & 15) return SDQ_ERR_ALIGNMENT;
   if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2 || ldw < K) return SDQ_ERR_SHAPE;
   if (((uintptr_t)W & 15) || ((uintptr_t)packed_buf & 15) || (ldw % 8)) return SDQ_ERR_ALIGNMENT;
   const bool tc = is_tensor_core_reading(*cfg);
-  const PackedOffsets off = packed_offsets(N, K, cfg->out_n, cfg->in_block == 32);
+  const PackedOffsets off = packed_offsets(N, K, cfg->out_n, cfg->in_block == 32, cfg->in_gran == SDQ_GRAN_DENSE);
   const PlainPackedOffsets poff = plain_packed_offsets(N, K, *cfg);
   if (packed_bytes < (tc ? off.total : poff.total)) return SDQ_ERR_BUFFER_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
@@ -299,7 +338,8 @@ extern "C" sdq_status_t sdq_decompose_metric(const void* W, int64_t N, int64_t K
 
 extern "C" sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canonical_t* out, void* stream)
 {
-  if (!P || !out || !P->dev || !out->in_code || !out->in_meta || !out->in_scale || !out->out_sexp) return SDQ_ERR_INVALID_ARG;
+  if (!P || !out || !P->dev || !out->in_code || !out->in_scale || !out->out_sexp) return SDQ_ERR_INVALID_ARG;
+  if (!out->in_meta && P->cfg.in_gran != SDQ_GRAN_DENSE) return SDQ_ERR_INVALID_ARG;
   if (P->cfg.out_n > 0 && (!out->out_code || !out->out_idx)) return SDQ_ERR_INVALID_ARG;
   if (!is_tensor_core_reading(P->cfg)) {
     // the buffer already holds the canonical arrays
@@ -317,7 +357,7 @@ extern "C" sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canon
     ok = ok && cudaMemcpyAsync(out->out_sexp, b + o.osexp, n * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
     return ok ? SDQ_OK : SDQ_ERR_CUDA;
   }
-  const PackedOffsets off = packed_offsets(P->N, P->K, P->cfg.out_n, P->cfg.in_block == 32);
+  const PackedOffsets off = packed_offsets(P->N, P->K, P->cfg.out_n, P->cfg.in_block == 32, P->cfg.in_gran == SDQ_GRAN_DENSE);
   export_packed_kernel<<<(unsigned)P->N, 128, 0, (cudaStream_t)stream>>>((const uint8_t*)P->dev, P->N, P->K, P->cfg, off, *out);
   return cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
 }

@@ -103,6 +103,17 @@ __device__ __forceinline__ void tc_cp_32x128b_warpx4(uint32_t taddr, uint64_t sd
   asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
 }
 
+// D[128 x N] (+)= A[128 x 64 K] * B[N x 64]^T, dense E2M1 operands, one E8M0 scale per 32 K (two bytes of the scale
+// word, chosen by the scale-factor ids of the instruction descriptor: 0 -> bytes 0, 1; 2 -> bytes 2, 3)
+__device__ __forceinline__ void mma_mxf4(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t sfa, uint32_t sfb,
+                                         uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n}" ::"r"(d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
+      : "memory");
+}
+
 // D[128 x N] (+)= A_sparse[128 x 128 logical K] * B[N x 128]^T, E2M1 operands, one E8M0 scale per 64 K
 __device__ __forceinline__ void mma_sp_mxf4(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t e_tmem,
                                             uint32_t sfa, uint32_t sfb, uint32_t accumulate) {

@@ -14,8 +14,8 @@ def sdq():
     return m
 
 
-def ocfg(out_n=1, rule=0, block=64):
-    return so.Config(out_n, so.GRAN_PAIR, block, rule)
+def ocfg(out_n=1, rule=0, block=64, gran=so.GRAN_PAIR):
+    return so.Config(out_n, gran, block, rule)
 
 
 def y_close(y_gpu, y_ref):
@@ -25,9 +25,9 @@ def y_close(y_gpu, y_ref):
     return d, tol
 
 
-def run_case(M, N, K, seed, out_n=1, rule=0, n_out_ch=None, check_rows=None, block=64):
+def run_case(M, N, K, seed, out_n=1, rule=0, n_out_ch=None, check_rows=None, block=64, gran=so.GRAN_PAIR):
     m = sdq()
-    cfg = m.Config(out_n, m.GRAN_PAIR, block, rule)
+    cfg = m.Config(out_n, gran, block, rule)
     W = sdq_synth.make_weight(N, K, seed)
     X = sdq_synth.make_act(M, K, seed, n_outlier_channels=n_out_ch)
     p = m.sdq_decompose(W.cuda(), cfg)
@@ -35,8 +35,8 @@ def run_case(M, N, K, seed, out_n=1, rule=0, n_out_ch=None, check_rows=None, blo
     y32 = m.sdq_linear(xq, p, f32=True)
     y16 = m.sdq_linear(xq, p)
     assert m.device_status() == 0
-    op = so.decompose(sdq_synth.bf16_bits(W), ocfg(out_n, rule, block))
-    oq = so.quantize_act(sdq_synth.bf16_bits(X), ocfg(out_n, rule, block))
+    op = so.decompose(sdq_synth.bf16_bits(W), ocfg(out_n, rule, block, gran))
+    oq = so.quantize_act(sdq_synth.bf16_bits(X), ocfg(out_n, rule, block, gran))
     pe = {k: v.cpu().numpy() for k, v in m.packed_export(p).items()}
     ae = {k: v.cpu().numpy() for k, v in m.act_export(xq).items()}
     for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp"):
@@ -134,6 +134,45 @@ def test_block_32_one_hot_readback():
     W_in, W_out = so.dequant_weights(so.decompose(sdq_synth.bf16_bits(W), ocfg(block=32)))
     assert np.array_equal(y, (W_in + W_out).T)
     assert m.device_status() == 0
+
+
+@pytest.mark.parametrize("M,N,K,out_n,rule", [(8, 256, 256, 1, 0), (1, 512, 2048, 1, 0), (16, 256, 4096, 2, 1), (33, 128, 768, 0, 0),
+                                              (100, 256, 2816, 1, 0), (128, 1024, 4096, 1, 0), (129, 256, 512, 1, 1),
+                                              (300, 512, 1024, 2, 0), (520, 6400, 256, 1, 0), (700, 2560, 1024, 1, 1)])
+def test_dense_inliers_through_the_tensor_core(M, N, K, out_n, rule):
+    """no Stage 1 (8:8 split as out_n:8 outliers + dense 4-bit inliers, one scale per 32 K): packed arrays bit-exact, the
+    inlier product on the dense kind::mxf4 MMA; few tokens, cluster split K, several hundred tokens, persistent CTAs"""
+    run_case(M, N, K, 1200 + M, out_n=out_n, rule=rule, block=32, gran=so.GRAN_DENSE)
+
+
+def test_dense_inliers_one_hot_readback_and_workspace_split():
+    m = sdq()
+    cfg = m.Config(1, m.GRAN_DENSE, 32, 0)
+    N, K = 256, 512
+    W = sdq_synth.make_weight(N, K, 71)
+    p = m.sdq_decompose(W.cuda(), cfg)
+    X = torch.eye(K, dtype=torch.bfloat16)
+    xq = m.sdq_quantize_act(X.cuda(), cfg)
+    y = m.sdq_linear(xq, p, f32=True).cpu().numpy().astype(np.float64)
+    op = so.decompose(sdq_synth.bf16_bits(W), ocfg(block=32, gran=so.GRAN_DENSE))
+    W_in, W_out = so.dequant_weights(op)
+    assert np.array_equal(y, (W_in + W_out).T)
+    # K split through a caller workspace: same criterion, identical from call to call
+    M = 7
+    Xs = sdq_synth.make_act(M, K, 72)
+    xs = m.sdq_quantize_act(Xs.cuda(), cfg)
+    ws = m.make_workspace(M, N, K, cfg, "cuda")
+    assert ws is not None
+    y1 = m.sdq_linear(xs, p, f32=True, workspace=ws)
+    y2 = m.sdq_linear(xs, p, f32=True, workspace=ws)
+    assert torch.equal(y1, y2)
+    d, tol = y_close(y1.cpu().numpy(), so.linear(so.quantize_act(sdq_synth.bf16_bits(Xs), op.cfg), op))
+    assert (d <= tol).all()
+    assert m.device_status() == 0
+    # the dense 4-bit tensor-core kind has no scale per 64 K
+    with pytest.raises(m.SdqError) as e:
+        m.sdq_decompose(W.cuda(), m.Config(1, m.GRAN_DENSE, 64, 0))
+    assert e.value.code == 4
 
 
 def test_one_hot_readback_512_tokens():
@@ -260,7 +299,7 @@ def test_activation_quantizer_row_lengths(M, K, rule, block):
         assert np.array_equal(ae[name], getattr(oq, name)), name
 
 
-@pytest.mark.parametrize("gran,block", [(1, 64), (0, 32), (0, 64)])
+@pytest.mark.parametrize("gran,block", [(1, 64), (0, 32), (0, 64), (2, 32)])
 @pytest.mark.parametrize("out_n", [0, 1, 2])
 def test_product_metric_packer(gran, block, out_n):
     """sdq_decompose_metric: selections by |w| * c[k]; packed arrays bit-exact against the oracle for the tensor-core
@@ -282,8 +321,11 @@ def test_product_metric_packer(gran, block, out_n):
         assert np.array_equal(pe[name], getattr(op, name)), name
     # it does change the selection (otherwise the test would prove nothing)
     om = so.decompose(sdq_synth.bf16_bits(W), oc)
-    assert not np.array_equal(op.in_meta, om.in_meta)
-    if gran == m.GRAN_PAIR and block == 64:
+    if gran == m.GRAN_DENSE:
+        assert out_n == 0 or not np.array_equal(op.out_idx, om.out_idx)
+    else:
+        assert not np.array_equal(op.in_meta, om.in_meta)
+    if gran != m.GRAN_ELEM:
         X = sdq_synth.make_act(M, K, 41)
         xq = m.sdq_quantize_act(X.cuda(), cfg)
         y = m.sdq_linear(xq, p, f32=True).cpu().numpy()
