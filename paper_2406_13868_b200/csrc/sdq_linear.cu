@@ -80,7 +80,8 @@ __device__ __forceinline__ TileCoord tile_coord(int ksplit, int tile, int RT, in
 // geometry constant known at compile time -- the single-thread issue loops are latency-bound, so each runtime
 // parameter they touch costs time.  FLEX = true: geometry from the launch parameters (few tokens, split K).
 // B32 (many-token instantiation only): one scale per 32 K, four ring slots of 45 KB.
-template <bool F32_OUT, bool FLEX, bool B32>
+// DENSE (many-token instantiation only): dense inliers with one scale per 32 K, four ring slots of 51 KB.
+template <bool F32_OUT, bool FLEX, bool B32, bool DENSE>
 __global__ void __maxnreg__(96)   // two 9-warp CTAs share an SM only below ~100 registers per thread
 sdq_linear_kernel(const LinearParams p)
 {
@@ -90,7 +91,10 @@ sdq_linear_kernel(const LinearParams p)
   const int ksplit = FLEX ? p.ksplit : 1, cluster_ks = FLEX ? p.cluster_ks : 1;
   const bool release = FLEX ? (p.release != 0) : true;
   // the transpose buffer and the barriers follow the ring (many tokens: 5 x 45056, or 4 x 46080 with one scale per 32 K)
-  const uint32_t SM_STG = FLEX ? (uint32_t)p.ring_bytes : (B32 ? 4u * 46080u : (uint32_t)RING_BYTES), SM_BARS = SM_STG + 4096;
+  static_assert(!(FLEX && (B32 || DENSE)) && !(B32 && DENSE), "B32 and DENSE name many-token instantiations");
+  constexpr bool S32 = B32 || DENSE;                       // many tokens with one scale per 32 K
+  constexpr uint32_t SLOT_FIXED = DENSE ? 52224u : (B32 ? 46080u : 45056u), NSLOT_FIXED = S32 ? 4u : 5u;
+  const uint32_t SM_STG = FLEX ? (uint32_t)p.ring_bytes : (S32 ? NSLOT_FIXED * SLOT_FIXED : (uint32_t)RING_BYTES), SM_BARS = SM_STG + 4096;
   const uint32_t TM_I = FLEX ? (uint32_t)p.meta_col : 256u, TM_EO = TM_I + 64, TM_SFA_OUT = TM_I + 72, TM_SFB_OUT = TM_I + 76;
   const uint32_t tmem_cols = FLEX ? (uint32_t)p.tmem_cols : 512u;
   uint64_t* full = reinterpret_cast<uint64_t*>(sm + SM_BARS);
@@ -106,10 +110,10 @@ sdq_linear_kernel(const LinearParams p)
   const int RT = (int)(p.N / TILE_ROWS);
   const int T1 = p.out_n ? (int)(p.K / K1) : 0, T2 = (int)(p.K / K2);
   const int n_atiles = (n_tile + TILE_TOK - 1) / TILE_TOK;     // 128-token activation tiles per token tile
-  const uint32_t nslot = FLEX ? (uint32_t)p.nslot : (B32 ? 4u : 5u), slot_bytes = FLEX ? (uint32_t)p.slot_bytes : (B32 ? 46080u : 45056u);
-  const bool b32 = FLEX ? (p.b32 != 0) : B32;              // one scale per 32 K
-  const bool dense = FLEX ? (p.dense != 0) : false;        // dense inliers (always with one scale per 32 K)
-  constexpr uint32_t MS = B32 ? 32u : 16u;                 // many tokens: metadata / scale columns per ring slot
+  const uint32_t nslot = FLEX ? (uint32_t)p.nslot : NSLOT_FIXED, slot_bytes = FLEX ? (uint32_t)p.slot_bytes : SLOT_FIXED;
+  const bool b32 = FLEX ? (p.b32 != 0) : S32;              // one scale per 32 K
+  const bool dense = FLEX ? (p.dense != 0) : DENSE;        // dense inliers (always with one scale per 32 K)
+  constexpr uint32_t MS = S32 ? 32u : 16u;                 // many tokens: metadata / scale columns per ring slot
   const uint32_t wib = (uint32_t)wi_bytes(b32, dense), xib = (uint32_t)xi_bytes(b32), na = b32 ? 2u : 1u;
   const uint32_t sl_b = wib;                               // B4 / B8 follow the (longest) weight record
   const uint32_t sl_sf = sl_b + (uint32_t)n_tile * 128u;
@@ -244,7 +248,12 @@ sdq_linear_kernel(const LinearParams p)
             const uint64_t so = (uint64_t)(s * slot16);
             const uint32_t mb = tmem + 256u + MS * s;
             if (k < ni) {
-              if constexpr (B32) {
+              if constexpr (DENSE) {
+#pragma unroll
+                for (uint32_t j = 0; j < 4; ++j)
+                  ptx::mma_mxf4(tmem + TM_D, d_a + so + ((4096 * j) >> 4), d_b + so + ((256 * j) >> 4), idd[j & 1], mb + 4 + 4 * (j >> 1),
+                                mb + 12 + 8 * (j >> 1), j ? 1u : acc);
+              } else if constexpr (B32) {
                 ptx::mma_sp_nvf4(tmem + TM_D, d_a + so, d_b + so, id4[0], mb, mb + 4, mb + 12, acc);
                 ptx::mma_sp_nvf4(tmem + TM_D, d_a + so + (4096 >> 4), d_b + so + (512 >> 4), id4[0], mb + 2, mb + 8, mb + 20, 1u);
               } else {
@@ -333,7 +342,7 @@ sdq_linear_kernel(const LinearParams p)
       const uint32_t smb = ptx::smem_u32(sm);
       uint32_t s = 0, ph = 0, tcount = 0;
       const uint64_t d_e_in = ptx::smem_desc(smb + SL_A + A_IN_BYTES, 0, 128);
-      const uint64_t d_sfa_in = ptx::smem_desc(smb + SL_A + A_IN_BYTES + E_IN_BYTES, 0, 128);
+      const uint64_t d_sfa_in = ptx::smem_desc(smb + SL_A + (DENSE ? 2 * A_IN_BYTES : A_IN_BYTES + E_IN_BYTES), 0, 128);
       const uint64_t d_e_out = ptx::smem_desc(smb + SL_A + A_OUT_BYTES, 0, 128);
       const uint64_t d_sf0 = ptx::smem_desc(smb + sl_sf, 0, 128), d_sf1 = ptx::smem_desc(smb + sl_sf + SF_ATOM_BYTES, 0, 128);
       const uint64_t d_sf2 = ptx::smem_desc(smb + sl_sf + 2 * SF_ATOM_BYTES, 0, 128);
@@ -346,9 +355,9 @@ sdq_linear_kernel(const LinearParams p)
           const uint64_t so = (uint64_t)(s * slot16);
           const uint32_t mb = tmem + 256u + MS * s;
           if (k < T2) {
-            ptx::tc_cp_128x128b(mb + 0, d_e_in + so);
+            if constexpr (!DENSE) ptx::tc_cp_128x128b(mb + 0, d_e_in + so);
             ptx::tc_cp_32x128b_warpx4(mb + 4, d_sfa_in + so);
-            if constexpr (B32) {
+            if constexpr (S32) {
               // scale words: weights K-block 0 / 1 at +4 / +8; tokens K-block kb, token tile a at +12 + 4 (2 kb + a), staged
               // as [token tile][K-block]
               ptx::tc_cp_32x128b_warpx4(mb + 8, d_sfa_in + so + (SF_ATOM_BYTES >> 4));
@@ -598,12 +607,15 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   if (((uintptr_t)Y & 15) || (ldy % 8) || ((uintptr_t)ws & 15)) return SDQ_ERR_ALIGNMENT;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(sdq_linear_kernel<true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
-        cudaFuncSetAttribute(sdq_linear_kernel<false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
-        cudaFuncSetAttribute(sdq_linear_kernel<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
-        cudaFuncSetAttribute(sdq_linear_kernel<false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
-        cudaFuncSetAttribute(sdq_linear_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess ||
-        cudaFuncSetAttribute(sdq_linear_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, LIN_SMEM_MAX) != cudaSuccess)
+    const cudaFuncAttribute a = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    if (cudaFuncSetAttribute(sdq_linear_kernel<true, true, false, false>, a, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<false, true, false, false>, a, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<true, false, false, false>, a, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<false, false, false, false>, a, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<true, false, true, false>, a, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<false, false, true, false>, a, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<true, false, false, true>, a, LIN_SMEM_MAX) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_kernel<false, false, false, true>, a, LIN_SMEM_MAX) != cudaSuccess)
       return SDQ_ERR_CUDA;
     attr_set = true;
   }
@@ -712,11 +724,12 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   }
   lc.attrs = attr;
   lc.numAttrs = na;
-  const bool flex = p.dense || !(p.n_tile == 256 && p.ksplit == 1 && p.nslot == (p.b32 ? 4 : 5) && p.release == 1);
+  const bool flex = !(p.n_tile == 256 && p.ksplit == 1 && p.nslot == (p.b32 ? 4 : 5) && p.release == 1);
   cudaError_t le;
-  if (flex) le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, true, false>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, true, false>, p);
-  else if (p.b32) le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, false, true>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, false, true>, p);
-  else le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, false, false>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, false, false>, p);
+  if (flex) le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, true, false, false>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, true, false, false>, p);
+  else if (p.dense) le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, false, false, true>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, false, false, true>, p);
+  else if (p.b32) le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, false, true, false>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, false, true, false>, p);
+  else le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, false, false, false>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, false, false, false>, p);
   return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
 }
 
