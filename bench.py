@@ -272,7 +272,12 @@ def run_ours(args):
     decode = measure_decode(sdq, cfg, dev, peaks)
     # ---- the same step with one scale per 32 K (the literal block-32 MXFP4 wording), timed the same way
     cfg32 = sdq.Config(1, sdq.GRAN_PAIR, 32, sdq.SCALE_OCP_FLOOR)
-    b32 = measure_block32_step(sdq, cfg32, dev, rank, X, H, (Yg, Yu, Yd), flops_step, args.steps)
+    b32 = measure_variant_step(sdq, cfg32, dev, rank, X, H, (Yg, Yu, Yd), flops_step, args.steps,
+                               "the same step with one E8M0 scale per 32 K for inlier weights and 4-bit activations")
+    # ---- and without Stage 1: 8:8 split as 1:8 FP8 outliers + dense MXFP4 inliers (dense kind::mxf4, one scale per 32 K)
+    cfgd = sdq.Config(1, sdq.GRAN_DENSE, 32, sdq.SCALE_OCP_FLOOR)
+    dns = measure_variant_step(sdq, cfgd, dev, rank, X, H, (Yg, Yu, Yd), flops_step, args.steps,
+                               "the same step without pruning: 1:8 FP8 outliers + dense MXFP4 inliers, one scale per 32 K")
     # ---- end to end through the public API with host buffers (pinned), copies inside the timed region
     e2e = measure_e2e(sdq, cfg, dev, X, H, (Pg, Pu, Pd), (bx, bh), (Yg, Yu, Yd), flops_step, max(3, args.steps // 2))
     sample = OracleSample(rows_x=1024)
@@ -284,7 +289,7 @@ def run_ours(args):
             "config": {"workload": WORKLOAD, "tokens_per_gpu": M_PREFILL, "l2": "packed weights + activations of one step exceed L2 (150 MB > 126 MB)",
                        "parallelism": "dp%d (independent batches, no collective)" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "quantizer_roofline": quant, "scale_block_32": b32, "decode": decode,
+            "roofline": roofline, "quantizer_roofline": quant, "scale_block_32": b32, "dense_inliers": dns, "decode": decode,
             "cpu_baseline": {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc, "seconds": dt}}
     print(json.dumps(line))
 
@@ -337,9 +342,10 @@ def measure_decode(sdq, cfg, dev, peaks, layers: int = 32, reps: int = 20):
     return out
 
 
-def measure_block32_step(sdq, cfg, dev, rank, X, H, outs, flops_step, steps):
-    """The benchmark step with in_block = 32 (kind::mxf4nvf4 .block16): fresh packed weights of the same shapes, the
-    same inputs and output buffers; whole-step throughput from one event pair around `steps` steps."""
+def measure_variant_step(sdq, cfg, dev, rank, X, H, outs, flops_step, steps, workload):
+    """The benchmark step under another configuration (in_block = 32 on kind::mxf4nvf4 .block16; dense inliers on the
+    dense kind::mxf4): fresh packed weights of the same shapes, the same inputs and output buffers; whole-step
+    throughput from one event pair around `steps` steps."""
     seed = 3000 + rank
     packs = []
     for i, (n, k) in enumerate(((D_FF, D_MODEL), (D_FF, D_MODEL), (D_MODEL, D_FF))):
@@ -366,8 +372,7 @@ def measure_block32_step(sdq, cfg, dev, rank, X, H, outs, flops_step, steps):
     torch.cuda.synchronize()
     ms = a.elapsed_time(b) / steps
     assert sdq.device_status() == 0
-    return {"value": flops_step / (ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms,
-            "workload": "the same step with one E8M0 scale per 32 K for inlier weights and 4-bit activations"}
+    return {"value": flops_step / (ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms, "workload": workload}
 
 
 def measure_e2e(sdq, cfg, dev, X, H, packs, bufs, outs, flops_step, steps):
@@ -498,15 +503,18 @@ def run_sweep(args):
         fl = 2.0 * M * 4096 * 16384
         c4[name] = {"fc1_ms": t1, "fc1_TFLOPs": fl / t1 / 1e9, "fc2_ms": t2, "fc2_TFLOPs": fl / t2 / 1e9}
         del P1, P2, xq, hq
-    # the same layers with one scale per 32 K (the literal block-32 MXFP4 wording), 1:8 outliers
-    cfg = sdq.Config(1, sdq.GRAN_PAIR, 32, 0)
-    P1, P2 = sdq.sdq_decompose(W1, cfg), sdq.sdq_decompose(W2, cfg)
-    xq, hq = sdq.sdq_quantize_act(X, cfg), sdq.sdq_quantize_act(H, cfg)
-    t1 = time_graph(lambda: sdq.sdq_linear(xq, P1, Y1))
-    t2 = time_graph(lambda: sdq.sdq_linear(hq, P2, Y2))
-    fl = 2.0 * M * 4096 * 16384
-    c4["1:8, scale block 32"] = {"fc1_ms": t1, "fc1_TFLOPs": fl / t1 / 1e9, "fc2_ms": t2, "fc2_TFLOPs": fl / t2 / 1e9}
-    del P1, P2, xq, hq
+    # the same layers with one scale per 32 K (the literal block-32 MXFP4 wording), and without pruning (dense MXFP4
+    # inliers, with 1:8 outliers and with none = a plain block-scaled 4-bit GEMM)
+    for name, cfg in (("1:8, scale block 32", sdq.Config(1, sdq.GRAN_PAIR, 32, 0)),
+                      ("1:8, dense inliers", sdq.Config(1, sdq.GRAN_DENSE, 32, 0)),
+                      ("none, dense inliers", sdq.Config(0, sdq.GRAN_DENSE, 32, 0))):
+        P1, P2 = sdq.sdq_decompose(W1, cfg), sdq.sdq_decompose(W2, cfg)
+        xq, hq = sdq.sdq_quantize_act(X, cfg), sdq.sdq_quantize_act(H, cfg)
+        t1 = time_graph(lambda: sdq.sdq_linear(xq, P1, Y1))
+        t2 = time_graph(lambda: sdq.sdq_linear(hq, P2, Y2))
+        fl = 2.0 * M * 4096 * 16384
+        c4[name] = {"fc1_ms": t1, "fc1_TFLOPs": fl / t1 / 1e9, "fc2_ms": t2, "fc2_TFLOPs": fl / t2 / 1e9}
+        del P1, P2, xq, hq
     out["opt67b_ffn_M4096_outlier_sweep"] = c4
     del X, H, W1, W2, Y1, Y2
     # ---- config 5: 32 layers x (q, k, v, o, gate, up, down)

@@ -32,6 +32,10 @@
 #define SDQO_GRAN_PAIR 0 /* inlier pattern: keep 2 of the 4 adjacent pairs in every 8 (pair-wise 4:8) */
 #define SDQO_GRAN_ELEM 1 /* inlier pattern: keep 2 of every 4 elements (element-wise 2:4)            */
 #define SDQO_GRAN_DENSE 2 /* no Stage 1: every non-outlier value stays an inlier (8:8 = out_n:8 + (8-out_n):8) */
+/* Stage 1 keeps the n most significant values of every S-Vector of 8 (n:8 sparsification, n = 2..8), of which out_n
+   become outliers and n - out_n stay inliers at whatever positions they have (the paper's flexible N:M patterns, e.g.
+   7:8 = 1:8 + 6:8); stored like the dense pattern, the dropped positions holding +0.  KEEP(8) is DENSE. */
+#define SDQO_GRAN_KEEP(n) (2 + (8 - (n)))
 #define SDQO_SCALE_OCP_FLOOR 0  /* E = floor(log2 amax) - 2   (OCP MX rule, may saturate in (6,8)) */
 #define SDQO_SCALE_CEIL_NOSAT 1 /* E = smallest integer with amax <= 6 * 2^E                        */
 
@@ -142,10 +146,10 @@ static int is_finite_bf16(uint16_t h) { return (h & 0x7F80) != 0x7F80; }
  *
  * W        [N][K] bf16 bit patterns, row-major (row = output feature, K contiguous)
  * Canonical outputs, one code per byte (layout-free parity surface):
- *   in_code  [N][K/2]      E2M1 codes of the kept inlier slots in ascending k   (DENSE: [N][K], every position)
+ *   in_code  [N][K/2]      E2M1 codes of the kept inlier slots in ascending k   (DENSE / KEEP(n): [N][K], every position)
  *   in_meta  [N][K/8] (PAIR: j0 | j1<<2, kept pair indices 0..3 of the group of 8)
  *            [N][K/4] (ELEM: i0 | i1<<2, kept element indices 0..3 of the group of 4)
- *            not touched for DENSE (there is no pattern to record)
+ *            not touched for DENSE / KEEP(n) (dropped and outlier positions simply hold +0)
  *   in_scale [N][K/in_block] E8M0 code
  *   out_code [N][K/8][out_n] E4M3 codes; out_idx same shape, position 0..7 inside the group, ascending
  *   out_sexp [N]           e of the per-row outlier scale 2^e (int32)
@@ -173,20 +177,24 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
       if (!(col_weight[k] >= 0.0f) || isinf(col_weight[k])) return -3;
   if (cfg->out_n < 0 || cfg->out_n > 2) return -1;
   if (cfg->in_block != 32 && cfg->in_block != 64) return -1;
-  if (cfg->in_gran != SDQO_GRAN_PAIR && cfg->in_gran != SDQO_GRAN_ELEM && cfg->in_gran != SDQO_GRAN_DENSE) return -1;
+  if (cfg->in_gran < 0 || cfg->in_gran > SDQO_GRAN_KEEP(2)) return -1;
+  const int keep_n = 10 - cfg->in_gran;                                /* n of KEEP(n); meaningful from DENSE on */
+  if (cfg->in_gran >= SDQO_GRAN_DENSE && keep_n <= cfg->out_n) return -1;
   const int on = cfg->out_n, Bs = cfg->in_block;
   const int64_t G8 = K / 8;
-  const int64_t slots = cfg->in_gran == SDQO_GRAN_DENSE ? K : K / 2;   /* inlier slots per row */
+  const int64_t slots = cfg->in_gran >= SDQO_GRAN_DENSE ? K : K / 2;   /* inlier slots per row */
   for (int64_t i = 0; i < N * K; ++i)
     if (!is_finite_bf16(W[i])) return -2;
 
   uint8_t* is_out = (uint8_t*)malloc((size_t)K);   /* 1 where the element went to W_o            */
   uint8_t* kept = (uint8_t*)malloc((size_t)K);     /* 1 where the element is a kept inlier SLOT  */
+  uint8_t* dropped = (uint8_t*)malloc((size_t)K);  /* KEEP(n): 1 where Stage 1 removed the value (its slot holds +0) */
   float* sig = (float*)malloc((size_t)K * sizeof(float));
   for (int64_t n = 0; n < N; ++n) {
     const uint16_t* w = W + n * K;
     memset(is_out, 0, (size_t)K);
     memset(kept, 0, (size_t)K);
+    memset(dropped, 0, (size_t)K);
     for (int64_t k = 0; k < K; ++k) sig[k] = significance(w[k], col_weight, k);
 
     /* Stage 2, local outlier extraction: the out_n most significant values of every S-Vector of 8
@@ -221,8 +229,23 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
 
     /* Stage 1 on the remaining values: N:M pruning by significance.  The dense configuration
        (Section 5, decomposition-stage study: 8:8 split as 1:8 outliers + 7:8 inliers) skips it. */
-    if (cfg->in_gran == SDQO_GRAN_DENSE) {
+    if (cfg->in_gran >= SDQO_GRAN_DENSE) {
+      /* n:8 sparsification then out_n:8 outlier extraction with one metric: the outliers are the out_n most
+         significant of the 8, the inliers the next n - out_n (largest first, ties to the lower index), the rest is
+         dropped -- in whichever order the two stages run.  Every position is a slot. */
       memset(kept, 1, (size_t)K);
+      for (int64_t g = 0; g < G8; ++g) {
+        uint8_t chosen[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        for (int t = 0; t < keep_n - on; ++t) {
+          int best = -1;
+          for (int i = 0; i < 8; ++i) {
+            if (is_out[8 * g + i] || chosen[i]) continue;
+            if (best < 0 || sig[8 * g + i] > sig[8 * g + best]) best = i;
+          }
+          chosen[best] = 1;
+        }
+        for (int i = 0; i < 8; ++i) dropped[8 * g + i] = (uint8_t)(!is_out[8 * g + i] && !chosen[i]);
+      }
     } else if (cfg->in_gran == SDQO_GRAN_PAIR) {
       for (int64_t g = 0; g < G8; ++g) {
         float score[4];
@@ -262,7 +285,7 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
     for (int64_t b = 0; b < K / Bs; ++b) {
       double amax = 0.0;
       for (int64_t k = b * Bs; k < (b + 1) * Bs; ++k)
-        if (kept[k] && !is_out[k]) {
+        if (kept[k] && !is_out[k] && !dropped[k]) {
           double a = fabs(sdqo_bf16_to_double(w[k]));
           if (a > amax) amax = a;
         }
@@ -272,7 +295,7 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
     for (int64_t k = 0; k < K; ++k) {
       if (!kept[k]) continue;
       uint8_t code = 0;
-      if (!is_out[k]) {
+      if (!is_out[k] && !dropped[k]) {
         int c = in_scale[n * (K / Bs) + k / Bs];
         code = sdqo_e2m1_encode(ldexp(sdqo_bf16_to_double(w[k]), 127 - c));
       }
@@ -281,6 +304,7 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
   }
   free(is_out);
   free(kept);
+  free(dropped);
   free(sig);
   return 0;
 }
@@ -303,7 +327,7 @@ int sdqo_dequant_weights(int64_t N, int64_t K, const sdqo_config* cfg,
   memset(W_out, 0, sizeof(double) * (size_t)(N * K));
   for (int64_t n = 0; n < N; ++n) {
     int64_t slot = 0;
-    if (cfg->in_gran == SDQO_GRAN_DENSE) {
+    if (cfg->in_gran >= SDQO_GRAN_DENSE) {
       for (int64_t k = 0; k < K; ++k)
         W_in[n * K + k] = sdqo_e2m1_decode(in_code[n * K + k]) * sdqo_e8m0_decode(in_scale[n * (K / Bs) + k / Bs]);
     } else if (cfg->in_gran == SDQO_GRAN_PAIR) {
@@ -410,7 +434,7 @@ int sdqo_linear(int64_t M, int64_t N, int64_t K, const sdqo_config* cfg,
     for (int64_t n = n_begin; n < n_end; ++n) {
       /* positions and values of the non-zeros of row n of W_i and W_o */
       int64_t ni = 0, no = 0, slot = 0;
-      if (cfg->in_gran == SDQO_GRAN_DENSE) {
+      if (cfg->in_gran >= SDQO_GRAN_DENSE) {
         for (int64_t k = 0; k < K; ++k) {
           ki[ni] = (int32_t)k;
           wi[ni++] = sdqo_e2m1_decode(in_code[n * K + k]) * sdqo_e8m0_decode(in_scale[n * (K / Bs) + k / Bs]);

@@ -19,6 +19,13 @@ _SRC = os.path.join(_HERE, "sdq_oracle.c")
 _LIB = os.path.join(_HERE, "libsdq_oracle.so")
 
 GRAN_PAIR, GRAN_ELEM, GRAN_DENSE = 0, 1, 2
+
+
+def gran_keep(n: int) -> int:
+    """in_gran value of the pattern that keeps the n most significant of every 8 (out_n outliers + n - out_n inliers at
+    any positions, stored like the dense pattern); gran_keep(8) == GRAN_DENSE."""
+    assert 2 <= n <= 8
+    return 2 + (8 - n)
 SCALE_OCP_FLOOR, SCALE_CEIL_NOSAT = 0, 1
 
 
@@ -90,8 +97,8 @@ class Packed:
     N: int
     K: int
     cfg: Config
-    in_code: np.ndarray    # [N, K/2] u8 E2M1 codes of kept slots, ascending k ([N, K] for GRAN_DENSE)
-    in_meta: np.ndarray    # [N, K/8] (pair) or [N, K/4] (elem) u8 nibble values ([N, 0] for GRAN_DENSE)
+    in_code: np.ndarray    # [N, K/2] u8 E2M1 codes of kept slots, ascending k ([N, K] from GRAN_DENSE on)
+    in_meta: np.ndarray    # [N, K/8] (pair) or [N, K/4] (elem) u8 nibble values ([N, 0] from GRAN_DENSE on)
     in_scale: np.ndarray   # [N, K/in_block] u8 E8M0 codes
     out_code: np.ndarray   # [N, K/8, out_n] u8 E4M3 codes
     out_idx: np.ndarray    # [N, K/8, out_n] u8 positions 0..7
@@ -115,8 +122,8 @@ def decompose(W_bits: np.ndarray, cfg: Config, col_weight=None) -> Packed:
     significance of an element is then the weight-activation product |w| * c[k] instead of the magnitude."""
     W_bits = np.ascontiguousarray(W_bits, dtype=np.uint16)
     N, K = W_bits.shape
-    nmeta = {GRAN_PAIR: K // 8, GRAN_DENSE: 0}.get(cfg.in_gran, K // 4)
-    nslot = K if cfg.in_gran == GRAN_DENSE else K // 2
+    nmeta = 0 if cfg.in_gran >= GRAN_DENSE else (K // 8 if cfg.in_gran == GRAN_PAIR else K // 4)
+    nslot = K if cfg.in_gran >= GRAN_DENSE else K // 2
     on = max(cfg.out_n, 0)
     p = Packed(N, K, cfg,
                np.zeros((N, nslot), np.uint8), np.zeros((N, nmeta), np.uint8),
@@ -200,8 +207,8 @@ def linear(q: QAct, p: Packed, n_begin: int = 0, n_end: int | None = None, threa
 def bits_per_weight(cfg: Config, K: int | None = None) -> float:
     """Average bits per weight element of the packed SDQ format (data + index + scale metadata)."""
     L = lib()
-    if cfg.in_gran == GRAN_DENSE:
-        # every position stored as a 4-bit value (the outlier positions hold +0): no index metadata
+    if cfg.in_gran >= GRAN_DENSE:
+        # every position stored as a 4-bit value (outlier and dropped positions hold +0): no index metadata
         inl = L.sdqo_bits_per_weight_part(8, 8, 4, 8, cfg.in_block)
     elif cfg.in_gran == GRAN_PAIR:
         # 2 of 4 pairs: per 8 elements 4 stored 4-bit values + two 2-bit pair indices

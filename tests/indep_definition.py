@@ -61,7 +61,8 @@ def top_mask(keys, n):
 def decompose_dense(W_bits, out_n, pair, block, rule_floor, col_weight=None):
     """returns (W_in_hat, W_out_hat, mask_in_slots, mask_out) as dense [N, K] arrays; with col_weight the
     selections rank by the fp32 product |w| * c[k] instead of |w| (the values that get quantized do not change);
-    pair: True = pair-wise 4:8, False = element-wise 2:4, None = no pruning"""
+    pair: True = pair-wise 4:8, False = element-wise 2:4, None = no pruning,
+    an integer n = the n most significant of every 8 survive (outliers included)"""
     W = bf16_to_f64(W_bits)
     N, K = W.shape
     A = np.abs(W)
@@ -71,6 +72,9 @@ def decompose_dense(W_bits, out_n, pair, block, rule_floor, col_weight=None):
     R = np.where(mask_out, 0.0, A)
     if pair is None:                      # no pruning: every non-outlier value stays an inlier
         slots = np.ones((N, K), bool)
+    elif pair is not True and pair is not False:   # an integer n: keep the n most significant of every 8 in total
+        keys = np.where(mask_out, -1.0, A).reshape(N, K // 8, 8)
+        slots = top_mask(keys, int(pair) - out_n).reshape(N, K)
     elif pair:
         r32 = R.astype(np.float32).reshape(N, K // 8, 4, 2)
         score = (r32[..., 0] + r32[..., 1]).astype(np.float32)

@@ -353,5 +353,62 @@ def test_dense_inliers_without_outliers_is_plain_block_scaled_4bit_quantization(
 
 
 def test_unknown_inlier_pattern_rejected():
-    with pytest.raises(ValueError):
-        so.decompose(tiny_W(8, 128, 0), so.Config(1, 3, 64, so.SCALE_OCP_FLOOR))
+    for out_n, gran in ((1, 9), (1, -1), (2, so.gran_keep(2))):      # the last: nothing would be left for the inliers
+        with pytest.raises(ValueError):
+            so.decompose(tiny_W(8, 128, 0), so.Config(out_n, gran, 64, so.SCALE_OCP_FLOOR))
+
+
+# ---------------------------------------------------------------- n:8 sparsification + out_n:8 outliers + (n - out_n):8 inliers
+KEEP_CFGS = [(7, 1, 32, so.SCALE_OCP_FLOOR), (6, 2, 32, so.SCALE_CEIL_NOSAT), (6, 1, 64, so.SCALE_OCP_FLOOR),
+             (4, 0, 32, so.SCALE_OCP_FLOOR), (3, 2, 32, so.SCALE_OCP_FLOOR)]
+
+
+@pytest.mark.parametrize("n,out_n,block,rule", KEEP_CFGS)
+def test_keep_n_of_8_matches_independent_dense_definition(n, out_n, block, rule):
+    cfg = so.Config(out_n, so.gran_keep(n), block, rule)
+    for seed, cw in ((2, None), (3, lognormal_channel_weight(512, 9))):
+        Wb = tiny_W(40, 512, seed)
+        p = so.decompose(Wb, cfg, cw)
+        W_in, W_out = so.dequant_weights(p)
+        ref_in, ref_out, slots, mask_out = decompose_dense(Wb, out_n, n, block, rule == so.SCALE_OCP_FLOOR, cw)
+        assert np.array_equal(W_out, ref_out) and np.array_equal(W_in, ref_in)
+        assert ((slots & ~mask_out).reshape(40, 64, 8).sum(-1) == n - out_n).all()
+        assert (((W_in != 0) | (W_out != 0)).reshape(40, 64, 8).sum(-1) <= n).all()
+        assert (p.in_code[~(slots & ~mask_out)] == 0).all()
+
+
+@pytest.mark.parametrize("n,out_n", [(7, 1), (6, 2), (5, 1)])
+def test_keep_n_of_8_is_the_papers_stage_order(n, out_n):
+    """sparsify to n:8 first, then take the out_n largest of the survivors (the paper's order), written out with numpy on
+    magnitudes that are distinct inside every S-Vector: same outliers, same inliers, same dropped values"""
+    rng = np.random.default_rng(21)
+    N, K = 24, 256
+    import torch
+    mags = np.stack([rng.permutation(8) for _ in range(N * K // 8)]).reshape(N, K) + 1.0     # 1..8, distinct per group
+    W = mags * rng.choice([-1.0, 1.0], size=(N, K)) * 0.03125
+    Wb = sdq_synth.bf16_bits(torch.from_numpy(W).to(torch.bfloat16))
+    assert np.array_equal(bf16_to_f64(Wb), W)
+    p = so.decompose(Wb, so.Config(out_n, so.gran_keep(n), 32, so.SCALE_CEIL_NOSAT))
+    W_in, W_out = so.dequant_weights(p)
+    g = mags.reshape(N, K // 8, 8)
+    survive = g > (8 - n)                       # Stage 1: the 8 - n smallest of every 8 go
+    outl = g > (8 - out_n)                      # Stage 2: the out_n largest survivors
+    inl = survive & ~outl
+    assert np.array_equal((W_out != 0).reshape(g.shape), outl)
+    # every surviving inlier is representable here (|w| * 32 in 1..8 with one scale per 32: at most one step of rounding,
+    # never to zero), so the support of W_in is exactly the inlier set
+    assert np.array_equal((W_in != 0).reshape(g.shape), inl)
+    assert np.array_equal(W_out, np.where(outl.reshape(N, K), W, 0.0))
+
+
+def test_keep_8_of_8_is_the_dense_pattern_and_keep_less_only_removes_values():
+    Wb = tiny_W(16, 256, 23)
+    d = so.decompose(Wb, so.Config(1, so.GRAN_DENSE, 32, so.SCALE_OCP_FLOOR))
+    assert so.gran_keep(8) == so.GRAN_DENSE
+    prev = so.dequant_weights(d)[0] != 0
+    for n in (7, 6, 5, 4, 3, 2):
+        p = so.decompose(Wb, so.Config(1, so.gran_keep(n), 32, so.SCALE_OCP_FLOOR))
+        assert np.array_equal(p.out_idx, d.out_idx) and np.array_equal(p.out_code, d.out_code)
+        nz = so.dequant_weights(p)[0] != 0
+        assert not (nz & ~prev).any()            # supports are nested as n shrinks
+        prev = nz

@@ -19,7 +19,8 @@ def make(M, N, K, seed, cfg=CFG):
 
 
 @pytest.mark.parametrize("cfg", [CFG, so.Config(2, so.GRAN_ELEM, 32, so.SCALE_CEIL_NOSAT), so.Config(0, so.GRAN_PAIR, 64, 0),
-                                 so.Config(1, so.GRAN_DENSE, 32, so.SCALE_OCP_FLOOR)])
+                                 so.Config(1, so.GRAN_DENSE, 32, so.SCALE_OCP_FLOOR),
+                                 so.Config(1, so.gran_keep(7), 32, so.SCALE_OCP_FLOOR)])
 def test_brute_force_triple_loop(cfg):
     Wb, Xb, p, q = make(3, 16, 128, 2, cfg)
     W_in, W_out = so.dequant_weights(p)
