@@ -39,6 +39,7 @@ typedef enum {
 } sdq_status_t;
 
 enum { SDQ_GRAN_PAIR = 0, SDQ_GRAN_ELEM = 1, SDQ_GRAN_DENSE = 2 }; /* inlier pattern            */
+#define SDQ_GRAN_KEEP(n) (2 + (8 - (n)))  /* n:8 sparsification, n = 2..8; SDQ_GRAN_KEEP(8) == SDQ_GRAN_DENSE */
 enum { SDQ_SCALE_OCP_FLOOR = 0, SDQ_SCALE_CEIL_NOSAT = 1 }; /* E8M0 Q-Vector scale rule        */
 
 /* "pattern, formats" of the decomposition (Section 5, Stages 1-3).
@@ -50,9 +51,13 @@ enum { SDQ_SCALE_OCP_FLOOR = 0, SDQ_SCALE_CEIL_NOSAT = 1 }; /* E8M0 Q-Vector sca
  *              of every 4 (decompose / export only: the buffer then holds the canonical arrays and
  *              sdq_linear returns SDQ_ERR_UNSUPPORTED).  SDQ_GRAN_DENSE skips Stage 1: every value that
  *              is not an outlier stays an inlier (the evaluation's configuration 8:8 = 1:8 outliers +
- *              7:8 inliers); sdq_linear runs W_i as a dense 4-bit operand.  The dense 4-bit tensor-core
- *              kind has one scale per 32 K only, so SDQ_GRAN_DENSE requires in_block = 32 (with 64 every
- *              call returns SDQ_ERR_UNSUPPORTED).
+ *              7:8 inliers); sdq_linear runs W_i as a dense 4-bit operand.  SDQ_GRAN_KEEP(n), n > out_n:
+ *              Stage 1 keeps the n most significant values of every S-Vector of 8, of which the out_n most
+ *              significant are the outliers and the other n - out_n the inliers, at whatever positions
+ *              they have (the evaluation's flexible N:M configurations, e.g. 7:8 = 1:8 + 6:8; largest
+ *              first, ties to the lower k); stored and executed like the dense pattern, the dropped
+ *              positions holding +0.  The dense 4-bit tensor-core kind has one scale per 32 K only, so
+ *              these patterns require in_block = 32 (with 64 every call returns SDQ_ERR_UNSUPPORTED).
  *   in_block   Q-Vector length: logical K sharing one E8M0 scale, for W_i and for the 4-bit
  *              activations: 64 or 32.  Both are executed by sdq_linear (64: kind::mxf4 .block32, the
  *              faster kernel; 32: kind::mxf4nvf4 .block16 with E8M0 scale codes).
@@ -93,9 +98,9 @@ typedef struct {
  * (all pointers: device memory, caller-owned, sizes in elements given beside each field). */
 typedef struct {
   uint8_t* in_code;   /* [N][K/2]   E2M1 codes of the kept inlier slots in ascending k
-                         (DENSE: [N][K], every position; outlier positions hold +0)                */
+                         (DENSE / KEEP: [N][K], every position; outlier and dropped ones hold +0)                */
   uint8_t* in_meta;   /* [N][K/8] (PAIR) or [N][K/4] (ELEM): i0 | i1<<2, kept indices, ascending
-                         (DENSE: not written, may be NULL)                                         */
+                         (DENSE / KEEP: not written, may be NULL)                                         */
   uint8_t* in_scale;  /* [N][K/in_block] E8M0 codes                                               */
   uint8_t* out_code;  /* [N][K/8][out_n] E4M3 codes                                               */
   uint8_t* out_idx;   /* [N][K/8][out_n] position 0..7 in the S-Vector, ascending                 */

@@ -16,6 +16,13 @@ import torch
 from .build import LIB, build
 
 GRAN_PAIR, GRAN_ELEM, GRAN_DENSE = 0, 1, 2
+
+
+def gran_keep(n: int) -> int:
+    """SDQ_GRAN_KEEP(n): Stage 1 keeps the n most significant of every 8 (out_n outliers + n - out_n inliers at any
+    positions); stored and executed like the dense pattern.  gran_keep(8) == GRAN_DENSE."""
+    assert 2 <= n <= 8
+    return 2 + (8 - n)
 SCALE_OCP_FLOOR, SCALE_CEIL_NOSAT = 0, 1
 
 STATUS = ["ok", "invalid_arg", "shape", "alignment", "unsupported", "buffer_too_small", "nonfinite", "cuda", "timeout"]
@@ -237,7 +244,7 @@ def sdq_linear_noalloc(xq: QuantAct, p: PackedWeight, out: torch.Tensor) -> torc
 def packed_export(p: PackedWeight) -> dict:
     N, K, on = p.N, p.K, p.cfg.out_n
     dev = p.buf.device
-    dense = p.cfg.in_gran == GRAN_DENSE
+    dense = p.cfg.in_gran >= GRAN_DENSE
     nmeta = 0 if dense else (K // 8 if p.cfg.in_gran == GRAN_PAIR else K // 4)
     t = dict(in_code=torch.zeros((N, K if dense else K // 2), dtype=torch.uint8, device=dev),
              in_meta=torch.zeros((N, nmeta), dtype=torch.uint8, device=dev),

@@ -603,7 +603,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   if (!Xq || !P || !Y || !Xq->dev || !P->dev) return SDQ_ERR_INVALID_ARG;
   if (Xq->K != P->K || Xq->M <= 0 || P->N <= 0 || P->N % TILE_ROWS || P->K % K2 || ldy < P->N) return SDQ_ERR_SHAPE;
   if (Xq->cfg.in_block != P->cfg.in_block || Xq->cfg.scale_rule != P->cfg.scale_rule) return SDQ_ERR_SHAPE;
-  if (P->cfg.in_gran != SDQ_GRAN_PAIR && !(P->cfg.in_gran == SDQ_GRAN_DENSE && P->cfg.in_block == 32)) return SDQ_ERR_UNSUPPORTED;
+  if (P->cfg.in_gran != SDQ_GRAN_PAIR && !(P->cfg.in_gran >= SDQ_GRAN_DENSE && P->cfg.in_block == 32)) return SDQ_ERR_UNSUPPORTED;
   if (((uintptr_t)Y & 15) || (ldy % 8) || ((uintptr_t)ws & 15)) return SDQ_ERR_ALIGNMENT;
   static bool attr_set = false;
   if (!attr_set) {
@@ -625,7 +625,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   p.w = (const uint8_t*)P->dev;
   p.x = (const uint8_t*)Xq->dev;
   p.b32 = P->cfg.in_block == 32 ? 1 : 0;
-  p.dense = P->cfg.in_gran == SDQ_GRAN_DENSE ? 1 : 0;
+  p.dense = P->cfg.in_gran >= SDQ_GRAN_DENSE ? 1 : 0;   // the n:8 patterns are stored and run like the dense one
   p.poff = packed_offsets(P->N, P->K, P->cfg.out_n, p.b32 != 0, p.dense != 0);
   p.aoff = act_offsets(Xq->M, Xq->K, p.b32 != 0);
   p.M = Xq->M; p.N = P->N; p.K = P->K;

@@ -96,7 +96,8 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
   const int64_t rt = n / TILE_ROWS;
   const uint32_t r = (uint32_t)(n % TILE_ROWS);
   const int T1 = (int)(K / K1), T2 = (int)(K / K2);
-  const bool b32 = cfg.in_block == 32, dense = cfg.in_gran == SDQ_GRAN_DENSE;
+  const bool b32 = cfg.in_block == 32, dense = cfg.in_gran >= SDQ_GRAN_DENSE;
+  const int keep_in = 10 - cfg.in_gran - out_n;     // dense family: inliers kept per S-Vector (8 - out_n without Stage 1)
   const int wib = wi_bytes(b32, dense);
   uint8_t* wi_base = blob + off.wi + (size_t)rt * T2 * wib;
   uint8_t* wo_base = blob + off.wo + (size_t)rt * T1 * WO_BYTES;
@@ -122,20 +123,28 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     uint8_t* wo = wo_base + (size_t)k1 * WO_BYTES;
 
     if (dense) {
-      // no Stage 1: all eight positions are inlier slots (an outlier position holds +0).  Stage 3 with one scale per
-      // 32 K = 4 S-Vectors = 4 lanes
+      // all eight positions are inlier slots; an outlier position holds +0, and so does a value that Stage 1 drops: a
+      // non-outlier survives if fewer than keep_in non-outliers rank before it (more significant, or equal with a
+      // lower index).  Stage 3 with one scale per 32 K = 4 S-Vectors = 4 lanes
+      uint32_t gone = 0;        // bit i: position i holds +0
       uint32_t ikey = 0;
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
-        if (i != o0 && i != o1) ikey = max(ikey, key[i]);
+      for (int i = 0; i < 8; ++i) {
+        int before = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          before += (j != o0 && j != o1 && (skey[j] > skey[i] || (skey[j] == skey[i] && j < i))) ? 1 : 0;
+        if (i == o0 || i == o1 || before >= keep_in) gone |= 1u << i;
+        else ikey = max(ikey, key[i]);
+      }
       ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 1));
       ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 2));
       const uint32_t c = e8m0_scale_code(bf16_bits_to_float(ikey), cfg.scale_rule);
       uint32_t codes = 0;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const float v0 = (2 * i == o0 || 2 * i == o1) ? 0.0f : bf16_bits_to_float(bits[2 * i]) * pow2_inv_e8m0(c);
-        const float v1 = (2 * i + 1 == o0 || 2 * i + 1 == o1) ? 0.0f : bf16_bits_to_float(bits[2 * i + 1]) * pow2_inv_e8m0(c);
+        const float v0 = ((gone >> (2 * i)) & 1) ? 0.0f : bf16_bits_to_float(bits[2 * i]) * pow2_inv_e8m0(c);
+        const float v1 = ((gone >> (2 * i + 1)) & 1) ? 0.0f : bf16_bits_to_float(bits[2 * i + 1]) * pow2_inv_e8m0(c);
         codes |= e2m1x2(v0, v1) << (8 * i);
       }
       // 32 S-Vectors per 256-K stage, 4 code bytes each: bytes 32 j .. 32 j + 31 = K-block j (64 K)
@@ -234,7 +243,7 @@ export_packed_kernel(const uint8_t* __restrict__ blob, int64_t N, int64_t K, sdq
   const int64_t rt = n / TILE_ROWS;
   const uint32_t r = (uint32_t)(n % TILE_ROWS);
   const int T2 = (int)(K / K2);
-  const bool b32 = cfg.in_block == 32, dense = cfg.in_gran == SDQ_GRAN_DENSE;
+  const bool b32 = cfg.in_block == 32, dense = cfg.in_gran >= SDQ_GRAN_DENSE;
   const int wib = wi_bytes(b32, dense);
   const uint8_t* wi_base = blob + off.wi + (size_t)rt * T2 * wib;
   for (int g = threadIdx.x; g < G; g += 128) {
@@ -271,22 +280,23 @@ export_packed_kernel(const uint8_t* __restrict__ blob, int64_t N, int64_t K, sdq
 using namespace sdq;
 
 static bool cfg_ok(const sdq_config_t* c) {
-  return c && c->out_n >= 0 && c->out_n <= 2 && (c->in_gran == SDQ_GRAN_PAIR || c->in_gran == SDQ_GRAN_ELEM || c->in_gran == SDQ_GRAN_DENSE) &&
+  return c && c->out_n >= 0 && c->out_n <= 2 && c->in_gran >= 0 && c->in_gran <= SDQ_GRAN_KEEP(2) &&
+         (c->in_gran < SDQ_GRAN_DENSE || 10 - c->in_gran > c->out_n) &&
          (c->in_block == 32 || c->in_block == 64) && (c->scale_rule == SDQ_SCALE_OCP_FLOOR || c->scale_rule == SDQ_SCALE_CEIL_NOSAT);
 }
 
 extern "C" sdq_status_t sdq_packed_size(int64_t N, int64_t K, const sdq_config_t* cfg, size_t* bytes, size_t* algorithmic_bytes)
 {
   if (!cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
-  if (cfg->in_gran == SDQ_GRAN_DENSE && cfg->in_block != 32) return SDQ_ERR_UNSUPPORTED;
+  if (cfg->in_gran >= SDQ_GRAN_DENSE && cfg->in_block != 32) return SDQ_ERR_UNSUPPORTED;
   if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2) return SDQ_ERR_SHAPE;
-  if (bytes) *bytes = is_tensor_core_reading(*cfg) ? packed_offsets(N, K, cfg->out_n, cfg->in_block == 32, cfg->in_gran == SDQ_GRAN_DENSE).total : plain_packed_offsets(N, K, *cfg).total;
+  if (bytes) *bytes = is_tensor_core_reading(*cfg) ? packed_offsets(N, K, cfg->out_n, cfg->in_block == 32, cfg->in_gran >= SDQ_GRAN_DENSE).total : plain_packed_offsets(N, K, *cfg).total;
   if (algorithmic_bytes) {
     // per weight: 4-bit values on half the positions (2) + index metadata (pair-wise: two 2-bit pair indices per 8 =
     // 0.5; element-wise: two 2-bit indices per 4 = 1) + one 8-bit scale per Q-Vector + out_n * (8 value + 3 index
     // bits) per 8; plus one 32-bit row scale
-    // (no pruning: a 4-bit value on every position and no index metadata)
-    const double inl = cfg->in_gran == SDQ_GRAN_DENSE ? 4.0 : 2.0 + (cfg->in_gran == SDQ_GRAN_PAIR ? 0.5 : 1.0);
+    // (dense storage: a 4-bit value on every position and no index metadata)
+    const double inl = cfg->in_gran >= SDQ_GRAN_DENSE ? 4.0 : 2.0 + (cfg->in_gran == SDQ_GRAN_PAIR ? 0.5 : 1.0);
     const double bits = inl + 8.0 / cfg->in_block + cfg->out_n * 11.0 / 8.0;
     *algorithmic_bytes = (size_t)((double)N * (double)K * bits / 8.0) + (cfg->out_n ? (size_t)N * 4 : 0);
   }
@@ -302,12 +312,12 @@ extern "C" sdq_status_t sdq_decompose_metric(const void* W, int64_t N, int64_t K
                                              void* stream)
 {
   if (!W || !packed_buf || !out || !cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
-  if (cfg->in_gran == SDQ_GRAN_DENSE && cfg->in_block != 32) return SDQ_ERR_UNSUPPORTED;
+  if (cfg->in_gran >= SDQ_GRAN_DENSE && cfg->in_block != 32) return SDQ_ERR_UNSUPPORTED;
   if ((uintptr_t)col_weight & 15) return SDQ_ERR_ALIGNMENT;
   if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2 || ldw < K) return SDQ_ERR_SHAPE;
   if (((uintptr_t)W & 15) || ((uintptr_t)packed_buf & 15) || (ldw % 8)) return SDQ_ERR_ALIGNMENT;
   const bool tc = is_tensor_core_reading(*cfg);
-  const PackedOffsets off = packed_offsets(N, K, cfg->out_n, cfg->in_block == 32, cfg->in_gran == SDQ_GRAN_DENSE);
+  const PackedOffsets off = packed_offsets(N, K, cfg->out_n, cfg->in_block == 32, cfg->in_gran >= SDQ_GRAN_DENSE);
   const PlainPackedOffsets poff = plain_packed_offsets(N, K, *cfg);
   if (packed_bytes < (tc ? off.total : poff.total)) return SDQ_ERR_BUFFER_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
@@ -339,7 +349,7 @@ extern "C" sdq_status_t sdq_decompose_metric(const void* W, int64_t N, int64_t K
 extern "C" sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canonical_t* out, void* stream)
 {
   if (!P || !out || !P->dev || !out->in_code || !out->in_scale || !out->out_sexp) return SDQ_ERR_INVALID_ARG;
-  if (!out->in_meta && P->cfg.in_gran != SDQ_GRAN_DENSE) return SDQ_ERR_INVALID_ARG;
+  if (!out->in_meta && P->cfg.in_gran < SDQ_GRAN_DENSE) return SDQ_ERR_INVALID_ARG;
   if (P->cfg.out_n > 0 && (!out->out_code || !out->out_idx)) return SDQ_ERR_INVALID_ARG;
   if (!is_tensor_core_reading(P->cfg)) {
     // the buffer already holds the canonical arrays
@@ -357,7 +367,7 @@ extern "C" sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canon
     ok = ok && cudaMemcpyAsync(out->out_sexp, b + o.osexp, n * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
     return ok ? SDQ_OK : SDQ_ERR_CUDA;
   }
-  const PackedOffsets off = packed_offsets(P->N, P->K, P->cfg.out_n, P->cfg.in_block == 32, P->cfg.in_gran == SDQ_GRAN_DENSE);
+  const PackedOffsets off = packed_offsets(P->N, P->K, P->cfg.out_n, P->cfg.in_block == 32, P->cfg.in_gran >= SDQ_GRAN_DENSE);
   export_packed_kernel<<<(unsigned)P->N, 128, 0, (cudaStream_t)stream>>>((const uint8_t*)P->dev, P->N, P->K, P->cfg, off, *out);
   return cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
 }

@@ -11,7 +11,7 @@ namespace sdq {
 // pair-wise 4:8 inliers with one scale per 64 K (kind::mxf4 .block32) or per 32 K (kind::mxf4nvf4 .block16), or dense
 // inliers with one scale per 32 K (dense kind::mxf4 .block32): tiled layout
 inline bool is_tensor_core_reading(const sdq_config_t& c) {
-  return (c.in_gran == SDQ_GRAN_PAIR && (c.in_block == 64 || c.in_block == 32)) || (c.in_gran == SDQ_GRAN_DENSE && c.in_block == 32);
+  return (c.in_gran == SDQ_GRAN_PAIR && (c.in_block == 64 || c.in_block == 32)) || (c.in_gran >= SDQ_GRAN_DENSE && c.in_block == 32);
 }
 
 struct PlainPackedOffsets {

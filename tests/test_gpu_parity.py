@@ -145,6 +145,16 @@ def test_dense_inliers_through_the_tensor_core(M, N, K, out_n, rule):
     run_case(M, N, K, 1200 + M, out_n=out_n, rule=rule, block=32, gran=so.GRAN_DENSE)
 
 
+@pytest.mark.parametrize("n,M,N,K,out_n,rule", [(7, 8, 256, 256, 1, 0), (7, 1, 512, 2048, 1, 0), (6, 16, 256, 4096, 2, 1), (4, 33, 128, 768, 0, 0),
+                                                (7, 100, 256, 2816, 1, 0), (6, 129, 256, 512, 1, 1), (3, 300, 512, 1024, 2, 0),
+                                                (7, 520, 6400, 256, 1, 0), (5, 64, 1024, 1024, 1, 0)])
+def test_n_of_8_sparsification_with_outliers_and_inliers_at_any_position(n, M, N, K, out_n, rule):
+    """SDQ_GRAN_KEEP(n): the n most significant of every 8 survive, out_n of them as FP8 outliers, the others as MXFP4
+    inliers wherever they sit (7:8 = 1:8 + 6:8 is the evaluation's headline pattern): packed arrays bit-exact, product
+    through the dense 4-bit MMA"""
+    run_case(M, N, K, 1500 + 10 * n + M, out_n=out_n, rule=rule, block=32, gran=so.gran_keep(n))
+
+
 def test_dense_inliers_one_hot_readback_and_workspace_split():
     m = sdq()
     cfg = m.Config(1, m.GRAN_DENSE, 32, 0)
@@ -173,6 +183,10 @@ def test_dense_inliers_one_hot_readback_and_workspace_split():
     with pytest.raises(m.SdqError) as e:
         m.sdq_decompose(W.cuda(), m.Config(1, m.GRAN_DENSE, 64, 0))
     assert e.value.code == 4
+    for out_n, gran in ((2, m.gran_keep(2)), (1, 9)):             # nothing left for the inliers; unknown pattern
+        with pytest.raises(m.SdqError) as e:
+            m.sdq_decompose(W.cuda(), m.Config(out_n, gran, 32, 0))
+        assert e.value.code == 1
 
 
 def test_one_hot_readback_512_tokens():
@@ -299,7 +313,7 @@ def test_activation_quantizer_row_lengths(M, K, rule, block):
         assert np.array_equal(ae[name], getattr(oq, name)), name
 
 
-@pytest.mark.parametrize("gran,block", [(1, 64), (0, 32), (0, 64), (2, 32)])
+@pytest.mark.parametrize("gran,block", [(1, 64), (0, 32), (0, 64), (2, 32), (3, 32)])
 @pytest.mark.parametrize("out_n", [0, 1, 2])
 def test_product_metric_packer(gran, block, out_n):
     """sdq_decompose_metric: selections by |w| * c[k]; packed arrays bit-exact against the oracle for the tensor-core
@@ -321,8 +335,13 @@ def test_product_metric_packer(gran, block, out_n):
         assert np.array_equal(pe[name], getattr(op, name)), name
     # it does change the selection (otherwise the test would prove nothing)
     om = so.decompose(sdq_synth.bf16_bits(W), oc)
-    if gran == m.GRAN_DENSE:
-        assert out_n == 0 or not np.array_equal(op.out_idx, om.out_idx)
+    if gran >= m.GRAN_DENSE:
+        # no pattern metadata: the metric shows in the outlier positions, or (7:8 with no outliers) in what is dropped;
+        # 8:8 with no outliers has no selection at all
+        if out_n:
+            assert not np.array_equal(op.out_idx, om.out_idx)
+        elif gran > m.GRAN_DENSE:
+            assert not np.array_equal(op.in_code, om.in_code)
     else:
         assert not np.array_equal(op.in_meta, om.in_meta)
     if gran != m.GRAN_ELEM:
