@@ -20,10 +20,10 @@ def sdq():
     return m
 
 
-def check_sampled(M, N, K, seed, out_n=1, n_tok=12, use_ws=False, block=64):
+def check_sampled(M, N, K, seed, out_n=1, n_tok=12, use_ws=False, block=64, gran=so.GRAN_PAIR):
     m = sdq()
-    cfg = m.Config(out_n, m.GRAN_PAIR, block, 0)
-    ocfg = so.Config(out_n, so.GRAN_PAIR, block, 0)
+    cfg = m.Config(out_n, gran, block, 0)
+    ocfg = so.Config(out_n, gran, block, 0)
     W = sdq_synth.make_weight(N, K, seed, device="cuda")
     X = sdq_synth.make_act(M, K, seed + 1, device="cuda")
     p = m.sdq_decompose(W, cfg)
@@ -75,6 +75,12 @@ def test_llama7b_mlp_prefill(N, K):
 def test_scale_block_32_at_full_size(M, N, K):
     """configs 2 and 3 with one scale per 32 K (the literal block-32 MXFP4 wording)"""
     check_sampled(M, N, K, 3500 + M, block=32)
+
+
+@pytest.mark.parametrize("M,N,K,n", [(16, 4096, 4096, 7), (2048, 11008, 4096, 7), (2048, 4096, 11008, 8), (4096, 16384, 4096, 7)])
+def test_n_of_8_patterns_at_full_size(M, N, K, n):
+    """configs 2, 3 and 4 with the evaluation's patterns 7:8 = 1:8 + 6:8 and 8:8 = 1:8 + 7:8 (inliers stored dense)"""
+    check_sampled(M, N, K, 3700 + M + n, block=32, gran=so.gran_keep(n))
 
 
 @pytest.mark.parametrize("out_n", [1, 2, 0])
