@@ -436,7 +436,11 @@ def run_case(args):
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
     cfg = sdq.Config(1, sdq.GRAN_PAIR, 64, sdq.SCALE_OCP_FLOOR)
-    if args.case == "gemm_prefill":
+    if args.case == "gemm_prefill_dense":        # 8:8 = 1:8 FP8 outliers + dense MXFP4 inliers
+        cfg = sdq.Config(1, sdq.GRAN_DENSE, 32, sdq.SCALE_OCP_FLOOR)
+    elif args.case == "gemm_prefill_mxfp4":      # no outliers, no pruning: a plain block-scaled 4-bit GEMM
+        cfg = sdq.Config(0, sdq.GRAN_DENSE, 32, sdq.SCALE_OCP_FLOOR)
+    if args.case.startswith("gemm_prefill"):
         M, K, N = M_PREFILL, D_MODEL, D_FF
     elif args.case == "gemm_decode":
         M, K, N = 16, 4096, 4096
@@ -563,7 +567,7 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--sweep", action="store_true", help="measure the other configurations (OPT FFN outlier sweep, whole-model pass) and exit")
-    ap.add_argument("--case", default=None, choices=["gemm_prefill", "gemm_decode", "quant"],
+    ap.add_argument("--case", default=None, choices=["gemm_prefill", "gemm_prefill_dense", "gemm_prefill_mxfp4", "gemm_decode", "quant"],
                     help="run only a small single-kernel case (for profiler captures) and exit")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)

@@ -94,6 +94,15 @@ def test_persistent_many_token_kernel(M, N, K, out_n):
     run_case(M, N, K, 200 + M, out_n=out_n)
 
 
+@pytest.mark.parametrize("M,N,K,out_n,rule", [(600, 8192, 512, 1, 0), (161, 38400, 256, 1, 0), (481, 12800, 256, 2, 1), (640, 8192, 256, 0, 0),
+                                              (1000, 5120, 768, 1, 0), (329, 19200, 256, 1, 1)])
+def test_many_tokens_more_tiles_than_sms(M, N, K, out_n, rule):
+    """many tokens and more 128 x 256 tiles than SMs, so that persistent CTAs run several tiles each; ragged last token
+    tile, with and without a second 128-token record in it; sampled row tiles checked"""
+    rows = (0, 256) if N <= 8192 else (N - 384, N - 128)
+    run_case(M, N, K, 1700 + M, out_n=out_n, rule=rule, check_rows=rows)
+
+
 def _random_shapes(n, seed):
     rng = np.random.default_rng(seed)
     out = []
