@@ -28,6 +28,7 @@
 
 namespace sdq {
 
+constexpr int LIN_THREADS_MANY = 416;   // many-token instantiations: warps 9..12 = a second epilogue group (tokens 128..255 of the tile)
 constexpr int LIN_THREADS = 288;   // warps: 0 weight producer, 1 MMA issuer, 2..5 epilogue, 6 activation producer, 7 scale-atom producer,
                                    // 8 metadata / scale mover (many-token instantiation only)
 constexpr int MAX_SLOTS = 16;
@@ -82,8 +83,8 @@ __device__ __forceinline__ TileCoord tile_coord(int ksplit, int tile, int RT, in
 // B32 (many-token instantiation only): one scale per 32 K, four ring slots of 45 KB.
 // DENSE (many-token instantiation only): dense inliers with one scale per 32 K, four ring slots of 51 KB.
 template <bool F32_OUT, bool FLEX, bool B32, bool DENSE>
-__global__ void __maxnreg__(96)   // two 9-warp CTAs share an SM only below ~100 registers per thread
-sdq_linear_kernel(const LinearParams p)
+__global__ void __maxnreg__(FLEX ? 96 : 128)   // runtime geometry: two 9-warp CTAs share an SM only below ~100 registers per thread;
+sdq_linear_kernel(const LinearParams p)       // many tokens: 13 warps, four of them on one sub-partition of 16 K registers
 {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -132,7 +133,7 @@ sdq_linear_kernel(const LinearParams p)
       ptx::mbar_init(&full_w[s], 2);
     }
     ptx::mbar_init(acc_full, 1);
-    ptx::mbar_init(acc_empty, 4);
+    ptx::mbar_init(acc_empty, FLEX ? 4 : 8);
     ptx::fence_barrier_init();
   }
   if (warp == 1) ptx::tmem_alloc(tmem_slot, tmem_cols);
@@ -383,10 +384,12 @@ sdq_linear_kernel(const LinearParams p)
       }
       if (!ok) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
     }
-  } else if (warp >= 2 && warp <= 5) {
-    // ---------------- epilogue: warp w owns TMEM lanes 32*(w%4) .. +31 (weight rows), columns = tokens
+  } else if ((warp >= 2 && warp <= 5) || warp >= 9) {
+    // ---------------- epilogue: warp w owns TMEM lanes 32*(w%4) .. +31 (weight rows), columns = tokens; many tokens: a
+    // second group of four warps (9..12) takes tokens 128..255 of the tile
     const uint32_t q = warp & 3;
-    const uint32_t et = (warp - 2) * 32 + lane;     // 0..127 among the epilogue threads
+    const uint32_t grp = warp >= 9 ? 1u : 0u;
+    const uint32_t et = (warp - (grp ? 9u : 2u)) * 32 + lane;     // 0..127 among the epilogue threads of the group
     uint32_t tcount = 0;
     bool ok = true;
     ptx::griddep_wait();                            // Y and the workspace may still be in use by the previous kernel
@@ -403,6 +406,68 @@ sdq_linear_kernel(const LinearParams p)
       if (cluster_ks > 1) part = reinterpret_cast<float*>(sm);   // the ring is idle once the accumulator is complete
       else if (ksplit > 1)
         part = p.ws_partial + ((size_t)(tc.rt * p.n_mtiles + tc.mtile) * ksplit + tc.split) * (size_t)n_tile * TILE_ROWS;
+      if constexpr (!FLEX && F32_OUT) {
+        if (grp) {                                  // fp32 output (tests): the first group stores everything
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(acc_empty);
+          continue;
+        }
+      }
+      if constexpr (!FLEX && !F32_OUT) {
+        // many tokens, bf16 output: the accumulator cannot be double-buffered (TMEM is full), so the epilogue first
+        // drains it into registers -- one weight row x 128 tokens per thread as 64 packed bf16 pairs -- hands TMEM back,
+        // and only then transposes and stores: the stores run under the next tile's K loop
+        uint32_t pk[64];
+        {
+          uint32_t va[16], vb[16];
+          const uint32_t tbase = tmem + ((q * 32u) << 16) + TM_D + 128u * grp;
+          ptx::tmem_ld_32x32b_x16(tbase, va);
+#pragma unroll
+          for (int c = 0; c < 128; c += 32) {
+            ptx::tmem_ld_wait();
+            ptx::tmem_ld_32x32b_x16(tbase + (uint32_t)(c + 16), vb);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(va[2 * j]), __uint_as_float(va[2 * j + 1]));
+              pk[c / 2 + j] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+            ptx::tmem_ld_wait();
+            if (c + 32 < 128) ptx::tmem_ld_32x32b_x16(tbase + (uint32_t)(c + 32), va);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(vb[2 * j]), __uint_as_float(vb[2 * j + 1]));
+              pk[c / 2 + 8 + j] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+          }
+        }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(acc_empty);
+        // transpose through shared memory, 8 tokens at a time per group: [8 tokens][128 features] bf16, then one 16-byte
+        // store per thread (full 256 B rows)
+        uint16_t* stg = reinterpret_cast<uint16_t*>(sm + SM_STG) + grp * 1024u;
+        __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(p.Y);
+        const int g0 = 128 * (int)grp;
+#pragma unroll
+        for (int c0 = 0; c0 < 128; c0 += 8) {
+          if (g0 + c0 < n_valid) {                  // uniform over the four warps of the group
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              stg[(2 * j) * 128 + q * 32 + lane] = (uint16_t)(pk[c0 / 2 + j] & 0xFFFFu);
+              stg[(2 * j + 1) * 128 + q * 32 + lane] = (uint16_t)(pk[c0 / 2 + j] >> 16);
+            }
+            ptx::named_bar_sync(1 + grp, 128);
+            const uint32_t tok = et >> 4, seg = et & 15;
+            if (g0 + c0 + (int)tok < n_valid) {
+              const uint4 w = *reinterpret_cast<const uint4*>(stg + tok * 128 + seg * 8);
+              *reinterpret_cast<uint4*>(Y + (m0 + g0 + c0 + tok) * p.ldy + n0 + seg * 8) = w;
+            }
+            ptx::named_bar_sync(1 + grp, 128);       // the buffer is rewritten by the next chunk
+          }
+        }
+        continue;
+      }
       if (part) {
         // split K: all n_tile token columns of the partial tile go out (the reduction reads only the valid ones); the
         // TMEM load of the next 16 columns is in flight while the current 16 are stored
@@ -706,7 +771,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   const int smem = p.ring_bytes + SM_TAIL;
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3((unsigned)grid_x);
-  lc.blockDim = dim3(LIN_THREADS);
+  lc.blockDim = dim3(LIN_THREADS);   // the many-token instantiations get LIN_THREADS_MANY below
   lc.dynamicSmemBytes = (size_t)smem;
   lc.stream = (cudaStream_t)stream;
   // the kernel may be scheduled while the previous one in the stream drains: set-up and weight copies overlap its tail
@@ -725,6 +790,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   lc.attrs = attr;
   lc.numAttrs = na;
   const bool flex = !(p.n_tile == 256 && p.ksplit == 1 && p.nslot == (p.b32 ? 4 : 5) && p.release == 1);
+  if (!flex) lc.blockDim = dim3(LIN_THREADS_MANY);
   cudaError_t le;
   if (flex) le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, true, false, false>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, true, false, false>, p);
   else if (p.dense) le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, false, false, true>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, false, false, true>, p);
