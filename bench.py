@@ -246,7 +246,7 @@ def run_ours(args):
                 "frac": gemm_tf / mixed_peak,
                 # dram__bytes_read.sum + dram__bytes_write.sum of one captured launch of the gate / up shape
                 # (profiles/sdq_linear_kernel_prefill_M2048_N11008_K4096.md); the down shape was not captured
-                "traffic": 90.8e6, "traffic_unit": "bytes per launch (gate/up shape)",
+                "traffic": 87.7e6, "traffic_unit": "bytes per launch (gate/up shape)",
                 "peak_basis": "%s bf16 burst %.1f TF/s x 8/3 (sparse FP4 at 8x + sparse FP8 at 4x per dense-equivalent flop)" % (peaks["source"], peaks["bf16"]),
                 "avg_launch_ms": gemm_ms / gemm_n, "launches": gemm_n,
                 "frac_of_sparse_fp4_peak": gemm_tf / (8 * peaks["bf16"])}
