@@ -6,12 +6,15 @@
 // then its outlier K loop
 //   2 x tcgen05.mma.sp kind::mxf8f6f4 per 128 K (1:8 / 2:8 E4M3 outliers embedded in 2:4 x E4M3 activations;
 //                                                the power-of-two row / token scales ride in as E8M0 factors)
-// both into ONE fp32 TMEM accumulator.  Persistent CTAs walk tiles of 128 rows x up to 256 tokens.
+// both into ONE fp32 TMEM accumulator (dense / n:8 inliers: 4 x dense tcgen05.mma kind::mxf4 of 64 K per 256 K instead;
+// one scale per 32 K: kind::mxf4nvf4 .block16).  Persistent CTAs walk tiles of 128 rows x up to 256 tokens.
 // Warp roles: warps 0, 6, 7 = bulk-copy (TMA) producers for weights, activations and scale atoms (issuing a
 // bulk copy costs one thread ~50 ns, so the copies of a stage are spread over three threads), warp 1 = TMEM
 // owner + MMA issuer, warps 2..5 = epilogue (tcgen05.ld, convert, shared-memory transpose, 16-byte row stores),
-// warp 8 = mover of metadata and scale atoms smem -> TMEM (tcgen05.cp) in the many-token instantiation; with
-// runtime geometry the MMA issuer does those copies itself.
+// warp 8 = mover of metadata and scale atoms smem -> TMEM (tcgen05.cp) in the many-token instantiations; with
+// runtime geometry the MMA issuer does those copies itself.  The many-token instantiations run four more warps
+// (9..12), a second epilogue group: the eight epilogue warps load the accumulator into registers, hand TMEM back
+// and store under the next tile's K loop.
 // For few tokens the K range of a row tile is split over several CTAs: either a thread-block cluster whose members
 // keep their fp32 partial tiles in shared memory and each add one slice of rows over all members in rank order
 // (no global scratch), or, with a caller-provided workspace, partial tiles in global memory that the last CTA to
