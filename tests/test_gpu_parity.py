@@ -402,6 +402,93 @@ def test_leading_dimensions_larger_than_the_row(M):
     assert (Ybig[:, N:] == 123.0).all() and (Y32big[:, N:] == 123.0).all()
 
 
+def test_leading_dimension_of_y_in_the_many_token_kernel():
+    """ldy > N where persistent thread blocks run several tiles each (the epilogue that stores under the next tile's K
+    loop): sampled row tiles against the oracle, bf16 = rounded fp32, nothing written outside the view"""
+    m = sdq()
+    cfg = m.Config()
+    M, N, K = 601, 6400, 256
+    W = sdq_synth.make_weight(N, K, 73)
+    X = sdq_synth.make_act(M, K, 74)
+    p = m.sdq_decompose(W.cuda(), cfg)
+    xq = m.sdq_quantize_act(X.cuda(), cfg)
+    Ybig = torch.full((M + 3, N + 72), 123.0, dtype=torch.bfloat16, device="cuda")
+    Y32big = torch.full((M + 3, N + 8), 123.0, dtype=torch.float32, device="cuda")
+    m.sdq_linear(xq, p, Ybig[:M, :N])
+    m.sdq_linear(xq, p, Y32big[:M, :N], f32=True)
+    assert m.device_status() == 0
+    assert (Ybig[:, N:] == 123.0).all() and (Ybig[M:] == 123.0).all()
+    assert (Y32big[:, N:] == 123.0).all() and (Y32big[M:] == 123.0).all()
+    assert torch.equal(Ybig[:M, :N], Y32big[:M, :N].to(torch.bfloat16))
+    oq = so.quantize_act(sdq_synth.bf16_bits(X), ocfg())
+    for t in (0, 24, 49):
+        op = so.decompose(sdq_synth.bf16_bits(W[128 * t:128 * t + 128]), ocfg())
+        d, tol = y_close(Y32big[:M, 128 * t:128 * t + 128].cpu().numpy(), so.linear(oq, op))
+        assert (d <= tol).all(), (t, d.max())
+
+
+@pytest.mark.parametrize("M,N,K", [(16, 1024, 2048), (700, 6400, 512)])
+def test_streams_and_graph_replay_give_the_eager_result(M, N, K):
+    """the quantizer + GEMM chain on two streams at once (separate buffers) and captured in a CUDA graph replayed
+    twice: bit-identical to the eager result on the default stream"""
+    m = sdq()
+    cfg = m.Config()
+    W = sdq_synth.make_weight(N, K, 81).cuda()
+    X = sdq_synth.make_act(M, K, 82).cuda()
+    p = m.sdq_decompose(W, cfg)
+    y_eager = m.sdq_linear(m.sdq_quantize_act(X, cfg), p)
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream() for _ in range(2)]
+    bufs = [torch.empty(m.act_size(M, K, cfg), dtype=torch.uint8, device="cuda") for _ in range(2)]
+    outs = [torch.zeros((M, N), dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    for _ in range(3):
+        for st, b, o in zip(streams, bufs, outs):
+            with torch.cuda.stream(st):
+                m.sdq_linear(m.sdq_quantize_act(X, cfg, b), p, o)
+    torch.cuda.synchronize()
+    assert torch.equal(outs[0], y_eager) and torch.equal(outs[1], y_eager)
+    g = torch.cuda.CUDAGraph()
+    yg = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        m.sdq_linear(m.sdq_quantize_act(X, cfg, bufs[0]), p, yg)     # warm-up outside the capture
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(g):
+        m.sdq_linear(m.sdq_quantize_act(X, cfg, bufs[0]), p, yg)
+    for _ in range(2):
+        yg.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(yg, y_eager)
+    assert m.device_status() == 0
+
+
+@pytest.mark.parametrize("M,N,K,out_n", [(8, 128, 32768, 1), (20001, 256, 256, 1), (3, 128, 16640, 2)])
+def test_extreme_shapes_long_rows_and_many_tokens(M, N, K, out_n):
+    """the longest rows (128 inlier + 256 outlier stages per tile; a row length only the two-pass quantizer takes) and
+    tens of thousands of tokens with a ragged last tile; tokens sampled for the oracle"""
+    m = sdq()
+    cfg = m.Config(out_n, m.GRAN_PAIR, 64, 0)
+    W = sdq_synth.make_weight(N, K, 91 + M % 7)
+    X = sdq_synth.make_act(M, K, 92 + M % 7)
+    p = m.sdq_decompose(W.cuda(), cfg)
+    xq = m.sdq_quantize_act(X.cuda(), cfg)
+    y = m.sdq_linear(xq, p, f32=True)
+    y16 = m.sdq_linear(xq, p)
+    assert m.device_status() == 0
+    assert torch.equal(y16, y.to(torch.bfloat16))
+    toks = np.unique(np.concatenate([[0, M - 1], np.random.default_rng(M).integers(0, M, size=min(M, 24))]))
+    op = so.decompose(sdq_synth.bf16_bits(W), ocfg(out_n))
+    oq = so.quantize_act(sdq_synth.bf16_bits(X[toks]), ocfg(out_n))
+    ae = m.act_export(xq)
+    for name in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp"):
+        assert np.array_equal(ae[name][torch.from_numpy(toks).cuda()].cpu().numpy(), getattr(oq, name)), name
+    d, tol = y_close(y[torch.from_numpy(toks).cuda()].cpu().numpy(), so.linear(oq, op))
+    assert (d <= tol).all(), (d.max(), (d / tol).max())
+
+
 @pytest.mark.parametrize("M,K", [(1, 256), (77, 512), (2048, 4096)])
 def test_channel_norm_and_calibrated_decomposition(M, K):
     """sdq_channel_norm against the fp64 definition (fp64 accumulation on both sides: equal after rounding to fp32, one
