@@ -38,6 +38,12 @@
 #define SDQO_GRAN_KEEP(n) (2 + (8 - (n)))
 #define SDQO_SCALE_OCP_FLOOR 0  /* E = floor(log2 amax) - 2   (OCP MX rule, may saturate in (6,8)) */
 #define SDQO_SCALE_CEIL_NOSAT 1 /* E = smallest integer with amax <= 6 * 2^E                        */
+/* Two-level scaling with 8-bit floating-point Q-Vector scales (the quantization-stage study: scale factors in
+   fp8-e4m3 work best): a vector (the kept inliers of a weight row, or a token) gets a power-of-two factor 2^t,
+   t = the exponent of its 8-bit scale (smallest t with amax <= 448 * 2^t); a Q-Vector gets the unsigned E4M3 scale
+   nearest to amax_q / (6 * 2^t) (ties to the even code; never below the smallest positive one unless the Q-Vector is
+   all zero); an element is the E2M1 value nearest to x / (scale * 2^t), ties to even, saturating at 6. */
+#define SDQO_SCALE_UE4M3 2
 
 typedef struct {
   int out_n;      /* outliers kept per S-Vector of 8 along K: 0, 1 or 2          */
@@ -138,6 +144,17 @@ int sdqo_fp8_scale_exp(double amax) {
   return e;
 }
 
+/* unsigned-E4M3 code (0x00..0x7E) of a Q-Vector scale under SDQO_SCALE_UE4M3, and the scaled E2M1 code of an element */
+uint8_t sdqo_ue4m3_scale_code(double amax_q, int t) {
+  if (amax_q == 0.0) return 0;
+  uint8_t c = sdqo_e4m3_encode(ldexp(amax_q, -t) / 6.0);
+  return c == 0 ? 1 : c;
+}
+static uint8_t e2m1_of_quotient(double x, uint8_t scale_code, int t) {
+  if (scale_code == 0) return 0;
+  return sdqo_e2m1_encode(x / ldexp(sdqo_e4m3_decode(scale_code), t));
+}
+
 /* magnitude key used by every "largest" selection: the 15 low bits of the bf16 pattern */
 
 static int is_finite_bf16(uint16_t h) { return (h & 0x7F80) != 0x7F80; }
@@ -150,7 +167,8 @@ static int is_finite_bf16(uint16_t h) { return (h & 0x7F80) != 0x7F80; }
  *   in_meta  [N][K/8] (PAIR: j0 | j1<<2, kept pair indices 0..3 of the group of 8)
  *            [N][K/4] (ELEM: i0 | i1<<2, kept element indices 0..3 of the group of 4)
  *            not touched for DENSE / KEEP(n) (dropped and outlier positions simply hold +0)
- *   in_scale [N][K/in_block] E8M0 code
+ *   in_scale [N][K/in_block] E8M0 code (SDQO_SCALE_UE4M3: unsigned E4M3 code, times 2^in_texp[n])
+ *   in_texp  [N]           SDQO_SCALE_UE4M3: exponent t of the row's power-of-two factor (int32); else 0 (may be NULL)
  *   out_code [N][K/8][out_n] E4M3 codes; out_idx same shape, position 0..7 inside the group, ascending
  *   out_sexp [N]           e of the per-row outlier scale 2^e (int32)
  * returns 0, or -1 on a bad argument, -2 if W holds a non-finite value.
@@ -170,13 +188,14 @@ static float significance(uint16_t w, const float* col_weight, int64_t k) {
 
 int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_config* cfg, const float* col_weight,
                           uint8_t* in_code, uint8_t* in_meta, uint8_t* in_scale,
-                          uint8_t* out_code, uint8_t* out_idx, int32_t* out_sexp) {
+                          uint8_t* out_code, uint8_t* out_idx, int32_t* out_sexp, int32_t* in_texp) {
   if (!W || !cfg || N <= 0 || K <= 0 || K % 64 != 0) return -1;
   if (col_weight)
     for (int64_t k = 0; k < K; ++k)
       if (!(col_weight[k] >= 0.0f) || isinf(col_weight[k])) return -3;
   if (cfg->out_n < 0 || cfg->out_n > 2) return -1;
   if (cfg->in_block != 32 && cfg->in_block != 64) return -1;
+  if (cfg->scale_rule < 0 || cfg->scale_rule > SDQO_SCALE_UE4M3 || (cfg->scale_rule == SDQO_SCALE_UE4M3 && !in_texp)) return -1;
   if (cfg->in_gran < 0 || cfg->in_gran > SDQO_GRAN_KEEP(2)) return -1;
   const int keep_n = 10 - cfg->in_gran;                                /* n of KEEP(n); meaningful from DENSE on */
   if (cfg->in_gran >= SDQO_GRAN_DENSE && keep_n <= cfg->out_n) return -1;
@@ -282,6 +301,18 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
 
     /* Stage 3 for inliers: per Q-Vector E8M0 scale over the kept inlier values, then E2M1 codes.
        A kept slot that holds an outlier position carries the value +0. */
+    const int ue = cfg->scale_rule == SDQO_SCALE_UE4M3;
+    int t = 0;                                   /* two-level scaling: the row's power-of-two factor */
+    if (ue) {
+      double row_amax = 0.0;
+      for (int64_t k = 0; k < K; ++k)
+        if (kept[k] && !is_out[k] && !dropped[k]) {
+          double a = fabs(sdqo_bf16_to_double(w[k]));
+          if (a > row_amax) row_amax = a;
+        }
+      t = sdqo_fp8_scale_exp(row_amax);
+    }
+    if (in_texp) in_texp[n] = t;
     for (int64_t b = 0; b < K / Bs; ++b) {
       double amax = 0.0;
       for (int64_t k = b * Bs; k < (b + 1) * Bs; ++k)
@@ -289,7 +320,7 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
           double a = fabs(sdqo_bf16_to_double(w[k]));
           if (a > amax) amax = a;
         }
-      in_scale[n * (K / Bs) + b] = sdqo_e8m0_scale_code(amax, cfg->scale_rule);
+      in_scale[n * (K / Bs) + b] = ue ? sdqo_ue4m3_scale_code(amax, t) : sdqo_e8m0_scale_code(amax, cfg->scale_rule);
     }
     int64_t slot = 0;
     for (int64_t k = 0; k < K; ++k) {
@@ -297,7 +328,8 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
       uint8_t code = 0;
       if (!is_out[k] && !dropped[k]) {
         int c = in_scale[n * (K / Bs) + k / Bs];
-        code = sdqo_e2m1_encode(ldexp(sdqo_bf16_to_double(w[k]), 127 - c));
+        code = ue ? e2m1_of_quotient(sdqo_bf16_to_double(w[k]), (uint8_t)c, t)
+                  : sdqo_e2m1_encode(ldexp(sdqo_bf16_to_double(w[k]), 127 - c));
       }
       in_code[n * slots + slot++] = code;
     }
@@ -312,14 +344,20 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
 /* magnitude metric: the decomposition of Section 5 with |w| as the significance */
 int sdqo_decompose(const uint16_t* W, int64_t N, int64_t K, const sdqo_config* cfg,
                    uint8_t* in_code, uint8_t* in_meta, uint8_t* in_scale,
-                   uint8_t* out_code, uint8_t* out_idx, int32_t* out_sexp) {
-  return sdqo_decompose_metric(W, N, K, cfg, (const float*)0, in_code, in_meta, in_scale, out_code, out_idx, out_sexp);
+                   uint8_t* out_code, uint8_t* out_idx, int32_t* out_sexp, int32_t* in_texp) {
+  return sdqo_decompose_metric(W, N, K, cfg, (const float*)0, in_code, in_meta, in_scale, out_code, out_idx, out_sexp, in_texp);
 }
 
-/* Dequantize the canonical arrays of ONE weight matrix back to dense W_i and W_o (fp64, [N][K]). */
+/* value of a Q-Vector scale code: E8M0, or unsigned E4M3 times the vector's power-of-two factor 2^t */
+static double scale_value(const sdqo_config* cfg, uint8_t code, int t) {
+  return cfg->scale_rule == SDQO_SCALE_UE4M3 ? ldexp(sdqo_e4m3_decode(code), t) : sdqo_e8m0_decode(code);
+}
+
+/* Dequantize the canonical arrays of ONE weight matrix back to dense W_i and W_o (fp64, [N][K]).
+   in_texp [N]: the rows' power-of-two factors (read under SDQO_SCALE_UE4M3 only). */
 int sdqo_dequant_weights(int64_t N, int64_t K, const sdqo_config* cfg,
                          const uint8_t* in_code, const uint8_t* in_meta, const uint8_t* in_scale,
-                         const uint8_t* out_code, const uint8_t* out_idx, const int32_t* out_sexp,
+                         const uint8_t* out_code, const uint8_t* out_idx, const int32_t* out_sexp, const int32_t* in_texp,
                          double* W_in, double* W_out) {
   const int on = cfg->out_n, Bs = cfg->in_block;
   const int64_t G8 = K / 8;
@@ -329,7 +367,7 @@ int sdqo_dequant_weights(int64_t N, int64_t K, const sdqo_config* cfg,
     int64_t slot = 0;
     if (cfg->in_gran >= SDQO_GRAN_DENSE) {
       for (int64_t k = 0; k < K; ++k)
-        W_in[n * K + k] = sdqo_e2m1_decode(in_code[n * K + k]) * sdqo_e8m0_decode(in_scale[n * (K / Bs) + k / Bs]);
+        W_in[n * K + k] = sdqo_e2m1_decode(in_code[n * K + k]) * scale_value(cfg, in_scale[n * (K / Bs) + k / Bs], in_texp ? in_texp[n] : 0);
     } else if (cfg->in_gran == SDQO_GRAN_PAIR) {
       for (int64_t g = 0; g < G8; ++g) {
         int nib = in_meta[n * G8 + g];
@@ -338,7 +376,7 @@ int sdqo_dequant_weights(int64_t N, int64_t K, const sdqo_config* cfg,
           for (int u = 0; u < 2; ++u) {
             int64_t k = 8 * g + 2 * jj[t] + u;
             W_in[n * K + k] = sdqo_e2m1_decode(in_code[n * (K / 2) + slot++]) *
-                              sdqo_e8m0_decode(in_scale[n * (K / Bs) + k / Bs]);
+                              scale_value(cfg, in_scale[n * (K / Bs) + k / Bs], in_texp ? in_texp[n] : 0);
           }
       }
     } else {
@@ -348,7 +386,7 @@ int sdqo_dequant_weights(int64_t N, int64_t K, const sdqo_config* cfg,
         for (int t = 0; t < 2; ++t) {
           int64_t k = 4 * h + ii[t];
           W_in[n * K + k] = sdqo_e2m1_decode(in_code[n * (K / 2) + slot++]) *
-                            sdqo_e8m0_decode(in_scale[n * (K / Bs) + k / Bs]);
+                            scale_value(cfg, in_scale[n * (K / Bs) + k / Bs], in_texp ? in_texp[n] : 0);
         }
       }
     }
@@ -362,13 +400,15 @@ int sdqo_dequant_weights(int64_t N, int64_t K, const sdqo_config* cfg,
 }
 
 /* ------------------------------------------------------------------ activations: A -> A_i (4-bit), A_o (8-bit)
- * X [M][K] bf16 patterns.  xq4_code [M][K] E2M1 codes, xq4_scale [M][K/in_block] E8M0 codes,
+ * X [M][K] bf16 patterns.  xq4_code [M][K] E2M1 codes, xq4_scale [M][K/in_block] E8M0 codes (SDQO_SCALE_UE4M3:
+ * unsigned E4M3 codes; the Q-Vector scale is then that value times 2^xq8_sexp[m]),
  * xq8_code [M][K] E4M3 codes, xq8_sexp [M] exponent e of the per-token scale 2^e.
  * +-Inf saturates to the largest finite value; NaN is rejected (-2). */
 int sdqo_quantize_act(const uint16_t* X, int64_t M, int64_t K, const sdqo_config* cfg,
                       uint8_t* xq4_code, uint8_t* xq4_scale, uint8_t* xq8_code, int32_t* xq8_sexp) {
   if (!X || !cfg || M <= 0 || K <= 0) return -1;
   if (cfg->in_block != 32 && cfg->in_block != 64) return -1;
+  if (cfg->scale_rule < 0 || cfg->scale_rule > SDQO_SCALE_UE4M3) return -1;
   if (K % cfg->in_block != 0) return -1;
   const int Bs = cfg->in_block;
   const double BF16_MAX = 3.3895313892515355e38;
@@ -378,6 +418,15 @@ int sdqo_quantize_act(const uint16_t* X, int64_t M, int64_t K, const sdqo_config
     for (int64_t k = 0; k < K; ++k) {
       if ((x[k] & 0x7F80) == 0x7F80 && (x[k] & 0x007F)) return -2; /* NaN */
     }
+    const int ue = cfg->scale_rule == SDQO_SCALE_UE4M3;
+    for (int64_t k = 0; k < K; ++k) {
+      double a = fabs(sdqo_bf16_to_double(x[k]));
+      if (isinf(a)) a = BF16_MAX;
+      if (a > row_amax) row_amax = a;
+    }
+    /* the token's 8-bit scale exponent; under two-level scaling also the power-of-two factor of its 4-bit Q-Vectors */
+    const int e = sdqo_fp8_scale_exp(row_amax);
+    xq8_sexp[m] = e;
     for (int64_t b = 0; b < K / Bs; ++b) {
       double amax = 0.0;
       for (int64_t k = b * Bs; k < (b + 1) * Bs; ++k) {
@@ -385,17 +434,14 @@ int sdqo_quantize_act(const uint16_t* X, int64_t M, int64_t K, const sdqo_config
         if (isinf(a)) a = BF16_MAX;
         if (a > amax) amax = a;
       }
-      if (amax > row_amax) row_amax = amax;
-      uint8_t c = sdqo_e8m0_scale_code(amax, cfg->scale_rule);
+      uint8_t c = ue ? sdqo_ue4m3_scale_code(amax, e) : sdqo_e8m0_scale_code(amax, cfg->scale_rule);
       xq4_scale[m * (K / Bs) + b] = c;
       for (int64_t k = b * Bs; k < (b + 1) * Bs; ++k) {
         double v = sdqo_bf16_to_double(x[k]);
         if (isinf(v)) v = copysign(BF16_MAX, v);
-        xq4_code[m * K + k] = sdqo_e2m1_encode(ldexp(v, 127 - (int)c));
+        xq4_code[m * K + k] = ue ? e2m1_of_quotient(v, c, e) : sdqo_e2m1_encode(ldexp(v, 127 - (int)c));
       }
     }
-    const int e = sdqo_fp8_scale_exp(row_amax);
-    xq8_sexp[m] = e;
     for (int64_t k = 0; k < K; ++k) {
       double v = sdqo_bf16_to_double(x[k]);
       if (isinf(v)) v = copysign(BF16_MAX, v);
@@ -411,7 +457,7 @@ int sdqo_quantize_act(const uint16_t* X, int64_t M, int64_t K, const sdqo_config
  * Only the non-zero weights are visited; every term is formed and added in fp64. */
 int sdqo_linear(int64_t M, int64_t N, int64_t K, const sdqo_config* cfg,
                 const uint8_t* in_code, const uint8_t* in_meta, const uint8_t* in_scale,
-                const uint8_t* out_code, const uint8_t* out_idx, const int32_t* out_sexp,
+                const uint8_t* out_code, const uint8_t* out_idx, const int32_t* out_sexp, const int32_t* in_texp,
                 const uint8_t* xq4_code, const uint8_t* xq4_scale, const uint8_t* xq8_code, const int32_t* xq8_sexp,
                 int64_t n_begin, int64_t n_end, double* Y, int n_threads) {
   if (n_begin < 0 || n_end > N || n_begin > n_end) return -1;
@@ -421,7 +467,7 @@ int sdqo_linear(int64_t M, int64_t N, int64_t K, const sdqo_config* cfg,
   double* A_o = (double*)malloc(sizeof(double) * (size_t)(M * K));
   for (int64_t m = 0; m < M; ++m)
     for (int64_t k = 0; k < K; ++k) {
-      A_i[m * K + k] = sdqo_e2m1_decode(xq4_code[m * K + k]) * sdqo_e8m0_decode(xq4_scale[m * (K / Bs) + k / Bs]);
+      A_i[m * K + k] = sdqo_e2m1_decode(xq4_code[m * K + k]) * scale_value(cfg, xq4_scale[m * (K / Bs) + k / Bs], xq8_sexp[m]);
       A_o[m * K + k] = ldexp(sdqo_e4m3_decode(xq8_code[m * K + k]), xq8_sexp[m]);
     }
 #pragma omp parallel num_threads(n_threads > 0 ? n_threads : 1)
@@ -437,7 +483,7 @@ int sdqo_linear(int64_t M, int64_t N, int64_t K, const sdqo_config* cfg,
       if (cfg->in_gran >= SDQO_GRAN_DENSE) {
         for (int64_t k = 0; k < K; ++k) {
           ki[ni] = (int32_t)k;
-          wi[ni++] = sdqo_e2m1_decode(in_code[n * K + k]) * sdqo_e8m0_decode(in_scale[n * (K / Bs) + k / Bs]);
+          wi[ni++] = sdqo_e2m1_decode(in_code[n * K + k]) * scale_value(cfg, in_scale[n * (K / Bs) + k / Bs], in_texp ? in_texp[n] : 0);
         }
       } else if (cfg->in_gran == SDQO_GRAN_PAIR) {
         for (int64_t g = 0; g < G8; ++g) {
@@ -448,7 +494,7 @@ int sdqo_linear(int64_t M, int64_t N, int64_t K, const sdqo_config* cfg,
               int64_t k = 8 * g + 2 * jj[t] + u;
               ki[ni] = (int32_t)k;
               wi[ni++] = sdqo_e2m1_decode(in_code[n * (K / 2) + slot++]) *
-                         sdqo_e8m0_decode(in_scale[n * (K / Bs) + k / Bs]);
+                         scale_value(cfg, in_scale[n * (K / Bs) + k / Bs], in_texp ? in_texp[n] : 0);
             }
         }
       } else {
@@ -459,7 +505,7 @@ int sdqo_linear(int64_t M, int64_t N, int64_t K, const sdqo_config* cfg,
             int64_t k = 4 * h + ii[t];
             ki[ni] = (int32_t)k;
             wi[ni++] = sdqo_e2m1_decode(in_code[n * (K / 2) + slot++]) *
-                       sdqo_e8m0_decode(in_scale[n * (K / Bs) + k / Bs]);
+                       scale_value(cfg, in_scale[n * (K / Bs) + k / Bs], in_texp ? in_texp[n] : 0);
           }
         }
       }

@@ -26,7 +26,7 @@ def gran_keep(n: int) -> int:
     any positions, stored like the dense pattern); gran_keep(8) == GRAN_DENSE."""
     assert 2 <= n <= 8
     return 2 + (8 - n)
-SCALE_OCP_FLOOR, SCALE_CEIL_NOSAT = 0, 1
+SCALE_OCP_FLOOR, SCALE_CEIL_NOSAT, SCALE_UE4M3 = 0, 1, 2
 
 
 def build(force: bool = False) -> str:
@@ -72,6 +72,8 @@ def lib():
             getattr(L, name).argtypes = [ctypes.c_double]
         L.sdqo_e8m0_scale_code.restype = ctypes.c_uint8
         L.sdqo_e8m0_scale_code.argtypes = [ctypes.c_double, ctypes.c_int]
+        L.sdqo_ue4m3_scale_code.restype = ctypes.c_uint8
+        L.sdqo_ue4m3_scale_code.argtypes = [ctypes.c_double, ctypes.c_int]
         L.sdqo_fp8_scale_exp.restype = ctypes.c_int
         L.sdqo_fp8_scale_exp.argtypes = [ctypes.c_double]
         L.sdqo_bits_per_weight_part.restype = ctypes.c_double
@@ -103,6 +105,7 @@ class Packed:
     out_code: np.ndarray   # [N, K/8, out_n] u8 E4M3 codes
     out_idx: np.ndarray    # [N, K/8, out_n] u8 positions 0..7
     out_sexp: np.ndarray   # [N] i32, outlier scale = 2^out_sexp
+    in_texp: np.ndarray = None   # [N] i32, SCALE_UE4M3: inlier scale = E4M3(in_scale) * 2^in_texp (zeros otherwise)
 
 
 @dataclass
@@ -129,7 +132,7 @@ def decompose(W_bits: np.ndarray, cfg: Config, col_weight=None) -> Packed:
                np.zeros((N, nslot), np.uint8), np.zeros((N, nmeta), np.uint8),
                np.zeros((N, K // cfg.in_block), np.uint8),
                np.zeros((N, K // 8, on), np.uint8), np.zeros((N, K // 8, on), np.uint8),
-               np.zeros((N,), np.int32))
+               np.zeros((N,), np.int32), np.zeros((N,), np.int32))
     c = cfg.c()
     if col_weight is None:
         cw = None
@@ -139,7 +142,7 @@ def decompose(W_bits: np.ndarray, cfg: Config, col_weight=None) -> Packed:
         cw = _p(cw_arr)
     rc = lib().sdqo_decompose_metric(_p(W_bits), ctypes.c_int64(N), ctypes.c_int64(K), ctypes.byref(c), cw,
                                      _p(p.in_code), _p(p.in_meta), _p(p.in_scale), _p(p.out_code), _p(p.out_idx),
-                                     _p(p.out_sexp))
+                                     _p(p.out_sexp), _p(p.in_texp))
     if rc != 0:
         raise ValueError("sdqo_decompose failed: %d" % rc)
     return p
@@ -160,7 +163,7 @@ def dequant_weights(p: Packed):
     c = p.cfg.c()
     rc = lib().sdqo_dequant_weights(ctypes.c_int64(p.N), ctypes.c_int64(p.K), ctypes.byref(c),
                                     _p(p.in_code), _p(p.in_meta), _p(p.in_scale), _p(p.out_code), _p(p.out_idx),
-                                    _p(p.out_sexp), _p(W_in), _p(W_out))
+                                    _p(p.out_sexp), _p(p.in_texp), _p(W_in), _p(W_out))
     assert rc == 0
     return W_in, W_out
 
@@ -183,7 +186,10 @@ def dequant_act(q: QAct):
     L = lib()
     e2m1 = np.array([L.sdqo_e2m1_decode(c) for c in range(16)])
     e4m3 = np.array([L.sdqo_e4m3_decode(c) for c in range(256)])
-    sc = np.repeat(np.ldexp(1.0, q.xq4_scale.astype(np.int64) - 127), q.cfg.in_block, axis=1)
+    if q.cfg.scale_rule == SCALE_UE4M3:
+        sc = np.repeat(np.ldexp(e4m3[q.xq4_scale], q.xq8_sexp[:, None].astype(np.int64)), q.cfg.in_block, axis=1)
+    else:
+        sc = np.repeat(np.ldexp(1.0, q.xq4_scale.astype(np.int64) - 127), q.cfg.in_block, axis=1)
     A_i = e2m1[q.xq4_code] * sc
     A_o = np.ldexp(e4m3[q.xq8_code], q.xq8_sexp[:, None].astype(np.int64))
     return A_i, A_o
@@ -198,7 +204,7 @@ def linear(q: QAct, p: Packed, n_begin: int = 0, n_end: int | None = None, threa
     c = p.cfg.c()
     rc = lib().sdqo_linear(ctypes.c_int64(q.M), ctypes.c_int64(p.N), ctypes.c_int64(p.K), ctypes.byref(c),
                            _p(p.in_code), _p(p.in_meta), _p(p.in_scale), _p(p.out_code), _p(p.out_idx),
-                           _p(p.out_sexp), _p(q.xq4_code), _p(q.xq4_scale), _p(q.xq8_code), _p(q.xq8_sexp),
+                           _p(p.out_sexp), _p(p.in_texp), _p(q.xq4_code), _p(q.xq4_scale), _p(q.xq8_code), _p(q.xq8_sexp),
                            ctypes.c_int64(n_begin), ctypes.c_int64(n_end), _p(Y), ctypes.c_int(threads))
     assert rc == 0
     return Y

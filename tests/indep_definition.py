@@ -61,6 +61,7 @@ def top_mask(keys, n):
 def decompose_dense(W_bits, out_n, pair, block, rule_floor, col_weight=None):
     """returns (W_in_hat, W_out_hat, mask_in_slots, mask_out) as dense [N, K] arrays; with col_weight the
     selections rank by the fp32 product |w| * c[k] instead of |w| (the values that get quantized do not change);
+    rule_floor: True = OCP floor rule, False = ceil rule, "ue4m3" = two-level scaling with e4m3 scales;
     pair: True = pair-wise 4:8, False = element-wise 2:4, None = no pruning,
     an integer n = the n most significant of every 8 survive (outliers included)"""
     W = bf16_to_f64(W_bits)
@@ -85,10 +86,13 @@ def decompose_dense(W_bits, out_n, pair, block, rule_floor, col_weight=None):
         slots = top_mask(keys, 2).reshape(N, K)
     inl = slots & ~mask_out
     Win = np.where(inl, W, 0.0)
-    amax = np.abs(Win).reshape(N, K // block, block).max(-1)
-    E = block_scale_exp(amax, rule_floor)
-    Es = np.repeat(E, block, axis=1)
-    Win_hat = np.where(inl, np.ldexp(q_e2m1(np.ldexp(Win, -Es)), Es), 0.0)
+    if rule_floor == "ue4m3":
+        Win_hat, _ = two_level_quantize(Win, inl, block)
+    else:
+        amax = np.abs(Win).reshape(N, K // block, block).max(-1)
+        E = block_scale_exp(amax, rule_floor)
+        Es = np.repeat(E, block, axis=1)
+        Win_hat = np.where(inl, np.ldexp(q_e2m1(np.ldexp(Win, -Es)), Es), 0.0)
     Wout = np.where(mask_out, W, 0.0)
     oamax = np.abs(Wout).max(axis=1)
     e = np.where(oamax > 0, ceil_exp(np.where(oamax > 0, oamax, 1.0), 448.0), 0)[:, None]
@@ -99,10 +103,31 @@ def decompose_dense(W_bits, out_n, pair, block, rule_floor, col_weight=None):
 def quantize_act_dense(X_bits, block, rule_floor):
     X = bf16_to_f64(X_bits)
     M, K = X.shape
-    amax = np.abs(X).reshape(M, K // block, block).max(-1)
-    Es = np.repeat(block_scale_exp(amax, rule_floor), block, axis=1)
-    A_i = np.ldexp(q_e2m1(np.ldexp(X, -Es)), Es)
+    if rule_floor == "ue4m3":
+        A_i, _ = two_level_quantize(X, np.ones(X.shape, bool), block)
+    else:
+        amax = np.abs(X).reshape(M, K // block, block).max(-1)
+        Es = np.repeat(block_scale_exp(amax, rule_floor), block, axis=1)
+        A_i = np.ldexp(q_e2m1(np.ldexp(X, -Es)), Es)
     ramax = np.abs(X).max(axis=1)
     e = np.where(ramax > 0, ceil_exp(np.where(ramax > 0, ramax, 1.0), 448.0), 0)[:, None]
     A_o = np.ldexp(q_e4m3(np.ldexp(X, -e)), e)
     return A_i, A_o
+
+
+def two_level_quantize(V, counted, block):
+    """Two-level scaling with fp8-e4m3 Q-Vector scales, stated with numpy and torch's own float8 cast: per row a
+    power-of-two factor 2^t (smallest t with amax <= 448 * 2^t over the counted elements), per block the e4m3 value
+    nearest to amax_b / (6 * 2^t) (at least 2^-9 unless the block is all zero), per element the E2M1 value nearest
+    to v / scale.  V [R, K] fp64, counted [R, K] bool (elements that exist); returns the dequantized values."""
+    R, K = V.shape
+    A = np.where(counted, np.abs(V), 0.0)
+    ramax = A.max(axis=1)
+    t = np.where(ramax > 0, ceil_exp(np.where(ramax > 0, ramax, 1.0), 448.0), 0)[:, None]
+    bamax = A.reshape(R, K // block, block).max(-1)
+    y = np.ldexp(bamax, -t) / 6.0
+    s = torch.from_numpy(y.astype(np.float32)).to(torch.float8_e4m3fn).double().numpy()
+    s = np.where((bamax > 0) & (s == 0), 2.0 ** -9, s)
+    S = np.repeat(np.ldexp(s, t), block, axis=1)
+    q = np.where(S > 0, V / np.where(S > 0, S, 1.0), 0.0)
+    return np.where(counted, q_e2m1(q) * S, 0.0), t[:, 0]

@@ -6,7 +6,7 @@ import pytest
 
 import sdq_synth
 from oracle import sdq_oracle as so
-from tests.indep_definition import bf16_to_f64, decompose_dense, quantize_act_dense
+from tests.indep_definition import bf16_to_f64, decompose_dense, quantize_act_dense, two_level_quantize
 
 CFGS = [so.Config(1, so.GRAN_PAIR, 64, so.SCALE_OCP_FLOOR),
         so.Config(1, so.GRAN_ELEM, 32, so.SCALE_OCP_FLOOR),
@@ -412,3 +412,104 @@ def test_keep_8_of_8_is_the_dense_pattern_and_keep_less_only_removes_values():
         nz = so.dequant_weights(p)[0] != 0
         assert not (nz & ~prev).any()            # supports are nested as n shrinks
         prev = nz
+
+
+# ---------------------------------------------------------------- two-level scaling with fp8-e4m3 Q-Vector scales
+def _e4m3_values():
+    import torch
+    return torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).double().numpy()
+
+
+def test_ue4m3_scale_code_closed_forms():
+    """amax = 6 * v * 2^t returns the code of v for every positive e4m3 value; just above / below a midpoint goes to the
+    right neighbour, the midpoint itself to the even code; zero gives 0, anything tiny the smallest positive code"""
+    L = so.lib()
+    vals = _e4m3_values()
+    for t in (-20, 0, 7):
+        for c in range(1, 0x7F):
+            assert L.sdqo_ue4m3_scale_code(6.0 * vals[c] * 2.0 ** t, t) == c
+        for c in range(1, 0x7E):
+            mid = 3.0 * (vals[c] + vals[c + 1]) * 2.0 ** t
+            assert L.sdqo_ue4m3_scale_code(mid, t) == (c if c % 2 == 0 else c + 1)
+            assert L.sdqo_ue4m3_scale_code(mid * (1 + 2.0 ** -30), t) == c + 1
+            assert L.sdqo_ue4m3_scale_code(mid * (1 - 2.0 ** -30), t) == c
+    assert L.sdqo_ue4m3_scale_code(0.0, 3) == 0
+    assert L.sdqo_ue4m3_scale_code(1e-30, 0) == 1
+
+
+@pytest.mark.parametrize("gran,block,out_n", [(so.GRAN_PAIR, 32, 1), (so.GRAN_PAIR, 64, 2), (so.GRAN_ELEM, 32, 0), (so.GRAN_DENSE, 32, 1)])
+def test_ue4m3_weights_match_independent_definition(gran, block, out_n):
+    cfg = so.Config(out_n, gran, block, so.SCALE_UE4M3)
+    for seed in (0, 1):
+        Wb = tiny_W(48, 512, seed)
+        p = so.decompose(Wb, cfg)
+        W_in, W_out = so.dequant_weights(p)
+        pair = {so.GRAN_PAIR: True, so.GRAN_ELEM: False, so.GRAN_DENSE: None}[gran]
+        ref_in, ref_out, slots, mask_out = decompose_dense(Wb, out_n, pair, block, "ue4m3")
+        assert np.array_equal(W_out, ref_out)
+        assert np.array_equal(W_in, ref_in)
+        _, t = two_level_quantize(np.where(slots & ~mask_out, bf16_to_f64(Wb), 0.0), slots & ~mask_out, block)
+        assert np.array_equal(p.in_texp, t)
+        assert (p.in_scale <= 0x7E).all()
+        # the selections do not depend on the scale format
+        p0 = so.decompose(Wb, so.Config(out_n, gran, block, so.SCALE_OCP_FLOOR))
+        assert np.array_equal(p.in_meta, p0.in_meta) and np.array_equal(p.out_idx, p0.out_idx)
+        assert np.array_equal(p.out_code, p0.out_code)
+
+
+def test_ue4m3_scales_on_power_of_two_blocks_equal_the_ceil_rule():
+    """blocks whose largest kept magnitude is 6 * 2^j get the scale 2^j under both rules: identical W_in"""
+    rng = np.random.default_rng(31)
+    N, K = 16, 256
+    import torch
+    W = rng.choice([-1.0, 1.0], size=(N, K)) * rng.choice([0.5, 1.0, 1.5, 2.0, 3.0, 4.0], size=(N, K))
+    j = rng.integers(-4, 3, size=(N, K // 32))
+    W[:, ::32] = 6.0                                       # every block reaches 6 (kept: the pair (0,1) has the largest sum)
+    W[:, 1::32] = 4.0
+    W = W * np.repeat(2.0 ** j, 32, axis=1)
+    Wb = sdq_synth.bf16_bits(torch.from_numpy(W).to(torch.bfloat16))
+    a = so.dequant_weights(so.decompose(Wb, so.Config(0, so.GRAN_PAIR, 32, so.SCALE_UE4M3)))[0]
+    b = so.dequant_weights(so.decompose(Wb, so.Config(0, so.GRAN_PAIR, 32, so.SCALE_CEIL_NOSAT)))[0]
+    assert np.array_equal(a, b)
+    assert np.array_equal(a != 0, b != 0) and (np.abs(a).reshape(N, K // 32, 32).max(-1) == 6.0 * 2.0 ** j).all()
+
+
+def test_ue4m3_scales_lower_the_inlier_error():
+    """the quantization-stage observation restated on synthetic weights: e4m3 Q-Vector scales give a smaller inlier
+    error than power-of-two scales under either rule (same kept positions, same block)"""
+    Wb = tiny_W(128, 1024, 41)
+    W = bf16_to_f64(Wb)
+    errs = {}
+    for rule in (so.SCALE_OCP_FLOOR, so.SCALE_CEIL_NOSAT, so.SCALE_UE4M3):
+        p = so.decompose(Wb, so.Config(1, so.GRAN_PAIR, 32, rule))
+        W_in, W_out = so.dequant_weights(p)
+        kept = np.repeat(np.zeros_like(p.in_meta, bool), 8, axis=1)
+        j0, j1 = p.in_meta & 3, (p.in_meta >> 2) & 3
+        for u in range(2):
+            np.put_along_axis(kept.reshape(128, -1, 8), (2 * j0 + u)[..., None], True, axis=-1)
+            np.put_along_axis(kept.reshape(128, -1, 8), (2 * j1 + u)[..., None], True, axis=-1)
+        kept &= (W_out == 0)
+        errs[rule] = np.sqrt((((W - W_in) * kept) ** 2).sum())
+    assert errs[so.SCALE_UE4M3] < 0.9 * min(errs[so.SCALE_OCP_FLOOR], errs[so.SCALE_CEIL_NOSAT]), errs
+
+
+@pytest.mark.parametrize("block", [32, 64])
+def test_ue4m3_activations_match_independent_definition(block):
+    Xb = sdq_synth.bf16_bits(sdq_synth.make_act(24, 512, 5, n_outlier_channels=5))
+    Xb[3, :] = 0                                           # an all-zero token: factor 2^0, scale codes 0
+    Xb[5, 64:128] = 0                                      # all-zero Q-Vectors inside a live token
+    q = so.quantize_act(Xb, so.Config(1, so.GRAN_PAIR, block, so.SCALE_UE4M3))
+    A_i, A_o = so.dequant_act(q)
+    ref_i, ref_o = quantize_act_dense(Xb, block, "ue4m3")
+    assert np.array_equal(A_i, ref_i) and np.array_equal(A_o, ref_o)
+    assert (q.xq4_scale[3] == 0).all() and q.xq8_sexp[3] == 0 and (q.xq4_scale[5, 64 // block:128 // block] == 0).all()
+    # the 8-bit part does not depend on the 4-bit scale format
+    q0 = so.quantize_act(Xb, so.Config(1, so.GRAN_PAIR, block, so.SCALE_OCP_FLOOR))
+    assert np.array_equal(q.xq8_code, q0.xq8_code) and np.array_equal(q.xq8_sexp, q0.xq8_sexp)
+    # a Q-Vector 2^20 below the token's largest value still gets the smallest positive scale, not zero
+    import torch
+    X = torch.zeros((1, 256), dtype=torch.bfloat16)
+    X[0, 0] = 256.0
+    X[0, 40] = 2.0 ** -12
+    q1 = so.quantize_act(sdq_synth.bf16_bits(X), so.Config(1, so.GRAN_PAIR, 32, so.SCALE_UE4M3))
+    assert q1.xq8_sexp[0] == 0 and q1.xq4_scale[0, 1] == 1 and q1.xq4_scale[0, 0] == so.lib().sdqo_ue4m3_scale_code(256.0, 0)

@@ -20,7 +20,8 @@ def make(M, N, K, seed, cfg=CFG):
 
 @pytest.mark.parametrize("cfg", [CFG, so.Config(2, so.GRAN_ELEM, 32, so.SCALE_CEIL_NOSAT), so.Config(0, so.GRAN_PAIR, 64, 0),
                                  so.Config(1, so.GRAN_DENSE, 32, so.SCALE_OCP_FLOOR),
-                                 so.Config(1, so.gran_keep(7), 32, so.SCALE_OCP_FLOOR)])
+                                 so.Config(1, so.gran_keep(7), 32, so.SCALE_OCP_FLOOR),
+                                 so.Config(1, so.GRAN_PAIR, 32, so.SCALE_UE4M3)])
 def test_brute_force_triple_loop(cfg):
     Wb, Xb, p, q = make(3, 16, 128, 2, cfg)
     W_in, W_out = so.dequant_weights(p)
@@ -68,6 +69,14 @@ def test_dense_inliers_match_independent_definition_end_to_end():
     err_dense = np.linalg.norm(so.linear(q, p) - X @ W.T)
     err_pruned = np.linalg.norm(so.linear(so.quantize_act(Xb, cfg_p), so.decompose(Wb, cfg_p)) - X @ W.T)
     assert err_dense < err_pruned
+
+
+def test_ue4m3_scales_match_independent_definition_end_to_end():
+    cfg = so.Config(1, so.GRAN_PAIR, 32, so.SCALE_UE4M3)
+    Wb, Xb, p, q = make(8, 64, 256, 11, cfg)
+    Win, Wout, _, _ = decompose_dense(Wb, 1, True, 32, "ue4m3")
+    Ai, Ao = quantize_act_dense(Xb, 32, "ue4m3")
+    assert np.allclose(so.linear(q, p), Ai @ Win.T + Ao @ Wout.T, rtol=1e-12, atol=1e-12)
 
 
 def test_one_hot_readback_returns_columns_of_W_in_plus_W_out():
