@@ -40,7 +40,7 @@ typedef enum {
 
 enum { SDQ_GRAN_PAIR = 0, SDQ_GRAN_ELEM = 1, SDQ_GRAN_DENSE = 2 }; /* inlier pattern            */
 #define SDQ_GRAN_KEEP(n) (2 + (8 - (n)))  /* n:8 sparsification, n = 2..8; SDQ_GRAN_KEEP(8) == SDQ_GRAN_DENSE */
-enum { SDQ_SCALE_OCP_FLOOR = 0, SDQ_SCALE_CEIL_NOSAT = 1 }; /* E8M0 Q-Vector scale rule        */
+enum { SDQ_SCALE_OCP_FLOOR = 0, SDQ_SCALE_CEIL_NOSAT = 1, SDQ_SCALE_UE4M3 = 2 }; /* Q-Vector scale rule */
 
 /* "pattern, formats" of the decomposition (Section 5, Stages 1-3).
  *   out_n      outliers extracted per S-Vector of 8 consecutive K (Stage 2): 0, 1 or 2; stored as
@@ -62,7 +62,15 @@ enum { SDQ_SCALE_OCP_FLOOR = 0, SDQ_SCALE_CEIL_NOSAT = 1 }; /* E8M0 Q-Vector sca
  *              activations: 64 or 32.  Both are executed by sdq_linear (64: kind::mxf4 .block32, the
  *              faster kernel; 32: kind::mxf4nvf4 .block16 with E8M0 scale codes).
  *   scale_rule E8M0 exponent from the Q-Vector's largest magnitude a: OCP_FLOOR = floor(log2 a) - 2,
- *              CEIL_NOSAT = smallest E with a <= 6 * 2^E.
+ *              CEIL_NOSAT = smallest E with a <= 6 * 2^E.  SDQ_SCALE_UE4M3 (the quantization-stage study's
+ *              preferred scale-factor format, fp8-e4m3): two-level scaling -- a vector (the kept inliers
+ *              of a weight row; a token) has a power-of-two factor 2^t, t = smallest integer with its
+ *              largest magnitude <= 448 * 2^t (for a token: the exponent of its 8-bit scale); a Q-Vector's
+ *              scale code is the unsigned E4M3 value nearest to a / (6 * 2^t) (ties to even, at least the
+ *              smallest positive one unless a = 0); an element is the E2M1 value nearest to x / (scale *
+ *              2^t).  Requires in_gran = SDQ_GRAN_PAIR and in_block = 32 (kind::mxf4nvf4 .block16 with
+ *              UE4M3 scale codes), else every call returns SDQ_ERR_UNSUPPORTED; rows or tokens whose largest
+ *              magnitude is below 2^-100 are outside its range.
  */
 typedef struct {
   int32_t out_n;
@@ -74,7 +82,8 @@ typedef struct {
 /* Host-side descriptor of a packed weight matrix (filled by sdq_decompose; plain data, may be
  * copied; `dev` stays owned by the caller).  off[] are byte offsets of the sections inside dev:
  *   0 inlier stages  1 outlier stages (tensor-core 2:4 form)  2 outlier row-scale atoms
- *   3 compact outlier codes  4 compact outlier indices  5 outlier scale exponents  6,7 reserved */
+ *   3 compact outlier codes  4 compact outlier indices  5 outlier scale exponents
+ *   6 inlier row-factor exponents (SDQ_SCALE_UE4M3; zeros otherwise)  7 reserved */
 typedef struct {
   void* dev;
   size_t bytes;
@@ -105,11 +114,13 @@ typedef struct {
   uint8_t* out_code;  /* [N][K/8][out_n] E4M3 codes                                               */
   uint8_t* out_idx;   /* [N][K/8][out_n] position 0..7 in the S-Vector, ascending                 */
   int32_t* out_sexp;  /* [N] exponent e of the row scale 2^e                                      */
+  int32_t* in_texp;   /* [N] SDQ_SCALE_UE4M3: exponent t of the row's inlier factor 2^t (in_scale then
+                         holds unsigned E4M3 codes); zeros otherwise; may be NULL                  */
 } sdq_canonical_t;
 
 typedef struct {
   uint8_t* xq4_code;  /* [M][K] E2M1 codes           */
-  uint8_t* xq4_scale; /* [M][K/in_block] E8M0 codes  */
+  uint8_t* xq4_scale; /* [M][K/in_block] E8M0 codes (SDQ_SCALE_UE4M3: unsigned E4M3 codes, times 2^xq8_sexp[m]) */
   uint8_t* xq8_code;  /* [M][K] E4M3 codes           */
   int32_t* xq8_sexp;  /* [M] exponent e of the per-token scale 2^e */
 } sdq_act_canonical_t;

@@ -23,7 +23,7 @@ def gran_keep(n: int) -> int:
     positions); stored and executed like the dense pattern.  gran_keep(8) == GRAN_DENSE."""
     assert 2 <= n <= 8
     return 2 + (8 - n)
-SCALE_OCP_FLOOR, SCALE_CEIL_NOSAT = 0, 1
+SCALE_OCP_FLOOR, SCALE_CEIL_NOSAT, SCALE_UE4M3 = 0, 1, 2
 
 STATUS = ["ok", "invalid_arg", "shape", "alignment", "unsupported", "buffer_too_small", "nonfinite", "cuda", "timeout"]
 
@@ -54,7 +54,7 @@ class _Act(ctypes.Structure):
 
 
 class _Canon(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_void_p) for n in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp")]
+    _fields_ = [(n, ctypes.c_void_p) for n in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp", "in_texp")]
 
 
 class _ActCanon(ctypes.Structure):
@@ -251,8 +251,9 @@ def packed_export(p: PackedWeight) -> dict:
              in_scale=torch.zeros((N, K // p.cfg.in_block), dtype=torch.uint8, device=dev),
              out_code=torch.zeros((N, K // 8, max(on, 1)), dtype=torch.uint8, device=dev),
              out_idx=torch.zeros((N, K // 8, max(on, 1)), dtype=torch.uint8, device=dev),
-             out_sexp=torch.zeros((N,), dtype=torch.int32, device=dev))
-    c = _Canon(*[t[n].data_ptr() for n in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp")])
+             out_sexp=torch.zeros((N,), dtype=torch.int32, device=dev),
+             in_texp=torch.zeros((N,), dtype=torch.int32, device=dev))
+    c = _Canon(*[t[n].data_ptr() for n in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp", "in_texp")])
     _check(lib().sdq_packed_export(ctypes.byref(p.desc), ctypes.byref(c), _stream()), "sdq_packed_export")
     if on == 0:
         t["out_code"] = t["out_code"][:, :, :0]

@@ -46,6 +46,20 @@ __device__ __forceinline__ int fp8_scale_exp(float amax) {
 __device__ __forceinline__ float pow2_inv_e8m0(uint32_t c) { return __uint_as_float((254u - c) << 23); }
 __device__ __forceinline__ float pow2_neg(int e) { return __uint_as_float((uint32_t)(127 - e) << 23); }
 
+// Two-level scaling (SDQ_SCALE_UE4M3): unsigned E4M3 code of the Q-Vector scale nearest to amax / (6 * 2^t), at least
+// the smallest positive code unless amax == 0, and the value scale * 2^t the elements are divided by (0 for code 0).
+// amax * 2^-t is exact (amax <= 448 * 2^t); the one rounding of the division is far from every E4M3 midpoint or
+// lands on it exactly, so the converter's round-to-nearest-even is that of the exact quotient.
+__device__ __forceinline__ uint32_t ue4m3_scale_code(float amax, int t) {
+  if (amax == 0.0f) return 0u;
+  const uint32_t c = (uint32_t)__nv_cvt_float_to_fp8(__fdiv_rn(scalbnf(amax, -t), 6.0f), __NV_SATFINITE, __NV_E4M3);
+  return c == 0u ? 1u : c;
+}
+__device__ __forceinline__ float ue4m3_scale_value(uint32_t c, int t) {
+  const __half_raw h = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)c, __NV_E4M3);
+  return scalbnf(__half2float(__half(h)), t);
+}
+
 // two floats -> two E2M1 codes in one byte (x in the low nibble)
 __device__ __forceinline__ uint32_t e2m1x2(float x, float y) {
   return (uint32_t)__nv_cvt_float2_to_fp4x2(make_float2(x, y), __NV_E2M1, cudaRoundNearest);

@@ -23,7 +23,8 @@
 //            embedding of the 1:8 / 2:8 outliers), same addressing as A_in
 //     E_out: 128 rows x 16 B  (one 4-bit index pair per 4 logical K over 128 K)
 //   section SFA_out[rt]: 512 B, the per-row outlier scale as an E8M0 code, scale-atom form, 4 copies
-//   sections compact outlier codes / indices [N][K/8][out_n] u8 and row scale exponents [N] i32
+//   sections compact outlier codes / indices [N][K/8][out_n] u8, row scale exponents [N] i32, inlier row-factor
+//   exponents [N] i32 (two-level scaling with E4M3 Q-Vector scales; zeros otherwise)
 //
 // Activation buffer (per 128-token tile mt)
 //   section XI[mt][k2] = | B4 16384 | SFB_in 512 |            (one scale per 32 K: SFB_in 2 x 512, as for the weights)
@@ -83,7 +84,7 @@ __host__ __device__ inline uint32_t sf_off(uint32_t row, uint32_t s) { return (r
 constexpr size_t HEADER_BYTES = 256;
 
 struct PackedOffsets {
-  size_t wi, wo, sfa_out, ocode, oidx, osexp, total;
+  size_t wi, wo, sfa_out, ocode, oidx, osexp, wtexp, total;
 };
 inline PackedOffsets packed_offsets(int64_t N, int64_t K, int out_n, bool b32 = false, bool dense = false) {
   PackedOffsets o;
@@ -95,7 +96,8 @@ inline PackedOffsets packed_offsets(int64_t N, int64_t K, int out_n, bool b32 = 
   o.ocode = al(o.sfa_out + RT * SF_ATOM_BYTES);
   o.oidx = al(o.ocode + (size_t)N * (size_t)(K / 8) * (size_t)out_n);
   o.osexp = al(o.oidx + (size_t)N * (size_t)(K / 8) * (size_t)out_n);
-  o.total = al(o.osexp + (size_t)N * 4);
+  o.wtexp = al(o.osexp + (size_t)N * 4);                          // inlier row-factor exponents [N] i32 (two-level scaling)
+  o.total = al(o.wtexp + (size_t)N * 4);
   return o;
 }
 

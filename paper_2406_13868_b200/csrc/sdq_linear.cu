@@ -672,6 +672,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   if (Xq->K != P->K || Xq->M <= 0 || P->N <= 0 || P->N % TILE_ROWS || P->K % K2 || ldy < P->N) return SDQ_ERR_SHAPE;
   if (Xq->cfg.in_block != P->cfg.in_block || Xq->cfg.scale_rule != P->cfg.scale_rule) return SDQ_ERR_SHAPE;
   if (P->cfg.in_gran != SDQ_GRAN_PAIR && !(P->cfg.in_gran >= SDQ_GRAN_DENSE && P->cfg.in_block == 32)) return SDQ_ERR_UNSUPPORTED;
+  if (P->cfg.scale_rule == SDQ_SCALE_UE4M3) return SDQ_ERR_UNSUPPORTED;
   if (((uintptr_t)Y & 15) || (ldy % 8) || ((uintptr_t)ws & 15)) return SDQ_ERR_ALIGNMENT;
   static bool attr_set = false;
   if (!attr_set) {

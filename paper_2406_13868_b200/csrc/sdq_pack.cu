@@ -49,6 +49,30 @@ __device__ __forceinline__ void load_group(const __nv_bfloat16* w, uint32_t (&bi
   }
 }
 
+// Stage 1, pair-wise 4:8: the 2 pairs (of 4) with the largest summed significance among the non-outliers (one fp32 add
+// per pair, largest first, ties to the lower index), ascending
+__device__ __forceinline__ void select_pairs(const uint32_t (&key)[8], const uint32_t (&skey)[8], bool weighted, int o0, int o1,
+                                             int& j0, int& j1) {
+  float score[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float a0 = (2 * j == o0 || 2 * j == o1) ? 0.0f : key_value(key[2 * j], skey[2 * j], weighted);
+    const float a1 = (2 * j + 1 == o0 || 2 * j + 1 == o1) ? 0.0f : key_value(key[2 * j + 1], skey[2 * j + 1], weighted);
+    score[j] = __fadd_rn(a0, a1);
+  }
+  j0 = 0;
+#pragma unroll
+  for (int j = 1; j < 4; ++j)
+    if (score[j] > score[j0]) j0 = j;
+  j1 = -1;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (j == j0) continue;
+    if (j1 < 0 || score[j] > score[j1]) j1 = j;
+  }
+  if (j0 > j1) { int t = j0; j0 = j1; j1 = t; }
+}
+
 __global__ void __launch_bounds__(128)
 pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t ldw, sdq_config_t cfg, const float* __restrict__ colw,
             uint8_t* __restrict__ blob, PackedOffsets off, uint32_t* __restrict__ flags)
@@ -58,11 +82,12 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
   const int G = (int)(K / 8);
   const int out_n = cfg.out_n;
   const __nv_bfloat16* wrow = W + n * ldw;
-  __shared__ uint32_t s_red[4];
-  __shared__ int s_e;
+  __shared__ uint32_t s_red[4], s_red_in[4];
+  __shared__ int s_e, s_t;
+  const bool ue = cfg.scale_rule == SDQ_SCALE_UE4M3;     // two-level scaling with E4M3 Q-Vector scales (pair-wise, block 32)
 
-  // ---- pass 1: largest outlier magnitude of the row, non-finite check
-  uint32_t okey_max = 0, bad = 0;
+  // ---- pass 1: largest outlier magnitude of the row (and, for two-level scaling, largest kept inlier), non-finite check
+  uint32_t okey_max = 0, ikey_max = 0, bad = 0;
   for (int g = tid; g < G; g += 128) {
     uint32_t bits[8], key[8];
     load_group(wrow + 8 * g, bits);
@@ -77,21 +102,32 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     select_outliers(skey, out_n, o0, o1);
     if (o0 >= 0) okey_max = max(okey_max, key[o0]);
     if (o1 >= 0) okey_max = max(okey_max, key[o1]);
+    if (ue) {
+      int j0, j1;
+      select_pairs(key, skey, colw != nullptr, o0, o1, j0, j1);
+      const int pos[4] = {2 * j0, 2 * j0 + 1, 2 * j1, 2 * j1 + 1};
+#pragma unroll
+      for (int s = 0; s < 4; ++s)
+        if (pos[s] != o0 && pos[s] != o1) ikey_max = max(ikey_max, key[pos[s]]);
+    }
   }
 #pragma unroll
   for (int s = 16; s > 0; s >>= 1) {
     okey_max = max(okey_max, __shfl_xor_sync(0xffffffffu, okey_max, s));
+    ikey_max = max(ikey_max, __shfl_xor_sync(0xffffffffu, ikey_max, s));
     bad |= __shfl_xor_sync(0xffffffffu, bad, s);
   }
-  if ((tid & 31) == 0) s_red[tid >> 5] = okey_max;
+  if ((tid & 31) == 0) { s_red[tid >> 5] = okey_max; s_red_in[tid >> 5] = ikey_max; }
   if (bad && (tid & 31) == 0) atomicOr(&flags[FLAG_NONFINITE], 1u);
   __syncthreads();
   if (tid == 0) {
     uint32_t m = max(max(s_red[0], s_red[1]), max(s_red[2], s_red[3]));
     s_e = fp8_scale_exp(bf16_bits_to_float(m));
+    const uint32_t mi = max(max(s_red_in[0], s_red_in[1]), max(s_red_in[2], s_red_in[3]));
+    s_t = ue ? fp8_scale_exp(bf16_bits_to_float(mi)) : 0;   // exponent of the row's inlier factor 2^t
   }
   __syncthreads();
-  const int e = s_e;
+  const int e = s_e, tw = s_t;
 
   const int64_t rt = n / TILE_ROWS;
   const uint32_t r = (uint32_t)(n % TILE_ROWS);
@@ -104,7 +140,10 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
 
   if (tid == 0) {
     reinterpret_cast<int32_t*>(blob + off.osexp)[n] = e;
-    const uint32_t c = (uint32_t)(e + 127);
+    reinterpret_cast<int32_t*>(blob + off.wtexp)[n] = tw;
+    // the accumulator of a row is kept in units of 2^tw (the inlier scale codes leave that factor out), so the outlier
+    // row scale is 2^(e - tw); the GEMM's epilogue multiplies the factor back in
+    const uint32_t c = (uint32_t)min(max(e - tw + 127, 0), 254);
     *reinterpret_cast<uint32_t*>(blob + off.sfa_out + (size_t)rt * SF_ATOM_BYTES + sf_off(r, 0)) = c * 0x01010101u;
   }
 
@@ -152,24 +191,8 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
       if ((g & 3) == 0) wi[a_in_bytes(true) + in_sf_off(true, r, (uint32_t)((g >> 2) & 7))] = (uint8_t)c;
     } else {
     // Stage 1 on the remaining values: keep the 2 pairs (of 4) with the largest summed significance
-    float score[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float a0 = (2 * j == o0 || 2 * j == o1) ? 0.0f : key_value(key[2 * j], skey[2 * j], colw != nullptr);
-      const float a1 = (2 * j + 1 == o0 || 2 * j + 1 == o1) ? 0.0f : key_value(key[2 * j + 1], skey[2 * j + 1], colw != nullptr);
-      score[j] = __fadd_rn(a0, a1);
-    }
-    int j0 = 0;
-#pragma unroll
-    for (int j = 1; j < 4; ++j)
-      if (score[j] > score[j0]) j0 = j;
-    int j1 = -1;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (j == j0) continue;
-      if (j1 < 0 || score[j] > score[j1]) j1 = j;
-    }
-    if (j0 > j1) { int t = j0; j0 = j1; j1 = t; }
+    int j0, j1;
+    select_pairs(key, skey, colw != nullptr, o0, o1, j0, j1);
     const int slot_pos[4] = {2 * j0, 2 * j0 + 1, 2 * j1, 2 * j1 + 1};
 
     // Stage 3, inliers: Q-Vector (64 K = 8 S-Vectors = 8 lanes, or 32 K = 4 lanes) largest kept magnitude -> E8M0 scale
@@ -182,12 +205,14 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 1));
     ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 2));
     if (!b32) ikey = max(ikey, __shfl_xor_sync(0xffffffffu, ikey, 4));
-    const uint32_t c = e8m0_scale_code(bf16_bits_to_float(ikey), cfg.scale_rule);
+    const uint32_t c = ue ? ue4m3_scale_code(bf16_bits_to_float(ikey), tw) : e8m0_scale_code(bf16_bits_to_float(ikey), cfg.scale_rule);
+    const float sv = ue ? ue4m3_scale_value(c, tw) : 0.0f;
     float v[4];
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
       const int p = slot_pos[s];
-      v[s] = (p == o0 || p == o1) ? 0.0f : bf16_bits_to_float(bits[p]) * pow2_inv_e8m0(c);
+      const float w = bf16_bits_to_float(bits[p]);
+      v[s] = (p == o0 || p == o1) ? 0.0f : (ue ? (c ? __fdiv_rn(w, sv) : 0.0f) : w * pow2_inv_e8m0(c));
     }
     const uint32_t codes = e2m1x2(v[0], v[1]) | (e2m1x2(v[2], v[3]) << 8);
 
@@ -272,7 +297,10 @@ export_packed_kernel(const uint8_t* __restrict__ blob, int64_t N, int64_t K, sdq
       out.out_idx[((size_t)n * G + g) * out_n + t] = blob[off.oidx + ((size_t)n * G + g) * out_n + t];
     }
   }
-  if (threadIdx.x == 0) out.out_sexp[n] = reinterpret_cast<const int32_t*>(blob + off.osexp)[n];
+  if (threadIdx.x == 0) {
+    out.out_sexp[n] = reinterpret_cast<const int32_t*>(blob + off.osexp)[n];
+    if (out.in_texp) out.in_texp[n] = reinterpret_cast<const int32_t*>(blob + off.wtexp)[n];
+  }
 }
 
 }  // namespace sdq
@@ -282,13 +310,18 @@ using namespace sdq;
 static bool cfg_ok(const sdq_config_t* c) {
   return c && c->out_n >= 0 && c->out_n <= 2 && c->in_gran >= 0 && c->in_gran <= SDQ_GRAN_KEEP(2) &&
          (c->in_gran < SDQ_GRAN_DENSE || 10 - c->in_gran > c->out_n) &&
-         (c->in_block == 32 || c->in_block == 64) && (c->scale_rule == SDQ_SCALE_OCP_FLOOR || c->scale_rule == SDQ_SCALE_CEIL_NOSAT);
+         (c->in_block == 32 || c->in_block == 64) && c->scale_rule >= SDQ_SCALE_OCP_FLOOR && c->scale_rule <= SDQ_SCALE_UE4M3;
+}
+// valid configurations this kernel set does not carry out
+static bool cfg_unsupported(const sdq_config_t* c) {
+  return (c->in_gran >= SDQ_GRAN_DENSE && c->in_block != 32) ||
+         (c->scale_rule == SDQ_SCALE_UE4M3 && !(c->in_gran == SDQ_GRAN_PAIR && c->in_block == 32));
 }
 
 extern "C" sdq_status_t sdq_packed_size(int64_t N, int64_t K, const sdq_config_t* cfg, size_t* bytes, size_t* algorithmic_bytes)
 {
   if (!cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
-  if (cfg->in_gran >= SDQ_GRAN_DENSE && cfg->in_block != 32) return SDQ_ERR_UNSUPPORTED;
+  if (cfg_unsupported(cfg)) return SDQ_ERR_UNSUPPORTED;
   if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2) return SDQ_ERR_SHAPE;
   if (bytes) *bytes = is_tensor_core_reading(*cfg) ? packed_offsets(N, K, cfg->out_n, cfg->in_block == 32, cfg->in_gran >= SDQ_GRAN_DENSE).total : plain_packed_offsets(N, K, *cfg).total;
   if (algorithmic_bytes) {
@@ -312,7 +345,7 @@ extern "C" sdq_status_t sdq_decompose_metric(const void* W, int64_t N, int64_t K
                                              void* stream)
 {
   if (!W || !packed_buf || !out || !cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
-  if (cfg->in_gran >= SDQ_GRAN_DENSE && cfg->in_block != 32) return SDQ_ERR_UNSUPPORTED;
+  if (cfg_unsupported(cfg)) return SDQ_ERR_UNSUPPORTED;
   if ((uintptr_t)col_weight & 15) return SDQ_ERR_ALIGNMENT;
   if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2 || ldw < K) return SDQ_ERR_SHAPE;
   if (((uintptr_t)W & 15) || ((uintptr_t)packed_buf & 15) || (ldw % 8)) return SDQ_ERR_ALIGNMENT;
@@ -338,7 +371,7 @@ extern "C" sdq_status_t sdq_decompose_metric(const void* W, int64_t N, int64_t K
   for (int i = 0; i < 8; ++i) out->off[i] = 0;
   if (tc) {
     out->off[0] = off.wi; out->off[1] = off.wo; out->off[2] = off.sfa_out;
-    out->off[3] = off.ocode; out->off[4] = off.oidx; out->off[5] = off.osexp;
+    out->off[3] = off.ocode; out->off[4] = off.oidx; out->off[5] = off.osexp; out->off[6] = off.wtexp;
   } else {
     out->off[0] = poff.in_code; out->off[1] = poff.in_meta; out->off[2] = poff.in_scale;
     out->off[3] = poff.out_code; out->off[4] = poff.out_idx; out->off[5] = poff.osexp;

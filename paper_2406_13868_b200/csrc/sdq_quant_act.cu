@@ -68,6 +68,7 @@ act_amax_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int64
   }
 }
 
+template <bool UE>                                      // UE: two-level scaling with E4M3 Q-Vector scales
 __global__ void __launch_bounds__(QA_THREADS)
 quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int64_t ldx, sdq_config_t cfg, uint8_t* __restrict__ buf,
                  ActOffsets off, const float* __restrict__ partial, int n_chunks)
@@ -94,12 +95,15 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
   const uint32_t tk = (uint32_t)(m % TILE_TOK);
   const int T1 = (int)(K / K1), T2 = (int)(K / K2);
   const bool b32 = cfg.in_block == 32;               // one scale per 32 K: a Q-Vector is a lane pair
+  constexpr bool ue = UE;
   const int xib = xi_bytes(b32);
   uint8_t* xi_base = buf + off.xi + (size_t)mt * T2 * xib;
   uint8_t* xo_base = buf + off.xo + (size_t)mt * T1 * XO_BYTES;
   if (live && blockIdx.y == 0 && warp == 0 && l == 0) {
     reinterpret_cast<int32_t*>(buf + off.sexp)[m] = e;
-    *reinterpret_cast<uint32_t*>(buf + off.sfb_out + (size_t)mt * SF_ATOM_BYTES + sf_off(tk, 0)) = (uint32_t)(e + 127) * 0x01010101u;
+    // two-level scaling keeps a token's accumulator column in units of 2^e (the 4-bit scale codes leave that factor out):
+    // the 8-bit product then takes the scale 1 here and the GEMM's epilogue multiplies 2^e back in
+    *reinterpret_cast<uint32_t*>(buf + off.sfb_out + (size_t)mt * SF_ATOM_BYTES + sf_off(tk, 0)) = (uint32_t)(ue ? 127 : e + 127) * 0x01010101u;
   }
 
 #pragma unroll
@@ -120,14 +124,20 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
     }
     bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
     if (!b32) bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
-    const uint32_t c = e8m0_scale_code(bmax, cfg.scale_rule);
+    const uint32_t c = ue ? ue4m3_scale_code(bmax, e) : e8m0_scale_code(bmax, cfg.scale_rule);
     uint32_t q4[2] = {0, 0}, q8[4] = {0, 0, 0, 0};
-    const float s4 = pow2_inv_e8m0(c);
+    if (!ue) {
+      const float s4 = pow2_inv_e8m0(c);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      q4[j >> 2] |= e2m1x2(v[2 * j] * s4, v[2 * j + 1] * s4) << (8 * (j & 3));
-      q8[j >> 1] |= e4m3x2(v[2 * j] * s8, v[2 * j + 1] * s8) << (16 * (j & 1));
+      for (int j = 0; j < 8; ++j) q4[j >> 2] |= e2m1x2(v[2 * j] * s4, v[2 * j + 1] * s4) << (8 * (j & 3));
+    } else if (c) {
+      // two-level scaling: the Q-Vector scale E4M3(c) * 2^e is not a power of two, the elements are divided by it
+      const float sv = ue4m3_scale_value(c, e);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) q4[j >> 2] |= e2m1x2(__fdiv_rn(v[2 * j], sv), __fdiv_rn(v[2 * j + 1], sv)) << (8 * (j & 3));
     }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) q8[j >> 1] |= e4m3x2(v[2 * j] * s8, v[2 * j + 1] * s8) << (16 * (j & 1));
     if (!live) continue;
     const uint32_t k = (uint32_t)b * 64 + l * 16;          // first element of this lane
     uint8_t* xi = xi_base + (size_t)(k >> 8) * xib;
@@ -144,8 +154,8 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
 // memory, and the codes are produced from the registers.  Same arithmetic as the two-kernel path, which stays for
 // rows too long for the register budget (K > 64 * QA_WARPS * QF_MAX_IT * 8 = 16384) and for the block-32 reading.
 constexpr int QF_MAX_IT = 4;                             // Q-Vectors per warp
-template <int IT>
-__global__ void __launch_bounds__(QA_THREADS, 4)
+template <int IT, bool UE>
+__global__ void __launch_bounds__(QA_THREADS, UE ? 3 : 4)
 quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int64_t ldx, sdq_config_t cfg, uint8_t* __restrict__ buf,
                        ActOffsets off)
 {
@@ -215,12 +225,15 @@ quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K
   const uint32_t tk = (uint32_t)(m % TILE_TOK);
   const int T1 = (int)(K / K1), T2 = (int)(K / K2);
   const bool b32 = cfg.in_block == 32;               // one scale per 32 K: a Q-Vector is a lane pair
+  constexpr bool ue = UE;
   const int xib = xi_bytes(b32);
   uint8_t* xi_base = buf + off.xi + (size_t)mt * T2 * xib;
   uint8_t* xo_base = buf + off.xo + (size_t)mt * T1 * XO_BYTES;
   if (live && rank == 0 && warp == 0 && l == 0) {
     reinterpret_cast<int32_t*>(buf + off.sexp)[m] = e;
-    *reinterpret_cast<uint32_t*>(buf + off.sfb_out + (size_t)mt * SF_ATOM_BYTES + sf_off(tk, 0)) = (uint32_t)(e + 127) * 0x01010101u;
+    // two-level scaling keeps a token's accumulator column in units of 2^e (the 4-bit scale codes leave that factor out):
+    // the 8-bit product then takes the scale 1 here and the GEMM's epilogue multiplies 2^e back in
+    *reinterpret_cast<uint32_t*>(buf + off.sfb_out + (size_t)mt * SF_ATOM_BYTES + sf_off(tk, 0)) = (uint32_t)(ue ? 127 : e + 127) * 0x01010101u;
   }
 #pragma unroll
   for (int i = 0; i < IT; ++i) {
@@ -241,14 +254,20 @@ quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K
     bm = max(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
     if (!b32) bm = max(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
     const float bmax = __uint_as_float(bm << 16);
-    const uint32_t c = e8m0_scale_code(bmax, cfg.scale_rule);
+    const uint32_t c = ue ? ue4m3_scale_code(bmax, e) : e8m0_scale_code(bmax, cfg.scale_rule);
     uint32_t q4[2] = {0, 0}, q8[4] = {0, 0, 0, 0};
-    const float s4 = pow2_inv_e8m0(c);
+    if (!ue) {
+      const float s4 = pow2_inv_e8m0(c);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      q4[j >> 2] |= e2m1x2(v[2 * j] * s4, v[2 * j + 1] * s4) << (8 * (j & 3));
-      q8[j >> 1] |= e4m3x2(v[2 * j] * s8, v[2 * j + 1] * s8) << (16 * (j & 1));
+      for (int j = 0; j < 8; ++j) q4[j >> 2] |= e2m1x2(v[2 * j] * s4, v[2 * j + 1] * s4) << (8 * (j & 3));
+    } else if (c) {
+      // two-level scaling: the Q-Vector scale E4M3(c) * 2^e is not a power of two, the elements are divided by it
+      const float sv = ue4m3_scale_value(c, e);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) q4[j >> 2] |= e2m1x2(__fdiv_rn(v[2 * j], sv), __fdiv_rn(v[2 * j + 1], sv)) << (8 * (j & 3));
     }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) q8[j >> 1] |= e4m3x2(v[2 * j] * s8, v[2 * j + 1] * s8) << (16 * (j & 1));
     if (!live) continue;
     const uint32_t k = (uint32_t)b * 64 + l * 16;          // first element of this lane
     uint8_t* xi = xi_base + (size_t)(k >> 8) * xib;
@@ -289,12 +308,13 @@ using namespace sdq;
 
 static bool act_cfg_ok(const sdq_config_t* c) {
   return c && c->out_n >= 0 && c->out_n <= 2 && (c->in_block == 32 || c->in_block == 64) &&
-         (c->scale_rule == SDQ_SCALE_OCP_FLOOR || c->scale_rule == SDQ_SCALE_CEIL_NOSAT);
+         c->scale_rule >= SDQ_SCALE_OCP_FLOOR && c->scale_rule <= SDQ_SCALE_UE4M3;
 }
 
 extern "C" sdq_status_t sdq_act_size(int64_t M, int64_t K, const sdq_config_t* cfg, size_t* bytes)
 {
   if (!act_cfg_ok(cfg) || !bytes) return SDQ_ERR_INVALID_ARG;
+  if (cfg->scale_rule == SDQ_SCALE_UE4M3 && cfg->in_block != 32) return SDQ_ERR_UNSUPPORTED;
   if (M <= 0 || K <= 0 || K % K2) return SDQ_ERR_SHAPE;
   *bytes = act_offsets(M, K, cfg->in_block == 32).total;
   return SDQ_OK;
@@ -304,6 +324,7 @@ extern "C" sdq_status_t sdq_quantize_act(const void* X, int64_t M, int64_t K, in
                                          size_t xq_bytes, sdq_act_t* out, void* stream)
 {
   if (!X || !xq_buf || !out || !act_cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
+  if (cfg->scale_rule == SDQ_SCALE_UE4M3 && cfg->in_block != 32) return SDQ_ERR_UNSUPPORTED;
   if (M <= 0 || K <= 0 || K % K2 || ldx < K) return SDQ_ERR_SHAPE;
   if (((uintptr_t)X & 15) || ((uintptr_t)xq_buf & 15) || (ldx % 8)) return SDQ_ERR_ALIGNMENT;
   const bool b32 = cfg->in_block == 32;
@@ -333,16 +354,28 @@ extern "C" sdq_status_t sdq_quantize_act(const void* X, int64_t M, int64_t K, in
     const __nv_bfloat16* Xb = (const __nv_bfloat16*)X;
     uint8_t* bufp = (uint8_t*)xq_buf;
     cudaError_t le;
-    switch (it) {
-      case 1: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<1>, Xb, M, K, ldx, *cfg, bufp, off); break;
-      case 2: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<2>, Xb, M, K, ldx, *cfg, bufp, off); break;
-      case 3: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<3>, Xb, M, K, ldx, *cfg, bufp, off); break;
-      default: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<4>, Xb, M, K, ldx, *cfg, bufp, off); break;
+    if (cfg->scale_rule == SDQ_SCALE_UE4M3) {
+      switch (it) {
+        case 1: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<1, true>, Xb, M, K, ldx, *cfg, bufp, off); break;
+        case 2: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<2, true>, Xb, M, K, ldx, *cfg, bufp, off); break;
+        case 3: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<3, true>, Xb, M, K, ldx, *cfg, bufp, off); break;
+        default: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<4, true>, Xb, M, K, ldx, *cfg, bufp, off); break;
+      }
+    } else {
+      switch (it) {
+        case 1: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<1, false>, Xb, M, K, ldx, *cfg, bufp, off); break;
+        case 2: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<2, false>, Xb, M, K, ldx, *cfg, bufp, off); break;
+        case 3: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<3, false>, Xb, M, K, ldx, *cfg, bufp, off); break;
+        default: le = cudaLaunchKernelEx(&lc, quant_act_fused_kernel<4, false>, Xb, M, K, ldx, *cfg, bufp, off); break;
+      }
     }
     if (le != cudaSuccess || cudaGetLastError() != cudaSuccess) return SDQ_ERR_CUDA;
   } else {
   act_amax_kernel<<<grid, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, partial, n_chunks);
-  quant_act_kernel<<<grid, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, *cfg, (uint8_t*)xq_buf, off, partial, n_chunks);
+  if (cfg->scale_rule == SDQ_SCALE_UE4M3)
+    quant_act_kernel<true><<<grid, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, *cfg, (uint8_t*)xq_buf, off, partial, n_chunks);
+  else
+    quant_act_kernel<false><<<grid, QA_THREADS, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, M, K, ldx, *cfg, (uint8_t*)xq_buf, off, partial, n_chunks);
   if (cudaGetLastError() != cudaSuccess) return SDQ_ERR_CUDA;
   }
   out->dev = xq_buf;

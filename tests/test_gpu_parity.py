@@ -39,7 +39,7 @@ def run_case(M, N, K, seed, out_n=1, rule=0, n_out_ch=None, check_rows=None, blo
     oq = so.quantize_act(sdq_synth.bf16_bits(X), ocfg(out_n, rule, block, gran))
     pe = {k: v.cpu().numpy() for k, v in m.packed_export(p).items()}
     ae = {k: v.cpu().numpy() for k, v in m.act_export(xq).items()}
-    for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp"):
+    for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp", "in_texp"):
         assert np.array_equal(pe[name], getattr(op, name)), name
     for name in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp"):
         assert np.array_equal(ae[name], getattr(oq, name)), name
@@ -196,6 +196,49 @@ def test_dense_inliers_one_hot_readback_and_workspace_split():
         with pytest.raises(m.SdqError) as e:
             m.sdq_decompose(W.cuda(), m.Config(out_n, gran, 32, 0))
         assert e.value.code == 1
+
+
+@pytest.mark.parametrize("M,K", [(13, 256), (21, 11008), (3, 16640)])
+def test_two_level_e4m3_scales_quantizer(M, K):
+    """SDQ_SCALE_UE4M3 activations (single-pass and two-pass quantizer): E4M3 scale codes and element codes bit-exact,
+    including an all-zero token, all-zero Q-Vectors, an infinity and a Q-Vector far below the token's maximum"""
+    m = sdq()
+    cfg = m.Config(1, m.GRAN_PAIR, 32, m.SCALE_UE4M3)
+    X = sdq_synth.make_act(M, K, 2100 + M)
+    X[1, :] = 0
+    X[2, 64:160] = 0
+    X[0, 5] = float("inf")
+    X[2, 200:232] = X[2, 200:232] * 2.0 ** -22
+    xq = m.sdq_quantize_act(X.cuda(), cfg)
+    oq = so.quantize_act(sdq_synth.bf16_bits(X), so.Config(1, so.GRAN_PAIR, 32, so.SCALE_UE4M3))
+    ae = {k: v.cpu().numpy() for k, v in m.act_export(xq).items()}
+    for name in ("xq4_scale", "xq4_code", "xq8_code", "xq8_sexp"):
+        assert np.array_equal(ae[name], getattr(oq, name)), name
+    with pytest.raises(m.SdqError) as e:
+        m.sdq_quantize_act(X.cuda(), m.Config(1, m.GRAN_PAIR, 64, m.SCALE_UE4M3))
+    assert e.value.code == 4
+
+
+@pytest.mark.parametrize("out_n", [0, 1, 2])
+def test_two_level_e4m3_scales_packer(out_n):
+    m = sdq()
+    N, K = 256, 1024
+    W = sdq_synth.make_weight(N, K, 2200 + out_n)
+    W[3, :] = 0
+    W[5, 32:96] = 0
+    W[7, :] = W[7, :] * 2.0 ** -30
+    rng = np.random.default_rng(3)
+    c = np.exp(rng.normal(0.0, 1.0, K)).astype(np.float32)
+    for cw in (None, c):
+        p = m.sdq_decompose(W.cuda(), m.Config(out_n, m.GRAN_PAIR, 32, m.SCALE_UE4M3), col_weight=None if cw is None else torch.from_numpy(cw).cuda())
+        op = so.decompose(sdq_synth.bf16_bits(W), so.Config(out_n, so.GRAN_PAIR, 32, so.SCALE_UE4M3), col_weight=cw)
+        pe = {k: v.cpu().numpy() for k, v in m.packed_export(p).items()}
+        for name in ("in_texp", "in_scale", "in_code", "in_meta", "out_code", "out_idx", "out_sexp"):
+            assert np.array_equal(pe[name], getattr(op, name)), name
+    for gran, block in ((m.GRAN_ELEM, 32), (m.GRAN_PAIR, 64), (m.GRAN_DENSE, 32)):
+        with pytest.raises(m.SdqError) as e:
+            m.sdq_decompose(W.cuda(), m.Config(out_n, gran, block, m.SCALE_UE4M3))
+        assert e.value.code == 4
 
 
 def test_one_hot_readback_512_tokens():
