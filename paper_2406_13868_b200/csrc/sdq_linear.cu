@@ -58,6 +58,9 @@ __host__ __device__ inline int slot_bytes_for(int n_tile, bool b32 = false, bool
   return wi_bytes(b32, dense) + n_tile * 128 + atoms * SF_ATOM_BYTES;
 }
 
+// 2^ex as a float (ex limited to the normal range), for the exact rescaling of two-level-scaled accumulators
+__device__ __forceinline__ float pow2i(int ex) { return __int_as_float((min(max(ex, -126), 127) + 127) << 23); }
+
 struct TileCoord {
   int rt, mtile, split;
   int i0, i1, o0, o1;   // inlier stages [i0, i1) of T2, outlier stages [o0, o1) of T1
@@ -216,7 +219,8 @@ sdq_linear_kernel(const LinearParams p)       // many tokens: 13 warps, four of 
       const uint32_t smb = ptx::smem_u32(sm);
       uint32_t s = 0, ph = 0, tcount = 0;
       bool ready = false;
-      const uint32_t id4[2] = {ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, true, 0, 0),
+      // (two-level scaling: the .block16 kind reads its scale codes as unsigned E4M3 when bit 23 is clear)
+      const uint32_t id4[2] = {ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, true, 0, 0) ^ (p.tw ? (1u << 23) : 0u),
                                ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, true, 2, 2)};
       const uint32_t id8 = ptx::idesc_block_scaled(128, (uint32_t)n_tile, 0, true, 0, 0);
       const uint32_t idd[2] = {ptx::idesc_block_scaled(128, (uint32_t)n_tile, 1, false, 0, 0),      // dense inliers
@@ -404,6 +408,12 @@ sdq_linear_kernel(const LinearParams p)       // many tokens: 13 warps, four of 
       ptx::tc_fence_after();
       if (!ok) break;
       const int64_t n0 = (int64_t)tc.rt * TILE_ROWS;
+      const int twr = p.tw ? __ldg(p.tw + n0 + q * 32 + lane) : 0;     // two-level scaling: this thread's row factor
+      auto rescale = [&](uint32_t (&v)[16], int c0) {                  // columns c0 .. c0 + 15 of the tile, by 2^(tw + tx)
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (c0 + j < n_valid) v[j] = __float_as_uint(__uint_as_float(v[j]) * pow2i(twr + __ldg(p.tx + m0 + c0 + j)));
+      };
       // split-K: this CTA's fp32 partial tile [token][128 rows] in the workspace
       float* part = nullptr;
       if (cluster_ks > 1) part = reinterpret_cast<float*>(sm);   // the ring is idle once the accumulator is complete
@@ -457,8 +467,16 @@ sdq_linear_kernel(const LinearParams p)       // many tokens: 13 warps, four of 
           if (g0 + c0 < n_valid) {                  // uniform over the four warps of the group
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-              stg[(2 * j) * 128 + q * 32 + lane] = (uint16_t)(pk[c0 / 2 + j] & 0xFFFFu);
-              stg[(2 * j + 1) * 128 + q * 32 + lane] = (uint16_t)(pk[c0 / 2 + j] >> 16);
+              uint32_t lo = pk[c0 / 2 + j] << 16, hi = pk[c0 / 2 + j] & 0xFFFF0000u;
+              if (p.tw) {
+                // two-level scaling: multiplying the rounded value by the power of two is the rounding of the multiplied
+                // value, so the factors go in here, after TMEM has been handed back
+                const int t = g0 + c0 + 2 * j;
+                if (t < n_valid) lo = __float_as_uint(__uint_as_float(lo) * pow2i(twr + __ldg(p.tx + m0 + t)));
+                if (t + 1 < n_valid) hi = __float_as_uint(__uint_as_float(hi) * pow2i(twr + __ldg(p.tx + m0 + t + 1)));
+              }
+              stg[(2 * j) * 128 + q * 32 + lane] = (uint16_t)(lo >> 16);
+              stg[(2 * j + 1) * 128 + q * 32 + lane] = (uint16_t)(hi >> 16);
             }
             ptx::named_bar_sync(1 + grp, 128);
             const uint32_t tok = et >> 4, seg = et & 15;
@@ -508,6 +526,7 @@ sdq_linear_kernel(const LinearParams p)       // many tokens: 13 warps, four of 
           if (lane == 0) ptx::mbar_arrive(acc_empty);
         }
         if (c0 >= n_valid) continue;  // uniform over the four epilogue warps
+        if (p.tw) rescale(v, c0);
         if (F32_OUT) {
           float* Y = reinterpret_cast<float*>(p.Y);
 #pragma unroll
@@ -556,6 +575,12 @@ sdq_linear_kernel(const LinearParams p)       // many tokens: 13 warps, four of 
 #pragma unroll
               for (int j = 0; j < 8; ++j) acc[j] += v[j];
             }
+            if (p.tw) {
+              const int twe = __ldg(p.tw + n0 + et);
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                if (t0 + j < n_valid) acc[j] *= pow2i(twe + __ldg(p.tx + m0 + t0 + j));
+            }
 #pragma unroll
             for (int j = 0; j < 8; ++j)
               if (t0 + j < n_valid) {
@@ -587,8 +612,13 @@ sdq_linear_kernel(const LinearParams p)       // many tokens: 13 warps, four of 
       const uint32_t q_per = rows_per >> 2;                    // 4, 8 or 16 (ks = 8, 4, 2): a power of two
       const uint32_t q_shift = 31u - (uint32_t)__clz((int)q_per);
       const uint32_t n_items = q_per * (uint32_t)n_valid;
-      auto out4 = [&](uint32_t idx, const float4& acc) {
+      auto out4 = [&](uint32_t idx, float4 acc) {
         const uint32_t row = rank * rows_per + ((idx & (q_per - 1)) << 2), tok = idx >> q_shift;
+        if (p.tw) {
+          const int4 t4 = __ldg(reinterpret_cast<const int4*>(p.tw + n0 + row));
+          const int txe = __ldg(p.tx + m0 + tok);
+          acc.x *= pow2i(t4.x + txe); acc.y *= pow2i(t4.y + txe); acc.z *= pow2i(t4.z + txe); acc.w *= pow2i(t4.w + txe);
+        }
         if (F32_OUT) {
           *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.Y) + (m0 + tok) * p.ldy + n0 + row) = acc;
         } else {
@@ -672,7 +702,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   if (Xq->K != P->K || Xq->M <= 0 || P->N <= 0 || P->N % TILE_ROWS || P->K % K2 || ldy < P->N) return SDQ_ERR_SHAPE;
   if (Xq->cfg.in_block != P->cfg.in_block || Xq->cfg.scale_rule != P->cfg.scale_rule) return SDQ_ERR_SHAPE;
   if (P->cfg.in_gran != SDQ_GRAN_PAIR && !(P->cfg.in_gran >= SDQ_GRAN_DENSE && P->cfg.in_block == 32)) return SDQ_ERR_UNSUPPORTED;
-  if (P->cfg.scale_rule == SDQ_SCALE_UE4M3) return SDQ_ERR_UNSUPPORTED;
+  if (P->cfg.scale_rule == SDQ_SCALE_UE4M3 && !(P->cfg.in_gran == SDQ_GRAN_PAIR && P->cfg.in_block == 32)) return SDQ_ERR_UNSUPPORTED;
   if (((uintptr_t)Y & 15) || (ldy % 8) || ((uintptr_t)ws & 15)) return SDQ_ERR_ALIGNMENT;
   static bool attr_set = false;
   if (!attr_set) {
@@ -694,9 +724,12 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   p.w = (const uint8_t*)P->dev;
   p.x = (const uint8_t*)Xq->dev;
   p.b32 = P->cfg.in_block == 32 ? 1 : 0;
+  const bool ue = P->cfg.scale_rule == SDQ_SCALE_UE4M3;
   p.dense = P->cfg.in_gran >= SDQ_GRAN_DENSE ? 1 : 0;   // the n:8 patterns are stored and run like the dense one
   p.poff = packed_offsets(P->N, P->K, P->cfg.out_n, p.b32 != 0, p.dense != 0);
   p.aoff = act_offsets(Xq->M, Xq->K, p.b32 != 0);
+  p.tw = ue ? reinterpret_cast<const int32_t*>(p.w + p.poff.wtexp) : nullptr;
+  p.tx = reinterpret_cast<const int32_t*>(p.x + p.aoff.sexp);
   p.M = Xq->M; p.N = P->N; p.K = P->K;
   p.out_n = P->cfg.out_n;
   const int64_t M = Xq->M;

@@ -24,6 +24,10 @@ struct LinearParams {
   int tmem_cols;         // TMEM columns to allocate (128, 256 or 512)
   int meta_col;          // first TMEM column of the metadata / scale buffers
   int b32;               // 1: one inlier / activation scale per 32 K (kind::mxf4nvf4 .block16), runtime geometry only
+  // two-level scaling (E4M3 Q-Vector scale codes): the accumulator of row n and token m is in units of 2^(tw[n] + tx[m]);
+  // the epilogue multiplies that factor back in.  tw == nullptr: not in use.
+  const int32_t* tw;     // [N] exponents of the rows' inlier factors (packed weights)
+  const int32_t* tx;     // [tokens] exponents of the tokens' 8-bit scales (quantized activations)
   int dense;             // 1: dense inliers (no Stage 1): 4 dense kind::mxf4 MMAs of 64 K per stage, runtime geometry only
   int ksplit;            // CTAs sharing the K range of one row tile (1 = no split)
   int cluster_ks;        // > 1: those CTAs form a cluster and reduce through distributed shared memory

@@ -20,10 +20,10 @@ def sdq():
     return m
 
 
-def check_sampled(M, N, K, seed, out_n=1, n_tok=12, use_ws=False, block=64, gran=so.GRAN_PAIR):
+def check_sampled(M, N, K, seed, out_n=1, n_tok=12, use_ws=False, block=64, gran=so.GRAN_PAIR, rule=0):
     m = sdq()
-    cfg = m.Config(out_n, gran, block, 0)
-    ocfg = so.Config(out_n, gran, block, 0)
+    cfg = m.Config(out_n, gran, block, rule)
+    ocfg = so.Config(out_n, gran, block, rule)
     W = sdq_synth.make_weight(N, K, seed, device="cuda")
     X = sdq_synth.make_act(M, K, seed + 1, device="cuda")
     p = m.sdq_decompose(W, cfg)
@@ -43,7 +43,7 @@ def check_sampled(M, N, K, seed, out_n=1, n_tok=12, use_ws=False, block=64, gran
 
     op = so.decompose(sdq_synth.bf16_bits(W[rows_t]), ocfg)
     pe = m.packed_export(p)
-    for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp"):
+    for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp", "in_texp"):
         assert np.array_equal(pe[name][rows_t].cpu().numpy(), getattr(op, name)), name
     oq = so.quantize_act(sdq_synth.bf16_bits(X[toks_t]), ocfg)
     ae = m.act_export(xq)
@@ -81,6 +81,12 @@ def test_scale_block_32_at_full_size(M, N, K):
 def test_n_of_8_patterns_at_full_size(M, N, K, n):
     """configs 2, 3 and 4 with the evaluation's patterns 7:8 = 1:8 + 6:8 and 8:8 = 1:8 + 7:8 (inliers stored dense)"""
     check_sampled(M, N, K, 3700 + M + n, block=32, gran=so.gran_keep(n))
+
+
+@pytest.mark.parametrize("M,N,K", [(16, 4096, 4096), (2048, 11008, 4096), (2048, 4096, 11008)])
+def test_two_level_e4m3_scales_at_full_size(M, N, K):
+    """configs 2 and 3 with E4M3 Q-Vector scales and power-of-two row / token factors"""
+    check_sampled(M, N, K, 3900 + M, block=32, rule=2)
 
 
 @pytest.mark.parametrize("out_n", [1, 2, 0])

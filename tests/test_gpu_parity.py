@@ -198,6 +198,48 @@ def test_dense_inliers_one_hot_readback_and_workspace_split():
         assert e.value.code == 1
 
 
+@pytest.mark.parametrize("M,N,K,out_n", [(8, 256, 256, 1), (1, 512, 2048, 1), (16, 256, 4096, 2), (33, 128, 768, 0), (100, 256, 2816, 1),
+                                         (128, 1024, 4096, 1), (129, 256, 512, 1), (300, 512, 1024, 2), (520, 6400, 256, 1),
+                                         (700, 2560, 1024, 1)])
+def test_two_level_e4m3_scales_through_the_tensor_core(M, N, K, out_n):
+    """SDQ_SCALE_UE4M3: E4M3 Q-Vector scale codes for inlier weights and 4-bit activations (kind::mxf4nvf4 .block16 with
+    its scale format switched), accumulator in units of the row and token factors, multiplied back in by the epilogue:
+    few tokens, cluster split K, several hundred tokens, persistent tiles"""
+    run_case(M, N, K, 2300 + M, out_n=out_n, rule=2, block=32)
+
+
+def test_two_level_e4m3_scales_one_hot_readback_and_workspace_split():
+    m = sdq()
+    cfg = m.Config(1, m.GRAN_PAIR, 32, m.SCALE_UE4M3)
+    oc = so.Config(1, so.GRAN_PAIR, 32, so.SCALE_UE4M3)
+    N, K = 256, 512
+    W = sdq_synth.make_weight(N, K, 2401)
+    W[9, :] = W[9, :] * 2.0 ** -14                     # a row with a very different factor
+    p = m.sdq_decompose(W.cuda(), cfg)
+    X = torch.eye(K, dtype=torch.bfloat16)            # 1.0 is exact in the 8-bit format, not with a 4-bit code times an E4M3 scale
+    xq = m.sdq_quantize_act(X.cuda(), cfg)
+    y = m.sdq_linear(xq, p, f32=True).cpu().numpy().astype(np.float64)
+    op = so.decompose(sdq_synth.bf16_bits(W), oc)
+    oq = so.quantize_act(sdq_synth.bf16_bits(X), oc)
+    A_i, A_o = so.dequant_act(oq)
+    W_in, W_out = so.dequant_weights(op)
+    # one non-zero per token: every output is a single product pair, exact in fp32 up to the final sum of the two parts
+    a_i, a_o = np.diag(A_i), np.diag(A_o)
+    assert (a_o == 1.0).all()
+    ref = (W_in * a_i[None, :] + W_out).T
+    assert np.allclose(y, ref, rtol=2e-7, atol=0)
+    M = 7
+    Xs = sdq_synth.make_act(M, K, 2402)
+    xs = m.sdq_quantize_act(Xs.cuda(), cfg)
+    ws = m.make_workspace(M, N, K, cfg, "cuda")
+    y1 = m.sdq_linear(xs, p, f32=True, workspace=ws)
+    y2 = m.sdq_linear(xs, p, f32=True, workspace=ws)
+    assert torch.equal(y1, y2)
+    d, tol = y_close(y1.cpu().numpy(), so.linear(so.quantize_act(sdq_synth.bf16_bits(Xs), oc), op))
+    assert (d <= tol).all()
+    assert m.device_status() == 0
+
+
 @pytest.mark.parametrize("M,K", [(13, 256), (21, 11008), (3, 16640)])
 def test_two_level_e4m3_scales_quantizer(M, K):
     """SDQ_SCALE_UE4M3 activations (single-pass and two-pass quantizer): E4M3 scale codes and element codes bit-exact,
