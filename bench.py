@@ -283,13 +283,17 @@ def run_ours(args):
     sample = OracleSample(rows_x=1024)
     v, dt = sample.run()
     threads, desc = sample.threads, sample.desc
+    # ---- and with E4M3 Q-Vector scales under power-of-two row / token factors (the scale-factor format the paper prefers)
+    cfge = sdq.Config(1, sdq.GRAN_PAIR, 32, sdq.SCALE_UE4M3)
+    e4 = measure_variant_step(sdq, cfge, dev, rank, X, H, (Yg, Yu, Yd), flops_step, args.steps,
+                              "the same step with E4M3 scale codes per 32 K and power-of-two row / token factors (two-level scaling)")
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp4+fp8 (E2M1/E4M3 products, fp32 accumulate)",
             "data": "synthetic",
             "config": {"workload": WORKLOAD, "tokens_per_gpu": M_PREFILL, "l2": "packed weights + activations of one step exceed L2 (150 MB > 126 MB)",
                        "parallelism": "dp%d (independent batches, no collective)" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "quantizer_roofline": quant, "scale_block_32": b32, "dense_inliers": dns, "decode": decode,
+            "roofline": roofline, "quantizer_roofline": quant, "scale_block_32": b32, "dense_inliers": dns, "e4m3_scales": e4, "decode": decode,
             "cpu_baseline": {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc, "seconds": dt}}
     print(json.dumps(line))
 

@@ -20,7 +20,8 @@
  * Pins (tests/ -m "not gpu"): exhaustive codec checks against closed forms and torch CPU casts,
  * N:M invariants from the paper, brute force over all C(8,n) selections, an independent dense
  * "definition" of the decomposition, brute-force matmul, one-hot read-back, exact power-of-two
- * scaling, and the paper's printed bits-per-weight / throughput arithmetic.
+ * scaling, the paper's printed bits-per-weight / throughput arithmetic, and for the E4M3 scale rule closed forms at every
+ * representable scale and midpoint plus an independent definition built on torch's float8 cast.
  * Parity unpinned: none of the functions in this file (model-quality numbers of the paper are not
  * computed here at all).
  */
