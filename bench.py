@@ -564,6 +564,26 @@ def run_sweep(args):
         c5["M%d" % M] = {"ms_per_model_pass": ms, "dense_equiv_TFLOPs": flops / ms / 1e9, "weight_GBps_algorithmic": algo / ms / 1e6,
                          "frac_of_hbm_peak": algo / ms / 1e6 / peaks["hbm"], "frac_of_mixed_tensor_peak": flops / ms / 1e9 / (peaks["bf16"] * MIXED_PEAK_OVER_BF16)}
     out["llama7b_32_layers_224_linears"] = c5
+    del layers
+    # ---- output error of every configuration against the unquantized product on the synthetic layer (a proxy only:
+    # the paper's quality numbers are perplexities of real models): ||Y - X W^T|| / ||X W^T||, fp64 reference on the GPU
+    M, K, N = 512, 4096, 4096
+    X = sdq_synth.make_act(M, K, 6001, device="cuda")
+    W = sdq_synth.make_weight(N, K, 6002, device="cuda")
+    ref = X.double() @ W.double().T
+    err = {}
+    for name, cfg in (("4:8 pair-wise, no outliers", sdq.Config(0, sdq.GRAN_PAIR, 64, 0)),
+                      ("4:8 pair-wise + 1:8", sdq.Config(1, sdq.GRAN_PAIR, 64, 0)),
+                      ("4:8 pair-wise + 2:8", sdq.Config(2, sdq.GRAN_PAIR, 64, 0)),
+                      ("4:8 pair-wise + 1:8, scale per 32", sdq.Config(1, sdq.GRAN_PAIR, 32, 0)),
+                      ("4:8 pair-wise + 1:8, E4M3 scales per 32", sdq.Config(1, sdq.GRAN_PAIR, 32, sdq.SCALE_UE4M3)),
+                      ("6:8 = 2:8 + 4:8 at any position", sdq.Config(2, sdq.gran_keep(6), 32, 0)),
+                      ("7:8 = 1:8 + 6:8", sdq.Config(1, sdq.gran_keep(7), 32, 0)),
+                      ("8:8 = 1:8 + 7:8", sdq.Config(1, sdq.GRAN_DENSE, 32, 0)),
+                      ("8:8 dense 4-bit, no outliers", sdq.Config(0, sdq.GRAN_DENSE, 32, 0))):
+        Y = sdq.sdq_linear(sdq.sdq_quantize_act(X, cfg), sdq.sdq_decompose(W, cfg), f32=True)
+        err[name] = float((Y.double() - ref).norm() / ref.norm())
+    out["relative_output_error_M512_4096x4096"] = err
     assert sdq.device_status() == 0
     print(json.dumps(out))
 
