@@ -283,6 +283,35 @@ def test_two_level_e4m3_scales_packer(out_n):
         assert e.value.code == 4
 
 
+@pytest.mark.parametrize("rule,block", [(0, 64), (1, 64), (0, 32), (1, 32), (2, 32)])
+def test_values_on_rounding_boundaries(rule, block):
+    """inputs built from exact ties (element quotients on E2M1 midpoints, block maxima on E4M3 midpoints, blocks far below
+    the row maximum): quantizer and packer (pair-wise and un-pruned) bit-exact against the oracle, product within the
+    criterion"""
+    from tests.tie_cases import make_tie_matrix
+    m = sdq()
+    for seed in (0, 1):
+        X = make_tie_matrix(40, 1024, 10 + seed)
+        W = make_tie_matrix(128, 1024, 20 + seed)
+        grans = [m.GRAN_PAIR] + ([m.GRAN_DENSE] if (block == 32 and rule != 2) else [])
+        for gran in grans:
+            for out_n in (0, 1):
+                cfg, oc = m.Config(out_n, gran, block, rule), so.Config(out_n, gran, block, rule)
+                xq = m.sdq_quantize_act(X.cuda(), cfg)
+                p = m.sdq_decompose(W.cuda(), cfg)
+                oq = so.quantize_act(sdq_synth.bf16_bits(X), oc)
+                op = so.decompose(sdq_synth.bf16_bits(W), oc)
+                ae = {k: v.cpu().numpy() for k, v in m.act_export(xq).items()}
+                pe = {k: v.cpu().numpy() for k, v in m.packed_export(p).items()}
+                for name in ("xq4_scale", "xq4_code", "xq8_code", "xq8_sexp"):
+                    assert np.array_equal(ae[name], getattr(oq, name)), (name, gran, out_n)
+                for name in ("in_texp", "in_scale", "in_code", "in_meta", "out_code", "out_idx", "out_sexp"):
+                    assert np.array_equal(pe[name], getattr(op, name)), (name, gran, out_n)
+                d, tol = y_close(m.sdq_linear(xq, p, f32=True).cpu().numpy(), so.linear(oq, op))
+                assert (d <= tol).all(), (gran, out_n, d.max())
+    assert m.device_status() == 0
+
+
 def test_one_hot_readback_512_tokens():
     m = sdq()
     cfg = m.Config()

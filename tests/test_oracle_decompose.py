@@ -513,3 +513,21 @@ def test_ue4m3_activations_match_independent_definition(block):
     X[0, 40] = 2.0 ** -12
     q1 = so.quantize_act(sdq_synth.bf16_bits(X), so.Config(1, so.GRAN_PAIR, 32, so.SCALE_UE4M3))
     assert q1.xq8_sexp[0] == 0 and q1.xq4_scale[0, 1] == 1 and q1.xq4_scale[0, 0] == so.lib().sdqo_ue4m3_scale_code(256.0, 0)
+
+
+@pytest.mark.parametrize("rule,block", [(so.SCALE_OCP_FLOOR, 32), (so.SCALE_CEIL_NOSAT, 64), (so.SCALE_UE4M3, 32), (so.SCALE_UE4M3, 64)])
+def test_values_on_rounding_boundaries_match_the_independent_definition(rule, block):
+    """inputs built from exact ties (element quotients on E2M1 midpoints, block maxima on E4M3 midpoints): the oracle and
+    the independent definition must break every tie the same way, for activations and for un-pruned weights"""
+    from tests.tie_cases import make_tie_matrix
+    tag = {so.SCALE_OCP_FLOOR: True, so.SCALE_CEIL_NOSAT: False, so.SCALE_UE4M3: "ue4m3"}[rule]
+    for seed in (0, 1, 2):
+        Xb = sdq_synth.bf16_bits(make_tie_matrix(24, 512, seed))
+        q = so.quantize_act(Xb, so.Config(1, so.GRAN_PAIR, block, rule))
+        A_i, A_o = so.dequant_act(q)
+        ref_i, ref_o = quantize_act_dense(Xb, block, tag)
+        assert np.array_equal(A_i, ref_i) and np.array_equal(A_o, ref_o)
+        p = so.decompose(Xb, so.Config(0, so.GRAN_DENSE, block, rule))
+        W_in, _ = so.dequant_weights(p)
+        assert np.array_equal(W_in, decompose_dense(Xb, 0, None, block, tag)[0])
+        assert np.array_equal(W_in, A_i)          # un-pruned weights without outliers = the activation 4-bit quantizer
