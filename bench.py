@@ -565,6 +565,38 @@ def run_sweep(args):
                          "frac_of_hbm_peak": algo / ms / 1e6 / peaks["hbm"], "frac_of_mixed_tensor_peak": flops / ms / 1e9 / (peaks["bf16"] * MIXED_PEAK_OVER_BF16)}
     out["llama7b_32_layers_224_linears"] = c5
     del layers
+    # ---- the same model with q, k, v packed as one 12288-row matrix and gate, up as one 22016-row matrix (the usual
+    # fused projections: the rows of a linear layer are independent, so concatenating weight matrices that read the
+    # same activations changes no output): 4 GEMMs + 4 quantizer launches per layer
+    fshapes = [(12288, 4096), (4096, 4096), (22016, 4096), (4096, 11008)]
+    flayers = []
+    for l in range(32):
+        ps = []
+        for i, (N, K) in enumerate(fshapes):
+            W = sdq_synth.make_weight(N, K, 7000 + 10 * l + i, device="cuda")
+            ps.append(sdq.sdq_decompose(W, cfg))
+            del W
+        flayers.append(ps)
+    c6 = {}
+    for M in (1, 16, 128, 1024):
+        X = sdq_synth.make_act(M, 4096, 5500 + M, n_outlier_channels=41, device="cuda")
+        Hh = sdq_synth.make_act(M, 11008, 5600 + M, n_outlier_channels=110, device="cuda")
+        bx = torch.empty(sdq.act_size(M, 4096, cfg), dtype=torch.uint8, device=dev)
+        bh = torch.empty(sdq.act_size(M, 11008, cfg), dtype=torch.uint8, device=dev)
+        Ys = [torch.empty((M, n), dtype=torch.bfloat16, device=dev) for n, _ in fshapes]
+
+        def fmodel():
+            for ps in flayers:
+                sdq.sdq_linear(sdq.sdq_quantize_act(X, cfg, bx), ps[0], Ys[0])     # q, k, v
+                sdq.sdq_linear(sdq.sdq_quantize_act(X, cfg, bx), ps[1], Ys[1])     # o
+                sdq.sdq_linear(sdq.sdq_quantize_act(X, cfg, bx), ps[2], Ys[2])     # gate, up
+                sdq.sdq_linear(sdq.sdq_quantize_act(Hh, cfg, bh), ps[3], Ys[3])    # down
+        ms = time_graph(fmodel, reps=3 if M >= 1024 else 10)
+        flops = 2.0 * M * sum(n * k for n, k in fshapes) * 32
+        c6["M%d" % M] = {"ms_per_model_pass": ms, "dense_equiv_TFLOPs": flops / ms / 1e9, "weight_GBps_algorithmic": algo / ms / 1e6,
+                         "frac_of_hbm_peak": algo / ms / 1e6 / peaks["hbm"]}
+    out["llama7b_32_layers_fused_qkv_gate_up_128_linears"] = c6
+    del flayers
     # ---- output error of every configuration against the unquantized product on the synthetic layer (a proxy only:
     # the paper's quality numbers are perplexities of real models): ||Y - X W^T|| / ||X W^T||, fp64 reference on the GPU
     M, K, N = 512, 4096, 4096

@@ -754,6 +754,10 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
       // per SM leave only three ring slots, which pays only when one per SM would leave many SMs idle
       ks = split_for((M <= 64 ? 2 : 1) * sm_count);
       if (M > 64 && ks * tiles * 5 <= sm_count * 3) ks = split_for(2 * sm_count);
+      // more row tiles than SMs: one CTA per SM walking whole-K tiles streams a tile in ~19 us however few tiles its
+      // last round holds (149 tiles took 38 us, 148 took 16), while two half-K CTAs per SM keep more bytes in flight;
+      // split in two and let the grid run in waves of two CTAs per SM (K >= 2048: below that the halves are too short)
+      if (ks == 1 && tiles > sm_count && T2c >= 8) ks = 2;
     } else if (tiles * 2 <= sm_count) {
       // a few hundred tokens against a narrow weight matrix: fewer 256-token tiles than half the SMs
       ks = split_for(sm_count);

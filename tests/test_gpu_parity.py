@@ -376,6 +376,28 @@ def test_cluster_split_k_few_tokens(M, N, K, out_n):
     assert (d <= tol).all(), (d.max(), (d / tol).max())
 
 
+@pytest.mark.parametrize("M,N,K,out_n", [(5, 19200, 2048, 1), (64, 22016, 2304, 1), (100, 19200, 2048, 2), (16, 38400, 2048, 0), (7, 19200, 512, 1)])
+def test_few_tokens_more_row_tiles_than_sms(M, N, K, out_n):
+    """few tokens against a very wide matrix: more row tiles than SMs, K still split in two, the grid runs in waves"""
+    m = sdq()
+    cfg = m.Config(out_n, m.GRAN_PAIR, 64, 0)
+    W = sdq_synth.make_weight(N, K, 2500 + M)
+    X = sdq_synth.make_act(M, K, 2501 + M)
+    p = m.sdq_decompose(W.cuda(), cfg)
+    xq = m.sdq_quantize_act(X.cuda(), cfg)
+    y1 = m.sdq_linear(xq, p, f32=True)
+    y2 = m.sdq_linear(xq, p, f32=True)
+    y16 = m.sdq_linear(xq, p)
+    assert m.device_status() == 0
+    assert torch.equal(y1, y2) and torch.equal(y16, y1.to(torch.bfloat16))
+    oq = so.quantize_act(sdq_synth.bf16_bits(X), ocfg(out_n))
+    RT = N // 128
+    for t in (0, 1, RT // 2, RT - 2, RT - 1):
+        op = so.decompose(sdq_synth.bf16_bits(W[128 * t:128 * t + 128]), ocfg(out_n))
+        d, tol = y_close(y1[:, 128 * t:128 * t + 128].cpu().numpy(), so.linear(oq, op))
+        assert (d <= tol).all(), (t, d.max())
+
+
 def test_one_hot_readback_through_the_tensor_core():
     """X = identity rows (1.0 is exact in both activation formats): Y^T must equal W_in + W_out exactly"""
     m = sdq()
