@@ -682,6 +682,10 @@ static int choose_ksplit(int64_t M, int64_t N, int64_t K, int sm_count) {
   if (ks > 32) ks = 32;
   return ks < 1 ? 1 : ks;
 }
+// CTAs a few-token grid may have per SM, in tenths (two small CTAs fit an SM; a little more runs a short second wave)
+#ifndef SDQ_FEW_TOKEN_CTA_BUDGET_TENTHS
+#define SDQ_FEW_TOKEN_CTA_BUDGET_TENTHS 20
+#endif
 static int n_tile_for(int64_t M) { return M > 128 ? 256 : (M > 64 ? 128 : (M > 32 ? 64 : (M > 16 ? 32 : 16))); }
 
 extern "C" sdq_status_t sdq_workspace_size(int64_t M, int64_t N, int64_t K, const sdq_config_t* cfg, size_t* bytes)
@@ -752,7 +756,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
     if (M <= 128) {
       // CTAs the grid may have: up to 64 tokens the CTAs are small enough for two per SM; from 65 to 128 tokens two
       // per SM leave only three ring slots, which pays only when one per SM would leave many SMs idle
-      ks = split_for((M <= 64 ? 2 : 1) * sm_count);
+      ks = split_for((M <= 64 ? SDQ_FEW_TOKEN_CTA_BUDGET_TENTHS * sm_count / 10 : sm_count));
       if (M > 64 && ks * tiles * 5 <= sm_count * 3) ks = split_for(2 * sm_count);
       // more row tiles than SMs: one CTA per SM walking whole-K tiles streams a tile in ~19 us however few tiles its
       // last round holds (149 tiles took 38 us, 148 took 16), while two half-K CTAs per SM keep more bytes in flight;
