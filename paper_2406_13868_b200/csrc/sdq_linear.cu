@@ -596,24 +596,25 @@ sdq_linear_kernel(const LinearParams p)       // many tokens: 13 warps, four of 
     if (!ok && lane == 0) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
   }
   if (cluster_ks > 1) {
-    // ---------------- cluster split-K: one tile per CTA; CTA r adds rows [r*128/ks, (r+1)*128/ks) of all members
+    // ---------------- cluster split-K: one tile per CTA; CTA r adds its share of the tile's rows over all members
     ptx::cluster_sync();                         // every member's partial tile is in its shared memory
     if (warp >= 2 && warp <= 5) {
       const uint32_t et = (warp - 2) * 32 + lane;
       const uint32_t ks = (uint32_t)cluster_ks, rank = ptx::cluster_ctarank();
-      const uint32_t rows_per = TILE_ROWS / ks;
       const int n_valid = (int)min((int64_t)n_tile, p.M - (int64_t)first_tc.mtile * n_tile);
       const int64_t m0 = (int64_t)first_tc.mtile * n_tile, n0 = (int64_t)first_tc.rt * TILE_ROWS;
       const uint32_t local = ptx::smem_u32(sm);
-      // four rows x one token per item: one 16-byte load per member, added in rank order
+      // four rows x one token per item: one 16-byte load per member, added in rank order.  The 32 quads of rows are
+      // dealt out evenly over the members (ks need not divide 32: 3 members take 10, 11 and 11 quads)
       uint32_t peer[8];
 #pragma unroll
       for (uint32_t sp = 0; sp < 8; ++sp) peer[sp] = ptx::mapa_u32(local, sp < ks ? sp : 0u);
-      const uint32_t q_per = rows_per >> 2;                    // 4, 8 or 16 (ks = 8, 4, 2): a power of two
-      const uint32_t q_shift = 31u - (uint32_t)__clz((int)q_per);
+      const uint32_t q_begin = rank * 32u / ks, q_per = (rank + 1) * 32u / ks - q_begin;
       const uint32_t n_items = q_per * (uint32_t)n_valid;
+      auto item_row = [&](uint32_t idx, uint32_t& tok) { tok = idx / q_per; return (q_begin + (idx - tok * q_per)) << 2; };
       auto out4 = [&](uint32_t idx, float4 acc) {
-        const uint32_t row = rank * rows_per + ((idx & (q_per - 1)) << 2), tok = idx >> q_shift;
+        uint32_t tok;
+        const uint32_t row = item_row(idx, tok);
         if (p.tw) {
           const int4 t4 = __ldg(reinterpret_cast<const int4*>(p.tw + n0 + row));
           const int txe = __ldg(p.tx + m0 + tok);
@@ -629,7 +630,7 @@ sdq_linear_kernel(const LinearParams p)       // many tokens: 13 warps, four of 
           *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.Y) + (m0 + tok) * p.ldy + n0 + row) = w;
         }
       };
-      auto item_off = [&](uint32_t idx) { return ((idx >> q_shift) * TILE_ROWS + rank * rows_per + ((idx & (q_per - 1)) << 2)) * 4; };
+      auto item_off = [&](uint32_t idx) { uint32_t tok; const uint32_t row = item_row(idx, tok); return (tok * TILE_ROWS + row) * 4; };
       // two items per round: up to 16 loads of 16 bytes in flight per thread
       for (uint32_t idx = et; idx < n_items; idx += 256) {
         const uint32_t idx2 = idx + 128;
@@ -745,12 +746,17 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   p.ws_counter = nullptr;
   p.ws_partial = nullptr;
   if (!ws) {
-    // cluster split-K: power-of-two cluster of up to 8 CTAs per (row tile, token tile), one tile per CTA
+    // cluster split-K: a cluster of up to 8 CTAs per (row tile, token tile), one tile per CTA
     const int tiles = (int)(P->N / TILE_ROWS) * p.n_mtiles, T2c = (int)(P->K / K2);
+    // as many members (1..8) as the budget and the inlier stages allow.  Clusters are placed inside one GPC, whose SM count
+    // varies: sizes 3, 5, 6, 7 pack worse than powers of two, and a grid that needs every slot then runs a second wave
+    // (96 clusters of 3 took 21 us, 96 of 2 take 14), so odd sizes only get 88 % of the budget
     auto split_for = [&](int cta_budget) {
-      int k = 8;
-      while (k > 1 && ((int64_t)k * tiles > cta_budget || k > T2c)) k >>= 1;
-      return k;
+      for (int k = 8; k > 1; --k) {
+        const bool pow2 = (k & (k - 1)) == 0;
+        if (k <= T2c && (int64_t)k * tiles <= (pow2 ? cta_budget : cta_budget * 22 / 25)) return k;
+      }
+      return 1;
     };
     int ks = 1;
     if (M <= 128) {
