@@ -37,6 +37,10 @@
    become outliers and n - out_n stay inliers at whatever positions they have (the paper's flexible N:M patterns, e.g.
    7:8 = 1:8 + 6:8); stored like the dense pattern, the dropped positions holding +0.  KEEP(8) is DENSE. */
 #define SDQO_GRAN_KEEP(n) (2 + (8 - (n)))
+/* S-Vectors of 4 (the evaluation's 3:4 = 1:4 + 2:4 configuration): Stage 1 keeps the 3 most significant of every 4,
+   Stage 2 takes the most significant of every 4 as the outlier (out_n = 2 per 8 consecutive K; out_n = 0: none), the
+   others stay inliers at whatever positions they have; stored like the dense pattern. */
+#define SDQO_GRAN_3OF4 9
 #define SDQO_SCALE_OCP_FLOOR 0  /* E = floor(log2 amax) - 2   (OCP MX rule, may saturate in (6,8)) */
 #define SDQO_SCALE_CEIL_NOSAT 1 /* E = smallest integer with amax <= 6 * 2^E                        */
 /* Two-level scaling with 8-bit floating-point Q-Vector scales (the quantization-stage study: scale factors in
@@ -197,9 +201,13 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
   if (cfg->out_n < 0 || cfg->out_n > 2) return -1;
   if (cfg->in_block != 32 && cfg->in_block != 64) return -1;
   if (cfg->scale_rule < 0 || cfg->scale_rule > SDQO_SCALE_UE4M3 || (cfg->scale_rule == SDQO_SCALE_UE4M3 && !in_texp)) return -1;
-  if (cfg->in_gran < 0 || cfg->in_gran > SDQO_GRAN_KEEP(2)) return -1;
-  const int keep_n = 10 - cfg->in_gran;                                /* n of KEEP(n); meaningful from DENSE on */
-  if (cfg->in_gran >= SDQO_GRAN_DENSE && keep_n <= cfg->out_n) return -1;
+  if (cfg->in_gran < 0 || cfg->in_gran > SDQO_GRAN_3OF4) return -1;
+  /* S-Vector length, values that survive Stage 1 per S-Vector (meaningful from DENSE on), outliers per S-Vector */
+  const int sv = cfg->in_gran == SDQO_GRAN_3OF4 ? 4 : 8;
+  const int keep_n = cfg->in_gran == SDQO_GRAN_3OF4 ? 3 : 10 - cfg->in_gran;
+  if (cfg->in_gran == SDQO_GRAN_3OF4 && cfg->out_n == 1) return -1;    /* one outlier per 4 is two per 8 */
+  const int on_sv = cfg->out_n * sv / 8;
+  if (cfg->in_gran >= SDQO_GRAN_DENSE && keep_n <= on_sv) return -1;
   const int on = cfg->out_n, Bs = cfg->in_block;
   const int64_t G8 = K / 8;
   const int64_t slots = cfg->in_gran >= SDQO_GRAN_DENSE ? K : K / 2;   /* inlier slots per row */
@@ -217,20 +225,22 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
     memset(dropped, 0, (size_t)K);
     for (int64_t k = 0; k < K; ++k) sig[k] = significance(w[k], col_weight, k);
 
-    /* Stage 2, local outlier extraction: the out_n most significant values of every S-Vector of 8
-       (largest first, ties to the lower index) */
+    /* Stage 2, local outlier extraction: the most significant values of every S-Vector (out_n of 8; with S-Vectors of
+       4, one of 4), largest first, ties to the lower index */
     double out_amax = 0.0;
     for (int64_t g = 0; g < G8; ++g) {
       int chosen[2] = {-1, -1};
-      for (int t = 0; t < on; ++t) {
-        int best = -1;
-        for (int i = 0; i < 8; ++i) {
-          if (is_out[8 * g + i]) continue;
-          if (best < 0 || sig[8 * g + i] > sig[8 * g + best]) best = i;
+      int nc = 0;
+      for (int sub = 0; sub < 8 / sv; ++sub)
+        for (int t = 0; t < on_sv; ++t) {
+          int best = -1;
+          for (int i = sub * sv; i < (sub + 1) * sv; ++i) {
+            if (is_out[8 * g + i]) continue;
+            if (best < 0 || sig[8 * g + i] > sig[8 * g + best]) best = i;
+          }
+          is_out[8 * g + best] = 1;
+          chosen[nc++] = best;
         }
-        is_out[8 * g + best] = 1;
-        chosen[t] = best;
-      }
       if (on == 2 && chosen[0] > chosen[1]) { int t = chosen[0]; chosen[0] = chosen[1]; chosen[1] = t; }
       for (int t = 0; t < on; ++t) {
         out_idx[(n * G8 + g) * on + t] = (uint8_t)chosen[t];
@@ -256,14 +266,15 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
       memset(kept, 1, (size_t)K);
       for (int64_t g = 0; g < G8; ++g) {
         uint8_t chosen[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        for (int t = 0; t < keep_n - on; ++t) {
-          int best = -1;
-          for (int i = 0; i < 8; ++i) {
-            if (is_out[8 * g + i] || chosen[i]) continue;
-            if (best < 0 || sig[8 * g + i] > sig[8 * g + best]) best = i;
+        for (int sub = 0; sub < 8 / sv; ++sub)
+          for (int t = 0; t < keep_n - on_sv; ++t) {
+            int best = -1;
+            for (int i = sub * sv; i < (sub + 1) * sv; ++i) {
+              if (is_out[8 * g + i] || chosen[i]) continue;
+              if (best < 0 || sig[8 * g + i] > sig[8 * g + best]) best = i;
+            }
+            chosen[best] = 1;
           }
-          chosen[best] = 1;
-        }
         for (int i = 0; i < 8; ++i) dropped[8 * g + i] = (uint8_t)(!is_out[8 * g + i] && !chosen[i]);
       }
     } else if (cfg->in_gran == SDQO_GRAN_PAIR) {

@@ -19,6 +19,7 @@ _SRC = os.path.join(_HERE, "sdq_oracle.c")
 _LIB = os.path.join(_HERE, "libsdq_oracle.so")
 
 GRAN_PAIR, GRAN_ELEM, GRAN_DENSE = 0, 1, 2
+GRAN_3OF4 = 9      # S-Vectors of 4: 3:4 sparsification, one outlier per 4 (out_n = 2 per 8, or 0), two inliers per 4; stored dense
 
 
 def gran_keep(n: int) -> int:

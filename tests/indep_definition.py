@@ -69,9 +69,15 @@ def decompose_dense(W_bits, out_n, pair, block, rule_floor, col_weight=None):
     A = np.abs(W)
     if col_weight is not None:
         A = (A.astype(np.float32) * np.asarray(col_weight, dtype=np.float32)[None, :]).astype(np.float32).astype(np.float64)
-    mask_out = top_mask(A.reshape(N, K // 8, 8), out_n).reshape(N, K) if out_n else np.zeros((N, K), bool)
+    if pair == "3of4":                    # S-Vectors of 4: the largest of every 4 is the outlier, the next two stay
+        mask_out = top_mask(A.reshape(N, K // 4, 4), 1).reshape(N, K) if out_n else np.zeros((N, K), bool)
+    else:
+        mask_out = top_mask(A.reshape(N, K // 8, 8), out_n).reshape(N, K) if out_n else np.zeros((N, K), bool)
     R = np.where(mask_out, 0.0, A)
-    if pair is None:                      # no pruning: every non-outlier value stays an inlier
+    if pair == "3of4":
+        keys = np.where(mask_out, -1.0, A).reshape(N, K // 4, 4)
+        slots = top_mask(keys, 3 - (1 if out_n else 0)).reshape(N, K)
+    elif pair is None:                      # no pruning: every non-outlier value stays an inlier
         slots = np.ones((N, K), bool)
     elif pair is not True and pair is not False:   # an integer n: keep the n most significant of every 8 in total
         keys = np.where(mask_out, -1.0, A).reshape(N, K // 8, 8)

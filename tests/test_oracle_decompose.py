@@ -531,3 +531,34 @@ def test_values_on_rounding_boundaries_match_the_independent_definition(rule, bl
         W_in, _ = so.dequant_weights(p)
         assert np.array_equal(W_in, decompose_dense(Xb, 0, None, block, tag)[0])
         assert np.array_equal(W_in, A_i)          # un-pruned weights without outliers = the activation 4-bit quantizer
+
+
+@pytest.mark.parametrize("out_n,block,rule", [(2, 32, so.SCALE_OCP_FLOOR), (0, 32, so.SCALE_CEIL_NOSAT), (2, 64, so.SCALE_OCP_FLOOR)])
+def test_s_vectors_of_4_match_independent_definition(out_n, block, rule):
+    """3:4 = 1:4 + 2:4: per 4 consecutive K the largest is the outlier, the next two are inliers, the smallest goes"""
+    cfg = so.Config(out_n, so.GRAN_3OF4, block, rule)
+    for seed, cw in ((4, None), (5, lognormal_channel_weight(512, 11))):
+        Wb = tiny_W(40, 512, seed)
+        p = so.decompose(Wb, cfg, cw)
+        W_in, W_out = so.dequant_weights(p)
+        ref_in, ref_out, slots, mask_out = decompose_dense(Wb, out_n, "3of4", block, rule == so.SCALE_OCP_FLOOR, cw)
+        assert np.array_equal(W_out, ref_out) and np.array_equal(W_in, ref_in)
+        assert ((W_out != 0).reshape(40, 128, 4).sum(-1) <= (1 if out_n else 0)).all()
+        assert ((slots & ~mask_out).reshape(40, 128, 4).sum(-1) == 3 - (1 if out_n else 0)).all()
+        if out_n:
+            assert (p.out_idx[..., 0] < 4).all() and (p.out_idx[..., 1] >= 4).all()
+    with pytest.raises(ValueError):
+        so.decompose(tiny_W(8, 128, 0), so.Config(1, so.GRAN_3OF4, 32, so.SCALE_OCP_FLOOR))
+
+
+def test_s_vectors_of_4_hand_example():
+    """one row, magnitudes 1..8 in two groups of 4: (4, 1, 3, 2 | 5, 8, 6, 7) -> outliers 4 and 8, dropped 1 and 5"""
+    import torch
+    row = np.array([4.0, 1.0, 3.0, 2.0, 5.0, 8.0, 6.0, 7.0] * 8) * 0.0625
+    W = np.tile(row, (2, 1))
+    Wb = sdq_synth.bf16_bits(torch.from_numpy(W).to(torch.bfloat16))
+    p = so.decompose(Wb, so.Config(2, so.GRAN_3OF4, 32, so.SCALE_CEIL_NOSAT))
+    W_in, W_out = so.dequant_weights(p)
+    assert (p.out_idx == np.array([0, 5])).all()
+    assert np.array_equal(W_out[0, :8], np.array([4.0, 0, 0, 0, 0, 8.0, 0, 0]) * 0.0625)
+    assert np.array_equal(W_in[0, :8] != 0, np.array([0, 0, 1, 1, 0, 0, 1, 1], bool))
