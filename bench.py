@@ -611,6 +611,7 @@ def run_sweep(args):
                       ("4:8 pair-wise + 1:8, E4M3 scales per 32", sdq.Config(1, sdq.GRAN_PAIR, 32, sdq.SCALE_UE4M3)),
                       ("6:8 = 2:8 + 4:8 at any position", sdq.Config(2, sdq.gran_keep(6), 32, 0)),
                       ("7:8 = 1:8 + 6:8", sdq.Config(1, sdq.gran_keep(7), 32, 0)),
+                      ("3:4 = 1:4 + 2:4 (S-Vectors of 4)", sdq.Config(2, sdq.GRAN_3OF4, 32, 0)),
                       ("8:8 = 1:8 + 7:8", sdq.Config(1, sdq.GRAN_DENSE, 32, 0)),
                       ("8:8 dense 4-bit, no outliers", sdq.Config(0, sdq.GRAN_DENSE, 32, 0))):
         Y = sdq.sdq_linear(sdq.sdq_quantize_act(X, cfg), sdq.sdq_decompose(W, cfg), f32=True)

@@ -40,6 +40,7 @@ typedef enum {
 
 enum { SDQ_GRAN_PAIR = 0, SDQ_GRAN_ELEM = 1, SDQ_GRAN_DENSE = 2 }; /* inlier pattern            */
 #define SDQ_GRAN_KEEP(n) (2 + (8 - (n)))  /* n:8 sparsification, n = 2..8; SDQ_GRAN_KEEP(8) == SDQ_GRAN_DENSE */
+#define SDQ_GRAN_3OF4 9                   /* S-Vectors of 4: 3:4 = 1:4 outliers + 2:4 inliers                 */
 enum { SDQ_SCALE_OCP_FLOOR = 0, SDQ_SCALE_CEIL_NOSAT = 1, SDQ_SCALE_UE4M3 = 2 }; /* Q-Vector scale rule */
 
 /* "pattern, formats" of the decomposition (Section 5, Stages 1-3).
@@ -56,7 +57,10 @@ enum { SDQ_SCALE_OCP_FLOOR = 0, SDQ_SCALE_CEIL_NOSAT = 1, SDQ_SCALE_UE4M3 = 2 };
  *              significant are the outliers and the other n - out_n the inliers, at whatever positions
  *              they have (the evaluation's flexible N:M configurations, e.g. 7:8 = 1:8 + 6:8; largest
  *              first, ties to the lower k); stored and executed like the dense pattern, the dropped
- *              positions holding +0.  The dense 4-bit tensor-core kind has one scale per 32 K only, so
+ *              positions holding +0.  SDQ_GRAN_3OF4 (the evaluation's 3:4 = 1:4 + 2:4): per 4 consecutive K
+ *              the most significant value is the outlier (out_n must be 2, i.e. two per 8, or 0), the
+ *              next two stay inliers, the last is dropped; stored and executed like the dense pattern.
+ *              The dense 4-bit tensor-core kind has one scale per 32 K only, so
  *              these patterns require in_block = 32 (with 64 every call returns SDQ_ERR_UNSUPPORTED).
  *   in_block   Q-Vector length: logical K sharing one E8M0 scale, for W_i and for the 4-bit
  *              activations: 64 or 32.  Both are executed by sdq_linear (64: kind::mxf4 .block32, the
@@ -150,7 +154,8 @@ sdq_status_t sdq_decompose(const void* W_bf16, int64_t N, int64_t K, int64_t ldw
  * k; a pair's score is the fp32 sum of its two products) instead of |w|.  Values, scales and formats
  * are untouched by the metric.
  *   col_weight (device) [K] fp32, 16-byte aligned, every entry finite and >= 0 -- typically the norm
- *   of input channel k over a calibration set.  NULL gives sdq_decompose exactly.
+ *   of input channel k over a calibration set (any per-channel saliency weight fits: an error-based
+ *   saliency w^2 / [H^-1]_kk ranks like |w| * c[k] with c[k] = [H^-1]_kk^(-1/2)).  NULL gives sdq_decompose exactly.
  *   Errors as sdq_decompose; a negative, infinite or NaN channel weight reports NONFINITE. */
 sdq_status_t sdq_decompose_metric(const void* W_bf16, int64_t N, int64_t K, int64_t ldw, const sdq_config_t* cfg,
                                   const float* col_weight, void* packed_buf, size_t packed_bytes,

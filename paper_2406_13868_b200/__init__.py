@@ -16,6 +16,7 @@ import torch
 from .build import LIB, build
 
 GRAN_PAIR, GRAN_ELEM, GRAN_DENSE = 0, 1, 2
+GRAN_3OF4 = 9      # S-Vectors of 4: 3:4 = 1:4 outliers (out_n = 2 per 8, or 0) + 2:4 inliers, stored and run like the dense pattern
 
 
 def gran_keep(n: int) -> int:

@@ -39,6 +39,16 @@ __device__ __forceinline__ void select_outliers(const uint32_t (&key)[8], int ou
   }
 }
 
+// S-Vectors of 4: the most significant of positions 0..3 and of positions 4..7 (ties to the lower index)
+__device__ __forceinline__ void select_outliers_per_4(const uint32_t (&key)[8], int& o0, int& o1) {
+  o0 = 0; o1 = 4;
+#pragma unroll
+  for (int i = 1; i < 4; ++i) {
+    if (key[i] > key[o0]) o0 = i;
+    if (key[4 + i] > key[o1]) o1 = 4 + i;
+  }
+}
+
 __device__ __forceinline__ void load_group(const __nv_bfloat16* w, uint32_t (&bits)[8]) {
   const uint4 v = *reinterpret_cast<const uint4*>(w);
   const uint32_t r[4] = {v.x, v.y, v.z, v.w};
@@ -84,6 +94,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
   const __nv_bfloat16* wrow = W + n * ldw;
   __shared__ uint32_t s_red[4], s_red_in[4];
   __shared__ int s_e, s_t;
+  const bool sv4 = cfg.in_gran == SDQ_GRAN_3OF4;          // S-Vectors of 4: one outlier and two inliers per 4
   const bool ue = cfg.scale_rule == SDQ_SCALE_UE4M3;     // two-level scaling with E4M3 Q-Vector scales (pair-wise, block 32)
 
   // ---- pass 1: largest outlier magnitude of the row (and, for two-level scaling, largest kept inlier), non-finite check
@@ -99,7 +110,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     uint32_t skey[8];
     bad |= selection_keys(key, colw, g, skey);
     int o0, o1;
-    select_outliers(skey, out_n, o0, o1);
+    if (sv4 && out_n) select_outliers_per_4(skey, o0, o1); else select_outliers(skey, out_n, o0, o1);
     if (o0 >= 0) okey_max = max(okey_max, key[o0]);
     if (o1 >= 0) okey_max = max(okey_max, key[o1]);
     if (ue) {
@@ -133,7 +144,8 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
   const uint32_t r = (uint32_t)(n % TILE_ROWS);
   const int T1 = (int)(K / K1), T2 = (int)(K / K2);
   const bool b32 = cfg.in_block == 32, dense = cfg.in_gran >= SDQ_GRAN_DENSE;
-  const int keep_in = 10 - cfg.in_gran - out_n;     // dense family: inliers kept per S-Vector (8 - out_n without Stage 1)
+  // dense family: inliers kept per S-Vector (8 - out_n without Stage 1; S-Vectors of 4: 3 minus the outlier)
+  const int keep_in = sv4 ? (out_n ? 2 : 3) : 10 - cfg.in_gran - out_n;
   const int wib = wi_bytes(b32, dense);
   uint8_t* wi_base = blob + off.wi + (size_t)rt * T2 * wib;
   uint8_t* wo_base = blob + off.wo + (size_t)rt * T1 * WO_BYTES;
@@ -156,7 +168,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     uint32_t skey[8];
     selection_keys(key, colw, g, skey);
     int o0, o1;
-    select_outliers(skey, out_n, o0, o1);
+    if (sv4 && out_n) select_outliers_per_4(skey, o0, o1); else select_outliers(skey, out_n, o0, o1);
     const int k1 = g >> 4, k2 = g >> 5;
     uint8_t* wi = wi_base + (size_t)k2 * wib;
     uint8_t* wo = wo_base + (size_t)k1 * WO_BYTES;
@@ -172,7 +184,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
         int before = 0;
 #pragma unroll
         for (int j = 0; j < 8; ++j)
-          before += (j != o0 && j != o1 && (skey[j] > skey[i] || (skey[j] == skey[i] && j < i))) ? 1 : 0;
+          before += (j != o0 && j != o1 && (!sv4 || (j >> 2) == (i >> 2)) && (skey[j] > skey[i] || (skey[j] == skey[i] && j < i))) ? 1 : 0;
         if (i == o0 || i == o1 || before >= keep_in) gone |= 1u << i;
         else ikey = max(ikey, key[i]);
       }
@@ -308,8 +320,9 @@ export_packed_kernel(const uint8_t* __restrict__ blob, int64_t N, int64_t K, sdq
 using namespace sdq;
 
 static bool cfg_ok(const sdq_config_t* c) {
-  return c && c->out_n >= 0 && c->out_n <= 2 && c->in_gran >= 0 && c->in_gran <= SDQ_GRAN_KEEP(2) &&
-         (c->in_gran < SDQ_GRAN_DENSE || 10 - c->in_gran > c->out_n) &&
+  return c && c->out_n >= 0 && c->out_n <= 2 && c->in_gran >= 0 && c->in_gran <= SDQ_GRAN_3OF4 &&
+         (c->in_gran < SDQ_GRAN_DENSE || c->in_gran == SDQ_GRAN_3OF4 || 10 - c->in_gran > c->out_n) &&
+         (c->in_gran != SDQ_GRAN_3OF4 || c->out_n != 1) &&
          (c->in_block == 32 || c->in_block == 64) && c->scale_rule >= SDQ_SCALE_OCP_FLOOR && c->scale_rule <= SDQ_SCALE_UE4M3;
 }
 // valid configurations this kernel set does not carry out

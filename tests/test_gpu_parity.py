@@ -164,6 +164,13 @@ def test_n_of_8_sparsification_with_outliers_and_inliers_at_any_position(n, M, N
     run_case(M, N, K, 1500 + 10 * n + M, out_n=out_n, rule=rule, block=32, gran=so.gran_keep(n))
 
 
+@pytest.mark.parametrize("M,N,K,out_n,rule", [(8, 256, 256, 2, 0), (1, 512, 2048, 2, 0), (33, 128, 768, 0, 1), (129, 256, 512, 2, 1),
+                                              (520, 6400, 256, 2, 0)])
+def test_s_vectors_of_4(M, N, K, out_n, rule):
+    """SDQ_GRAN_3OF4 (3:4 = 1:4 + 2:4): packed arrays bit-exact, product through the dense 4-bit MMA"""
+    run_case(M, N, K, 2600 + M, out_n=out_n, rule=rule, block=32, gran=so.GRAN_3OF4)
+
+
 def test_dense_inliers_one_hot_readback_and_workspace_split():
     m = sdq()
     cfg = m.Config(1, m.GRAN_DENSE, 32, 0)
@@ -458,7 +465,7 @@ def test_activation_quantizer_row_lengths(M, K, rule, block):
         assert np.array_equal(ae[name], getattr(oq, name)), name
 
 
-@pytest.mark.parametrize("gran,block", [(1, 64), (0, 32), (0, 64), (2, 32), (3, 32)])
+@pytest.mark.parametrize("gran,block", [(1, 64), (0, 32), (0, 64), (2, 32), (3, 32), (9, 32)])
 @pytest.mark.parametrize("out_n", [0, 1, 2])
 def test_product_metric_packer(gran, block, out_n):
     """sdq_decompose_metric: selections by |w| * c[k]; packed arrays bit-exact against the oracle for the tensor-core
@@ -469,6 +476,11 @@ def test_product_metric_packer(gran, block, out_n):
     cfg = m.Config(out_n, gran, block, 0)
     oc = so.Config(out_n, gran, block, 0)
     W = sdq_synth.make_weight(N, K, 40 + out_n)
+    if gran == m.GRAN_3OF4 and out_n == 1:          # one outlier per 4 is two per 8: there is no such configuration
+        with pytest.raises(m.SdqError) as ei:
+            m.sdq_decompose(W.cuda(), cfg)
+        assert ei.value.code == 1
+        return
     rng = np.random.default_rng(17)
     c = np.exp(rng.normal(0.0, 1.0, K)).astype(np.float32)
     c[rng.integers(0, K, 12)] *= 30.0
