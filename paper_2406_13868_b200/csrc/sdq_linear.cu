@@ -38,7 +38,9 @@ constexpr int MAX_SLOTS = 16;
 constexpr int SL_A = 0;                        // WI record (A_in | E_in | SFA_in) or WO record (A_out | E_out)
 constexpr int RING_BYTES = 225280;             // largest ring: nslot slots of slot_bytes each
 constexpr int SM_TAIL = 4096 + 640 + 128;      // epilogue transpose buffer (16 tokens x 128 features bf16) + barriers + slack
-constexpr int LIN_SMEM_MAX = RING_BYTES + SM_TAIL;
+constexpr int SM_TAIL_B32 = 640 + 128;         // many tokens, one scale per 32 K: five 46080-byte slots leave no room for the
+                                               // transpose buffer; that instantiation stores from registers
+constexpr int LIN_SMEM_MAX = 5 * 46080 + SM_TAIL_B32;   // the largest request
 
 // TMEM columns: accumulator at 0 (n_tile columns, tokens), then metadata / scales.
 // Runtime geometry: 84 columns at `meta_col`:
@@ -100,8 +102,9 @@ sdq_linear_kernel(const LinearParams p)       // many tokens: 13 warps, four of 
   // the transpose buffer and the barriers follow the ring (many tokens: 5 x 45056, or 4 x 46080 with one scale per 32 K)
   static_assert(!(FLEX && (B32 || DENSE)) && !(B32 && DENSE), "B32 and DENSE name many-token instantiations");
   constexpr bool S32 = B32 || DENSE;                       // many tokens with one scale per 32 K
-  constexpr uint32_t SLOT_FIXED = DENSE ? 52224u : (B32 ? 46080u : 45056u), NSLOT_FIXED = S32 ? 4u : 5u;
-  const uint32_t SM_STG = FLEX ? (uint32_t)p.ring_bytes : (S32 ? NSLOT_FIXED * SLOT_FIXED : (uint32_t)RING_BYTES), SM_BARS = SM_STG + 4096;
+  constexpr uint32_t SLOT_FIXED = DENSE ? 52224u : (B32 ? 46080u : 45056u), NSLOT_FIXED = DENSE ? 4u : 5u;
+  // the transpose buffer and then the barriers follow the ring (B32: no transpose buffer)
+  const uint32_t SM_STG = FLEX ? (uint32_t)p.ring_bytes : NSLOT_FIXED * SLOT_FIXED, SM_BARS = B32 ? SM_STG : SM_STG + 4096;
   const uint32_t TM_I = FLEX ? (uint32_t)p.meta_col : 256u, TM_EO = TM_I + 64, TM_SFA_OUT = TM_I + 72, TM_SFB_OUT = TM_I + 76;
   const uint32_t tmem_cols = FLEX ? (uint32_t)p.tmem_cols : 512u;
   uint64_t* full = reinterpret_cast<uint64_t*>(sm + SM_BARS);
@@ -457,34 +460,47 @@ sdq_linear_kernel(const LinearParams p)       // many tokens: 13 warps, four of 
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(acc_empty);
-        // transpose through shared memory, 8 tokens at a time per group: [8 tokens][128 features] bf16, then one 16-byte
-        // store per thread (full 256 B rows)
-        uint16_t* stg = reinterpret_cast<uint16_t*>(sm + SM_STG) + grp * 1024u;
-        __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(p.Y);
         const int g0 = 128 * (int)grp;
+        if constexpr (B32) {
+          // no room for a transpose buffer beside five slots: every thread stores its row's 128 tokens itself (for one
+          // token the 32 lanes of a warp write 64 contiguous bytes); measured 2-4 % slower than the transposed stores
+          // below, which the fifth slot more than pays for
+          uint16_t* Y = reinterpret_cast<uint16_t*>(p.Y) + n0 + q * 32 + lane;
 #pragma unroll
-        for (int c0 = 0; c0 < 128; c0 += 8) {
-          if (g0 + c0 < n_valid) {                  // uniform over the four warps of the group
+          for (int j = 0; j < 64; ++j) {
+            const int t = g0 + 2 * j;
+            if (t >= n_valid) break;                  // uniform over the warp
+            uint32_t lo = pk[j] << 16, hi = pk[j] & 0xFFFF0000u;
+            if (p.tw) {
+              // two-level scaling: multiplying the rounded value by the power of two is the rounding of the multiplied
+              // value, so the factors go in here, after TMEM has been handed back
+              lo = __float_as_uint(__uint_as_float(lo) * pow2i(twr + __ldg(p.tx + m0 + t)));
+              if (t + 1 < n_valid) hi = __float_as_uint(__uint_as_float(hi) * pow2i(twr + __ldg(p.tx + m0 + t + 1)));
+            }
+            Y[(m0 + t) * p.ldy] = (uint16_t)(lo >> 16);
+            if (t + 1 < n_valid) Y[(m0 + t + 1) * p.ldy] = (uint16_t)(hi >> 16);
+          }
+        } else {
+          // transpose through shared memory, 8 tokens at a time per group: [8 tokens][128 features] bf16, then one
+          // 16-byte store per thread (full 256 B rows)
+          uint16_t* stg = reinterpret_cast<uint16_t*>(sm + SM_STG) + grp * 1024u;
+          __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(p.Y);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              uint32_t lo = pk[c0 / 2 + j] << 16, hi = pk[c0 / 2 + j] & 0xFFFF0000u;
-              if (p.tw) {
-                // two-level scaling: multiplying the rounded value by the power of two is the rounding of the multiplied
-                // value, so the factors go in here, after TMEM has been handed back
-                const int t = g0 + c0 + 2 * j;
-                if (t < n_valid) lo = __float_as_uint(__uint_as_float(lo) * pow2i(twr + __ldg(p.tx + m0 + t)));
-                if (t + 1 < n_valid) hi = __float_as_uint(__uint_as_float(hi) * pow2i(twr + __ldg(p.tx + m0 + t + 1)));
+          for (int c0 = 0; c0 < 128; c0 += 8) {
+            if (g0 + c0 < n_valid) {                  // uniform over the four warps of the group
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                stg[(2 * j) * 128 + q * 32 + lane] = (uint16_t)(pk[c0 / 2 + j] & 0xFFFFu);
+                stg[(2 * j + 1) * 128 + q * 32 + lane] = (uint16_t)(pk[c0 / 2 + j] >> 16);
               }
-              stg[(2 * j) * 128 + q * 32 + lane] = (uint16_t)(lo >> 16);
-              stg[(2 * j + 1) * 128 + q * 32 + lane] = (uint16_t)(hi >> 16);
+              ptx::named_bar_sync(1 + grp, 128);
+              const uint32_t tok = et >> 4, seg = et & 15;
+              if (g0 + c0 + (int)tok < n_valid) {
+                const uint4 w = *reinterpret_cast<const uint4*>(stg + tok * 128 + seg * 8);
+                *reinterpret_cast<uint4*>(Y + (m0 + g0 + c0 + tok) * p.ldy + n0 + seg * 8) = w;
+              }
+              ptx::named_bar_sync(1 + grp, 128);       // the buffer is rewritten by the next chunk
             }
-            ptx::named_bar_sync(1 + grp, 128);
-            const uint32_t tok = et >> 4, seg = et & 15;
-            if (g0 + c0 + (int)tok < n_valid) {
-              const uint4 w = *reinterpret_cast<const uint4*>(stg + tok * 128 + seg * 8);
-              *reinterpret_cast<uint4*>(Y + (m0 + g0 + c0 + tok) * p.ldy + n0 + seg * 8) = w;
-            }
-            ptx::named_bar_sync(1 + grp, 128);       // the buffer is rewritten by the next chunk
           }
         }
         continue;
@@ -793,7 +809,9 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   // much shared memory as its stages take (so that small CTAs share an SM) and skips the slot-release traffic
   const int T1 = p.out_n ? (int)(P->K / K1) : 0, T2 = (int)(P->K / K2);
   const int stages_per_tile = (T2 + p.ksplit - 1) / p.ksplit + (T1 + p.ksplit - 1) / p.ksplit;
-  int max_slots = RING_BYTES / p.slot_bytes;
+  // many tokens without K split: the instantiations with compile-time geometry (five ring slots; four with dense inliers)
+  const bool many = p.n_tile == 256 && p.ksplit == 1;
+  int max_slots = many ? (p.dense ? 4 : 5) : RING_BYTES / p.slot_bytes;
   if (p.cluster_ks > 1 && p.total_tiles > sm_count) {
     // cluster split K with more CTAs than SMs (few tokens, one tile per CTA): the grid is one wave only if two CTAs
     // share an SM, so a ring gets half of an SM's shared memory (228 KB, 1 KB of it reserved per CTA)
@@ -819,7 +837,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   p.meta_col = p.n_tile < 32 ? 32 : p.n_tile;
   int cols = p.meta_col + (int)TM_META_COLS;
   p.tmem_cols = cols <= 128 ? 128 : (cols <= 256 ? 256 : 512);
-  const int smem = p.ring_bytes + SM_TAIL;
+  const int smem = p.ring_bytes + (many && p.b32 && !p.dense ? SM_TAIL_B32 : SM_TAIL);
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3((unsigned)grid_x);
   lc.blockDim = dim3(LIN_THREADS);   // the many-token instantiations get LIN_THREADS_MANY below
@@ -840,7 +858,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   }
   lc.attrs = attr;
   lc.numAttrs = na;
-  const bool flex = !(p.n_tile == 256 && p.ksplit == 1 && p.nslot == (p.b32 ? 4 : 5) && p.release == 1);
+  const bool flex = !many;
   if (!flex) lc.blockDim = dim3(LIN_THREADS_MANY);
   cudaError_t le;
   if (flex) le = f32 ? cudaLaunchKernelEx(&lc, sdq_linear_kernel<true, true, false, false>, p) : cudaLaunchKernelEx(&lc, sdq_linear_kernel<false, true, false, false>, p);
