@@ -440,7 +440,11 @@ def run_case(args):
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
     cfg = sdq.Config(1, sdq.GRAN_PAIR, 64, sdq.SCALE_OCP_FLOOR)
-    if args.case == "gemm_prefill_dense":        # 8:8 = 1:8 FP8 outliers + dense MXFP4 inliers
+    if args.case == "gemm_prefill_b32":          # one scale per 32 K
+        cfg = sdq.Config(1, sdq.GRAN_PAIR, 32, sdq.SCALE_OCP_FLOOR)
+    elif args.case == "gemm_prefill_e4m3":       # E4M3 scale codes per 32 K, power-of-two row / token factors
+        cfg = sdq.Config(1, sdq.GRAN_PAIR, 32, sdq.SCALE_UE4M3)
+    elif args.case == "gemm_prefill_dense":      # 8:8 = 1:8 FP8 outliers + dense MXFP4 inliers
         cfg = sdq.Config(1, sdq.GRAN_DENSE, 32, sdq.SCALE_OCP_FLOOR)
     elif args.case == "gemm_prefill_mxfp4":      # no outliers, no pruning: a plain block-scaled 4-bit GEMM
         cfg = sdq.Config(0, sdq.GRAN_DENSE, 32, sdq.SCALE_OCP_FLOOR)
@@ -624,7 +628,7 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--sweep", action="store_true", help="measure the other configurations (OPT FFN outlier sweep, whole-model pass) and exit")
-    ap.add_argument("--case", default=None, choices=["gemm_prefill", "gemm_prefill_dense", "gemm_prefill_mxfp4", "gemm_decode", "quant"],
+    ap.add_argument("--case", default=None, choices=["gemm_prefill", "gemm_prefill_b32", "gemm_prefill_e4m3", "gemm_prefill_dense", "gemm_prefill_mxfp4", "gemm_decode", "quant"],
                     help="run only a small single-kernel case (for profiler captures) and exit")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
