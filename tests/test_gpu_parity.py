@@ -319,6 +319,26 @@ def test_values_on_rounding_boundaries(rule, block):
     assert m.device_status() == 0
 
 
+def test_error_order_of_the_configurations_on_the_gpu():
+    """the whole CUDA path against the unquantized product (fp64 on the GPU) on a synthetic layer: outliers lower the
+    error, 7:8 = 1:8 + 6:8 beats dense 4-bit, 50 % sparsity costs most, E4M3 scales help"""
+    m = sdq()
+    M, N, K = 256, 1024, 4096
+    X = sdq_synth.make_act(M, K, 2701).cuda()
+    W = sdq_synth.make_weight(N, K, 2702).cuda()
+    ref = X.double() @ W.double().T
+
+    def err(cfg):
+        y = m.sdq_linear(m.sdq_quantize_act(X, cfg), m.sdq_decompose(W, cfg), f32=True)
+        return float((y.double() - ref).norm() / ref.norm())
+    e48_0, e48_1, e48_2 = (err(m.Config(n, m.GRAN_PAIR, 32, 0)) for n in (0, 1, 2))
+    e78, e88, e88_0 = err(m.Config(1, m.gran_keep(7), 32, 0)), err(m.Config(1, m.GRAN_DENSE, 32, 0)), err(m.Config(0, m.GRAN_DENSE, 32, 0))
+    e34, e_ue = err(m.Config(2, m.GRAN_3OF4, 32, 0)), err(m.Config(1, m.GRAN_PAIR, 32, m.SCALE_UE4M3))
+    assert m.device_status() == 0
+    assert e48_0 > e48_1 > e48_2 and e88 < e78 < e48_2 and e78 < e88_0 and e88 < e34 < e48_1 and e_ue < e48_1, \
+        (e48_0, e48_1, e48_2, e78, e88, e88_0, e34, e_ue)
+
+
 def test_one_hot_readback_512_tokens():
     m = sdq()
     cfg = m.Config()

@@ -122,6 +122,28 @@ def test_error_against_unquantized_product_is_small():
     assert np.corrcoef(Y.ravel(), ref.ravel())[0, 1] > 0.8
 
 
+def test_error_order_of_the_configurations():
+    """the paper's qualitative findings on the synthetic layer: outlier extraction lowers the output error, dropping one
+    of eight values costs little, 50 % sparsity costs most, and 1:8 outliers + 6:8 inliers beat plain dense 4-bit"""
+    Wb = sdq_synth.bf16_bits(sdq_synth.make_weight(96, 2048, 21))
+    Xb = sdq_synth.bf16_bits(sdq_synth.make_act(16, 2048, 22))
+    W = torch.from_numpy(Wb.view(np.int16)).view(torch.bfloat16).double().numpy()
+    X = torch.from_numpy(Xb.view(np.int16)).view(torch.bfloat16).double().numpy()
+    ref = X @ W.T
+
+    def err(cfg):
+        return np.linalg.norm(so.linear(so.quantize_act(Xb, cfg), so.decompose(Wb, cfg)) - ref) / np.linalg.norm(ref)
+    e48_0, e48_1, e48_2 = (err(so.Config(n, so.GRAN_PAIR, 32, 0)) for n in (0, 1, 2))
+    e78, e88, e88_0 = err(so.Config(1, so.gran_keep(7), 32, 0)), err(so.Config(1, so.GRAN_DENSE, 32, 0)), err(so.Config(0, so.GRAN_DENSE, 32, 0))
+    e34 = err(so.Config(2, so.GRAN_3OF4, 32, 0))
+    e_ue = err(so.Config(1, so.GRAN_PAIR, 32, so.SCALE_UE4M3))
+    assert e48_0 > e48_1 > e48_2
+    assert e88 < e78 < e48_2
+    assert e78 < e88_0                      # the headline claim: 7:8 = 1:8 + 6:8 beats dense 4-bit quantization
+    assert e88 < e34 < e48_1
+    assert e_ue < e48_1
+
+
 def golden():
     vals = {}
     with open(os.path.join(os.path.dirname(__file__), "golden", "paper_arithmetic.txt")) as f:
