@@ -41,6 +41,10 @@
    Stage 2 takes the most significant of every 4 as the outlier (out_n = 2 per 8 consecutive K; out_n = 0: none), the
    others stay inliers at whatever positions they have; stored like the dense pattern. */
 #define SDQO_GRAN_3OF4 9
+/* Stage 2 order (decomposition-stage study): "Large" takes the most significant values as outliers (the method),
+   "Small" the least significant ones (the study's control: the wrong values in high precision) */
+#define SDQO_ORDER_LARGE 0
+#define SDQO_ORDER_SMALL 1
 #define SDQO_SCALE_OCP_FLOOR 0  /* E = floor(log2 amax) - 2   (OCP MX rule, may saturate in (6,8)) */
 #define SDQO_SCALE_CEIL_NOSAT 1 /* E = smallest integer with amax <= 6 * 2^E                        */
 /* Two-level scaling with 8-bit floating-point Q-Vector scales (the quantization-stage study: scale factors in
@@ -55,6 +59,7 @@ typedef struct {
   int in_gran;    /* SDQO_GRAN_*                                                */
   int in_block;   /* Q-Vector: logical K per inlier / 4-bit activation scale (32|64) */
   int scale_rule; /* SDQO_SCALE_*                                               */
+  int out_order;  /* SDQO_ORDER_*: which end of the metric's order Stage 2 takes     */
 } sdqo_config;
 
 /* ------------------------------------------------------------------ number formats */
@@ -199,6 +204,7 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
     for (int64_t k = 0; k < K; ++k)
       if (!(col_weight[k] >= 0.0f) || isinf(col_weight[k])) return -3;
   if (cfg->out_n < 0 || cfg->out_n > 2) return -1;
+  if (cfg->out_order != SDQO_ORDER_LARGE && cfg->out_order != SDQO_ORDER_SMALL) return -1;
   if (cfg->in_block != 32 && cfg->in_block != 64) return -1;
   if (cfg->scale_rule < 0 || cfg->scale_rule > SDQO_SCALE_UE4M3 || (cfg->scale_rule == SDQO_SCALE_UE4M3 && !in_texp)) return -1;
   if (cfg->in_gran < 0 || cfg->in_gran > SDQO_GRAN_3OF4) return -1;
@@ -236,12 +242,13 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
           int best = -1;
           for (int i = sub * sv; i < (sub + 1) * sv; ++i) {
             if (is_out[8 * g + i]) continue;
-            if (best < 0 || sig[8 * g + i] > sig[8 * g + best]) best = i;
+            if (best < 0 || (cfg->out_order == SDQO_ORDER_SMALL ? sig[8 * g + i] < sig[8 * g + best]
+                                                                : sig[8 * g + i] > sig[8 * g + best])) best = i;
           }
           is_out[8 * g + best] = 1;
           chosen[nc++] = best;
         }
-      if (on == 2 && chosen[0] > chosen[1]) { int t = chosen[0]; chosen[0] = chosen[1]; chosen[1] = t; }
+      if (nc == 2 && chosen[0] > chosen[1]) { int t = chosen[0]; chosen[0] = chosen[1]; chosen[1] = t; }
       for (int t = 0; t < on; ++t) {
         out_idx[(n * G8 + g) * on + t] = (uint8_t)chosen[t];
         double a = fabs(sdqo_bf16_to_double(w[8 * g + chosen[t]]));

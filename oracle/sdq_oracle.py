@@ -28,6 +28,7 @@ def gran_keep(n: int) -> int:
     assert 2 <= n <= 8
     return 2 + (8 - n)
 SCALE_OCP_FLOOR, SCALE_CEIL_NOSAT, SCALE_UE4M3 = 0, 1, 2
+ORDER_LARGE, ORDER_SMALL = 0, 1
 
 
 def build(force: bool = False) -> str:
@@ -42,7 +43,7 @@ def build(force: bool = False) -> str:
 
 class _Cfg(ctypes.Structure):
     _fields_ = [("out_n", ctypes.c_int), ("in_gran", ctypes.c_int), ("in_block", ctypes.c_int),
-                ("scale_rule", ctypes.c_int)]
+                ("scale_rule", ctypes.c_int), ("out_order", ctypes.c_int)]
 
 
 @dataclass(frozen=True)
@@ -51,9 +52,10 @@ class Config:
     in_gran: int = GRAN_PAIR
     in_block: int = 64
     scale_rule: int = SCALE_OCP_FLOOR
+    out_order: int = 0          # ORDER_LARGE; ORDER_SMALL takes the least significant values as outliers (study control)
 
     def c(self) -> _Cfg:
-        return _Cfg(self.out_n, self.in_gran, self.in_block, self.scale_rule)
+        return _Cfg(self.out_n, self.in_gran, self.in_block, self.scale_rule, self.out_order)
 
 
 _lib = None

@@ -58,7 +58,7 @@ def top_mask(keys, n):
     return mask
 
 
-def decompose_dense(W_bits, out_n, pair, block, rule_floor, col_weight=None):
+def decompose_dense(W_bits, out_n, pair, block, rule_floor, col_weight=None, small=False):
     """returns (W_in_hat, W_out_hat, mask_in_slots, mask_out) as dense [N, K] arrays; with col_weight the
     selections rank by the fp32 product |w| * c[k] instead of |w| (the values that get quantized do not change);
     rule_floor: True = OCP floor rule, False = ceil rule, "ue4m3" = two-level scaling with e4m3 scales;
@@ -69,10 +69,11 @@ def decompose_dense(W_bits, out_n, pair, block, rule_floor, col_weight=None):
     A = np.abs(W)
     if col_weight is not None:
         A = (A.astype(np.float32) * np.asarray(col_weight, dtype=np.float32)[None, :]).astype(np.float32).astype(np.float64)
+    Ao = -A if small else A               # "Small": the least significant values become the outliers
     if pair == "3of4":                    # S-Vectors of 4: the largest of every 4 is the outlier, the next two stay
-        mask_out = top_mask(A.reshape(N, K // 4, 4), 1).reshape(N, K) if out_n else np.zeros((N, K), bool)
+        mask_out = top_mask(Ao.reshape(N, K // 4, 4), 1).reshape(N, K) if out_n else np.zeros((N, K), bool)
     else:
-        mask_out = top_mask(A.reshape(N, K // 8, 8), out_n).reshape(N, K) if out_n else np.zeros((N, K), bool)
+        mask_out = top_mask(Ao.reshape(N, K // 8, 8), out_n).reshape(N, K) if out_n else np.zeros((N, K), bool)
     R = np.where(mask_out, 0.0, A)
     if pair == "3of4":
         keys = np.where(mask_out, -1.0, A).reshape(N, K // 4, 4)

@@ -562,3 +562,28 @@ def test_s_vectors_of_4_hand_example():
     assert (p.out_idx == np.array([0, 5])).all()
     assert np.array_equal(W_out[0, :8], np.array([4.0, 0, 0, 0, 0, 8.0, 0, 0]) * 0.0625)
     assert np.array_equal(W_in[0, :8] != 0, np.array([0, 0, 1, 1, 0, 0, 1, 1], bool))
+
+
+@pytest.mark.parametrize("gran,block,out_n", [(so.GRAN_PAIR, 64, 1), (so.GRAN_PAIR, 32, 2), (so.gran_keep(7), 32, 1)])
+def test_small_order_takes_the_least_significant_values(gran, block, out_n):
+    """the decomposition-stage study's "Small" control: outliers in ascending order of the metric"""
+    cfg = so.Config(out_n, gran, block, so.SCALE_OCP_FLOOR, so.ORDER_SMALL)
+    pair = True if gran == so.GRAN_PAIR else 7
+    for seed, cw in ((6, None), (7, lognormal_channel_weight(512, 13))):
+        Wb = tiny_W(40, 512, seed)
+        p = so.decompose(Wb, cfg, cw)
+        W_in, W_out = so.dequant_weights(p)
+        ref_in, ref_out, slots, mask_out = decompose_dense(Wb, out_n, pair, block, True, cw, small=True)
+        assert np.array_equal(W_out, ref_out) and np.array_equal(W_in, ref_in)
+    # magnitudes 1..8 in every group: "Small" picks 1 (and 2), "Large" 8 (and 7)
+    import torch
+    rng = np.random.default_rng(5)
+    mags = np.stack([rng.permutation(8) for _ in range(4 * 64)]).reshape(4, 512) + 1.0
+    Wb = sdq_synth.bf16_bits(torch.from_numpy(mags * 0.25).to(torch.bfloat16))
+    ps = so.decompose(Wb, so.Config(out_n, so.GRAN_PAIR, 64, 0, so.ORDER_SMALL))
+    pl = so.decompose(Wb, so.Config(out_n, so.GRAN_PAIR, 64, 0, so.ORDER_LARGE))
+    g = mags.reshape(4, 64, 8)
+    assert np.array_equal(np.sort(np.take_along_axis(g, ps.out_idx.astype(int), -1), -1), np.tile(np.arange(1, out_n + 1.0), (4, 64, 1)))
+    assert np.array_equal(np.sort(np.take_along_axis(g, pl.out_idx.astype(int), -1), -1), np.tile(np.arange(9 - out_n, 9.0), (4, 64, 1)))
+    with pytest.raises(ValueError):
+        so.decompose(Wb, so.Config(1, so.GRAN_PAIR, 64, 0, 2))
