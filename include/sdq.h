@@ -42,6 +42,7 @@ enum { SDQ_GRAN_PAIR = 0, SDQ_GRAN_ELEM = 1, SDQ_GRAN_DENSE = 2 }; /* inlier pat
 #define SDQ_GRAN_KEEP(n) (2 + (8 - (n)))  /* n:8 sparsification, n = 2..8; SDQ_GRAN_KEEP(8) == SDQ_GRAN_DENSE */
 #define SDQ_GRAN_3OF4 9                   /* S-Vectors of 4: 3:4 = 1:4 outliers + 2:4 inliers                 */
 enum { SDQ_SCALE_OCP_FLOOR = 0, SDQ_SCALE_CEIL_NOSAT = 1, SDQ_SCALE_UE4M3 = 2 }; /* Q-Vector scale rule */
+enum { SDQ_ORDER_LARGE = 0, SDQ_ORDER_SMALL = 1 };          /* Stage 2 takes the most / least significant values */
 
 /* "pattern, formats" of the decomposition (Section 5, Stages 1-3).
  *   out_n      outliers extracted per S-Vector of 8 consecutive K (Stage 2): 0, 1 or 2; stored as
@@ -81,6 +82,8 @@ typedef struct {
   int32_t in_gran;
   int32_t in_block;
   int32_t scale_rule;
+  int32_t out_order;   /* SDQ_ORDER_LARGE (the method) or SDQ_ORDER_SMALL: outliers in ascending order of the
+                          metric, the decomposition-stage study's control; sdq_quantize_act ignores it */
 } sdq_config_t;
 
 /* Host-side descriptor of a packed weight matrix (filled by sdq_decompose; plain data, may be

@@ -25,6 +25,7 @@ def gran_keep(n: int) -> int:
     assert 2 <= n <= 8
     return 2 + (8 - n)
 SCALE_OCP_FLOOR, SCALE_CEIL_NOSAT, SCALE_UE4M3 = 0, 1, 2
+ORDER_LARGE, ORDER_SMALL = 0, 1
 
 STATUS = ["ok", "invalid_arg", "shape", "alignment", "unsupported", "buffer_too_small", "nonfinite", "cuda", "timeout"]
 
@@ -38,10 +39,10 @@ class SdqError(RuntimeError):
 class Config(ctypes.Structure):
     """`pattern, formats` of the decomposition (sdq_config_t)."""
     _fields_ = [("out_n", ctypes.c_int32), ("in_gran", ctypes.c_int32), ("in_block", ctypes.c_int32),
-                ("scale_rule", ctypes.c_int32)]
+                ("scale_rule", ctypes.c_int32), ("out_order", ctypes.c_int32)]
 
-    def __init__(self, out_n=1, in_gran=GRAN_PAIR, in_block=64, scale_rule=SCALE_OCP_FLOOR):
-        super().__init__(out_n, in_gran, in_block, scale_rule)
+    def __init__(self, out_n=1, in_gran=GRAN_PAIR, in_block=64, scale_rule=SCALE_OCP_FLOOR, out_order=0):
+        super().__init__(out_n, in_gran, in_block, scale_rule, out_order)
 
 
 class _Packed(ctypes.Structure):

@@ -17,14 +17,14 @@ struct GroupSel {
   int o0, o1;        // outlier positions (ascending), -1 if absent
 };
 
-// positions of the out_n largest magnitudes, ties to the lower index
-__device__ __forceinline__ void select_outliers(const uint32_t (&key)[8], int out_n, int& o0, int& o1) {
+// positions of the out_n most (small: least) significant values, ties to the lower index
+__device__ __forceinline__ void select_outliers(const uint32_t (&key)[8], int out_n, bool small, int& o0, int& o1) {
   o0 = o1 = -1;
   if (out_n >= 1) {
     int b = 0;
 #pragma unroll
     for (int i = 1; i < 8; ++i)
-      if (key[i] > key[b]) b = i;
+      if (small ? key[i] < key[b] : key[i] > key[b]) b = i;
     o0 = b;
   }
   if (out_n >= 2) {
@@ -32,7 +32,7 @@ __device__ __forceinline__ void select_outliers(const uint32_t (&key)[8], int ou
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       if (i == o0) continue;
-      if (b < 0 || key[i] > key[b]) b = i;
+      if (b < 0 || (small ? key[i] < key[b] : key[i] > key[b])) b = i;
     }
     o1 = b;
     if (o0 > o1) { int t = o0; o0 = o1; o1 = t; }
@@ -40,12 +40,12 @@ __device__ __forceinline__ void select_outliers(const uint32_t (&key)[8], int ou
 }
 
 // S-Vectors of 4: the most significant of positions 0..3 and of positions 4..7 (ties to the lower index)
-__device__ __forceinline__ void select_outliers_per_4(const uint32_t (&key)[8], int& o0, int& o1) {
+__device__ __forceinline__ void select_outliers_per_4(const uint32_t (&key)[8], bool small, int& o0, int& o1) {
   o0 = 0; o1 = 4;
 #pragma unroll
   for (int i = 1; i < 4; ++i) {
-    if (key[i] > key[o0]) o0 = i;
-    if (key[4 + i] > key[o1]) o1 = 4 + i;
+    if (small ? key[i] < key[o0] : key[i] > key[o0]) o0 = i;
+    if (small ? key[4 + i] < key[o1] : key[4 + i] > key[o1]) o1 = 4 + i;
   }
 }
 
@@ -95,6 +95,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
   __shared__ uint32_t s_red[4], s_red_in[4];
   __shared__ int s_e, s_t;
   const bool sv4 = cfg.in_gran == SDQ_GRAN_3OF4;          // S-Vectors of 4: one outlier and two inliers per 4
+  const bool small = cfg.out_order == SDQ_ORDER_SMALL;   // Stage 2 takes the least significant values (study control)
   const bool ue = cfg.scale_rule == SDQ_SCALE_UE4M3;     // two-level scaling with E4M3 Q-Vector scales (pair-wise, block 32)
 
   // ---- pass 1: largest outlier magnitude of the row (and, for two-level scaling, largest kept inlier), non-finite check
@@ -110,7 +111,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     uint32_t skey[8];
     bad |= selection_keys(key, colw, g, skey);
     int o0, o1;
-    if (sv4 && out_n) select_outliers_per_4(skey, o0, o1); else select_outliers(skey, out_n, o0, o1);
+    if (sv4 && out_n) select_outliers_per_4(skey, small, o0, o1); else select_outliers(skey, out_n, small, o0, o1);
     if (o0 >= 0) okey_max = max(okey_max, key[o0]);
     if (o1 >= 0) okey_max = max(okey_max, key[o1]);
     if (ue) {
@@ -168,7 +169,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     uint32_t skey[8];
     selection_keys(key, colw, g, skey);
     int o0, o1;
-    if (sv4 && out_n) select_outliers_per_4(skey, o0, o1); else select_outliers(skey, out_n, o0, o1);
+    if (sv4 && out_n) select_outliers_per_4(skey, small, o0, o1); else select_outliers(skey, out_n, small, o0, o1);
     const int k1 = g >> 4, k2 = g >> 5;
     uint8_t* wi = wi_base + (size_t)k2 * wib;
     uint8_t* wo = wo_base + (size_t)k1 * WO_BYTES;
@@ -321,6 +322,7 @@ using namespace sdq;
 
 static bool cfg_ok(const sdq_config_t* c) {
   return c && c->out_n >= 0 && c->out_n <= 2 && c->in_gran >= 0 && c->in_gran <= SDQ_GRAN_3OF4 &&
+         (c->out_order == SDQ_ORDER_LARGE || c->out_order == SDQ_ORDER_SMALL) &&
          (c->in_gran < SDQ_GRAN_DENSE || c->in_gran == SDQ_GRAN_3OF4 || 10 - c->in_gran > c->out_n) &&
          (c->in_gran != SDQ_GRAN_3OF4 || c->out_n != 1) &&
          (c->in_block == 32 || c->in_block == 64) && c->scale_rule >= SDQ_SCALE_OCP_FLOOR && c->scale_rule <= SDQ_SCALE_UE4M3;

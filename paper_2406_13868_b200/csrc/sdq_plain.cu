@@ -19,13 +19,13 @@ __device__ __forceinline__ void load_group8(const __nv_bfloat16* w, uint32_t (&b
     bits[2 * i + 1] = r[i] >> 16;
   }
 }
-__device__ __forceinline__ void pick_outliers(const uint32_t (&key)[8], int out_n, int& o0, int& o1) {
+__device__ __forceinline__ void pick_outliers(const uint32_t (&key)[8], int out_n, bool small, int& o0, int& o1) {
   o0 = o1 = -1;
   if (out_n >= 1) {
     int b = 0;
 #pragma unroll
     for (int i = 1; i < 8; ++i)
-      if (key[i] > key[b]) b = i;
+      if (small ? key[i] < key[b] : key[i] > key[b]) b = i;
     o0 = b;
   }
   if (out_n >= 2) {
@@ -33,7 +33,7 @@ __device__ __forceinline__ void pick_outliers(const uint32_t (&key)[8], int out_
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       if (i == o0) continue;
-      if (b < 0 || key[i] > key[b]) b = i;
+      if (b < 0 || (small ? key[i] < key[b] : key[i] > key[b])) b = i;
     }
     o1 = b;
     if (o0 > o1) { int t = o0; o0 = o1; o1 = t; }
@@ -64,7 +64,7 @@ pack_plain_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int
     uint32_t skey[8];
     bad |= selection_keys(key, colw, g, skey);
     int o0, o1;
-    pick_outliers(skey, out_n, o0, o1);
+    pick_outliers(skey, out_n, cfg.out_order == SDQ_ORDER_SMALL, o0, o1);
     if (o0 >= 0) okey_max = max(okey_max, key[o0]);
     if (o1 >= 0) okey_max = max(okey_max, key[o1]);
   }
@@ -89,7 +89,7 @@ pack_plain_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int
     uint32_t skey[8];
     selection_keys(key, colw, g, skey);
     int o0, o1;
-    pick_outliers(skey, out_n, o0, o1);
+    pick_outliers(skey, out_n, cfg.out_order == SDQ_ORDER_SMALL, o0, o1);
     int slot_pos[4];
     if (pair) {
       float score[4];

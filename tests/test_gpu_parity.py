@@ -171,6 +171,31 @@ def test_s_vectors_of_4(M, N, K, out_n, rule):
     run_case(M, N, K, 2600 + M, out_n=out_n, rule=rule, block=32, gran=so.GRAN_3OF4)
 
 
+@pytest.mark.parametrize("gran,block,out_n", [(0, 64, 1), (0, 32, 2), (1, 32, 1), (3, 32, 1), (9, 32, 2)])
+def test_small_order_packer_and_product(gran, block, out_n):
+    """SDQ_ORDER_SMALL (the decomposition-stage study's control): the least significant values become the outliers;
+    packed arrays bit-exact for every layout, the product within the criterion where the GEMM runs the pattern"""
+    m = sdq()
+    N, K, M = 256, 1024, 24
+    cfg = m.Config(out_n, gran, block, 0, m.ORDER_SMALL)
+    oc = so.Config(out_n, gran, block, 0, so.ORDER_SMALL)
+    W = sdq_synth.make_weight(N, K, 2800 + gran)
+    p = m.sdq_decompose(W.cuda(), cfg)
+    op = so.decompose(sdq_synth.bf16_bits(W), oc)
+    pe = {k: v.cpu().numpy() for k, v in m.packed_export(p).items()}
+    for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp"):
+        assert np.array_equal(pe[name], getattr(op, name)), name
+    assert not np.array_equal(op.out_idx, so.decompose(sdq_synth.bf16_bits(W), so.Config(out_n, gran, block, 0)).out_idx)
+    if gran != m.GRAN_ELEM:
+        X = sdq_synth.make_act(M, K, 2801)
+        xq = m.sdq_quantize_act(X.cuda(), cfg)
+        d, tol = y_close(m.sdq_linear(xq, p, f32=True).cpu().numpy(), so.linear(so.quantize_act(sdq_synth.bf16_bits(X), oc), op))
+        assert (d <= tol).all()
+    with pytest.raises(m.SdqError) as e:
+        m.sdq_decompose(W.cuda(), m.Config(out_n, gran, block, 0, 2))
+    assert e.value.code == 1
+
+
 def test_dense_inliers_one_hot_readback_and_workspace_split():
     m = sdq()
     cfg = m.Config(1, m.GRAN_DENSE, 32, 0)
