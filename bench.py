@@ -613,6 +613,7 @@ def run_sweep(args):
                       ("4:8 pair-wise + 2:8", sdq.Config(2, sdq.GRAN_PAIR, 64, 0)),
                       ("4:8 pair-wise + 1:8, scale per 32", sdq.Config(1, sdq.GRAN_PAIR, 32, 0)),
                       ("4:8 pair-wise + 1:8, E4M3 scales per 32", sdq.Config(1, sdq.GRAN_PAIR, 32, sdq.SCALE_UE4M3)),
+                      ("2:4 element-wise + 1:8, scale per 32 (literal wording)", sdq.Config(1, sdq.GRAN_ELEM, 32, 0)),
                       ("6:8 = 2:8 + 4:8 at any position", sdq.Config(2, sdq.gran_keep(6), 32, 0)),
                       ("7:8 = 1:8 + 6:8", sdq.Config(1, sdq.gran_keep(7), 32, 0)),
                       ("3:4 = 1:4 + 2:4 (S-Vectors of 4)", sdq.Config(2, sdq.GRAN_3OF4, 32, 0)),

@@ -50,8 +50,10 @@ enum { SDQ_ORDER_LARGE = 0, SDQ_ORDER_SMALL = 1 };          /* Stage 2 takes the
  *   in_gran    how the remaining values are pruned to 50% (Stage 1, magnitude metric):
  *              SDQ_GRAN_PAIR keeps the 2 adjacent pairs (of 4) with the largest |a|+|b| in every 8
  *              (the pattern the sparse FP4 tensor core consumes); SDQ_GRAN_ELEM keeps the 2 largest
- *              of every 4 (decompose / export only: the buffer then holds the canonical arrays and
- *              sdq_linear returns SDQ_ERR_UNSUPPORTED).  SDQ_GRAN_DENSE skips Stage 1: every value that
+ *              of every 4 (with in_block = 32 the inliers are stored and executed like the dense
+ *              pattern below, the dropped positions holding +0; with in_block = 64 decompose / export
+ *              only: the buffer then holds the canonical arrays and sdq_linear returns
+ *              SDQ_ERR_UNSUPPORTED).  SDQ_GRAN_DENSE skips Stage 1: every value that
  *              is not an outlier stays an inlier (the evaluation's configuration 8:8 = 1:8 outliers +
  *              7:8 inliers); sdq_linear runs W_i as a dense 4-bit operand.  SDQ_GRAN_KEEP(n), n > out_n:
  *              Stage 1 keeps the n most significant values of every S-Vector of 8, of which the out_n most
@@ -197,7 +199,7 @@ sdq_status_t sdq_act_export(const sdq_act_t* Xq, const sdq_act_canonical_t* out,
  *   weights) while the previous kernel of the stream is still finishing, and waits for that kernel before it
  *   reads Xq or writes Y.  The packed weights must therefore be complete before the call is enqueued
  *   (sdq_decompose synchronises its stream, so a buffer it returned always is).
- *   Errors: INVALID_ARG, SHAPE, ALIGNMENT, UNSUPPORTED (in_gran == ELEM), CUDA. */
+ *   Errors: INVALID_ARG, SHAPE, ALIGNMENT, UNSUPPORTED (in_gran == ELEM with in_block == 64), CUDA. */
 sdq_status_t sdq_linear(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y_bf16, int64_t ldy, void* stream);
 
 /* Same product, storing the fp32 accumulator itself (the value the bf16 output is rounded from). */

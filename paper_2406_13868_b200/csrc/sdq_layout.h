@@ -24,7 +24,8 @@
 //     E_out: 128 rows x 16 B  (one 4-bit index pair per 4 logical K over 128 K)
 //   section SFA_out[rt]: 512 B, the per-row outlier scale as an E8M0 code, scale-atom form, 4 copies
 //   sections compact outlier codes / indices [N][K/8][out_n] u8, row scale exponents [N] i32, inlier row-factor
-//   exponents [N] i32 (two-level scaling with E4M3 Q-Vector scales; zeros otherwise)
+//   exponents [N] i32 (two-level scaling with E4M3 Q-Vector scales; zeros otherwise); element-wise 2:4 inliers with one
+//   scale per 32 K are stored like dense inliers, plus their kept indices [N][K/4] u8 for the exporter
 //
 // Activation buffer (per 128-token tile mt)
 //   section XI[mt][k2] = | B4 16384 | SFB_in 512 |            (one scale per 32 K: SFB_in 2 x 512, as for the weights)
@@ -84,9 +85,9 @@ __host__ __device__ inline uint32_t sf_off(uint32_t row, uint32_t s) { return (r
 constexpr size_t HEADER_BYTES = 256;
 
 struct PackedOffsets {
-  size_t wi, wo, sfa_out, ocode, oidx, osexp, wtexp, total;
+  size_t wi, wo, sfa_out, ocode, oidx, osexp, wtexp, emeta, total;
 };
-inline PackedOffsets packed_offsets(int64_t N, int64_t K, int out_n, bool b32 = false, bool dense = false) {
+inline PackedOffsets packed_offsets(int64_t N, int64_t K, int out_n, bool b32 = false, bool dense = false, bool elem = false) {
   PackedOffsets o;
   const size_t RT = (size_t)(N / TILE_ROWS), T1 = (size_t)(K / K1), T2 = (size_t)(K / K2);
   auto al = [](size_t x) { return (x + 255) & ~(size_t)255; };
@@ -97,7 +98,8 @@ inline PackedOffsets packed_offsets(int64_t N, int64_t K, int out_n, bool b32 = 
   o.oidx = al(o.ocode + (size_t)N * (size_t)(K / 8) * (size_t)out_n);
   o.osexp = al(o.oidx + (size_t)N * (size_t)(K / 8) * (size_t)out_n);
   o.wtexp = al(o.osexp + (size_t)N * 4);                          // inlier row-factor exponents [N] i32 (two-level scaling)
-  o.total = al(o.wtexp + (size_t)N * 4);
+  o.emeta = al(o.wtexp + (size_t)N * 4);                          // element-wise 2:4 stored dense: kept indices [N][K/4] u8
+  o.total = al(o.emeta + (elem ? (size_t)N * (size_t)(K / 4) : 0));
   return o;
 }
 

@@ -27,6 +27,7 @@
 #include "sdq_internal.h"
 #include "sdq_layout.h"
 #include "sdq_linear.h"
+#include "sdq_plain.h"
 #include "sdq_ptx.cuh"
 
 namespace sdq {
@@ -722,7 +723,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   if (!Xq || !P || !Y || !Xq->dev || !P->dev) return SDQ_ERR_INVALID_ARG;
   if (Xq->K != P->K || Xq->M <= 0 || P->N <= 0 || P->N % TILE_ROWS || P->K % K2 || ldy < P->N) return SDQ_ERR_SHAPE;
   if (Xq->cfg.in_block != P->cfg.in_block || Xq->cfg.scale_rule != P->cfg.scale_rule) return SDQ_ERR_SHAPE;
-  if (P->cfg.in_gran != SDQ_GRAN_PAIR && !(P->cfg.in_gran >= SDQ_GRAN_DENSE && P->cfg.in_block == 32)) return SDQ_ERR_UNSUPPORTED;
+  if (!is_tensor_core_reading(P->cfg)) return SDQ_ERR_UNSUPPORTED;
   if (P->cfg.scale_rule == SDQ_SCALE_UE4M3 && !(P->cfg.in_gran == SDQ_GRAN_PAIR && P->cfg.in_block == 32)) return SDQ_ERR_UNSUPPORTED;
   if (((uintptr_t)Y & 15) || (ldy % 8) || ((uintptr_t)ws & 15)) return SDQ_ERR_ALIGNMENT;
   static bool attr_set = false;
@@ -746,8 +747,8 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   p.x = (const uint8_t*)Xq->dev;
   p.b32 = P->cfg.in_block == 32 ? 1 : 0;
   const bool ue = P->cfg.scale_rule == SDQ_SCALE_UE4M3;
-  p.dense = P->cfg.in_gran >= SDQ_GRAN_DENSE ? 1 : 0;   // the n:8 patterns are stored and run like the dense one
-  p.poff = packed_offsets(P->N, P->K, P->cfg.out_n, p.b32 != 0, p.dense != 0);
+  p.dense = is_dense_layout(P->cfg) ? 1 : 0;   // the n:8, 3:4 and element-wise 2:4 patterns are stored and run like the dense one
+  p.poff = tiled_offsets(P->N, P->K, P->cfg);
   p.aoff = act_offsets(Xq->M, Xq->K, p.b32 != 0);
   p.tw = ue ? reinterpret_cast<const int32_t*>(p.w + p.poff.wtexp) : nullptr;
   p.tx = reinterpret_cast<const int32_t*>(p.x + p.aoff.sexp);

@@ -144,9 +144,11 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
   const int64_t rt = n / TILE_ROWS;
   const uint32_t r = (uint32_t)(n % TILE_ROWS);
   const int T1 = (int)(K / K1), T2 = (int)(K / K2);
-  const bool b32 = cfg.in_block == 32, dense = cfg.in_gran >= SDQ_GRAN_DENSE;
-  // dense family: inliers kept per S-Vector (8 - out_n without Stage 1; S-Vectors of 4: 3 minus the outlier)
-  const int keep_in = sv4 ? (out_n ? 2 : 3) : 10 - cfg.in_gran - out_n;
+  const bool b32 = cfg.in_block == 32, dense = is_dense_layout(cfg);
+  const bool elem = cfg.in_gran == SDQ_GRAN_ELEM;        // element-wise 2:4: the 2 most significant non-outliers of every 4
+  const bool grp4 = sv4 || elem;                         // Stage 1 ranks inside groups of 4
+  // dense family: inliers kept per group (8 - out_n without Stage 1; groups of 4: 3 minus the outlier, or 2 for 2:4)
+  const int keep_in = elem ? 2 : (sv4 ? (out_n ? 2 : 3) : 10 - cfg.in_gran - out_n);
   const int wib = wi_bytes(b32, dense);
   uint8_t* wi_base = blob + off.wi + (size_t)rt * T2 * wib;
   uint8_t* wo_base = blob + off.wo + (size_t)rt * T1 * WO_BYTES;
@@ -185,7 +187,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
         int before = 0;
 #pragma unroll
         for (int j = 0; j < 8; ++j)
-          before += (j != o0 && j != o1 && (!sv4 || (j >> 2) == (i >> 2)) && (skey[j] > skey[i] || (skey[j] == skey[i] && j < i))) ? 1 : 0;
+          before += (j != o0 && j != o1 && (!grp4 || (j >> 2) == (i >> 2)) && (skey[j] > skey[i] || (skey[j] == skey[i] && j < i))) ? 1 : 0;
         if (i == o0 || i == o1 || before >= keep_in) gone |= 1u << i;
         else ikey = max(ikey, key[i]);
       }
@@ -202,6 +204,15 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
       // 32 S-Vectors per 256-K stage, 4 code bytes each: bytes 32 j .. 32 j + 31 = K-block j (64 K)
       *reinterpret_cast<uint32_t*>(wi + a_off(r, (uint32_t)(g & 31) * 4)) = codes;
       if ((g & 3) == 0) wi[a_in_bytes(true) + in_sf_off(true, r, (uint32_t)((g >> 2) & 7))] = (uint8_t)c;
+      if (elem) {
+        // the kept indices (two ascending 2-bit values per group of 4) are only needed by the exporter
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const uint32_t kept = (~(gone >> (4 * h))) & 15u;            // exactly two bits
+          const int i0 = __ffs((int)kept) - 1, i1 = 31 - __clz((int)kept);
+          blob[off.emeta + (size_t)n * (size_t)(K / 4) + 2 * g + h] = (uint8_t)(i0 | (i1 << 2));
+        }
+      }
     } else {
     // Stage 1 on the remaining values: keep the 2 pairs (of 4) with the largest summed significance
     int j0, j1;
@@ -281,16 +292,28 @@ export_packed_kernel(const uint8_t* __restrict__ blob, int64_t N, int64_t K, sdq
   const int64_t rt = n / TILE_ROWS;
   const uint32_t r = (uint32_t)(n % TILE_ROWS);
   const int T2 = (int)(K / K2);
-  const bool b32 = cfg.in_block == 32, dense = cfg.in_gran >= SDQ_GRAN_DENSE;
+  const bool b32 = cfg.in_block == 32, dense = is_dense_layout(cfg), elem = cfg.in_gran == SDQ_GRAN_ELEM;
   const int wib = wi_bytes(b32, dense);
   const uint8_t* wi_base = blob + off.wi + (size_t)rt * T2 * wib;
   for (int g = threadIdx.x; g < G; g += 128) {
     const uint8_t* wi = wi_base + (size_t)(g >> 5) * wib;
     if (dense) {
       const uint32_t codes = *reinterpret_cast<const uint32_t*>(wi + a_off(r, (uint32_t)(g & 31) * 4));
+      if (elem) {
+        // element-wise 2:4: the canonical arrays hold the two kept slots of every 4 and their indices
+        uint8_t* ic = out.in_code + (size_t)n * (K / 2) + 4 * g;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const uint32_t mb = blob[off.emeta + (size_t)n * (size_t)(K / 4) + 2 * g + h];
+          out.in_meta[(size_t)n * (K / 4) + 2 * g + h] = (uint8_t)mb;
+          ic[2 * h] = (codes >> (4 * (4 * h + (mb & 3)))) & 15;
+          ic[2 * h + 1] = (codes >> (4 * (4 * h + ((mb >> 2) & 3)))) & 15;
+        }
+      } else {
       uint8_t* ic = out.in_code + (size_t)n * K + 8 * g;
 #pragma unroll
       for (int i = 0; i < 8; ++i) ic[i] = (codes >> (4 * i)) & 15;
+      }
       if ((g & 3) == 0) out.in_scale[(size_t)n * (K / 32) + (g >> 2)] = wi[a_in_bytes(true) + in_sf_off(true, r, (uint32_t)((g >> 2) & 7))];
       for (int t = 0; t < out_n; ++t) {
         out.out_code[((size_t)n * G + g) * out_n + t] = blob[off.ocode + ((size_t)n * G + g) * out_n + t];
@@ -338,13 +361,13 @@ extern "C" sdq_status_t sdq_packed_size(int64_t N, int64_t K, const sdq_config_t
   if (!cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
   if (cfg_unsupported(cfg)) return SDQ_ERR_UNSUPPORTED;
   if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2) return SDQ_ERR_SHAPE;
-  if (bytes) *bytes = is_tensor_core_reading(*cfg) ? packed_offsets(N, K, cfg->out_n, cfg->in_block == 32, cfg->in_gran >= SDQ_GRAN_DENSE).total : plain_packed_offsets(N, K, *cfg).total;
+  if (bytes) *bytes = is_tensor_core_reading(*cfg) ? tiled_offsets(N, K, *cfg).total : plain_packed_offsets(N, K, *cfg).total;
   if (algorithmic_bytes) {
     // per weight: 4-bit values on half the positions (2) + index metadata (pair-wise: two 2-bit pair indices per 8 =
     // 0.5; element-wise: two 2-bit indices per 4 = 1) + one 8-bit scale per Q-Vector + out_n * (8 value + 3 index
     // bits) per 8; plus one 32-bit row scale
     // (dense storage: a 4-bit value on every position and no index metadata)
-    const double inl = cfg->in_gran >= SDQ_GRAN_DENSE ? 4.0 : 2.0 + (cfg->in_gran == SDQ_GRAN_PAIR ? 0.5 : 1.0);
+    const double inl = cfg->in_gran >= SDQ_GRAN_DENSE ? 4.0 : 2.0 + (cfg->in_gran == SDQ_GRAN_PAIR ? 0.5 : 1.0);   // 2:4: the paper's form
     const double bits = inl + 8.0 / cfg->in_block + cfg->out_n * 11.0 / 8.0;
     *algorithmic_bytes = (size_t)((double)N * (double)K * bits / 8.0) + (cfg->out_n ? (size_t)N * 4 : 0);
   }
@@ -365,7 +388,7 @@ extern "C" sdq_status_t sdq_decompose_metric(const void* W, int64_t N, int64_t K
   if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2 || ldw < K) return SDQ_ERR_SHAPE;
   if (((uintptr_t)W & 15) || ((uintptr_t)packed_buf & 15) || (ldw % 8)) return SDQ_ERR_ALIGNMENT;
   const bool tc = is_tensor_core_reading(*cfg);
-  const PackedOffsets off = packed_offsets(N, K, cfg->out_n, cfg->in_block == 32, cfg->in_gran >= SDQ_GRAN_DENSE);
+  const PackedOffsets off = tiled_offsets(N, K, *cfg);
   const PlainPackedOffsets poff = plain_packed_offsets(N, K, *cfg);
   if (packed_bytes < (tc ? off.total : poff.total)) return SDQ_ERR_BUFFER_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
@@ -397,7 +420,7 @@ extern "C" sdq_status_t sdq_decompose_metric(const void* W, int64_t N, int64_t K
 extern "C" sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canonical_t* out, void* stream)
 {
   if (!P || !out || !P->dev || !out->in_code || !out->in_scale || !out->out_sexp) return SDQ_ERR_INVALID_ARG;
-  if (!out->in_meta && P->cfg.in_gran < SDQ_GRAN_DENSE) return SDQ_ERR_INVALID_ARG;
+  if (!out->in_meta && P->cfg.in_gran < SDQ_GRAN_DENSE) return SDQ_ERR_INVALID_ARG;   // PAIR and ELEM record their pattern
   if (P->cfg.out_n > 0 && (!out->out_code || !out->out_idx)) return SDQ_ERR_INVALID_ARG;
   if (!is_tensor_core_reading(P->cfg)) {
     // the buffer already holds the canonical arrays
@@ -415,7 +438,7 @@ extern "C" sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canon
     ok = ok && cudaMemcpyAsync(out->out_sexp, b + o.osexp, n * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
     return ok ? SDQ_OK : SDQ_ERR_CUDA;
   }
-  const PackedOffsets off = packed_offsets(P->N, P->K, P->cfg.out_n, P->cfg.in_block == 32, P->cfg.in_gran >= SDQ_GRAN_DENSE);
+  const PackedOffsets off = tiled_offsets(P->N, P->K, P->cfg);
   export_packed_kernel<<<(unsigned)P->N, 128, 0, (cudaStream_t)stream>>>((const uint8_t*)P->dev, P->N, P->K, P->cfg, off, *out);
   return cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
 }

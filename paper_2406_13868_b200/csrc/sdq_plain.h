@@ -5,13 +5,23 @@
 #include <stdint.h>
 
 #include "sdq_internal.h"
+#include "sdq_layout.h"
 
 namespace sdq {
 
 // pair-wise 4:8 inliers with one scale per 64 K (kind::mxf4 .block32) or per 32 K (kind::mxf4nvf4 .block16), or dense
-// inliers with one scale per 32 K (dense kind::mxf4 .block32): tiled layout
+// inliers with one scale per 32 K (dense kind::mxf4 .block32), which also carries element-wise 2:4 inliers with one
+// scale per 32 K: tiled layout
 inline bool is_tensor_core_reading(const sdq_config_t& c) {
-  return (c.in_gran == SDQ_GRAN_PAIR && (c.in_block == 64 || c.in_block == 32)) || (c.in_gran >= SDQ_GRAN_DENSE && c.in_block == 32);
+  return (c.in_gran == SDQ_GRAN_PAIR && (c.in_block == 64 || c.in_block == 32)) || (c.in_gran >= SDQ_GRAN_DENSE && c.in_block == 32) ||
+         (c.in_gran == SDQ_GRAN_ELEM && c.in_block == 32);
+}
+// inliers stored as a dense 4-bit operand: no pruning, n:8 / 3:4 sparsification, or element-wise 2:4 with one scale per 32 K
+__host__ __device__ inline bool is_dense_layout(const sdq_config_t& c) {
+  return c.in_block == 32 && (c.in_gran >= SDQ_GRAN_DENSE || c.in_gran == SDQ_GRAN_ELEM);
+}
+inline PackedOffsets tiled_offsets(int64_t N, int64_t K, const sdq_config_t& c) {
+  return packed_offsets(N, K, c.out_n, c.in_block == 32, is_dense_layout(c), c.in_gran == SDQ_GRAN_ELEM && c.in_block == 32);
 }
 
 struct PlainPackedOffsets {

@@ -196,6 +196,14 @@ def test_small_order_packer_and_product(gran, block, out_n):
     assert e.value.code == 1
 
 
+@pytest.mark.parametrize("M,N,K,out_n,rule", [(8, 256, 256, 1, 0), (1, 512, 2048, 1, 0), (16, 256, 4096, 2, 1), (33, 128, 768, 0, 0),
+                                              (129, 256, 512, 1, 1), (300, 512, 1024, 2, 0), (520, 6400, 256, 1, 0)])
+def test_element_wise_2of4_block_32_through_the_tensor_core(M, N, K, out_n, rule):
+    """the literal wording (element-wise 2:4 inliers, one scale per 32 K): packed arrays bit-exact in their own canonical
+    form (two kept slots and their indices per 4), the product on the dense 4-bit MMA with the dropped positions at +0"""
+    run_case(M, N, K, 2900 + M, out_n=out_n, rule=rule, block=32, gran=so.GRAN_ELEM)
+
+
 def test_dense_inliers_one_hot_readback_and_workspace_split():
     m = sdq()
     cfg = m.Config(1, m.GRAN_DENSE, 32, 0)
@@ -754,8 +762,8 @@ def test_errors_are_status_codes():
     with pytest.raises(m.SdqError) as e:
         m.sdq_decompose(W[:, :128].contiguous())           # K not a multiple of 256
     assert e.value.code == 2
-    p_elem = m.sdq_decompose(W, m.Config(1, m.GRAN_ELEM, 32, 0))            # decompose-only reading ...
-    xq32 = m.sdq_quantize_act(sdq_synth.make_act(4, 256, 0).cuda(), m.Config(1, m.GRAN_ELEM, 32, 0))
+    p_elem = m.sdq_decompose(W, m.Config(1, m.GRAN_ELEM, 64, 0))            # decompose-only reading ...
+    xq32 = m.sdq_quantize_act(sdq_synth.make_act(4, 256, 0).cuda(), m.Config(1, m.GRAN_ELEM, 64, 0))
     with pytest.raises(m.SdqError) as e:
         m.sdq_linear(xq32, p_elem)                                          # ... which the tensor core cannot run
     assert e.value.code == 4
