@@ -249,6 +249,11 @@ def run_ours(args):
                 "traffic": 87.7e6, "traffic_unit": "bytes per launch (gate/up shape)",
                 "peak_basis": "%s bf16 burst %.1f TF/s x 8/3 (sparse FP4 at 8x + sparse FP8 at 4x per dense-equivalent flop)" % (peaks["source"], peaks["bf16"]),
                 "avg_launch_ms": gemm_ms / gemm_n, "launches": gemm_n,
+                # what actually bounds the kernel: bytes staged from L2 into shared memory per launch (688 tiles x 2.09 MB for
+                # the gate / up shape, l1tex__m_xbar2l1tex_read_bytes of the same ncu capture) against the 19.5 TB/s that 148
+                # SMs pulling together reach in a copy-only microbenchmark on this pool
+                "l2_to_sm": {"bytes_per_launch": 1.438e9, "achieved_TBps": 1.438e9 / (gemm_ms / gemm_n * 1e-3) / 1e12,
+                             "measured_ceiling_TBps": 19.5, "frac": 1.438e9 / (gemm_ms / gemm_n * 1e-3) / 19.5e12},
                 "frac_of_sparse_fp4_peak": gemm_tf / (8 * peaks["bf16"])}
     # activation quantizer alone (quant_act_fused_kernel), back to back on the larger input so that
     # host launch overhead does not count: bytes = bf16 read + 4-bit codes + 8-bit codes + one scale byte per 64
