@@ -240,6 +240,18 @@ sdq_status_t sdq_linear_f32_ws(const sdq_act_t* Xq, const sdq_packed_t* P, float
 #define SDQ_STATIC_WS_BYTES (4u << 20)
 sdq_status_t sdq_linear_noalloc(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y_bf16, int64_t ldy, void* stream);
 
+/* Measurement aid (no counterpart in the paper): enqueues a copy-only kernel in which every SM keeps `nslot` bulk
+ * copies of `slot_bytes` in flight from its own region of `src` (device, 16-byte aligned; walked cyclically) into
+ * shared memory, `iters` copies per SM, nothing consuming them.  *bytes_moved receives the bytes the launch stages
+ * in total; the caller times the launch with events.  With a source smaller than L2 this is the ceiling of the
+ * L2 -> shared-memory path that bounds the many-token product kernel.
+ *   slot_bytes a multiple of 128, >= 1024; nslot 1..16; nslot * slot_bytes <= 220 KB; src_bytes / #SMs >= slot_bytes;
+ *   issuers 1..4: threads per SM that issue the copies (the slots are dealt out over them).
+ *   Asynchronous on `stream`.  Errors: INVALID_ARG, ALIGNMENT, SHAPE, CUDA; a bounded wait that gives up sets the
+ *   sticky device status. */
+sdq_status_t sdq_diag_l2_copy(const void* src, size_t src_bytes, int slot_bytes, int nslot, int issuers, int iters,
+                              size_t* bytes_moved, void* stream);
+
 /* Synchronises `stream` and returns the sticky device-side status (SDQ_OK or SDQ_ERR_TIMEOUT when a
  * bounded wait inside a kernel gave up), clearing it. */
 sdq_status_t sdq_device_status(void* stream);

@@ -65,7 +65,7 @@ class _ActCanon(ctypes.Structure):
 
 EXPORTS = ["sdq_packed_size", "sdq_decompose", "sdq_decompose_metric", "sdq_channel_norm", "sdq_packed_export", "sdq_act_size", "sdq_quantize_act", "sdq_act_export",
            "sdq_linear", "sdq_linear_f32", "sdq_workspace_size", "sdq_workspace_init", "sdq_linear_ws", "sdq_linear_f32_ws", "sdq_linear_noalloc",
-           "sdq_device_status", "sdq_status_string"]
+           "sdq_diag_l2_copy", "sdq_device_status", "sdq_status_string"]
 
 _lib = None
 
@@ -83,6 +83,7 @@ def lib() -> ctypes.CDLL:
         L.sdq_decompose.argtypes = [vp, i64, i64, i64, ctypes.POINTER(Config), vp, sz, ctypes.POINTER(_Packed), vp]
         L.sdq_decompose_metric.argtypes = [vp, i64, i64, i64, ctypes.POINTER(Config), vp, vp, sz, ctypes.POINTER(_Packed), vp]
         L.sdq_channel_norm.argtypes = [vp, i64, i64, i64, vp, vp]
+        L.sdq_diag_l2_copy.argtypes = [vp, sz, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.POINTER(sz), vp]
         L.sdq_packed_export.argtypes = [ctypes.POINTER(_Packed), ctypes.POINTER(_Canon), vp]
         L.sdq_act_size.argtypes = [i64, i64, ctypes.POINTER(Config), ctypes.POINTER(sz)]
         L.sdq_quantize_act.argtypes = [vp, i64, i64, i64, ctypes.POINTER(Config), vp, sz, ctypes.POINTER(_Act), vp]
@@ -229,6 +230,15 @@ def sdq_linear(xq: QuantAct, p: PackedWeight, out: torch.Tensor | None = None, f
         _check(fn(ctypes.byref(xq.desc), ctypes.byref(p.desc), out.data_ptr(), out.stride(0), workspace.data_ptr(),
                   workspace.numel(), _stream()), "sdq_linear_ws")
     return out
+
+
+def diag_l2_copy(src: torch.Tensor, slot_bytes: int, nslot: int, iters: int, issuers: int = 1) -> int:
+    """Enqueues the copy-only L2 -> shared-memory kernel on `src` (uint8 CUDA tensor); returns the bytes it stages."""
+    _need_cuda(src, "src")
+    n = ctypes.c_size_t(0)
+    _check(lib().sdq_diag_l2_copy(src.data_ptr(), src.numel() * src.element_size(), slot_bytes, nslot, issuers, iters, ctypes.byref(n), _stream()),
+           "sdq_diag_l2_copy")
+    return int(n.value)
 
 
 STATIC_WS_BYTES = 4 << 20

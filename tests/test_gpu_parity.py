@@ -756,6 +756,20 @@ def test_literal_readings_element_wise_2of4_and_block32(gran, block, out_n):
         assert np.array_equal(pe[name], getattr(op, name)), name
 
 
+def test_l2_copy_diagnostic_runs_and_reports_bytes():
+    m = sdq()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    src = torch.zeros(sms * (128 << 10), dtype=torch.uint8, device="cuda")
+    for issuers, iters in ((1, 50), (3, 50), (4, 3), (2, 1)):
+        moved = m.diag_l2_copy(src, 16384, 4, iters, issuers)
+        torch.cuda.synchronize()
+        assert moved == sms * iters * 16384 and m.device_status() == 0
+    for args, code in (((1000, 4, 10), 2), ((16384, 17, 10), 2), ((1 << 20, 4, 10), 2), ((16384, 4, 10, 5), 2)):
+        with pytest.raises(m.SdqError) as e:
+            m.diag_l2_copy(src, *args)
+        assert e.value.code == code
+
+
 def test_errors_are_status_codes():
     m = sdq()
     W = sdq_synth.make_weight(128, 256, 0).cuda()
