@@ -48,7 +48,8 @@ constexpr int LIN_SMEM_MAX = 5 * 46080 + SM_TAIL_B32;   // the largest request
 //   +0  2 buffers x 32: E_in 4 | SFA_in 4 or 8 | SFB_in up to 16     +64 2 buffers x 4: E_out     +72 SFA_out 4     +76 SFB_out 8
 //   (one scale per 64 K: SFA_in 4, SFB_in 4 per token tile; per 32 K: one scale word per 128-K block, so twice as many)
 // Many tokens (512 columns): 16 columns per ring slot at 256 + 16 s (E 4 | SFA 4 | SFB 8; an outlier stage uses the
-// first 4) and two alternating 12-column buffers of outlier row / token scales at 336.
+// first 4; 32 per slot with one scale per 32 K: E 4 | SFA 8 | SFB 16) and, behind the slots' columns, two alternating
+// 12-column buffers of outlier row / token scales.
 constexpr uint32_t TM_D = 0;
 constexpr uint32_t TM_META_COLS = 84;
 
