@@ -1,15 +1,37 @@
 // Status plumbing of the C-ABI: sticky device flags and status strings.
+#include <mutex>
+
 #include "sdq_internal.h"
 
 namespace sdq {
+
+static DeviceInfo g_device_info[MAX_DEVICES];
+static std::mutex g_device_mutex;
+
+DeviceInfo* device_info_slot(int dev) { return (dev >= 0 && dev < MAX_DEVICES) ? &g_device_info[dev] : nullptr; }
+
+DeviceInfo* device_info() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+  DeviceInfo* d = device_info_slot(dev);
+  if (!d) return nullptr;
+  std::lock_guard<std::mutex> lock(g_device_mutex);
+  if (!d->sm_count) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return nullptr;
+    d->sm_count = n;
+  }
+  return d;
+}
 
 __device__ uint32_t g_flags[FLAG_COUNT];
 
 uint32_t* device_flags() {
   // resolved once per device (the symbol lives in every context that loads the library)
-  static uint32_t* cache[64] = {nullptr};
+  static uint32_t* cache[MAX_DEVICES] = {nullptr};
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return nullptr;
+  std::lock_guard<std::mutex> lock(g_device_mutex);
   if (!cache[dev]) {
     void* ptr = nullptr;
     if (cudaGetSymbolAddress(&ptr, g_flags) != cudaSuccess) return nullptr;

@@ -61,17 +61,16 @@ extern "C" sdq_status_t sdq_diag_l2_copy(const void* src, size_t src_bytes, int 
 {
   if (!src || !bytes_moved) return SDQ_ERR_INVALID_ARG;
   if ((uintptr_t)src & 15) return SDQ_ERR_ALIGNMENT;
-  int dev = 0, sm_count = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
-    return SDQ_ERR_CUDA;
+  DeviceInfo* dinfo = device_info();
+  if (!dinfo) return SDQ_ERR_CUDA;
+  const int sm_count = dinfo->sm_count;
   const size_t region = (src_bytes / (size_t)sm_count) & ~(size_t)127;
   if (slot_bytes < 1024 || (slot_bytes & 127) || nslot < 1 || nslot > 16 || issuers < 1 || issuers > 4 || iters < 1 || (size_t)nslot * slot_bytes > 220 * 1024 ||
       region < (size_t)slot_bytes)
     return SDQ_ERR_SHAPE;
-  static bool attr_set = false;
-  if (!attr_set) {
+  if (!dinfo->diag_attr) {
     if (cudaFuncSetAttribute(l2_copy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024 + 128) != cudaSuccess) return SDQ_ERR_CUDA;
-    attr_set = true;
+    dinfo->diag_attr = 1;
   }
   uint32_t* flags = device_flags();
   if (!flags) return SDQ_ERR_CUDA;

@@ -681,13 +681,10 @@ sdq_linear_kernel(const LinearParams p)       // many tokens: 13 warps, four of 
 
 using namespace sdq;
 
-static int sm_count_cached() {
-  static int sm_count = 0;
-  if (!sm_count) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sm_count = 0;
-  }
-  return sm_count;
+// SM count of the current device (0 on failure)
+static int sm_count_current() {
+  const DeviceInfo* d = device_info();
+  return d ? d->sm_count : 0;
 }
 
 // number of K splits for a call: only for M <= 128 (one token tile), as many as keep one CTA per SM,
@@ -711,7 +708,7 @@ extern "C" sdq_status_t sdq_workspace_size(int64_t M, int64_t N, int64_t K, cons
 {
   if (!cfg || !bytes) return SDQ_ERR_INVALID_ARG;
   if (M <= 0 || N <= 0 || K <= 0 || N % TILE_ROWS || K % K2) return SDQ_ERR_SHAPE;
-  const int ks = choose_ksplit(M, N, K, sm_count_cached());
+  const int ks = choose_ksplit(M, N, K, sm_count_current());
   const size_t RT = (size_t)(N / TILE_ROWS);
   // counters first (one per row tile, 256 B aligned), then ks fp32 partial tiles per row tile
   *bytes = ks > 1 ? ((RT * 4 + 255) & ~(size_t)255) + RT * (size_t)ks * (size_t)n_tile_for(M) * TILE_ROWS * 4 : 0;
@@ -727,8 +724,9 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   if (!is_tensor_core_reading(P->cfg)) return SDQ_ERR_UNSUPPORTED;
   if (P->cfg.scale_rule == SDQ_SCALE_UE4M3 && !(P->cfg.in_gran == SDQ_GRAN_PAIR && P->cfg.in_block == 32)) return SDQ_ERR_UNSUPPORTED;
   if (((uintptr_t)Y & 15) || (ldy % 8) || ((uintptr_t)ws & 15)) return SDQ_ERR_ALIGNMENT;
-  static bool attr_set = false;
-  if (!attr_set) {
+  DeviceInfo* dinfo = device_info();
+  if (!dinfo) return SDQ_ERR_CUDA;
+  if (!dinfo->linear_attr) {     // function attributes belong to the device's context: once per device
     const cudaFuncAttribute a = cudaFuncAttributeMaxDynamicSharedMemorySize;
     if (cudaFuncSetAttribute(sdq_linear_kernel<true, true, false, false>, a, LIN_SMEM_MAX) != cudaSuccess ||
         cudaFuncSetAttribute(sdq_linear_kernel<false, true, false, false>, a, LIN_SMEM_MAX) != cudaSuccess ||
@@ -739,10 +737,9 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
         cudaFuncSetAttribute(sdq_linear_kernel<true, false, false, true>, a, LIN_SMEM_MAX) != cudaSuccess ||
         cudaFuncSetAttribute(sdq_linear_kernel<false, false, false, true>, a, LIN_SMEM_MAX) != cudaSuccess)
       return SDQ_ERR_CUDA;
-    attr_set = true;
+    dinfo->linear_attr = 1;
   }
-  const int sm_count = sm_count_cached();
-  if (!sm_count) return SDQ_ERR_CUDA;
+  const int sm_count = dinfo->sm_count;
   LinearParams p;
   p.w = (const uint8_t*)P->dev;
   p.x = (const uint8_t*)Xq->dev;
@@ -813,6 +810,11 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   const int stages_per_tile = (T2 + p.ksplit - 1) / p.ksplit + (T1 + p.ksplit - 1) / p.ksplit;
   // many tokens without K split: the instantiations with compile-time geometry (five ring slots; four with dense inliers)
   const bool many = p.n_tile == 256 && p.ksplit == 1;
+  // ... as CTA pairs on tiles of 256 rows x 256 tokens wherever the shape allows (fewer L2 bytes per output)
+  if (many && pair_kernel_applies(M, P->N, P->K) && !getenv("SDQ_NO_PAIR")) {
+    const cudaError_t pe = launch_linear_pair(p, f32, sm_count, (cudaStream_t)stream, &dinfo->pair_attr);
+    return pe == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
+  }
   int max_slots = many ? (p.dense ? 4 : 5) : RING_BYTES / p.slot_bytes;
   if (p.cluster_ks > 1 && p.total_tiles > sm_count) {
     // cluster split K with more CTAs than SMs (few tokens, one tile per CTA): the grid is one wave only if two CTAs
