@@ -40,7 +40,7 @@ struct LinearParams {
 
 // CTA-pair (tcgen05 cta_group::2) many-token kernel: tiles of 256 weight rows x 256 tokens (sdq_linear_pair.cu).
 // `attr_mask` is the calling device's record of which instantiations already carry their shared-memory attribute.
-bool pair_kernel_applies(int64_t M, int64_t N, int64_t K);
+bool pair_kernel_applies(int64_t M, int64_t N, int64_t K, int out_n);
 cudaError_t launch_linear_pair(LinearParams p, bool f32_out, int sm_count, cudaStream_t stream, uint32_t* attr_mask);
 
 }  // namespace sdq

@@ -7,12 +7,19 @@
 // shared memory -- 27 KB per CTA and stage instead of 43 KB for the same MMA time.  The stage sequence of a tile is
 // that of the single-CTA kernel (all inlier stages of 256 K, then all outlier stages of 128 K, one fp32 accumulator).
 //
-// Per CTA: warps 0 / 6 / 7 bulk-copy producers (weight records / own activation codes / scale atoms of both token
-// halves), warps 2..5 and 9..12 epilogue (own 128 rows x 256 tokens: TMEM -> registers as packed bf16, TMEM handed
-// back, transposed 16-byte stores under the next tile's K loop).  Even CTA (leader): warp 8 moves metadata and scales
-// of both CTAs to TMEM (pair-wide tcgen05.cp), warp 1 issues the pair-wide MMAs; its tcgen05.commit signals "slot
-// consumed" / "accumulator complete" to the barriers of both CTAs.  Odd CTA: one thread of warp 8 and one of warp 1
+// Per CTA: warps 0 / 6 / 7 bulk-copy producers (own weight records / own activation codes / scale atoms of both token
+// halves; two lanes each, see there), warps 2..5 and 9..12 epilogue (own 128 rows x 256 tokens: TMEM -> registers as
+// packed bf16, TMEM handed back, transposed stores under the next tile's K loop).  Even CTA (leader): warp 1 copies
+// metadata and scales of both CTAs to TMEM (pair-wide tcgen05.cp) and issues the pair-wide MMAs; its tcgen05.commit
+// signals "slots consumed" / "accumulator complete" to the barriers of both CTAs.  Odd CTA: two lanes of warp 1
 // forward "my part of the slot has landed" to the leader's barriers.  Every wait is bounded.
+//
+// What was measured on the way (B200, 2048 tokens, 4096 -> 11008, 1:8 outliers; the single-CTA kernel takes 84 us):
+// a first version with one release per slot, a separate TMEM-mover thread and cluster-scope release / acquire on the
+// forwarding hop took 213 us -- a remote mbarrier arrive with .release.cluster costs ~0.8 us under load (the default
+// semantics suffice: the data was written by the bulk-copy engine and is read by the tensor core, both outside the
+// forwarding thread's view of memory) -> 94 us; warp-uniform issue loops, the copies to TMEM folded into the MMA issuer,
+// one barrier per slot and batches of landed slots -> 78 us; two lanes per producer -> 67 us (2.75 PFLOP/s).
 #include <cuda_bf16.h>
 #include <stdlib.h>
 
@@ -22,14 +29,6 @@
 #include "sdq_ptx.cuh"
 
 namespace sdq {
-
-#ifdef SDQ_PAIR_TRACE
-__device__ unsigned long long g_trace[2 * 8 * 512];
-__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define TRACE(ev, k) do { if (pair == 0 && trace_tile) g_trace[(rank * 8 + (ev)) * 512 + (k)] = gtime(); } while (0)
-#else
-#define TRACE(ev, k) do { } while (0)
-#endif
 
 constexpr int PAIR_THREADS = 416;            // 13 warps
 constexpr int PAIR_MAX_SLOTS = 8;
@@ -93,81 +92,91 @@ sdq_linear_pair_kernel(const LinearParams p)
   const uint32_t tmem = *tmem_slot;
 
   if (warp == 0 || warp == 6 || warp == 7) {
-    if (lane == 0) {
-      // ---------------- producers (both CTAs): role 0 = own weight records, 1 = own activation codes, 2 = scale atoms
+    if (lane < 2) {
+      // ---------------- producers (both CTAs): role 0 = own weight records, 1 = own activation codes, 2 = scale atoms.
+      // One trip of a producer's loop (barrier wait, address arithmetic, expect-tx, copy) takes ~0.3 us, which one thread
+      // per role cannot hide at two MMAs per stage; ring slots are released in pairs, so lanes 0 and 1 of the warp run the
+      // loop in lockstep, lane l filling the slots of parity l: two stages per trip.
       const int role = warp == 0 ? 0 : (int)warp - 5;
       if (role != 0) ptx::griddep_wait();    // activations come from an earlier kernel; weights do not
+      const int S = T2 + T1;
+      const int my_tiles = p.total_tiles > pair ? (p.total_tiles - pair + n_pairs - 1) / n_pairs : 0;
+      const int total = my_tiles * S;                                        // stages of this CTA, numbered through its tiles
+      const size_t xi_tile = (size_t)T2 * xib, xo_tile = (size_t)T1 * XO_BYTES;
       bool ok = true;
-      uint32_t s = 0, wrapped = 0, ph = 0;
-      for (int tile = pair; tile < p.total_tiles && ok; tile += n_pairs) {
-        const bool trace_tile = (tile == pair + n_pairs); (void)trace_tile;
-        const int rt = 2 * (tile % RTP) + (int)rank, mtile = tile / RTP;
-        const int mt0 = 2 * mtile;                                           // first activation tile of the token tile
-        const int have = min(2, (int)p.aoff.MT - mt0);                       // activation tiles that exist (1 or 2)
-        const bool own = (int)rank < have;                                   // this CTA's 128 tokens exist
-        const uint8_t* wi = p.w + p.poff.wi + (size_t)rt * T2 * G::WIB;
-        const uint8_t* wo = p.w + p.poff.wo + (size_t)rt * T1 * WO_BYTES;
-        const size_t xi_tile = (size_t)T2 * xib, xo_tile = (size_t)T1 * XO_BYTES;
-        const uint8_t* xi = p.x + p.aoff.xi + (size_t)mt0 * xi_tile;         // activation tile mt0, stage 0
-        const uint8_t* xo = p.x + p.aoff.xo + (size_t)mt0 * xo_tile;
-        for (int k = 0; k < T2 + T1; ++k) {
-          if (wrapped && !(ok = ptx::mbar_wait(&empty[s >> 1], ph ^ 1))) break;
-          uint8_t* st = sm + (size_t)s * SLOT;
-          const bool first_o = (k == T2);
-          TRACE(role, k);
-          if (role == 0) {
-            if (k < T2) {
-              ptx::mbar_expect_tx(&full[s], G::WIB);
-              ptx::bulk_g2s(st, wi, G::WIB, &full[s]);
-              wi += G::WIB;
-            } else {
-              ptx::mbar_expect_tx(&full[s], WO_BYTES + (first_o ? SF_ATOM_BYTES : 0u));
-              ptx::bulk_g2s(st, wo, WO_BYTES, &full[s]);
-              if (first_o) ptx::bulk_g2s(st + G::SL_SF, p.w + p.poff.sfa_out + (size_t)rt * SF_ATOM_BYTES, SF_ATOM_BYTES, &full[s]);
-              wo += WO_BYTES;
-            }
-          } else if (role == 1) {
-            if (!own) {
-              ptx::mbar_arrive(&full[s]);
-            } else if (k < T2) {
-              ptx::mbar_expect_tx(&full[s], B4_BYTES);
-              ptx::bulk_g2s(st + G::SL_B, xi + rank * xi_tile, B4_BYTES, &full[s]);
-            } else {
-              ptx::mbar_expect_tx(&full[s], B8_BYTES);
-              ptx::bulk_g2s(st + G::SL_B, xo + rank * xo_tile, B8_BYTES, &full[s]);
-            }
-            if (k < T2) xi += xib; else xo += XO_BYTES;
-          } else {
-            if (k < T2) {
-              ptx::mbar_expect_tx(&full[s], (uint32_t)have * NA * SF_ATOM_BYTES);
-              for (int a = 0; a < have; ++a)
-                ptx::bulk_g2s(st + G::SL_SF + a * NA * SF_ATOM_BYTES, xi + a * xi_tile + B4_BYTES, NA * SF_ATOM_BYTES, &full[s]);
-              xi += xib;
-            } else if (first_o) {
-              ptx::mbar_expect_tx(&full[s], (uint32_t)have * SF_ATOM_BYTES);
-              for (int a = 0; a < have; ++a)
-                ptx::bulk_g2s(st + G::SL_SF + (1 + a) * SF_ATOM_BYTES, p.x + p.aoff.sfb_out + (size_t)(mt0 + a) * SF_ATOM_BYTES, SF_ATOM_BYTES,
-                              &full[s]);
-            } else {
-              ptx::mbar_arrive(&full[s]);
-            }
-          }
-          if (++s == NSLOT) { s = 0; wrapped = 1; ph ^= 1; }
+      uint32_t s = lane, wrapped = 0, ph = 0;
+      int tseq = 0, k = (int)lane;                                           // this lane's stage: tile number in the CTA's sequence, stage in the tile
+      if (k >= S) { k -= S; ++tseq; }                                        // (S >= 2)
+      int cur = -1, rt = 0, mt0 = 0, have = 0;
+      bool own = false;
+      for (int i = (int)lane; i < total && ok; i += 2) {
+        if (tseq != cur) {
+          cur = tseq;
+          const int tile = pair + tseq * n_pairs;
+          rt = 2 * (tile % RTP) + (int)rank;
+          mt0 = 2 * (tile / RTP);                                            // first activation tile of the token tile
+          have = min(2, (int)p.aoff.MT - mt0);                               // activation tiles that exist (1 or 2)
+          own = (int)rank < have;                                            // this CTA's 128 tokens exist
         }
+        if (wrapped && !(ok = ptx::mbar_wait(&empty[s >> 1], ph ^ 1))) break;
+        uint8_t* st = sm + (size_t)s * SLOT;
+        const bool inl = k < T2, first_o = (k == T2);
+        const int ko = k - T2;                                               // outlier stage number
+        if (role == 0) {
+          if (inl) {
+            ptx::mbar_expect_tx(&full[s], G::WIB);
+            ptx::bulk_g2s(st, p.w + p.poff.wi + ((size_t)rt * T2 + k) * G::WIB, G::WIB, &full[s]);
+          } else {
+            ptx::mbar_expect_tx(&full[s], WO_BYTES + (first_o ? SF_ATOM_BYTES : 0u));
+            ptx::bulk_g2s(st, p.w + p.poff.wo + ((size_t)rt * T1 + ko) * WO_BYTES, WO_BYTES, &full[s]);
+            if (first_o) ptx::bulk_g2s(st + G::SL_SF, p.w + p.poff.sfa_out + (size_t)rt * SF_ATOM_BYTES, SF_ATOM_BYTES, &full[s]);
+          }
+        } else if (role == 1) {
+          if (!own) {
+            ptx::mbar_arrive(&full[s]);
+          } else if (inl) {
+            ptx::mbar_expect_tx(&full[s], B4_BYTES);
+            ptx::bulk_g2s(st + G::SL_B, p.x + p.aoff.xi + (size_t)(mt0 + (int)rank) * xi_tile + (size_t)k * xib, B4_BYTES, &full[s]);
+          } else {
+            ptx::mbar_expect_tx(&full[s], B8_BYTES);
+            ptx::bulk_g2s(st + G::SL_B, p.x + p.aoff.xo + (size_t)(mt0 + (int)rank) * xo_tile + (size_t)ko * XO_BYTES, B8_BYTES, &full[s]);
+          }
+        } else {
+          if (inl) {
+            ptx::mbar_expect_tx(&full[s], (uint32_t)have * NA * SF_ATOM_BYTES);
+            for (int a = 0; a < have; ++a)
+              ptx::bulk_g2s(st + G::SL_SF + a * NA * SF_ATOM_BYTES, p.x + p.aoff.xi + (size_t)(mt0 + a) * xi_tile + (size_t)k * xib + B4_BYTES,
+                            NA * SF_ATOM_BYTES, &full[s]);
+          } else if (first_o) {
+            ptx::mbar_expect_tx(&full[s], (uint32_t)have * SF_ATOM_BYTES);
+            for (int a = 0; a < have; ++a)
+              ptx::bulk_g2s(st + G::SL_SF + (1 + a) * SF_ATOM_BYTES, p.x + p.aoff.sfb_out + (size_t)(mt0 + a) * SF_ATOM_BYTES, SF_ATOM_BYTES,
+                            &full[s]);
+          } else {
+            ptx::mbar_arrive(&full[s]);
+          }
+        }
+        s += 2;
+        if (s >= NSLOT) { s -= NSLOT; wrapped = 1; ph ^= 1; }
+        k += 2;
+        if (k >= S) { k -= S; ++tseq; }
       }
       if (!ok) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
     }
   } else if (warp == 1 && rank == 1) {
-    if (lane == 0) {
-      // ---------------- odd CTA: forward "my part of the slot has landed" to the leader's barrier
+    if (lane < 2) {
+      // ---------------- odd CTA: forward "my part of the slot has landed" to the leader's barrier (lane l: slots of parity l)
+      const int S = T2 + T1;
+      const int my_tiles = p.total_tiles > pair ? (p.total_tiles - pair + n_pairs - 1) / n_pairs : 0;
+      const int total = my_tiles * S;
       bool ok = true;
-      uint32_t s = 0, ph = 0;
-      for (int tile = pair; tile < p.total_tiles && ok; tile += n_pairs)
-        for (int k = 0; k < T2 + T1; ++k) {
-          if (!(ok = ptx::mbar_wait(&full[s], ph))) break;
-          ptx::mbar_arrive_remote(&full[s], 0);
-          if (++s == NSLOT) { s = 0; ph ^= 1; }
-        }
+      uint32_t s = lane, ph = 0;
+      for (int i = (int)lane; i < total; i += 2) {
+        if (!(ok = ptx::mbar_wait(&full[s], ph))) break;
+        ptx::mbar_arrive_remote(&full[s], 0);
+        s += 2;
+        if (s >= NSLOT) { s -= NSLOT; ph ^= 1; }
+      }
       if (!ok) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
     }
   } else if (warp == 1) {
@@ -206,10 +215,10 @@ sdq_linear_pair_kernel(const LinearParams p)
           const uint32_t idx = s + lane, sl = idx >= NSLOT ? idx - NSLOT : idx;
           const bool r = (int)lane < min((int)NSLOT, S - k) && ptx::mbar_test(&full[sl], idx >= NSLOT ? ph ^ 1 : ph);
           int n = __ffs(~__ballot_sync(0xffffffffu, r)) - 1;     // length of the run of ready slots
-          if (n == 0) {
+          if (n == 0) {   // nothing yet: wait for the next slot, then look again (its neighbours tend to land with it)
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(&full[s], ph));
             if (!ok) break;
-            n = 1;
+            continue;
           }
           if (k == 0 && tcount > 0) {   // the epilogues of both CTAs must have drained the accumulator of the previous tile
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_empty, (tcount - 1) & 1));
@@ -406,11 +415,13 @@ static cudaError_t launch_one(const LinearParams& p, int pairs, cudaStream_t str
   return cudaLaunchKernelEx(&lc, kern, p);
 }
 
-bool pair_kernel_applies(int64_t M, int64_t N, int64_t K)
+bool pair_kernel_applies(int64_t M, int64_t N, int64_t K, int out_n)
 {
-  // K = 256 is left to the single-CTA kernel: with one inlier stage per tile and seven ring slots the outlier scales of
-  // the tile after next could reach TMEM while this tile's last MMAs still read theirs
-  return M > 128 && N % (2 * TILE_ROWS) == 0 && K >= 2 * K2;
+  // The accumulator is not double-buffered, so every tile pays for the epilogue's drain of TMEM (~1 us); tiles of fewer
+  // than 32 stages (no outlier part and K <= 7936, or K < 2816 with one) run faster on the single-CTA kernel's smaller
+  // tiles (measured: 4096 -> 11008 without outliers 40 against 36 us; 11008 -> 4096 without outliers 30 against 34 us).
+  const int64_t stages = K / K2 + (out_n ? K / K1 : 0);
+  return M > 128 && N % (2 * TILE_ROWS) == 0 && stages >= 32;
 }
 
 cudaError_t launch_linear_pair(LinearParams p, bool f32_out, int sm_count, cudaStream_t stream, uint32_t* attr_mask)
@@ -432,8 +443,3 @@ cudaError_t launch_linear_pair(LinearParams p, bool f32_out, int sm_count, cudaS
 
 }  // namespace sdq
 
-#ifdef SDQ_PAIR_TRACE
-extern "C" int sdq_pair_trace_read(unsigned long long* host) {
-  return (int)cudaMemcpyFromSymbol(host, sdq::g_trace, sizeof(sdq::g_trace));
-}
-#endif
