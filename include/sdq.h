@@ -91,7 +91,8 @@ typedef struct {
 /* Host-side descriptor of a packed weight matrix (filled by sdq_decompose; plain data, may be
  * copied; `dev` stays owned by the caller).  off[] are byte offsets of the sections inside dev:
  *   0 inlier stages  1 outlier stages (tensor-core 2:4 form)  2 outlier row-scale atoms
- *   3 compact outlier codes  4 compact outlier indices  5 outlier scale exponents
+ *   3 outlier stages in compact form (8-bit code + position nibble per outlier; tiled configurations; the
+ *     decompose-only reading keeps plain code / index arrays at 3 and 4)  4 see 3  5 outlier scale exponents
  *   6 inlier row-factor exponents (SDQ_SCALE_UE4M3; zeros otherwise)  7 reserved */
 typedef struct {
   void* dev;
@@ -220,6 +221,24 @@ sdq_status_t sdq_linear_ws(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y_b
                            void* stream);
 sdq_status_t sdq_linear_f32_ws(const sdq_act_t* Xq, const sdq_packed_t* P, float* Y_f32, int64_t ldy, void* ws, size_t ws_bytes,
                                void* stream);
+
+/* Several independent layers in one call: Y[i] = A_i,in W_i,in^T + A_i,out W_i,out^T for i = 0 .. n - 1
+ * (Section 5.1, O = O_i + O_o, once per layer; Section 5, Stage 3 supplies each layer's quantized operands).  The
+ * layers must not depend on one another (q / k / v projections or gate / up, which may share one Xq; the layers of a
+ * benchmark rotation): they may run in any order and concurrently.
+ *   Xq, P, Y, ldy: host arrays of n entries (descriptors and pointers as for sdq_linear; the arrays themselves are read
+ *   during the call only).  Outputs must not overlap.
+ *   When every layer has at most 32 tokens, the primary format (SDQ_GRAN_PAIR, in_block 64, out_n <= 1, power-of-two
+ *   scales), n <= 32 and the layers together have at least half as many 128-row tiles as the GPU has SMs, the call is ONE
+ *   persistent kernel launch that streams all weights once, the outlier part in its compact form (8-bit code + position per
+ *   S-Vector, rebuilt into the tensor core's 2:4 form in shared memory); the summation order over K of an output differs
+ *   from sdq_linear's split-K paths, so results agree to fp32 rounding, not bit for bit.  Otherwise the layers are
+ *   enqueued one after the other exactly as sdq_linear would.
+ *   Asynchronous on `stream`; allocates nothing.  Errors as sdq_linear (the first failing layer's). */
+sdq_status_t sdq_linear_group(int n, const sdq_act_t* const* Xq, const sdq_packed_t* const* P, void* const* Y_bf16,
+                              const int64_t* ldy, void* stream);
+sdq_status_t sdq_linear_group_f32(int n, const sdq_act_t* const* Xq, const sdq_packed_t* const* P, float* const* Y_f32,
+                                  const int64_t* ldy, void* stream);
 
 /* Built-in scratch variant of sdq_linear_ws (the paper has no counterpart: this is a packaging choice of the
  * library, not part of the method).

@@ -65,7 +65,7 @@ class _ActCanon(ctypes.Structure):
 
 EXPORTS = ["sdq_packed_size", "sdq_decompose", "sdq_decompose_metric", "sdq_channel_norm", "sdq_packed_export", "sdq_act_size", "sdq_quantize_act", "sdq_act_export",
            "sdq_linear", "sdq_linear_f32", "sdq_workspace_size", "sdq_workspace_init", "sdq_linear_ws", "sdq_linear_f32_ws", "sdq_linear_noalloc",
-           "sdq_diag_l2_copy", "sdq_device_status", "sdq_status_string"]
+           "sdq_linear_group", "sdq_linear_group_f32", "sdq_diag_l2_copy", "sdq_device_status", "sdq_status_string"]
 
 _lib = None
 
@@ -95,6 +95,8 @@ def lib() -> ctypes.CDLL:
         L.sdq_linear_ws.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_Packed), vp, i64, vp, sz, vp]
         L.sdq_linear_f32_ws.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_Packed), vp, i64, vp, sz, vp]
         L.sdq_linear_noalloc.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_Packed), vp, i64, vp]
+        L.sdq_linear_group.argtypes = [ctypes.c_int, vp, vp, vp, vp, vp]
+        L.sdq_linear_group_f32.argtypes = [ctypes.c_int, vp, vp, vp, vp, vp]
         L.sdq_device_status.argtypes = [vp]
         L.sdq_status_string.argtypes = [ctypes.c_int]
         L.sdq_status_string.restype = ctypes.c_char_p
@@ -230,6 +232,25 @@ def sdq_linear(xq: QuantAct, p: PackedWeight, out: torch.Tensor | None = None, f
         _check(fn(ctypes.byref(xq.desc), ctypes.byref(p.desc), out.data_ptr(), out.stride(0), workspace.data_ptr(),
                   workspace.numel(), _stream()), "sdq_linear_ws")
     return out
+
+
+def sdq_linear_group(xqs, ps, outs=None, f32: bool = False):
+    """Y[i] = sdq_linear(xqs[i], ps[i]) for independent layers in one call (one persistent launch when every layer has few
+    tokens and the group is large enough; see sdq_linear_group in include/sdq.h).  Returns the list of outputs."""
+    n = len(ps)
+    assert n == len(xqs) and n > 0
+    dt = torch.float32 if f32 else torch.bfloat16
+    if outs is None:
+        outs = [torch.empty((x.M, p.N), dtype=dt, device=p.buf.device) for x, p in zip(xqs, ps)]
+    for o, x, p in zip(outs, xqs, ps):
+        assert o.dtype == dt and o.shape == (x.M, p.N) and o.stride(1) == 1
+    XA = (ctypes.POINTER(_Act) * n)(*[ctypes.pointer(x.desc) for x in xqs])
+    PA = (ctypes.POINTER(_Packed) * n)(*[ctypes.pointer(p.desc) for p in ps])
+    YA = (ctypes.c_void_p * n)(*[o.data_ptr() for o in outs])
+    LD = (ctypes.c_int64 * n)(*[o.stride(0) for o in outs])
+    fn = lib().sdq_linear_group_f32 if f32 else lib().sdq_linear_group
+    _check(fn(n, XA, PA, YA, LD, _stream()), "sdq_linear_group")
+    return outs
 
 
 def diag_l2_copy(src: torch.Tensor, slot_bytes: int, nslot: int, iters: int, issuers: int = 1) -> int:

@@ -23,9 +23,15 @@
 //            embedding of the 1:8 / 2:8 outliers), same addressing as A_in
 //     E_out: 128 rows x 16 B  (one 4-bit index pair per 4 logical K over 128 K)
 //   section SFA_out[rt]: 512 B, the per-row outlier scale as an E8M0 code, scale-atom form, 4 copies
-//   sections compact outlier codes / indices [N][K/8][out_n] u8, row scale exponents [N] i32, inlier row-factor
-//   exponents [N] i32 (two-level scaling with E4M3 Q-Vector scales; zeros otherwise); element-wise 2:4 inliers with one
-//   scale per 32 K are stored like dense inliers, plus their kept indices [N][K/4] u8 for the exporter
+//   section WC[rt][k1] = | codes 128 rows x 16 out_n B | positions 128 rows x 8 out_n B |   (3072 out_n B)
+//     the outliers in the form the method states them (one 8-bit code + one 3-bit position per S-Vector of 8 and
+//     outlier, 12 of the 11 algorithmic bits): row r, S-Vector g (0..15 inside the 128-K stage), outlier t: code byte at
+//     r * 16 out_n + g * out_n + t; position (0..7) in nibble (g * out_n + t) & 1 of byte
+//     2048 out_n + r * 8 out_n + (g * out_n + t) / 2.  Few-token calls stream this section instead of WO and rebuild
+//     the 2:4 form in shared memory; the exporter reads it.
+//   sections row scale exponents [N] i32, inlier row-factor exponents [N] i32 (two-level scaling with E4M3 Q-Vector
+//   scales; zeros otherwise); element-wise 2:4 inliers with one scale per 32 K are stored like dense inliers, plus their
+//   kept indices [N][K/4] u8 for the exporter
 //
 // Activation buffer (per 128-token tile mt)
 //   section XI[mt][k2] = | B4 16384 | SFB_in 512 |            (one scale per 32 K: SFB_in 2 x 512, as for the weights)
@@ -51,6 +57,9 @@ constexpr int WI_BYTES = A_IN_BYTES + E_IN_BYTES + SF_ATOM_BYTES;   // 10752
 constexpr int A_OUT_BYTES = 8192;     // per 128 K
 constexpr int E_OUT_BYTES = 2048;
 constexpr int WO_BYTES = A_OUT_BYTES + E_OUT_BYTES;                  // 10240
+constexpr int WC_CODE_BYTES = 2048;   // per 128 K and outlier of the S-Vector: 128 rows x 16 code bytes
+constexpr int WC_POS_BYTES = 1024;    //                                        128 rows x 16 position nibbles
+__host__ __device__ inline int wc_bytes(int out_n) { return (WC_CODE_BYTES + WC_POS_BYTES) * out_n; }
 constexpr int B4_BYTES = 16384;       // 128 tokens x 256 K
 constexpr int XI_BYTES = B4_BYTES + SF_ATOM_BYTES;                   // 16896
 constexpr int B8_BYTES = 16384;       // 128 tokens x 128 K
@@ -85,7 +94,7 @@ __host__ __device__ inline uint32_t sf_off(uint32_t row, uint32_t s) { return (r
 constexpr size_t HEADER_BYTES = 256;
 
 struct PackedOffsets {
-  size_t wi, wo, sfa_out, ocode, oidx, osexp, wtexp, emeta, total;
+  size_t wi, wo, sfa_out, wc, osexp, wtexp, emeta, total;
 };
 inline PackedOffsets packed_offsets(int64_t N, int64_t K, int out_n, bool b32 = false, bool dense = false, bool elem = false) {
   PackedOffsets o;
@@ -94,9 +103,8 @@ inline PackedOffsets packed_offsets(int64_t N, int64_t K, int out_n, bool b32 = 
   o.wi = HEADER_BYTES;
   o.wo = al(o.wi + RT * T2 * (size_t)wi_bytes(b32, dense));
   o.sfa_out = al(o.wo + (out_n ? RT * T1 * WO_BYTES : 0));
-  o.ocode = al(o.sfa_out + RT * SF_ATOM_BYTES);
-  o.oidx = al(o.ocode + (size_t)N * (size_t)(K / 8) * (size_t)out_n);
-  o.osexp = al(o.oidx + (size_t)N * (size_t)(K / 8) * (size_t)out_n);
+  o.wc = al(o.sfa_out + RT * SF_ATOM_BYTES);
+  o.osexp = al(o.wc + RT * T1 * (size_t)wc_bytes(out_n));
   o.wtexp = al(o.osexp + (size_t)N * 4);                          // inlier row-factor exponents [N] i32 (two-level scaling)
   o.emeta = al(o.wtexp + (size_t)N * 4);                          // element-wise 2:4 stored dense: kept indices [N][K/4] u8
   o.total = al(o.emeta + (elem ? (size_t)N * (size_t)(K / 4) : 0));

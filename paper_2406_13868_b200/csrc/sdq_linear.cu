@@ -894,6 +894,69 @@ extern "C" sdq_status_t sdq_linear_f32_ws(const sdq_act_t* Xq, const sdq_packed_
 { return launch_linear(Xq, P, (void*)Y, ldy, ws, ws_bytes, stream, true); }
 
 // ---------------------------------------------------------------------------------------------------------
+// Several independent layers in one call (see include/sdq.h).  Few tokens everywhere and enough row tiles to occupy
+// the GPU: one persistent launch of the grouped kernel; otherwise the layers are enqueued one after the other.
+static sdq_status_t launch_group(int n, const sdq_act_t* const* Xq, const sdq_packed_t* const* P, void* const* Y, const int64_t* ldy,
+                                 void* stream, bool f32)
+{
+  if (n <= 0 || !Xq || !P || !Y || !ldy) return SDQ_ERR_INVALID_ARG;
+  DeviceInfo* dinfo = device_info();
+  if (!dinfo) return SDQ_ERR_CUDA;
+  bool fused = n <= GROUP_MAX;
+  int64_t items = 0, max_m = 0;
+  for (int i = 0; i < n; ++i) {
+    const sdq_act_t* x = Xq[i];
+    const sdq_packed_t* w = P[i];
+    if (!x || !w || !Y[i] || !x->dev || !w->dev) return SDQ_ERR_INVALID_ARG;
+    if (x->K != w->K || x->M <= 0 || w->N <= 0 || w->N % TILE_ROWS || w->K % K2 || ldy[i] < w->N) return SDQ_ERR_SHAPE;
+    if (x->cfg.in_block != w->cfg.in_block || x->cfg.scale_rule != w->cfg.scale_rule) return SDQ_ERR_SHAPE;
+    if (!is_tensor_core_reading(w->cfg)) return SDQ_ERR_UNSUPPORTED;
+    if (((uintptr_t)Y[i] & 15) || (ldy[i] % 8)) return SDQ_ERR_ALIGNMENT;
+    // the grouped kernel carries the primary format: pair-wise 4:8 inliers, one E8M0 scale per 64 K, at most one outlier per S-Vector
+    fused = fused && x->M <= 32 && w->cfg.in_gran == SDQ_GRAN_PAIR && w->cfg.in_block == 64 && w->cfg.scale_rule != SDQ_SCALE_UE4M3 &&
+            w->cfg.out_n <= 1;
+    items += w->N / TILE_ROWS;
+    if (x->M > max_m) max_m = x->M;
+  }
+  fused = fused && items * 2 >= dinfo->sm_count && items < (1 << 30) && !getenv("SDQ_NO_GROUP");
+  if (!fused) {
+    for (int i = 0; i < n; ++i) {
+      const sdq_status_t st = launch_linear(Xq[i], P[i], Y[i], ldy[i], nullptr, 0, stream, f32);
+      if (st != SDQ_OK) return st;
+    }
+    return SDQ_OK;
+  }
+  GroupParams g;
+  g.n = n;
+  g.n_tile = max_m <= 16 ? 16 : 32;
+  g.total_items = (int)items;
+  g.flags = device_flags();
+  if (!g.flags) return SDQ_ERR_CUDA;
+  int item0 = 0;
+  for (int i = 0; i < n; ++i) {
+    const PackedOffsets po = tiled_offsets(P[i]->N, P[i]->K, P[i]->cfg);
+    const ActOffsets ao = act_offsets(Xq[i]->M, Xq[i]->K, false);
+    GroupMat& m = g.m[i];
+    m.w = (const uint8_t*)P[i]->dev; m.x = (const uint8_t*)Xq[i]->dev; m.Y = Y[i]; m.ldy = ldy[i];
+    m.wi = po.wi; m.wc = po.wc; m.sfa_out = po.sfa_out;
+    m.xi = ao.xi; m.xo = ao.xo; m.sfb_out = ao.sfb_out;
+    m.M = (int)Xq[i]->M; m.T2 = (int)(P[i]->K / K2); m.out_n = P[i]->cfg.out_n;
+    m.item0 = item0;
+    item0 += (int)(P[i]->N / TILE_ROWS);
+  }
+  const cudaError_t e = launch_linear_group(g, f32, dinfo->sm_count, (cudaStream_t)stream, &dinfo->group_attr);
+  return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
+}
+
+extern "C" sdq_status_t sdq_linear_group(int n, const sdq_act_t* const* Xq, const sdq_packed_t* const* P, void* const* Y,
+                                         const int64_t* ldy, void* stream)
+{ return launch_group(n, Xq, P, Y, ldy, stream, false); }
+
+extern "C" sdq_status_t sdq_linear_group_f32(int n, const sdq_act_t* const* Xq, const sdq_packed_t* const* P, float* const* Y,
+                                             const int64_t* ldy, void* stream)
+{ return launch_group(n, Xq, P, (void* const*)Y, ldy, stream, true); }
+
+// ---------------------------------------------------------------------------------------------------------
 // Allocation-free variant of sdq_linear_ws (see include/sdq.h).  The split-K scratch lives in this library's
 // own device image instead of a caller buffer.
 namespace sdq {

@@ -38,6 +38,26 @@ struct LinearParams {
   uint32_t* flags;
 };
 
+// Grouped few-token kernel (sdq_linear_group.cu): one persistent launch over the (matrix, 128-row tile) work items of
+// up to GROUP_MAX independent linear layers.
+constexpr int GROUP_MAX = 32;
+struct GroupMat {
+  const uint8_t* w;      // packed weights
+  const uint8_t* x;      // quantized activations
+  void* Y;
+  int64_t ldy;
+  uint64_t wi, wc, sfa_out;       // sections of w: inlier stages, compact outlier stages, outlier row-scale atoms
+  uint64_t xi, xo, sfb_out;       // sections of x: 4-bit stages, 8-bit stages, token-scale atom
+  int M, T2, out_n;      // tokens, K / 256, outliers per S-Vector (0 or 1)
+  int item0;             // number of the matrix's first work item (= row tiles of the matrices before it)
+};
+struct GroupParams {
+  int n, n_tile, nslot, slot_bytes, total_items;
+  uint32_t* flags;
+  GroupMat m[GROUP_MAX];
+};
+cudaError_t launch_linear_group(GroupParams p, bool f32_out, int sm_count, cudaStream_t stream, uint32_t* attr_done);
+
 // CTA-pair (tcgen05 cta_group::2) many-token kernel: tiles of 256 weight rows x 256 tokens (sdq_linear_pair.cu).
 // `attr_mask` is the calling device's record of which instantiations already carry their shared-memory attribute.
 bool pair_kernel_applies(int64_t M, int64_t N, int64_t K, int out_n);

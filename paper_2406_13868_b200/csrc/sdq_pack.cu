@@ -255,11 +255,17 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
       // FP8 tensor-core path consumes (per 4 K: two ascending slot indices, unused slots hold +0)
       const uint32_t c0 = e4m3x1(bf16_bits_to_float(bits[o0]) * pow2_neg(e));
       const uint32_t c1 = (o1 >= 0) ? e4m3x1(bf16_bits_to_float(bits[o1]) * pow2_neg(e)) : 0u;
-      uint8_t* oc = blob + off.ocode + ((size_t)n * G + g) * out_n;
-      uint8_t* oi = blob + off.oidx + ((size_t)n * G + g) * out_n;
-      oc[0] = (uint8_t)c0;
-      oi[0] = (uint8_t)o0;
-      if (out_n == 2) { oc[1] = (uint8_t)c1; oi[1] = (uint8_t)o1; }
+      // compact record of the 128-K stage: codes, then position nibbles (two S-Vectors share a byte when out_n = 1)
+      uint8_t* wc = blob + off.wc + ((size_t)rt * T1 + k1) * (size_t)wc_bytes(out_n);
+      const uint32_t gi = (uint32_t)(g & 15);
+      if (out_n == 1) {
+        wc[r * 16 + gi] = (uint8_t)c0;
+        const uint32_t pos_hi = __shfl_down_sync(0xffffffffu, (uint32_t)o0, 1);
+        if ((g & 1) == 0) wc[WC_CODE_BYTES + r * 8 + (gi >> 1)] = (uint8_t)((uint32_t)o0 | (pos_hi << 4));
+      } else {
+        *reinterpret_cast<uint16_t*>(wc + r * 32 + gi * 2) = (uint16_t)(c0 | (c1 << 8));
+        wc[2 * WC_CODE_BYTES + r * 16 + gi] = (uint8_t)((uint32_t)o0 | ((uint32_t)o1 << 4));
+      }
       uint32_t stored = 0, meta = 0;
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
@@ -283,6 +289,17 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
   }
 }
 
+// outlier t of S-Vector g of row r in row tile rt, from the compact records: code and position
+__device__ __forceinline__ uint8_t wc_code(const uint8_t* blob, const PackedOffsets& off, int64_t rt, int T1, uint32_t r, int g, int out_n, int t) {
+  const uint8_t* wc = blob + off.wc + ((size_t)rt * T1 + (g >> 4)) * (size_t)wc_bytes(out_n);
+  return wc[r * 16 * out_n + (g & 15) * out_n + t];
+}
+__device__ __forceinline__ uint8_t wc_pos(const uint8_t* blob, const PackedOffsets& off, int64_t rt, int T1, uint32_t r, int g, int out_n, int t) {
+  const uint8_t* wc = blob + off.wc + ((size_t)rt * T1 + (g >> 4)) * (size_t)wc_bytes(out_n);
+  const int e = (g & 15) * out_n + t;
+  return (uint8_t)((wc[WC_CODE_BYTES * out_n + r * 8 * out_n + (e >> 1)] >> (4 * (e & 1))) & 15);
+}
+
 // packed buffer -> canonical arrays (one code per byte)
 __global__ void __launch_bounds__(128)
 export_packed_kernel(const uint8_t* __restrict__ blob, int64_t N, int64_t K, sdq_config_t cfg, PackedOffsets off, sdq_canonical_t out)
@@ -291,7 +308,7 @@ export_packed_kernel(const uint8_t* __restrict__ blob, int64_t N, int64_t K, sdq
   const int G = (int)(K / 8), out_n = cfg.out_n;
   const int64_t rt = n / TILE_ROWS;
   const uint32_t r = (uint32_t)(n % TILE_ROWS);
-  const int T2 = (int)(K / K2);
+  const int T1 = (int)(K / K1), T2 = (int)(K / K2);
   const bool b32 = cfg.in_block == 32, dense = is_dense_layout(cfg), elem = cfg.in_gran == SDQ_GRAN_ELEM;
   const int wib = wi_bytes(b32, dense);
   const uint8_t* wi_base = blob + off.wi + (size_t)rt * T2 * wib;
@@ -316,8 +333,8 @@ export_packed_kernel(const uint8_t* __restrict__ blob, int64_t N, int64_t K, sdq
       }
       if ((g & 3) == 0) out.in_scale[(size_t)n * (K / 32) + (g >> 2)] = wi[a_in_bytes(true) + in_sf_off(true, r, (uint32_t)((g >> 2) & 7))];
       for (int t = 0; t < out_n; ++t) {
-        out.out_code[((size_t)n * G + g) * out_n + t] = blob[off.ocode + ((size_t)n * G + g) * out_n + t];
-        out.out_idx[((size_t)n * G + g) * out_n + t] = blob[off.oidx + ((size_t)n * G + g) * out_n + t];
+        out.out_code[((size_t)n * G + g) * out_n + t] = wc_code(blob, off, rt, T1, r, g, out_n, t);
+        out.out_idx[((size_t)n * G + g) * out_n + t] = wc_pos(blob, off, rt, T1, r, g, out_n, t);
       }
       continue;
     }
@@ -329,8 +346,8 @@ export_packed_kernel(const uint8_t* __restrict__ blob, int64_t N, int64_t K, sdq
     if (b32) { if ((g & 3) == 0) out.in_scale[(size_t)n * (K / 32) + (g >> 2)] = wi[A_IN_BYTES + E_IN_BYTES + in_sf_off(true, r, (uint32_t)((g >> 2) & 7))]; }
     else if ((g & 7) == 0) out.in_scale[(size_t)n * (K / 64) + (g >> 3)] = wi[A_IN_BYTES + E_IN_BYTES + in_sf_off(false, r, (uint32_t)((g >> 3) & 3))];
     for (int t = 0; t < out_n; ++t) {
-      out.out_code[((size_t)n * G + g) * out_n + t] = blob[off.ocode + ((size_t)n * G + g) * out_n + t];
-      out.out_idx[((size_t)n * G + g) * out_n + t] = blob[off.oidx + ((size_t)n * G + g) * out_n + t];
+      out.out_code[((size_t)n * G + g) * out_n + t] = wc_code(blob, off, rt, T1, r, g, out_n, t);
+      out.out_idx[((size_t)n * G + g) * out_n + t] = wc_pos(blob, off, rt, T1, r, g, out_n, t);
     }
   }
   if (threadIdx.x == 0) {
@@ -409,7 +426,7 @@ extern "C" sdq_status_t sdq_decompose_metric(const void* W, int64_t N, int64_t K
   for (int i = 0; i < 8; ++i) out->off[i] = 0;
   if (tc) {
     out->off[0] = off.wi; out->off[1] = off.wo; out->off[2] = off.sfa_out;
-    out->off[3] = off.ocode; out->off[4] = off.oidx; out->off[5] = off.osexp; out->off[6] = off.wtexp;
+    out->off[3] = off.wc; out->off[4] = 0; out->off[5] = off.osexp; out->off[6] = off.wtexp;
   } else {
     out->off[0] = poff.in_code; out->off[1] = poff.in_meta; out->off[2] = poff.in_scale;
     out->off[3] = poff.out_code; out->off[4] = poff.out_idx; out->off[5] = poff.osexp;
