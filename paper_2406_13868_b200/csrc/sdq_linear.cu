@@ -914,7 +914,7 @@ static sdq_status_t launch_group(int n, const sdq_act_t* const* Xq, const sdq_pa
     if (((uintptr_t)Y[i] & 15) || (ldy[i] % 8)) return SDQ_ERR_ALIGNMENT;
     // the grouped kernel carries the primary format: pair-wise 4:8 inliers, one E8M0 scale per 64 K, at most one outlier per S-Vector
     fused = fused && x->M <= 32 && w->cfg.in_gran == SDQ_GRAN_PAIR && w->cfg.in_block == 64 && w->cfg.scale_rule != SDQ_SCALE_UE4M3 &&
-            w->cfg.out_n <= 1;
+            w->cfg.out_n <= 1 && w->cfg.out_n == P[0]->cfg.out_n;
     items += w->N / TILE_ROWS;
     if (x->M > max_m) max_m = x->M;
   }
@@ -929,6 +929,7 @@ static sdq_status_t launch_group(int n, const sdq_act_t* const* Xq, const sdq_pa
   GroupParams g;
   g.n = n;
   g.n_tile = max_m <= 16 ? 16 : 32;
+  g.out_n = P[0]->cfg.out_n;
   g.total_items = (int)items;
   g.flags = device_flags();
   if (!g.flags) return SDQ_ERR_CUDA;
@@ -940,7 +941,7 @@ static sdq_status_t launch_group(int n, const sdq_act_t* const* Xq, const sdq_pa
     m.w = (const uint8_t*)P[i]->dev; m.x = (const uint8_t*)Xq[i]->dev; m.Y = Y[i]; m.ldy = ldy[i];
     m.wi = po.wi; m.wc = po.wc; m.sfa_out = po.sfa_out;
     m.xi = ao.xi; m.xo = ao.xo; m.sfb_out = ao.sfb_out;
-    m.M = (int)Xq[i]->M; m.T2 = (int)(P[i]->K / K2); m.out_n = P[i]->cfg.out_n;
+    m.M = (int)Xq[i]->M; m.T2 = (int)(P[i]->K / K2);
     m.item0 = item0;
     item0 += (int)(P[i]->N / TILE_ROWS);
   }
