@@ -44,8 +44,10 @@ constexpr int GRP_BAR_BYTES = (3 * GRP_MAX_UNITS + 2 + 4) * 8 + 8;
 
 // inlier slot: | WI record | 4-bit codes of the tokens | their scale atom |
 __host__ __device__ inline int group_is_bytes(int n_tile) { return WI_BYTES + n_tile * 128 + SF_ATOM_BYTES; }
-// outlier slot: | two compact records (128 K each) | 8-bit codes of the tokens, 2 x 128 K | row / token scale atoms (first unit only) |
-__host__ __device__ inline int group_os_bytes(int n_tile) { return 2 * wc_bytes(1) + 2 * n_tile * 128 + 2 * SF_ATOM_BYTES; }
+// outlier slot: | two compact records (128 K each) | 8-bit codes of the tokens, 2 x 128 K |
+__host__ __device__ inline int group_os_bytes(int n_tile) { return 2 * wc_bytes(1) + 2 * n_tile * 128; }
+// beside the ring: two container pairs and, alternating per item, the outlier row / token scale atoms (SFA_out | SFB_out)
+constexpr int GRP_SIDE_BYTES = 4 * WO_BYTES + 2 * 2 * SF_ATOM_BYTES;
 
 // matrix of work item `item` (items are numbered matrix by matrix)
 __device__ __forceinline__ int group_mat_of(const GroupParams& p, int item) {
@@ -65,7 +67,8 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
   const uint32_t xb = (uint32_t)p.n_tile * 128u, isb = (uint32_t)group_is_bytes(p.n_tile), osb = p.out_n ? (uint32_t)group_os_bytes(p.n_tile) : 0u;
   const uint32_t ub = isb + osb;                                             // bytes of a unit: inlier slot, then outlier slot
   uint8_t* cbuf = sm + NU * ub;                                              // two container pairs: 2 x (2 x WO_BYTES)
-  uint64_t* full_is = reinterpret_cast<uint64_t*>(cbuf + (p.out_n ? 4 * WO_BYTES : 0));   // inlier slot of ring position v has landed
+  uint8_t* sfbuf = cbuf + 4 * WO_BYTES;                                      // 2 x (SFA_out | SFB_out) of the item, alternating
+  uint64_t* full_is = reinterpret_cast<uint64_t*>(cbuf + (p.out_n ? GRP_SIDE_BYTES : 0));   // inlier slot of ring position v has landed
   uint64_t* full_os = full_is + GRP_MAX_UNITS;                               // outlier slot of ring position v has landed
   uint64_t* done = full_os + GRP_MAX_UNITS;                                  // the MMAs of the unit at ring position v have completed
   uint64_t* built = done + GRP_MAX_UNITS;                                    // [2] container pair is rebuilt
@@ -97,13 +100,14 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
       bool ok = true;
       int item = first, k2 = (int)lane;          // this lane's position: work item and 256-K unit inside the item
       int mat = -1, rt = 0;
+      uint32_t iseq = 0;                         // number of the item in this CTA's sequence
       uint32_t v = lane, wrapped = 0, ph = 0;    // ring position, whether the ring has wrapped, parity of `done` to wait for
       for (;;) {
         for (;;) {                               // advance to the item that holds unit k2
           if (item >= p.total_items) break;
           if (mat < 0) { mat = group_mat_of(p, item); rt = item - p.m[mat].item0; }
           if (k2 < p.m[mat].T2) break;
-          k2 -= p.m[mat].T2; item += stride; mat = -1;
+          k2 -= p.m[mat].T2; item += stride; mat = -1; ++iseq;
         }
         if (item >= p.total_items) break;
         const GroupMat& m = p.m[mat];
@@ -122,9 +126,10 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
           ptx::bulk_g2s(st, m.w + m.wc + ((size_t)rt * 2 * m.T2 + 2 * k2) * (size_t)wc_bytes(1), wcb, &full_os[v]);
           ptx::bulk_g2s(st + wcb, xo, xb, &full_os[v]);
           ptx::bulk_g2s(st + wcb + xb, xo + XO_BYTES, xb, &full_os[v]);
-          if (k2 == 0) {
-            ptx::bulk_g2s(st + wcb + 2 * xb, m.w + m.sfa_out + (size_t)rt * SF_ATOM_BYTES, SF_ATOM_BYTES, &full_os[v]);
-            ptx::bulk_g2s(st + wcb + 2 * xb + SF_ATOM_BYTES, m.x + m.sfb_out, SF_ATOM_BYTES, &full_os[v]);
+          if (k2 == 0) {   // the item's outlier scale atoms ride on its first unit's barrier
+            uint8_t* sf = sfbuf + (iseq & 1) * 2 * SF_ATOM_BYTES;
+            ptx::bulk_g2s(sf, m.w + m.sfa_out + (size_t)rt * SF_ATOM_BYTES, SF_ATOM_BYTES, &full_os[v]);
+            ptx::bulk_g2s(sf + SF_ATOM_BYTES, m.x + m.sfb_out, SF_ATOM_BYTES, &full_os[v]);
           }
         }
         k2 += 2;
@@ -170,8 +175,9 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
           if (p.out_n) {
             const uint32_t ob = sb + isb;
             if (k2 == 0) {
-              ptx::tc_cp_32x128b_warpx4(so, ptx::smem_desc(ob + wcb + 2 * xb, 0, 128));
-              ptx::tc_cp_32x128b_warpx4(so + 4, ptx::smem_desc(ob + wcb + 2 * xb + SF_ATOM_BYTES, 0, 128));
+              const uint32_t sf = cbb + 4 * WO_BYTES + ab * 2 * SF_ATOM_BYTES;
+              ptx::tc_cp_32x128b_warpx4(so, ptx::smem_desc(sf, 0, 128));
+              ptx::tc_cp_32x128b_warpx4(so + 4, ptx::smem_desc(sf + SF_ATOM_BYTES, 0, 128));
             }
 #pragma unroll
             for (uint32_t h = 0; h < 2; ++h) {
@@ -200,9 +206,12 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
       const GroupMat& m = p.m[mat];
       const int64_t n0 = (int64_t)(item - m.item0) * TILE_ROWS;
       const uint32_t ab = itc & 1;
-      ok = ptx::mbar_wait(&acc_full[ab], (itc >> 1) & 1);
+      // one thread polls the barrier and releases the other 127 through a hardware barrier: many threads polling an mbarrier
+      // slow every other barrier operation of the CTA down
+      if (warp == 2 && lane == 0 && !ptx::mbar_wait(&acc_full[ab], (itc >> 1) & 1)) *timed_out = 1u;
+      ptx::named_bar_sync(3, 128);
+      if (*timed_out) { ok = false; break; }
       ptx::tc_fence_after();
-      if (!ok) break;
       uint32_t val[32];
       {
         uint32_t a[16], b[16];
@@ -254,20 +263,21 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
         const uint4 codes = *reinterpret_cast<const uint4*>(st + r * 16);
         const uint2 pos = *reinterpret_cast<const uint2*>(st + WC_CODE_BYTES + r * 8);
         const uint32_t cw[4] = {codes.x, codes.y, codes.z, codes.w}, pw[2] = {pos.x, pos.y};
-        uint32_t stored[16], meta[4] = {0u, 0u, 0u, 0u};
+        // position ps (0..7) of the outlier in its S-Vector: it sits in the group of 4 number ps >> 2 at p = ps & 3.  Stored
+        // bytes of the S-Vector (two per group of 4): the code moves to byte (p == 3) + 2 (ps >> 2); metadata byte = the two
+        // groups' slot-index nibbles, (p, 3) or (0, 3) for p = 3 where the outlier is, (0, 1) elsewhere.  Both come from
+        // 8-entry byte tables held in two registers each, and one byte-permute looks up four S-Vectors at a time: the four
+        // position nibbles of a 16-bit piece of the position word are its selector.
+        uint32_t stored[16], meta[4], shw[4];
 #pragma unroll
-        for (int g = 0; g < 16; ++g) {
-          // position ps (0..7) of the outlier in its S-Vector: it sits in the group of 4 number ps >> 2 at p = ps & 3.  Stored
-          // bytes of the S-Vector (two per group of 4): the code moves to byte (p == 3) + 2 (ps >> 2); metadata byte = the two
-          // groups' slot-index nibbles, (p, 3) or (0, 3) for p = 3 where the outlier is, (0, 1) elsewhere -- both from
-          // 8-entry byte tables held in two registers each
-          const uint32_t code = __byte_perm(cw[g >> 2], 0u, 0x4440u + (uint32_t)(g & 3));
-          const uint32_t ps = (pw[g >> 3] >> (4 * (g & 7))) & 7u;
-          const uint32_t sh = __byte_perm(0x08000000u, 0x18101010u, ps) & 0xFFu;
-          stored[g] = code << sh;
-          const uint32_t mbyte = __byte_perm(0x4C4E4D4Cu, 0xC4E4D4C4u, ps) & 0xFFu;
-          meta[g >> 2] |= mbyte << (8 * (g & 3));
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t sel = pw[i >> 1] >> (16 * (i & 1));
+          meta[i] = __byte_perm(0x4C4E4D4Cu, 0xC4E4D4C4u, sel);
+          shw[i] = __byte_perm(0x08000000u, 0x18101010u, sel);
         }
+#pragma unroll
+        for (int g = 0; g < 16; ++g)
+          stored[g] = __byte_perm(cw[g >> 2], 0u, 0x4440u + (uint32_t)(g & 3)) << ((shw[g >> 2] >> (8 * (g & 3))) & 0xFFu);
         uint8_t* cb = cbuf + (size_t)((u & 1) * 2 + h) * WO_BYTES;
         // row r: bytes 0..31 of its 64 stored bytes belong to K-block 0, 32..63 to K-block 1; 16-byte chunks 128 B apart
         uint8_t* arow = cb + (r >> 3) * 256 + (r & 7) * 16;
@@ -290,7 +300,7 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
 
 // units the ring holds for `n_tile` tokens per tile: as many as fit beside the container pairs (an even number)
 static int group_units(int n_tile, int out_n) {
-  const int avail = 232448 - 128 - (out_n ? 4 * WO_BYTES : 0) - GRP_BAR_BYTES;
+  const int avail = 232448 - 128 - (out_n ? GRP_SIDE_BYTES : 0) - GRP_BAR_BYTES;
   int n = avail / (group_is_bytes(n_tile) + (out_n ? group_os_bytes(n_tile) : 0));
   n &= ~1;
   return n > GRP_MAX_UNITS ? GRP_MAX_UNITS : n;
@@ -300,7 +310,7 @@ cudaError_t launch_linear_group(GroupParams p, bool f32_out, int sm_count, cudaS
 {
   p.nslot = group_units(p.n_tile, p.out_n);
   p.slot_bytes = group_is_bytes(p.n_tile) + (p.out_n ? group_os_bytes(p.n_tile) : 0);
-  const int smem = p.nslot * p.slot_bytes + (p.out_n ? 4 * WO_BYTES : 0) + GRP_BAR_BYTES + 128;
+  const int smem = p.nslot * p.slot_bytes + (p.out_n ? GRP_SIDE_BYTES : 0) + GRP_BAR_BYTES + 128;
   if (!*attr_done) {
     cudaError_t e = cudaFuncSetAttribute(sdq_linear_group_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(sdq_linear_group_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
