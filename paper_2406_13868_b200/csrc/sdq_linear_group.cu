@@ -22,8 +22,8 @@
 //
 // Warps: 0 and 10 bulk-copy producers (inlier / outlier slots, two lanes each), 1 MMA issuer (warp-uniform loop, one
 // elected lane issues; also copies metadata and scales to TMEM), 2..5 epilogue (two alternating accumulators of 32
-// columns: the next item's MMAs never wait for the stores), 6..9 and 11..14 container builders.  Every wait is
-// bounded; a timeout sets the sticky flag.
+// columns: the next item's MMAs never wait for the stores), 6..9, 11..14 and 15..22 container builders (two groups).
+// Every wait is bounded; a timeout sets the sticky flag.
 #include <cuda_bf16.h>
 
 #include "sdq_internal.h"
@@ -33,7 +33,7 @@
 
 namespace sdq {
 
-constexpr int GRP_THREADS = 480;                 // 15 warps
+constexpr int GRP_THREADS = 736;                 // 23 warps
 constexpr int GRP_MAX_UNITS = 8;                 // units the ring may hold
 constexpr uint32_t GRP_TM_ACC = 0;               // two accumulators of 32 columns
 constexpr uint32_t GRP_TM_I = 64;                // 2 x 12: E_in 4 | SFA_in 4 | SFB_in 4
@@ -236,58 +236,67 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
     }
     if (!ok && lane == 0) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
   } else if (p.out_n) {
-    // ---------------- outlier container builders (warps 6..9: first 128-K stage of the unit, 11..14: second): thread r
-    // rebuilds weight row r of its stage from 16 codes + 16 positions: per S-Vector of 8 the code goes to the 2:4 slot of
-    // its group of 4 (two ascending slot indices per 4: (p, 3) with the value first, or (0, 3) with the value second when
-    // p = 3; a group without outlier gets (0, 1) and zeros), the form the packer writes for the many-token kernels.
-    const uint32_t h = warp >= 11 ? 1u : 0u, r = (warp - (h ? 11u : 6u)) * 32 + lane;
+    // ---------------- outlier container builders: two groups of eight warps; group g (warps 6..9 + 11..14, or 15..22)
+    // rebuilds container pair g for the units u = g, g + 2, ...  Inside a group the first four warps take the unit's first
+    // 128-K stage and the other four the second; thread r rebuilds weight row r of its stage from 16 codes + 16 positions:
+    // per S-Vector of 8 the code goes to the 2:4 slot of its group of 4 (two ascending slot indices per 4: (p, 3) with the
+    // value first, or (0, 3) with the value second when p = 3; a group without outlier gets (0, 1) and zeros), the form
+    // the packer writes for the many-token kernels.  Two groups, because a trip is mostly latency (barriers, the
+    // dependent load -> permute -> store chain, the proxy fence): they overlap in time.
+    const uint32_t grp = warp >= 15 ? 1u : 0u;
+    const uint32_t wg = grp ? warp - 15 : (warp >= 11 ? warp - 7 : warp - 6);   // 0..7 inside the group
+    const uint32_t h = wg >> 2, r = (wg & 3) * 32 + lane;
+    const bool poller = wg == 0;
     bool ok = true;
-    uint32_t v = 0, ph = 0, u = 0;
+    uint32_t v = 0, ph = 0, u = 0;               // position of the unit in the ring, lap parity, unit count
+    uint8_t* const cb = cbuf + (size_t)(grp * 2 + h) * WO_BYTES;
+    uint8_t* const arow = cb + (r >> 3) * 256 + (r & 7) * 16;
+    const uint32_t row_off = isb + h * (uint32_t)wc_bytes(1) + r * 16, pos_off = isb + h * (uint32_t)wc_bytes(1) + WC_CODE_BYTES + r * 8;
     for (int item = first; item < p.total_items && ok; item += stride) {
       const int T2 = p.m[group_mat_of(p, item)].T2;
       for (int k2 = 0; k2 < T2; ++k2, ++u) {
-        // Only ONE warp waits on the mbarriers (lane 0: the unit's outlier slot has landed; lane 1: the MMAs of the unit that
-        // last used this container pair -- two units back: ring position v - 2, in the previous lap when v < 2 -- have
-        // completed) and then releases the other seven through a hardware barrier: with eight warps waiting on the same
-        // mbarrier some of them noticed its completion more than a microsecond late.
-        if (warp == 6) {
-          const uint32_t vb = v >= 2 ? v - 2 : v + NU - 2;
-          uint64_t* bar = lane == 0 ? &full_os[v] : &done[vb];
-          const uint32_t par = lane == 0 ? ph : (v >= 2 ? ph : ph ^ 1);
-          const bool need = lane == 0 || (lane == 1 && u >= 2);
-          if (!__all_sync(0xffffffffu, need ? ptx::mbar_wait(bar, par) : true) && lane == 0) *timed_out = 1u;
-        }
-        ptx::named_bar_sync(2, 256);
-        if (*timed_out) { ok = false; break; }
-        const uint8_t* st = sm + (size_t)v * ub + isb + h * (uint32_t)wc_bytes(1);
-        const uint4 codes = *reinterpret_cast<const uint4*>(st + r * 16);
-        const uint2 pos = *reinterpret_cast<const uint2*>(st + WC_CODE_BYTES + r * 8);
-        const uint32_t cw[4] = {codes.x, codes.y, codes.z, codes.w}, pw[2] = {pos.x, pos.y};
-        // position ps (0..7) of the outlier in its S-Vector: it sits in the group of 4 number ps >> 2 at p = ps & 3.  Stored
-        // bytes of the S-Vector (two per group of 4): the code moves to byte (p == 3) + 2 (ps >> 2); metadata byte = the two
-        // groups' slot-index nibbles, (p, 3) or (0, 3) for p = 3 where the outlier is, (0, 1) elsewhere.  Both come from
-        // 8-entry byte tables held in two registers each, and one byte-permute looks up four S-Vectors at a time: the four
-        // position nibbles of a 16-bit piece of the position word are its selector.
-        uint32_t stored[16], meta[4], shw[4];
+        if ((u & 1) == grp) {
+          // Only ONE warp of the group waits on the mbarriers (lane 0: the unit's outlier slot has landed; lane 1: the MMAs of
+          // the unit that last used this container pair -- two units back: ring position v - 2, in the previous lap when
+          // v < 2 -- have completed) and then releases the other seven through a hardware barrier: with eight warps waiting
+          // on the same mbarrier some of them noticed its completion more than a microsecond late.
+          if (poller) {
+            const uint32_t vb = v >= 2 ? v - 2 : v + NU - 2;
+            uint64_t* bar = lane == 0 ? &full_os[v] : &done[vb];
+            const uint32_t par = lane == 0 ? ph : (v >= 2 ? ph : ph ^ 1);
+            const bool need = lane == 0 || (lane == 1 && u >= 2);
+            if (!__all_sync(0xffffffffu, need ? ptx::mbar_wait(bar, par) : true) && lane == 0) *timed_out = 1u;
+          }
+          ptx::named_bar_sync(4 + grp, 256);   // (barrier 3 belongs to the epilogue)
+          if (*timed_out) { ok = false; break; }
+          const uint8_t* st = sm + (size_t)v * ub;
+          const uint4 codes = *reinterpret_cast<const uint4*>(st + row_off);
+          const uint2 pos = *reinterpret_cast<const uint2*>(st + pos_off);
+          const uint32_t cw[4] = {codes.x, codes.y, codes.z, codes.w}, pw[2] = {pos.x, pos.y};
+          // position ps (0..7) of the outlier in its S-Vector: it sits in the group of 4 number ps >> 2 at p = ps & 3.  Stored
+          // bytes of the S-Vector (two per group of 4): the code moves to byte (p == 3) + 2 (ps >> 2); metadata byte = the two
+          // groups' slot-index nibbles, (p, 3) or (0, 3) for p = 3 where the outlier is, (0, 1) elsewhere.  Both come from
+          // 8-entry byte tables held in two registers each, and one byte-permute looks up four S-Vectors at a time: the four
+          // position nibbles of a 16-bit piece of the position word are its selector.
+          uint32_t stored[16], meta[4], shw[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const uint32_t sel = pw[i >> 1] >> (16 * (i & 1));
-          meta[i] = __byte_perm(0x4C4E4D4Cu, 0xC4E4D4C4u, sel);
-          shw[i] = __byte_perm(0x08000000u, 0x18101010u, sel);
-        }
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t sel = pw[i >> 1] >> (16 * (i & 1));
+            meta[i] = __byte_perm(0x4C4E4D4Cu, 0xC4E4D4C4u, sel);
+            shw[i] = __byte_perm(0x08000000u, 0x18101010u, sel);
+          }
 #pragma unroll
-        for (int g = 0; g < 16; ++g)
-          stored[g] = __byte_perm(cw[g >> 2], 0u, 0x4440u + (uint32_t)(g & 3)) << ((shw[g >> 2] >> (8 * (g & 3))) & 0xFFu);
-        uint8_t* cb = cbuf + (size_t)((u & 1) * 2 + h) * WO_BYTES;
-        // row r: bytes 0..31 of its 64 stored bytes belong to K-block 0, 32..63 to K-block 1; 16-byte chunks 128 B apart
-        uint8_t* arow = cb + (r >> 3) * 256 + (r & 7) * 16;
-        *reinterpret_cast<uint4*>(arow) = make_uint4(stored[0], stored[1], stored[2], stored[3]);
-        *reinterpret_cast<uint4*>(arow + 128) = make_uint4(stored[4], stored[5], stored[6], stored[7]);
-        *reinterpret_cast<uint4*>(arow + 4096) = make_uint4(stored[8], stored[9], stored[10], stored[11]);
-        *reinterpret_cast<uint4*>(arow + 4096 + 128) = make_uint4(stored[12], stored[13], stored[14], stored[15]);
-        *reinterpret_cast<uint4*>(cb + A_OUT_BYTES + r * 16) = make_uint4(meta[0], meta[1], meta[2], meta[3]);
-        ptx::fence_proxy_async();                          // generic-proxy writes -> visible to the tensor core's reads
-        ptx::mbar_arrive(&built[u & 1]);
+          for (int g = 0; g < 16; ++g)
+            stored[g] = __byte_perm(cw[g >> 2], 0u, 0x4440u + (uint32_t)(g & 3)) << ((shw[g >> 2] >> (8 * (g & 3))) & 0xFFu);
+          // row r: bytes 0..31 of its 64 stored bytes belong to K-block 0, 32..63 to K-block 1; 16-byte chunks 128 B apart
+          *reinterpret_cast<uint4*>(arow) = make_uint4(stored[0], stored[1], stored[2], stored[3]);
+          *reinterpret_cast<uint4*>(arow + 128) = make_uint4(stored[4], stored[5], stored[6], stored[7]);
+          *reinterpret_cast<uint4*>(arow + 4096) = make_uint4(stored[8], stored[9], stored[10], stored[11]);
+          *reinterpret_cast<uint4*>(arow + 4096 + 128) = make_uint4(stored[12], stored[13], stored[14], stored[15]);
+          *reinterpret_cast<uint4*>(cb + A_OUT_BYTES + r * 16) = make_uint4(meta[0], meta[1], meta[2], meta[3]);
+          ptx::fence_proxy_async();                        // generic-proxy writes -> visible to the tensor core's reads
+          ptx::mbar_arrive(&built[grp]);
+        }
         if (++v == NU) { v = 0; ph ^= 1; }
       }
     }
