@@ -811,7 +811,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   // many tokens without K split: the instantiations with compile-time geometry (five ring slots; four with dense inliers)
   const bool many = p.n_tile == 256 && p.ksplit == 1;
   // ... as CTA pairs on tiles of 256 rows x 256 tokens wherever the shape allows (fewer L2 bytes per output)
-  if (many && pair_kernel_applies(M, P->N, P->K, p.out_n) && !getenv("SDQ_NO_PAIR")) {
+  if (many && pair_kernel_applies(M, P->N, P->K, p.out_n)) {
     const cudaError_t pe = launch_linear_pair(p, f32, sm_count, (cudaStream_t)stream, &dinfo->pair_attr);
     return pe == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
   }
@@ -918,7 +918,7 @@ static sdq_status_t launch_group(int n, const sdq_act_t* const* Xq, const sdq_pa
     items += w->N / TILE_ROWS;
     if (x->M > max_m) max_m = x->M;
   }
-  fused = fused && items * 2 >= dinfo->sm_count && items < (1 << 30) && !getenv("SDQ_NO_GROUP");
+  fused = fused && items * 2 >= dinfo->sm_count && items < (1 << 30);
   if (!fused) {
     for (int i = 0; i < n; ++i) {
       const sdq_status_t st = launch_linear(Xq[i], P[i], Y[i], ldy[i], nullptr, 0, stream, f32);

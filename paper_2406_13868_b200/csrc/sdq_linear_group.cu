@@ -20,9 +20,10 @@
 // has long completed and a tcgen05 instruction ~40 to issue, so every role keeps its trips few and its waits parallel:
 // where a role waits for several barriers, different lanes wait for them at the same time.
 //
-// Warps: 0 and 10 bulk-copy producers (inlier / outlier slots, two lanes each), 1 MMA issuer (warp-uniform loop, one
-// elected lane issues; also copies metadata and scales to TMEM), 2..5 epilogue (two alternating accumulators of 32
-// columns: the next item's MMAs never wait for the stores), 6..9, 11..14 and 15..22 container builders (two groups).
+// Warps: 0 and 10 bulk-copy producers (inlier / outlier slots, two lanes each), 1 and 23 MMA issuers (inlier / outlier
+// product, each into its own accumulator; warp-uniform loops, one elected lane issues; they also copy metadata and scales
+// to TMEM), 2..5 epilogue (adds the two accumulators; accumulator pairs alternate per item, so the next item's MMAs never
+// wait for the stores), 6..9, 11..14 and 15..22 container builders (two groups).
 // Every wait is bounded; a timeout sets the sticky flag.
 #include <cuda_bf16.h>
 
@@ -33,13 +34,13 @@
 
 namespace sdq {
 
-constexpr int GRP_THREADS = 736;                 // 23 warps
+constexpr int GRP_THREADS = 768;                 // 24 warps
 constexpr int GRP_MAX_UNITS = 8;                 // units the ring may hold
-constexpr uint32_t GRP_TM_ACC = 0;               // two accumulators of 32 columns
-constexpr uint32_t GRP_TM_I = 64;                // 2 x 12: E_in 4 | SFA_in 4 | SFB_in 4
-constexpr uint32_t GRP_TM_EO = 88;               // 2 x 4: E_out of the unit's two 128-K stages
-constexpr uint32_t GRP_TM_SO = 96;               // 2 x 8: SFA_out 4 | SFB_out 4 (per item)
-constexpr uint32_t GRP_TMEM_COLS = 128;
+constexpr uint32_t GRP_TM_ACC = 0;               // per item parity 64 columns: O_i at +0, O_o at +32 (32 columns each)
+constexpr uint32_t GRP_TM_I = 128;               // 2 x 12: E_in 4 | SFA_in 4 | SFB_in 4
+constexpr uint32_t GRP_TM_EO = 152;              // 2 x 4: E_out of the unit's two 128-K stages
+constexpr uint32_t GRP_TM_SO = 160;              // 2 x 8: SFA_out 4 | SFB_out 4 (per item)
+constexpr uint32_t GRP_TMEM_COLS = 256;
 constexpr int GRP_BAR_BYTES = (3 * GRP_MAX_UNITS + 2 + 4) * 8 + 8;
 
 // inlier slot: | WI record | 4-bit codes of the tokens | their scale atom |
@@ -80,8 +81,9 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
   if (tid == 0) ptx::griddep_launch_dependents();
   if (tid == 0) {
     *timed_out = 0u;
-    for (uint32_t v = 0; v < NU; ++v) { ptx::mbar_init(&full_is[v], 1); ptx::mbar_init(&full_os[v], 1); ptx::mbar_init(&done[v], 1); }
-    for (int a = 0; a < 2; ++a) { ptx::mbar_init(&built[a], 256); ptx::mbar_init(&acc_full[a], 1); ptx::mbar_init(&acc_empty[a], 4); }
+    const uint32_t issuers = p.out_n ? 2u : 1u;   // MMA-issuing warps: both commit to `done` and `acc_full`
+    for (uint32_t v = 0; v < NU; ++v) { ptx::mbar_init(&full_is[v], 1); ptx::mbar_init(&full_os[v], 1); ptx::mbar_init(&done[v], issuers); }
+    for (int a = 0; a < 2; ++a) { ptx::mbar_init(&built[a], 256); ptx::mbar_init(&acc_full[a], issuers); ptx::mbar_init(&acc_empty[a], 4); }
     ptx::fence_barrier_init();
   }
   if (warp == 1) ptx::tmem_alloc(tmem_slot, GRP_TMEM_COLS);
@@ -99,15 +101,15 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
       ptx::griddep_wait();                       // activations come from an earlier kernel
       bool ok = true;
       int item = first, k2 = (int)lane;          // this lane's position: work item and 256-K unit inside the item
-      int mat = -1, rt = 0;
+      int mat = -1, rt = 0, T2 = 0;
       uint32_t iseq = 0;                         // number of the item in this CTA's sequence
       uint32_t v = lane, wrapped = 0, ph = 0;    // ring position, whether the ring has wrapped, parity of `done` to wait for
       for (;;) {
         for (;;) {                               // advance to the item that holds unit k2
           if (item >= p.total_items) break;
-          if (mat < 0) { mat = group_mat_of(p, item); rt = item - p.m[mat].item0; }
-          if (k2 < p.m[mat].T2) break;
-          k2 -= p.m[mat].T2; item += stride; mat = -1; ++iseq;
+          if (mat < 0) { mat = group_mat_of(p, item); rt = item - p.m[mat].item0; T2 = p.m[mat].T2; }
+          if (k2 < T2) break;
+          k2 -= T2; item += stride; mat = -1; ++iseq;
         }
         if (item >= p.total_items) break;
         const GroupMat& m = p.m[mat];
@@ -138,63 +140,73 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
       }
       if (!ok) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer: warp-uniform loop, one elected lane issues (descriptors and TMEM addresses are
-    // uniform-register operands).  tcgen05.cp and tcgen05.mma of one thread execute in issue order, so metadata and
-    // scales need no barrier of their own; their TMEM buffers alternate.  One trip per unit: lanes 0 / 1 / 2 wait for the
-    // inlier slot / the outlier slot / the container pair at the same time; one commit releases all of the unit.
-    bool ok = true;
-    const uint32_t smb = ptx::smem_u32(sm), cbb = ptx::smem_u32(cbuf);
-    const uint32_t id4[2] = {ptx::idesc_block_scaled(128, (uint32_t)p.n_tile, 1, true, 0, 0), ptx::idesc_block_scaled(128, (uint32_t)p.n_tile, 1, true, 2, 2)};
-    const uint32_t id8 = ptx::idesc_block_scaled(128, (uint32_t)p.n_tile, 0, true, 0, 0);
-    const uint32_t wcb = 2u * (uint32_t)wc_bytes(1);
-    const uint32_t nwait = p.out_n ? 3u : 1u;
-    uint32_t v = 0, ph = 0, u = 0, itc = 0;      // ring position and its parity, unit count, item count
-    for (int item = first; item < p.total_items && ok; item += stride, ++itc) {
-      const int T2 = p.m[group_mat_of(p, item)].T2;
-      const uint32_t ab = itc & 1, acc_col = tmem + GRP_TM_ACC + 32u * ab, so = tmem + GRP_TM_SO + 8u * ab;
-      if (itc >= 2) {    // the epilogue has read this accumulator's previous item
-        ok = __all_sync(0xffffffffu, ptx::mbar_wait(&acc_empty[ab], ((itc >> 1) - 1) & 1));
-        if (!ok) break;
-      }
-      for (int k2 = 0; k2 < T2; ++k2, ++u) {
-        uint64_t* bar = lane == 0 ? &full_is[v] : (lane == 1 ? &full_os[v] : &built[u & 1]);
-        const uint32_t par = lane == 2 ? ((u >> 1) & 1) : ph;
-        ok = __all_sync(0xffffffffu, lane < nwait ? ptx::mbar_wait(bar, par) : true);
-        if (!ok) break;
-        ptx::tc_fence_after();
-        if (ptx::elect_one()) {
-          const uint32_t sb = smb + v * ub, mb = tmem + GRP_TM_I + 12u * (uint32_t)(k2 & 1);
-          ptx::tc_cp_128x128b(mb, ptx::smem_desc(sb + A_IN_BYTES, 0, 128));
-          ptx::tc_cp_32x128b_warpx4(mb + 4, ptx::smem_desc(sb + A_IN_BYTES + E_IN_BYTES, 0, 128));
-          ptx::tc_cp_32x128b_warpx4(mb + 8, ptx::smem_desc(sb + WI_BYTES + xb, 0, 128));
-          ptx::mma_sp_mxf4(acc_col, ptx::smem_desc(sb, 128, 256), ptx::smem_desc(sb + WI_BYTES, 128, 1024), id4[0], mb, mb + 4, mb + 8,
-                           k2 ? 1u : 0u);
-          ptx::mma_sp_mxf4(acc_col, ptx::smem_desc(sb + 4096, 128, 256), ptx::smem_desc(sb + WI_BYTES + 512, 128, 1024), id4[1], mb + 2,
-                           mb + 4, mb + 8, 1u);
-          if (p.out_n) {
-            const uint32_t ob = sb + isb;
-            if (k2 == 0) {
-              const uint32_t sf = cbb + 4 * WO_BYTES + ab * 2 * SF_ATOM_BYTES;
-              ptx::tc_cp_32x128b_warpx4(so, ptx::smem_desc(sf, 0, 128));
-              ptx::tc_cp_32x128b_warpx4(so + 4, ptx::smem_desc(sf + SF_ATOM_BYTES, 0, 128));
-            }
-#pragma unroll
-            for (uint32_t h = 0; h < 2; ++h) {
-              const uint32_t ca = cbb + ((u & 1) * 2 + h) * WO_BYTES, eb = tmem + GRP_TM_EO + 4u * h, xa = ob + wcb + h * xb;
-              ptx::tc_cp_128x128b(eb, ptx::smem_desc(ca + A_OUT_BYTES, 0, 128));
-              ptx::mma_sp_mxf8(acc_col, ptx::smem_desc(ca, 128, 256), ptx::smem_desc(xa, 128, 1024), id8, eb, so, so + 4, 1u);
-              ptx::mma_sp_mxf8(acc_col, ptx::smem_desc(ca + 4096, 128, 256), ptx::smem_desc(xa + 512, 128, 1024), id8, eb + 2, so, so + 4, 1u);
-            }
-          }
-          ptx::tc_commit(&done[v]);
-          if (k2 == T2 - 1) ptx::tc_commit(&acc_full[ab]);
+  } else if (warp == 1 || warp == 23) {
+    // ---------------- MMA issuers: warp 1 the inlier product O_i, warp 23 the outlier product O_o, each into its own
+    // accumulator (the epilogue adds them: O = O_i + O_o) -- a tcgen05 instruction costs its issuing thread ~45 cycles, and
+    // the 13 of a 256-K unit in one thread were the longest serial piece of the kernel.  Warp-uniform loops, one elected
+    // lane issues (descriptors and TMEM addresses are uniform-register operands).  tcgen05.cp and tcgen05.mma of one
+    // thread execute in issue order, so metadata and scales need no barrier of their own; their TMEM buffers alternate.
+    // The unit is released when both warps' commits have arrived.
+    const bool outw = warp == 23;
+    if (!outw || p.out_n) {
+      bool ok = true;
+      const uint32_t smb = ptx::smem_u32(sm), cbb = ptx::smem_u32(cbuf);
+      const uint32_t id4[2] = {ptx::idesc_block_scaled(128, (uint32_t)p.n_tile, 1, true, 0, 0), ptx::idesc_block_scaled(128, (uint32_t)p.n_tile, 1, true, 2, 2)};
+      const uint32_t id8 = ptx::idesc_block_scaled(128, (uint32_t)p.n_tile, 0, true, 0, 0);
+      const uint32_t wcb = 2u * (uint32_t)wc_bytes(1);
+      uint32_t v = 0, ph = 0, u = 0, itc = 0;      // ring position and its parity, unit count, item count
+      for (int item = first; item < p.total_items && ok; item += stride, ++itc) {
+        const int T2 = p.m[group_mat_of(p, item)].T2;
+        const uint32_t ab = itc & 1, acc_col = tmem + GRP_TM_ACC + 64u * ab + (outw ? 32u : 0u), so = tmem + GRP_TM_SO + 8u * ab;
+        if (itc >= 2) {    // the epilogue has read this accumulator pair's previous item
+          ok = __all_sync(0xffffffffu, ptx::mbar_wait(&acc_empty[ab], ((itc >> 1) - 1) & 1));
+          if (!ok) break;
         }
-        __syncwarp();
-        if (++v == NU) { v = 0; ph ^= 1; }
+        for (int k2 = 0; k2 < T2; ++k2, ++u) {
+          if (!outw) {
+            ok = __all_sync(0xffffffffu, ptx::mbar_wait(&full_is[v], ph));
+          } else {   // lane 0: the outlier slot has landed; lane 1: its containers are rebuilt
+            uint64_t* bar = lane == 0 ? &full_os[v] : &built[u & 1];
+            const uint32_t par = lane == 0 ? ph : ((u >> 1) & 1);
+            ok = __all_sync(0xffffffffu, lane < 2 ? ptx::mbar_wait(bar, par) : true);
+          }
+          if (!ok) break;
+          ptx::tc_fence_after();
+          if (ptx::elect_one()) {
+            const uint32_t sb = smb + v * ub;
+            if (!outw) {
+              const uint32_t mb = tmem + GRP_TM_I + 12u * (uint32_t)(k2 & 1);
+              ptx::tc_cp_128x128b(mb, ptx::smem_desc(sb + A_IN_BYTES, 0, 128));
+              ptx::tc_cp_32x128b_warpx4(mb + 4, ptx::smem_desc(sb + A_IN_BYTES + E_IN_BYTES, 0, 128));
+              ptx::tc_cp_32x128b_warpx4(mb + 8, ptx::smem_desc(sb + WI_BYTES + xb, 0, 128));
+              ptx::mma_sp_mxf4(acc_col, ptx::smem_desc(sb, 128, 256), ptx::smem_desc(sb + WI_BYTES, 128, 1024), id4[0], mb, mb + 4, mb + 8,
+                               k2 ? 1u : 0u);
+              ptx::mma_sp_mxf4(acc_col, ptx::smem_desc(sb + 4096, 128, 256), ptx::smem_desc(sb + WI_BYTES + 512, 128, 1024), id4[1], mb + 2,
+                               mb + 4, mb + 8, 1u);
+            } else {
+              const uint32_t ob = sb + isb;
+              if (k2 == 0) {
+                const uint32_t sf = cbb + 4 * WO_BYTES + ab * 2 * SF_ATOM_BYTES;
+                ptx::tc_cp_32x128b_warpx4(so, ptx::smem_desc(sf, 0, 128));
+                ptx::tc_cp_32x128b_warpx4(so + 4, ptx::smem_desc(sf + SF_ATOM_BYTES, 0, 128));
+              }
+#pragma unroll
+              for (uint32_t h = 0; h < 2; ++h) {
+                const uint32_t ca = cbb + ((u & 1) * 2 + h) * WO_BYTES, eb = tmem + GRP_TM_EO + 4u * h, xa = ob + wcb + h * xb;
+                ptx::tc_cp_128x128b(eb, ptx::smem_desc(ca + A_OUT_BYTES, 0, 128));
+                ptx::mma_sp_mxf8(acc_col, ptx::smem_desc(ca, 128, 256), ptx::smem_desc(xa, 128, 1024), id8, eb, so, so + 4, (k2 | h) ? 1u : 0u);
+                ptx::mma_sp_mxf8(acc_col, ptx::smem_desc(ca + 4096, 128, 256), ptx::smem_desc(xa + 512, 128, 1024), id8, eb + 2, so, so + 4, 1u);
+              }
+            }
+            ptx::tc_commit(&done[v]);
+            if (k2 == T2 - 1) ptx::tc_commit(&acc_full[ab]);
+          }
+          __syncwarp();
+          if (++v == NU) { v = 0; ph ^= 1; }
+        }
       }
+      if (!ok && lane == 0) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
     }
-    if (!ok && lane == 0) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
   } else if (warp >= 2 && warp <= 5) {
     // ---------------- epilogue: warp w owns TMEM lanes 32 (w % 4) .. + 31 (weight rows), columns = tokens
     const uint32_t qd = warp & 3;
@@ -214,13 +226,22 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
       ptx::tc_fence_after();
       uint32_t val[32];
       {
+        // O = O_i + O_o: the two partial products of the item, added in fp32
         uint32_t a[16], b[16];
-        const uint32_t tb = tmem + ((qd * 32u) << 16) + GRP_TM_ACC + 32u * ab;
-        ptx::tmem_ld_32x32b_x16(tb, a);
-        if (p.n_tile > 16) ptx::tmem_ld_32x32b_x16(tb + 16, b);
-        ptx::tmem_ld_wait();
+        const uint32_t tb = tmem + ((qd * 32u) << 16) + GRP_TM_ACC + 64u * ab;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) { val[i] = a[i]; val[16 + i] = (p.n_tile > 16) ? b[i] : 0u; }
+        for (uint32_t c = 0; c < 32; c += 16) {
+          if (c < (uint32_t)p.n_tile) {
+            ptx::tmem_ld_32x32b_x16(tb + c, a);
+            if (p.out_n) ptx::tmem_ld_32x32b_x16(tb + 32 + c, b);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) val[c + i] = p.out_n ? __float_as_uint(__uint_as_float(a[i]) + __uint_as_float(b[i])) : a[i];
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) val[c + i] = 0u;
+          }
+        }
       }
       ptx::tc_fence_before();
       __syncwarp();
@@ -235,7 +256,7 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
       }
     }
     if (!ok && lane == 0) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
-  } else if (p.out_n) {
+  } else if (p.out_n && warp >= 6 && warp <= 22) {
     // ---------------- outlier container builders: two groups of eight warps; group g (warps 6..9 + 11..14, or 15..22)
     // rebuilds container pair g for the units u = g, g + 2, ...  Inside a group the first four warps take the unit's first
     // 128-K stage and the other four the second; thread r rebuilds weight row r of its stage from 16 codes + 16 positions:

@@ -21,7 +21,6 @@
 // forwarding thread's view of memory) -> 94 us; warp-uniform issue loops, the copies to TMEM folded into the MMA issuer,
 // one barrier per slot and batches of landed slots -> 78 us; two lanes per producer -> 67 us (2.75 PFLOP/s).
 #include <cuda_bf16.h>
-#include <stdlib.h>
 
 #include "sdq_internal.h"
 #include "sdq_layout.h"
