@@ -14,7 +14,8 @@
  *   host memory.  The library never allocates or frees device memory: every buffer is owned by the
  *   caller and sized with the *_size queries.  All launches go to the caller's stream; nothing
  *   synchronises unless stated.  Every function returns a status code; nothing throws or aborts.
- *   Preconditions: N % 128 == 0, K % 256 == 0, M >= 1, 16-byte aligned pointers, finite weights.
+ *   Preconditions: N % 128 == 0, K % 256 == 0 (the inlier metadata and scale atoms of the sparse 4-bit tensor-core
+ *   kind cover 256 K: a record of the packed layout is one such atom), M >= 1, 16-byte aligned pointers, finite weights.
  */
 #ifndef SDQ_H_
 #define SDQ_H_
@@ -153,7 +154,7 @@ sdq_status_t sdq_decompose(const void* W_bf16, int64_t N, int64_t K, int64_t ldw
                            void* packed_buf, size_t packed_bytes, sdq_packed_t* out, void* stream);
 
 /* The same decomposition with the weight-activation product as the significance metric (Section 5,
- * Stage 1: "a weight value itself is tiny, [but] the corresponding activation is huge"; the
+ * Stage 1, calibration-based metrics: a small weight that meets a large activation matters; the
  * decomposition-stage study finds product-based outlier extraction best): the selections -- which
  * out_n values of an S-Vector are outliers and which inlier pairs / elements survive pruning -- rank
  * by |w[n][k]| * col_weight[k] (one fp32 round-to-nearest multiply, largest first, ties to the lower
@@ -177,10 +178,20 @@ sdq_status_t sdq_channel_norm(const void* X_bf16, int64_t M, int64_t K, int64_t 
 /* Untile a packed weight buffer into the canonical arrays (parity surface). Asynchronous. */
 sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canonical_t* out, void* stream);
 
+/* Packed buffers are self-describing: sdq_decompose writes a 256-byte header (magic, layout version, configuration, N,
+ * K, total bytes, section offsets) in front of the sections, so a buffer can be saved and restored with plain memcpy
+ * (device -> file -> device, or to another process) and turned back into a descriptor without the original weights.
+ *   sdq_packed_attach: `dev` (device, 16-byte aligned) holds `bytes` bytes of a packed buffer.  Reads the header
+ *   (synchronises `stream`), checks magic, version, configuration, shape and that the recorded section offsets are the
+ *   ones this library computes for that configuration and shape, and fills *out.  The buffer stays owned by the caller.
+ *   Errors: INVALID_ARG (null pointer), ALIGNMENT, UNSUPPORTED (not a packed buffer of this layout version),
+ *   SHAPE (header inconsistent with itself), BUFFER_TOO_SMALL (bytes < the size the header records), CUDA. */
+sdq_status_t sdq_packed_attach(const void* dev, size_t bytes, sdq_packed_t* out, void* stream);
+
 /* Size of the quantized-activation buffer for M tokens of K features. */
 sdq_status_t sdq_act_size(int64_t M, int64_t K, const sdq_config_t* cfg, size_t* bytes);
 
-/* "We also quantize activations accordingly" (Section 5, Stage 3; A -> A_o, A_i in Section 5.1):
+/* activation quantization (Section 5, Stage 3; A -> A_o, A_i in Section 5.1):
  * per token and Q-Vector an E8M0 scale and E2M1 codes (A_i); per token a power-of-two scale and
  * E4M3 codes (A_o).  X (device) [M][ldx] bf16; xq_buf (device) >= sdq_act_size bytes; out (host).
  * +-Inf saturates, NaN input is undefined.  Asynchronous on `stream`; for K <= 16384 the one kernel it
@@ -258,18 +269,6 @@ sdq_status_t sdq_linear_group_f32(int n, const sdq_act_t* const* Xq, const sdq_p
  *   sdq_linear_ws with separate workspaces. */
 #define SDQ_STATIC_WS_BYTES (4u << 20)
 sdq_status_t sdq_linear_noalloc(const sdq_act_t* Xq, const sdq_packed_t* P, void* Y_bf16, int64_t ldy, void* stream);
-
-/* Measurement aid (no counterpart in the paper): enqueues a copy-only kernel in which every SM keeps `nslot` bulk
- * copies of `slot_bytes` in flight from its own region of `src` (device, 16-byte aligned; walked cyclically) into
- * shared memory, `iters` copies per SM, nothing consuming them.  *bytes_moved receives the bytes the launch stages
- * in total; the caller times the launch with events.  With a source smaller than L2 this is the ceiling of the
- * L2 -> shared-memory path that bounds the many-token product kernel.
- *   slot_bytes a multiple of 128, >= 1024; nslot 1..16; nslot * slot_bytes <= 220 KB; src_bytes / #SMs >= slot_bytes;
- *   issuers 1..4: threads per SM that issue the copies (the slots are dealt out over them).
- *   Asynchronous on `stream`.  Errors: INVALID_ARG, ALIGNMENT, SHAPE, CUDA; a bounded wait that gives up sets the
- *   sticky device status. */
-sdq_status_t sdq_diag_l2_copy(const void* src, size_t src_bytes, int slot_bytes, int nslot, int issuers, int iters,
-                              size_t* bytes_moved, void* stream);
 
 /* Synchronises `stream` and returns the sticky device-side status (SDQ_OK or SDQ_ERR_TIMEOUT when a
  * bounded wait inside a kernel gave up), clearing it. */

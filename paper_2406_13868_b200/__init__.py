@@ -63,9 +63,9 @@ class _ActCanon(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp")]
 
 
-EXPORTS = ["sdq_packed_size", "sdq_decompose", "sdq_decompose_metric", "sdq_channel_norm", "sdq_packed_export", "sdq_act_size", "sdq_quantize_act", "sdq_act_export",
+EXPORTS = ["sdq_packed_size", "sdq_decompose", "sdq_decompose_metric", "sdq_channel_norm", "sdq_packed_export", "sdq_packed_attach", "sdq_act_size", "sdq_quantize_act", "sdq_act_export",
            "sdq_linear", "sdq_linear_f32", "sdq_workspace_size", "sdq_workspace_init", "sdq_linear_ws", "sdq_linear_f32_ws", "sdq_linear_noalloc",
-           "sdq_linear_group", "sdq_linear_group_f32", "sdq_diag_l2_copy", "sdq_device_status", "sdq_status_string"]
+           "sdq_linear_group", "sdq_linear_group_f32", "sdq_diag_l2_copy", "sdq_diag_wait_timeout", "sdq_device_status", "sdq_status_string"]
 
 _lib = None
 
@@ -85,6 +85,8 @@ def lib() -> ctypes.CDLL:
         L.sdq_channel_norm.argtypes = [vp, i64, i64, i64, vp, vp]
         L.sdq_diag_l2_copy.argtypes = [vp, sz, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.POINTER(sz), vp]
         L.sdq_packed_export.argtypes = [ctypes.POINTER(_Packed), ctypes.POINTER(_Canon), vp]
+        L.sdq_packed_attach.argtypes = [vp, sz, ctypes.POINTER(_Packed), vp]
+        L.sdq_diag_wait_timeout.argtypes = [ctypes.c_int, vp]
         L.sdq_act_size.argtypes = [i64, i64, ctypes.POINTER(Config), ctypes.POINTER(sz)]
         L.sdq_quantize_act.argtypes = [vp, i64, i64, i64, ctypes.POINTER(Config), vp, sz, ctypes.POINTER(_Act), vp]
         L.sdq_act_export.argtypes = [ctypes.POINTER(_Act), ctypes.POINTER(_ActCanon), vp]
@@ -173,6 +175,22 @@ def sdq_decompose(W: torch.Tensor, cfg: Config | None = None, buf: torch.Tensor 
         _check(lib().sdq_decompose_metric(W.data_ptr(), N, K, W.stride(0), ctypes.byref(cfg), col_weight.data_ptr(), buf.data_ptr(),
                                           buf.numel(), ctypes.byref(d), _stream()), "sdq_decompose_metric")
     return PackedWeight(buf, d, N, K, cfg, algo)
+
+
+def packed_attach(buf: torch.Tensor) -> PackedWeight:
+    """uint8 CUDA tensor holding a packed buffer (e.g. restored from a file) -> PackedWeight, from the buffer's own header."""
+    _need_cuda(buf, "buf")
+    assert buf.dtype == torch.uint8 and buf.is_contiguous()
+    d = _Packed()
+    _check(lib().sdq_packed_attach(buf.data_ptr(), buf.numel(), ctypes.byref(d), _stream()), "sdq_packed_attach")
+    cfg = Config(d.cfg.out_n, d.cfg.in_gran, d.cfg.in_block, d.cfg.scale_rule, d.cfg.out_order)
+    _, algo = packed_size(d.N, d.K, cfg)
+    return PackedWeight(buf, d, d.N, d.K, cfg, algo)
+
+
+def diag_wait_timeout(polls: int = 64) -> None:
+    """Enqueues the failure-detection self-test: a bounded device-side wait that is made to run out (include/sdq_diag.h)."""
+    _check(lib().sdq_diag_wait_timeout(polls, _stream()), "sdq_diag_wait_timeout")
 
 
 def channel_norm(X: torch.Tensor) -> torch.Tensor:

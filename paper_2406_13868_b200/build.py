@@ -8,7 +8,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libsdq_b200.so")
 SOURCES = ["sdq_api.cu", "sdq_pack.cu", "sdq_quant_act.cu", "sdq_linear.cu", "sdq_linear_pair.cu", "sdq_linear_group.cu", "sdq_plain.cu", "sdq_calib.cu", "sdq_diag.cu"]
-HEADERS = ["sdq_internal.h", "sdq_layout.h", "sdq_linear.h", "sdq_plain.h", "sdq_ptx.cuh", "sdq_codec.cuh", os.path.join("..", "..", "include", "sdq.h")]
+HEADERS = ["sdq_internal.h", "sdq_layout.h", "sdq_linear.h", "sdq_plain.h", "sdq_ptx.cuh", "sdq_codec.cuh", os.path.join("..", "..", "include", "sdq.h"), os.path.join("..", "..", "include", "sdq_diag.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
               "-Xcompiler", "-fPIC"]
 

@@ -1,4 +1,5 @@
-// Measurement aid, not part of the method: the rate at which all SMs together can stage bytes from L2 into shared
+// Measurement and self-test aids, not part of the method (declared in include/sdq_diag.h).
+// Copy rate: the rate at which all SMs together can stage bytes from L2 into shared
 // memory with bulk copies.  The many-token GEMM is bound by exactly this path (a 128 x 256 tile pulls 2.09 MB of
 // operands through it), so the benchmark measures its ceiling live beside the kernel.
 //
@@ -6,6 +7,7 @@
 // cyclically, so the source stays L2-resident after a first pass) and re-issues a slot as soon as its copy has landed;
 // nothing consumes the data.  The slots are dealt out over `issuers` threads (one per warp), as the GEMM spreads its
 // copies over three producer threads.  Every wait is bounded.
+#include "../../include/sdq_diag.h"
 #include "sdq_internal.h"
 #include "sdq_ptx.cuh"
 
@@ -52,9 +54,27 @@ l2_copy_kernel(const uint8_t* __restrict__ src, size_t region_bytes, int iters, 
   if (!ok) atomicOr(&flags[FLAG_TIMEOUT], 1u);
 }
 
+// a bounded wait that is made to run out: nothing ever arrives on the barrier
+__global__ void wait_timeout_kernel(uint32_t polls, uint32_t* __restrict__ flags)
+{
+  __shared__ __align__(8) uint64_t bar;
+  ptx::mbar_init(&bar, 1);
+  ptx::fence_barrier_init();
+  if (!ptx::mbar_wait(&bar, 0, polls)) atomicOr(&flags[FLAG_TIMEOUT], 1u);
+}
+
 }  // namespace sdq
 
 using namespace sdq;
+
+extern "C" sdq_status_t sdq_diag_wait_timeout(int polls, void* stream)
+{
+  if (polls < 1 || polls > 4096) return SDQ_ERR_SHAPE;
+  uint32_t* flags = device_flags();
+  if (!flags) return SDQ_ERR_CUDA;
+  wait_timeout_kernel<<<1, 1, 0, (cudaStream_t)stream>>>((uint32_t)polls, flags);
+  return cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
+}
 
 extern "C" sdq_status_t sdq_diag_l2_copy(const void* src, size_t src_bytes, int slot_bytes, int nslot, int issuers, int iters,
                                          size_t* bytes_moved, void* stream)

@@ -92,6 +92,20 @@ __host__ __device__ inline uint32_t b_off(uint32_t tok, uint32_t byte /*0..127*/
 __host__ __device__ inline uint32_t sf_off(uint32_t row, uint32_t s) { return (row & 31) * 16 + (row >> 5) * 4 + s; }
 
 constexpr size_t HEADER_BYTES = 256;
+// What the first HEADER_BYTES of a packed buffer hold (the rest of the 256 bytes is zero): enough to rebuild the host
+// descriptor from the bytes alone.
+constexpr uint64_t BLOB_MAGIC = 0x0030303242514453ull;   // "SDQB200\0", little endian
+constexpr uint32_t BLOB_VERSION = 2;                     // layout version: 2 = compact outlier records tiled per 128 K (WC)
+struct BlobHeader {
+  uint64_t magic;
+  uint32_t version, header_bytes;
+  int32_t cfg[5];          // out_n, in_gran, in_block, scale_rule, out_order
+  uint32_t tiled;          // 1: stage-tiled tensor-core layout, 0: canonical arrays (decompose-only reading)
+  int64_t N, K;
+  uint64_t total;          // bytes of the whole buffer
+  uint64_t off[8];         // the section offsets of sdq_packed_t
+};
+static_assert(sizeof(BlobHeader) <= HEADER_BYTES, "header fits its reservation");
 
 struct PackedOffsets {
   size_t wi, wo, sfa_out, wc, osexp, wtexp, emeta, total;

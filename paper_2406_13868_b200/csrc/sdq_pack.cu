@@ -373,6 +373,17 @@ static bool cfg_unsupported(const sdq_config_t* c) {
          (c->scale_rule == SDQ_SCALE_UE4M3 && !(c->in_gran == SDQ_GRAN_PAIR && c->in_block == 32));
 }
 
+static void fill_header(BlobHeader* h, const sdq_packed_t& d, bool tiled) {
+  h->magic = BLOB_MAGIC;
+  h->version = BLOB_VERSION;
+  h->header_bytes = (uint32_t)HEADER_BYTES;
+  h->cfg[0] = d.cfg.out_n; h->cfg[1] = d.cfg.in_gran; h->cfg[2] = d.cfg.in_block; h->cfg[3] = d.cfg.scale_rule; h->cfg[4] = d.cfg.out_order;
+  h->tiled = tiled ? 1u : 0u;
+  h->N = d.N; h->K = d.K;
+  h->total = d.bytes;
+  for (int i = 0; i < 8; ++i) h->off[i] = d.off[i];
+}
+
 extern "C" sdq_status_t sdq_packed_size(int64_t N, int64_t K, const sdq_config_t* cfg, size_t* bytes, size_t* algorithmic_bytes)
 {
   if (!cfg_ok(cfg)) return SDQ_ERR_INVALID_ARG;
@@ -417,7 +428,6 @@ extern "C" sdq_status_t sdq_decompose_metric(const void* W, int64_t N, int64_t K
   if (cudaGetLastError() != cudaSuccess) return SDQ_ERR_CUDA;
   uint32_t nonfinite = 0;
   if (cudaMemcpyAsync(&nonfinite, flags + FLAG_NONFINITE, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SDQ_ERR_CUDA;
-  if (cudaStreamSynchronize(st) != cudaSuccess) return SDQ_ERR_CUDA;
   out->dev = packed_buf;
   out->bytes = tc ? off.total : poff.total;
   out->N = N;
@@ -431,7 +441,52 @@ extern "C" sdq_status_t sdq_decompose_metric(const void* W, int64_t N, int64_t K
     out->off[0] = poff.in_code; out->off[1] = poff.in_meta; out->off[2] = poff.in_scale;
     out->off[3] = poff.out_code; out->off[4] = poff.out_idx; out->off[5] = poff.osexp;
   }
+  // the self-describing header (read back by sdq_packed_attach); the copy is complete before `hdr` goes out of scope
+  // because the stream is synchronised below
+  alignas(16) unsigned char hdr[HEADER_BYTES] = {0};
+  fill_header(reinterpret_cast<BlobHeader*>(hdr), *out, tc);
+  if (cudaMemcpyAsync(packed_buf, hdr, HEADER_BYTES, cudaMemcpyHostToDevice, st) != cudaSuccess) return SDQ_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return SDQ_ERR_CUDA;
   return nonfinite ? SDQ_ERR_NONFINITE : SDQ_OK;
+}
+
+extern "C" sdq_status_t sdq_packed_attach(const void* dev, size_t bytes, sdq_packed_t* out, void* stream)
+{
+  if (!dev || !out) return SDQ_ERR_INVALID_ARG;
+  if ((uintptr_t)dev & 15) return SDQ_ERR_ALIGNMENT;
+  if (bytes < HEADER_BYTES) return SDQ_ERR_BUFFER_TOO_SMALL;
+  alignas(16) unsigned char raw[HEADER_BYTES];
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(raw, dev, HEADER_BYTES, cudaMemcpyDeviceToHost, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+    return SDQ_ERR_CUDA;
+  const BlobHeader* h = reinterpret_cast<const BlobHeader*>(raw);
+  if (h->magic != BLOB_MAGIC || h->version != BLOB_VERSION || h->header_bytes != HEADER_BYTES) return SDQ_ERR_UNSUPPORTED;
+  sdq_config_t cfg;
+  cfg.out_n = h->cfg[0]; cfg.in_gran = h->cfg[1]; cfg.in_block = h->cfg[2]; cfg.scale_rule = h->cfg[3]; cfg.out_order = h->cfg[4];
+  if (!cfg_ok(&cfg) || cfg_unsupported(&cfg)) return SDQ_ERR_SHAPE;
+  if (h->N <= 0 || h->K <= 0 || h->N % TILE_ROWS || h->K % K2) return SDQ_ERR_SHAPE;
+  // the sections must sit where this library puts them for that configuration and shape
+  const bool tc = is_tensor_core_reading(cfg);
+  if ((h->tiled != 0) != tc) return SDQ_ERR_SHAPE;
+  sdq_packed_t d;
+  d.dev = const_cast<void*>(dev);
+  d.N = h->N; d.K = h->K; d.cfg = cfg;
+  for (int i = 0; i < 8; ++i) d.off[i] = 0;
+  if (tc) {
+    const PackedOffsets off = tiled_offsets(h->N, h->K, cfg);
+    d.bytes = off.total;
+    d.off[0] = off.wi; d.off[1] = off.wo; d.off[2] = off.sfa_out; d.off[3] = off.wc; d.off[5] = off.osexp; d.off[6] = off.wtexp;
+  } else {
+    const PlainPackedOffsets poff = plain_packed_offsets(h->N, h->K, cfg);
+    d.bytes = poff.total;
+    d.off[0] = poff.in_code; d.off[1] = poff.in_meta; d.off[2] = poff.in_scale; d.off[3] = poff.out_code; d.off[4] = poff.out_idx; d.off[5] = poff.osexp;
+  }
+  if (h->total != d.bytes) return SDQ_ERR_SHAPE;
+  for (int i = 0; i < 8; ++i)
+    if (h->off[i] != d.off[i]) return SDQ_ERR_SHAPE;
+  if (bytes < d.bytes) return SDQ_ERR_BUFFER_TOO_SMALL;
+  *out = d;
+  return SDQ_OK;
 }
 
 extern "C" sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canonical_t* out, void* stream)

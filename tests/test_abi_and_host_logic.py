@@ -20,9 +20,13 @@ def m():
 
 
 def declared_symbols():
-    src = open(os.path.join(ROOT, "include", "sdq.h")).read()
-    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
-    return sorted(set(re.findall(r"\b(sdq_[a-z0-9_]+)\s*\(", src)))
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for f in sorted(os.listdir(inc)):                    # every header of the boundary: sdq.h and sdq_diag.h
+        if f.endswith(".h"):
+            src = re.sub(r"/\*.*?\*/", "", open(os.path.join(inc, f)).read(), flags=re.S)
+            names |= set(re.findall(r"\b(sdq_[a-z0-9_]+)\s*\(", src))
+    return sorted(names)
 
 
 def test_library_exports_every_declared_symbol(m):
@@ -93,3 +97,14 @@ def test_weak_scaling_aggregation_two_ranks_gloo(tmp_path):
     for p, o in zip(procs, outs):
         assert p.returncode == 0, o
         assert "ok" in o
+
+
+def test_attach_group_and_selftest_argument_errors_without_a_gpu(m):
+    L = m.lib()
+    d = m._Packed()
+    assert L.sdq_packed_attach(None, 1 << 20, ctypes.byref(d), None) == 1          # null buffer
+    assert L.sdq_packed_attach(ctypes.c_void_p(0x1008), 1 << 20, ctypes.byref(d), None) == 3   # not 16-byte aligned
+    assert L.sdq_packed_attach(ctypes.c_void_p(0x1000), 100, ctypes.byref(d), None) == 5       # smaller than a header
+    assert L.sdq_linear_group(0, None, None, None, None, None) == 1
+    assert L.sdq_linear_group(2, None, None, None, None, None) == 1
+    assert L.sdq_diag_wait_timeout(0, None) == 2 and L.sdq_diag_wait_timeout(5000, None) == 2  # polls outside 1 .. 4096

@@ -224,3 +224,68 @@ def test_rows_and_tokens_of_subnormal_magnitude():
     assert m.device_status() == 0
     d, tol = y_close(y, so.linear(oq, op))
     assert (d <= tol).all()
+
+
+# ---------------------------------------------------------------------------------------------- saved and restored buffers
+@pytest.mark.parametrize("cfg_args,M", [((1, so.GRAN_PAIR, 64, 0), 5), ((2, so.GRAN_PAIR, 32, 1), 200), ((1, so.GRAN_DENSE, 32, 0), 33),
+                                        ((1, so.GRAN_PAIR, 32, 2), 16), ((1, so.GRAN_ELEM, 64, 0), 0)])
+def test_packed_buffer_survives_a_plain_copy_and_attach(cfg_args, M):
+    """device -> host bytes -> another device buffer -> sdq_packed_attach: the descriptor is rebuilt from the buffer's own
+    header and sdq_linear gives the original result bit for bit."""
+    m = sdq()
+    cfg = m.Config(*cfg_args)
+    N, K = 256, 1024
+    p = m.sdq_decompose(sdq_synth.make_weight(N, K, 4800).cuda(), cfg)
+    saved = p.buf.cpu().numpy().tobytes()                      # what a file would hold
+    pad = torch.zeros(len(saved) + 4096, dtype=torch.uint8, device="cuda")
+    restored = pad[:len(saved)]
+    restored.copy_(torch.frombuffer(bytearray(saved), dtype=torch.uint8))
+    q = m.packed_attach(restored)
+    assert (q.N, q.K) == (N, K)
+    assert [q.cfg.out_n, q.cfg.in_gran, q.cfg.in_block, q.cfg.scale_rule, q.cfg.out_order] == \
+           [cfg.out_n, cfg.in_gran, cfg.in_block, cfg.scale_rule, cfg.out_order]
+    assert list(q.desc.off) == list(p.desc.off) and q.desc.bytes == p.desc.bytes
+    a, b = m.packed_export(p), m.packed_export(q)
+    assert all(torch.equal(a[k], b[k]) for k in a)
+    if M:
+        xq = m.sdq_quantize_act(sdq_synth.make_act(M, K, 4801).cuda(), cfg)
+        assert torch.equal(m.sdq_linear(xq, q), m.sdq_linear(xq, p))
+    assert m.device_status() == 0
+
+
+def test_attach_refuses_what_is_not_a_packed_buffer():
+    m = sdq()
+    cfg = m.Config()
+    p = m.sdq_decompose(sdq_synth.make_weight(128, 256, 4810).cuda(), cfg)
+    junk = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    with pytest.raises(m.SdqError) as e:
+        m.packed_attach(junk)
+    assert e.value.code == 4                                   # no magic: SDQ_ERR_UNSUPPORTED
+    cut = p.buf[:p.buf.numel() // 2].clone()
+    with pytest.raises(m.SdqError) as e:
+        m.packed_attach(cut)
+    assert e.value.code == 5                                   # shorter than its header says
+    bad = p.buf.clone()
+    bad[16] = 7                                                # out_n = 7 in the header's configuration (byte 16)
+    with pytest.raises(m.SdqError) as e:
+        m.packed_attach(bad)
+    assert e.value.code == 2
+
+
+def test_a_bounded_wait_that_runs_out_sets_the_sticky_status_and_the_context_stays_usable():
+    """Failure detection without a fault: a kernel waits, for 64 polls, on a barrier nothing completes; it returns, the
+    sticky status word reports the timeout once, and the next call runs normally."""
+    m = sdq()
+    assert m.device_status() == 0
+    m.diag_wait_timeout(64)
+    assert m.device_status() == 8                              # SDQ_ERR_TIMEOUT
+    assert m.device_status() == 0                              # reading cleared it
+    cfg = m.Config()
+    p = m.sdq_decompose(sdq_synth.make_weight(128, 256, 4820).cuda(), cfg)
+    xq = m.sdq_quantize_act(sdq_synth.make_act(3, 256, 4821).cuda(), cfg)
+    y = m.sdq_linear(xq, p, f32=True).cpu().numpy()
+    assert m.device_status() == 0
+    oc = ocfg(1)
+    d, tol = y_close(y, so.linear(so.quantize_act(sdq_synth.bf16_bits(sdq_synth.make_act(3, 256, 4821)), oc),
+                                  so.decompose(sdq_synth.bf16_bits(sdq_synth.make_weight(128, 256, 4820)), oc)))
+    assert (d <= tol).all()

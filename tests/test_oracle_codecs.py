@@ -136,3 +136,27 @@ def test_scale_of_zero_block():
     assert L.sdqo_e8m0_scale_code(0.0, so.SCALE_OCP_FLOOR) == 0
     assert L.sdqo_e8m0_scale_code(0.0, so.SCALE_CEIL_NOSAT) == 0
     assert L.sdqo_fp8_scale_exp(0.0) == 0
+
+
+def test_scale_exponents_clamp_to_the_e8m0_range():
+    """E8M0 holds exponents -127 .. 127 (codes 0 .. 254; 255 is NaN and never produced), and the power-of-two scale of the
+    8-bit operands is carried as such a code too.  Stated from that definition: whatever the rule asks for is clamped to
+    the nearest representable exponent.  bf16 subnormal blocks (largest magnitude below 2^-126) reach the lower clamp."""
+    # 4-bit Q-Vector scale: the floor rule wants floor(log2 a) - 2
+    assert L.sdqo_e8m0_scale_code(2.0 ** -125, so.SCALE_OCP_FLOOR) == 0          # -127: the last unclamped exponent
+    assert L.sdqo_e8m0_scale_code(2.0 ** -126, so.SCALE_OCP_FLOOR) == 0          # -128 -> clamped to -127
+    assert L.sdqo_e8m0_scale_code(127 * 2.0 ** -133, so.SCALE_OCP_FLOOR) == 0    # the largest bf16 subnormal
+    assert L.sdqo_e8m0_scale_code(2.0 ** -133, so.SCALE_OCP_FLOOR) == 0          # the smallest
+    assert L.sdqo_e8m0_scale_code(2.0 ** -124, so.SCALE_OCP_FLOOR) == 1
+    assert L.sdqo_e8m0_scale_code(6.0 * 2.0 ** -127, so.SCALE_CEIL_NOSAT) == 0
+    assert L.sdqo_e8m0_scale_code(6.0 * 2.0 ** -140, so.SCALE_CEIL_NOSAT) == 0   # far below: still code 0
+    big = float(np.float32(2.0) ** 127 * np.float32(1.9921875))                   # the largest finite bf16
+    assert L.sdqo_e8m0_scale_code(big, so.SCALE_OCP_FLOOR) == 125 + 127          # floor(log2) - 2 = 125: inside the range
+    assert L.sdqo_e8m0_scale_code(big, so.SCALE_CEIL_NOSAT) == 126 + 127         # 6 * 2^126 >= big > 6 * 2^125
+    # 8-bit operands: smallest e with a <= 448 * 2^e
+    assert L.sdqo_fp8_scale_exp(448.0 * 2.0 ** -127) == -127                     # exactly representable at the bound
+    assert L.sdqo_fp8_scale_exp(447.0 * 2.0 ** -127) == -127
+    assert L.sdqo_fp8_scale_exp(448.0 * 2.0 ** -128) == -127                     # would be -128: clamped
+    assert L.sdqo_fp8_scale_exp(2.0 ** -133) == -127
+    assert L.sdqo_fp8_scale_exp(big) == 120                                      # 448 * 2^119 = 1.75 * 2^127 < big <= 448 * 2^120
+    assert L.sdqo_fp8_scale_exp(1e300) == 127                                    # beyond every bf16: the upper clamp

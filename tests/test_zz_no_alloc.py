@@ -41,6 +41,12 @@ def test_noalloc_matches_workspace_variant_twice_in_a_row(M, N, K):
     assert torch.equal(out2, ref)
     d = (out1.float() - ref.float()).abs()
     assert (d <= 1e-3 * (ref.float().abs() + 1e-2)).all()
+    # and against the CPU oracle itself: the bf16 output lies within one bf16 rounding of the oracle's value
+    from oracle import sdq_oracle as so
+    oc = so.Config(1, so.GRAN_PAIR, 64, so.SCALE_OCP_FLOOR)
+    yref = so.linear(so.quantize_act(sdq_synth.bf16_bits(X.cpu()), oc), so.decompose(sdq_synth.bf16_bits(W.cpu()), oc))
+    err = np.abs(out2.float().cpu().numpy().astype(np.float64) - yref)
+    assert (err <= 2.0 ** -8 * np.abs(yref) + 1e-3 * (np.abs(yref) + 1e-2)).all()
 
 
 def test_noalloc_refuses_shapes_beyond_its_fixed_scratch_and_runs_shapes_without_scratch():
