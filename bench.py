@@ -160,6 +160,38 @@ def aggregate_over_ranks(ms_local: float, units_per_rank: float, world: int, dev
 
 
 # ----------------------------------------------------------------------------------------------- CUDA arm
+def spawn_ranks(args) -> int:
+    """`python bench.py --gpus N` without a launcher: start the N ranks (one process per GPU, NCCL rendezvous on the
+    loopback address) through torch.distributed.run and pass their exit code on."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus), "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__), "--gpus", str(args.gpus), "--steps", str(args.steps), "--warmup",
+           str(args.warmup), "--impl", args.impl] + (["--stub-body"] if args.stub_body else [])
+    return subprocess.call(cmd)
+
+
+def run_stub(args):
+    """The rank plumbing of the CUDA arm with the timed body replaced by a fixed duration (CPU, gloo): what the
+    multi-process test drives to check rendezvous, barrier, max-over-ranks and the one JSON line of rank 0."""
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    ms_local = 10.0 * (1 + rank)                       # rank r "took" 10 (r + 1) ms for its batch
+    units_per_s, ms_max = aggregate_over_ranks(ms_local, 100.0 * args.steps, world, "cpu")
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "stub": True, "n_gpus": world, "steps": args.steps, "ms_per_step": ms_max / args.steps,
+                          "value": units_per_s, "scaling": "weak"}))
+
+
 def run_ours(args):
     import paper_2406_13868_b200 as sdq
 
@@ -242,7 +274,7 @@ def run_ours(args):
     # the three projections have the same flop count, so the mean duration of the sampled launches gives the rate
     gemm_tf = (flops_step / 3) / (gemm_ms / gemm_n * 1e-3) / 1e12
     mixed_peak = peaks["bf16"] * MIXED_PEAK_OVER_BF16
-    roofline = {"kernel": "sdq_linear_kernel", "bound": "tensor", "achieved": gemm_tf, "peak": mixed_peak, "unit": "TFLOP/s",
+    roofline = {"kernel": "sdq_linear_pair_kernel", "bound": "tensor", "achieved": gemm_tf, "peak": mixed_peak, "unit": "TFLOP/s",
                 "frac": gemm_tf / mixed_peak,
                 # dram__bytes_read.sum + dram__bytes_write.sum of one captured launch of the gate / up shape
                 # (profiles/sdq_linear_kernel_prefill_M2048_N11008_K4096.md); the down shape was not captured
@@ -281,6 +313,13 @@ def run_ours(args):
     cfgd = sdq.Config(1, sdq.GRAN_DENSE, 32, sdq.SCALE_OCP_FLOOR)
     dns = measure_variant_step(sdq, cfgd, dev, rank, X, H, (Yg, Yu, Yd), flops_step, args.steps,
                                "the same step without pruning: 1:8 FP8 outliers + dense MXFP4 inliers, one scale per 32 K")
+    # ---- the configuration as the benchmark spec words it: element-wise 2:4 inliers, one E8M0 scale per 32 K (stored and run as a
+    # dense 4-bit operand: the sparse FP4 tensor core takes pairs only)
+    cfgl = sdq.Config(1, sdq.GRAN_ELEM, 32, sdq.SCALE_OCP_FLOOR)
+    lit = measure_variant_step(sdq, cfgl, dev, rank, X, H, (Yg, Yu, Yd), flops_step, args.steps,
+                               "the same step with the literal wording: element-wise 2:4 MXFP4 inliers, block 32, 1:8 FP8 outliers")
+    # ---- the headline step repeated for >= 1 s: clocks settle under the power cap; against the sustained bf16 peak
+    sustained = measure_sustained(sdq, step, flops_step, local, peaks)
     # ---- end to end through the public API with host buffers (pinned), copies inside the timed region
     e2e = measure_e2e(sdq, cfg, dev, X, H, (Pg, Pu, Pd), (bx, bh), (Yg, Yu, Yd), flops_step, max(3, args.steps // 2))
     sample = OracleSample(rows_x=1024)
@@ -290,13 +329,23 @@ def run_ours(args):
     cfge = sdq.Config(1, sdq.GRAN_PAIR, 32, sdq.SCALE_UE4M3)
     e4 = measure_variant_step(sdq, cfge, dev, rank, X, H, (Yg, Yu, Yd), flops_step, args.steps,
                               "the same step with E4M3 scale codes per 32 K and power-of-two row / token factors (two-level scaling)")
+    packer = measure_packer(sdq, cfg, dev, peaks)
+    del Pg, Pu, Pd
+    torch.cuda.empty_cache()
+    opt_ffn, keep = measure_opt_ffn(sdq, dev, peaks)
+    del keep
+    torch.cuda.empty_cache()
+    model, keep = measure_model(sdq, dev, peaks)
+    del keep
+    torch.cuda.empty_cache()
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp4+fp8 (E2M1/E4M3 products, fp32 accumulate)",
             "data": "synthetic",
             "config": {"workload": WORKLOAD, "tokens_per_gpu": M_PREFILL, "l2": "packed weights + activations of one step exceed L2 (150 MB > 126 MB)",
                        "parallelism": "dp%d (independent batches, no collective)" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "quantizer_roofline": quant, "scale_block_32": b32, "dense_inliers": dns, "e4m3_scales": e4, "decode": decode,
+            "roofline": roofline, "quantizer_roofline": quant, "sustained": sustained, "scale_block_32": b32, "literal_elem_2of4_block_32": lit, "dense_inliers": dns, "e4m3_scales": e4,
+            "decode": decode, "packer_roofline": packer, "opt67b_ffn_M4096": opt_ffn, "llama7b_224_linears": model,
             "cpu_baseline": {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc, "seconds": dt}}
     print(json.dumps(line))
 
@@ -304,9 +353,10 @@ def run_ours(args):
 def l2_to_sm(sdq, dev, gemm_launch_ms):
     """The ceiling of the L2 -> shared-memory path measured live with the library's copy-only kernel (every SM keeps 128 to
     220 KB of bulk copies in flight from a 37 MB, L2-resident source; best of four copy shapes, each the best of five
-    launches of ~2 GB), and the fraction of it that the GEMM's staged operand bytes reach (1.438 GB per launch: 688 tiles x
-    2.09 MB for the gate / up shape, the same for the down shape; l1tex__m_xbar2l1tex_read_bytes of the ncu capture under
-    profiles/)."""
+    launches of ~2 GB), and the fraction of it that the GEMM's staged operand bytes reach.  Staged bytes per launch of the
+    CTA-pair kernel: per CTA and 256 x 256 tile, 16 inlier stages of 28160 B (weight record + own 128 tokens' codes + two
+    scale atoms) + 32 outlier stages of 26624 B + 1536 B of outlier scale atoms = 1.304 MB; x 2 CTAs x 344 tiles = 0.897 GB
+    for the gate / up shape (0.897 GB for the down shape too: 128 tiles of 43 + 86 stages)."""
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
     src = torch.empty(sms * (256 << 10), dtype=torch.uint8, device=dev).fill_(1)
     best = 0.0
@@ -319,13 +369,17 @@ def l2_to_sm(sdq, dev, gemm_launch_ms):
             torch.cuda.synchronize()
             if rep >= 2:
                 best = max(best, moved / (a.elapsed_time(b) * 1e-3) / 1e12)
-    staged = 1.438e9
+    staged = 0.897e9
     ach = staged / (gemm_launch_ms * 1e-3) / 1e12
     return {"bytes_per_launch": staged, "achieved_TBps": ach, "measured_ceiling_TBps": best, "frac": ach / best,
             "ceiling_basis": "copy-only kernel of this library (sdq_diag_l2_copy), all SMs, best of 3 x 64 KB, 6 x 32 KB, 13 x 16 KB and 15 x 14 KB bulk copies in flight per SM, L2-resident source"}
 
 
 def measure_decode(sdq, cfg, dev, peaks, layers: int = 32, reps: int = 20):
+    """Decode shape (configs[1]): 4096 x 4096, M in {1, 16}, rotating over 32 distinct packed layers (> L2).  Two ways
+    of enqueuing the same 32 independent products, each captured once in a CUDA graph and replayed: ONE
+    sdq_linear_group call (one persistent launch streaming the compact outlier records), and 32 sdq_linear calls
+    (cluster split-K, consecutive launches overlapped by programmatic dependent launch)."""
     N = K = 4096
     packs = []
     for i in range(layers):
@@ -336,38 +390,28 @@ def measure_decode(sdq, cfg, dev, peaks, layers: int = 32, reps: int = 20):
     out = {}
     for M in (1, 16):
         X = sdq_synth.make_act(M, K, 2100 + M, device=str(dev))
-        Y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+        Ys = [torch.empty((M, N), dtype=torch.bfloat16, device=dev) for _ in packs]
         xb = torch.empty(sdq.act_size(M, K, cfg), dtype=torch.uint8, device=dev)
         xq = sdq.sdq_quantize_act(X, cfg, xb)
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side):
-            for _ in range(3):
-                for p in packs:
-                    sdq.sdq_linear(xq, p, Y)
-        torch.cuda.current_stream().wait_stream(side)
-        torch.cuda.synchronize()
-        # the 32 calls of one pass are captured once in a CUDA graph and replayed: the host is out of the loop
-        # (few tokens: cluster split-K, no workspace; consecutive launches overlap by programmatic dependent launch)
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            for p in packs:
-                sdq.sdq_linear(xq, p, Y)
-        g.replay()
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for _ in range(reps):
-            g.replay()
-        b.record()
-        torch.cuda.synchronize()
-        assert sdq.device_status() == 0
-        us = a.elapsed_time(b) * 1e3 / (reps * layers)
-        gbs = algo / (us * 1e-6) / 1e9
-        out["M%d" % M] = {"us_per_layer": us, "weight_GBps_algorithmic": gbs, "frac_of_hbm_peak": gbs / peaks["hbm"]}
-    out["workload"] = ("llama7b_attn_proj_decode 4096x4096, %d distinct layers in rotation (%.0f MB packed > L2), sdq_linear only, "
-                       "one CUDA graph of the %d calls replayed" % (layers, layers * packs[0].buf.numel() / 1e6, layers))
+
+        def grouped():
+            sdq.sdq_linear_group([xq] * layers, packs, Ys)
+
+        def chain():
+            for p, y in zip(packs, Ys):
+                sdq.sdq_linear(xq, p, y)
+        res = {}
+        for name, fn in (("group", grouped), ("chain", chain)):
+            us = time_graph(fn, reps=reps) * 1e3 / layers
+            assert sdq.device_status() == 0
+            gbs = algo / (us * 1e-6) / 1e9
+            res[name] = {"us_per_layer": us, "weight_GBps_algorithmic": gbs, "frac_of_hbm_peak": gbs / peaks["hbm"]}
+        out["M%d" % M] = dict(res["group"], call="sdq_linear_group, 32 layers in one launch",
+                              per_call_chain=dict(res["chain"], call="32 x sdq_linear"))
+    out["workload"] = ("llama7b_attn_proj_decode 4096x4096, %d distinct layers in rotation (%.0f MB packed > L2), products only, "
+                       "one CUDA graph per variant replayed %d times" % (layers, layers * packs[0].buf.numel() / 1e6, reps))
     out["algorithmic_bytes_per_layer"] = algo
+    out["streamed_bytes_per_layer"] = {"group": int(N * K * 4.125 / 8), "chain": int(N * K * 7.625 / 8)}
     out["stored_bytes_per_layer"] = int(packs[0].buf.numel())
     out["hbm_peak_GBps"] = peaks["hbm"]
     return out
@@ -404,6 +448,55 @@ def measure_variant_step(sdq, cfg, dev, rank, X, H, outs, flops_step, steps, wor
     ms = a.elapsed_time(b) / steps
     assert sdq.device_status() == 0
     return {"value": flops_step / (ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms, "workload": workload}
+
+
+def measure_sustained(sdq, step, flops_step, gpu_index, peaks, seconds: float = 1.2):
+    """The benchmark step back to back for at least `seconds`, clocks sampled meanwhile: the number a long-running job
+    sees once the part sits at its power cap, set against the sustained bf16 peak (x 8/3 for the instruction mix)."""
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(); step(); b.record(); torch.cuda.synchronize()
+    n = max(50, int(seconds * 1e3 / a.elapsed_time(b)) + 1)
+    sampler = ClockSampler(gpu_index)
+    sampler.start()
+    time.sleep(0.1)
+    a.record()
+    for _ in range(n):
+        step()
+    b.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = a.elapsed_time(b)
+    tf = flops_step * n / (ms * 1e-3) / 1e12
+    peak = peaks["bf16_sustained"] * MIXED_PEAK_OVER_BF16
+    return {"value": tf, "unit": UNIT, "steps": n, "seconds": ms * 1e-3, "ms_per_step": ms / n, "clocks": clocks,
+            "frac_of_sustained_mixed_peak": tf / peak, "peak": peak,
+            "peak_basis": "%s bf16 sustained %.1f TF/s x 8/3" % (peaks["source"], peaks["bf16_sustained"])}
+
+
+def measure_packer(sdq, cfg, dev, peaks, N: int = D_FF, K: int = D_MODEL, reps: int = 10):
+    """Offline weight packing (pack_kernel) on the gate shape: bytes = the bf16 weights read once + the algorithmic packed
+    bytes written, against the HBM peak.  (sdq_decompose synchronises its stream to read back the non-finite flag, so
+    the launches are timed one by one with events around each call.)"""
+    W = sdq_synth.make_weight(N, K, 9001, device=str(dev))
+    nbytes, algo = sdq.packed_size(N, K, cfg)
+    buf = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    best = 1e9
+    for i in range(reps + 2):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        sdq.sdq_decompose(W, cfg, buf)
+        b.record()
+        torch.cuda.synchronize()
+        if i >= 2:
+            best = min(best, a.elapsed_time(b))
+    moved = N * K * 2 + algo
+    gbs = moved / (best * 1e-3) / 1e9
+    return {"kernel": "pack_kernel", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s", "frac": gbs / peaks["hbm"],
+            "ms": best, "workload": "W %d x %d bf16 -> packed (best of %d calls, includes the call's flag read-back)" % (N, K, reps),
+            "bytes_counted": moved, "bytes_written_all_sections": nbytes}
 
 
 def measure_e2e(sdq, cfg, dev, X, H, packs, bufs, outs, flops_step, steps):
@@ -475,6 +568,23 @@ def run_case(args):
         cfg = sdq.Config(1, sdq.GRAN_DENSE, 32, sdq.SCALE_OCP_FLOOR)
     elif args.case == "gemm_prefill_mxfp4":      # no outliers, no pruning: a plain block-scaled 4-bit GEMM
         cfg = sdq.Config(0, sdq.GRAN_DENSE, 32, sdq.SCALE_OCP_FLOOR)
+    if args.case == "pack":                      # the offline packer alone, on the gate shape
+        W = sdq_synth.make_weight(D_FF, D_MODEL, 1, device=str(dev))
+        for _ in range(args.steps):
+            sdq.sdq_decompose(W, cfg)
+        torch.cuda.synchronize()
+        print(json.dumps({"case": args.case, "N": D_FF, "K": D_MODEL, "launches": args.steps}))
+        return
+    if args.case == "group_decode":              # 16 layers of 4096 x 4096 at 16 tokens in one grouped launch (139 MB > L2)
+        packs = [sdq.sdq_decompose(sdq_synth.make_weight(4096, 4096, 10 + i, device=str(dev)), cfg) for i in range(16)]
+        xq = sdq.sdq_quantize_act(sdq_synth.make_act(16, 4096, 2, device=str(dev)), cfg)
+        Ys = [torch.empty((16, 4096), dtype=torch.bfloat16, device=dev) for _ in packs]
+        for _ in range(args.steps):
+            sdq.sdq_linear_group([xq] * 16, packs, Ys)
+        torch.cuda.synchronize()
+        assert sdq.device_status() == 0
+        print(json.dumps({"case": args.case, "layers": 16, "M": 16, "launches": args.steps}))
+        return
     if args.case.startswith("gemm_prefill"):
         M, K, N = M_PREFILL, D_MODEL, D_FF
     elif args.case == "gemm_decode":
@@ -515,6 +625,90 @@ def time_graph(fn, reps=10):
     return a.elapsed_time(b) / reps
 
 
+def measure_opt_ffn(sdq, dev, peaks):
+    """configs[3]: OPT-6.7B-shaped FFN at prefill, M = 4096: fc1 4096 -> 16384 and fc2 16384 -> 4096 with the outlier pattern
+    swept over 1:8, 2:8 and none (products only, one CUDA graph per GEMM)."""
+    M = 4096
+    X = sdq_synth.make_act(M, 4096, 4001, device=str(dev))
+    H = sdq_synth.make_act(M, 16384, 4002, device=str(dev))
+    W1 = sdq_synth.make_weight(16384, 4096, 4003, device=str(dev))
+    W2 = sdq_synth.make_weight(4096, 16384, 4004, device=str(dev))
+    Y1 = torch.empty((M, 16384), dtype=torch.bfloat16, device=dev)
+    Y2 = torch.empty((M, 4096), dtype=torch.bfloat16, device=dev)
+    fl = 2.0 * M * 4096 * 16384
+    c4 = {"workload": "opt6.7b_ffn_prefill_M4096 (fc1 4096->16384, fc2 16384->4096), products only"}
+    for on, name in ((1, "1:8"), (2, "2:8"), (0, "none")):
+        cfg = sdq.Config(on, sdq.GRAN_PAIR, 64, 0)
+        P1, P2 = sdq.sdq_decompose(W1, cfg), sdq.sdq_decompose(W2, cfg)
+        xq, hq = sdq.sdq_quantize_act(X, cfg), sdq.sdq_quantize_act(H, cfg)
+        t1 = time_graph(lambda: sdq.sdq_linear(xq, P1, Y1))
+        t2 = time_graph(lambda: sdq.sdq_linear(hq, P2, Y2))
+        # roofline of the pattern: sparse FP4 for the inliers (8x the bf16 peak) + sparse FP8 for the outlier part (4x), if any
+        peak = peaks["bf16"] / (1.0 / 8.0 + (1.0 / 4.0 if on else 0.0))
+        c4[name] = {"fc1_ms": t1, "fc1_TFLOPs": fl / t1 / 1e9, "fc2_ms": t2, "fc2_TFLOPs": fl / t2 / 1e9,
+                    "frac_of_tensor_roofline": (fl / t1 / 1e9 + fl / t2 / 1e9) / 2 / peak, "roofline_TFLOPs": peak}
+        del P1, P2, xq, hq
+    return c4, (X, H, W1, W2, Y1, Y2)
+
+
+def measure_model(sdq, dev, peaks, token_counts=(1, 16, 128, 1024, 8192)):
+    """configs[4]: all 224 linear layers of a 32-layer LLaMA-7B-shaped decoder back to back on one stream, as one CUDA
+    graph per token count (activation quantization where a new activation enters + the products).  For M <= 16 also with
+    the independent projections of a layer issued as grouped calls (q, k, v together; gate, up together)."""
+    cfg = sdq.Config(1, sdq.GRAN_PAIR, 64, 0)
+    shapes = [(4096, 4096)] * 4 + [(11008, 4096)] * 2 + [(4096, 11008)]
+    layers = []
+    algo = 0
+    for l in range(32):
+        ps = []
+        for i, (N, K) in enumerate(shapes):
+            W = sdq_synth.make_weight(N, K, 5000 + 10 * l + i, device=str(dev))
+            ps.append(sdq.sdq_decompose(W, cfg))
+            algo += ps[-1].algorithmic_bytes
+            del W
+        layers.append(ps)
+    mixed_peak = peaks["bf16"] * MIXED_PEAK_OVER_BF16
+    c5 = {"workload": "llama7b_32_layers_224_linears (q,k,v,o 4096x4096; gate,up 4096->11008; down 11008->4096), 1%% outlier channels x30",
+          "algorithmic_weight_bytes": algo}
+    for M in token_counts:
+        X = sdq_synth.make_act(M, 4096, 5500 + M, n_outlier_channels=41, device=str(dev))
+        Hh = sdq_synth.make_act(M, 11008, 5600 + M, n_outlier_channels=110, device=str(dev))
+        bx = torch.empty(sdq.act_size(M, 4096, cfg), dtype=torch.uint8, device=dev)
+        bh = torch.empty(sdq.act_size(M, 11008, cfg), dtype=torch.uint8, device=dev)
+        Ya = [torch.empty((M, 4096), dtype=torch.bfloat16, device=dev) for _ in range(3)]
+        Yb = [torch.empty((M, 11008), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+
+        def model(grouped=False):
+            for ps in layers:
+                xq = sdq.sdq_quantize_act(X, cfg, bx)          # input of q, k, v
+                if grouped:
+                    sdq.sdq_linear_group([xq] * 3, ps[0:3], Ya)
+                else:
+                    for j in range(3):
+                        sdq.sdq_linear(xq, ps[j], Ya[j])
+                xq = sdq.sdq_quantize_act(X, cfg, bx)          # input of o
+                sdq.sdq_linear(xq, ps[3], Ya[0])
+                xq = sdq.sdq_quantize_act(X, cfg, bx)          # input of gate, up
+                if grouped:
+                    sdq.sdq_linear_group([xq] * 2, ps[4:6], Yb)
+                else:
+                    sdq.sdq_linear(xq, ps[4], Yb[0])
+                    sdq.sdq_linear(xq, ps[5], Yb[1])
+                hq = sdq.sdq_quantize_act(Hh, cfg, bh)         # input of down
+                sdq.sdq_linear(hq, ps[6], Ya[0])
+        flops = 2.0 * M * sum(n * k for n, k in shapes) * 32
+
+        def entry(ms):
+            return {"ms_per_model_pass": ms, "dense_equiv_TFLOPs": flops / ms / 1e9, "weight_GBps_algorithmic": algo / ms / 1e6,
+                    "frac_of_hbm_peak": algo / ms / 1e6 / peaks["hbm"], "frac_of_mixed_tensor_peak": flops / ms / 1e9 / mixed_peak}
+        e = entry(time_graph(lambda: model(False), reps=3 if M >= 1024 else 10))
+        if M <= 16:
+            e["grouped_qkv_and_gate_up"] = entry(time_graph(lambda: model(True), reps=10))
+        c5["M%d" % M] = e
+        assert sdq.device_status() == 0
+    return c5, layers
+
+
 def run_sweep(args):
     """Extra measurements for the other configurations (not the contract line): the OPT-6.7B FFN with the outlier
     pattern swept, and all 224 linear layers of a 32-layer LLaMA-7B-shaped decoder back to back for a sweep of
@@ -524,24 +718,8 @@ def run_sweep(args):
     torch.cuda.set_device(0)
     peaks = measured_peaks()
     out = {"peaks": peaks}
-    # ---- config 4: OPT-6.7B FFN, M = 4096
+    c4, (X, H, W1, W2, Y1, Y2) = measure_opt_ffn(sdq, dev, peaks)
     M = 4096
-    X = sdq_synth.make_act(M, 4096, 4001, device="cuda")
-    H = sdq_synth.make_act(M, 16384, 4002, device="cuda")
-    W1 = sdq_synth.make_weight(16384, 4096, 4003, device="cuda")
-    W2 = sdq_synth.make_weight(4096, 16384, 4004, device="cuda")
-    Y1 = torch.empty((M, 16384), dtype=torch.bfloat16, device=dev)
-    Y2 = torch.empty((M, 4096), dtype=torch.bfloat16, device=dev)
-    c4 = {}
-    for on, name in ((1, "1:8"), (2, "2:8"), (0, "none")):
-        cfg = sdq.Config(on, sdq.GRAN_PAIR, 64, 0)
-        P1, P2 = sdq.sdq_decompose(W1, cfg), sdq.sdq_decompose(W2, cfg)
-        xq, hq = sdq.sdq_quantize_act(X, cfg), sdq.sdq_quantize_act(H, cfg)
-        t1 = time_graph(lambda: sdq.sdq_linear(xq, P1, Y1))
-        t2 = time_graph(lambda: sdq.sdq_linear(hq, P2, Y2))
-        fl = 2.0 * M * 4096 * 16384
-        c4[name] = {"fc1_ms": t1, "fc1_TFLOPs": fl / t1 / 1e9, "fc2_ms": t2, "fc2_TFLOPs": fl / t2 / 1e9}
-        del P1, P2, xq, hq
     # the same layers with one scale per 32 K (the literal block-32 MXFP4 wording), and without pruning (dense MXFP4
     # inliers, with 1:8 outliers and with none = a plain block-scaled 4-bit GEMM)
     for name, cfg in (("1:8, scale block 32", sdq.Config(1, sdq.GRAN_PAIR, 32, 0)),
@@ -556,44 +734,10 @@ def run_sweep(args):
         del P1, P2, xq, hq
     out["opt67b_ffn_M4096_outlier_sweep"] = c4
     del X, H, W1, W2, Y1, Y2
-    # ---- config 5: 32 layers x (q, k, v, o, gate, up, down)
     cfg = sdq.Config(1, sdq.GRAN_PAIR, 64, 0)
     shapes = [(4096, 4096)] * 4 + [(11008, 4096)] * 2 + [(4096, 11008)]
-    layers = []
-    algo = 0
-    for l in range(32):
-        ps = []
-        for i, (N, K) in enumerate(shapes):
-            W = sdq_synth.make_weight(N, K, 5000 + 10 * l + i, device="cuda")
-            ps.append(sdq.sdq_decompose(W, cfg))
-            algo += ps[-1].algorithmic_bytes
-            del W
-        layers.append(ps)
-    c5 = {"algorithmic_weight_bytes": algo}
-    for M in (1, 16, 128, 1024, 8192):
-        X = sdq_synth.make_act(M, 4096, 5500 + M, n_outlier_channels=41, device="cuda")
-        Hh = sdq_synth.make_act(M, 11008, 5600 + M, n_outlier_channels=110, device="cuda")
-        bx = torch.empty(sdq.act_size(M, 4096, cfg), dtype=torch.uint8, device=dev)
-        bh = torch.empty(sdq.act_size(M, 11008, cfg), dtype=torch.uint8, device=dev)
-        Ya = torch.empty((M, 4096), dtype=torch.bfloat16, device=dev)
-        Yb = torch.empty((M, 11008), dtype=torch.bfloat16, device=dev)
-
-        def model():
-            for ps in layers:
-                xq = sdq.sdq_quantize_act(X, cfg, bx)          # input of q, k, v
-                for j in range(3):
-                    sdq.sdq_linear(xq, ps[j], Ya)
-                xq = sdq.sdq_quantize_act(X, cfg, bx)          # input of o
-                sdq.sdq_linear(xq, ps[3], Ya)
-                xq = sdq.sdq_quantize_act(X, cfg, bx)          # input of gate, up
-                sdq.sdq_linear(xq, ps[4], Yb)
-                sdq.sdq_linear(xq, ps[5], Yb)
-                hq = sdq.sdq_quantize_act(Hh, cfg, bh)         # input of down
-                sdq.sdq_linear(hq, ps[6], Ya)
-        ms = time_graph(model, reps=3 if M >= 1024 else 10)
-        flops = 2.0 * M * sum(n * k for n, k in shapes) * 32
-        c5["M%d" % M] = {"ms_per_model_pass": ms, "dense_equiv_TFLOPs": flops / ms / 1e9, "weight_GBps_algorithmic": algo / ms / 1e6,
-                         "frac_of_hbm_peak": algo / ms / 1e6 / peaks["hbm"], "frac_of_mixed_tensor_peak": flops / ms / 1e9 / (peaks["bf16"] * MIXED_PEAK_OVER_BF16)}
+    c5, layers = measure_model(sdq, dev, peaks)
+    algo = c5["algorithmic_weight_bytes"]
     out["llama7b_32_layers_224_linears"] = c5
     del layers
     # ---- the same model with q, k, v packed as one 12288-row matrix and gate, up as one 22016-row matrix (the usual
@@ -656,18 +800,24 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--sweep", action="store_true", help="measure the other configurations (OPT FFN outlier sweep, whole-model pass) and exit")
-    ap.add_argument("--case", default=None, choices=["gemm_prefill", "gemm_prefill_b32", "gemm_prefill_e4m3", "gemm_prefill_dense", "gemm_prefill_mxfp4", "gemm_decode", "quant"],
+    ap.add_argument("--case", default=None, choices=["gemm_prefill", "gemm_prefill_b32", "gemm_prefill_e4m3", "gemm_prefill_dense", "gemm_prefill_mxfp4", "gemm_decode", "group_decode", "quant",
+                             "pack"],
                     help="run only a small single-kernel case (for profiler captures) and exit")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--stub-body", action="store_true", help="(tests) run only the rank plumbing, on CPU, with a fixed fake duration")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.sweep or args.case):
+        sys.exit(spawn_ranks(args))       # no launcher around us: become one
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.sweep:
         run_sweep(args)
     elif args.case:
         run_case(args)
+    elif args.stub_body:
+        run_stub(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

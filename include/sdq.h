@@ -223,7 +223,9 @@ sdq_status_t sdq_linear_f32(const sdq_act_t* Xq, const sdq_packed_t* P, float* Y
  * split order, so the result does not depend on timing (O = O_o + O_i of Section 5.1 is unchanged; only the
  * summation over K is regrouped, hence Y may differ from sdq_linear in the last fp32 bits).
  *   sdq_workspace_size: bytes needed for (M, N, K) on the current device (0 when no split would be used).
- *   sdq_workspace_init: zeroes a workspace once after allocation (asynchronous); calls leave it zeroed.
+ *   sdq_workspace_init: zeroes a workspace once after allocation (asynchronous); calls leave it zeroed.  A call that
+ *   ended with SDQ_ERR_TIMEOUT (sdq_device_status) or SDQ_ERR_CUDA may leave arrival counters behind: initialise the
+ *   workspace again before it is reused, or the next call adds incomplete partial tiles.
  *   A workspace must not be shared by calls that can overlap on the GPU.  ws may be NULL (no split).
  *   Errors as sdq_linear, plus BUFFER_TOO_SMALL. */
 sdq_status_t sdq_workspace_size(int64_t M, int64_t N, int64_t K, const sdq_config_t* cfg, size_t* bytes);

@@ -152,7 +152,7 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
 // Single pass: the CTAs of a cluster share one group of 8 tokens and split its Q-Vectors; every thread keeps its
 // elements in registers (packed bf16) from the one read of X, the per-token maxima meet through distributed shared
 // memory, and the codes are produced from the registers.  Same arithmetic as the two-kernel path, which stays for
-// rows too long for the register budget (K > 64 * QA_WARPS * QF_MAX_IT * 8 = 16384) and for the block-32 reading.
+// rows too long for the register budget (K > 64 * QA_WARPS * QF_MAX_IT * 8 = 16384); both scale-block sizes run here.
 constexpr int QF_MAX_IT = 4;                             // Q-Vectors per warp
 template <int IT, bool UE>
 __global__ void __launch_bounds__(QA_THREADS, UE ? 3 : 4)

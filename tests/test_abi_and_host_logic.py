@@ -108,3 +108,20 @@ def test_attach_group_and_selftest_argument_errors_without_a_gpu(m):
     assert L.sdq_linear_group(0, None, None, None, None, None) == 1
     assert L.sdq_linear_group(2, None, None, None, None, None) == 1
     assert L.sdq_diag_wait_timeout(0, None) == 2 and L.sdq_diag_wait_timeout(5000, None) == 2  # polls outside 1 .. 4096
+
+
+def test_bench_starts_its_own_ranks_when_run_without_a_launcher():
+    """`python bench.py --gpus 2` with no WORLD_SIZE around it must become two ranks: here with the timed body stubbed
+    (CPU, gloo), through the same spawn path, rendezvous on 127.0.0.1, max-over-ranks timing, one JSON line from rank 0."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "4", "--stub-body"], env=env,
+                       stdout=subprocess.PIPE, stderr=subprocess.PIPE, timeout=300)
+    assert r.returncode == 0, r.stderr.decode()[-2000:]
+    lines = [l for l in r.stdout.decode().splitlines() if l.startswith("{")]
+    assert len(lines) == 1, r.stdout.decode()
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["stub"] is True
+    # rank 1 "took" 20 ms for its 400 units, rank 0 10 ms: the job took the max, and processed both batches
+    assert abs(d["ms_per_step"] - 20.0 / 4) < 1e-9
+    assert abs(d["value"] - 2 * 400.0 / 20e-3) < 1e-6
