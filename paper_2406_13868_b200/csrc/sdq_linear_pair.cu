@@ -66,6 +66,7 @@ sdq_linear_pair_kernel(const LinearParams p)
   uint64_t* acc_full = empty + PAIR_MAX_SLOTS;
   uint64_t* acc_empty = acc_full + 1;                              // leader: all 16 epilogue warps of the pair have drained TMEM
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
+  volatile uint32_t* timed_out = tmem_slot + 1;                    // an epilogue group's wait gave up
 
   const uint32_t rank = ptx::cluster_ctarank();                    // 0 = leader
   const int pair = (int)(blockIdx.x >> 1), n_pairs = (int)(gridDim.x >> 1);
@@ -75,6 +76,7 @@ sdq_linear_pair_kernel(const LinearParams p)
 
   if (tid == 0) ptx::griddep_launch_dependents();
   if (tid == 0) {
+    *timed_out = 0u;
     for (uint32_t s = 0; s < NSLOT; ++s) {
       ptx::mbar_init(&full[s], rank == 0 ? 4 : 3);
       if (!(s & 1)) ptx::mbar_init(&empty[s >> 1], 1);
@@ -299,9 +301,12 @@ sdq_linear_pair_kernel(const LinearParams p)
       const int rt = 2 * (tile % RTP) + (int)rank, mtile = tile / RTP;
       const int64_t m0 = (int64_t)mtile * 256;
       const int n_valid = (int)min((int64_t)256, p.M - m0);
-      ok = ptx::mbar_wait(acc_full, tcount & 1);
+      // one thread per group polls the barrier and releases the other 127 through a hardware barrier: hundreds of threads
+      // polling one mbarrier notice its completion late and slow the CTA's other barrier traffic down
+      if (et == 0 && !ptx::mbar_wait(acc_full, tcount & 1)) *timed_out = 1u;
+      ptx::named_bar_sync(3 + grp, 128);
+      if (*timed_out) { ok = false; break; }
       ptx::tc_fence_after();
-      if (!ok) break;
       const int64_t n0 = (int64_t)rt * TILE_ROWS;
       const int twr = p.tw ? __ldg(p.tw + n0 + q * 32 + lane) : 0;     // two-level scaling: this thread's row factor
       if constexpr (F32_OUT) {
