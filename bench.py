@@ -277,8 +277,8 @@ def run_ours(args):
     roofline = {"kernel": "sdq_linear_pair_kernel", "bound": "tensor", "achieved": gemm_tf, "peak": mixed_peak, "unit": "TFLOP/s",
                 "frac": gemm_tf / mixed_peak,
                 # dram__bytes_read.sum + dram__bytes_write.sum of one captured launch of the gate / up shape
-                # (profiles/sdq_linear_kernel_prefill_M2048_N11008_K4096.md); the down shape was not captured
-                "traffic": 87.7e6, "traffic_unit": "bytes per launch (gate/up shape)",
+                # (profiles/sdq_linear_pair_kernel_prefill_M2048_N11008_K4096.md); the down shape was not captured
+                "traffic": 84.1e6, "traffic_unit": "bytes per launch (gate/up shape)",
                 "peak_basis": "%s bf16 burst %.1f TF/s x 8/3 (sparse FP4 at 8x + sparse FP8 at 4x per dense-equivalent flop)" % (peaks["source"], peaks["bf16"]),
                 "avg_launch_ms": gemm_ms / gemm_n, "launches": gemm_n,
                 # what actually bounds the kernel: bytes staged from L2 into shared memory per launch against the rate that
