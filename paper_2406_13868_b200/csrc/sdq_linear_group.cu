@@ -9,21 +9,25 @@
 // as many row tiles as SMs.
 //
 // The outlier part is streamed in the form the method states it -- an 8-bit code and a position per S-Vector (the WC
-// section, 1.5 bits per weight) -- not as the 2:4 FP8 container of the many-token kernels (5 bits per weight): eight
-// warps rebuild the containers of each 256-K unit in shared memory (one weight row of one 128-K stage per thread, 80
-// bytes written) while the tensor core works on earlier units.  Streamed bytes: 2.625 + 1.5 = 4.125 bits per weight
-// against 4.0 algorithmic.
+// section, 1.5 bits per weight) -- not as the 2:4 FP8 container of the many-token kernels (5 bits per weight): sixteen
+// warps rebuild the containers of each 256-K unit (one weight row of one 128-K stage per thread) and write them with
+// tcgen05.st into tensor memory, from where the outlier MMAs take their A operand and their metadata, while the tensor
+// core works on earlier units.  Shared memory carries every streamed byte once in (bulk copy) and once out (operand
+// read); an earlier version that rebuilt the containers in shared memory moved 86 KB per unit through it, two thirds of
+// its bandwidth at the rate aimed for, and had room for two container pairs only, whose build -> multiply -> release
+// cycle set the pace.  Streamed bytes: 2.625 + 1.5 = 4.125 bits per weight against 4.0 algorithmic.
 //
 // The ring is organised in units of 256 K of one item: an inlier slot (the WI record with the tokens' 4-bit codes and
-// scale atom) and an outlier slot (two compact records with the tokens' 8-bit codes), plus one of two container
-// pairs.  All of a unit is released by ONE tcgen05.commit.  An mbarrier test costs ~150 cycles even when the phase
-// has long completed and a tcgen05 instruction ~40 to issue, so every role keeps its trips few and its waits parallel:
-// where a role waits for several barriers, different lanes wait for them at the same time.
+// scale atom) and an outlier slot (two compact records with the tokens' 8-bit codes); tensor memory holds one container
+// set per ring position.  All of a unit is released by ONE tcgen05.commit per issuer.  An mbarrier test costs 15..50 cycles
+// when the phase has completed, a tcgen05 instruction ~40 to issue, but a hand-over between roles (complete -> noticed)
+// several hundred, so every role keeps its trips few and its waits parallel: where a role waits for several barriers,
+// different lanes wait for them at the same time.
 //
-// Warps: 0 and 10 bulk-copy producers (inlier / outlier slots, two lanes each), 1 and 23 MMA issuers (inlier / outlier
-// product, each into its own accumulator; warp-uniform loops, one elected lane issues; they also copy metadata and scales
-// to TMEM), 2..5 epilogue (adds the two accumulators; accumulator pairs alternate per item, so the next item's MMAs never
-// wait for the stores), 6..9, 11..14 and 15..22 container builders (two groups).
+// Warps: 0 and 10 bulk-copy producers (inlier / outlier slots, six lanes each), 1 and 23 MMA issuers (inlier / outlier
+// product, each into its own accumulator; warp-uniform loops, one elected lane issues; they also copy the inlier metadata
+// and the scales to TMEM), 2..5 epilogue (adds the two accumulators; accumulator pairs alternate per item, so the next
+// item's MMAs never wait for the stores), 6..9, 11..14 and 15..22 container builders (two groups).
 // Every wait is bounded; a timeout sets the sticky flag.
 #include <cuda_bf16.h>
 
@@ -35,20 +39,21 @@
 namespace sdq {
 
 constexpr int GRP_THREADS = 768;                 // 24 warps
-constexpr int GRP_MAX_UNITS = 8;                 // units the ring may hold
+constexpr int GRP_MAX_UNITS = 8;                 // units the ring may hold (and container sets tensor memory holds)
 constexpr uint32_t GRP_TM_ACC = 0;               // per item parity 64 columns: O_i at +0, O_o at +32 (32 columns each)
 constexpr uint32_t GRP_TM_I = 128;               // 2 x 12: E_in 4 | SFA_in 4 | SFB_in 4
-constexpr uint32_t GRP_TM_EO = 152;              // 2 x 4: E_out of the unit's two 128-K stages
-constexpr uint32_t GRP_TM_SO = 160;              // 2 x 8: SFA_out 4 | SFB_out 4 (per item)
-constexpr uint32_t GRP_TMEM_COLS = 256;
-constexpr int GRP_BAR_BYTES = (3 * GRP_MAX_UNITS + 2 + 4) * 8 + 8;
+constexpr uint32_t GRP_TM_SO = 152;              // 2 x 8: SFA_out 4 | SFB_out 4 (per item parity)
+constexpr uint32_t GRP_TM_C = 168;               // per ring position 40: A_out of the unit's two 128-K stages 2 x 16 | E_out 2 x 4
+constexpr uint32_t GRP_TM_C_COLS = 40;
+constexpr uint32_t GRP_TMEM_COLS = 512;
+constexpr int GRP_BAR_BYTES = (4 * GRP_MAX_UNITS + 4 + 2) * 8 + 8;
 
 // inlier slot: | WI record | 4-bit codes of the tokens | their scale atom |
 __host__ __device__ inline int group_is_bytes(int n_tile) { return WI_BYTES + n_tile * 128 + SF_ATOM_BYTES; }
 // outlier slot: | two compact records (128 K each) | 8-bit codes of the tokens, 2 x 128 K |
 __host__ __device__ inline int group_os_bytes(int n_tile) { return 2 * wc_bytes(1) + 2 * n_tile * 128; }
-// beside the ring: two container pairs and, alternating per item, the outlier row / token scale atoms (SFA_out | SFB_out)
-constexpr int GRP_SIDE_BYTES = 4 * WO_BYTES + 2 * 2 * SF_ATOM_BYTES;
+// beside the ring: alternating per item, the outlier row / token scale atoms (SFA_out | SFB_out)
+constexpr int GRP_SIDE_BYTES = 2 * 2 * SF_ATOM_BYTES;
 
 // matrix of work item `item` (items are numbered matrix by matrix)
 __device__ __forceinline__ int group_mat_of(const GroupParams& p, int item) {
@@ -67,23 +72,25 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
   const uint32_t NU = (uint32_t)p.nslot;                                     // units in the ring
   const uint32_t xb = (uint32_t)p.n_tile * 128u, isb = (uint32_t)group_is_bytes(p.n_tile), osb = p.out_n ? (uint32_t)group_os_bytes(p.n_tile) : 0u;
   const uint32_t ub = isb + osb;                                             // bytes of a unit: inlier slot, then outlier slot
-  uint8_t* cbuf = sm + NU * ub;                                              // two container pairs: 2 x (2 x WO_BYTES)
-  uint8_t* sfbuf = cbuf + 4 * WO_BYTES;                                      // 2 x (SFA_out | SFB_out) of the item, alternating
-  uint64_t* full_is = reinterpret_cast<uint64_t*>(cbuf + (p.out_n ? GRP_SIDE_BYTES : 0));   // inlier slot of ring position v has landed
+  uint8_t* sfbuf = sm + NU * ub;                                             // 2 x (SFA_out | SFB_out) of the item, alternating
+  uint64_t* full_is = reinterpret_cast<uint64_t*>(sfbuf + (p.out_n ? GRP_SIDE_BYTES : 0));  // inlier slot of ring position v has landed
   uint64_t* full_os = full_is + GRP_MAX_UNITS;                               // outlier slot of ring position v has landed
   uint64_t* done = full_os + GRP_MAX_UNITS;                                  // the MMAs of the unit at ring position v have completed
-  uint64_t* built = done + GRP_MAX_UNITS;                                    // [2] container pair is rebuilt
-  uint64_t* acc_full = built + 2;                                            // [2]
+  uint64_t* built = done + GRP_MAX_UNITS;                                    // the containers of the unit at ring position v are in tensor memory
+  uint64_t* acc_full = built + GRP_MAX_UNITS;                                // [2]
   uint64_t* acc_empty = acc_full + 2;                                        // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* sf_full = acc_empty + 2;                                         // [2] outlier scale atoms of the item have landed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sf_full + 2);
   volatile uint32_t* timed_out = tmem_slot + 1;                              // a container builder's wait gave up
 
   if (tid == 0) ptx::griddep_launch_dependents();
   if (tid == 0) {
     *timed_out = 0u;
     const uint32_t issuers = p.out_n ? 2u : 1u;   // MMA-issuing warps: both commit to `done` and `acc_full`
-    for (uint32_t v = 0; v < NU; ++v) { ptx::mbar_init(&full_is[v], 1); ptx::mbar_init(&full_os[v], 1); ptx::mbar_init(&done[v], issuers); }
-    for (int a = 0; a < 2; ++a) { ptx::mbar_init(&built[a], 256); ptx::mbar_init(&acc_full[a], issuers); ptx::mbar_init(&acc_empty[a], 4); }
+    for (uint32_t v = 0; v < NU; ++v) {
+      ptx::mbar_init(&full_is[v], 1); ptx::mbar_init(&full_os[v], 1); ptx::mbar_init(&done[v], issuers); ptx::mbar_init(&built[v], 8);
+    }
+    for (int a = 0; a < 2; ++a) { ptx::mbar_init(&acc_full[a], issuers); ptx::mbar_init(&acc_empty[a], 4); ptx::mbar_init(&sf_full[a], 1); }
     ptx::fence_barrier_init();
   }
   if (warp == 1) ptx::tmem_alloc(tmem_slot, GRP_TMEM_COLS);
@@ -94,16 +101,20 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
   const int first = (int)blockIdx.x, stride = (int)gridDim.x;
 
   if (warp == 0 || warp == 10) {
-    // ---------------- producers: warp 0 fills the inlier slots, warp 10 the outlier slots; two lanes each in lockstep, lane l
-    // taking the units u = l, l + 2, ... of this CTA's sequence (NU is even, so a lane's ring positions keep its parity)
+    // ---------------- producers: warp 0 fills the inlier slots, warp 10 the outlier slots.  Six lanes each, in lockstep: lane
+    // 2 c + l issues copy c (of three) of the units u = l, l + 2, ... of this CTA's sequence (NU is even, so a lane's ring
+    // positions keep its parity) -- issuing a bulk copy costs its thread ~100 ns, so one instruction issues a copy for
+    // each of the six lanes instead of one thread issuing six in a row.
     const bool outl = warp == 10;
-    if (lane < 2 && (!outl || p.out_n)) {
+    const uint32_t l = lane & 1, c = lane >> 1;
+    if (c < 3 && (!outl || p.out_n)) {
       ptx::griddep_wait();                       // activations come from an earlier kernel
       bool ok = true;
-      int item = first, k2 = (int)lane;          // this lane's position: work item and 256-K unit inside the item
+      int item = first, k2 = (int)l;             // this lane's position: work item and 256-K unit inside the item
       int mat = -1, rt = 0, T2 = 0;
       uint32_t iseq = 0;                         // number of the item in this CTA's sequence
-      uint32_t v = lane, wrapped = 0, ph = 0;    // ring position, whether the ring has wrapped, parity of `done` to wait for
+      uint32_t v = l, wrapped = 0, ph = 0;       // ring position, whether the ring has wrapped, parity of `done` to wait for
+      const uint32_t wcb = 2u * (uint32_t)wc_bytes(1);
       for (;;) {
         for (;;) {                               // advance to the item that holds unit k2
           if (item >= p.total_items) break;
@@ -117,21 +128,26 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
         uint8_t* st = sm + (size_t)v * ub + (outl ? isb : 0u);
         if (!outl) {
           const uint8_t* xi = m.x + m.xi + (size_t)k2 * XI_BYTES;
-          ptx::mbar_expect_tx(&full_is[v], WI_BYTES + xb + SF_ATOM_BYTES);
-          ptx::bulk_g2s(st, m.w + m.wi + ((size_t)rt * m.T2 + k2) * WI_BYTES, WI_BYTES, &full_is[v]);
-          ptx::bulk_g2s(st + WI_BYTES, xi, xb, &full_is[v]);
-          ptx::bulk_g2s(st + WI_BYTES + xb, xi + B4_BYTES, SF_ATOM_BYTES, &full_is[v]);
+          if (c == 0) ptx::mbar_expect_tx(&full_is[v], WI_BYTES + xb + SF_ATOM_BYTES);
+          const uint8_t* src = c == 0 ? m.w + m.wi + ((size_t)rt * m.T2 + k2) * WI_BYTES : (c == 1 ? xi : xi + B4_BYTES);
+          const uint32_t off = c == 0 ? 0u : (c == 1 ? (uint32_t)WI_BYTES : (uint32_t)WI_BYTES + xb);
+          ptx::bulk_g2s(st + off, src, c == 0 ? (uint32_t)WI_BYTES : (c == 1 ? xb : (uint32_t)SF_ATOM_BYTES), &full_is[v]);
         } else {
-          const uint32_t wcb = 2u * (uint32_t)wc_bytes(1);
           const uint8_t* xo = m.x + m.xo + (size_t)(2 * k2) * XO_BYTES;
-          ptx::mbar_expect_tx(&full_os[v], wcb + 2 * xb + (k2 == 0 ? 2u * SF_ATOM_BYTES : 0u));
-          ptx::bulk_g2s(st, m.w + m.wc + ((size_t)rt * 2 * m.T2 + 2 * k2) * (size_t)wc_bytes(1), wcb, &full_os[v]);
-          ptx::bulk_g2s(st + wcb, xo, xb, &full_os[v]);
-          ptx::bulk_g2s(st + wcb + xb, xo + XO_BYTES, xb, &full_os[v]);
-          if (k2 == 0) {   // the item's outlier scale atoms ride on its first unit's barrier
-            uint8_t* sf = sfbuf + (iseq & 1) * 2 * SF_ATOM_BYTES;
-            ptx::bulk_g2s(sf, m.w + m.sfa_out + (size_t)rt * SF_ATOM_BYTES, SF_ATOM_BYTES, &full_os[v]);
-            ptx::bulk_g2s(sf + SF_ATOM_BYTES, m.x + m.sfb_out, SF_ATOM_BYTES, &full_os[v]);
+          if (c == 0) ptx::mbar_expect_tx(&full_os[v], wcb + 2 * xb);
+          const uint8_t* src = c == 0 ? m.w + m.wc + ((size_t)rt * 2 * m.T2 + 2 * k2) * (size_t)wc_bytes(1) : (c == 1 ? xo : xo + XO_BYTES);
+          ptx::bulk_g2s(st + (c == 0 ? 0u : wcb + (c - 1) * xb), src, c == 0 ? wcb : xb, &full_os[v]);
+          if (k2 == 0 && c >= 1) {
+            // the item's outlier scale atoms (lane c = 1: of the weight rows, c = 2: of the tokens): a buffer and a barrier
+            // of their own per item parity.  The buffer is free once every MMA of the item two back has completed (`acc_full`
+            // of that item: it cannot complete again before these atoms land, since the next item on that accumulator needs
+            // them) -- the ring alone does not say so when an item has fewer units than half the ring.
+            const uint32_t sb = iseq & 1;
+            if (iseq >= 2 && !(ok = ptx::mbar_wait(&acc_full[sb], ((iseq >> 1) - 1) & 1))) break;
+            uint8_t* sf = sfbuf + sb * 2 * SF_ATOM_BYTES;
+            if (c == 1) ptx::mbar_expect_tx(&sf_full[sb], 2u * SF_ATOM_BYTES);
+            ptx::bulk_g2s(sf + (c - 1) * SF_ATOM_BYTES, c == 1 ? m.w + m.sfa_out + (size_t)rt * SF_ATOM_BYTES : m.x + m.sfb_out, SF_ATOM_BYTES,
+                          &sf_full[sb]);
           }
         }
         k2 += 2;
@@ -143,18 +159,19 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
   } else if (warp == 1 || warp == 23) {
     // ---------------- MMA issuers: warp 1 the inlier product O_i, warp 23 the outlier product O_o, each into its own
     // accumulator (the epilogue adds them: O = O_i + O_o) -- a tcgen05 instruction costs its issuing thread ~45 cycles, and
-    // the 13 of a 256-K unit in one thread were the longest serial piece of the kernel.  Warp-uniform loops, one elected
+    // all of a 256-K unit's in one thread were the longest serial piece of the kernel.  Warp-uniform loops, one elected
     // lane issues (descriptors and TMEM addresses are uniform-register operands).  tcgen05.cp and tcgen05.mma of one
-    // thread execute in issue order, so metadata and scales need no barrier of their own; their TMEM buffers alternate.
+    // thread execute in issue order, so the inlier metadata and the scales need no barrier of their own; their TMEM buffers
+    // alternate.  The outlier product takes its A operand and metadata from tensor memory, where the builders put them.
     // The unit is released when both warps' commits have arrived.
     const bool outw = warp == 23;
     if (!outw || p.out_n) {
       bool ok = true;
-      const uint32_t smb = ptx::smem_u32(sm), cbb = ptx::smem_u32(cbuf);
+      const uint32_t smb = ptx::smem_u32(sm);
       const uint32_t id4[2] = {ptx::idesc_block_scaled(128, (uint32_t)p.n_tile, 1, true, 0, 0), ptx::idesc_block_scaled(128, (uint32_t)p.n_tile, 1, true, 2, 2)};
       const uint32_t id8 = ptx::idesc_block_scaled(128, (uint32_t)p.n_tile, 0, true, 0, 0);
       const uint32_t wcb = 2u * (uint32_t)wc_bytes(1);
-      uint32_t v = 0, ph = 0, u = 0, itc = 0;      // ring position and its parity, unit count, item count
+      uint32_t v = 0, ph = 0, itc = 0;             // ring position and its lap parity, item count
       for (int item = first; item < p.total_items && ok; item += stride, ++itc) {
         const int T2 = p.m[group_mat_of(p, item)].T2;
         const uint32_t ab = itc & 1, acc_col = tmem + GRP_TM_ACC + 64u * ab + (outw ? 32u : 0u), so = tmem + GRP_TM_SO + 8u * ab;
@@ -162,13 +179,13 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
           ok = __all_sync(0xffffffffu, ptx::mbar_wait(&acc_empty[ab], ((itc >> 1) - 1) & 1));
           if (!ok) break;
         }
-        for (int k2 = 0; k2 < T2; ++k2, ++u) {
+        for (int k2 = 0; k2 < T2; ++k2) {
           if (!outw) {
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(&full_is[v], ph));
-          } else {   // lane 0: the outlier slot has landed; lane 1: its containers are rebuilt
-            uint64_t* bar = lane == 0 ? &full_os[v] : &built[u & 1];
-            const uint32_t par = lane == 0 ? ph : ((u >> 1) & 1);
-            ok = __all_sync(0xffffffffu, lane < 2 ? ptx::mbar_wait(bar, par) : true);
+          } else {   // lane 0: the unit's containers are in tensor memory; lane 1: its outlier slot has landed; lane 2: the item's scale atoms
+            uint64_t* bar = lane == 0 ? &built[v] : (lane == 1 ? &full_os[v] : &sf_full[ab]);
+            const uint32_t par = lane < 2 ? ph : ((itc >> 1) & 1);
+            ok = __all_sync(0xffffffffu, (lane < 2 || (lane == 2 && k2 == 0)) ? ptx::mbar_wait(bar, par) : true);
           }
           if (!ok) break;
           ptx::tc_fence_after();
@@ -184,18 +201,17 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
               ptx::mma_sp_mxf4(acc_col, ptx::smem_desc(sb + 4096, 128, 256), ptx::smem_desc(sb + WI_BYTES + 512, 128, 1024), id4[1], mb + 2,
                                mb + 4, mb + 8, 1u);
             } else {
-              const uint32_t ob = sb + isb;
               if (k2 == 0) {
-                const uint32_t sf = cbb + 4 * WO_BYTES + ab * 2 * SF_ATOM_BYTES;
+                const uint32_t sf = ptx::smem_u32(sfbuf) + ab * 2 * SF_ATOM_BYTES;
                 ptx::tc_cp_32x128b_warpx4(so, ptx::smem_desc(sf, 0, 128));
                 ptx::tc_cp_32x128b_warpx4(so + 4, ptx::smem_desc(sf + SF_ATOM_BYTES, 0, 128));
               }
 #pragma unroll
               for (uint32_t h = 0; h < 2; ++h) {
-                const uint32_t ca = cbb + ((u & 1) * 2 + h) * WO_BYTES, eb = tmem + GRP_TM_EO + 4u * h, xa = ob + wcb + h * xb;
-                ptx::tc_cp_128x128b(eb, ptx::smem_desc(ca + A_OUT_BYTES, 0, 128));
-                ptx::mma_sp_mxf8(acc_col, ptx::smem_desc(ca, 128, 256), ptx::smem_desc(xa, 128, 1024), id8, eb, so, so + 4, (k2 | h) ? 1u : 0u);
-                ptx::mma_sp_mxf8(acc_col, ptx::smem_desc(ca + 4096, 128, 256), ptx::smem_desc(xa + 512, 128, 1024), id8, eb + 2, so, so + 4, 1u);
+                const uint32_t ca = tmem + GRP_TM_C + GRP_TM_C_COLS * v + 16u * h, eb = tmem + GRP_TM_C + GRP_TM_C_COLS * v + 32u + 4u * h;
+                const uint32_t xa = sb + isb + wcb + h * xb;
+                ptx::mma_sp_mxf8_ta(acc_col, ca, ptx::smem_desc(xa, 128, 1024), id8, eb, so, so + 4, (k2 | h) ? 1u : 0u);
+                ptx::mma_sp_mxf8_ta(acc_col, ca + 8, ptx::smem_desc(xa + 512, 128, 1024), id8, eb + 2, so, so + 4, 1u);
               }
             }
             ptx::tc_commit(&done[v]);
@@ -258,36 +274,31 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
     if (!ok && lane == 0) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
   } else if (p.out_n && warp >= 6 && warp <= 22) {
     // ---------------- outlier container builders: two groups of eight warps; group g (warps 6..9 + 11..14, or 15..22)
-    // rebuilds container pair g for the units u = g, g + 2, ...  Inside a group the first four warps take the unit's first
-    // 128-K stage and the other four the second; thread r rebuilds weight row r of its stage from 16 codes + 16 positions:
+    // rebuilds the containers of the units u = g, g + 2, ... -- straight into tensor memory, where the outlier MMAs read their
+    // A operand and metadata: shared memory is written once (by the bulk copies) and never again.  Inside a group the first
+    // four warps take the unit's first 128-K stage and the other four the second; a warp can reach the 32 TMEM lanes
+    // 32 (warp % 4) .., so its thread `lane` rebuilds weight row 32 (warp % 4) + lane of its stage from 16 codes + 16 positions:
     // per S-Vector of 8 the code goes to the 2:4 slot of its group of 4 (two ascending slot indices per 4: (p, 3) with the
     // value first, or (0, 3) with the value second when p = 3; a group without outlier gets (0, 1) and zeros), the form
-    // the packer writes for the many-token kernels.  Two groups, because a trip is mostly latency (barriers, the
-    // dependent load -> permute -> store chain, the proxy fence): they overlap in time.
+    // the packer writes for the many-token kernels.  A row's 64 stored bytes are 16 columns of its lane, its 16 metadata
+    // bytes 4 columns.  Two groups, because a trip is mostly latency (the barrier, the dependent load -> permute -> store
+    // chain): they overlap in time.  Container set v is free when the unit's outlier slot has landed at ring position v: the
+    // producer refills a position only after the MMAs of its previous unit have completed.
     const uint32_t grp = warp >= 15 ? 1u : 0u;
-    const uint32_t wg = grp ? warp - 15 : (warp >= 11 ? warp - 7 : warp - 6);   // 0..7 inside the group
-    const uint32_t h = wg >> 2, r = (wg & 3) * 32 + lane;
-    const bool poller = wg == 0;
+    const uint32_t h = grp ? (warp >= 19 ? 1u : 0u) : (warp >= 11 ? 1u : 0u);
+    const uint32_t r = (warp & 3) * 32 + lane;
+    const bool poller = grp ? warp == 15 : warp == 6;
     bool ok = true;
     uint32_t v = 0, ph = 0, u = 0;               // position of the unit in the ring, lap parity, unit count
-    uint8_t* const cb = cbuf + (size_t)(grp * 2 + h) * WO_BYTES;
-    uint8_t* const arow = cb + (r >> 3) * 256 + (r & 7) * 16;
     const uint32_t row_off = isb + h * (uint32_t)wc_bytes(1) + r * 16, pos_off = isb + h * (uint32_t)wc_bytes(1) + WC_CODE_BYTES + r * 8;
+    const uint32_t tlane = tmem + (((warp & 3) * 32u) << 16) + GRP_TM_C;
     for (int item = first; item < p.total_items && ok; item += stride) {
       const int T2 = p.m[group_mat_of(p, item)].T2;
       for (int k2 = 0; k2 < T2; ++k2, ++u) {
         if ((u & 1) == grp) {
-          // Only ONE warp of the group waits on the mbarriers (lane 0: the unit's outlier slot has landed; lane 1: the MMAs of
-          // the unit that last used this container pair -- two units back: ring position v - 2, in the previous lap when
-          // v < 2 -- have completed) and then releases the other seven through a hardware barrier: with eight warps waiting
-          // on the same mbarrier some of them noticed its completion more than a microsecond late.
-          if (poller) {
-            const uint32_t vb = v >= 2 ? v - 2 : v + NU - 2;
-            uint64_t* bar = lane == 0 ? &full_os[v] : &done[vb];
-            const uint32_t par = lane == 0 ? ph : (v >= 2 ? ph : ph ^ 1);
-            const bool need = lane == 0 || (lane == 1 && u >= 2);
-            if (!__all_sync(0xffffffffu, need ? ptx::mbar_wait(bar, par) : true) && lane == 0) *timed_out = 1u;
-          }
+          // Only ONE thread of the group waits on the mbarrier and then releases the others through a hardware barrier: with
+          // eight warps waiting on the same mbarrier some of them noticed its completion more than a microsecond late.
+          if (poller && lane == 0 && !ptx::mbar_wait(&full_os[v], ph)) *timed_out = 1u;
           ptx::named_bar_sync(4 + grp, 256);   // (barrier 3 belongs to the epilogue)
           if (*timed_out) { ok = false; break; }
           const uint8_t* st = sm + (size_t)v * ub;
@@ -309,14 +320,14 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
 #pragma unroll
           for (int g = 0; g < 16; ++g)
             stored[g] = __byte_perm(cw[g >> 2], 0u, 0x4440u + (uint32_t)(g & 3)) << ((shw[g >> 2] >> (8 * (g & 3))) & 0xFFu);
-          // row r: bytes 0..31 of its 64 stored bytes belong to K-block 0, 32..63 to K-block 1; 16-byte chunks 128 B apart
-          *reinterpret_cast<uint4*>(arow) = make_uint4(stored[0], stored[1], stored[2], stored[3]);
-          *reinterpret_cast<uint4*>(arow + 128) = make_uint4(stored[4], stored[5], stored[6], stored[7]);
-          *reinterpret_cast<uint4*>(arow + 4096) = make_uint4(stored[8], stored[9], stored[10], stored[11]);
-          *reinterpret_cast<uint4*>(arow + 4096 + 128) = make_uint4(stored[12], stored[13], stored[14], stored[15]);
-          *reinterpret_cast<uint4*>(cb + A_OUT_BYTES + r * 16) = make_uint4(meta[0], meta[1], meta[2], meta[3]);
-          ptx::fence_proxy_async();                        // generic-proxy writes -> visible to the tensor core's reads
-          ptx::mbar_arrive(&built[grp]);
+          // columns 0..7 of the stage: the row's stored bytes of K-block 0 (the first MMA's A), 8..15: of K-block 1
+          const uint32_t tc = tlane + GRP_TM_C_COLS * v;
+          ptx::tmem_st_32x32b_x16(tc + 16u * h, stored);
+          ptx::tmem_st_32x32b_x4(tc + 32u + 4u * h, meta);
+          ptx::tmem_st_wait();
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&built[v]);      // one arrival per warp
         }
         if (++v == NU) { v = 0; ph ^= 1; }
       }
@@ -328,7 +339,7 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
   if (warp == 1) ptx::tmem_dealloc(tmem, GRP_TMEM_COLS);
 }
 
-// units the ring holds for `n_tile` tokens per tile: as many as fit beside the container pairs (an even number)
+// units the ring holds for `n_tile` tokens per tile: as many as fit (an even number)
 static int group_units(int n_tile, int out_n) {
   const int avail = 232448 - 128 - (out_n ? GRP_SIDE_BYTES : 0) - GRP_BAR_BYTES;
   int n = avail / (group_is_bytes(n_tile) + (out_n ? group_os_bytes(n_tile) : 0));
