@@ -179,46 +179,65 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
           ok = __all_sync(0xffffffffu, ptx::mbar_wait(&acc_empty[ab], ((itc >> 1) - 1) & 1));
           if (!ok) break;
         }
-        for (int k2 = 0; k2 < T2; ++k2) {
-          if (!outw) {
-            ok = __all_sync(0xffffffffu, ptx::mbar_wait(&full_is[v], ph));
-          } else {   // lane 0: the unit's containers are in tensor memory; lane 1: its outlier slot has landed; lane 2: the item's scale atoms
-            uint64_t* bar = lane == 0 ? &built[v] : (lane == 1 ? &full_os[v] : &sf_full[ab]);
-            const uint32_t par = lane < 2 ? ph : ((itc >> 1) & 1);
-            ok = __all_sync(0xffffffffu, (lane < 2 || (lane == 2 && k2 == 0)) ? ptx::mbar_wait(bar, par) : true);
+        for (int k2 = 0; k2 < T2 && ok;) {
+          // Up to four units of the item per trip: lane i tests unit k2 + i (for the outlier product: its containers are in
+          // tensor memory, which implies that its slot has landed -- the builders waited for that), lane 4 the item's scale
+          // atoms; the units ready in a row from k2 on are issued together.  A trip costs several hundred cycles beside the
+          // instructions it issues (test, vote, fence, election, reconvergence), so taking what is ready in one trip keeps
+          // the issuer ahead whenever it has fallen behind.  With nothing ready it waits for unit k2 and votes again.
+          const int nb = T2 - k2 < 4 ? T2 - k2 : 4;
+          uint32_t vi = v + lane, phi = ph;
+          if (vi >= NU) { vi -= NU; phi ^= 1; }
+          const bool sf_lane = outw && k2 == 0 && lane == 4;
+          uint64_t* bar = sf_lane ? &sf_full[ab] : (outw ? &built[vi < NU ? vi : 0] : &full_is[vi < NU ? vi : 0]);
+          const uint32_t par = sf_lane ? ((itc >> 1) & 1) : phi;
+          const bool mine = (int)lane < nb || sf_lane;
+          const uint32_t ready = __ballot_sync(0xffffffffu, mine ? ptx::mbar_test(bar, par) : (lane == 4));
+          int n = __ffs((int)~ready) - 1;          // units ready in a row (lane 4 votes yes when it has nothing to test)
+          if (n > nb) n = nb;
+          if (!(ready & 16u)) n = 0;
+          if (n == 0) {
+            ok = __all_sync(0xffffffffu, (lane == 0 || sf_lane) ? ptx::mbar_wait(bar, par) : true);
+            continue;
           }
-          if (!ok) break;
           ptx::tc_fence_after();
           if (ptx::elect_one()) {
-            const uint32_t sb = smb + v * ub;
-            if (!outw) {
-              const uint32_t mb = tmem + GRP_TM_I + 12u * (uint32_t)(k2 & 1);
-              ptx::tc_cp_128x128b(mb, ptx::smem_desc(sb + A_IN_BYTES, 0, 128));
-              ptx::tc_cp_32x128b_warpx4(mb + 4, ptx::smem_desc(sb + A_IN_BYTES + E_IN_BYTES, 0, 128));
-              ptx::tc_cp_32x128b_warpx4(mb + 8, ptx::smem_desc(sb + WI_BYTES + xb, 0, 128));
-              ptx::mma_sp_mxf4(acc_col, ptx::smem_desc(sb, 128, 256), ptx::smem_desc(sb + WI_BYTES, 128, 1024), id4[0], mb, mb + 4, mb + 8,
-                               k2 ? 1u : 0u);
-              ptx::mma_sp_mxf4(acc_col, ptx::smem_desc(sb + 4096, 128, 256), ptx::smem_desc(sb + WI_BYTES + 512, 128, 1024), id4[1], mb + 2,
-                               mb + 4, mb + 8, 1u);
-            } else {
-              if (k2 == 0) {
-                const uint32_t sf = ptx::smem_u32(sfbuf) + ab * 2 * SF_ATOM_BYTES;
-                ptx::tc_cp_32x128b_warpx4(so, ptx::smem_desc(sf, 0, 128));
-                ptx::tc_cp_32x128b_warpx4(so + 4, ptx::smem_desc(sf + SF_ATOM_BYTES, 0, 128));
-              }
+            uint32_t vv = v;
+            for (int i = 0; i < n; ++i) {
+              const int kk = k2 + i;
+              const uint32_t sb = smb + vv * ub;
+              if (!outw) {
+                const uint32_t mb = tmem + GRP_TM_I + 12u * (uint32_t)(kk & 1);
+                ptx::tc_cp_128x128b(mb, ptx::smem_desc(sb + A_IN_BYTES, 0, 128));
+                ptx::tc_cp_32x128b_warpx4(mb + 4, ptx::smem_desc(sb + A_IN_BYTES + E_IN_BYTES, 0, 128));
+                ptx::tc_cp_32x128b_warpx4(mb + 8, ptx::smem_desc(sb + WI_BYTES + xb, 0, 128));
+                ptx::mma_sp_mxf4(acc_col, ptx::smem_desc(sb, 128, 256), ptx::smem_desc(sb + WI_BYTES, 128, 1024), id4[0], mb, mb + 4, mb + 8,
+                                 kk ? 1u : 0u);
+                ptx::mma_sp_mxf4(acc_col, ptx::smem_desc(sb + 4096, 128, 256), ptx::smem_desc(sb + WI_BYTES + 512, 128, 1024), id4[1], mb + 2,
+                                 mb + 4, mb + 8, 1u);
+              } else {
+                if (kk == 0) {
+                  const uint32_t sf = ptx::smem_u32(sfbuf) + ab * 2 * SF_ATOM_BYTES;
+                  ptx::tc_cp_32x128b_warpx4(so, ptx::smem_desc(sf, 0, 128));
+                  ptx::tc_cp_32x128b_warpx4(so + 4, ptx::smem_desc(sf + SF_ATOM_BYTES, 0, 128));
+                }
 #pragma unroll
-              for (uint32_t h = 0; h < 2; ++h) {
-                const uint32_t ca = tmem + GRP_TM_C + GRP_TM_C_COLS * v + 16u * h, eb = tmem + GRP_TM_C + GRP_TM_C_COLS * v + 32u + 4u * h;
-                const uint32_t xa = sb + isb + wcb + h * xb;
-                ptx::mma_sp_mxf8_ta(acc_col, ca, ptx::smem_desc(xa, 128, 1024), id8, eb, so, so + 4, (k2 | h) ? 1u : 0u);
-                ptx::mma_sp_mxf8_ta(acc_col, ca + 8, ptx::smem_desc(xa + 512, 128, 1024), id8, eb + 2, so, so + 4, 1u);
+                for (uint32_t h = 0; h < 2; ++h) {
+                  const uint32_t ca = tmem + GRP_TM_C + GRP_TM_C_COLS * vv + 16u * h, eb = tmem + GRP_TM_C + GRP_TM_C_COLS * vv + 32u + 4u * h;
+                  const uint32_t xa = sb + isb + wcb + h * xb;
+                  ptx::mma_sp_mxf8_ta(acc_col, ca, ptx::smem_desc(xa, 128, 1024), id8, eb, so, so + 4, (kk | (int)h) ? 1u : 0u);
+                  ptx::mma_sp_mxf8_ta(acc_col, ca + 8, ptx::smem_desc(xa + 512, 128, 1024), id8, eb + 2, so, so + 4, 1u);
+                }
               }
+              ptx::tc_commit(&done[vv]);
+              if (kk == T2 - 1) ptx::tc_commit(&acc_full[ab]);
+              if (++vv == NU) vv = 0;
             }
-            ptx::tc_commit(&done[v]);
-            if (k2 == T2 - 1) ptx::tc_commit(&acc_full[ab]);
           }
           __syncwarp();
-          if (++v == NU) { v = 0; ph ^= 1; }
+          k2 += n;
+          v += (uint32_t)n;
+          if (v >= NU) { v -= NU; ph ^= 1; }
         }
       }
       if (!ok && lane == 0) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
