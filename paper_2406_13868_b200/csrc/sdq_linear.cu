@@ -914,7 +914,8 @@ static sdq_status_t launch_group(int n, const sdq_act_t* const* Xq, const sdq_pa
     if (((uintptr_t)Y[i] & 15) || (ldy[i] % 8)) return SDQ_ERR_ALIGNMENT;
     // the grouped kernel carries the primary format: pair-wise 4:8 inliers, one E8M0 scale per 64 K, at most one outlier per S-Vector
     fused = fused && x->M <= 32 && w->cfg.in_gran == SDQ_GRAN_PAIR && w->cfg.in_block == 64 && w->cfg.scale_rule != SDQ_SCALE_UE4M3 &&
-            w->cfg.out_n <= 1 && w->cfg.out_n == P[0]->cfg.out_n;
+            w->cfg.out_n <= 1 && w->cfg.out_n == P[0]->cfg.out_n &&
+            w->K >= 4 * K2;   // an item spans at least half the ring: the kernel's per-item barriers then never run two phases apart
     items += w->N / TILE_ROWS;
     if (x->M > max_m) max_m = x->M;
   }
