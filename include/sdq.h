@@ -241,10 +241,10 @@ sdq_status_t sdq_linear_f32_ws(const sdq_act_t* Xq, const sdq_packed_t* P, float
  * benchmark rotation): they may run in any order and concurrently.
  *   Xq, P, Y, ldy: host arrays of n entries (descriptors and pointers as for sdq_linear; the arrays themselves are read
  *   during the call only).  Outputs must not overlap.
- *   When every layer has at most 32 tokens, the primary format (SDQ_GRAN_PAIR, in_block 64, out_n <= 1, power-of-two
- *   scales), n <= 32 and the layers together have at least half as many 128-row tiles as the GPU has SMs, the call is ONE
- *   persistent kernel launch that streams all weights once, the outlier part in its compact form (8-bit code + position per
- *   S-Vector, rebuilt into the tensor core's 2:4 form in shared memory); the summation order over K of an output differs
+ *   When every layer has at most 32 tokens, K >= 1024, the primary format (SDQ_GRAN_PAIR, in_block 64, out_n <= 1,
+ *   power-of-two scales), n <= 32 and the layers together have at least half as many 128-row tiles as the GPU has SMs, the
+ *   call is ONE persistent kernel launch that streams all weights once, the outlier part in its compact form (8-bit code +
+ *   position per S-Vector, rebuilt into the tensor core's 2:4 form in tensor memory); the summation order over K of an output differs
  *   from sdq_linear's split-K paths, so results agree to fp32 rounding, not bit for bit.  Otherwise the layers are
  *   enqueued one after the other exactly as sdq_linear would.
  *   Asynchronous on `stream`; allocates nothing.  Errors as sdq_linear (the first failing layer's). */

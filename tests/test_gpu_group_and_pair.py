@@ -46,11 +46,12 @@ def _check_against_oracle(m, Ws, Xs, ys32, ys16, cfg_args, rows=None):
     ([(4096, 4096)] * 3, [16] * 3, 1, True),                 # the same sharing one quantized X
     ([(11008, 4096)] * 2, [7] * 2, 1, True),                 # gate / up
     ([(4096, 4096), (11008, 4096), (4096, 11008)], [5, 5, 5], 1, False),   # different N and K in one call
-    ([(2048, 512)] * 10, [3] * 10, 1, False),                # many small layers, two 256-K units each
+    ([(2048, 1024)] * 10, [3] * 10, 1, False),               # many small layers, four 256-K units each: the shortest items of the fused kernel
     ([(4096, 2048)] * 4, [32] * 4, 1, False),                # 32 tokens: the wider token tile
     ([(4096, 2048)] * 4, [17, 20, 32, 1], 1, False),         # token counts differ inside the group
     ([(4096, 4096)] * 3, [16] * 3, 0, False),                # no outlier part
-    ([(1152, 256)] * 10, [2] * 10, 1, False),                # one unit per item: the ring wraps across items at once
+    ([(1152, 1280)] * 10, [2] * 10, 1, False),               # an odd number of units per item: items start on either ring parity
+    ([(1152, 256)] * 10, [2] * 10, 1, False),                # K below the fused kernel's range: enqueued layer by layer
 ])
 def test_group_call_matches_oracle(shapes, Ms, out_n, share_x):
     cfg_args = (out_n, so.GRAN_PAIR, 64, 0)
@@ -102,6 +103,7 @@ def test_group_call_runs_twice_in_a_row_and_inside_a_graph():
     ([(4096, 1024)] * 3, [8] * 3, (1, so.GRAN_PAIR, 32, 0)),      # one scale per 32 K
     ([(4096, 1024)] * 3, [8] * 3, (2, so.GRAN_PAIR, 64, 0)),      # two outliers per S-Vector
     ([(256, 1024)] * 2, [8] * 2, (1, so.GRAN_PAIR, 64, 0)),       # too few row tiles for the persistent kernel
+    ([(4096, 512)] * 3, [8] * 3, (1, so.GRAN_PAIR, 64, 0)),       # items shorter than half the ring
     ([(4096, 1024)] * 3, [8] * 3, (1, so.GRAN_DENSE, 32, 0)),     # dense inliers
 ])
 def test_group_call_outside_the_fused_kernels_range_equals_single_calls(shapes, Ms, cfg_args):
