@@ -22,6 +22,9 @@
  * "definition" of the decomposition, brute-force matmul, one-hot read-back, exact power-of-two
  * scaling, the paper's printed bits-per-weight / throughput arithmetic, and for the E4M3 scale rule closed forms at every
  * representable scale and midpoint plus an independent definition built on torch's float8 cast.
+ * The int8 outlier format is pinned by closed forms (codes of k * amax / 127 are k, the half-way points go to the even
+ * integer, nothing exceeds 127), by numpy's own fp32 division and rint on random rows, and by a product that must equal an
+ * exact integer matrix product times the two scales.
  * Parity unpinned: none of the functions in this file (model-quality numbers of the paper are not
  * computed here at all).
  */
@@ -53,6 +56,11 @@
    nearest to amax_q / (6 * 2^t) (ties to the even code; never below the smallest positive one unless the Q-Vector is
    all zero); an element is the E2M1 value nearest to x / (scale * 2^t), ties to even, saturating at 6. */
 #define SDQO_SCALE_UE4M3 2
+/* 8-bit format of the outlier operands W_o and A_o: E4M3 with a power-of-two scale per weight row / token, or the
+   evaluation's int8 (Section 6 configuration names "1:8int8"; Section 5.1: "quantize 1:8 W_o as int8 ... A would be
+   quantized to int8 A_o"): symmetric, one fp32 scale per weight row / token */
+#define SDQO_OUT_E4M3 0
+#define SDQO_OUT_INT8 1
 
 typedef struct {
   int out_n;      /* outliers kept per S-Vector of 8 along K: 0, 1 or 2          */
@@ -60,6 +68,7 @@ typedef struct {
   int in_block;   /* Q-Vector: logical K per inlier / 4-bit activation scale (32|64) */
   int scale_rule; /* SDQO_SCALE_*                                               */
   int out_order;  /* SDQO_ORDER_*: which end of the metric's order Stage 2 takes     */
+  int out_fmt;    /* SDQO_OUT_*: 8-bit format of W_o and A_o                          */
 } sdqo_config;
 
 /* ------------------------------------------------------------------ number formats */
@@ -154,6 +163,27 @@ int sdqo_fp8_scale_exp(double amax) {
   return e;
 }
 
+/* int8 operands: scale s = amax / 127 (amax = 0: s = 1) and code = the integer nearest to x / s, ties to the even
+ * integer, limited to [-127, 127].  The scale is not a power of two, so x / s rounds; both the scale and the quotient
+ * are formed in fp32 (one IEEE division each, round to nearest even), the precision in which the code is decided.
+ * x is a bf16 value (exact in fp32).  The scale is handed on as its fp32 bit pattern. */
+float sdqo_int8_scale(double amax) { return amax == 0.0 ? 1.0f : (float)amax / 127.0f; }
+int8_t sdqo_int8_encode(double x, float s) {
+  volatile float q = (float)x / s;   /* fp32 quotient (volatile: no wider intermediate) */
+  float r = nearbyintf(q);           /* default rounding mode: to nearest, ties to even */
+  if (r > 127.0f) r = 127.0f;
+  if (r < -127.0f) r = -127.0f;
+  return (int8_t)r;
+}
+static int32_t float_bits(float f) { int32_t u; memcpy(&u, &f, 4); return u; }
+static float bits_float(int32_t u) { float f; memcpy(&f, &u, 4); return f; }
+/* value of an 8-bit operand code under the configuration's format; sexp = the exponent of the power-of-two scale
+ * (E4M3) or the bit pattern of the fp32 scale (int8) */
+static double out_value(const sdqo_config* cfg, uint8_t code, int32_t sexp) {
+  if (cfg->out_fmt == SDQO_OUT_INT8) return (double)(int8_t)code * (double)bits_float(sexp);
+  return ldexp(sdqo_e4m3_decode(code), sexp);
+}
+
 /* unsigned-E4M3 code (0x00..0x7E) of a Q-Vector scale under SDQO_SCALE_UE4M3, and the scaled E2M1 code of an element */
 uint8_t sdqo_ue4m3_scale_code(double amax_q, int t) {
   if (amax_q == 0.0) return 0;
@@ -180,7 +210,8 @@ static int is_finite_bf16(uint16_t h) { return (h & 0x7F80) != 0x7F80; }
  *   in_scale [N][K/in_block] E8M0 code (SDQO_SCALE_UE4M3: unsigned E4M3 code, times 2^in_texp[n])
  *   in_texp  [N]           SDQO_SCALE_UE4M3: exponent t of the row's power-of-two factor (int32); else 0 (may be NULL)
  *   out_code [N][K/8][out_n] E4M3 codes; out_idx same shape, position 0..7 inside the group, ascending
- *   out_sexp [N]           e of the per-row outlier scale 2^e (int32)
+ *   out_sexp [N]           e of the per-row outlier scale 2^e (int32); SDQO_OUT_INT8: out_code holds int8 codes and
+ *                          out_sexp the bit pattern of the row's fp32 scale
  * returns 0, or -1 on a bad argument, -2 if W holds a non-finite value.
  */
 /* Significance of element k of a row for the selections of Stage 2 (which values are outliers) and Stage 1 (which
@@ -205,6 +236,7 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
       if (!(col_weight[k] >= 0.0f) || isinf(col_weight[k])) return -3;
   if (cfg->out_n < 0 || cfg->out_n > 2) return -1;
   if (cfg->out_order != SDQO_ORDER_LARGE && cfg->out_order != SDQO_ORDER_SMALL) return -1;
+  if (cfg->out_fmt != SDQO_OUT_E4M3 && cfg->out_fmt != SDQO_OUT_INT8) return -1;
   if (cfg->in_block != 32 && cfg->in_block != 64) return -1;
   if (cfg->scale_rule < 0 || cfg->scale_rule > SDQO_SCALE_UE4M3 || (cfg->scale_rule == SDQO_SCALE_UE4M3 && !in_texp)) return -1;
   if (cfg->in_gran < 0 || cfg->in_gran > SDQO_GRAN_3OF4) return -1;
@@ -255,14 +287,24 @@ int sdqo_decompose_metric(const uint16_t* W, int64_t N, int64_t K, const sdqo_co
         if (a > out_amax) out_amax = a;
       }
     }
-    /* Stage 3 for outliers: per-row power-of-two scale, E4M3 codes of w / 2^e */
-    const int e = sdqo_fp8_scale_exp(out_amax);
-    out_sexp[n] = e;
-    for (int64_t g = 0; g < G8; ++g)
-      for (int t = 0; t < on; ++t) {
-        int i = out_idx[(n * G8 + g) * on + t];
-        out_code[(n * G8 + g) * on + t] = sdqo_e4m3_encode(ldexp(sdqo_bf16_to_double(w[8 * g + i]), -e));
-      }
+    /* Stage 3 for outliers: per-row power-of-two scale, E4M3 codes of w / 2^e -- or int8 codes of w / s, s = amax / 127 */
+    if (cfg->out_fmt == SDQO_OUT_INT8) {
+      const float sw = sdqo_int8_scale(out_amax);
+      out_sexp[n] = float_bits(sw);
+      for (int64_t g = 0; g < G8; ++g)
+        for (int t = 0; t < on; ++t) {
+          int i = out_idx[(n * G8 + g) * on + t];
+          out_code[(n * G8 + g) * on + t] = (uint8_t)sdqo_int8_encode(sdqo_bf16_to_double(w[8 * g + i]), sw);
+        }
+    } else {
+      const int e = sdqo_fp8_scale_exp(out_amax);
+      out_sexp[n] = e;
+      for (int64_t g = 0; g < G8; ++g)
+        for (int t = 0; t < on; ++t) {
+          int i = out_idx[(n * G8 + g) * on + t];
+          out_code[(n * G8 + g) * on + t] = sdqo_e4m3_encode(ldexp(sdqo_bf16_to_double(w[8 * g + i]), -e));
+        }
+    }
 
     /* Stage 1 on the remaining values: N:M pruning by significance.  The dense configuration
        (Section 5, decomposition-stage study: 8:8 split as 1:8 outliers + 7:8 inliers) skips it. */
@@ -412,7 +454,7 @@ int sdqo_dequant_weights(int64_t N, int64_t K, const sdqo_config* cfg,
     for (int64_t g = 0; g < G8; ++g)
       for (int t = 0; t < on; ++t) {
         int64_t k = 8 * g + out_idx[(n * G8 + g) * on + t];
-        W_out[n * K + k] = ldexp(sdqo_e4m3_decode(out_code[(n * G8 + g) * on + t]), out_sexp[n]);
+        W_out[n * K + k] = out_value(cfg, out_code[(n * G8 + g) * on + t], out_sexp[n]);
       }
   }
   return 0;
@@ -421,7 +463,8 @@ int sdqo_dequant_weights(int64_t N, int64_t K, const sdqo_config* cfg,
 /* ------------------------------------------------------------------ activations: A -> A_i (4-bit), A_o (8-bit)
  * X [M][K] bf16 patterns.  xq4_code [M][K] E2M1 codes, xq4_scale [M][K/in_block] E8M0 codes (SDQO_SCALE_UE4M3:
  * unsigned E4M3 codes; the Q-Vector scale is then that value times 2^xq8_sexp[m]),
- * xq8_code [M][K] E4M3 codes, xq8_sexp [M] exponent e of the per-token scale 2^e.
+ * xq8_code [M][K] E4M3 codes, xq8_sexp [M] exponent e of the per-token scale 2^e (SDQO_OUT_INT8: int8 codes and the bit
+ * pattern of the token's fp32 scale amax / 127; not combined with SDQO_SCALE_UE4M3, whose 4-bit scales hang on e).
  * +-Inf saturates to the largest finite value; NaN is rejected (-2). */
 int sdqo_quantize_act(const uint16_t* X, int64_t M, int64_t K, const sdqo_config* cfg,
                       uint8_t* xq4_code, uint8_t* xq4_scale, uint8_t* xq8_code, int32_t* xq8_sexp) {
@@ -429,6 +472,7 @@ int sdqo_quantize_act(const uint16_t* X, int64_t M, int64_t K, const sdqo_config
   if (cfg->in_block != 32 && cfg->in_block != 64) return -1;
   if (cfg->scale_rule < 0 || cfg->scale_rule > SDQO_SCALE_UE4M3) return -1;
   if (K % cfg->in_block != 0) return -1;
+  if (cfg->out_fmt != SDQO_OUT_E4M3 && (cfg->out_fmt != SDQO_OUT_INT8 || cfg->scale_rule == SDQO_SCALE_UE4M3)) return -1;
   const int Bs = cfg->in_block;
   const double BF16_MAX = 3.3895313892515355e38;
   for (int64_t m = 0; m < M; ++m) {
@@ -445,7 +489,8 @@ int sdqo_quantize_act(const uint16_t* X, int64_t M, int64_t K, const sdqo_config
     }
     /* the token's 8-bit scale exponent; under two-level scaling also the power-of-two factor of its 4-bit Q-Vectors */
     const int e = sdqo_fp8_scale_exp(row_amax);
-    xq8_sexp[m] = e;
+    const float sx = sdqo_int8_scale(row_amax);
+    xq8_sexp[m] = cfg->out_fmt == SDQO_OUT_INT8 ? float_bits(sx) : e;
     for (int64_t b = 0; b < K / Bs; ++b) {
       double amax = 0.0;
       for (int64_t k = b * Bs; k < (b + 1) * Bs; ++k) {
@@ -464,7 +509,7 @@ int sdqo_quantize_act(const uint16_t* X, int64_t M, int64_t K, const sdqo_config
     for (int64_t k = 0; k < K; ++k) {
       double v = sdqo_bf16_to_double(x[k]);
       if (isinf(v)) v = copysign(BF16_MAX, v);
-      xq8_code[m * K + k] = sdqo_e4m3_encode(ldexp(v, -e));
+      xq8_code[m * K + k] = cfg->out_fmt == SDQO_OUT_INT8 ? (uint8_t)sdqo_int8_encode(v, sx) : sdqo_e4m3_encode(ldexp(v, -e));
     }
   }
   return 0;
@@ -487,7 +532,7 @@ int sdqo_linear(int64_t M, int64_t N, int64_t K, const sdqo_config* cfg,
   for (int64_t m = 0; m < M; ++m)
     for (int64_t k = 0; k < K; ++k) {
       A_i[m * K + k] = sdqo_e2m1_decode(xq4_code[m * K + k]) * scale_value(cfg, xq4_scale[m * (K / Bs) + k / Bs], xq8_sexp[m]);
-      A_o[m * K + k] = ldexp(sdqo_e4m3_decode(xq8_code[m * K + k]), xq8_sexp[m]);
+      A_o[m * K + k] = out_value(cfg, xq8_code[m * K + k], xq8_sexp[m]);
     }
 #pragma omp parallel num_threads(n_threads > 0 ? n_threads : 1)
   {
@@ -531,7 +576,7 @@ int sdqo_linear(int64_t M, int64_t N, int64_t K, const sdqo_config* cfg,
       for (int64_t g = 0; g < G8; ++g)
         for (int t = 0; t < on; ++t) {
           ko[no] = (int32_t)(8 * g + out_idx[(n * G8 + g) * on + t]);
-          wo[no++] = ldexp(sdqo_e4m3_decode(out_code[(n * G8 + g) * on + t]), out_sexp[n]);
+          wo[no++] = out_value(cfg, out_code[(n * G8 + g) * on + t], out_sexp[n]);
         }
       for (int64_t m = 0; m < M; ++m) {
         double acc = 0.0;

@@ -29,6 +29,7 @@ def gran_keep(n: int) -> int:
     return 2 + (8 - n)
 SCALE_OCP_FLOOR, SCALE_CEIL_NOSAT, SCALE_UE4M3 = 0, 1, 2
 ORDER_LARGE, ORDER_SMALL = 0, 1
+OUT_E4M3, OUT_INT8 = 0, 1      # 8-bit format of W_o / A_o: E4M3 with power-of-two scales, or int8 with fp32 scales amax / 127
 
 
 def build(force: bool = False) -> str:
@@ -43,7 +44,7 @@ def build(force: bool = False) -> str:
 
 class _Cfg(ctypes.Structure):
     _fields_ = [("out_n", ctypes.c_int), ("in_gran", ctypes.c_int), ("in_block", ctypes.c_int),
-                ("scale_rule", ctypes.c_int), ("out_order", ctypes.c_int)]
+                ("scale_rule", ctypes.c_int), ("out_order", ctypes.c_int), ("out_fmt", ctypes.c_int)]
 
 
 @dataclass(frozen=True)
@@ -53,9 +54,10 @@ class Config:
     in_block: int = 64
     scale_rule: int = SCALE_OCP_FLOOR
     out_order: int = 0          # ORDER_LARGE; ORDER_SMALL takes the least significant values as outliers (study control)
+    out_fmt: int = 0            # OUT_E4M3; OUT_INT8: int8 outlier operands (out_sexp / xq8_sexp then hold fp32 bit patterns)
 
     def c(self) -> _Cfg:
-        return _Cfg(self.out_n, self.in_gran, self.in_block, self.scale_rule, self.out_order)
+        return _Cfg(self.out_n, self.in_gran, self.in_block, self.scale_rule, self.out_order, self.out_fmt)
 
 
 _lib = None
@@ -79,6 +81,10 @@ def lib():
         L.sdqo_ue4m3_scale_code.argtypes = [ctypes.c_double, ctypes.c_int]
         L.sdqo_fp8_scale_exp.restype = ctypes.c_int
         L.sdqo_fp8_scale_exp.argtypes = [ctypes.c_double]
+        L.sdqo_int8_scale.restype = ctypes.c_float
+        L.sdqo_int8_scale.argtypes = [ctypes.c_double]
+        L.sdqo_int8_encode.restype = ctypes.c_int8
+        L.sdqo_int8_encode.argtypes = [ctypes.c_double, ctypes.c_float]
         L.sdqo_bits_per_weight_part.restype = ctypes.c_double
         L.sdqo_bits_per_weight_part.argtypes = [ctypes.c_int] * 5
         L.sdqo_relative_cost.restype = ctypes.c_double
@@ -194,7 +200,10 @@ def dequant_act(q: QAct):
     else:
         sc = np.repeat(np.ldexp(1.0, q.xq4_scale.astype(np.int64) - 127), q.cfg.in_block, axis=1)
     A_i = e2m1[q.xq4_code] * sc
-    A_o = np.ldexp(e4m3[q.xq8_code], q.xq8_sexp[:, None].astype(np.int64))
+    if q.cfg.out_fmt == OUT_INT8:
+        A_o = q.xq8_code.view(np.int8).astype(np.float64) * q.xq8_sexp.view(np.float32)[:, None].astype(np.float64)
+    else:
+        A_o = np.ldexp(e4m3[q.xq8_code], q.xq8_sexp[:, None].astype(np.int64))
     return A_i, A_o
 
 
