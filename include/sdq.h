@@ -44,6 +44,14 @@ enum { SDQ_GRAN_PAIR = 0, SDQ_GRAN_ELEM = 1, SDQ_GRAN_DENSE = 2 }; /* inlier pat
 #define SDQ_GRAN_3OF4 9                   /* S-Vectors of 4: 3:4 = 1:4 outliers + 2:4 inliers                 */
 enum { SDQ_SCALE_OCP_FLOOR = 0, SDQ_SCALE_CEIL_NOSAT = 1, SDQ_SCALE_UE4M3 = 2 }; /* Q-Vector scale rule */
 enum { SDQ_ORDER_LARGE = 0, SDQ_ORDER_SMALL = 1 };          /* Stage 2 takes the most / least significant values */
+/* 8-bit format of the outlier operands.  SDQ_OUT_E4M3: FP8 E4M3 with a power-of-two scale per weight row / token, applied by
+ * the tensor core, so that O_i and O_o can share an accumulator.  SDQ_OUT_INT8 (Section 5.1 "quantize 1:8 W_o as int8 ...
+ * A would be quantized to int8 A_o"): symmetric int8, one fp32 scale amax / 127 per weight row and per token (1 for an
+ * all-zero vector), code = integer nearest to x / s (ties to even, |code| <= 127), both quotients formed in fp32; O_o is
+ * accumulated exactly in int32 and scaled in the epilogue.  Pair-wise 4:8 inliers with in_block 64 only; computed by
+ * sdq_linear_group's fused kernel (other calls return SDQ_ERR_UNSUPPORTED for it).  out_sexp / xq8_sexp of the canonical
+ * exports then hold the bit patterns of the fp32 scales. */
+enum { SDQ_OUT_E4M3 = 0, SDQ_OUT_INT8 = 1 };
 
 /* "pattern, formats" of the decomposition (Section 5, Stages 1-3).
  *   out_n      outliers extracted per S-Vector of 8 consecutive K (Stage 2): 0, 1 or 2; stored as
@@ -87,6 +95,8 @@ typedef struct {
   int32_t scale_rule;
   int32_t out_order;   /* SDQ_ORDER_LARGE (the method) or SDQ_ORDER_SMALL: outliers in ascending order of the
                           metric, the decomposition-stage study's control; sdq_quantize_act ignores it */
+  int32_t out_fmt;     /* SDQ_OUT_E4M3, or SDQ_OUT_INT8: the 8-bit operands W_o and A_o in int8 (Section 5.1; the
+                          evaluation's "1:8int8" configurations) */
 } sdq_config_t;
 
 /* Host-side descriptor of a packed weight matrix (filled by sdq_decompose; plain data, may be

@@ -26,6 +26,7 @@ def gran_keep(n: int) -> int:
     return 2 + (8 - n)
 SCALE_OCP_FLOOR, SCALE_CEIL_NOSAT, SCALE_UE4M3 = 0, 1, 2
 ORDER_LARGE, ORDER_SMALL = 0, 1
+OUT_E4M3, OUT_INT8 = 0, 1
 
 STATUS = ["ok", "invalid_arg", "shape", "alignment", "unsupported", "buffer_too_small", "nonfinite", "cuda", "timeout"]
 
@@ -39,10 +40,10 @@ class SdqError(RuntimeError):
 class Config(ctypes.Structure):
     """`pattern, formats` of the decomposition (sdq_config_t)."""
     _fields_ = [("out_n", ctypes.c_int32), ("in_gran", ctypes.c_int32), ("in_block", ctypes.c_int32),
-                ("scale_rule", ctypes.c_int32), ("out_order", ctypes.c_int32)]
+                ("scale_rule", ctypes.c_int32), ("out_order", ctypes.c_int32), ("out_fmt", ctypes.c_int32)]
 
-    def __init__(self, out_n=1, in_gran=GRAN_PAIR, in_block=64, scale_rule=SCALE_OCP_FLOOR, out_order=0):
-        super().__init__(out_n, in_gran, in_block, scale_rule, out_order)
+    def __init__(self, out_n=1, in_gran=GRAN_PAIR, in_block=64, scale_rule=SCALE_OCP_FLOOR, out_order=0, out_fmt=0):
+        super().__init__(out_n, in_gran, in_block, scale_rule, out_order, out_fmt)
 
 
 class _Packed(ctypes.Structure):
@@ -183,7 +184,7 @@ def packed_attach(buf: torch.Tensor) -> PackedWeight:
     assert buf.dtype == torch.uint8 and buf.is_contiguous()
     d = _Packed()
     _check(lib().sdq_packed_attach(buf.data_ptr(), buf.numel(), ctypes.byref(d), _stream()), "sdq_packed_attach")
-    cfg = Config(d.cfg.out_n, d.cfg.in_gran, d.cfg.in_block, d.cfg.scale_rule, d.cfg.out_order)
+    cfg = Config(d.cfg.out_n, d.cfg.in_gran, d.cfg.in_block, d.cfg.scale_rule, d.cfg.out_order, d.cfg.out_fmt)
     _, algo = packed_size(d.N, d.K, cfg)
     return PackedWeight(buf, d, d.N, d.K, cfg, algo)
 

@@ -29,6 +29,15 @@ __device__ __forceinline__ uint32_t e8m0_scale_code(float amax, int rule) {
   return (uint32_t)min(max(c, 0), 254);
 }
 
+// int8 operands (Section 5.1: W_o and A_o in int8): scale amax / 127 (1 for an all-zero vector) and code = the integer
+// nearest to x / s, ties to even, limited to +-127 -- both quotients in fp32, IEEE round-to-nearest divisions, the
+// precision in which the code is decided; returns the code's byte
+__device__ __forceinline__ float int8_scale(float amax) { return amax == 0.0f ? 1.0f : __fdiv_rn(amax, 127.0f); }
+__device__ __forceinline__ uint32_t int8_code(float x, float s) {
+  const float r = fminf(fmaxf(rintf(__fdiv_rn(x, s)), -127.0f), 127.0f);
+  return (uint32_t)(int)r & 0xFFu;
+}
+
 // exponent e of the power-of-two scale of an 8-bit (E4M3, max 448 = 1.75 * 2^8) operand:
 // the smallest integer with amax <= 448 * 2^e, limited to what an E8M0 byte can carry
 __device__ __forceinline__ int fp8_scale_exp(float amax) {

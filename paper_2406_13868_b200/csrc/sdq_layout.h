@@ -95,11 +95,11 @@ constexpr size_t HEADER_BYTES = 256;
 // What the first HEADER_BYTES of a packed buffer hold (the rest of the 256 bytes is zero): enough to rebuild the host
 // descriptor from the bytes alone.
 constexpr uint64_t BLOB_MAGIC = 0x0030303242514453ull;   // "SDQB200\0", little endian
-constexpr uint32_t BLOB_VERSION = 2;                     // layout version: 2 = compact outlier records tiled per 128 K (WC)
+constexpr uint32_t BLOB_VERSION = 3;                     // layout version: 2 = compact outlier records tiled per 128 K (WC); 3 = six configuration words
 struct BlobHeader {
   uint64_t magic;
   uint32_t version, header_bytes;
-  int32_t cfg[5];          // out_n, in_gran, in_block, scale_rule, out_order
+  int32_t cfg[6];          // out_n, in_gran, in_block, scale_rule, out_order, out_fmt
   uint32_t tiled;          // 1: stage-tiled tensor-core layout, 0: canonical arrays (decompose-only reading)
   int64_t N, K;
   uint64_t total;          // bytes of the whole buffer

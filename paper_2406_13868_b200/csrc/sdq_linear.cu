@@ -722,6 +722,8 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   if (Xq->K != P->K || Xq->M <= 0 || P->N <= 0 || P->N % TILE_ROWS || P->K % K2 || ldy < P->N) return SDQ_ERR_SHAPE;
   if (Xq->cfg.in_block != P->cfg.in_block || Xq->cfg.scale_rule != P->cfg.scale_rule) return SDQ_ERR_SHAPE;
   if (!is_tensor_core_reading(P->cfg)) return SDQ_ERR_UNSUPPORTED;
+  if (P->cfg.out_n > 0 && Xq->cfg.out_fmt != P->cfg.out_fmt) return SDQ_ERR_SHAPE;
+  if (P->cfg.out_n > 0 && P->cfg.out_fmt == SDQ_OUT_INT8) return SDQ_ERR_UNSUPPORTED;   // int8 outliers: the grouped few-token kernel only
   if (P->cfg.scale_rule == SDQ_SCALE_UE4M3 && !(P->cfg.in_gran == SDQ_GRAN_PAIR && P->cfg.in_block == 32)) return SDQ_ERR_UNSUPPORTED;
   if (((uintptr_t)Y & 15) || (ldy % 8) || ((uintptr_t)ws & 15)) return SDQ_ERR_ALIGNMENT;
   DeviceInfo* dinfo = device_info();
@@ -911,10 +913,11 @@ static sdq_status_t launch_group(int n, const sdq_act_t* const* Xq, const sdq_pa
     if (x->K != w->K || x->M <= 0 || w->N <= 0 || w->N % TILE_ROWS || w->K % K2 || ldy[i] < w->N) return SDQ_ERR_SHAPE;
     if (x->cfg.in_block != w->cfg.in_block || x->cfg.scale_rule != w->cfg.scale_rule) return SDQ_ERR_SHAPE;
     if (!is_tensor_core_reading(w->cfg)) return SDQ_ERR_UNSUPPORTED;
+    if (w->cfg.out_n > 0 && x->cfg.out_fmt != w->cfg.out_fmt) return SDQ_ERR_SHAPE;
     if (((uintptr_t)Y[i] & 15) || (ldy[i] % 8)) return SDQ_ERR_ALIGNMENT;
     // the grouped kernel carries the primary format: pair-wise 4:8 inliers, one E8M0 scale per 64 K, at most one outlier per S-Vector
     fused = fused && x->M <= 32 && w->cfg.in_gran == SDQ_GRAN_PAIR && w->cfg.in_block == 64 && w->cfg.scale_rule != SDQ_SCALE_UE4M3 &&
-            w->cfg.out_n <= 1 && w->cfg.out_n == P[0]->cfg.out_n &&
+            w->cfg.out_n <= 1 && w->cfg.out_n == P[0]->cfg.out_n && w->cfg.out_fmt == P[0]->cfg.out_fmt &&
             w->K >= 4 * K2;   // an item spans at least half the ring: the kernel's per-item barriers then never run two phases apart
     items += w->N / TILE_ROWS;
     if (x->M > max_m) max_m = x->M;
@@ -931,6 +934,7 @@ static sdq_status_t launch_group(int n, const sdq_act_t* const* Xq, const sdq_pa
   g.n = n;
   g.n_tile = max_m <= 16 ? 16 : 32;
   g.out_n = P[0]->cfg.out_n;
+  g.out_i8 = g.out_n > 0 && P[0]->cfg.out_fmt == SDQ_OUT_INT8;
   g.total_items = (int)items;
   g.flags = device_flags();
   if (!g.flags) return SDQ_ERR_CUDA;
@@ -942,6 +946,7 @@ static sdq_status_t launch_group(int n, const sdq_act_t* const* Xq, const sdq_pa
     m.w = (const uint8_t*)P[i]->dev; m.x = (const uint8_t*)Xq[i]->dev; m.Y = Y[i]; m.ldy = ldy[i];
     m.wi = po.wi; m.wc = po.wc; m.sfa_out = po.sfa_out;
     m.xi = ao.xi; m.xo = ao.xo; m.sfb_out = ao.sfb_out;
+    m.wsc = po.osexp; m.xsc = ao.sexp;
     m.M = (int)Xq[i]->M; m.T2 = (int)(P[i]->K / K2);
     m.item0 = item0;
     item0 += (int)(P[i]->N / TILE_ROWS);

@@ -48,12 +48,14 @@ struct GroupMat {
   int64_t ldy;
   uint64_t wi, wc, sfa_out;       // sections of w: inlier stages, compact outlier stages, outlier row-scale atoms
   uint64_t xi, xo, sfb_out;       // sections of x: 4-bit stages, 8-bit stages, token-scale atom
+  uint64_t wsc, xsc;              // int8 outliers: the fp32 row scales [N] of w and token scales [M] of x
   int M, T2;             // tokens, K / 256
   int item0;             // number of the matrix's first work item (= row tiles of the matrices before it)
 };
 struct GroupParams {
   int n, n_tile, nslot, slot_bytes, total_items;
   int out_n;             // outliers per S-Vector, the same for every matrix of the call (0 or 1)
+  int out_i8;            // the outlier operands are int8 with fp32 scales (else E4M3 with power-of-two scale atoms)
   uint32_t* flags;
   GroupMat m[GROUP_MAX];
 };

@@ -137,7 +137,7 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
           if (c == 0) ptx::mbar_expect_tx(&full_os[v], wcb + 2 * xb);
           const uint8_t* src = c == 0 ? m.w + m.wc + ((size_t)rt * 2 * m.T2 + 2 * k2) * (size_t)wc_bytes(1) : (c == 1 ? xo : xo + XO_BYTES);
           ptx::bulk_g2s(st + (c == 0 ? 0u : wcb + (c - 1) * xb), src, c == 0 ? wcb : xb, &full_os[v]);
-          if (k2 == 0 && c >= 1) {
+          if (k2 == 0 && c >= 1 && !p.out_i8) {     // (int8 outliers take fp32 scales in the epilogue: no scale atoms)
             // the item's outlier scale atoms (lane c = 1: of the weight rows, c = 2: of the tokens): a buffer and a barrier
             // of their own per item parity.  The buffer is free once every MMA of the item two back has completed (`acc_full`
             // of that item: it cannot complete again before these atoms land, since the next item on that accumulator needs
@@ -169,7 +169,7 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
       bool ok = true;
       const uint32_t smb = ptx::smem_u32(sm);
       const uint32_t id4[2] = {ptx::idesc_block_scaled(128, (uint32_t)p.n_tile, 1, true, 0, 0), ptx::idesc_block_scaled(128, (uint32_t)p.n_tile, 1, true, 2, 2)};
-      const uint32_t id8 = ptx::idesc_block_scaled(128, (uint32_t)p.n_tile, 0, true, 0, 0);
+      const uint32_t id8 = p.out_i8 ? ptx::idesc_i8(128, (uint32_t)p.n_tile, true) : ptx::idesc_block_scaled(128, (uint32_t)p.n_tile, 0, true, 0, 0);
       const uint32_t wcb = 2u * (uint32_t)wc_bytes(1);
       uint32_t v = 0, ph = 0, itc = 0;             // ring position and its lap parity, item count
       for (int item = first; item < p.total_items && ok; item += stride, ++itc) {
@@ -188,7 +188,7 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
           const int nb = T2 - k2 < 4 ? T2 - k2 : 4;
           uint32_t vi = v + lane, phi = ph;
           if (vi >= NU) { vi -= NU; phi ^= 1; }
-          const bool sf_lane = outw && k2 == 0 && lane == 4;
+          const bool sf_lane = outw && k2 == 0 && lane == 4 && !p.out_i8;
           uint64_t* bar = sf_lane ? &sf_full[ab] : (outw ? &built[vi < NU ? vi : 0] : &full_is[vi < NU ? vi : 0]);
           const uint32_t par = sf_lane ? ((itc >> 1) & 1) : phi;
           const bool mine = (int)lane < nb || sf_lane;
@@ -216,7 +216,7 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
                 ptx::mma_sp_mxf4(acc_col, ptx::smem_desc(sb + 4096, 128, 256), ptx::smem_desc(sb + WI_BYTES + 512, 128, 1024), id4[1], mb + 2,
                                  mb + 4, mb + 8, 1u);
               } else {
-                if (kk == 0) {
+                if (kk == 0 && !p.out_i8) {
                   const uint32_t sf = ptx::smem_u32(sfbuf) + ab * 2 * SF_ATOM_BYTES;
                   ptx::tc_cp_32x128b_warpx4(so, ptx::smem_desc(sf, 0, 128));
                   ptx::tc_cp_32x128b_warpx4(so + 4, ptx::smem_desc(sf + SF_ATOM_BYTES, 0, 128));
@@ -225,8 +225,13 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
                 for (uint32_t h = 0; h < 2; ++h) {
                   const uint32_t ca = tmem + GRP_TM_C + GRP_TM_C_COLS * vv + 16u * h, eb = tmem + GRP_TM_C + GRP_TM_C_COLS * vv + 32u + 4u * h;
                   const uint32_t xa = sb + isb + wcb + h * xb;
-                  ptx::mma_sp_mxf8_ta(acc_col, ca, ptx::smem_desc(xa, 128, 1024), id8, eb, so, so + 4, (kk | (int)h) ? 1u : 0u);
-                  ptx::mma_sp_mxf8_ta(acc_col, ca + 8, ptx::smem_desc(xa + 512, 128, 1024), id8, eb + 2, so, so + 4, 1u);
+                  if (p.out_i8) {     // the same containers and token codes as integers, int32 accumulator
+                    ptx::mma_sp_i8_ta(acc_col, ca, ptx::smem_desc(xa, 128, 1024), id8, eb, (kk | (int)h) ? 1u : 0u);
+                    ptx::mma_sp_i8_ta(acc_col, ca + 8, ptx::smem_desc(xa + 512, 128, 1024), id8, eb + 2, 1u);
+                  } else {
+                    ptx::mma_sp_mxf8_ta(acc_col, ca, ptx::smem_desc(xa, 128, 1024), id8, eb, so, so + 4, (kk | (int)h) ? 1u : 0u);
+                    ptx::mma_sp_mxf8_ta(acc_col, ca + 8, ptx::smem_desc(xa + 512, 128, 1024), id8, eb + 2, so, so + 4, 1u);
+                  }
                 }
               }
               ptx::tc_commit(&done[vv]);
@@ -259,6 +264,9 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
       ptx::named_bar_sync(3, 128);
       if (*timed_out) { ok = false; break; }
       ptx::tc_fence_after();
+      // int8 outliers: O_o = s_w[row] s_x[token] (exact int32 sum of code products); this thread's row scale
+      const float sw = p.out_i8 ? __ldg(reinterpret_cast<const float*>(m.w + m.wsc) + n0 + qd * 32 + lane) : 0.0f;
+      const float* sxp = reinterpret_cast<const float*>(m.x + m.xsc);
       uint32_t val[32];
       {
         // O = O_i + O_o: the two partial products of the item, added in fp32
@@ -271,7 +279,12 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
             if (p.out_n) ptx::tmem_ld_32x32b_x16(tb + 32 + c, b);
             ptx::tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 16; ++i) val[c + i] = p.out_n ? __float_as_uint(__uint_as_float(a[i]) + __uint_as_float(b[i])) : a[i];
+            for (int i = 0; i < 16; ++i) {
+              float o = 0.0f;
+              if (p.out_i8) { if ((int)(c + i) < m.M) o = (float)(int)b[i] * (sw * __ldg(sxp + c + i)); }
+              else if (p.out_n) o = __uint_as_float(b[i]);
+              val[c + i] = p.out_n ? __float_as_uint(__uint_as_float(a[i]) + o) : a[i];
+            }
           } else {
 #pragma unroll
             for (int i = 0; i < 16; ++i) val[c + i] = 0u;

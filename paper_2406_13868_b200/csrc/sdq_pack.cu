@@ -97,6 +97,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
   const bool sv4 = cfg.in_gran == SDQ_GRAN_3OF4;          // S-Vectors of 4: one outlier and two inliers per 4
   const bool small = cfg.out_order == SDQ_ORDER_SMALL;   // Stage 2 takes the least significant values (study control)
   const bool ue = cfg.scale_rule == SDQ_SCALE_UE4M3;     // two-level scaling with E4M3 Q-Vector scales (pair-wise, block 32)
+  const bool i8 = cfg.out_fmt == SDQ_OUT_INT8;           // int8 outliers with an fp32 row scale
 
   // ---- pass 1: largest outlier magnitude of the row (and, for two-level scaling, largest kept inlier), non-finite check
   uint32_t okey_max = 0, ikey_max = 0, bad = 0;
@@ -134,7 +135,8 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
   __syncthreads();
   if (tid == 0) {
     uint32_t m = max(max(s_red[0], s_red[1]), max(s_red[2], s_red[3]));
-    s_e = fp8_scale_exp(bf16_bits_to_float(m));
+    // int8 outliers: the row's fp32 scale amax / 127 travels as its bit pattern in the place of the exponent
+    s_e = i8 ? __float_as_int(int8_scale(bf16_bits_to_float(m))) : fp8_scale_exp(bf16_bits_to_float(m));
     const uint32_t mi = max(max(s_red_in[0], s_red_in[1]), max(s_red_in[2], s_red_in[3]));
     s_t = ue ? fp8_scale_exp(bf16_bits_to_float(mi)) : 0;   // exponent of the row's inlier factor 2^t
   }
@@ -158,7 +160,7 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     reinterpret_cast<int32_t*>(blob + off.wtexp)[n] = tw;
     // the accumulator of a row is kept in units of 2^tw (the inlier scale codes leave that factor out), so the outlier
     // row scale is 2^(e - tw); the GEMM's epilogue multiplies the factor back in
-    const uint32_t c = (uint32_t)min(max(e - tw + 127, 0), 254);
+    const uint32_t c = i8 ? 127u : (uint32_t)min(max(e - tw + 127, 0), 254);    // (int8: the epilogue applies the scales)
     *reinterpret_cast<uint32_t*>(blob + off.sfa_out + (size_t)rt * SF_ATOM_BYTES + sf_off(r, 0)) = c * 0x01010101u;
   }
 
@@ -253,8 +255,9 @@ pack_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t l
     if (out_n > 0) {
       // Stage 3, outliers: E4M3 codes of w / 2^e; compact arrays plus the 2:4 embedding the sparse
       // FP8 tensor-core path consumes (per 4 K: two ascending slot indices, unused slots hold +0)
-      const uint32_t c0 = e4m3x1(bf16_bits_to_float(bits[o0]) * pow2_neg(e));
-      const uint32_t c1 = (o1 >= 0) ? e4m3x1(bf16_bits_to_float(bits[o1]) * pow2_neg(e)) : 0u;
+      // (or int8 codes of w / s, Section 5.1)
+      const uint32_t c0 = i8 ? int8_code(bf16_bits_to_float(bits[o0]), __int_as_float(e)) : e4m3x1(bf16_bits_to_float(bits[o0]) * pow2_neg(e));
+      const uint32_t c1 = (o1 >= 0) ? (i8 ? int8_code(bf16_bits_to_float(bits[o1]), __int_as_float(e)) : e4m3x1(bf16_bits_to_float(bits[o1]) * pow2_neg(e))) : 0u;
       // compact record of the 128-K stage: codes, then position nibbles (two S-Vectors share a byte when out_n = 1)
       uint8_t* wc = blob + off.wc + ((size_t)rt * T1 + k1) * (size_t)wc_bytes(out_n);
       const uint32_t gi = (uint32_t)(g & 15);
@@ -365,19 +368,21 @@ static bool cfg_ok(const sdq_config_t* c) {
          (c->out_order == SDQ_ORDER_LARGE || c->out_order == SDQ_ORDER_SMALL) &&
          (c->in_gran < SDQ_GRAN_DENSE || c->in_gran == SDQ_GRAN_3OF4 || 10 - c->in_gran > c->out_n) &&
          (c->in_gran != SDQ_GRAN_3OF4 || c->out_n != 1) &&
-         (c->in_block == 32 || c->in_block == 64) && c->scale_rule >= SDQ_SCALE_OCP_FLOOR && c->scale_rule <= SDQ_SCALE_UE4M3;
+         (c->in_block == 32 || c->in_block == 64) && c->scale_rule >= SDQ_SCALE_OCP_FLOOR && c->scale_rule <= SDQ_SCALE_UE4M3 &&
+         (c->out_fmt == SDQ_OUT_E4M3 || (c->out_fmt == SDQ_OUT_INT8 && c->scale_rule != SDQ_SCALE_UE4M3));
 }
 // valid configurations this kernel set does not carry out
 static bool cfg_unsupported(const sdq_config_t* c) {
   return (c->in_gran >= SDQ_GRAN_DENSE && c->in_block != 32) ||
-         (c->scale_rule == SDQ_SCALE_UE4M3 && !(c->in_gran == SDQ_GRAN_PAIR && c->in_block == 32));
+         (c->scale_rule == SDQ_SCALE_UE4M3 && !(c->in_gran == SDQ_GRAN_PAIR && c->in_block == 32)) ||
+         (c->out_fmt == SDQ_OUT_INT8 && !(c->in_gran == SDQ_GRAN_PAIR && c->in_block == 64));   // int8 outliers: the primary format only
 }
 
 static void fill_header(BlobHeader* h, const sdq_packed_t& d, bool tiled) {
   h->magic = BLOB_MAGIC;
   h->version = BLOB_VERSION;
   h->header_bytes = (uint32_t)HEADER_BYTES;
-  h->cfg[0] = d.cfg.out_n; h->cfg[1] = d.cfg.in_gran; h->cfg[2] = d.cfg.in_block; h->cfg[3] = d.cfg.scale_rule; h->cfg[4] = d.cfg.out_order;
+  h->cfg[0] = d.cfg.out_n; h->cfg[1] = d.cfg.in_gran; h->cfg[2] = d.cfg.in_block; h->cfg[3] = d.cfg.scale_rule; h->cfg[4] = d.cfg.out_order; h->cfg[5] = d.cfg.out_fmt;
   h->tiled = tiled ? 1u : 0u;
   h->N = d.N; h->K = d.K;
   h->total = d.bytes;
@@ -462,7 +467,7 @@ extern "C" sdq_status_t sdq_packed_attach(const void* dev, size_t bytes, sdq_pac
   const BlobHeader* h = reinterpret_cast<const BlobHeader*>(raw);
   if (h->magic != BLOB_MAGIC || h->version != BLOB_VERSION || h->header_bytes != HEADER_BYTES) return SDQ_ERR_UNSUPPORTED;
   sdq_config_t cfg;
-  cfg.out_n = h->cfg[0]; cfg.in_gran = h->cfg[1]; cfg.in_block = h->cfg[2]; cfg.scale_rule = h->cfg[3]; cfg.out_order = h->cfg[4];
+  cfg.out_n = h->cfg[0]; cfg.in_gran = h->cfg[1]; cfg.in_block = h->cfg[2]; cfg.scale_rule = h->cfg[3]; cfg.out_order = h->cfg[4]; cfg.out_fmt = h->cfg[5];
   if (!cfg_ok(&cfg) || cfg_unsupported(&cfg)) return SDQ_ERR_SHAPE;
   if (h->N <= 0 || h->K <= 0 || h->N % TILE_ROWS || h->K % K2) return SDQ_ERR_SHAPE;
   // the sections must sit where this library puts them for that configuration and shape

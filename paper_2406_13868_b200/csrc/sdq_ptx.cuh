@@ -113,6 +113,12 @@ __device__ __forceinline__ uint32_t idesc_block_scaled(uint32_t M, uint32_t N, u
          ((M >> 4) << 24) | (a_sf_id << 29);
 }
 
+// instruction descriptor of kind::i8: signed 8-bit A and B, int32 accumulate, K-major A and B (no scales: bits 4..5 are
+// the accumulator format, 2 = S32; operand formats 1 = signed)
+__device__ __forceinline__ uint32_t idesc_i8(uint32_t M, uint32_t N, bool sparse) {
+  return ((sparse ? 1u : 0u) << 2) | (2u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
 // smem -> TMEM copies: 128 rows x 16 B (sparsity metadata) and 32 rows x 16 B replicated to the
 // four 32-lane quarters (scale-factor atoms)
 __device__ __forceinline__ void tc_cp_128x128b(uint32_t taddr, uint64_t sdesc) {
@@ -169,6 +175,14 @@ __device__ __forceinline__ void mma_sp_mxf8_ta(uint32_t d, uint32_t a_tmem, uint
       "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
       "tcgen05.mma.sp.cta_group::1.kind::mxf8f6f4.block_scale [%0], [%1], %2, [%7], %3, [%5], [%6], p;\n}" ::"r"(d),
       "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb), "r"(e_tmem)
+      : "memory");
+}
+// 2:4-sparse int8 product into an int32 accumulator, A (stored half) and metadata in tensor memory: K = 64 per instruction
+__device__ __forceinline__ void mma_sp_i8_ta(uint32_t d, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t e_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.sp.cta_group::1.kind::i8 [%0], [%1], %2, [%5], %3, p;\n}" ::"r"(d),
+      "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(e_tmem)
       : "memory");
 }
 // all previously issued tcgen05 async ops of this thread arrive on the mbarrier when complete

@@ -90,6 +90,8 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
   ramax = fmaxf(ramax, __shfl_xor_sync(0xffffffffu, ramax, 2));
   const int e = fp8_scale_exp(ramax);
   const float s8 = pow2_neg(e);
+  const bool i8 = cfg.out_fmt == SDQ_OUT_INT8;       // A_o in int8: fp32 token scale amax / 127, handed on as its bit pattern
+  const float sx = int8_scale(ramax);
 
   const int64_t mt = m / TILE_TOK;
   const uint32_t tk = (uint32_t)(m % TILE_TOK);
@@ -100,10 +102,10 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
   uint8_t* xi_base = buf + off.xi + (size_t)mt * T2 * xib;
   uint8_t* xo_base = buf + off.xo + (size_t)mt * T1 * XO_BYTES;
   if (live && blockIdx.y == 0 && warp == 0 && l == 0) {
-    reinterpret_cast<int32_t*>(buf + off.sexp)[m] = e;
+    reinterpret_cast<int32_t*>(buf + off.sexp)[m] = i8 ? __float_as_int(sx) : e;
     // two-level scaling keeps a token's accumulator column in units of 2^e (the 4-bit scale codes leave that factor out):
     // the 8-bit product then takes the scale 1 here and the GEMM's epilogue multiplies 2^e back in
-    *reinterpret_cast<uint32_t*>(buf + off.sfb_out + (size_t)mt * SF_ATOM_BYTES + sf_off(tk, 0)) = (uint32_t)(ue ? 127 : e + 127) * 0x01010101u;
+    *reinterpret_cast<uint32_t*>(buf + off.sfb_out + (size_t)mt * SF_ATOM_BYTES + sf_off(tk, 0)) = (uint32_t)((ue || i8) ? 127 : e + 127) * 0x01010101u;
   }
 
 #pragma unroll
@@ -137,7 +139,8 @@ quant_act_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K, int6
       for (int j = 0; j < 8; ++j) q4[j >> 2] |= e2m1x2(__fdiv_rn(v[2 * j], sv), __fdiv_rn(v[2 * j + 1], sv)) << (8 * (j & 3));
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) q8[j >> 1] |= e4m3x2(v[2 * j] * s8, v[2 * j + 1] * s8) << (16 * (j & 1));
+    for (int j = 0; j < 8; ++j)
+      q8[j >> 1] |= (i8 ? (int8_code(v[2 * j], sx) | (int8_code(v[2 * j + 1], sx) << 8)) : e4m3x2(v[2 * j] * s8, v[2 * j + 1] * s8)) << (16 * (j & 1));
     if (!live) continue;
     const uint32_t k = (uint32_t)b * 64 + l * 16;          // first element of this lane
     uint8_t* xi = xi_base + (size_t)(k >> 8) * xib;
@@ -220,6 +223,8 @@ quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K
   for (uint32_t c = 0; c < cx; ++c) ramax = fmaxf(ramax, s_all[c][t]);
   const int e = fp8_scale_exp(ramax);
   const float s8 = pow2_neg(e);
+  const bool i8 = cfg.out_fmt == SDQ_OUT_INT8;       // A_o in int8: fp32 token scale amax / 127, handed on as its bit pattern
+  const float sx = int8_scale(ramax);
 
   const int64_t mt = m / TILE_TOK;
   const uint32_t tk = (uint32_t)(m % TILE_TOK);
@@ -230,10 +235,10 @@ quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K
   uint8_t* xi_base = buf + off.xi + (size_t)mt * T2 * xib;
   uint8_t* xo_base = buf + off.xo + (size_t)mt * T1 * XO_BYTES;
   if (live && rank == 0 && warp == 0 && l == 0) {
-    reinterpret_cast<int32_t*>(buf + off.sexp)[m] = e;
+    reinterpret_cast<int32_t*>(buf + off.sexp)[m] = i8 ? __float_as_int(sx) : e;
     // two-level scaling keeps a token's accumulator column in units of 2^e (the 4-bit scale codes leave that factor out):
     // the 8-bit product then takes the scale 1 here and the GEMM's epilogue multiplies 2^e back in
-    *reinterpret_cast<uint32_t*>(buf + off.sfb_out + (size_t)mt * SF_ATOM_BYTES + sf_off(tk, 0)) = (uint32_t)(ue ? 127 : e + 127) * 0x01010101u;
+    *reinterpret_cast<uint32_t*>(buf + off.sfb_out + (size_t)mt * SF_ATOM_BYTES + sf_off(tk, 0)) = (uint32_t)((ue || i8) ? 127 : e + 127) * 0x01010101u;
   }
 #pragma unroll
   for (int i = 0; i < IT; ++i) {
@@ -267,7 +272,8 @@ quant_act_fused_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int64_t K
       for (int j = 0; j < 8; ++j) q4[j >> 2] |= e2m1x2(__fdiv_rn(v[2 * j], sv), __fdiv_rn(v[2 * j + 1], sv)) << (8 * (j & 3));
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) q8[j >> 1] |= e4m3x2(v[2 * j] * s8, v[2 * j + 1] * s8) << (16 * (j & 1));
+    for (int j = 0; j < 8; ++j)
+      q8[j >> 1] |= (i8 ? (int8_code(v[2 * j], sx) | (int8_code(v[2 * j + 1], sx) << 8)) : e4m3x2(v[2 * j] * s8, v[2 * j + 1] * s8)) << (16 * (j & 1));
     if (!live) continue;
     const uint32_t k = (uint32_t)b * 64 + l * 16;          // first element of this lane
     uint8_t* xi = xi_base + (size_t)(k >> 8) * xib;
@@ -308,7 +314,8 @@ using namespace sdq;
 
 static bool act_cfg_ok(const sdq_config_t* c) {
   return c && c->out_n >= 0 && c->out_n <= 2 && (c->in_block == 32 || c->in_block == 64) &&
-         c->scale_rule >= SDQ_SCALE_OCP_FLOOR && c->scale_rule <= SDQ_SCALE_UE4M3;
+         c->scale_rule >= SDQ_SCALE_OCP_FLOOR && c->scale_rule <= SDQ_SCALE_UE4M3 &&
+         (c->out_fmt == SDQ_OUT_E4M3 || (c->out_fmt == SDQ_OUT_INT8 && c->scale_rule != SDQ_SCALE_UE4M3));
 }
 
 extern "C" sdq_status_t sdq_act_size(int64_t M, int64_t K, const sdq_config_t* cfg, size_t* bytes)

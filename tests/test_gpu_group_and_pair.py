@@ -291,3 +291,100 @@ def test_a_bounded_wait_that_runs_out_sets_the_sticky_status_and_the_context_sta
     d, tol = y_close(y, so.linear(so.quantize_act(sdq_synth.bf16_bits(sdq_synth.make_act(3, 256, 4821)), oc),
                                   so.decompose(sdq_synth.bf16_bits(sdq_synth.make_weight(128, 256, 4820)), oc)))
     assert (d <= tol).all()
+
+
+# ---------------------------------------------------------------------------------------------------------------------
+# int8 outlier operands (Section 5.1: W_o and A_o in int8; the evaluation's "1:8int8" configurations)
+
+I8_ARGS = (1, so.GRAN_PAIR, 64, 0, 0, so.OUT_INT8)
+
+
+def _i8_cfgs():
+    m = sdq()
+    return m, m.Config(*I8_ARGS), so.Config(*I8_ARGS)
+
+
+@pytest.mark.parametrize("N,K,M", [(256, 512, 9), (1152, 1280, 130), (128, 16640, 3)])
+def test_int8_outlier_codes_and_scales_match_the_oracle_bit_for_bit(N, K, M):
+    """packer and activation quantizer: int8 codes, positions and the bit patterns of the fp32 scales (short and long rows:
+    the one-launch and the two-launch quantizer)"""
+    m, cfg, oc = _i8_cfgs()
+    W, X = sdq_synth.make_weight(N, K, 77), sdq_synth.make_act(M, K, 78)
+    p, xq = m.sdq_decompose(W.cuda(), cfg), m.sdq_quantize_act(X.cuda(), cfg)
+    assert m.device_status() == 0
+    op, oq = so.decompose(sdq_synth.bf16_bits(W), oc), so.quantize_act(sdq_synth.bf16_bits(X), oc)
+    pe = {k: v.cpu().numpy() for k, v in m.packed_export(p).items()}
+    ae = {k: v.cpu().numpy() for k, v in m.act_export(xq).items()}
+    for name in ("in_code", "in_meta", "in_scale", "out_code", "out_idx", "out_sexp"):
+        assert np.array_equal(pe[name], getattr(op, name)), name
+    for name in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp"):
+        assert np.array_equal(ae[name], getattr(oq, name)), name
+    # an all-zero row and an all-zero token: scale 1, codes 0
+    W2 = W.clone(); W2[5] = 0
+    X2 = X.clone(); X2[0] = 0
+    p2, x2 = m.sdq_decompose(W2.cuda(), cfg), m.sdq_quantize_act(X2.cuda(), cfg)
+    assert m.packed_export(p2)["out_sexp"].cpu().numpy().view(np.float32)[5] == 1.0
+    assert m.act_export(x2)["xq8_sexp"].cpu().numpy().view(np.float32)[0] == 1.0
+    assert not m.act_export(x2)["xq8_code"].cpu().numpy()[0].any()
+
+
+@pytest.mark.parametrize("shapes,Ms", [
+    ([(4096, 4096)] * 3, [1, 16, 5]),                      # q / k / v
+    ([(4096, 1024), (11008, 4096), (4096, 11008)], [7, 7, 7]),   # different widths and depths: up to 1376 outliers per row
+    ([(4096, 2048)] * 4, [32, 17, 20, 2]),                 # the wider token tile
+])
+def test_int8_outlier_group_call_matches_oracle(shapes, Ms):
+    m, cfg, oc = _i8_cfgs()
+    Ws = [sdq_synth.make_weight(N, K, 4700 + i) for i, (N, K) in enumerate(shapes)]
+    Xs = [sdq_synth.make_act(M, K, 4750 + i) for i, ((N, K), M) in enumerate(zip(shapes, Ms))]
+    ps = [m.sdq_decompose(W.cuda(), cfg) for W in Ws]
+    xqs = [m.sdq_quantize_act(X.cuda(), cfg) for X in Xs]
+    ys32 = m.sdq_linear_group(xqs, ps, f32=True)
+    ys16 = m.sdq_linear_group(xqs, ps)
+    assert m.device_status() == 0
+    for W, X, y32, y16 in zip(Ws, Xs, ys32, ys16):
+        op, oq = so.decompose(sdq_synth.bf16_bits(W), oc), so.quantize_act(sdq_synth.bf16_bits(X), oc)
+        N = W.shape[0]
+        for n0, n1 in ((0, 512), (N - 128, N)):
+            yref = so.linear(oq, op, n0, n1)
+            d, tol = y_close(y32[:, n0:n1].cpu().numpy(), yref)
+            assert (d <= tol).all(), (d.max(), (d / tol).max())
+        assert torch.equal(y16, y32.to(torch.bfloat16))
+    # the outlier part alone: weights whose only non-zeros are outliers give O = O_o = s_x s_w (integer sum), which the
+    # kernel forms exactly in int32 and scales once
+    N, K, M = 4096, 1024, 4
+    g = torch.Generator().manual_seed(9)
+    W = torch.zeros((N, K))
+    pos = torch.randint(0, 8, (N, K // 8), generator=g)
+    vals = torch.randn((N, K // 8), generator=g) * 0.05 + 0.001
+    W.view(N, K // 8, 8).scatter_(2, pos.unsqueeze(-1), vals.unsqueeze(-1))
+    W = W.to(torch.bfloat16)
+    X = sdq_synth.make_act(M, K, 10)
+    ps, xq = [m.sdq_decompose(W.cuda(), cfg)] * 3, m.sdq_quantize_act(X.cuda(), cfg)
+    y = m.sdq_linear_group([xq] * 3, ps, f32=True)[2].cpu().numpy()
+    op, oq = so.decompose(sdq_synth.bf16_bits(W), oc), so.quantize_act(sdq_synth.bf16_bits(X), oc)
+    qw = np.zeros((N, K), dtype=np.int64)
+    np.put_along_axis(qw.reshape(N, K // 8, 8), op.out_idx.astype(np.int64), op.out_code.view(np.int8).astype(np.int64), axis=2)
+    isum = oq.xq8_code.view(np.int8).astype(np.int64) @ qw.T
+    sx, sw = oq.xq8_sexp.view(np.float32), op.out_sexp.view(np.float32)
+    want = isum.astype(np.float32) * (sw[None, :] * sx[:, None])          # the kernel's own two fp32 roundings
+    assert np.array_equal(y, want)
+
+
+def test_int8_outliers_outside_the_grouped_kernel_are_refused():
+    m, cfg, oc = _i8_cfgs()
+    p = m.sdq_decompose(sdq_synth.make_weight(256, 1024, 1).cuda(), cfg)
+    x = m.sdq_quantize_act(sdq_synth.make_act(4, 1024, 1).cuda(), cfg)
+    with pytest.raises(RuntimeError):
+        m.sdq_linear(x, p)                                   # a single call
+    with pytest.raises(RuntimeError):
+        m.sdq_linear_group([x, x], [p, p])                   # too few row tiles for the fused kernel
+    x_e4m3 = m.sdq_quantize_act(sdq_synth.make_act(4, 1024, 1).cuda(), m.Config(1, so.GRAN_PAIR, 64, 0))
+    big = m.sdq_decompose(sdq_synth.make_weight(4096, 1024, 2).cuda(), cfg)
+    with pytest.raises(RuntimeError):
+        m.sdq_linear_group([x_e4m3] * 3, [big] * 3)          # the activations' 8-bit format differs from the weights'
+    with pytest.raises(RuntimeError):
+        m.sdq_decompose(sdq_synth.make_weight(256, 1024, 1).cuda(), m.Config(1, so.GRAN_PAIR, 32, 0, 0, so.OUT_INT8))   # block 32
+    # the blob header carries the format
+    q = m.packed_attach(big.buf.clone())
+    assert q.cfg.out_fmt == so.OUT_INT8
