@@ -408,6 +408,24 @@ def measure_decode(sdq, cfg, dev, peaks, layers: int = 32, reps: int = 20):
             res[name] = {"us_per_layer": us, "weight_GBps_algorithmic": gbs, "frac_of_hbm_peak": gbs / peaks["hbm"]}
         out["M%d" % M] = dict(res["group"], call="sdq_linear_group, 32 layers in one launch",
                               per_call_chain=dict(res["chain"], call="32 x sdq_linear"))
+    # the evaluation's outlier format (int8 with fp32 scales, Section 5.1) through the same grouped call
+    cfg8 = sdq.Config(cfg.out_n, cfg.in_gran, cfg.in_block, cfg.scale_rule, cfg.out_order, sdq.OUT_INT8)
+    packs8 = []
+    for i in range(layers):
+        W = sdq_synth.make_weight(N, K, 2000 + i, device=str(dev))
+        packs8.append(sdq.sdq_decompose(W, cfg8))
+        del W
+    out["int8_outliers"] = {}
+    for M in (1, 16):
+        X = sdq_synth.make_act(M, K, 2100 + M, device=str(dev))
+        Ys = [torch.empty((M, N), dtype=torch.bfloat16, device=dev) for _ in packs8]
+        xq = sdq.sdq_quantize_act(X, cfg8)
+        us = time_graph(lambda: sdq.sdq_linear_group([xq] * layers, packs8, Ys), reps=reps) * 1e3 / layers
+        assert sdq.device_status() == 0
+        gbs = algo / (us * 1e-6) / 1e9
+        out["int8_outliers"]["M%d" % M] = {"us_per_layer": us, "weight_GBps_algorithmic": gbs, "frac_of_hbm_peak": gbs / peaks["hbm"],
+                                           "call": "sdq_linear_group, 32 layers in one launch, SDQ_OUT_INT8"}
+    del packs8
     out["workload"] = ("llama7b_attn_proj_decode 4096x4096, %d distinct layers in rotation (%.0f MB packed > L2), products only, "
                        "one CUDA graph per variant replayed %d times" % (layers, layers * packs[0].buf.numel() / 1e6, reps))
     out["algorithmic_bytes_per_layer"] = algo
