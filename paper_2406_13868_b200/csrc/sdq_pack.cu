@@ -17,28 +17,6 @@ struct GroupSel {
   int o0, o1;        // outlier positions (ascending), -1 if absent
 };
 
-// positions of the out_n most (small: least) significant values, ties to the lower index
-__device__ __forceinline__ void select_outliers(const uint32_t (&key)[8], int out_n, bool small, int& o0, int& o1) {
-  o0 = o1 = -1;
-  if (out_n >= 1) {
-    int b = 0;
-#pragma unroll
-    for (int i = 1; i < 8; ++i)
-      if (small ? key[i] < key[b] : key[i] > key[b]) b = i;
-    o0 = b;
-  }
-  if (out_n >= 2) {
-    int b = -1;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      if (i == o0) continue;
-      if (b < 0 || (small ? key[i] < key[b] : key[i] > key[b])) b = i;
-    }
-    o1 = b;
-    if (o0 > o1) { int t = o0; o0 = o1; o1 = t; }
-  }
-}
-
 // S-Vectors of 4: the most significant of positions 0..3 and of positions 4..7 (ties to the lower index)
 __device__ __forceinline__ void select_outliers_per_4(const uint32_t (&key)[8], bool small, int& o0, int& o1) {
   o0 = 0; o1 = 4;
@@ -46,16 +24,6 @@ __device__ __forceinline__ void select_outliers_per_4(const uint32_t (&key)[8], 
   for (int i = 1; i < 4; ++i) {
     if (small ? key[i] < key[o0] : key[i] > key[o0]) o0 = i;
     if (small ? key[4 + i] < key[o1] : key[4 + i] > key[o1]) o1 = 4 + i;
-  }
-}
-
-__device__ __forceinline__ void load_group(const __nv_bfloat16* w, uint32_t (&bits)[8]) {
-  const uint4 v = *reinterpret_cast<const uint4*>(w);
-  const uint32_t r[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    bits[2 * i] = r[i] & 0xFFFFu;
-    bits[2 * i + 1] = r[i] >> 16;
   }
 }
 

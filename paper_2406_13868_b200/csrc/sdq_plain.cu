@@ -10,36 +10,6 @@
 
 namespace sdq {
 
-__device__ __forceinline__ void load_group8(const __nv_bfloat16* w, uint32_t (&bits)[8]) {
-  const uint4 v = *reinterpret_cast<const uint4*>(w);
-  const uint32_t r[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    bits[2 * i] = r[i] & 0xFFFFu;
-    bits[2 * i + 1] = r[i] >> 16;
-  }
-}
-__device__ __forceinline__ void pick_outliers(const uint32_t (&key)[8], int out_n, bool small, int& o0, int& o1) {
-  o0 = o1 = -1;
-  if (out_n >= 1) {
-    int b = 0;
-#pragma unroll
-    for (int i = 1; i < 8; ++i)
-      if (small ? key[i] < key[b] : key[i] > key[b]) b = i;
-    o0 = b;
-  }
-  if (out_n >= 2) {
-    int b = -1;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      if (i == o0) continue;
-      if (b < 0 || (small ? key[i] < key[b] : key[i] > key[b])) b = i;
-    }
-    o1 = b;
-    if (o0 > o1) { int t = o0; o0 = o1; o1 = t; }
-  }
-}
-
 __global__ void __launch_bounds__(128)
 pack_plain_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int64_t ldw, sdq_config_t cfg, const float* __restrict__ colw,
                   uint8_t* __restrict__ blob, PlainPackedOffsets off, uint32_t* __restrict__ flags)
@@ -55,7 +25,7 @@ pack_plain_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int
   uint32_t okey_max = 0, bad = 0;
   for (int g = tid; g < G; g += 128) {
     uint32_t bits[8], key[8];
-    load_group8(wrow + 8 * g, bits);
+    load_group(wrow + 8 * g, bits);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       key[i] = bits[i] & 0x7FFFu;
@@ -64,7 +34,7 @@ pack_plain_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int
     uint32_t skey[8];
     bad |= selection_keys(key, colw, g, skey);
     int o0, o1;
-    pick_outliers(skey, out_n, cfg.out_order == SDQ_ORDER_SMALL, o0, o1);
+    select_outliers(skey, out_n, cfg.out_order == SDQ_ORDER_SMALL, o0, o1);
     if (o0 >= 0) okey_max = max(okey_max, key[o0]);
     if (o1 >= 0) okey_max = max(okey_max, key[o1]);
   }
@@ -83,13 +53,13 @@ pack_plain_kernel(const __nv_bfloat16* __restrict__ W, int64_t N, int64_t K, int
 
   for (int g = tid; g < G; g += 128) {
     uint32_t bits[8], key[8];
-    load_group8(wrow + 8 * g, bits);
+    load_group(wrow + 8 * g, bits);
 #pragma unroll
     for (int i = 0; i < 8; ++i) key[i] = bits[i] & 0x7FFFu;
     uint32_t skey[8];
     selection_keys(key, colw, g, skey);
     int o0, o1;
-    pick_outliers(skey, out_n, cfg.out_order == SDQ_ORDER_SMALL, o0, o1);
+    select_outliers(skey, out_n, cfg.out_order == SDQ_ORDER_SMALL, o0, o1);
     int slot_pos[4];
     if (pair) {
       float score[4];
