@@ -263,6 +263,23 @@ sdq_status_t sdq_linear_group(int n, const sdq_act_t* const* Xq, const sdq_packe
 sdq_status_t sdq_linear_group_f32(int n, const sdq_act_t* const* Xq, const sdq_packed_t* const* P, float* const* Y_f32,
                                   const int64_t* ldy, void* stream);
 
+/* sdq_linear_group with the activation quantization inside the kernel (Section 5, Stage 3 fused into the linear layers'
+ * load path): Y_i = Q(X) W_i,in^T + Q'(X) W_i,out^T for n independent layers that read the SAME activations -- q / k / v, or
+ * gate / up, of a few tokens.
+ *   X_bf16: device, [M][K] bf16, row stride ldx elements (16-byte aligned, ldx % 8 == 0), M <= 16.  Every CTA of the one
+ *   persistent launch quantizes X into its own shared memory (the codes, scales and arithmetic of sdq_quantize_act, so
+ *   the results are bit-identical to sdq_quantize_act followed by sdq_linear_group) while the first weights stream in;
+ *   no quantized buffer exists in device memory and no second kernel runs.
+ *   P, Y, ldy as for sdq_linear_group; every P[i]->K == K.  The 8-bit format of A_o is the weights' (cfg.out_fmt).
+ *   Range: the fused kernel's (primary format, out_n <= 1, power-of-two scales, n <= 32, at least half as many 128-row
+ *   tiles as SMs) with 1024 <= K <= 4096 (X has to fit beside the weight ring); outside it the call returns
+ *   SDQ_ERR_UNSUPPORTED and launches nothing: quantize with sdq_quantize_act and use sdq_linear_group then.
+ *   Asynchronous on `stream`; allocates nothing. */
+sdq_status_t sdq_linear_group_x(int n, const void* X_bf16, int64_t M, int64_t K, int64_t ldx, const sdq_packed_t* const* P,
+                                void* const* Y_bf16, const int64_t* ldy, void* stream);
+sdq_status_t sdq_linear_group_x_f32(int n, const void* X_bf16, int64_t M, int64_t K, int64_t ldx, const sdq_packed_t* const* P,
+                                    float* const* Y_f32, const int64_t* ldy, void* stream);
+
 /* Built-in scratch variant of sdq_linear_ws (the paper has no counterpart: this is a packaging choice of the
  * library, not part of the method).
  *   For callers that hold nothing but their input and output pointers and cannot obtain device memory: a

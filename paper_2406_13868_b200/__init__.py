@@ -66,7 +66,7 @@ class _ActCanon(ctypes.Structure):
 
 EXPORTS = ["sdq_packed_size", "sdq_decompose", "sdq_decompose_metric", "sdq_channel_norm", "sdq_packed_export", "sdq_packed_attach", "sdq_act_size", "sdq_quantize_act", "sdq_act_export",
            "sdq_linear", "sdq_linear_f32", "sdq_workspace_size", "sdq_workspace_init", "sdq_linear_ws", "sdq_linear_f32_ws", "sdq_linear_noalloc",
-           "sdq_linear_group", "sdq_linear_group_f32", "sdq_diag_l2_copy", "sdq_diag_wait_timeout", "sdq_device_status", "sdq_status_string"]
+           "sdq_linear_group", "sdq_linear_group_f32", "sdq_linear_group_x", "sdq_linear_group_x_f32", "sdq_diag_l2_copy", "sdq_diag_wait_timeout", "sdq_device_status", "sdq_status_string"]
 
 _lib = None
 
@@ -269,6 +269,27 @@ def sdq_linear_group(xqs, ps, outs=None, f32: bool = False):
     LD = (ctypes.c_int64 * n)(*[o.stride(0) for o in outs])
     fn = lib().sdq_linear_group_f32 if f32 else lib().sdq_linear_group
     _check(fn(n, XA, PA, YA, LD, _stream()), "sdq_linear_group")
+    return outs
+
+
+def sdq_linear_group_x(X: torch.Tensor, ps, outs=None, f32: bool = False):
+    """Y[i] = sdq_linear(sdq_quantize_act(X), ps[i]) for layers that share the bf16 activations X [M <= 16, K], the quantizer
+    fused into the one persistent launch (see sdq_linear_group_x in include/sdq.h).  Returns the list of outputs."""
+    _need_cuda(X, "X")
+    assert X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    n, M, K = len(ps), X.shape[0], X.shape[1]
+    assert n > 0
+    dt = torch.float32 if f32 else torch.bfloat16
+    if outs is None:
+        outs = [torch.empty((M, p.N), dtype=dt, device=X.device) for p in ps]
+    for o, p in zip(outs, ps):
+        assert o.dtype == dt and o.shape == (M, p.N) and o.stride(1) == 1
+    PA = (ctypes.POINTER(_Packed) * n)(*[ctypes.pointer(p.desc) for p in ps])
+    YA = (ctypes.c_void_p * n)(*[o.data_ptr() for o in outs])
+    LD = (ctypes.c_int64 * n)(*[o.stride(0) for o in outs])
+    fn = lib().sdq_linear_group_x_f32 if f32 else lib().sdq_linear_group_x
+    _check(fn(n, ctypes.c_void_p(X.data_ptr()), ctypes.c_int64(M), ctypes.c_int64(K), ctypes.c_int64(X.stride(0)), PA, YA, LD, _stream()),
+           "sdq_linear_group_x")
     return outs
 
 

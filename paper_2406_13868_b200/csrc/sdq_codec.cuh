@@ -103,6 +103,10 @@ __device__ __forceinline__ float key_value(uint32_t key, uint32_t skey, bool wei
   return weighted ? __uint_as_float(skey) : bf16_bits_to_float(key);
 }
 
+// |x| with +-Inf replaced by the largest finite bf16 (saturation)
+__device__ __forceinline__ float sat_abs(float x) { return fminf(fabsf(x), 3.3895313892515355e38f); }
+__device__ __forceinline__ float sat(float x) { return copysignf(sat_abs(x), x); }
+
 // ---- Stage 2 helpers shared by the tiled and the plain packer (one thread per S-Vector of 8 weights) ----------
 // the 8 bf16 bit patterns of an S-Vector (one 16-byte load)
 __device__ __forceinline__ void load_group(const __nv_bfloat16* w, uint32_t (&bits)[8]) {

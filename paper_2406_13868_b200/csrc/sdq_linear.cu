@@ -935,6 +935,7 @@ static sdq_status_t launch_group(int n, const sdq_act_t* const* Xq, const sdq_pa
   g.n_tile = max_m <= 16 ? 16 : 32;
   g.out_n = P[0]->cfg.out_n;
   g.out_i8 = g.out_n > 0 && P[0]->cfg.out_fmt == SDQ_OUT_INT8;
+  g.x_bf16 = nullptr; g.x_ld = 0; g.x_M = 0; g.scale_rule = P[0]->cfg.scale_rule;
   g.total_items = (int)items;
   g.flags = device_flags();
   if (!g.flags) return SDQ_ERR_CUDA;
@@ -954,6 +955,63 @@ static sdq_status_t launch_group(int n, const sdq_act_t* const* Xq, const sdq_pa
   const cudaError_t e = launch_linear_group(g, f32, dinfo->sm_count, (cudaStream_t)stream, &dinfo->group_attr);
   return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
 }
+
+// The same with the activation quantizer inside the kernel: all layers read one bf16 X (see include/sdq.h).
+static sdq_status_t launch_group_x(int n, const void* X, int64_t M, int64_t K, int64_t ldx, const sdq_packed_t* const* P, void* const* Y,
+                                   const int64_t* ldy, void* stream, bool f32)
+{
+  if (n <= 0 || !X || !P || !Y || !ldy) return SDQ_ERR_INVALID_ARG;
+  if (M <= 0 || K <= 0 || K % K2 || ldx < K) return SDQ_ERR_SHAPE;
+  if (((uintptr_t)X & 15) || (ldx % 8)) return SDQ_ERR_ALIGNMENT;
+  DeviceInfo* dinfo = device_info();
+  if (!dinfo) return SDQ_ERR_CUDA;
+  int64_t items = 0;
+  for (int i = 0; i < n; ++i) {
+    const sdq_packed_t* w = P[i];
+    if (!w || !Y[i] || !w->dev) return SDQ_ERR_INVALID_ARG;
+    if (w->K != K || w->N <= 0 || w->N % TILE_ROWS || ldy[i] < w->N) return SDQ_ERR_SHAPE;
+    if (!is_tensor_core_reading(w->cfg)) return SDQ_ERR_UNSUPPORTED;
+    if (((uintptr_t)Y[i] & 15) || (ldy[i] % 8)) return SDQ_ERR_ALIGNMENT;
+    const sdq_config_t& c = w->cfg, &c0 = P[0]->cfg;
+    if (c.in_gran != SDQ_GRAN_PAIR || c.in_block != 64 || c.scale_rule == SDQ_SCALE_UE4M3 || c.out_n > 1 || c.out_n != c0.out_n ||
+        c.out_fmt != c0.out_fmt || c.scale_rule != c0.scale_rule)
+      return SDQ_ERR_UNSUPPORTED;
+    items += w->N / TILE_ROWS;
+  }
+  if (n > GROUP_MAX || M > 16 || K < 4 * K2 || !group_xres_fits((int)(K / K2), P[0]->cfg.out_n) || items * 2 < dinfo->sm_count || items >= (1 << 30))
+    return SDQ_ERR_UNSUPPORTED;
+  GroupParams g;
+  g.n = n;
+  g.n_tile = 16;
+  g.out_n = P[0]->cfg.out_n;
+  g.out_i8 = g.out_n > 0 && P[0]->cfg.out_fmt == SDQ_OUT_INT8;
+  g.x_bf16 = X; g.x_ld = ldx; g.x_M = (int)M; g.scale_rule = P[0]->cfg.scale_rule;
+  g.total_items = (int)items;
+  g.flags = device_flags();
+  if (!g.flags) return SDQ_ERR_CUDA;
+  int item0 = 0;
+  for (int i = 0; i < n; ++i) {
+    const PackedOffsets po = tiled_offsets(P[i]->N, P[i]->K, P[i]->cfg);
+    GroupMat& m = g.m[i];
+    m.w = (const uint8_t*)P[i]->dev; m.x = nullptr; m.Y = Y[i]; m.ldy = ldy[i];
+    m.wi = po.wi; m.wc = po.wc; m.sfa_out = po.sfa_out;
+    m.xi = m.xo = m.sfb_out = m.xsc = 0;
+    m.wsc = po.osexp;
+    m.M = (int)M; m.T2 = (int)(K / K2);
+    m.item0 = item0;
+    item0 += (int)(P[i]->N / TILE_ROWS);
+  }
+  const cudaError_t e = launch_linear_group(g, f32, dinfo->sm_count, (cudaStream_t)stream, &dinfo->group_attr);
+  return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
+}
+
+extern "C" sdq_status_t sdq_linear_group_x(int n, const void* X_bf16, int64_t M, int64_t K, int64_t ldx, const sdq_packed_t* const* P,
+                                           void* const* Y, const int64_t* ldy, void* stream)
+{ return launch_group_x(n, X_bf16, M, K, ldx, P, Y, ldy, stream, false); }
+
+extern "C" sdq_status_t sdq_linear_group_x_f32(int n, const void* X_bf16, int64_t M, int64_t K, int64_t ldx, const sdq_packed_t* const* P,
+                                               float* const* Y, const int64_t* ldy, void* stream)
+{ return launch_group_x(n, X_bf16, M, K, ldx, P, (void* const*)Y, ldy, stream, true); }
 
 extern "C" sdq_status_t sdq_linear_group(int n, const sdq_act_t* const* Xq, const sdq_packed_t* const* P, void* const* Y,
                                          const int64_t* ldy, void* stream)

@@ -56,10 +56,16 @@ struct GroupParams {
   int n, n_tile, nslot, slot_bytes, total_items;
   int out_n;             // outliers per S-Vector, the same for every matrix of the call (0 or 1)
   int out_i8;            // the outlier operands are int8 with fp32 scales (else E4M3 with power-of-two scale atoms)
+  // activation-resident variant (launch_linear_group with x_bf16 set): all matrices share one bf16 X [x_M][K], which every
+  // CTA quantizes into its own shared memory before it starts; GroupMat::x and its section offsets are then unused
+  const void* x_bf16;
+  int64_t x_ld;
+  int x_M, scale_rule;
   uint32_t* flags;
   GroupMat m[GROUP_MAX];
 };
 cudaError_t launch_linear_group(GroupParams p, bool f32_out, int sm_count, cudaStream_t stream, uint32_t* attr_done);
+bool group_xres_fits(int T2, int out_n);   // the activation-resident variant's shared-memory budget for K = 256 T2
 
 // CTA-pair (tcgen05 cta_group::2) many-token kernel: tiles of 256 weight rows x 256 tokens (sdq_linear_pair.cu).
 // `attr_mask` is the calling device's record of which instantiations already carry their shared-memory attribute.

@@ -31,6 +31,7 @@
 // Every wait is bounded; a timeout sets the sticky flag.
 #include <cuda_bf16.h>
 
+#include "sdq_codec.cuh"
 #include "sdq_internal.h"
 #include "sdq_layout.h"
 #include "sdq_linear.h"
@@ -47,6 +48,13 @@ constexpr uint32_t GRP_TM_C = 168;               // per ring position 40: A_out 
 constexpr uint32_t GRP_TM_C_COLS = 40;
 constexpr uint32_t GRP_TMEM_COLS = 512;
 constexpr int GRP_BAR_BYTES = (4 * GRP_MAX_UNITS + 4 + 2) * 8 + 8;
+// activation-resident variant (16 tokens): per 256-K unit the tokens' 4-bit codes, their scale atom and the 8-bit codes of the
+// unit's two 128-K stages, in the operand layouts of the quantizer's buffer; then one atom of token scales for the outlier
+// product; then the quantizing warps' per-token maxima and the tokens' fp32 scales (int8 outliers)
+constexpr uint32_t GRP_XU = 16 * 128 + SF_ATOM_BYTES + 2 * 16 * 128;   // 6656
+constexpr int GRP_XQ_WARPS = 22;                                       // every warp but the two producers quantizes
+constexpr int GRP_X_TAIL = SF_ATOM_BYTES + GRP_XQ_WARPS * 8 * 4 + 16 * 4 + 64;
+__host__ __device__ inline int group_xres_bytes(int T2) { return T2 * (int)GRP_XU + GRP_X_TAIL; }
 
 // inlier slot: | WI record | 4-bit codes of the tokens | their scale atom |
 __host__ __device__ inline int group_is_bytes(int n_tile) { return WI_BYTES + n_tile * 128 + SF_ATOM_BYTES; }
@@ -62,7 +70,7 @@ __device__ __forceinline__ int group_mat_of(const GroupParams& p, int item) {
   return i;
 }
 
-template <bool F32_OUT>
+template <bool F32_OUT, bool XRES>
 __global__ void __launch_bounds__(GRP_THREADS, 1)
 sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
 {
@@ -70,9 +78,16 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint8_t* sm = smem_raw + ((128 - (ptx::smem_u32(smem_raw) & 127)) & 127);
   const uint32_t NU = (uint32_t)p.nslot;                                     // units in the ring
-  const uint32_t xb = (uint32_t)p.n_tile * 128u, isb = (uint32_t)group_is_bytes(p.n_tile), osb = p.out_n ? (uint32_t)group_os_bytes(p.n_tile) : 0u;
+  // (activation-resident variant: the slots hold the weight records only)
+  const uint32_t xb = (uint32_t)p.n_tile * 128u, isb = XRES ? (uint32_t)WI_BYTES : (uint32_t)group_is_bytes(p.n_tile);
+  const uint32_t osb = p.out_n ? (XRES ? 2u * (uint32_t)wc_bytes(1) : (uint32_t)group_os_bytes(p.n_tile)) : 0u;
   const uint32_t ub = isb + osb;                                             // bytes of a unit: inlier slot, then outlier slot
-  uint8_t* sfbuf = sm + NU * ub;                                             // 2 x (SFA_out | SFB_out) of the item, alternating
+  uint8_t* xres = sm + NU * ub;                                              // XRES: the quantized activations of all K
+  const uint32_t xres_main = XRES ? (uint32_t)p.m[0].T2 * GRP_XU : 0u;
+  uint8_t* x_sfb = xres + xres_main;                                         // XRES: token-scale atom of the outlier product
+  float* x_part = reinterpret_cast<float*>(x_sfb + SF_ATOM_BYTES);           // XRES: [quantizing warp][token of its group] maxima
+  float* x_sx = x_part + GRP_XQ_WARPS * 8;                                   // XRES: the tokens' fp32 scales (int8 outliers)
+  uint8_t* sfbuf = xres + (XRES ? (uint32_t)group_xres_bytes(p.m[0].T2) : 0u);   // 2 x (SFA_out | SFB_out) of the item, alternating
   uint64_t* full_is = reinterpret_cast<uint64_t*>(sfbuf + (p.out_n ? GRP_SIDE_BYTES : 0));  // inlier slot of ring position v has landed
   uint64_t* full_os = full_is + GRP_MAX_UNITS;                               // outlier slot of ring position v has landed
   uint64_t* done = full_os + GRP_MAX_UNITS;                                  // the MMAs of the unit at ring position v have completed
@@ -100,6 +115,86 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
   const uint32_t tmem = *tmem_slot;
   const int first = (int)blockIdx.x, stride = (int)gridDim.x;
 
+  if (XRES && warp != 0 && warp != 10) {
+    // ---------------- activation-resident variant: every warp but the producers quantizes the shared X (up to 16 tokens x K)
+    // into this CTA's shared memory, in the operand layouts and with the arithmetic of sdq_quantize_act (Section 5, Stage 3:
+    // A_i as E2M1 with one scale per 64 K, A_o as E4M3 or int8 per token), while the producers already stream the first
+    // weights.  A warp takes a group of 8 tokens and every 11th Q-Vector, 4 lanes per token as in the quantizer; X is read
+    // twice (L2): once for the tokens' maxima, once to encode.
+    ptx::griddep_wait();                         // X comes from an earlier kernel
+    const uint32_t qw = warp - (warp > 10 ? 2u : 1u);      // 0..21
+    const uint32_t tg = qw & 1u, t = lane >> 2, l = lane & 3;
+    const uint32_t mtok = tg * 8 + t;
+    const bool live = (int)mtok < p.x_M;
+    const __nv_bfloat16* xrow = reinterpret_cast<const __nv_bfloat16*>(p.x_bf16) + (int64_t)mtok * p.x_ld;
+    const int NB = p.m[0].T2 * 4;                // Q-Vectors of 64 per token
+    uint32_t m2 = 0;
+    for (int b = (int)(qw >> 1); b < NB; b += GRP_XQ_WARPS / 2) {
+      if (live) {
+        const uint4* src = reinterpret_cast<const uint4*>(xrow + (int64_t)b * 64 + l * 16);
+        const uint4 r0 = __ldg(src), r1 = __ldg(src + 1);
+        const uint32_t r[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+        uint32_t q = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) q = __vmaxu2(q, r[j] & 0x7FFF7FFFu);
+        m2 = max(m2, min(max(q & 0xFFFFu, q >> 16), 0x7F7Fu));     // (+-Inf counts as the largest finite bf16)
+      }
+    }
+    float amax = __uint_as_float(m2 << 16);
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+    if (l == 0) x_part[qw * 8 + t] = amax;
+    ptx::named_bar_sync(6, GRP_XQ_WARPS * 32);
+    float ramax = 0.0f;
+    for (uint32_t q2 = 0; q2 < GRP_XQ_WARPS / 2; ++q2) ramax = fmaxf(ramax, x_part[(2 * q2 + tg) * 8 + t]);
+    const int e = fp8_scale_exp(ramax);
+    const float s8 = pow2_neg(e), sx = int8_scale(ramax);
+    const bool i8 = p.out_i8 != 0;
+    if (qw < 2 && l == 0) {
+      x_sx[mtok] = sx;
+      *reinterpret_cast<uint32_t*>(x_sfb + sf_off(mtok, 0)) = (uint32_t)((i8 || !live) ? 127 : e + 127) * 0x01010101u;
+    }
+    for (int b = (int)(qw >> 1); b < NB; b += GRP_XQ_WARPS / 2) {
+      uint4 r0 = make_uint4(0, 0, 0, 0), r1 = r0;
+      if (live) {
+        const uint4* src = reinterpret_cast<const uint4*>(xrow + (int64_t)b * 64 + l * 16);
+        r0 = __ldg(src); r1 = __ldg(src + 1);
+      }
+      const uint32_t r[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+      float v[16];
+      uint32_t qm = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        v[2 * j] = __uint_as_float(r[j] << 16);
+        v[2 * j + 1] = __uint_as_float(r[j] & 0xFFFF0000u);
+        qm = __vmaxu2(qm, r[j] & 0x7FFF7FFFu);
+      }
+      qm = max(qm & 0xFFFFu, qm >> 16);
+      if (qm > 0x7F7Fu) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = sat(v[j]);
+      }
+      uint32_t bm = min(qm, 0x7F7Fu);
+      bm = max(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
+      bm = max(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
+      const uint32_t c = e8m0_scale_code(__uint_as_float(bm << 16), p.scale_rule);
+      const float s4 = pow2_inv_e8m0(c);
+      uint32_t q4[2] = {0, 0}, q8[4] = {0, 0, 0, 0};
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        q4[j >> 2] |= e2m1x2(v[2 * j] * s4, v[2 * j + 1] * s4) << (8 * (j & 3));
+        q8[j >> 1] |= (i8 ? (int8_code(v[2 * j], sx) | (int8_code(v[2 * j + 1], sx) << 8)) : e4m3x2(v[2 * j] * s8, v[2 * j + 1] * s8)) << (16 * (j & 1));
+      }
+      const uint32_t k = (uint32_t)b * 64 + l * 16;          // first element of this lane
+      uint8_t* xu = xres + (size_t)(k >> 8) * GRP_XU;
+      *reinterpret_cast<uint2*>(xu + b_off(mtok, (k & 255) >> 1)) = make_uint2(q4[0], q4[1]);
+      *reinterpret_cast<uint4*>(xu + 16 * 128 + SF_ATOM_BYTES + ((k >> 7) & 1) * 16 * 128 + b_off(mtok, k & 127)) = make_uint4(q8[0], q8[1], q8[2], q8[3]);
+      if (l == 0) xu[16 * 128 + in_sf_off(false, mtok, (uint32_t)(b & 3))] = (uint8_t)c;
+    }
+    ptx::fence_proxy_async();                    // generic-proxy writes -> visible to the tensor core's operand reads
+    ptx::named_bar_sync(6, GRP_XQ_WARPS * 32);
+  }
+
   if (warp == 0 || warp == 10) {
     // ---------------- producers: warp 0 fills the inlier slots, warp 10 the outlier slots.  Six lanes each, in lockstep: lane
     // 2 c + l issues copy c (of three) of the units u = l, l + 2, ... of this CTA's sequence (NU is even, so a lane's ring
@@ -107,8 +202,10 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
     // each of the six lanes instead of one thread issuing six in a row.
     const bool outl = warp == 10;
     const uint32_t l = lane & 1, c = lane >> 1;
-    if (c < 3 && (!outl || p.out_n)) {
-      ptx::griddep_wait();                       // activations come from an earlier kernel
+    // (activation-resident variant: one copy per inlier slot; per outlier slot the compact records, and lane c = 1 the row-scale
+    // atom of each item)
+    if (c < (XRES ? (outl ? 2u : 1u) : 3u) && (!outl || p.out_n)) {
+      if (!XRES) ptx::griddep_wait();            // activations come from an earlier kernel
       bool ok = true;
       int item = first, k2 = (int)l;             // this lane's position: work item and 256-K unit inside the item
       int mat = -1, rt = 0, T2 = 0;
@@ -126,7 +223,20 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
         const GroupMat& m = p.m[mat];
         if (wrapped && !(ok = ptx::mbar_wait(&done[v], ph ^ 1))) break;
         uint8_t* st = sm + (size_t)v * ub + (outl ? isb : 0u);
-        if (!outl) {
+        if (XRES) {
+          if (!outl) {
+            ptx::mbar_expect_tx(&full_is[v], WI_BYTES);
+            ptx::bulk_g2s(st, m.w + m.wi + ((size_t)rt * m.T2 + k2) * WI_BYTES, WI_BYTES, &full_is[v]);
+          } else if (c == 0) {
+            ptx::mbar_expect_tx(&full_os[v], wcb);
+            ptx::bulk_g2s(st, m.w + m.wc + ((size_t)rt * 2 * m.T2 + 2 * k2) * (size_t)wc_bytes(1), wcb, &full_os[v]);
+          } else if (k2 == 0 && !p.out_i8) {     // the item's row-scale atom (see below); the tokens' atom is resident
+            const uint32_t sb = iseq & 1;
+            if (iseq >= 2 && !(ok = ptx::mbar_wait(&acc_full[sb], ((iseq >> 1) - 1) & 1))) break;
+            ptx::mbar_expect_tx(&sf_full[sb], SF_ATOM_BYTES);
+            ptx::bulk_g2s(sfbuf + sb * 2 * SF_ATOM_BYTES, m.w + m.sfa_out + (size_t)rt * SF_ATOM_BYTES, SF_ATOM_BYTES, &sf_full[sb]);
+          }
+        } else if (!outl) {
           const uint8_t* xi = m.x + m.xi + (size_t)k2 * XI_BYTES;
           if (c == 0) ptx::mbar_expect_tx(&full_is[v], WI_BYTES + xb + SF_ATOM_BYTES);
           const uint8_t* src = c == 0 ? m.w + m.wi + ((size_t)rt * m.T2 + k2) * WI_BYTES : (c == 1 ? xi : xi + B4_BYTES);
@@ -206,25 +316,28 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
             for (int i = 0; i < n; ++i) {
               const int kk = k2 + i;
               const uint32_t sb = smb + vv * ub;
+              // the tokens' operands of unit kk: in the slot behind the weight records, or resident
+              const uint32_t xu = ptx::smem_u32(xres) + (uint32_t)kk * GRP_XU;
+              const uint32_t b4 = XRES ? xu : sb + WI_BYTES, sf4 = XRES ? xu + 16 * 128 : sb + WI_BYTES + xb;
               if (!outw) {
                 const uint32_t mb = tmem + GRP_TM_I + 12u * (uint32_t)(kk & 1);
                 ptx::tc_cp_128x128b(mb, ptx::smem_desc(sb + A_IN_BYTES, 0, 128));
                 ptx::tc_cp_32x128b_warpx4(mb + 4, ptx::smem_desc(sb + A_IN_BYTES + E_IN_BYTES, 0, 128));
-                ptx::tc_cp_32x128b_warpx4(mb + 8, ptx::smem_desc(sb + WI_BYTES + xb, 0, 128));
-                ptx::mma_sp_mxf4(acc_col, ptx::smem_desc(sb, 128, 256), ptx::smem_desc(sb + WI_BYTES, 128, 1024), id4[0], mb, mb + 4, mb + 8,
+                ptx::tc_cp_32x128b_warpx4(mb + 8, ptx::smem_desc(sf4, 0, 128));
+                ptx::mma_sp_mxf4(acc_col, ptx::smem_desc(sb, 128, 256), ptx::smem_desc(b4, 128, 1024), id4[0], mb, mb + 4, mb + 8,
                                  kk ? 1u : 0u);
-                ptx::mma_sp_mxf4(acc_col, ptx::smem_desc(sb + 4096, 128, 256), ptx::smem_desc(sb + WI_BYTES + 512, 128, 1024), id4[1], mb + 2,
+                ptx::mma_sp_mxf4(acc_col, ptx::smem_desc(sb + 4096, 128, 256), ptx::smem_desc(b4 + 512, 128, 1024), id4[1], mb + 2,
                                  mb + 4, mb + 8, 1u);
               } else {
                 if (kk == 0 && !p.out_i8) {
                   const uint32_t sf = ptx::smem_u32(sfbuf) + ab * 2 * SF_ATOM_BYTES;
                   ptx::tc_cp_32x128b_warpx4(so, ptx::smem_desc(sf, 0, 128));
-                  ptx::tc_cp_32x128b_warpx4(so + 4, ptx::smem_desc(sf + SF_ATOM_BYTES, 0, 128));
+                  ptx::tc_cp_32x128b_warpx4(so + 4, ptx::smem_desc(XRES ? ptx::smem_u32(x_sfb) : sf + SF_ATOM_BYTES, 0, 128));
                 }
 #pragma unroll
                 for (uint32_t h = 0; h < 2; ++h) {
                   const uint32_t ca = tmem + GRP_TM_C + GRP_TM_C_COLS * vv + 16u * h, eb = tmem + GRP_TM_C + GRP_TM_C_COLS * vv + 32u + 4u * h;
-                  const uint32_t xa = sb + isb + wcb + h * xb;
+                  const uint32_t xa = XRES ? xu + 16 * 128 + SF_ATOM_BYTES + h * 16 * 128 : sb + isb + wcb + h * xb;
                   if (p.out_i8) {     // the same containers and token codes as integers, int32 accumulator
                     ptx::mma_sp_i8_ta(acc_col, ca, ptx::smem_desc(xa, 128, 1024), id8, eb, (kk | (int)h) ? 1u : 0u);
                     ptx::mma_sp_i8_ta(acc_col, ca + 8, ptx::smem_desc(xa + 512, 128, 1024), id8, eb + 2, 1u);
@@ -281,7 +394,7 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
               float o = 0.0f;
-              if (p.out_i8) { if ((int)(c + i) < m.M) o = (float)(int)b[i] * (sw * __ldg(sxp + c + i)); }
+              if (p.out_i8) { if ((int)(c + i) < m.M) o = (float)(int)b[i] * (sw * (XRES ? x_sx[c + i] : __ldg(sxp + c + i))); }
               else if (p.out_n) o = __uint_as_float(b[i]);
               val[c + i] = p.out_n ? __float_as_uint(__uint_as_float(a[i]) + o) : a[i];
             }
@@ -372,22 +485,33 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
 }
 
 // units the ring holds for `n_tile` tokens per tile: as many as fit (an even number)
-static int group_units(int n_tile, int out_n) {
-  const int avail = 232448 - 128 - (out_n ? GRP_SIDE_BYTES : 0) - GRP_BAR_BYTES;
-  int n = avail / (group_is_bytes(n_tile) + (out_n ? group_os_bytes(n_tile) : 0));
+static int group_units(int n_tile, int out_n, int xres_bytes, int unit_bytes) {
+  const int avail = 232448 - 128 - (out_n ? GRP_SIDE_BYTES : 0) - GRP_BAR_BYTES - xres_bytes;
+  int n = avail / unit_bytes;
   n &= ~1;
   return n > GRP_MAX_UNITS ? GRP_MAX_UNITS : n;
 }
 
+// shared-memory budget of the activation-resident variant: does a ring of at least six units fit beside X of K / 256 = T2 units?
+bool group_xres_fits(int T2, int out_n) {
+  const int unit = WI_BYTES + (out_n ? 2 * wc_bytes(1) : 0);
+  return group_units(16, out_n, group_xres_bytes(T2), unit) >= 6;
+}
+
 cudaError_t launch_linear_group(GroupParams p, bool f32_out, int sm_count, cudaStream_t stream, uint32_t* attr_done)
 {
-  p.nslot = group_units(p.n_tile, p.out_n);
-  p.slot_bytes = group_is_bytes(p.n_tile) + (p.out_n ? group_os_bytes(p.n_tile) : 0);
-  const int smem = p.nslot * p.slot_bytes + (p.out_n ? GRP_SIDE_BYTES : 0) + GRP_BAR_BYTES + 128;
+  const bool xres = p.x_bf16 != nullptr;
+  const int xbytes = xres ? group_xres_bytes(p.m[0].T2) : 0;
+  p.slot_bytes = xres ? WI_BYTES + (p.out_n ? 2 * wc_bytes(1) : 0) : group_is_bytes(p.n_tile) + (p.out_n ? group_os_bytes(p.n_tile) : 0);
+  p.nslot = group_units(p.n_tile, p.out_n, xbytes, p.slot_bytes);
+  const int smem = p.nslot * p.slot_bytes + xbytes + (p.out_n ? GRP_SIDE_BYTES : 0) + GRP_BAR_BYTES + 128;
   if (!*attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(sdq_linear_group_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(sdq_linear_group_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
-    if (e != cudaSuccess) return e;
+    const cudaFuncAttribute a = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    if (cudaFuncSetAttribute(sdq_linear_group_kernel<false, false>, a, 232448) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_group_kernel<true, false>, a, 232448) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_group_kernel<false, true>, a, 232448) != cudaSuccess ||
+        cudaFuncSetAttribute(sdq_linear_group_kernel<true, true>, a, 232448) != cudaSuccess)
+      return cudaErrorUnknown;
     *attr_done = 1;
   }
   cudaLaunchConfig_t lc = {};
@@ -400,7 +524,8 @@ cudaError_t launch_linear_group(GroupParams p, bool f32_out, int sm_count, cudaS
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = attr;
   lc.numAttrs = 1;
-  return f32_out ? cudaLaunchKernelEx(&lc, sdq_linear_group_kernel<true>, p) : cudaLaunchKernelEx(&lc, sdq_linear_group_kernel<false>, p);
+  if (xres) return f32_out ? cudaLaunchKernelEx(&lc, sdq_linear_group_kernel<true, true>, p) : cudaLaunchKernelEx(&lc, sdq_linear_group_kernel<false, true>, p);
+  return f32_out ? cudaLaunchKernelEx(&lc, sdq_linear_group_kernel<true, false>, p) : cudaLaunchKernelEx(&lc, sdq_linear_group_kernel<false, false>, p);
 }
 
 }  // namespace sdq

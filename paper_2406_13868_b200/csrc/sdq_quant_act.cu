@@ -30,9 +30,6 @@ __device__ __forceinline__ void load16(const __nv_bfloat16* p, float (&x)[16]) {
     x[2 * i + 1] = __uint_as_float(r[i] & 0xFFFF0000u);
   }
 }
-// |x| with +-Inf replaced by the largest finite bf16 (saturation)
-__device__ __forceinline__ float sat_abs(float x) { return fminf(fabsf(x), 3.3895313892515355e38f); }
-__device__ __forceinline__ float sat(float x) { return copysignf(sat_abs(x), x); }
 
 // partial[m][chunk] = max |x| of token m over its 1024-K chunk
 __global__ void __launch_bounds__(QA_THREADS)

@@ -388,3 +388,61 @@ def test_int8_outliers_outside_the_grouped_kernel_are_refused():
     # the blob header carries the format
     q = m.packed_attach(big.buf.clone())
     assert q.cfg.out_fmt == so.OUT_INT8
+
+
+# ---------------------------------------------------------------------------------------------------------------------
+# the activation quantizer fused into the grouped kernel (Section 5, Stage 3 in the linear layers' load path)
+
+@pytest.mark.parametrize("shapes,M,cfg_args", [
+    ([(4096, 4096)] * 3, 1, (1, so.GRAN_PAIR, 64, 0)),                       # q / k / v, one token
+    ([(4096, 4096)] * 3, 16, (1, so.GRAN_PAIR, 64, 0)),
+    ([(11008, 4096)] * 2, 7, (1, so.GRAN_PAIR, 64, 1)),                      # gate / up, the ceil scale rule
+    ([(4096, 1024), (2048, 1024), (4096, 1024)], 5, (0, so.GRAN_PAIR, 64, 0)),   # no outlier part, the shortest K
+    ([(4096, 2048)] * 4, 13, I8_ARGS),                                       # int8 outlier operands
+])
+def test_fused_quantizer_group_call_equals_quantize_then_group(shapes, M, cfg_args):
+    m = sdq()
+    cfg = m.Config(*cfg_args)
+    K = shapes[0][1]
+    Ws = [sdq_synth.make_weight(N, K, 5100 + i) for i, (N, _) in enumerate(shapes)]
+    X = sdq_synth.make_act(M, K, 5150)
+    X[0, 5] = float("inf")                                                   # saturates like the stand-alone quantizer
+    if M > 2:
+        X[2] = 0                                                             # an all-zero token
+    ps = [m.sdq_decompose(W.cuda(), cfg) for W in Ws]
+    Xd = X.cuda()
+    xq = m.sdq_quantize_act(Xd, cfg)
+    ref32 = m.sdq_linear_group([xq] * len(ps), ps, f32=True)
+    ref16 = m.sdq_linear_group([xq] * len(ps), ps)
+    y32 = m.sdq_linear_group_x(Xd, ps, f32=True)
+    y16 = m.sdq_linear_group_x(Xd, ps)
+    assert m.device_status() == 0
+    for a, b, c, d in zip(y32, ref32, y16, ref16):
+        assert torch.equal(a, b) and torch.equal(c, d)                       # the same codes, scales and summation order
+    # and against the oracle directly (first layer, sampled rows)
+    oc = so.Config(*cfg_args)
+    op, oq = so.decompose(sdq_synth.bf16_bits(Ws[0]), oc), so.quantize_act(sdq_synth.bf16_bits(X), oc)
+    yref = so.linear(oq, op, 0, 256)
+    dd, tol = y_close(y32[0][:, :256].cpu().numpy(), yref)
+    assert (dd <= tol).all()
+    # a strided X (a slice of a wider buffer)
+    wide = torch.zeros((M, K + 64), dtype=torch.bfloat16, device="cuda")
+    wide[:, :K] = Xd
+    y_s = m.sdq_linear_group_x(wide[:, :K], ps)
+    assert all(torch.equal(a, b) for a, b in zip(y_s, ref16))
+
+
+def test_fused_quantizer_group_call_outside_its_range_is_refused():
+    m = sdq()
+    cfg = m.Config(1, so.GRAN_PAIR, 64, 0)
+    ps = [m.sdq_decompose(sdq_synth.make_weight(4096, 1024, 1).cuda(), cfg)] * 3
+    with pytest.raises(RuntimeError):
+        m.sdq_linear_group_x(sdq_synth.make_act(17, 1024, 1).cuda(), ps)                 # more than 16 tokens
+    p_long = [m.sdq_decompose(sdq_synth.make_weight(4096, 11008, 1).cuda(), cfg)] * 3
+    with pytest.raises(RuntimeError):
+        m.sdq_linear_group_x(sdq_synth.make_act(4, 11008, 1).cuda(), p_long)             # X does not fit beside the ring
+    with pytest.raises(RuntimeError):
+        m.sdq_linear_group_x(sdq_synth.make_act(4, 1024, 1).cuda(), ps[:1])              # too few row tiles
+    with pytest.raises(RuntimeError):
+        m.sdq_linear_group_x(sdq_synth.make_act(4, 2048, 1).cuda(), ps)                  # K of X and of the weights differ
+    assert m.device_status() == 0
