@@ -978,7 +978,8 @@ static sdq_status_t launch_group_x(int n, const void* X, int64_t M, int64_t K, i
       return SDQ_ERR_UNSUPPORTED;
     items += w->N / TILE_ROWS;
   }
-  if (n > GROUP_MAX || M > 16 || K < 4 * K2 || !group_xres_fits((int)(K / K2), P[0]->cfg.out_n) || items * 2 < dinfo->sm_count || items >= (1 << 30))
+  // (the in-kernel quantizer keeps a token's K <= 4096 elements in the registers of its 11 x 4 lanes)
+  if (n > GROUP_MAX || M > 16 || K < 4 * K2 || K > 16 * K2 || !group_xres_fits((int)(K / K2), P[0]->cfg.out_n) || items * 2 < dinfo->sm_count || items >= (1 << 30))
     return SDQ_ERR_UNSUPPORTED;
   GroupParams g;
   g.n = n;

@@ -119,8 +119,7 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
     // ---------------- activation-resident variant: every warp but the producers quantizes the shared X (up to 16 tokens x K)
     // into this CTA's shared memory, in the operand layouts and with the arithmetic of sdq_quantize_act (Section 5, Stage 3:
     // A_i as E2M1 with one scale per 64 K, A_o as E4M3 or int8 per token), while the producers already stream the first
-    // weights.  A warp takes a group of 8 tokens and every 11th Q-Vector, 4 lanes per token as in the quantizer; X is read
-    // twice (L2): once for the tokens' maxima, once to encode.
+    // weights.  A warp takes a group of 8 tokens and every 11th Q-Vector, 4 lanes per token as in the quantizer.
     ptx::griddep_wait();                         // X comes from an earlier kernel
     const uint32_t qw = warp - (warp > 10 ? 2u : 1u);      // 0..21
     const uint32_t tg = qw & 1u, t = lane >> 2, l = lane & 3;
@@ -128,17 +127,30 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
     const bool live = (int)mtok < p.x_M;
     const __nv_bfloat16* xrow = reinterpret_cast<const __nv_bfloat16*>(p.x_bf16) + (int64_t)mtok * p.x_ld;
     const int NB = p.m[0].T2 * 4;                // Q-Vectors of 64 per token
+    // one read of X: a lane keeps its (up to six) 16-element pieces in registers across the maxima's barrier
+    constexpr int XT = 6;                        // Q-Vectors per warp: K <= 4096 -> 64 / 11
+    uint4 raw[XT][2];
+    uint32_t qmax[XT];
     uint32_t m2 = 0;
-    for (int b = (int)(qw >> 1); b < NB; b += GRP_XQ_WARPS / 2) {
-      if (live) {
-        const uint4* src = reinterpret_cast<const uint4*>(xrow + (int64_t)b * 64 + l * 16);
-        const uint4 r0 = __ldg(src), r1 = __ldg(src + 1);
-        const uint32_t r[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
-        uint32_t q = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) q = __vmaxu2(q, r[j] & 0x7FFF7FFFu);
-        m2 = max(m2, min(max(q & 0xFFFFu, q >> 16), 0x7F7Fu));     // (+-Inf counts as the largest finite bf16)
+    for (int i = 0; i < XT; ++i) {
+      const int b = (int)(qw >> 1) + i * (GRP_XQ_WARPS / 2);
+      raw[i][0] = raw[i][1] = make_uint4(0, 0, 0, 0);
+      if (live && b < NB) {
+        const uint4* src = reinterpret_cast<const uint4*>(xrow + (int64_t)b * 64 + l * 16);
+        raw[i][0] = __ldg(src);
+        raw[i][1] = __ldg(src + 1);
       }
+    }
+#pragma unroll
+    for (int i = 0; i < XT; ++i) {
+      const uint32_t r[8] = {raw[i][0].x, raw[i][0].y, raw[i][0].z, raw[i][0].w, raw[i][1].x, raw[i][1].y, raw[i][1].z, raw[i][1].w};
+      uint32_t q = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) q = __vmaxu2(q, r[j] & 0x7FFF7FFFu);
+      q = max(q & 0xFFFFu, q >> 16);             // > 0x7F7F: the lane holds an infinity (counts as the largest finite bf16)
+      qmax[i] = q;
+      m2 = max(m2, min(q, 0x7F7Fu));
     }
     float amax = __uint_as_float(m2 << 16);
     amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
@@ -154,27 +166,22 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
       x_sx[mtok] = sx;
       *reinterpret_cast<uint32_t*>(x_sfb + sf_off(mtok, 0)) = (uint32_t)((i8 || !live) ? 127 : e + 127) * 0x01010101u;
     }
-    for (int b = (int)(qw >> 1); b < NB; b += GRP_XQ_WARPS / 2) {
-      uint4 r0 = make_uint4(0, 0, 0, 0), r1 = r0;
-      if (live) {
-        const uint4* src = reinterpret_cast<const uint4*>(xrow + (int64_t)b * 64 + l * 16);
-        r0 = __ldg(src); r1 = __ldg(src + 1);
-      }
-      const uint32_t r[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+#pragma unroll
+    for (int i = 0; i < XT; ++i) {
+      const int b = (int)(qw >> 1) + i * (GRP_XQ_WARPS / 2);     // uniform over the warp
+      if (b >= NB) break;
+      const uint32_t r[8] = {raw[i][0].x, raw[i][0].y, raw[i][0].z, raw[i][0].w, raw[i][1].x, raw[i][1].y, raw[i][1].z, raw[i][1].w};
       float v[16];
-      uint32_t qm = 0;
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         v[2 * j] = __uint_as_float(r[j] << 16);
         v[2 * j + 1] = __uint_as_float(r[j] & 0xFFFF0000u);
-        qm = __vmaxu2(qm, r[j] & 0x7FFF7FFFu);
       }
-      qm = max(qm & 0xFFFFu, qm >> 16);
-      if (qm > 0x7F7Fu) {
+      if (qmax[i] > 0x7F7Fu) {
 #pragma unroll
         for (int j = 0; j < 16; ++j) v[j] = sat(v[j]);
       }
-      uint32_t bm = min(qm, 0x7F7Fu);
+      uint32_t bm = min(qmax[i], 0x7F7Fu);
       bm = max(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
       bm = max(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
       const uint32_t c = e8m0_scale_code(__uint_as_float(bm << 16), p.scale_rule);
