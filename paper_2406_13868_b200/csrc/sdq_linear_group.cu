@@ -399,11 +399,13 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
             if (p.out_n) ptx::tmem_ld_32x32b_x16(tb + 32 + c, b);
             ptx::tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              float o = 0.0f;
-              if (p.out_i8) { if ((int)(c + i) < m.M) o = (float)(int)b[i] * (sw * (XRES ? x_sx[c + i] : __ldg(sxp + c + i))); }
-              else if (p.out_n) o = __uint_as_float(b[i]);
-              val[c + i] = p.out_n ? __float_as_uint(__uint_as_float(a[i]) + o) : a[i];
+            for (int i = 0; i < 16; ++i) val[c + i] = p.out_n ? __float_as_uint(__uint_as_float(a[i]) + __uint_as_float(b[i])) : a[i];
+            if (p.out_i8) {      // b holds exact int32 sums: scale them, tokens that exist only
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const float o = (int)(c + i) < m.M ? (float)(int)b[i] * (sw * (XRES ? x_sx[c + i] : __ldg(sxp + c + i))) : 0.0f;
+                val[c + i] = __float_as_uint(__uint_as_float(a[i]) + o);
+              }
             }
           } else {
 #pragma unroll
