@@ -10,7 +10,7 @@
 //
 // The outlier part is streamed in the form the method states it -- an 8-bit code and a position per S-Vector (the WC
 // section, 1.5 bits per weight) -- not as the 2:4 FP8 container of the many-token kernels (5 bits per weight): sixteen
-// warps rebuild the containers of each 256-K unit (one weight row of one 128-K stage per thread) and write them with
+// warps in groups of four rebuild the containers of each 256-K unit (one weight row per thread) and write them with
 // tcgen05.st into tensor memory, from where the outlier MMAs take their A operand and their metadata, while the tensor
 // core works on earlier units.  Shared memory carries every streamed byte once in (bulk copy) and once out (operand
 // read); an earlier version that rebuilt the containers in shared memory moved 86 KB per unit through it, two thirds of
@@ -27,7 +27,7 @@
 // Warps: 0 and 10 bulk-copy producers (inlier / outlier slots, six lanes each), 1 and 23 MMA issuers (inlier / outlier
 // product, each into its own accumulator; warp-uniform loops, one elected lane issues; they also copy the inlier metadata
 // and the scales to TMEM), 2..5 epilogue (adds the two accumulators; accumulator pairs alternate per item, so the next
-// item's MMAs never wait for the stores), 6..9, 11..14 and 15..22 container builders (two groups).
+// item's MMAs never wait for the stores), 6..9, 11..14, 15..18 and 19..22 container builders (up to four groups).
 // Every wait is bounded; a timeout sets the sticky flag.
 #include <cuda_bf16.h>
 
@@ -103,7 +103,7 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
     *timed_out = 0u;
     const uint32_t issuers = p.out_n ? 2u : 1u;   // MMA-issuing warps: both commit to `done` and `acc_full`
     for (uint32_t v = 0; v < NU; ++v) {
-      ptx::mbar_init(&full_is[v], 1); ptx::mbar_init(&full_os[v], 1); ptx::mbar_init(&done[v], issuers); ptx::mbar_init(&built[v], 8);
+      ptx::mbar_init(&full_is[v], 1); ptx::mbar_init(&full_os[v], 1); ptx::mbar_init(&done[v], issuers); ptx::mbar_init(&built[v], 4);
     }
     for (int a = 0; a < 2; ++a) { ptx::mbar_init(&acc_full[a], issuers); ptx::mbar_init(&acc_empty[a], 4); ptx::mbar_init(&sf_full[a], 1); }
     ptx::fence_barrier_init();
@@ -156,7 +156,7 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
     amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
     amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
     if (l == 0) x_part[qw * 8 + t] = amax;
-    ptx::named_bar_sync(6, GRP_XQ_WARPS * 32);
+    ptx::named_bar_sync(8, GRP_XQ_WARPS * 32);
     float ramax = 0.0f;
     for (uint32_t q2 = 0; q2 < GRP_XQ_WARPS / 2; ++q2) ramax = fmaxf(ramax, x_part[(2 * q2 + tg) * 8 + t]);
     const int e = fp8_scale_exp(ramax);
@@ -199,7 +199,7 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
       if (l == 0) xu[16 * 128 + in_sf_off(false, mtok, (uint32_t)(b & 3))] = (uint8_t)c;
     }
     ptx::fence_proxy_async();                    // generic-proxy writes -> visible to the tensor core's operand reads
-    ptx::named_bar_sync(6, GRP_XQ_WARPS * 32);
+    ptx::named_bar_sync(8, GRP_XQ_WARPS * 32);
   }
 
   if (warp == 0 || warp == 10) {
@@ -427,62 +427,66 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
     }
     if (!ok && lane == 0) atomicOr(&p.flags[FLAG_TIMEOUT], 1u);
   } else if (p.out_n && warp >= 6 && warp <= 22) {
-    // ---------------- outlier container builders: two groups of eight warps; group g (warps 6..9 + 11..14, or 15..22)
-    // rebuilds the containers of the units u = g, g + 2, ... -- straight into tensor memory, where the outlier MMAs read their
-    // A operand and metadata: shared memory is written once (by the bulk copies) and never again.  Inside a group the first
-    // four warps take the unit's first 128-K stage and the other four the second; a warp can reach the 32 TMEM lanes
-    // 32 (warp % 4) .., so its thread `lane` rebuilds weight row 32 (warp % 4) + lane of its stage from 16 codes + 16 positions:
-    // per S-Vector of 8 the code goes to the 2:4 slot of its group of 4 (two ascending slot indices per 4: (p, 3) with the
-    // value first, or (0, 3) with the value second when p = 3; a group without outlier gets (0, 1) and zeros), the form
-    // the packer writes for the many-token kernels.  A row's 64 stored bytes are 16 columns of its lane, its 16 metadata
-    // bytes 4 columns.  Two groups, because a trip is mostly latency (the barrier, the dependent load -> permute -> store
-    // chain): they overlap in time.  Container set v is free when the unit's outlier slot has landed at ring position v: the
-    // producer refills a position only after the MMAs of its previous unit have completed.
-    const uint32_t grp = warp >= 15 ? 1u : 0u;
-    const uint32_t h = grp ? (warp >= 19 ? 1u : 0u) : (warp >= 11 ? 1u : 0u);
+    // ---------------- outlier container builders: up to four groups of four warps (6..9, 11..14, 15..18, 19..22); group g
+    // rebuilds the containers of the units u = g, g + G, ... -- straight into tensor memory, where the outlier MMAs read their
+    // A operand and metadata: shared memory is written once (by the bulk copies) and never again.  A warp can reach the 32
+    // TMEM lanes 32 (warp % 4) .., so its thread `lane` rebuilds weight row 32 (warp % 4) + lane, both 128-K stages of the
+    // unit, each from 16 codes + 16 positions: per S-Vector of 8 the code goes to the 2:4 slot of its group of 4 (two
+    // ascending slot indices per 4: (p, 3) with the value first, or (0, 3) with the value second when p = 3; a group without
+    // outlier gets (0, 1) and zeros), the form the packer writes for the many-token kernels.  A row's 64 stored bytes per
+    // stage are 16 columns of its lane, its 16 metadata bytes 4 columns.  Several groups, because a trip is mostly latency
+    // (measured ~1800 cycles, a tenth of it arithmetic): they overlap in time.  G divides the ring, so that every phase of
+    // a slot's barrier is seen by the same group.  Container set v is free when the unit's outlier slot has landed at ring
+    // position v: the producer refills a position only after the MMAs of its previous unit have completed.
+    const uint32_t bw = warp - (warp >= 11 ? 7u : 6u);       // 0..15
+    const uint32_t grp = bw >> 2;
+    const uint32_t G = (NU & 3u) == 0 ? 4u : (NU % 3u == 0 ? 3u : 2u);
     const uint32_t r = (warp & 3) * 32 + lane;
-    const bool poller = grp ? warp == 15 : warp == 6;
+    const bool poller = (bw & 3u) == 0;
     bool ok = true;
-    uint32_t v = 0, ph = 0, u = 0;               // position of the unit in the ring, lap parity, unit count
-    const uint32_t row_off = isb + h * (uint32_t)wc_bytes(1) + r * 16, pos_off = isb + h * (uint32_t)wc_bytes(1) + WC_CODE_BYTES + r * 8;
+    uint32_t v = 0, ph = 0, gu = 0;              // position of the unit in the ring, lap parity, unit count modulo G
     const uint32_t tlane = tmem + (((warp & 3) * 32u) << 16) + GRP_TM_C;
-    for (int item = first; item < p.total_items && ok; item += stride) {
+    for (int item = first; item < p.total_items && ok && grp < G; item += stride) {
       const int T2 = p.m[group_mat_of(p, item)].T2;
-      for (int k2 = 0; k2 < T2; ++k2, ++u) {
-        if ((u & 1) == grp) {
+      for (int k2 = 0; k2 < T2; ++k2) {
+        if (gu == grp) {
           // Only ONE thread of the group waits on the mbarrier and then releases the others through a hardware barrier: with
-          // eight warps waiting on the same mbarrier some of them noticed its completion more than a microsecond late.
+          // every warp waiting on the same mbarrier some of them noticed its completion more than a microsecond late.
           if (poller && lane == 0 && !ptx::mbar_wait(&full_os[v], ph)) *timed_out = 1u;
-          ptx::named_bar_sync(4 + grp, 256);   // (barrier 3 belongs to the epilogue)
+          ptx::named_bar_sync(4 + grp, 128);   // (barrier 3 belongs to the epilogue)
           if (*timed_out) { ok = false; break; }
-          const uint8_t* st = sm + (size_t)v * ub;
-          const uint4 codes = *reinterpret_cast<const uint4*>(st + row_off);
-          const uint2 pos = *reinterpret_cast<const uint2*>(st + pos_off);
-          const uint32_t cw[4] = {codes.x, codes.y, codes.z, codes.w}, pw[2] = {pos.x, pos.y};
-          // position ps (0..7) of the outlier in its S-Vector: it sits in the group of 4 number ps >> 2 at p = ps & 3.  Stored
-          // bytes of the S-Vector (two per group of 4): the code moves to byte (p == 3) + 2 (ps >> 2); metadata byte = the two
-          // groups' slot-index nibbles, (p, 3) or (0, 3) for p = 3 where the outlier is, (0, 1) elsewhere.  Both come from
-          // 8-entry byte tables held in two registers each, and one byte-permute looks up four S-Vectors at a time: the four
-          // position nibbles of a 16-bit piece of the position word are its selector.
-          uint32_t stored[16], meta[4], shw[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint32_t sel = pw[i >> 1] >> (16 * (i & 1));
-            meta[i] = __byte_perm(0x4C4E4D4Cu, 0xC4E4D4C4u, sel);
-            shw[i] = __byte_perm(0x08000000u, 0x18101010u, sel);
-          }
-#pragma unroll
-          for (int g = 0; g < 16; ++g)
-            stored[g] = __byte_perm(cw[g >> 2], 0u, 0x4440u + (uint32_t)(g & 3)) << ((shw[g >> 2] >> (8 * (g & 3))) & 0xFFu);
-          // columns 0..7 of the stage: the row's stored bytes of K-block 0 (the first MMA's A), 8..15: of K-block 1
+          const uint8_t* st = sm + (size_t)v * ub + isb;
           const uint32_t tc = tlane + GRP_TM_C_COLS * v;
-          ptx::tmem_st_32x32b_x16(tc + 16u * h, stored);
-          ptx::tmem_st_32x32b_x4(tc + 32u + 4u * h, meta);
+#pragma unroll
+          for (uint32_t h = 0; h < 2; ++h) {
+            const uint4 codes = *reinterpret_cast<const uint4*>(st + h * (uint32_t)wc_bytes(1) + r * 16);
+            const uint2 pos = *reinterpret_cast<const uint2*>(st + h * (uint32_t)wc_bytes(1) + WC_CODE_BYTES + r * 8);
+            const uint32_t cw[4] = {codes.x, codes.y, codes.z, codes.w}, pw[2] = {pos.x, pos.y};
+            // position ps (0..7) of the outlier in its S-Vector: it sits in the group of 4 number ps >> 2 at p = ps & 3.  Stored
+            // bytes of the S-Vector (two per group of 4): the code moves to byte (p == 3) + 2 (ps >> 2); metadata byte = the two
+            // groups' slot-index nibbles, (p, 3) or (0, 3) for p = 3 where the outlier is, (0, 1) elsewhere.  Both come from
+            // 8-entry byte tables held in two registers each, and one byte-permute looks up four S-Vectors at a time: the four
+            // position nibbles of a 16-bit piece of the position word are its selector.
+            uint32_t stored[16], meta[4], shw[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint32_t sel = pw[i >> 1] >> (16 * (i & 1));
+              meta[i] = __byte_perm(0x4C4E4D4Cu, 0xC4E4D4C4u, sel);
+              shw[i] = __byte_perm(0x08000000u, 0x18101010u, sel);
+            }
+#pragma unroll
+            for (int g = 0; g < 16; ++g)
+              stored[g] = __byte_perm(cw[g >> 2], 0u, 0x4440u + (uint32_t)(g & 3)) << ((shw[g >> 2] >> (8 * (g & 3))) & 0xFFu);
+            // columns 0..7 of the stage: the row's stored bytes of K-block 0 (the first MMA's A), 8..15: of K-block 1
+            ptx::tmem_st_32x32b_x16(tc + 16u * h, stored);
+            ptx::tmem_st_32x32b_x4(tc + 32u + 4u * h, meta);
+          }
           ptx::tmem_st_wait();
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&built[v]);      // one arrival per warp
         }
+        if (++gu == G) gu = 0;
         if (++v == NU) { v = 0; ph ^= 1; }
       }
     }
