@@ -108,6 +108,20 @@ def test_attach_group_and_selftest_argument_errors_without_a_gpu(m):
     assert L.sdq_linear_group(0, None, None, None, None, None) == 1
     assert L.sdq_linear_group(2, None, None, None, None, None) == 1
     assert L.sdq_diag_wait_timeout(0, None) == 2 and L.sdq_diag_wait_timeout(5000, None) == 2  # polls outside 1 .. 4096
+    i64 = ctypes.c_int64
+    assert L.sdq_linear_group_x(1, None, i64(4), i64(1024), i64(1024), None, None, None, None) == 1                    # null X
+    pp, yy, ld = (ctypes.c_void_p * 1)(), (ctypes.c_void_p * 1)(), (ctypes.c_int64 * 1)(1024)
+    x = ctypes.c_void_p(0x1000)
+    assert L.sdq_linear_group_x(1, x, i64(4), i64(1000), i64(1024), pp, yy, ld, None) == 2                             # K % 256
+    assert L.sdq_linear_group_x(1, ctypes.c_void_p(0x1008), i64(4), i64(1024), i64(1024), pp, yy, ld, None) == 3       # X not 16-byte aligned
+    assert L.sdq_linear_group_x(1, x, i64(4), i64(1024), i64(1020), pp, yy, ld, None) == 2                             # row stride shorter than K
+    # the sixth configuration word: int8 outlier operands only with the primary inlier format and power-of-two inlier scales
+    b = ctypes.c_size_t()
+    assert L.sdq_packed_size(128, 256, ctypes.byref(m.Config(1, m.GRAN_PAIR, 64, 0, 0, m.OUT_INT8)), ctypes.byref(b), None) == 0
+    assert L.sdq_packed_size(128, 256, ctypes.byref(m.Config(1, m.GRAN_PAIR, 32, 0, 0, m.OUT_INT8)), ctypes.byref(b), None) == 4
+    assert L.sdq_packed_size(128, 256, ctypes.byref(m.Config(1, m.GRAN_PAIR, 32, m.SCALE_UE4M3, 0, m.OUT_INT8)), ctypes.byref(b), None) == 1
+    assert L.sdq_packed_size(128, 256, ctypes.byref(m.Config(1, m.GRAN_PAIR, 64, 0, 0, 7)), ctypes.byref(b), None) == 1
+    assert L.sdq_act_size(4, 256, ctypes.byref(m.Config(1, m.GRAN_PAIR, 64, 0, 0, 7)), ctypes.byref(b)) == 1
 
 
 def test_bench_starts_its_own_ranks_when_run_without_a_launcher():
