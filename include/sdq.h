@@ -198,6 +198,20 @@ sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canonical_t* out
  *   SHAPE (header inconsistent with itself), BUFFER_TOO_SMALL (bytes < the size the header records), CUDA. */
 sdq_status_t sdq_packed_attach(const void* dev, size_t bytes, sdq_packed_t* out, void* stream);
 
+/* The packed matrix without its 2:4 outlier containers: inlier records, compact outlier records (8-bit code + position per
+ * outlier), scales -- 4.2 instead of 9.1 bits per weight for the 1:8 + 4:8 configuration, i.e. what Section 3.3 counts plus
+ * the tensor core's metadata and padding.  This is all the fused few-token kernel of sdq_linear_group / sdq_linear_group_x
+ * streams (it rebuilds the containers in tensor memory), so a deployment that only decodes keeps just this form resident;
+ * calls that need the containers (sdq_linear and its variants, the layer-by-layer fallback of sdq_linear_group) return
+ * SDQ_ERR_UNSUPPORTED for it.  sdq_packed_export, sdq_packed_attach (the header says which form a buffer holds) and the
+ * grouped calls accept both forms; off[1] of a compact descriptor is 0.
+ *   sdq_packed_compact_size: bytes of the compact form (tiled configurations with out_n >= 1; SDQ_ERR_UNSUPPORTED otherwise).
+ *   sdq_packed_compact: copies P's sections into dst (device, 256-byte aligned, >= that many bytes, caller-owned, must not
+ *   overlap P->dev), writes its header and fills *out.  Device-to-device copies on `stream`, then one stream
+ *   synchronisation; allocates nothing.  P itself is unchanged and may be freed afterwards. */
+sdq_status_t sdq_packed_compact_size(int64_t N, int64_t K, const sdq_config_t* cfg, size_t* bytes);
+sdq_status_t sdq_packed_compact(const sdq_packed_t* P, void* dst, size_t dst_bytes, sdq_packed_t* out, void* stream);
+
 /* Size of the quantized-activation buffer for M tokens of K features. */
 sdq_status_t sdq_act_size(int64_t M, int64_t K, const sdq_config_t* cfg, size_t* bytes);
 

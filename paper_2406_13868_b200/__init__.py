@@ -64,7 +64,7 @@ class _ActCanon(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("xq4_code", "xq4_scale", "xq8_code", "xq8_sexp")]
 
 
-EXPORTS = ["sdq_packed_size", "sdq_decompose", "sdq_decompose_metric", "sdq_channel_norm", "sdq_packed_export", "sdq_packed_attach", "sdq_act_size", "sdq_quantize_act", "sdq_act_export",
+EXPORTS = ["sdq_packed_size", "sdq_decompose", "sdq_decompose_metric", "sdq_channel_norm", "sdq_packed_export", "sdq_packed_attach", "sdq_packed_compact_size", "sdq_packed_compact", "sdq_act_size", "sdq_quantize_act", "sdq_act_export",
            "sdq_linear", "sdq_linear_f32", "sdq_workspace_size", "sdq_workspace_init", "sdq_linear_ws", "sdq_linear_f32_ws", "sdq_linear_noalloc",
            "sdq_linear_group", "sdq_linear_group_f32", "sdq_linear_group_x", "sdq_linear_group_x_f32", "sdq_diag_l2_copy", "sdq_diag_wait_timeout", "sdq_device_status", "sdq_status_string"]
 
@@ -187,6 +187,18 @@ def packed_attach(buf: torch.Tensor) -> PackedWeight:
     cfg = Config(d.cfg.out_n, d.cfg.in_gran, d.cfg.in_block, d.cfg.scale_rule, d.cfg.out_order, d.cfg.out_fmt)
     _, algo = packed_size(d.N, d.K, cfg)
     return PackedWeight(buf, d, d.N, d.K, cfg, algo)
+
+
+def packed_compact(p: PackedWeight) -> PackedWeight:
+    """The packed matrix without its 2:4 outlier containers (4.2 instead of 9.1 bits per weight): the form the grouped
+    few-token calls stream.  Returns a new PackedWeight in its own buffer (see sdq_packed_compact in include/sdq.h)."""
+    n = ctypes.c_size_t(0)
+    _check(lib().sdq_packed_compact_size(ctypes.c_int64(p.N), ctypes.c_int64(p.K), ctypes.byref(p.cfg), ctypes.byref(n)), "sdq_packed_compact_size")
+    buf = torch.empty(int(n.value), dtype=torch.uint8, device=p.buf.device)
+    d = _Packed()
+    _check(lib().sdq_packed_compact(ctypes.byref(p.desc), ctypes.c_void_p(buf.data_ptr()), ctypes.c_size_t(buf.numel()), ctypes.byref(d), _stream()),
+           "sdq_packed_compact")
+    return PackedWeight(buf, d, p.N, p.K, p.cfg, p.algorithmic_bytes)
 
 
 def diag_wait_timeout(polls: int = 64) -> None:

@@ -100,7 +100,8 @@ struct BlobHeader {
   uint64_t magic;
   uint32_t version, header_bytes;
   int32_t cfg[6];          // out_n, in_gran, in_block, scale_rule, out_order, out_fmt
-  uint32_t tiled;          // 1: stage-tiled tensor-core layout, 0: canonical arrays (decompose-only reading)
+  uint32_t tiled;          // 1: stage-tiled tensor-core layout, 2: the same without the 2:4 outlier containers (compact),
+                           // 0: canonical arrays (decompose-only reading)
   int64_t N, K;
   uint64_t total;          // bytes of the whole buffer
   uint64_t off[8];         // the section offsets of sdq_packed_t
@@ -110,13 +111,15 @@ static_assert(sizeof(BlobHeader) <= HEADER_BYTES, "header fits its reservation")
 struct PackedOffsets {
   size_t wi, wo, sfa_out, wc, osexp, wtexp, emeta, total;
 };
-inline PackedOffsets packed_offsets(int64_t N, int64_t K, int out_n, bool b32 = false, bool dense = false, bool elem = false) {
+// compact: the buffer carries no 2:4 outlier containers (section WO empty), only the compact records -- the form the grouped
+// few-token kernel streams; 4.2 instead of 9.1 bits per weight
+inline PackedOffsets packed_offsets(int64_t N, int64_t K, int out_n, bool b32 = false, bool dense = false, bool elem = false, bool compact = false) {
   PackedOffsets o;
   const size_t RT = (size_t)(N / TILE_ROWS), T1 = (size_t)(K / K1), T2 = (size_t)(K / K2);
   auto al = [](size_t x) { return (x + 255) & ~(size_t)255; };
   o.wi = HEADER_BYTES;
   o.wo = al(o.wi + RT * T2 * (size_t)wi_bytes(b32, dense));
-  o.sfa_out = al(o.wo + (out_n ? RT * T1 * WO_BYTES : 0));
+  o.sfa_out = al(o.wo + ((out_n && !compact) ? RT * T1 * WO_BYTES : 0));
   o.wc = al(o.sfa_out + RT * SF_ATOM_BYTES);
   o.osexp = al(o.wc + RT * T1 * (size_t)wc_bytes(out_n));
   o.wtexp = al(o.osexp + (size_t)N * 4);                          // inlier row-factor exponents [N] i32 (two-level scaling)

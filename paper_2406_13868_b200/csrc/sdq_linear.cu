@@ -724,6 +724,7 @@ static sdq_status_t launch_linear(const sdq_act_t* Xq, const sdq_packed_t* P, vo
   if (!is_tensor_core_reading(P->cfg)) return SDQ_ERR_UNSUPPORTED;
   if (P->cfg.out_n > 0 && Xq->cfg.out_fmt != P->cfg.out_fmt) return SDQ_ERR_SHAPE;
   if (P->cfg.out_n > 0 && P->cfg.out_fmt == SDQ_OUT_INT8) return SDQ_ERR_UNSUPPORTED;   // int8 outliers: the grouped few-token kernel only
+  if (is_compact(*P)) return SDQ_ERR_UNSUPPORTED;                                       // no 2:4 containers in the buffer: likewise
   if (P->cfg.scale_rule == SDQ_SCALE_UE4M3 && !(P->cfg.in_gran == SDQ_GRAN_PAIR && P->cfg.in_block == 32)) return SDQ_ERR_UNSUPPORTED;
   if (((uintptr_t)Y & 15) || (ldy % 8) || ((uintptr_t)ws & 15)) return SDQ_ERR_ALIGNMENT;
   DeviceInfo* dinfo = device_info();
@@ -941,7 +942,7 @@ static sdq_status_t launch_group(int n, const sdq_act_t* const* Xq, const sdq_pa
   if (!g.flags) return SDQ_ERR_CUDA;
   int item0 = 0;
   for (int i = 0; i < n; ++i) {
-    const PackedOffsets po = tiled_offsets(P[i]->N, P[i]->K, P[i]->cfg);
+    const PackedOffsets po = tiled_offsets(*P[i]);
     const ActOffsets ao = act_offsets(Xq[i]->M, Xq[i]->K, false);
     GroupMat& m = g.m[i];
     m.w = (const uint8_t*)P[i]->dev; m.x = (const uint8_t*)Xq[i]->dev; m.Y = Y[i]; m.ldy = ldy[i];
@@ -992,7 +993,7 @@ static sdq_status_t launch_group_x(int n, const void* X, int64_t M, int64_t K, i
   if (!g.flags) return SDQ_ERR_CUDA;
   int item0 = 0;
   for (int i = 0; i < n; ++i) {
-    const PackedOffsets po = tiled_offsets(P[i]->N, P[i]->K, P[i]->cfg);
+    const PackedOffsets po = tiled_offsets(*P[i]);
     GroupMat& m = g.m[i];
     m.w = (const uint8_t*)P[i]->dev; m.x = nullptr; m.Y = Y[i]; m.ldy = ldy[i];
     m.wi = po.wi; m.wc = po.wc; m.sfa_out = po.sfa_out;

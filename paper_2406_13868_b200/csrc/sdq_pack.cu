@@ -5,6 +5,8 @@
 // outliers, prunes the rest pair-wise, derives the Q-Vector scales by an 8-lane shuffle reduction
 // (8 S-Vectors = 64 K), encodes, and scatters into the stage-tiled layout of sdq_layout.h.  Without Stage 1 (dense
 // inliers) every position that is not an outlier is encoded, with one scale per 32 K.
+#include <cstring>
+
 #include "sdq_codec.cuh"
 #include "sdq_internal.h"
 #include "sdq_layout.h"
@@ -446,9 +448,11 @@ extern "C" sdq_status_t sdq_packed_attach(const void* dev, size_t bytes, sdq_pac
   d.N = h->N; d.K = h->K; d.cfg = cfg;
   for (int i = 0; i < 8; ++i) d.off[i] = 0;
   if (tc) {
-    const PackedOffsets off = tiled_offsets(h->N, h->K, cfg);
+    const bool compact = h->tiled == 2;
+    if (h->tiled > 2 || (compact && cfg.out_n == 0)) return SDQ_ERR_SHAPE;
+    const PackedOffsets off = tiled_offsets(h->N, h->K, cfg, compact);
     d.bytes = off.total;
-    d.off[0] = off.wi; d.off[1] = off.wo; d.off[2] = off.sfa_out; d.off[3] = off.wc; d.off[5] = off.osexp; d.off[6] = off.wtexp;
+    d.off[0] = off.wi; d.off[1] = compact ? 0 : off.wo; d.off[2] = off.sfa_out; d.off[3] = off.wc; d.off[5] = off.osexp; d.off[6] = off.wtexp;
   } else {
     const PlainPackedOffsets poff = plain_packed_offsets(h->N, h->K, cfg);
     d.bytes = poff.total;
@@ -459,6 +463,44 @@ extern "C" sdq_status_t sdq_packed_attach(const void* dev, size_t bytes, sdq_pac
     if (h->off[i] != d.off[i]) return SDQ_ERR_SHAPE;
   if (bytes < d.bytes) return SDQ_ERR_BUFFER_TOO_SMALL;
   *out = d;
+  return SDQ_OK;
+}
+
+extern "C" sdq_status_t sdq_packed_compact_size(int64_t N, int64_t K, const sdq_config_t* cfg, size_t* bytes)
+{
+  if (!cfg_ok(cfg) || !bytes) return SDQ_ERR_INVALID_ARG;
+  if (cfg_unsupported(cfg) || !is_tensor_core_reading(*cfg) || cfg->out_n == 0) return SDQ_ERR_UNSUPPORTED;
+  if (N <= 0 || K <= 0 || N % TILE_ROWS || K % K2) return SDQ_ERR_SHAPE;
+  *bytes = tiled_offsets(N, K, *cfg, true).total;
+  return SDQ_OK;
+}
+
+extern "C" sdq_status_t sdq_packed_compact(const sdq_packed_t* P, void* dst, size_t dst_bytes, sdq_packed_t* out, void* stream)
+{
+  if (!P || !P->dev || !dst || !out) return SDQ_ERR_INVALID_ARG;
+  if (!cfg_ok(&P->cfg)) return SDQ_ERR_INVALID_ARG;
+  if (!is_tensor_core_reading(P->cfg) || P->cfg.out_n == 0 || is_compact(*P)) return SDQ_ERR_UNSUPPORTED;
+  if ((uintptr_t)dst & 255) return SDQ_ERR_ALIGNMENT;
+  const PackedOffsets src = tiled_offsets(P->N, P->K, P->cfg), off = tiled_offsets(P->N, P->K, P->cfg, true);
+  if (dst_bytes < off.total) return SDQ_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  const uint8_t* s = (const uint8_t*)P->dev;
+  uint8_t* d = (uint8_t*)dst;
+  // every section but the 2:4 containers, each to its place in the shorter buffer
+  bool ok = cudaMemcpyAsync(d + off.wi, s + src.wi, src.wo - src.wi, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(d + off.sfa_out, s + src.sfa_out, src.total - src.sfa_out, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (!ok) return SDQ_ERR_CUDA;
+  sdq_packed_t q;
+  q.dev = dst; q.bytes = off.total; q.N = P->N; q.K = P->K; q.cfg = P->cfg;
+  for (int i = 0; i < 8; ++i) q.off[i] = 0;
+  q.off[0] = off.wi; q.off[1] = 0; q.off[2] = off.sfa_out; q.off[3] = off.wc; q.off[5] = off.osexp; q.off[6] = off.wtexp;
+  alignas(16) static thread_local unsigned char raw[HEADER_BYTES];
+  memset(raw, 0, HEADER_BYTES);
+  fill_header(reinterpret_cast<BlobHeader*>(raw), q, true);
+  reinterpret_cast<BlobHeader*>(raw)->tiled = 2u;
+  if (cudaMemcpyAsync(dst, raw, HEADER_BYTES, cudaMemcpyHostToDevice, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+    return SDQ_ERR_CUDA;
+  *out = q;
   return SDQ_OK;
 }
 
@@ -483,7 +525,7 @@ extern "C" sdq_status_t sdq_packed_export(const sdq_packed_t* P, const sdq_canon
     ok = ok && cudaMemcpyAsync(out->out_sexp, b + o.osexp, n * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
     return ok ? SDQ_OK : SDQ_ERR_CUDA;
   }
-  const PackedOffsets off = tiled_offsets(P->N, P->K, P->cfg);
+  const PackedOffsets off = tiled_offsets(*P);
   export_packed_kernel<<<(unsigned)P->N, 128, 0, (cudaStream_t)stream>>>((const uint8_t*)P->dev, P->N, P->K, P->cfg, off, *out);
   return cudaGetLastError() == cudaSuccess ? SDQ_OK : SDQ_ERR_CUDA;
 }

@@ -20,9 +20,12 @@ inline bool is_tensor_core_reading(const sdq_config_t& c) {
 __host__ __device__ inline bool is_dense_layout(const sdq_config_t& c) {
   return c.in_block == 32 && (c.in_gran >= SDQ_GRAN_DENSE || c.in_gran == SDQ_GRAN_ELEM);
 }
-inline PackedOffsets tiled_offsets(int64_t N, int64_t K, const sdq_config_t& c) {
-  return packed_offsets(N, K, c.out_n, c.in_block == 32, is_dense_layout(c), c.in_gran == SDQ_GRAN_ELEM && c.in_block == 32);
+inline PackedOffsets tiled_offsets(int64_t N, int64_t K, const sdq_config_t& c, bool compact = false) {
+  return packed_offsets(N, K, c.out_n, c.in_block == 32, is_dense_layout(c), c.in_gran == SDQ_GRAN_ELEM && c.in_block == 32, compact);
 }
+// a tiled buffer made by sdq_packed_compact: it has outliers but no container section (its offset, never 0 in a full buffer, is 0)
+inline bool is_compact(const sdq_packed_t& p) { return p.cfg.out_n > 0 && p.off[1] == 0; }
+inline PackedOffsets tiled_offsets(const sdq_packed_t& p) { return tiled_offsets(p.N, p.K, p.cfg, is_compact(p)); }
 
 struct PlainPackedOffsets {
   size_t in_code, in_meta, in_scale, out_code, out_idx, osexp, total;

@@ -122,6 +122,15 @@ def test_attach_group_and_selftest_argument_errors_without_a_gpu(m):
     assert L.sdq_packed_size(128, 256, ctypes.byref(m.Config(1, m.GRAN_PAIR, 32, m.SCALE_UE4M3, 0, m.OUT_INT8)), ctypes.byref(b), None) == 1
     assert L.sdq_packed_size(128, 256, ctypes.byref(m.Config(1, m.GRAN_PAIR, 64, 0, 0, 7)), ctypes.byref(b), None) == 1
     assert L.sdq_act_size(4, 256, ctypes.byref(m.Config(1, m.GRAN_PAIR, 64, 0, 0, 7)), ctypes.byref(b)) == 1
+    # the compact form: 2.625 + 1.5 bits per weight plus scales and the header; only where there are outliers to compact
+    c, full = ctypes.c_size_t(), ctypes.c_size_t()
+    cfg = m.Config()
+    assert L.sdq_packed_compact_size(i64(4096), i64(4096), ctypes.byref(cfg), ctypes.byref(c)) == 0
+    assert L.sdq_packed_size(4096, 4096, ctypes.byref(cfg), ctypes.byref(full), None) == 0
+    assert c.value * 8 / 4096 ** 2 < 4.2 and full.value - c.value == 4096 * 4096 * 5 // 8
+    assert L.sdq_packed_compact_size(i64(4096), i64(4096), ctypes.byref(m.Config(0)), ctypes.byref(c)) == 4
+    assert L.sdq_packed_compact_size(i64(4096), i64(4000), ctypes.byref(cfg), ctypes.byref(c)) == 2
+    assert L.sdq_packed_compact(None, None, 0, None, None) == 1
 
 
 def test_bench_starts_its_own_ranks_when_run_without_a_launcher():

@@ -446,3 +446,44 @@ def test_fused_quantizer_group_call_outside_its_range_is_refused():
     with pytest.raises(RuntimeError):
         m.sdq_linear_group_x(sdq_synth.make_act(4, 2048, 1).cuda(), ps)                  # K of X and of the weights differ
     assert m.device_status() == 0
+
+
+# ---------------------------------------------------------------------------------------------------------------------
+# the packed buffer without its 2:4 outlier containers
+
+@pytest.mark.parametrize("cfg_args", [(1, so.GRAN_PAIR, 64, 0), I8_ARGS])
+def test_compact_buffer_serves_the_grouped_calls_and_nothing_else(cfg_args):
+    m = sdq()
+    cfg = m.Config(*cfg_args)
+    N, K, M = 4096, 2048, 6
+    Ws = [sdq_synth.make_weight(N, K, 6100 + i) for i in range(3)]
+    X = sdq_synth.make_act(M, K, 6150).cuda()
+    full = [m.sdq_decompose(W.cuda(), cfg) for W in Ws]
+    comp = [m.packed_compact(p) for p in full]
+    # 2.625 + 1.5 bits per weight, scales, padding: under 4.3; the full buffer carries the 5-bit containers on top
+    assert comp[0].buf.numel() * 8 / (N * K) < 4.3 and full[0].buf.numel() * 8 / (N * K) > 9.0
+    assert comp[0].desc.off[1] == 0 and comp[0].desc.off[3] > 0
+    xq = m.sdq_quantize_act(X, cfg)
+    ref = m.sdq_linear_group([xq] * 3, full, f32=True)
+    got = m.sdq_linear_group([xq] * 3, comp, f32=True)
+    gotx = m.sdq_linear_group_x(X, comp, f32=True)
+    assert m.device_status() == 0
+    for a, b, c in zip(ref, got, gotx):
+        assert torch.equal(a, b) and torch.equal(a, c)
+    # the canonical export reads the compact records: identical
+    ea, eb = m.packed_export(full[0]), m.packed_export(comp[0])
+    for k in ea:
+        assert torch.equal(ea[k], eb[k]), k
+    # save -> reload: the header says which form the buffer holds
+    re = m.packed_attach(comp[1].buf.clone())
+    assert re.desc.off[1] == 0 and torch.equal(m.sdq_linear_group([xq] * 3, [comp[0], re, comp[2]], f32=True)[1], ref[1])
+    # calls that need the containers refuse it: the single-layer call, the layer-by-layer path of a group too small to fuse,
+    # and compacting twice
+    with pytest.raises(RuntimeError):
+        m.sdq_linear(xq, comp[0])
+    small = m.packed_compact(m.sdq_decompose(sdq_synth.make_weight(256, K, 1).cuda(), cfg))
+    with pytest.raises(RuntimeError):
+        m.sdq_linear_group([xq], [small])
+    with pytest.raises(RuntimeError):
+        m.packed_compact(comp[0])
+    assert m.device_status() == 0
