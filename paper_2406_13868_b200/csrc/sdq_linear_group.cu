@@ -29,6 +29,15 @@
 // and the scales to TMEM), 2..5 epilogue (adds the two accumulators; accumulator pairs alternate per item, so the next
 // item's MMAs never wait for the stores), 6..9, 11..14, 15..18 and 19..22 container builders (up to four groups).
 // Every wait is bounded; a timeout sets the sticky flag.
+//
+// Variants.  Outlier operands in int8 (SDQ_OUT_INT8): the same containers and token codes read as integers by a sparse
+// kind::i8 MMA into an int32 accumulator; the epilogue converts the exact sums and applies the fp32 row and token scales.
+// Activation-resident (template XRES, sdq_linear_group_x): all layers read one bf16 X of up to 16 tokens, which every CTA
+// quantizes into its own shared memory (22 warps; the codes, scales and layouts of sdq_quantize_act) while its producers
+// already stream weights; the ring slots then hold the weight records only.
+//
+// What bounds it (measured): the SM's instruction issue is half used, more than half of it by the builders' byte
+// arithmetic; a CTA runs a unit in ~0.45-0.5 us against 0.38 us at the HBM peak.
 #include <cuda_bf16.h>
 
 #include "sdq_codec.cuh"
