@@ -105,3 +105,40 @@ def test_llama7b_layer_shapes_token_sweep(M):
     """config 5: the three weight shapes of a LLaMA-7B decoder layer at every token count of the sweep"""
     for i, (N, K) in enumerate([(4096, 4096), (11008, 4096), (4096, 11008)]):
         check_sampled(M, N, K, 5000 + 10 * M + i, n_tok=8)
+
+
+@pytest.mark.parametrize("M", [1, 16])
+@pytest.mark.parametrize("out_fmt", [so.OUT_E4M3, so.OUT_INT8])
+def test_llama7b_decode_32_layers_in_one_grouped_call_as_in_the_bench(M, out_fmt):
+    """config 2 in the launch configuration bench.py times for decode: 32 distinct 4096 x 4096 layers, compact packed form,
+    ONE grouped call; three layers (first, middle, last) are checked on sampled 128-row tiles, every token.  Also with the
+    activation quantizer inside the kernel (bit-identical) and with int8 outlier operands."""
+    m = sdq()
+    cfg = m.Config(1, so.GRAN_PAIR, 64, 0, 0, out_fmt)
+    ocfg = so.Config(1, so.GRAN_PAIR, 64, 0, 0, out_fmt)
+    N = K = 4096
+    layers = 32
+    Ws, ps = {}, []
+    for i in range(layers):
+        W = sdq_synth.make_weight(N, K, 2000 + i, device="cuda")
+        ps.append(m.packed_compact(m.sdq_decompose(W, cfg)))
+        if i in (0, 15, 31):
+            Ws[i] = W
+        del W
+    X = sdq_synth.make_act(M, K, 2100 + M, device="cuda")
+    xq = m.sdq_quantize_act(X, cfg)
+    ys = m.sdq_linear_group([xq] * layers, ps, f32=True)
+    ys16 = m.sdq_linear_group([xq] * layers, ps)
+    yx = m.sdq_linear_group_x(X, ps, f32=True)
+    assert m.device_status() == 0
+    oq = so.quantize_act(sdq_synth.bf16_bits(X), ocfg)
+    rows = np.concatenate([np.arange(128 * t, 128 * t + 128) for t in (0, 16, 31)])
+    rows_t = torch.from_numpy(rows).cuda()
+    for i, W in Ws.items():
+        op = so.decompose(sdq_synth.bf16_bits(W[rows_t]), ocfg)
+        yref = so.linear(oq, op)
+        d = np.abs(ys[i][:, rows_t].cpu().numpy().astype(np.float64) - yref)
+        tol = 1e-3 * (np.abs(yref) + 1e-2)
+        assert (d <= tol).all(), (i, float(d.max()), float((d / tol).max()))
+    for a, b, c in zip(ys, ys16, yx):
+        assert torch.equal(b, a.to(torch.bfloat16)) and torch.equal(a, c)
