@@ -485,7 +485,7 @@ sdq_linear_group_kernel(const __grid_constant__ GroupParams p)
             }
 #pragma unroll
             for (int g = 0; g < 16; ++g)
-              stored[g] = __byte_perm(cw[g >> 2], 0u, 0x4440u + (uint32_t)(g & 3)) << ((shw[g >> 2] >> (8 * (g & 3))) & 0xFFu);
+              stored[g] = __funnelshift_l(0u, __byte_perm(cw[g >> 2], 0u, 0x4440u + (uint32_t)(g & 3)), shw[g >> 2] >> (8 * (g & 3)));   // (shift count mod 32: the byte's 0 / 8 / 16 / 24)
             // columns 0..7 of the stage: the row's stored bytes of K-block 0 (the first MMA's A), 8..15: of K-block 1
             ptx::tmem_st_32x32b_x16(tc + 16u * h, stored);
             ptx::tmem_st_32x32b_x4(tc + 32u + 4u * h, meta);
